@@ -1,0 +1,582 @@
+/*
+ * RAC reference-aware activation codec -- plain CPU oracle (TEST INFRASTRUCTURE).
+ *
+ * This file is a slow, scalar restatement of the method, written from the
+ * paper's equations.  It exists only so that tests (and the reported CPU
+ * baseline of the benchmark) have something independent to compare the CUDA
+ * path with.  The product never calls it and it shares no code with the CUDA
+ * sources.
+ *
+ * What follows which passage of the paper (Sec. IV-B, IV-C):
+ *   orc_match_spans      Sec. IV-B.1, Eq. 3: w-token windows over the history,
+ *                        every hit extended to its longest exact match, at most
+ *                        K most recent hits per distinct window, selection by
+ *                        lexargmax(length, recency), scan advances by the span
+ *                        length or by one.
+ *   orc_encode           Sec. IV-C: grouped affine fit (Eq. 6) with the
+ *                        zero-variance rule, wire rounding of the coefficients,
+ *                        aligned reference and residual (Eq. 7), outlier split
+ *                        (unnumbered equation before Eq. 8, outlier values kept
+ *                        as FP16), symmetric b-bit quantisation with
+ *                        Qmax = 2^(b-1)-1 and round-to-nearest (Eq. 8), packing.
+ *   orc_reconstruct      Eq. 9: dequantise, restore outliers, add the aligned
+ *                        reference.  Sender and receiver run this same function.
+ *   orc_calibrate        "offline calibration" of Sec. IV-C reduced to the one
+ *                        thing the codec needs as an input: a per-channel step
+ *                        from the RMS of the aligned residual.
+ *
+ * Readings taken where the paper is silent (each is also listed in the design
+ * notes of the repository):
+ *   - one fit per (token, group): the "fitting positions" of Eq. 6 are the
+ *     channels of one group of one token;
+ *   - Round_wire of the coefficients is IEEE binary16 round-to-nearest-even,
+ *     saturating at +-65504;
+ *   - zero variance means centred Sxx <= 1e-12, or a slope that binary16 cannot
+ *     hold (|Sxy| >= 65504*Sxx), or no reference at all;
+ *   - the quantiser step is a static per-channel table (two rows: tokens with a
+ *     reference, tokens coded directly) instead of Eq. 8's per-group dynamic
+ *     scale, so dense values can clip; step 0 means "code 0";
+ *   - outliers are the k largest |e| per TOKEN (not per group), ranked on the
+ *     fp32 bit pattern of |e|, ties to the lower channel, stored with u16
+ *     absolute channel indices in ascending order;
+ *   - round-to-nearest is ties-to-even;
+ *   - the residual, the scaled value, the rounding decision and the
+ *     reconstruction are taken in binary32 with one rounding per operation
+ *     (fused multiply-add where written as fmaf), because these decide integer
+ *     codes and two endpoints must agree bit for bit; the fit itself is done
+ *     in binary64.
+ *
+ * Wire record of one token (all little endian), records back to back:
+ *   coef    J  x u32   binary16 alpha in bits 0..15, binary16 beta in bits 16..31
+ *   codes   d*b/8 B    code of channel c occupies stream bits [c*b, c*b+b),
+ *                      stream bit n is bit (n%8) of byte (n/8); two's complement
+ *   out_idx k  x u16   ascending
+ *   out_val k  x u16   binary16
+ *   padding to a multiple of 16 bytes (zero)
+ *
+ * Parity status: the LS fit, residual identity, quantiser bounds, packing,
+ * outlier selection and the matcher are pinned by tests against closed forms,
+ * library least squares, brute force and invariants.  The wire layout, the
+ * coefficient format, the static step table and the tie rules are this
+ * build's own definitions ("parity unpinned" by the paper): only round trips
+ * and the properties above pin them.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------ */
+/* number formats                                                      */
+/* ------------------------------------------------------------------ */
+
+static float bits_to_f32(uint32_t u) { float f; memcpy(&f, &u, 4); return f; }
+static uint32_t f32_to_bits(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+
+float orc_bf16_to_f32(uint16_t h) { return bits_to_f32((uint32_t)h << 16); }
+
+/* binary32 -> bfloat16, round to nearest even (NaN kept quiet). */
+uint16_t orc_f32_to_bf16(float f) {
+    uint32_t u = f32_to_bits(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+/* binary16 -> binary64 (exact). */
+double orc_f16_to_f64(uint16_t h) {
+    int sign = (h >> 15) & 1;
+    int ex = (h >> 10) & 0x1f;
+    int man = h & 0x3ff;
+    double v;
+    if (ex == 0) v = ldexp((double)man, -24);
+    else if (ex == 31) v = man ? NAN : INFINITY;
+    else v = ldexp((double)(man | 0x400), ex - 25);
+    return sign ? -v : v;
+}
+float orc_f16_to_f32(uint16_t h) { return (float)orc_f16_to_f64(h); }
+
+/* binary64 -> binary16, round to nearest even in ONE rounding, saturating to
+ * +-65504 (so never infinity).  NaN gives 0x7e00. */
+uint16_t orc_f64_to_f16(double x) {
+    if (isnan(x)) return 0x7e00;
+    uint16_t sign = signbit(x) ? 0x8000 : 0;
+    double a = fabs(x);
+    if (a >= 65504.0) return sign | 0x7bff;
+    if (a == 0.0) return sign;
+    int e;
+    (void)frexp(a, &e);               /* a = m * 2^e, m in [0.5,1) */
+    int ulp_exp = e - 11;             /* 11 significant bits for normals   */
+    if (ulp_exp < -24) ulp_exp = -24; /* subnormal spacing 2^-24           */
+    double scaled = ldexp(a, -ulp_exp);     /* exact                      */
+    double r = nearbyint(scaled);           /* default mode: ties to even  */
+    double v = ldexp(r, ulp_exp);
+    if (v >= 65520.0) return sign | 0x7bff;
+    /* re-encode v, which is exactly representable */
+    if (v == 0.0) return sign;
+    int e2;
+    double m2 = frexp(v, &e2);        /* v = m2 * 2^e2 */
+    if (e2 - 1 < -14) {               /* subnormal */
+        return sign | (uint16_t)ldexp(v, 24);
+    }
+    uint16_t ex = (uint16_t)(e2 - 1 + 15);
+    uint16_t man = (uint16_t)(ldexp(m2, 11)) & 0x3ff;
+    return sign | (uint16_t)(ex << 10) | man;
+}
+
+/* smallest binary16 value >= x, for x >= 0 (used for step tables so that the
+ * stored step never shrinks the range, mirroring RoundUp_wire of Eq. 8). */
+uint16_t orc_f64_to_f16_up(double x) {
+    uint16_t h = orc_f64_to_f16(x);
+    if (orc_f16_to_f64(h) < x && h < 0x7bff) h++;
+    return h;
+}
+
+/* ------------------------------------------------------------------ */
+/* record geometry                                                     */
+/* ------------------------------------------------------------------ */
+
+int64_t orc_record_bytes(int d, int group, int bits, int topk) {
+    int64_t raw = 4 * (int64_t)(d / group) + ((int64_t)d * bits) / 8 + 4 * (int64_t)topk;
+    return (raw + 15) / 16 * 16;
+}
+
+static int cfg_ok(int d, int group, int bits, int topk) {
+    if (d <= 0 || group <= 0 || d % group) return 0;
+    if (bits < 2 || bits > 8) return 0;
+    if (((int64_t)d * bits) % 8) return 0;
+    if (topk < 0 || topk > d || d > 65536) return 0;
+    return 1;
+}
+
+static void put_code(uint8_t *codes, int c, int bits, int q) {
+    uint32_t v = (uint32_t)q & ((1u << bits) - 1u);
+    int64_t bit = (int64_t)c * bits;
+    for (int n = 0; n < bits; n++, bit++) {
+        if ((v >> n) & 1u) codes[bit >> 3] |= (uint8_t)(1u << (bit & 7));
+    }
+}
+
+static int get_code(const uint8_t *codes, int c, int bits) {
+    uint32_t v = 0;
+    int64_t bit = (int64_t)c * bits;
+    for (int n = 0; n < bits; n++, bit++) {
+        v |= (uint32_t)((codes[bit >> 3] >> (bit & 7)) & 1u) << n;
+    }
+    if (v & (1u << (bits - 1))) return (int)v - (1 << bits);
+    return (int)v;
+}
+
+/* exported for the packing tests */
+void orc_pack_codes(const int32_t *q, int d, int bits, uint8_t *codes) {
+    memset(codes, 0, ((size_t)d * bits) / 8);
+    for (int c = 0; c < d; c++) put_code(codes, c, bits, q[c]);
+}
+void orc_unpack_codes(const uint8_t *codes, int d, int bits, int32_t *q) {
+    for (int c = 0; c < d; c++) q[c] = get_code(codes, c, bits);
+}
+
+/* ------------------------------------------------------------------ */
+/* reference row of one token                                          */
+/* ------------------------------------------------------------------ */
+
+/* Returns 1 when the token has a reference, 0 when it is coded directly, and
+ * -1 when ref_row points outside the buffer.  r[] receives the reference as
+ * binary32 (zeros when there is none).  The optional per-channel transform is
+ * the stand-in for the decode predictor of Eq. 5: r <- bf16(gain*r + bias). */
+static int resolve_ref(int d, int64_t t, const uint16_t *ref_base, int64_t ref_rows,
+                       const int32_t *ref_row, const uint16_t *gain, const uint16_t *bias,
+                       float *r) {
+    int64_t row = ref_row ? (int64_t)ref_row[t] : t;
+    if (!ref_base || row < 0) {
+        for (int c = 0; c < d; c++) r[c] = 0.0f;
+        return 0;
+    }
+    if (row >= ref_rows) return -1;
+    const uint16_t *src = ref_base + row * (int64_t)d;
+    for (int c = 0; c < d; c++) {
+        float v = orc_bf16_to_f32(src[c]);
+        if (gain) {
+            float gsc = orc_f16_to_f32(gain[c]);
+            float bsc = orc_f16_to_f32(bias[c]);
+            v = orc_bf16_to_f32(orc_f32_to_bf16(fmaf(gsc, v, bsc)));
+        }
+        r[c] = v;
+    }
+    return 1;
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 6: least-squares (alpha, beta) of one group                     */
+/* ------------------------------------------------------------------ */
+
+/* h, r: g values.  Outputs the unrounded optimum and the two means. */
+void orc_fit_group(const float *h, const float *r, int g, int has_ref,
+                   double *alpha_star, double *beta_star, double *hbar_out, double *rbar_out) {
+    double sr = 0.0, sh = 0.0;
+    for (int i = 0; i < g; i++) { sr += (double)r[i]; sh += (double)h[i]; }
+    double rbar = sr / g, hbar = sh / g;
+    double sxx = 0.0, sxy = 0.0;
+    for (int i = 0; i < g; i++) {
+        double dr = (double)r[i] - rbar;
+        double dh = (double)h[i] - hbar;
+        sxx += dr * dr;
+        sxy += dr * dh;
+    }
+    int degenerate = !has_ref || !(sxx > 1e-12) || !(fabs(sxy) < 65504.0 * sxx);
+    if (degenerate) { *alpha_star = 0.0; *beta_star = hbar; }
+    else { double a = sxy / sxx; *alpha_star = a; *beta_star = hbar - a * rbar; }
+    if (hbar_out) *hbar_out = hbar;
+    if (rbar_out) *rbar_out = rbar;
+}
+
+/* ------------------------------------------------------------------ */
+/* encode                                                              */
+/* ------------------------------------------------------------------ */
+
+static float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi); }
+
+/*
+ * X            bf16[T,d]
+ * ref_base     bf16[ref_rows,d] or NULL (every token direct)
+ * ref_row      int32[T] or NULL (identity); negative = direct
+ * gain, bias   binary16[d] or both NULL
+ * step,inv_step float[2,d]: row 0 for tokens with a reference, row 1 direct
+ * forced_coef  u32[T,J] or NULL; when given the fit is skipped and these wire
+ *              coefficients are used (tests use this to separate a coefficient
+ *              rounding flip from everything downstream of it)
+ * payload      T*record bytes out
+ * diag_*       optional outputs (NULL to skip): unrounded alpha, beta, the
+ *              group means (double[T,J] each), the binary32 residual e[T,d]
+ *              and the scaled value v[T,d] the rounding decision was taken on.
+ * returns 0, or -1 bad configuration, -2 ref_row out of range.
+ */
+int orc_encode(int d, int group, int bits, int topk,
+               const uint16_t *X, int64_t T,
+               const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
+               const uint16_t *gain, const uint16_t *bias,
+               const float *step, const float *inv_step,
+               const uint32_t *forced_coef,
+               uint8_t *payload,
+               double *diag_alpha, double *diag_beta, double *diag_hbar, double *diag_rbar,
+               float *diag_e, float *diag_v, int nthreads) {
+    if (!cfg_ok(d, group, bits, topk)) return -1;
+    if ((gain == NULL) != (bias == NULL)) return -1;
+    const int J = d / group;
+    const int64_t rec = orc_record_bytes(d, group, bits, topk);
+    const int qmax = (1 << (bits - 1)) - 1;
+    int err = 0;
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel num_threads(nthreads)
+    {
+        float *h = (float *)malloc(sizeof(float) * d);
+        float *r = (float *)malloc(sizeof(float) * d);
+        float *e = (float *)malloc(sizeof(float) * d);
+        uint8_t *is_out = (uint8_t *)malloc(d);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < T; t++) {
+            uint8_t *recp = payload + t * rec;
+            memset(recp, 0, rec);
+            uint32_t *coef = (uint32_t *)recp;
+            uint8_t *codes = recp + 4 * J;
+            uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
+            uint8_t *oval = oidx + 2 * topk;
+
+            for (int c = 0; c < d; c++) h[c] = orc_bf16_to_f32(X[t * (int64_t)d + c]);
+            int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
+            if (has_ref < 0) {
+#pragma omp atomic write
+                err = -2;
+                continue;
+            }
+            /* Eq. 6 + wire rounding, then Eq. 7 in binary32 */
+            for (int j = 0; j < J; j++) {
+                uint16_t a16, b16;
+                double as = 0, bs = 0, hb = 0, rb = 0;
+                orc_fit_group(h + j * group, r + j * group, group, has_ref, &as, &bs, &hb, &rb);
+                if (forced_coef) {
+                    uint32_t w = forced_coef[t * J + j];
+                    a16 = (uint16_t)(w & 0xffff); b16 = (uint16_t)(w >> 16);
+                } else {
+                    a16 = orc_f64_to_f16(as); b16 = orc_f64_to_f16(bs);
+                }
+                uint32_t w = (uint32_t)a16 | ((uint32_t)b16 << 16);
+                memcpy(&coef[j], &w, 4);
+                if (diag_alpha) diag_alpha[t * J + j] = as;
+                if (diag_beta) diag_beta[t * J + j] = bs;
+                if (diag_hbar) diag_hbar[t * J + j] = hb;
+                if (diag_rbar) diag_rbar[t * J + j] = rb;
+                float a = orc_f16_to_f32(a16), b = orc_f16_to_f32(b16);
+                for (int c = j * group; c < (j + 1) * group; c++) {
+                    float rt = fmaf(a, r[c], b);
+                    e[c] = h[c] - rt;
+                }
+            }
+            /* outlier split: k largest |e| of the token, ties to the lower channel */
+            memset(is_out, 0, d);
+            for (int n = 0; n < topk; n++) {
+                int best = -1; uint32_t bestkey = 0;
+                for (int c = 0; c < d; c++) {
+                    if (is_out[c]) continue;
+                    uint32_t key = f32_to_bits(e[c]) & 0x7fffffffu;
+                    if (best < 0 || key > bestkey) { best = c; bestkey = key; }
+                }
+                is_out[best] = 1;
+            }
+            {
+                int n = 0;
+                for (int c = 0; c < d; c++) {
+                    if (!is_out[c]) continue;
+                    uint16_t ci = (uint16_t)c;
+                    uint16_t hv = orc_f64_to_f16((double)clampf(e[c], -65504.0f, 65504.0f));
+                    memcpy(oidx + 2 * n, &ci, 2);
+                    memcpy(oval + 2 * n, &hv, 2);
+                    n++;
+                }
+            }
+            /* Eq. 8 with the static table, then packing */
+            const float *st = step + (has_ref ? 0 : d);
+            const float *ist = inv_step + (has_ref ? 0 : d);
+            for (int c = 0; c < d; c++) {
+                int q = 0;
+                float v = 0.0f;
+                if (st[c] != 0.0f && !is_out[c]) {
+                    v = e[c] * ist[c];
+                    q = (int)rintf(clampf(v, (float)-qmax, (float)qmax));
+                }
+                if (diag_v) diag_v[t * (int64_t)d + c] = v;
+                if (diag_e) diag_e[t * (int64_t)d + c] = e[c];
+                put_code(codes, c, bits, q);
+            }
+        }
+        free(h); free(r); free(e); free(is_out);
+    }
+    return err;
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 9: reconstruct (receiver and sender)                            */
+/* ------------------------------------------------------------------ */
+
+/* X_hat bf16[T,d] out.  status (optional, one word) gets bit 1 when a reserved
+ * code -2^(b-1) was seen.  returns 0, -1, -2 as orc_encode; -3 when an outlier
+ * index is >= d. */
+int orc_reconstruct(int d, int group, int bits, int topk,
+                    const uint8_t *payload, int64_t T,
+                    const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                    const uint16_t *gain, const uint16_t *bias,
+                    const float *step, uint16_t *X_hat, uint32_t *status, int nthreads) {
+    if (!cfg_ok(d, group, bits, topk)) return -1;
+    if ((gain == NULL) != (bias == NULL)) return -1;
+    const int J = d / group;
+    const int64_t rec = orc_record_bytes(d, group, bits, topk);
+    int err = 0;
+    uint32_t st_word = 0;
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel num_threads(nthreads)
+    {
+        float *r = (float *)malloc(sizeof(float) * d);
+        float *eh = (float *)malloc(sizeof(float) * d);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < T; t++) {
+            const uint8_t *recp = payload + t * rec;
+            const uint8_t *codes = recp + 4 * J;
+            const uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
+            const uint8_t *oval = oidx + 2 * topk;
+            int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
+            if (has_ref < 0) {
+#pragma omp atomic write
+                err = -2;
+                continue;
+            }
+            const float *st = step + (has_ref ? 0 : d);
+            for (int c = 0; c < d; c++) {
+                int q = get_code(codes, c, bits);
+                if (q == -(1 << (bits - 1))) {
+#pragma omp atomic
+                    st_word |= 2u;
+                }
+                eh[c] = (float)q * st[c];
+            }
+            for (int n = 0; n < topk; n++) {
+                uint16_t ci, hv;
+                memcpy(&ci, oidx + 2 * n, 2);
+                memcpy(&hv, oval + 2 * n, 2);
+                if (ci >= d) {
+#pragma omp atomic write
+                    err = -3;
+                    continue;
+                }
+                eh[ci] = orc_f16_to_f32(hv);
+            }
+            for (int j = 0; j < J; j++) {
+                uint32_t w;
+                memcpy(&w, recp + 4 * j, 4);
+                float a = orc_f16_to_f32((uint16_t)(w & 0xffff));
+                float b = orc_f16_to_f32((uint16_t)(w >> 16));
+                for (int c = j * group; c < (j + 1) * group; c++) {
+                    float rt = fmaf(a, r[c], b);
+                    float xh = rt + eh[c];
+                    X_hat[t * (int64_t)d + c] = orc_f32_to_bf16(xh);
+                }
+            }
+        }
+        free(r); free(eh);
+    }
+    if (status) *status |= st_word;
+    return err;
+}
+
+/* ------------------------------------------------------------------ */
+/* step tables from a calibration draw                                 */
+/* ------------------------------------------------------------------ */
+
+/* For every channel: sigma = sqrt(mean over tokens of e^2), separately over
+ * tokens with a reference (row 0) and direct tokens (row 1), e being the
+ * binary32 residual of Eq. 7 with wire coefficients.  step = smallest
+ * binary16 >= clip_sigmas*sigma/Qmax (held as float), inv_step = 1.0f/step in
+ * binary32; a row without tokens, or a channel with sigma 0, gets step 0 and
+ * inv_step 0. */
+int orc_calibrate(int d, int group, int bits,
+                  const uint16_t *X, int64_t T,
+                  const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                  const uint16_t *gain, const uint16_t *bias,
+                  double clip_sigmas, float *step, float *inv_step) {
+    if (!cfg_ok(d, group, bits, 0)) return -1;
+    const int J = d / group;
+    const int qmax = (1 << (bits - 1)) - 1;
+    double *acc = (double *)calloc((size_t)2 * d, sizeof(double));
+    int64_t cnt[2] = {0, 0};
+    float *h = (float *)malloc(sizeof(float) * d);
+    float *r = (float *)malloc(sizeof(float) * d);
+    int err = 0;
+    for (int64_t t = 0; t < T && !err; t++) {
+        for (int c = 0; c < d; c++) h[c] = orc_bf16_to_f32(X[t * (int64_t)d + c]);
+        int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
+        if (has_ref < 0) { err = -2; break; }
+        int row = has_ref ? 0 : 1;
+        cnt[row]++;
+        for (int j = 0; j < J; j++) {
+            double as, bs;
+            orc_fit_group(h + j * group, r + j * group, group, has_ref, &as, &bs, NULL, NULL);
+            float a = orc_f16_to_f32(orc_f64_to_f16(as));
+            float b = orc_f16_to_f32(orc_f64_to_f16(bs));
+            for (int c = j * group; c < (j + 1) * group; c++) {
+                float rt = fmaf(a, r[c], b);
+                float e = h[c] - rt;
+                acc[row * d + c] += (double)e * (double)e;
+            }
+        }
+    }
+    for (int row = 0; row < 2 && !err; row++) {
+        for (int c = 0; c < d; c++) {
+            float s = 0.0f, is = 0.0f;
+            if (cnt[row] > 0) {
+                double sigma = sqrt(acc[row * d + c] / (double)cnt[row]);
+                double want = clip_sigmas * sigma / (double)qmax;
+                if (want > 0.0) {
+                    s = orc_f16_to_f32(orc_f64_to_f16_up(want));
+                    if (s != 0.0f) is = 1.0f / s;
+                }
+            }
+            step[row * d + c] = s;
+            inv_step[row * d + c] = is;
+        }
+    }
+    free(acc); free(h); free(r);
+    return err;
+}
+
+/* ------------------------------------------------------------------ */
+/* Sec. IV-B.1: exact-token span match                                 */
+/* ------------------------------------------------------------------ */
+
+static const int32_t *g_sort_tok;
+static int g_sort_w;
+
+static int cmp_window_pos(const void *pa, const void *pb) {
+    int32_t a = *(const int32_t *)pa, b = *(const int32_t *)pb;
+    for (int m = 0; m < g_sort_w; m++) {
+        int32_t x = g_sort_tok[a + m], y = g_sort_tok[b + m];
+        if (x != y) return x < y ? -1 : 1;
+    }
+    return a < b ? -1 : (a > b ? 1 : 0);
+}
+
+/* compare the history window at position p with the query window at i */
+static int cmp_hist_query(const int32_t *hist, int32_t p, const int32_t *query, int64_t i, int w) {
+    for (int m = 0; m < w; m++) {
+        int32_t x = hist[p + m], y = query[i + m];
+        if (x != y) return x < y ? -1 : 1;
+    }
+    return 0;
+}
+
+/*
+ * ref_row  int32[n_query] out: history row of every covered query position, -1 otherwise
+ * spans    int32[3*cap]  out (q_start, h_start, len), cap >= n_query/w + 1; may be NULL
+ * n_spans  out
+ * max_hits K: only the K largest history starts of each distinct window are
+ *          candidates; 0 = all of them.
+ * Not thread safe (qsort comparator state).
+ */
+int orc_match_spans(const int32_t *hist, int64_t n_hist, const int32_t *query, int64_t n_query,
+                    int w, int max_hits, int32_t *ref_row, int32_t *spans, int32_t *n_spans) {
+    if (w < 1 || max_hits < 0) return -1;
+    for (int64_t i = 0; i < n_query; i++) ref_row[i] = -1;
+    *n_spans = 0;
+    int64_t nwin = n_hist - w + 1;
+    if (nwin <= 0) return 0;
+    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)nwin);
+    for (int64_t j = 0; j < nwin; j++) order[j] = (int32_t)j;
+    g_sort_tok = hist; g_sort_w = w;
+    qsort(order, (size_t)nwin, sizeof(int32_t), cmp_window_pos);
+
+    int64_t i = 0;
+    int32_t ns = 0;
+    while (i < n_query) {
+        if (i + w > n_query) { i++; continue; }
+        /* equal range of the query window in the sorted window list */
+        int64_t lo = 0, hi = nwin;
+        while (lo < hi) {
+            int64_t mid = (lo + hi) / 2;
+            if (cmp_hist_query(hist, order[mid], query, i, w) < 0) lo = mid + 1; else hi = mid;
+        }
+        int64_t first = lo;
+        hi = nwin;
+        while (lo < hi) {
+            int64_t mid = (lo + hi) / 2;
+            if (cmp_hist_query(hist, order[mid], query, i, w) <= 0) lo = mid + 1; else hi = mid;
+        }
+        int64_t last = lo;              /* [first,last): ascending history position */
+        if (first == last) { i++; continue; }
+        int64_t from = first;
+        if (max_hits > 0 && last - first > max_hits) from = last - max_hits;
+        int64_t bestL = -1; int32_t bestj = -1;
+        for (int64_t k = from; k < last; k++) {
+            int32_t j = order[k];
+            int64_t L = w;
+            while (i + L < n_query && j + L < n_hist && query[i + L] == hist[j + L]) L++;
+            if (L > bestL || (L == bestL && j > bestj)) { bestL = L; bestj = j; }
+        }
+        if (spans) { spans[3 * ns] = (int32_t)i; spans[3 * ns + 1] = bestj; spans[3 * ns + 2] = (int32_t)bestL; }
+        ns++;
+        for (int64_t m = 0; m < bestL; m++) ref_row[i + m] = bestj + (int32_t)m;
+        i += bestL;
+    }
+    *n_spans = ns;
+    free(order);
+    return 0;
+}
+
+int orc_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

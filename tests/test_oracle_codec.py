@@ -1,0 +1,344 @@
+"""Pins for the oracle's encode / reconstruct / calibrate (CPU only).
+
+Nothing here re-types the oracle's formulas.  The checks are: closed forms of
+the affine fit (Eq. 6), agreement with numpy's least squares, the zero-variance
+rule, the error identity of Eq. 10 observed from inputs and outputs only, the
+half-step bound of Eq. 11 outside the clip range and exact saturation inside
+it, exhaustive rounding at every half-way point, and brute-force outlier
+selection with crafted ties.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_04991_b200 import synth
+
+
+def bits_of(x):  # float array -> bf16 bits via torch (independent of the oracle's own rounding)
+    return synth.bf16_bits(torch.as_tensor(np.asarray(x, np.float32)).to(torch.bfloat16))
+
+
+def f16(bits):
+    return np.asarray(bits, np.uint16).view(np.float16).astype(np.float64)
+
+
+def flat_tables(d, step_val):
+    step = np.full((2, d), step_val, np.float32)
+    inv = (np.float32(1.0) / step).astype(np.float32)
+    return step, inv
+
+
+# ------------------------------------------------------------------ Eq. 6
+def test_fit_reference_equal_to_x_gives_identity_and_zero_codes(orc):
+    d, g, T = 256, 64, 5
+    gen = synth.generator(10)
+    X = synth.activations(T, d, synth.channel_scale(d, 0), gen)
+    Xb = synth.bf16_bits(X)
+    step, inv = flat_tables(d, 0.02)
+    for bits, k in [(4, 0), (3, 0), (2, 0), (4, 4)]:
+        payload = orc.encode(d, g, bits, k, Xb, ref_base=Xb, step=step, inv_step=inv)
+        coef, codes, oi, ov = orc.split_payload(payload, T, d, g, bits, k)
+        assert np.all((coef & 0xffff) == 0x3c00)      # alpha == 1.0
+        assert np.all(f16(coef >> 16) == 0.0)         # beta == +-0
+        assert not codes.any()                         # residual identically zero
+        if k:
+            # all |e| tie at zero: the k lowest channels win, values are zero
+            assert np.array_equal(oi, np.tile(np.arange(k, dtype=np.uint16), (T, 1)))
+            assert not (ov & 0x7fff).any()
+        xh = orc.reconstruct(d, g, bits, k, payload, T, ref_base=Xb, step=step)
+        assert np.array_equal(xh, Xb)
+
+
+def test_fit_recovers_exact_affine_map(orc):
+    # small-integer references and dyadic (a, b): X = a*R + b is exact in bf16, so the fit must return
+    # exactly (a, b), the residual is zero and the round trip is the identity.
+    rng = np.random.default_rng(11)
+    d, g, T = 256, 64, 16
+    J = d // g
+    R = rng.integers(-8, 9, size=(T, d)).astype(np.float32)
+    R[:, ::g] = 8.0  # make sure no group is constant
+    R[:, 1::g] = -8.0
+    a = rng.choice([0.75, 1.0, 1.25, 1.5, -0.5], size=(T, J)).astype(np.float32)
+    b = rng.choice([-0.5, 0.0, 0.25, 2.0], size=(T, J)).astype(np.float32)
+    X = np.repeat(a, g, axis=1) * R + np.repeat(b, g, axis=1)
+    Xb, Rb = bits_of(X), bits_of(R)
+    assert np.array_equal(orc.bf16_to_f32(Xb), X)  # exact by construction
+    step, inv = flat_tables(d, 0.01)
+    payload = orc.encode(d, g, 4, 0, Xb, ref_base=Rb, step=step, inv_step=inv)
+    coef, codes, _, _ = orc.split_payload(payload, T, d, g, 4, 0)
+    assert np.array_equal(f16(coef & 0xffff), a.astype(np.float64))
+    assert np.array_equal(f16(coef >> 16), b.astype(np.float64))
+    assert not codes.any()
+    assert np.array_equal(orc.reconstruct(d, g, 4, 0, payload, T, ref_base=Rb, step=step), Xb)
+
+
+def test_fit_zero_variance_and_missing_reference(orc):
+    rng = np.random.default_rng(12)
+    d, g, T = 128, 64, 4
+    X = rng.standard_normal((T, d)).astype(np.float32)
+    Xb = bits_of(X)
+    Xv = orc.bf16_to_f32(Xb).astype(np.float64)
+    mean = Xv.reshape(T, d // g, g).mean(axis=2)
+    step, inv = flat_tables(d, 0.05)
+    const = bits_of(np.full((T, d), 3.5, np.float32))
+    neg = np.full(T, -1, np.int32)
+    for kwargs in (dict(ref_base=const), dict(ref_base=None), dict(ref_base=const, ref_row=neg)):
+        payload, dg = orc.encode(d, g, 4, 0, Xb, step=step, inv_step=inv, diag=True, **kwargs)
+        coef, _, _, _ = orc.split_payload(payload, T, d, g, 4, 0)
+        assert np.all((coef & 0x7fff) == 0)  # alpha = 0
+        assert np.allclose(dg["beta"], mean, rtol=0, atol=1e-12)
+        assert np.all(np.abs(f16(coef >> 16) - mean) <= np.abs(mean) * 2.0 ** -11 + 2.0 ** -25)
+
+
+def test_fit_matches_library_least_squares_and_normal_equations(orc):
+    rng = np.random.default_rng(13)
+    for g in (32, 64, 128, 256):
+        for _ in range(20):
+            r = orc.bf16_to_f32(bits_of(rng.standard_normal(g) * rng.uniform(0.1, 30)))
+            h = orc.bf16_to_f32(bits_of(rng.uniform(-2, 2) * r + rng.uniform(-1, 1) + 0.3 * rng.standard_normal(g)))
+            a, b, hbar, rbar = orc.fit_group(h, r)
+            A = np.stack([r.astype(np.float64), np.ones(g)], axis=1)
+            sol = np.linalg.lstsq(A, h.astype(np.float64), rcond=None)[0]
+            assert np.allclose([a, b], sol, rtol=1e-9, atol=1e-11)
+            res = h.astype(np.float64) - (a * r.astype(np.float64) + b)
+            scale = np.abs(h).sum() + 1.0
+            assert abs(res.sum()) < 1e-10 * scale            # d/d(beta) = 0
+            assert abs((res * r).sum()) < 1e-9 * scale * np.abs(r).max()  # d/d(alpha) = 0
+            assert hbar == pytest.approx(h.astype(np.float64).mean(), abs=1e-12)
+            assert rbar == pytest.approx(r.astype(np.float64).mean(), abs=1e-12)
+
+
+def test_wire_coefficients_are_nearest_binary16(orc):
+    d, g, T = 512, 128, 32
+    gen = synth.generator(14)
+    X = synth.activations(T, d, synth.channel_scale(d, 1), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    step, inv = flat_tables(d, 0.02)
+    payload, dg = orc.encode(d, g, 4, 0, synth.bf16_bits(X), ref_base=synth.bf16_bits(R), step=step, inv_step=inv,
+                             diag=True)
+    coef, _, _, _ = orc.split_payload(payload, T, d, g, 4, 0)
+    want_a = dg["alpha"].astype(np.float16).view(np.uint16)  # numpy rounds binary64 -> binary16 in one step
+    want_b = dg["beta"].astype(np.float16).view(np.uint16)
+    assert np.array_equal(coef & 0xffff, want_a)
+    assert np.array_equal(coef >> 16, want_b)
+    # the fit is attenuated by the reference noise but sits near the drawn slope range
+    a = f16(coef & 0xffff)
+    assert 0.75 < a.min() and a.max() < 1.3
+
+
+# ------------------------------------------------------------------ Eq. 8-11
+@pytest.mark.parametrize("bits,topk", [(4, 0), (3, 0), (2, 0), (4, 8), (3, 8), (2, 8)])
+def test_round_trip_error_identity_and_bounds(orc, bits, topk):
+    d, g, T = 1024, 128, 48
+    gen = synth.generator(20 + bits)
+    scale = synth.channel_scale(d, 2)
+    X = synth.activations(T, d, scale, gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    Xb, Rb = synth.bf16_bits(X), synth.bf16_bits(R)
+    cal = synth.activations(256, d, scale, gen)
+    calr = synth.affine_noisy_reference(cal, g, gen)
+    # a tight 1.5-sigma clip so that saturation is exercised even after the outliers are taken out
+    step, inv = orc.calibrate(d, g, bits, synth.bf16_bits(cal), ref_base=synth.bf16_bits(calr), clip_sigmas=1.5)
+    assert np.all(step[0] > 0) and np.all(step[1] == 0)  # no direct tokens in the draw
+    payload, dg = orc.encode(d, g, bits, topk, Xb, ref_base=Rb, step=step, inv_step=inv, diag=True)
+    xh = orc.reconstruct(d, g, bits, topk, payload, T, ref_base=Rb, step=step)
+    coef, codes, oi, ov = orc.split_payload(payload, T, d, g, bits, topk)
+    qmax = (1 << (bits - 1)) - 1
+    h = orc.bf16_to_f32(Xb).astype(np.float64)
+    r = orc.bf16_to_f32(Rb).astype(np.float64)
+    x_hat = orc.bf16_to_f32(xh).astype(np.float64)
+    alpha = np.repeat(f16(coef & 0xffff), g, axis=1)
+    beta = np.repeat(f16(coef >> 16), g, axis=1)
+    e = h - (alpha * r + beta)  # Eq. 7 from the WIRE coefficients, in binary64
+    assert np.allclose(dg["e"], e, rtol=0, atol=np.abs(h).max() * 2.0 ** -22)
+    q = np.stack([orc.unpack_codes(codes[t], d, bits) for t in range(T)])
+    assert q.min() >= -qmax and q.max() <= qmax  # reserved code never produced
+    is_out = np.zeros((T, d), bool)
+    if topk:
+        is_out[np.arange(T)[:, None], oi.astype(np.int64)] = True
+        assert np.all(q[is_out] == 0)  # E^d = E - O: dense value at an outlier position is zero
+    # e_hat as the receiver sees it, from the payload alone
+    e_hat = q * step[0].astype(np.float64)
+    if topk:
+        e_hat[np.arange(T)[:, None], oi.astype(np.int64)] = f16(ov)
+    # Eq. 10: H - H_hat == E - E_hat, up to the final bf16 rounding of H_hat
+    lhs = h - x_hat
+    rhs = e - e_hat
+    assert np.all(np.abs(lhs - rhs) <= np.abs(x_hat) * 2.0 ** -8 + 1e-30)
+    # Eq. 11 with a static step: half a step inside the clip range, exact saturation outside
+    s = step[0].astype(np.float64)[None, :]
+    v = e / s
+    inside = (np.abs(v) <= qmax + 0.5) & ~is_out
+    assert np.all(np.abs(e - e_hat)[inside] <= 0.5 * s.repeat(T, 0)[inside] * (1 + 1e-6))
+    clipped = (np.abs(v) > qmax + 0.5 + 1e-3) & ~is_out
+    assert clipped.any()
+    assert np.all(q[clipped] == (np.sign(v[clipped]) * qmax).astype(np.int64))
+    if topk:
+        # outliers are reproduced exactly: the receiver's value IS the stored binary16, which is the
+        # nearest binary16 to the residual
+        eo = dg["e"][is_out].astype(np.float64)
+        assert np.array_equal(f16(ov).reshape(-1), eo.astype(np.float16).astype(np.float64))
+        # and they are the k largest magnitudes of the token (strictly larger than every dense value
+        # except for exact ties)
+        ae = np.abs(dg["e"])
+        kth = np.where(is_out, ae, np.inf).min(axis=1)
+        assert np.all(np.where(is_out, 0, ae).max(axis=1) <= kth)
+
+
+def test_step_zero_means_code_zero_and_direct_row_is_used(orc):
+    d, g, T = 128, 64, 6
+    rng = np.random.default_rng(30)
+    Xb = bits_of(rng.standard_normal((T, d)))
+    Rb = bits_of(rng.standard_normal((T, d)))
+    step = np.zeros((2, d), np.float32)
+    step[0, ::2] = 0.25          # referenced tokens: every second channel coded
+    step[1, :] = 0.5             # direct tokens: coarser table
+    inv = np.where(step > 0, 1.0 / np.where(step > 0, step, 1), 123.0).astype(np.float32)  # garbage where step==0
+    ref_row = np.array([0, -1, 2, -1, 4, 5], np.int32)
+    payload = orc.encode(d, g, 4, 0, Xb, ref_base=Rb, ref_row=ref_row, step=step, inv_step=inv)
+    coef, codes, _, _ = orc.split_payload(payload, T, d, g, 4, 0)
+    q = np.stack([orc.unpack_codes(codes[t], d, 4) for t in range(T)])
+    for t in range(T):
+        if ref_row[t] >= 0:
+            assert not q[t, 1::2].any() and q[t, ::2].any()
+        else:
+            assert np.all((coef[t] & 0x7fff) == 0)  # alpha = 0 for direct tokens
+            assert np.count_nonzero(q[t]) > d // 4
+    xh = orc.reconstruct(d, g, 4, 0, payload, T, ref_base=Rb, ref_row=ref_row, step=step)
+    h = orc.bf16_to_f32(Xb).astype(np.float64)
+    err = np.abs(h - orc.bf16_to_f32(xh))
+    direct = ref_row < 0
+    assert np.all(err[direct] <= 0.25 + np.abs(h[direct]) * 2.0 ** -8)  # half of the direct-row step
+
+
+def test_rounding_is_half_to_even_at_every_boundary(orc):
+    # reference constant -> alpha = 0, beta = mean(h); choose h so that mean is 0 and e = h exactly.
+    # With step = 1 the scaled value is e itself: put every n + 0.5 in the input and read the codes.
+    for bits in (2, 3, 4):
+        qmax = (1 << (bits - 1)) - 1
+        halves = np.arange(-qmax - 2, qmax + 2) + 0.5
+        vals = np.concatenate([halves, -halves])            # symmetric -> zero mean
+        d = g = 64
+        row = np.zeros(d, np.float32)
+        row[:vals.size] = vals
+        assert row.sum() == 0 and vals.size <= d
+        Xb = bits_of(row[None, :])
+        step, inv = flat_tables(d, 1.0)
+        payload = orc.encode(d, g, bits, 0, Xb, step=step, inv_step=inv)
+        coef, codes, _, _ = orc.split_payload(payload, 1, d, g, bits, 0)
+        assert coef[0, 0] & 0x7fffffff == 0
+        q = orc.unpack_codes(codes[0], d, bits)
+        want = np.clip(np.round(row), -qmax, qmax).astype(np.int32)  # numpy's round is half-to-even
+        assert np.array_equal(q, want)
+
+
+# ------------------------------------------------------------------ outliers
+def test_outliers_brute_force_and_ties_to_lower_index(orc):
+    rng = np.random.default_rng(40)
+    d, g, T, k = 128, 64, 64, 8
+    # direct coding with zero-mean groups of small integers/4 -> plenty of exact ties in |e|
+    vals = rng.integers(-12, 13, size=(T, d)).astype(np.float32) / 4
+    vals -= vals.reshape(T, d // g, g).mean(axis=2).repeat(g, axis=1)
+    Xb = bits_of(vals)
+    step, inv = flat_tables(d, 0.25)
+    payload, dg = orc.encode(d, g, 4, k, Xb, step=step, inv_step=inv, diag=True)
+    _, _, oi, ov = orc.split_payload(payload, T, d, g, 4, k)
+    ties_seen = 0
+    for t in range(T):
+        e = dg["e"][t]
+        # brute force: stable sort by descending magnitude keeps the lower index first among equals
+        order = sorted(range(d), key=lambda c: (-abs(float(e[c])), c))[:k]
+        assert list(oi[t]) == sorted(order)
+        assert np.all(np.diff(oi[t].astype(int)) > 0)
+        kth = abs(float(e[order[-1]]))
+        ties_seen += int(np.sum(np.abs(e) == kth) > 1)
+        assert np.array_equal(f16(ov[t]), e[oi[t].astype(int)].astype(np.float16).astype(np.float64))
+    assert ties_seen > T // 2  # the tie rule is really exercised
+
+
+def test_reconstruct_reports_reserved_code(orc):
+    d, g = 64, 64
+    step, _ = flat_tables(d, 0.5)
+    rec = orc.record_bytes(d, g, 4, 0)
+    payload = np.zeros(rec, np.uint8)
+    payload[4] = 0x08  # channel 0 carries -8, which the encoder never emits
+    xh, status = orc.reconstruct(d, g, 4, 0, payload, 1, step=step, return_status=True)
+    assert status & 2
+    assert orc.bf16_to_f32(xh)[0, 0] == -4.0 and not orc.bf16_to_f32(xh)[0, 1:].any()
+
+
+# ------------------------------------------------------------------ forced coefficients, predictor stand-in
+def test_forced_coefficients_and_gain_bias_transform(orc):
+    d, g, T = 256, 128, 8
+    gen = synth.generator(50)
+    X = synth.activations(T, d, synth.channel_scale(d, 3), gen)
+    prev = synth.activations(T, d, synth.channel_scale(d, 3), gen)
+    gain, bias = synth.predictor_gain_bias(d, 0)
+    Xb, Pb = synth.bf16_bits(X), synth.bf16_bits(prev)
+    gb, bb = synth.f16_bits(gain), synth.f16_bits(bias)
+    step, inv = flat_tables(d, 0.1)
+    # transform applied inside == transform applied outside with torch's own bf16 rounding
+    R_outside = (gain.float() * prev.float() + bias.float()).to(torch.bfloat16)
+    p_in = orc.encode(d, g, 3, 0, Xb, ref_base=Pb, gain=gb, bias=bb, step=step, inv_step=inv)
+    p_out = orc.encode(d, g, 3, 0, Xb, ref_base=synth.bf16_bits(R_outside), step=step, inv_step=inv)
+    # float32 multiply-add without fusion can differ from fmaf by one rounding before the bf16 cast;
+    # accept the rare double-rounding difference but require near-total agreement
+    assert np.mean(p_in != p_out) < 0.01
+    x_in = orc.reconstruct(d, g, 3, 0, p_in, T, ref_base=Pb, gain=gb, bias=bb, step=step)
+    err = np.abs(orc.bf16_to_f32(x_in).astype(np.float64) - orc.bf16_to_f32(Xb))
+    # forcing the coefficients the encoder chose itself changes nothing
+    coef, _, _, _ = orc.split_payload(p_in, T, d, g, 3, 0)
+    p_forced = orc.encode(d, g, 3, 0, Xb, ref_base=Pb, gain=gb, bias=bb, step=step, inv_step=inv,
+                          forced_coef=coef.reshape(-1).copy())
+    assert np.array_equal(p_forced, p_in)
+    # forcing alpha=0, beta=0 codes X directly: error bounded by clip or half a step
+    zero = np.zeros(T * (d // g), np.uint32)
+    p_zero = orc.encode(d, g, 3, 0, Xb, ref_base=Pb, gain=gb, bias=bb, step=step, inv_step=inv, forced_coef=zero)
+    x_zero = orc.bf16_to_f32(orc.reconstruct(d, g, 3, 0, p_zero, T, ref_base=Pb, gain=gb, bias=bb, step=step))
+    h = orc.bf16_to_f32(Xb)
+    small = np.abs(h) <= 3.5 * 0.1
+    assert np.all(np.abs(h - x_zero)[small] <= 0.05 + 2.0 ** -8 * np.abs(h[small]))
+    assert err.shape == (T, d)
+
+
+def test_thread_count_does_not_change_the_payload(orc):
+    d, g, T = 256, 64, 37
+    gen = synth.generator(60)
+    X = synth.activations(T, d, synth.channel_scale(d, 4), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    step, inv = flat_tables(d, 0.02)
+    a = orc.encode(d, g, 4, 8, synth.bf16_bits(X), ref_base=synth.bf16_bits(R), step=step, inv_step=inv, nthreads=1)
+    b = orc.encode(d, g, 4, 8, synth.bf16_bits(X), ref_base=synth.bf16_bits(R), step=step, inv_step=inv, nthreads=4)
+    assert np.array_equal(a, b)
+    xa = orc.reconstruct(d, g, 4, 8, a, T, ref_base=synth.bf16_bits(R), step=step, nthreads=1)
+    xb = orc.reconstruct(d, g, 4, 8, a, T, ref_base=synth.bf16_bits(R), step=step, nthreads=3)
+    assert np.array_equal(xa, xb)
+
+
+def test_calibrated_step_is_three_sigma_rounded_up(orc):
+    d, g, bits, T = 256, 128, 4, 512
+    gen = synth.generator(70)
+    scale = synth.channel_scale(d, 5)
+    X = synth.activations(T, d, scale, gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    step, inv = orc.calibrate(d, g, bits, synth.bf16_bits(X), ref_base=synth.bf16_bits(R))
+    # independent estimate of the residual RMS with numpy least squares per (token, group)
+    h = X.float().numpy().astype(np.float64).reshape(T, d // g, g)
+    r = R.float().numpy().astype(np.float64).reshape(T, d // g, g)
+    rc = r - r.mean(-1, keepdims=True)
+    hc = h - h.mean(-1, keepdims=True)
+    a = (rc * hc).sum(-1, keepdims=True) / (rc * rc).sum(-1, keepdims=True)
+    b = h.mean(-1, keepdims=True) - a * r.mean(-1, keepdims=True)
+    # the residual is taken with the coefficients as they travel (binary16): on a heavy channel the
+    # rounding of alpha alone moves the residual by a visible amount
+    a16 = a.astype(np.float16).astype(np.float64)
+    b16 = b.astype(np.float16).astype(np.float64)
+    e = h - (a16 * r + b16)
+    sigma = np.sqrt((e ** 2).mean(axis=0)).reshape(d)
+    want = 3 * sigma / 7
+    # step is a binary16 value, >= the target (up to the small effect of coefficient rounding) and within one ulp
+    assert np.array_equal(step[0], step[0].astype(np.float16).astype(np.float32))
+    assert np.all(step[0] >= want * (1 - 2e-3))
+    assert np.all(step[0] <= want * (1 + 2e-3) + np.spacing(step[0].astype(np.float16)).astype(np.float64))
+    assert np.array_equal(inv[0], (np.float32(1) / step[0]).astype(np.float32))
+    assert not step[1].any() and not inv[1].any()
