@@ -1,0 +1,176 @@
+/*
+ * rac.h -- C ABI of the B200 (sm_100a) hot path of the RAC reference-aware
+ * activation codec.
+ *
+ * The operations follow the paper's statement of the problem: a boundary hidden
+ * state H [T,d] is coded as the residual against a shared, affinely aligned
+ * reference (Sec. III-A, Eq. 2; Sec. IV-C), the receiver adds the dequantised
+ * residual back (Eq. 9), the sender runs the same reconstruction so that later
+ * references stay in sync (Sec. IV-C, first paragraph), and for prefill uplinks
+ * the reference row of every token is picked by exact-token span retrieval over
+ * a history (Sec. IV-B.1, Eq. 3).
+ *
+ * Conventions
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller.  The library
+ *    allocates no device memory and frees none.  `cfg` structs and scalar
+ *    arguments are host values.
+ *  - Every call is asynchronous on `stream` (a cudaStream_t passed as void*;
+ *    NULL is the default stream).  Nothing synchronises the device.
+ *  - Return value: RAC_OK or a negative error.  Errors that the host can see
+ *    (bad sizes, NULL or misaligned pointers, unsupported configuration) are
+ *    returned BEFORE anything is launched and leave every output untouched.
+ *  - Anomalies only the device can see never trap: the kernel ORs RAC_STATUS_*
+ *    bits into `*dev_status` (device uint32, may be NULL) and finishes.
+ *  - bf16 tensors are row major [rows, d]; rows must start on 16-byte
+ *    boundaries (d is a multiple of 32, base pointers 16-byte aligned).
+ *
+ * Wire record of one token (little endian), records back to back in `payload`:
+ *     coef    J x u32      binary16 alpha in bits 0..15, binary16 beta in 16..31,  J = d/group
+ *     codes   d*bits/8 B   code of channel c in stream bits [c*bits, c*bits+bits); stream bit n is
+ *                          bit n%8 of byte n/8; two's complement; -2^(bits-1) is never produced
+ *     out_idx topk x u16   channel indices, ascending
+ *     out_val topk x u16   binary16 residuals of those channels (their dense code is 0)
+ *     zero padding to a multiple of 16 bytes
+ * rac_record_bytes() gives the stride.  A token range is a contiguous byte range.
+ */
+#ifndef RAC_H_
+#define RAC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RAC_OK            0
+#define RAC_EINVAL       -1   /* NULL pointer, negative size, inconsistent arguments           */
+#define RAC_EALIGN       -2   /* a pointer that must be 16-byte aligned is not                 */
+#define RAC_ESIZE        -3   /* a caller buffer (payload_cap, workspace_bytes) is too small   */
+#define RAC_EUNSUPPORTED -4   /* a configuration this build has no kernel for                  */
+#define RAC_ECUDA        -5   /* a CUDA runtime call failed (launch error, wrong device, ...)  */
+
+/* bits ORed into *dev_status by the kernels */
+#define RAC_STATUS_REF_RANGE     1u   /* a ref_row entry >= ref_rows: the token was coded/decoded as direct   */
+#define RAC_STATUS_RESERVED_CODE 2u   /* decode met the code -2^(bits-1); it was dequantised as that value     */
+#define RAC_STATUS_NONFINITE     4u   /* encode met a NaN/Inf in X or in the reference; that record is garbage */
+#define RAC_STATUS_TIMEOUT       8u   /* an on-chip copy did not complete within the wait limit; the kernel
+                                         stopped early and its outputs are incomplete                        */
+#define RAC_STATUS_OUTLIER_RANGE 16u  /* decode met an outlier index >= d and ignored that outlier            */
+
+/* Codec configuration (Sec. IV-C: calibration picks (g_a, g_q, q, k) per phase and direction; here
+ * g_a == g_q == group).
+ *   d       hidden width; multiple of 32, <= 8192
+ *   group   channels per alignment/quantisation group; power of two, 32..1024, divides d
+ *   bits    code width: 2, 3 or 4            (Qmax = 2^(bits-1) - 1, Eq. 8a)
+ *   topk    outliers per token kept as binary16, 0..16 (Sec. IV-C "Outlier Metadata"; per token here)
+ *   coef_fmt   0 = binary16 pair (the only format)
+ *   scale_mode 0 = static per-channel step table (the only mode)
+ *   flags   must be 0 */
+typedef struct {
+    int32_t d, group, bits, topk, coef_fmt, scale_mode, flags;
+} rac_codec_cfg;
+
+/* One selected span (Eq. 3): query[q_start .. q_start+len) == history[h_start .. h_start+len). */
+typedef struct {
+    int32_t q_start, h_start, len;
+} rac_span;
+
+const char *rac_version(void);
+const char *rac_strerror(int err);
+
+/* Record stride in bytes (0 for an invalid configuration) and payload size of T tokens. */
+size_t rac_record_bytes(const rac_codec_cfg *cfg);
+size_t rac_payload_bytes(const rac_codec_cfg *cfg, int64_t T);
+
+/* ---------------------------------------------------------------------------------------------
+ * Span retrieval for prefill uplinks (Sec. IV-B.1, Eq. 3).
+ *
+ * Every window of `min_ngram` consecutive history tokens is indexed in a hash table (keys are
+ * verified token by token, so hash collisions cannot change the result); of each distinct window
+ * the `max_hits` most recent (largest) start positions are kept.  For every query position the
+ * candidates are extended forward to their longest exact match, bounded by the end of the query
+ * and of the history; the longest wins, ties go to the larger history start.  A left-to-right scan
+ * then selects spans: at position i with a candidate of length L the span (i, j, L) is emitted and
+ * the scan moves to i+L, otherwise to i+1.
+ *
+ *   hist_tok   int32[n_hist]     history token ids (row j of the history state buffer belongs to token j)
+ *   query_tok  int32[n_query]    tokens of the current prompt
+ *   min_ngram  w, 1..32
+ *   max_hits   K, 1..16
+ *   ref_row    int32[n_query]    out: history row of every covered position, -1 elsewhere
+ *   spans      rac_span[n_query/min_ngram + 1]  out, in query order; may be NULL
+ *   n_spans    int32[1]          out (device)
+ *   workspace  >= rac_match_workspace_bytes(n_hist, n_query, max_hits) bytes, 16-byte aligned;
+ *              contents are scratch, nothing persists between calls
+ * n_hist and n_query must be below 2^30.  n_query == 0 is allowed (only n_spans is written). */
+size_t rac_match_workspace_bytes(int64_t n_hist, int64_t n_query, int32_t max_hits);
+int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *query_tok, int64_t n_query,
+                    int32_t min_ngram, int32_t max_hits, int32_t *ref_row, rac_span *spans, int32_t *n_spans,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* Receiver side of the retrieval: spans travel as control metadata, tokens do not.  Expands
+ * `*n_spans` spans into ref_row[n_query] (-1 where no span covers).  Spans reaching outside
+ * [0, n_query) are clipped. */
+int rac_spans_to_rows(const rac_span *spans, const int32_t *n_spans, int64_t n_query, int32_t *ref_row,
+                      void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Encode (Sec. IV-C: Eq. 6 grouped affine fit with the zero-variance rule and wire rounding,
+ * Eq. 7 aligned residual, outlier split, Eq. 8 symmetric quantisation, packing).
+ *
+ *   X         bf16[T,d]          activations to send
+ *   ref_base  bf16[ref_rows,d]   reference rows; NULL = every token is coded directly
+ *   ref_row   int32[T]           row of ref_base used by token t; NULL = row t (needs ref_rows >= T);
+ *                                negative = token coded directly (zero reference, alpha = 0,
+ *                                beta = group mean, step table row 1)
+ *   ref_gain, ref_bias  binary16[d], both or neither: the reference row is first mapped per channel to
+ *                                bf16(gain*r + bias) (stand-in for the decode predictor of Eq. 5)
+ *   step, inv_step  float[2,d]   quantiser step and its reciprocal per channel; row 0 for tokens with a
+ *                                reference, row 1 for direct tokens; step 0 means "code 0"
+ *   payload   >= T*record bytes, 16-byte aligned; payload_cap is its capacity
+ * The per-group fit is taken in binary32 on the device; its result, rounded to binary16, is what both
+ * ends use, so any rounding difference against a binary64 fit shows up only in `coef`. */
+int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T,
+               const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+               const void *ref_gain, const void *ref_bias,
+               const float *step, const float *inv_step,
+               void *payload, size_t payload_cap, uint32_t *dev_status, void *stream);
+
+/* Receiver reconstruction (Eq. 9): X_hat = bf16( (alpha*r + beta) + e_hat ), e_hat = code*step or the
+ * stored binary16 outlier.  Arguments as rac_encode.  X_hat bf16[T,d] must not overlap payload.  X_hat
+ * may be the very buffer that ref_base points to ONLY with ref_row == NULL (token t reads row t and
+ * writes row t; each row is read completely before it is written). */
+int rac_decode_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_t T,
+                           const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                           const void *ref_gain, const void *ref_bias, const float *step,
+                           void *X_hat, uint32_t *dev_status, void *stream);
+
+/* Sender-side reconstruction (Sec. IV-C: the sender applies the same wire-format reconstruction as the
+ * receiver so that subsequent references stay synchronised).  Same device code as
+ * rac_decode_reconstruct, hence bit-identical output. */
+int rac_sender_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_t T,
+                           const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                           const void *ref_gain, const void *ref_bias, const float *step,
+                           void *X_hat, uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Step tables from a calibration draw (the part of the offline calibration of Sec. IV-C that the
+ * codec needs as an input).  Runs the fit and the residual of rac_encode over T calibration tokens and
+ * sets, per channel and per table row (0: tokens with a reference, 1: direct tokens),
+ *     step = smallest binary16 >= clip_sigmas * sqrt(mean e^2) / Qmax,   inv_step = 1/step (binary32),
+ * both 0 for a row without tokens or a channel whose residual is identically 0.
+ *   step, inv_step  float[2,d]  out
+ *   workspace  >= rac_calibrate_workspace_bytes(cfg) bytes, 16-byte aligned scratch
+ * Deterministic for a given device (fixed partition of tokens, fixed summation order). */
+size_t rac_calibrate_workspace_bytes(const rac_codec_cfg *cfg);
+int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T,
+                        const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                        const void *ref_gain, const void *ref_bias, float clip_sigmas,
+                        float *step, float *inv_step, void *workspace, size_t workspace_bytes,
+                        uint32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAC_H_ */

@@ -1,0 +1,209 @@
+"""ctypes binding of ``librac.so`` -- argument marshalling only.
+
+Every function has the name and the argument order of its C entry point in
+``include/rac.h``.  Arguments are either raw addresses (int) or torch tensors
+living where the C function expects them (device pointers for the ``rac_*``
+calls); the binding checks dtype, contiguity and device, takes
+``tensor.data_ptr()`` and the current CUDA stream, calls the library and raises
+on a non-zero return code.  No arithmetic of the method happens here and there
+is no fallback: if the library cannot be loaded, importing callers get an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librac.so")
+
+RAC_OK = 0
+STATUS_REF_RANGE = 1
+STATUS_RESERVED_CODE = 2
+STATUS_NONFINITE = 4
+STATUS_TIMEOUT = 8
+STATUS_OUTLIER_RANGE = 16
+
+EXPORTS = [
+    "rac_version", "rac_strerror", "rac_record_bytes", "rac_payload_bytes",
+    "rac_match_workspace_bytes", "rac_match_spans", "rac_spans_to_rows",
+    "rac_encode", "rac_decode_reconstruct", "rac_sender_reconstruct",
+    "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
+]
+
+
+class RacError(RuntimeError):
+    def __init__(self, fn: str, code: int, msg: str):
+        super().__init__(f"{fn} failed: {code} ({msg})")
+        self.code = code
+
+
+class CodecCfg(C.Structure):
+    """Mirror of ``rac_codec_cfg``."""
+    _fields_ = [(n, C.c_int32) for n in ("d", "group", "bits", "topk", "coef_fmt", "scale_mode", "flags")]
+
+    def __init__(self, d: int, group: int, bits: int, topk: int = 0):
+        super().__init__(d, group, bits, topk, 0, 0, 0)
+
+    def __repr__(self):
+        return f"CodecCfg(d={self.d}, group={self.group}, bits={self.bits}, topk={self.topk})"
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def load() -> C.CDLL:
+    """Load the C-ABI library.  Raises if it has not been built (``__graft_entry__.build()``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_04991_b200.build` "
+                           "(there is no CPU fallback)")
+    l = C.CDLL(LIB_PATH)
+    vp, i64, i32, sz = C.c_void_p, C.c_int64, C.c_int32, C.c_size_t
+    cfgp = C.POINTER(CodecCfg)
+    l.rac_version.restype = C.c_char_p
+    l.rac_version.argtypes = []
+    l.rac_strerror.restype = C.c_char_p
+    l.rac_strerror.argtypes = [C.c_int]
+    l.rac_record_bytes.restype = sz
+    l.rac_record_bytes.argtypes = [cfgp]
+    l.rac_payload_bytes.restype = sz
+    l.rac_payload_bytes.argtypes = [cfgp, i64]
+    l.rac_match_workspace_bytes.restype = sz
+    l.rac_match_workspace_bytes.argtypes = [i64, i64, i32]
+    l.rac_match_spans.restype = C.c_int
+    l.rac_match_spans.argtypes = [vp, i64, vp, i64, i32, i32, vp, vp, vp, vp, sz, vp]
+    l.rac_spans_to_rows.restype = C.c_int
+    l.rac_spans_to_rows.argtypes = [vp, vp, i64, vp, vp]
+    l.rac_encode.restype = C.c_int
+    l.rac_encode.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    for name in ("rac_decode_reconstruct", "rac_sender_reconstruct"):
+        f = getattr(l, name)
+        f.restype = C.c_int
+        f.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, vp]
+    l.rac_calibrate_workspace_bytes.restype = sz
+    l.rac_calibrate_workspace_bytes.argtypes = [cfgp]
+    l.rac_calibrate_steps.restype = C.c_int
+    l.rac_calibrate_steps.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, C.c_float, vp, vp, vp, sz, vp, vp]
+    _lib = l
+    return l
+
+
+def _check(fn: str, rc: int) -> None:
+    if rc != RAC_OK:
+        raise RacError(fn, rc, load().rac_strerror(rc).decode())
+
+
+def _ptr(t, dtype=None, name="tensor") -> Optional[int]:
+    """Address of a tensor (or pass an int / None through)."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if not isinstance(t, torch.Tensor):
+        raise TypeError(f"{name}: expected a torch tensor, an address or None")
+    if not t.is_cuda:
+        raise ValueError(f"{name}: must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+_BF16 = torch.bfloat16
+_F16 = torch.float16
+_I32 = torch.int32
+_F32 = torch.float32
+_U8 = (torch.uint8, torch.int8)
+
+
+# ----------------------------------------------------------------------------- plain queries
+def rac_version() -> str:
+    return load().rac_version().decode()
+
+
+def rac_strerror(code: int) -> str:
+    return load().rac_strerror(int(code)).decode()
+
+
+def rac_record_bytes(cfg: CodecCfg) -> int:
+    return int(load().rac_record_bytes(C.byref(cfg)))
+
+
+def rac_payload_bytes(cfg: CodecCfg, T: int) -> int:
+    return int(load().rac_payload_bytes(C.byref(cfg), int(T)))
+
+
+def rac_match_workspace_bytes(n_hist: int, n_query: int, max_hits: int) -> int:
+    return int(load().rac_match_workspace_bytes(int(n_hist), int(n_query), int(max_hits)))
+
+
+def rac_calibrate_workspace_bytes(cfg: CodecCfg) -> int:
+    return int(load().rac_calibrate_workspace_bytes(C.byref(cfg)))
+
+
+# ----------------------------------------------------------------------------- device calls
+def rac_match_spans(hist_tok, n_hist, query_tok, n_query, min_ngram, max_hits, ref_row, spans, n_spans,
+                    workspace, workspace_bytes, stream=None) -> None:
+    rc = load().rac_match_spans(_ptr(hist_tok, _I32, "hist_tok"), int(n_hist), _ptr(query_tok, _I32, "query_tok"),
+                                int(n_query), int(min_ngram), int(max_hits), _ptr(ref_row, _I32, "ref_row"),
+                                _ptr(spans, _I32, "spans"), _ptr(n_spans, _I32, "n_spans"),
+                                _ptr(workspace, None, "workspace"), int(workspace_bytes),
+                                _stream() if stream is None else stream)
+    _check("rac_match_spans", rc)
+
+
+def rac_spans_to_rows(spans, n_spans, n_query, ref_row, stream=None) -> None:
+    rc = load().rac_spans_to_rows(_ptr(spans, _I32, "spans"), _ptr(n_spans, _I32, "n_spans"), int(n_query),
+                                  _ptr(ref_row, _I32, "ref_row"), _stream() if stream is None else stream)
+    _check("rac_spans_to_rows", rc)
+
+
+def rac_encode(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload, payload_cap,
+               dev_status, stream=None) -> None:
+    rc = load().rac_encode(C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(ref_base, _BF16, "ref_base"), int(ref_rows),
+                           _ptr(ref_row, _I32, "ref_row"), _ptr(ref_gain, _F16, "ref_gain"),
+                           _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"), _ptr(inv_step, _F32, "inv_step"),
+                           _ptr(payload, _U8, "payload"), int(payload_cap), _ptr(dev_status, _I32, "dev_status"),
+                           _stream() if stream is None else stream)
+    _check("rac_encode", rc)
+
+
+def _reconstruct(fn, cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, X_hat, dev_status, stream):
+    rc = getattr(load(), fn)(C.byref(cfg), _ptr(payload, _U8, "payload"), int(T), _ptr(ref_base, _BF16, "ref_base"),
+                             int(ref_rows), _ptr(ref_row, _I32, "ref_row"), _ptr(ref_gain, _F16, "ref_gain"),
+                             _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"), _ptr(X_hat, _BF16, "X_hat"),
+                             _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
+    _check(fn, rc)
+
+
+def rac_decode_reconstruct(cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, X_hat,
+                           dev_status, stream=None) -> None:
+    _reconstruct("rac_decode_reconstruct", cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step,
+                 X_hat, dev_status, stream)
+
+
+def rac_sender_reconstruct(cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, X_hat,
+                           dev_status, stream=None) -> None:
+    _reconstruct("rac_sender_reconstruct", cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step,
+                 X_hat, dev_status, stream)
+
+
+def rac_calibrate_steps(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, clip_sigmas, step, inv_step,
+                        workspace, workspace_bytes, dev_status, stream=None) -> None:
+    rc = load().rac_calibrate_steps(C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(ref_base, _BF16, "ref_base"),
+                                    int(ref_rows), _ptr(ref_row, _I32, "ref_row"), _ptr(ref_gain, _F16, "ref_gain"),
+                                    _ptr(ref_bias, _F16, "ref_bias"), float(clip_sigmas), _ptr(step, _F32, "step"),
+                                    _ptr(inv_step, _F32, "inv_step"), _ptr(workspace, None, "workspace"),
+                                    int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"),
+                                    _stream() if stream is None else stream)
+    _check("rac_calibrate_steps", rc)

@@ -1,0 +1,310 @@
+// Exact-token span retrieval for prefill uplinks (Sec. IV-B.1, Eq. 3) on the GPU.
+//
+// Index: an open-addressing hash table with one slot per DISTINCT w-token window of the history.  A slot
+// stores one representative start position (used to verify a key token by token, so hash collisions can
+// never change the result) and the K largest start positions of that window, found by K rounds of
+// atomicMax ("largest start below the previous round's").  Because every round is a maximum, the
+// table contents do not depend on the order in which threads run.
+// Query: one thread per query position looks its window up, extends each of the <= K candidates forward
+// to the longest exact match and keeps lexargmax(length, start).
+// Selection: the left-to-right scan of Eq. 3 visits a position, jumps by the span length if it has a
+// candidate and by one otherwise.  "Next position at or after p that has a candidate" is a parallel
+// suffix scan; the remaining chain (one hop per selected span) is walked by a single thread, and the
+// spans are expanded to per-token rows in parallel.
+#include "rac_common.cuh"
+
+namespace rac {
+
+struct MatchParams {
+    const int32_t *hist;
+    const int32_t *query;
+    int32_t *ref_row;
+    rac_span *spans_out;   // may be null
+    int32_t *n_spans;
+    // workspace sections
+    int32_t *rep;          // [M]      representative start of the slot's window, -1 = empty
+    int32_t *top;          // [M*K]    r-th largest start of the slot's window, -1 = none
+    int32_t *slot_of;      // [nwin]
+    int2 *best;            // [N]      (length, history start) of the best candidate, length 0 = none
+    int2 *hop;             // [N]      (next position >= p with a candidate, position after its span)
+    rac_span *spans_ws;    // [N/w + 1]
+    int n_hist, n_query, nwin, w, K;
+    unsigned int mask;     // M - 1
+};
+
+__device__ __forceinline__ unsigned int window_hash(const int32_t *tok, int w) {
+    unsigned long long h = 0x9E3779B97F4A7C15ull;
+    for (int m = 0; m < w; m++) {
+        h ^= (unsigned long long)(unsigned int)tok[m];
+        h *= 0xff51afd7ed558ccdull;
+        h ^= h >> 32;
+    }
+    return (unsigned int)h;
+}
+
+__device__ __forceinline__ bool same_window(const int32_t *a, const int32_t *b, int w) {
+    for (int m = 0; m < w; m++)
+        if (a[m] != b[m]) return false;
+    return true;
+}
+
+__global__ void match_init_kernel(MatchParams p, long long table_ints) {
+    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long k = i; k < table_ints; k += stride) p.rep[k] = -1;  // rep and top are contiguous
+    for (long long k = i; k < p.n_query; k += stride) p.ref_row[k] = -1;
+    if (i == 0) *p.n_spans = 0;
+}
+
+// one slot per distinct window: claim an empty slot or find the slot that already holds this window
+__global__ void match_insert_kernel(MatchParams p) {
+    int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= p.nwin) return;
+    const int32_t *win = p.hist + j;
+    unsigned int s = window_hash(win, p.w) & p.mask;
+    int slot = -1;
+    for (unsigned int probe = 0; probe <= p.mask; probe++) {
+        int cur = atomicCAS(&p.rep[s], -1, j);
+        if (cur == -1 || cur == j || same_window(p.hist + cur, win, p.w)) { slot = (int)s; break; }
+        s = (s + 1) & p.mask;
+    }
+    p.slot_of[j] = slot;  // the table has >= 2*nwin slots, so a slot is always found
+}
+
+// round r: the largest start of each window that is below the start found in round r-1
+__global__ void match_round_kernel(MatchParams p, int r) {
+    int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= p.nwin) return;
+    int s = p.slot_of[j];
+    if (s < 0) return;
+    int32_t *lst = p.top + (long long)s * p.K;
+    if (r == 0 || j < lst[r - 1]) atomicMax(&lst[r], j);
+}
+
+__global__ void match_query_kernel(MatchParams p) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.n_query) return;
+    int bestL = 0, bestj = -1;
+    if (i + p.w <= p.n_query && p.nwin > 0) {
+        const int32_t *win = p.query + i;
+        unsigned int s = window_hash(win, p.w) & p.mask;
+        int slot = -1;
+        for (unsigned int probe = 0; probe <= p.mask; probe++) {
+            int cur = p.rep[s];
+            if (cur < 0) break;  // empty slot ends the probe sequence: the window is not in the history
+            if (same_window(p.hist + cur, win, p.w)) { slot = (int)s; break; }
+            s = (s + 1) & p.mask;
+        }
+        if (slot >= 0) {
+            const int32_t *lst = p.top + (long long)slot * p.K;
+            for (int r = 0; r < p.K; r++) {
+                int j = lst[r];
+                if (j < 0) break;
+                int L = p.w;
+                while (i + L < p.n_query && j + L < p.n_hist && p.query[i + L] == p.hist[j + L]) L++;
+                if (L > bestL || (L == bestL && j > bestj)) { bestL = L; bestj = j; }
+            }
+        }
+    }
+    p.best[i] = make_int2(bestL, bestj);
+}
+
+// Single CTA.  (1) hop[p] = (s, s + len(s)) with s the first position >= p that has a candidate (n_query
+// if none); (2) one thread follows the chain from 0 and lists the spans; (3) all threads expand them.
+__global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p) {
+    __shared__ int warp_first[32];
+    __shared__ int s_nspans;
+    const int N = p.n_query;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    // contiguous range of whole 32-position tiles per warp
+    const int tiles = (N + 31) / 32;
+    const int tiles_per_warp = (tiles + nwarps - 1) / nwarps;
+    const int t_lo = warp * tiles_per_warp, t_hi = min(tiles, t_lo + tiles_per_warp);
+
+    // pass A: first position with a candidate in this warp's range
+    int first = N;
+    for (int tl = t_lo; tl < t_hi; tl++) {
+        int i = tl * 32 + lane;
+        bool st = i < N && p.best[i].x > 0;
+        unsigned int b = __ballot_sync(0xffffffffu, st);
+        if (b) { first = tl * 32 + __ffs(b) - 1; break; }
+    }
+    if (lane == 0) warp_first[warp] = first;
+    __syncthreads();
+    // first candidate position after this warp's range
+    int carry = N;
+    for (int w = nwarps - 1; w > warp; w--) carry = min(carry, warp_first[w]);
+    int carry_next = carry < N ? carry + p.best[carry].x : N;
+
+    // pass B: tiles backwards, carrying the next candidate position
+    for (int tl = t_hi - 1; tl >= t_lo; tl--) {
+        int i = tl * 32 + lane;
+        int len = i < N ? p.best[i].x : 0;
+        unsigned int b = __ballot_sync(0xffffffffu, len > 0);
+        unsigned int at_or_after = b >> lane;
+        int s = carry, nx = carry_next;
+        const int src = at_or_after ? lane + __ffs(at_or_after) - 1 : lane;
+        const int len_src = __shfl_sync(0xffffffffu, len, src);  // one convergent shuffle for all lanes
+        if (at_or_after) {
+            s = tl * 32 + src;
+            nx = s + len_src;
+        }
+        if (i < N) p.hop[i] = make_int2(s, nx);
+        if (b) {
+            int f = __ffs(b) - 1;
+            carry = tl * 32 + f;
+            carry_next = carry + __shfl_sync(0xffffffffu, len, f);
+        }
+    }
+    __syncthreads();
+
+    // (2) the serial part of Eq. 3: one dependent load per selected span
+    if (tid == 0) {
+        int n = 0, pos = 0;
+        while (pos < N) {
+            int2 h = p.hop[pos];
+            if (h.x >= N) break;
+            p.spans_ws[n].q_start = h.x;
+            p.spans_ws[n].len = h.y - h.x;
+            n++;
+            pos = h.y;
+        }
+        s_nspans = n;
+        *p.n_spans = n;
+    }
+    __syncthreads();
+
+    // (3) history starts and per-token rows
+    const int ns = s_nspans;
+    for (int sidx = warp; sidx < ns; sidx += nwarps) {
+        int q0 = p.spans_ws[sidx].q_start, len = p.spans_ws[sidx].len;
+        int h0 = p.best[q0].y;
+        if (lane == 0 && p.spans_out) {
+            p.spans_out[sidx].q_start = q0;
+            p.spans_out[sidx].h_start = h0;
+            p.spans_out[sidx].len = len;
+        }
+        for (int m = lane; m < len; m += 32) p.ref_row[q0 + m] = h0 + m;
+    }
+}
+
+__global__ void spans_to_rows_kernel(const rac_span *spans, const int32_t *n_spans, long long n_query, int32_t *ref_row) {
+    const int ns = *n_spans;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    for (int s = gw; s < ns; s += warps) {
+        long long q0 = spans[s].q_start, len = spans[s].len;
+        int h0 = spans[s].h_start;
+        for (long long m = lane; m < len; m += 32) {
+            long long i = q0 + m;
+            if (i >= 0 && i < n_query) ref_row[i] = h0 + (int)m;
+        }
+    }
+}
+
+__global__ void fill_i32_kernel(int32_t *dst, long long n, int32_t v) {
+    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    long long stride = (long long)gridDim.x * blockDim.x;
+    for (; i < n; i += stride) dst[i] = v;
+}
+
+static size_t align16(size_t v) { return (v + 15) / 16 * 16; }
+
+struct MatchLayout {
+    size_t rep, top, slot_of, best, hop, spans, total;
+    unsigned int M;
+};
+static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
+    MatchLayout L;
+    unsigned long long M = 1024;
+    while (M < 2ull * (unsigned long long)(n_hist > 0 ? n_hist : 1)) M <<= 1;
+    L.M = (unsigned int)M;
+    size_t o = 0;
+    L.rep = o;      o += (size_t)M * 4;                       // rep and top must stay contiguous (one fill)
+    L.top = o;      o = align16(o + (size_t)M * K * 4);
+    L.slot_of = o;  o = align16(o + (size_t)(n_hist > 0 ? n_hist : 1) * 4);
+    L.best = o;     o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 8);
+    L.hop = o;      o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 8);
+    L.spans = o;    o = align16(o + (size_t)(n_query + 1) * sizeof(rac_span));
+    L.total = o;
+    return L;
+}
+
+}  // namespace rac
+
+using namespace rac;
+
+extern "C" {
+
+size_t rac_match_workspace_bytes(int64_t n_hist, int64_t n_query, int32_t max_hits) {
+    if (n_hist < 0 || n_query < 0 || max_hits < 1 || max_hits > 16) return 0;
+    if (n_hist >= (1ll << 30) || n_query >= (1ll << 30)) return 0;
+    return match_layout(n_hist, n_query, max_hits).total;
+}
+
+int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *query_tok, int64_t n_query,
+                    int32_t min_ngram, int32_t max_hits, int32_t *ref_row, rac_span *spans, int32_t *n_spans,
+                    void *workspace, size_t workspace_bytes, void *stream) {
+    if (n_hist < 0 || n_query < 0 || !n_spans) return RAC_EINVAL;
+    if (n_hist >= (1ll << 30) || n_query >= (1ll << 30)) return RAC_EUNSUPPORTED;
+    if (min_ngram < 1 || min_ngram > 32) return RAC_EUNSUPPORTED;
+    if (max_hits < 1 || max_hits > 16) return RAC_EUNSUPPORTED;
+    if ((n_hist > 0 && !hist_tok) || (n_query > 0 && (!query_tok || !ref_row))) return RAC_EINVAL;
+    if (!workspace) return RAC_EINVAL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 15u) return RAC_EALIGN;
+    MatchLayout L = match_layout(n_hist, n_query, max_hits);
+    if (workspace_bytes < L.total) return RAC_ESIZE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    MatchParams p;
+    p.hist = hist_tok;
+    p.query = query_tok;
+    p.ref_row = ref_row;
+    p.spans_out = spans;
+    p.n_spans = n_spans;
+    p.rep = reinterpret_cast<int32_t *>(ws + L.rep);
+    p.top = reinterpret_cast<int32_t *>(ws + L.top);
+    p.slot_of = reinterpret_cast<int32_t *>(ws + L.slot_of);
+    p.best = reinterpret_cast<int2 *>(ws + L.best);
+    p.hop = reinterpret_cast<int2 *>(ws + L.hop);
+    p.spans_ws = reinterpret_cast<rac_span *>(ws + L.spans);
+    p.n_hist = (int)n_hist;
+    p.n_query = (int)n_query;
+    p.nwin = (int)(n_hist - min_ngram + 1 > 0 ? n_hist - min_ngram + 1 : 0);
+    p.w = min_ngram;
+    p.K = max_hits;
+    p.mask = L.M - 1;
+
+    const long long table_ints = (long long)L.M * (1 + max_hits);
+    const int tb = 256;
+    long long work = table_ints > n_query ? table_ints : n_query;
+    int init_blocks = (int)((work + tb - 1) / tb);
+    if (init_blocks > 148 * 8) init_blocks = 148 * 8;
+    if (init_blocks < 1) init_blocks = 1;
+    match_init_kernel<<<init_blocks, tb, 0, st>>>(p, table_ints);
+    if (p.nwin > 0 && n_query > 0) {
+        int nb = (p.nwin + tb - 1) / tb;
+        match_insert_kernel<<<nb, tb, 0, st>>>(p);
+        for (int r = 0; r < max_hits; r++) match_round_kernel<<<nb, tb, 0, st>>>(p, r);
+    }
+    if (n_query > 0) {
+        match_query_kernel<<<(int)((n_query + tb - 1) / tb), tb, 0, st>>>(p);
+        match_select_kernel<<<1, 1024, 0, st>>>(p);
+    }
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+int rac_spans_to_rows(const rac_span *spans, const int32_t *n_spans, int64_t n_query, int32_t *ref_row, void *stream) {
+    if (n_query < 0 || !n_spans) return RAC_EINVAL;
+    if (n_query == 0) return RAC_OK;
+    if (!spans || !ref_row) return RAC_EINVAL;
+    if (n_query >= (1ll << 30)) return RAC_EUNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int blocks = (int)((n_query + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    fill_i32_kernel<<<blocks, 256, 0, st>>>(ref_row, n_query, -1);
+    spans_to_rows_kernel<<<148, 256, 0, st>>>(spans, n_spans, n_query, ref_row);
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,175 @@
+"""Parity protocol between the CUDA codec and the CPU oracle (helper, not a test module).
+
+The device fits (alpha, beta) in binary32, the oracle in binary64; both round the result to
+binary16.  When the exact optimum sits next to a binary16 rounding midpoint the two can land on
+different neighbours, and from there every code of that group may differ.  So the comparison is
+staged:
+
+1. coefficient words: equal, or the device value is what the oracle's unrounded optimum rounds to
+   after a perturbation no larger than the binary32 evaluation error (5e-3 of a binary16 step, plus
+   for beta the cancellation term 1e-6*(|hbar| + |alpha*rbar|)); such flips are counted and
+   reported; every coefficient is within 1e-3 relative of the optimum;
+2. the oracle re-encodes with the DEVICE's coefficient words forced: codes, outlier indices and
+   outlier values must then be bit-identical, token for token;
+3. reconstruction: the device's decode of any payload must equal the oracle's decode of the same
+   payload bit for bit.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2608_04991_b200 import binding as rac
+from paper_2608_04991_b200 import synth
+
+ALPHA_WINDOW_ULP = 5e-3
+REL_TOL = 1e-3
+
+
+def f16v(bits):
+    return np.asarray(bits, np.uint16).view(np.float16).astype(np.float64)
+
+
+@dataclass
+class EncodeReport:
+    groups: int
+    alpha_flips: int
+    beta_flips: int
+    tokens_with_flip: int
+
+    def __str__(self):
+        return (f"{self.groups} groups: alpha flips {self.alpha_flips}, beta flips {self.beta_flips}, "
+                f"tokens touched {self.tokens_with_flip}")
+
+
+def _check_flips(name, gpu16, orc16, exact, window_abs):
+    """A device coefficient that differs from the oracle's is accepted only if a perturbation of the
+    exact optimum no larger than the window (binary32 evaluation error) rounds to it: the interval
+    [exact - W, exact + W] must reach the device value's binary16 rounding cell.
+    gpu16: uint16 bit patterns of the mismatching entries; exact: binary64 optimum."""
+    g = np.asarray(gpu16, np.uint16).view(np.float16)
+    below = np.nextafter(g, np.float16(-np.inf)).astype(np.float64)
+    above = np.nextafter(g, np.float16(np.inf)).astype(np.float64)
+    gv = g.astype(np.float64)
+    W = window_abs + ALPHA_WINDOW_ULP * np.maximum(above - gv, gv - below)
+    lo_cell, hi_cell = (gv + below) / 2, (gv + above) / 2
+    ok = (exact + W >= lo_cell) & (exact - W <= hi_cell)
+    assert np.all(ok), (f"{name}: {int((~ok).sum())} device coefficients are not a rounding of the exact optimum "
+                        f"within the window; first: device {gv[~ok][0]!r}, oracle {f16v(orc16)[~ok][0]!r}, "
+                        f"exact {exact[~ok][0]!r}")
+
+
+def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None, gain=None, bias=None,
+                   step=None, inv_step=None) -> EncodeReport:
+    d, g, bits, k = cfg.d, cfg.group, cfg.bits, cfg.topk
+    T = Xb.size // d
+    nthr = oracle.max_threads()
+    o_payload, dg = oracle.encode(d, g, bits, k, Xb, ref_base=ref_base, ref_row=ref_row, gain=gain, bias=bias,
+                                  step=step, inv_step=inv_step, diag=True, nthreads=nthr)
+    g_coef = oracle.split_payload(gpu_payload, T, d, g, bits, k)[0]
+    o_coef = oracle.split_payload(o_payload, T, d, g, bits, k)[0]
+    ga, gb = (g_coef & 0xffff).astype(np.uint16), (g_coef >> 16).astype(np.uint16)
+    oa, ob = (o_coef & 0xffff).astype(np.uint16), (o_coef >> 16).astype(np.uint16)
+    # 1e-3 relative (with the floor of one binary16 subnormal, and for beta the cancellation in hbar - alpha*rbar)
+    a_exact, b_exact = dg["alpha"], dg["beta"]
+    cancel = 1e-6 * (np.abs(dg["hbar"]) + np.abs(a_exact * dg["rbar"]))
+    assert np.all(np.abs(f16v(ga) - a_exact) <= REL_TOL * np.abs(a_exact) + 2.0 ** -24), "alpha beyond 1e-3 relative"
+    assert np.all(np.abs(f16v(gb) - b_exact) <= REL_TOL * np.abs(b_exact) + 2.0 ** -24 + cancel), "beta beyond 1e-3 relative"
+    ma, mb = ga != oa, gb != ob
+    # +0 and -0 are the same coefficient
+    ma &= ~(((ga | oa) & 0x7fff) == 0)
+    mb &= ~(((gb | ob) & 0x7fff) == 0)
+    if ma.any():
+        _check_flips("alpha", ga[ma], oa[ma], a_exact[ma], 0.0)
+    if mb.any():
+        _check_flips("beta", gb[mb], ob[mb], b_exact[mb], cancel[mb])
+    # stage 2: same coefficients -> everything else bit-identical
+    forced = oracle.encode(d, g, bits, k, Xb, ref_base=ref_base, ref_row=ref_row, gain=gain, bias=bias,
+                           step=step, inv_step=inv_step, forced_coef=g_coef.reshape(-1).copy(), nthreads=nthr)
+    if not np.array_equal(forced, gpu_payload):
+        rec = oracle.record_bytes(d, g, bits, k)
+        bad = np.flatnonzero((forced.reshape(T, rec) != gpu_payload.reshape(T, rec)).any(axis=1))
+        t = int(bad[0])
+        off = np.flatnonzero(forced.reshape(T, rec)[t] != gpu_payload.reshape(T, rec)[t])
+        raise AssertionError(f"payload differs from the oracle in {bad.size} tokens; first token {t}, "
+                             f"byte offsets {off[:8].tolist()} of {rec} (coef {4 * (d // g)}, codes {d * bits // 8})")
+    return EncodeReport(ma.size, int(ma.sum()), int(mb.sum()), int((ma | mb).any(axis=1).sum()))
+
+
+def to_dev(a, dev, dtype=None):
+    if a is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.view(dtype)
+    return t.to(dev)
+
+
+def gpu_encode(cfg, X, ref_base, ref_row, gain, bias, step, inv_step, pad=64):
+    """Runs rac_encode into a canary-padded buffer; returns (payload numpy, status)."""
+    dev = X.device
+    T = X.shape[0]
+    rec = rac.rac_record_bytes(cfg)
+    buf = torch.full((T * rec + 2 * pad,), 0xA5, dtype=torch.uint8, device=dev)
+    payload = buf[pad:pad + T * rec]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rac.rac_encode(cfg, X, T, ref_base, 0 if ref_base is None else ref_base.shape[0], ref_row, gain, bias,
+                   step, inv_step, payload, T * rec, status)
+    torch.cuda.synchronize()
+    host = buf.cpu().numpy()
+    assert np.all(host[:pad] == 0xA5) and np.all(host[pad + T * rec:] == 0xA5), "encode wrote outside the payload"
+    return host[pad:pad + T * rec].copy(), int(status.item())
+
+
+def gpu_decode(cfg, payload_np, T, ref_base, ref_row, gain, bias, step, dev, fn=None, pad_rows=1):
+    fn = fn or rac.rac_decode_reconstruct
+    d = cfg.d
+    payload = torch.from_numpy(payload_np).to(dev)
+    buf = torch.full(((T + 2 * pad_rows), d), -7.0, dtype=torch.bfloat16, device=dev)
+    xh = buf[pad_rows:pad_rows + T]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    fn(cfg, payload, T, ref_base, 0 if ref_base is None else ref_base.shape[0], ref_row, gain, bias, step, xh, status)
+    torch.cuda.synchronize()
+    assert torch.all(buf[:pad_rows] == -7.0) and torch.all(buf[pad_rows + T:] == -7.0), "decode wrote outside X_hat"
+    return xh, int(status.item())
+
+
+def round_trip_case(cfg, X, ref_base=None, ref_row=None, gain=None, bias=None, step=None, inv_step=None):
+    """Full protocol on one input set (torch CUDA tensors; step tables numpy float32[2,d]).
+    Returns (EncodeReport, gpu payload numpy, X_hat tensor)."""
+    dev = X.device
+    d, g, bits, k = cfg.d, cfg.group, cfg.bits, cfg.topk
+    T = X.shape[0]
+    step_d, inv_d = to_dev(step, dev), to_dev(inv_step, dev)
+    Xb = synth.bf16_bits(X)
+    Rb = None if ref_base is None else synth.bf16_bits(ref_base)
+    rr = None if ref_row is None else ref_row.cpu().numpy()
+    gb = None if gain is None else synth.f16_bits(gain)
+    bb = None if bias is None else synth.f16_bits(bias)
+    pay, st = gpu_encode(cfg, X, ref_base, ref_row, gain, bias, step_d, inv_d)
+    assert st == 0, f"encode status {st}"
+    rep = compare_encode(cfg, pay, Xb, Rb, rr, gb, bb, step, inv_step)
+    # receiver and sender on the device payload, against the oracle's decode of the same bytes
+    xr, st = gpu_decode(cfg, pay, T, ref_base, ref_row, gain, bias, step_d, dev)
+    assert st == 0, f"decode status {st}"
+    xs, st = gpu_decode(cfg, pay, T, ref_base, ref_row, gain, bias, step_d, dev, fn=rac.rac_sender_reconstruct)
+    assert torch.equal(xr, xs), "sender and receiver reconstructions differ"
+    o_x = oracle.reconstruct(d, g, bits, k, pay, T, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step,
+                             nthreads=oracle.max_threads())
+    assert np.array_equal(o_x, synth.bf16_bits(xr)), "device reconstruction differs from the oracle's"
+    # and the device's decode of the ORACLE's own payload
+    o_pay = oracle.encode(d, g, bits, k, Xb, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step, inv_step=inv_step,
+                          nthreads=oracle.max_threads())
+    xo, st = gpu_decode(cfg, o_pay, T, ref_base, ref_row, gain, bias, step_d, dev)
+    o_xo = oracle.reconstruct(d, g, bits, k, o_pay, T, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step,
+                              nthreads=oracle.max_threads())
+    assert st == 0 and np.array_equal(o_xo, synth.bf16_bits(xo)), "device decode of the oracle payload differs"
+    # spec tolerance on the end-to-end activations where no coefficient flipped (implied by the above,
+    # stated explicitly): abs 2e-2 / rel 1e-2
+    a, b = synth.bf16_from_bits(o_xo).float(), xr.float().cpu()
+    if rep.tokens_with_flip == 0:
+        assert torch.all((a - b).abs() <= 2e-2 + 1e-2 * a.abs())
+    return rep, pay, xr

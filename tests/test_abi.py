@@ -1,0 +1,85 @@
+"""The C-ABI library loads, exports every symbol the header declares, and rejects bad
+arguments on the host before anything is launched (no GPU needed)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def rac():
+    from paper_2608_04991_b200 import build, binding
+    build.build()
+    binding.load()
+    return binding
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "rac.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rac_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(rac):
+    names = declared_symbols()
+    assert len(names) >= 12
+    lib = rac.load()
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in rac.h but not exported by librac.so"
+    assert sorted(rac.EXPORTS) == names
+    for n in names:
+        assert callable(getattr(rac, n)), f"binding lacks {n}"
+
+
+def test_record_geometry_matches_the_wire_format(rac, orc):
+    for d, g, b, k in [(4096, 128, 4, 0), (4096, 128, 4, 8), (3584, 128, 3, 0), (5120, 128, 4, 8), (4096, 64, 2, 8),
+                       (4096, 64, 3, 8), (8192, 256, 4, 16), (64, 32, 2, 0)]:
+        cfg = rac.CodecCfg(d, g, b, k)
+        assert rac.rac_record_bytes(cfg) == orc.record_bytes(d, g, b, k)
+        assert rac.rac_payload_bytes(cfg, 1000) == 1000 * orc.record_bytes(d, g, b, k)
+    assert rac.rac_record_bytes(rac.CodecCfg(4096, 100, 4, 0)) == 0   # group does not divide d
+    assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 5, 0)) == 0   # unsupported width
+    assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 4, 17)) == 0
+    assert "sm_100a" in rac.rac_version()
+
+
+def test_host_side_rejections_happen_before_any_launch(rac):
+    lib = rac.load()
+    cfg = rac.CodecCfg(4096, 128, 4, 8)
+    bad = rac.CodecCfg(4096, 96, 4, 8)
+    A = 0x10000  # a 16-byte aligned fake address: never dereferenced because the call is rejected first
+    args = dict(X=A, T=16, ref_base=A, ref_rows=16, ref_row=None, ref_gain=None, ref_bias=None, step=A, inv_step=A,
+                payload=A, payload_cap=16 * 2208, dev_status=None, stream=0)
+
+    def enc(c=cfg, **kw):
+        a = dict(args, **kw)
+        return lib.rac_encode(C.byref(c), a["X"], a["T"], a["ref_base"], a["ref_rows"], a["ref_row"], a["ref_gain"],
+                              a["ref_bias"], a["step"], a["inv_step"], a["payload"], a["payload_cap"], a["dev_status"],
+                              a["stream"])
+    assert enc(c=bad) == -1                      # d % group
+    assert enc(c=rac.CodecCfg(4100, 4100 // 4, 4, 0)) in (-1, -4)
+    assert enc(T=-1) == -1
+    assert enc(X=None) == -1
+    assert enc(X=A + 2) == -2                    # misaligned
+    assert enc(payload=A + 8) == -2
+    assert enc(payload_cap=16 * 2208 - 1) == -3
+    assert enc(ref_rows=8) == -1                 # identity rows need ref_rows >= T
+    assert enc(ref_gain=A) == -1                 # gain without bias
+    assert enc(T=0, X=None, payload=None) == 0   # nothing to do
+    dec = lib.rac_decode_reconstruct(C.byref(cfg), None, 4, A, 4, None, None, None, A, A, None, 0)
+    assert dec == -1
+    assert lib.rac_decode_reconstruct(C.byref(cfg), A, 4, A, 4, None, None, None, A, A + 4, None, 0) == -2
+    # matcher
+    assert rac.rac_match_workspace_bytes(1000, 100, 8) > 0
+    assert rac.rac_match_workspace_bytes(1000, 100, 0) == 0
+    assert rac.rac_match_workspace_bytes(1000, 100, 17) == 0
+    need = rac.rac_match_workspace_bytes(1000, 100, 8)
+    m = lambda **kw: lib.rac_match_spans(kw.get("h", A), kw.get("nh", 1000), A, 100, kw.get("w", 4), kw.get("K", 8), A, None, A,
+                                         kw.get("ws", A), kw.get("wsb", need), 0)
+    assert m(w=0) == -4 and m(K=0) == -4 and m(wsb=need - 1) == -3 and m(ws=A + 4) == -2 and m(h=None) == -1
+    assert rac.rac_strerror(-3) == "caller buffer too small"
+    with pytest.raises(rac.RacError):
+        rac._check("x", -1)
