@@ -63,7 +63,7 @@ struct CodecParams {
     long long T;
     long long ref_rows;
     // geometry
-    int d, J, lpg, topk, rec, code_bytes, stages;
+    int d, J, lpg, lpg_shift, topk, rec, code_bytes, stages;
     float inv_group;
 };
 
@@ -93,7 +93,7 @@ __host__ __device__ inline EncSmem enc_smem_layout(int d, int rec, int stages, i
     s.stage_bytes = 4 * d;  // X row + R row
     s.rec0 = s.stage0 + stages * s.stage_bytes;
     s.es0 = align_up(s.rec0 + (calib ? 0 : kRecBufs * rec), 16);
-    int es_bytes = calib ? 2 * nthreads * 32 * 4 : (topk ? nthreads * 32 * 4 : 0);
+    int es_bytes = calib ? 2 * nthreads * 32 * 4 : 0;  // calibration accumulators (residuals reuse the stage)
     s.hot0 = s.es0 + es_bytes;
     s.cand0 = align_up(s.hot0 + (topk ? nthreads * 4 * 2 : 0), 16);
     s.crank0 = s.cand0 + (topk ? kCandCap * 8 : 0);
@@ -119,6 +119,43 @@ __host__ __device__ inline DecSmem dec_smem_layout(int d, int rec, int stages) {
 // ------------------------------------------------------------------------------------------------
 // device helpers
 // ------------------------------------------------------------------------------------------------
+typedef unsigned long long u64;
+
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 pfma(u64 a, u64 b, u64 c) {
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ u64 padd(u64 a, u64 b) {
+    u64 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ u64 psub(u64 a, u64 b) {
+    u64 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ u64 pmul(u64 a, u64 b) {
+    u64 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// a 32-bit word of two bf16 -> packed (even channel, odd channel) binary32, exact
+__device__ __forceinline__ u64 bf16x2_to_p(uint32_t w) {
+    return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+// bits of a where m is set, bits of b elsewhere
+__device__ __forceinline__ uint32_t bitsel(uint32_t a, uint32_t b, uint32_t m) { return (a & m) | (b & ~m); }
+
 // rotate the four entries right by rot (new[j] = old[(j - rot) & 3])
 __device__ __forceinline__ void rot_right4(uint32_t (&w)[4], int rot) {
     if (rot & 1) { uint32_t t = w[3]; w[3] = w[2]; w[2] = w[1]; w[1] = w[0]; w[0] = t; }
@@ -130,20 +167,29 @@ __device__ __forceinline__ void rot_left4(uint32_t (&w)[4], int rot) {
     if (rot & 2) { uint32_t t = w[0]; w[0] = w[2]; w[2] = t; t = w[1]; w[1] = w[3]; w[3] = t; }
 }
 
+// low BITS bits of eight integers -> one word, element 0 in the lowest field
+template <int BITS>
+__device__ __forceinline__ uint32_t pack8(const uint32_t (&b)[8]) {
+    if (BITS == 4) {
+        uint32_t b01 = bitsel(b[0], b[1] << 4, 0x0fu), b23 = bitsel(b[2], b[3] << 4, 0x0fu);
+        uint32_t b45 = bitsel(b[4], b[5] << 4, 0x0fu), b67 = bitsel(b[6], b[7] << 4, 0x0fu);
+        return __byte_perm(__byte_perm(b01, b23, 0x0040), __byte_perm(b45, b67, 0x0040), 0x5410);
+    } else {
+        constexpr uint32_t m1 = (1u << BITS) - 1u, m2 = (1u << (2 * BITS)) - 1u, m4 = (1u << (4 * BITS)) - 1u;
+        constexpr uint32_t m8 = (BITS * 8 == 32) ? 0xffffffffu : ((1u << (BITS * 8 % 32)) - 1u);
+        uint32_t p0 = bitsel(b[0], b[1] << BITS, m1), p1 = bitsel(b[2], b[3] << BITS, m1);
+        uint32_t p2 = bitsel(b[4], b[5] << BITS, m1), p3 = bitsel(b[6], b[7] << BITS, m1);
+        uint32_t q0 = bitsel(p0, p1 << (2 * BITS), m2), q1 = bitsel(p2, p3 << (2 * BITS), m2);
+        return bitsel(q0, q1 << (4 * BITS), m4) & m8;
+    }
+}
+
 // reference values of one slot (8 channels starting at channel c) from shared memory, with the optional
 // per-channel transform r <- bf16(gain*r + bias)
-__device__ __forceinline__ void load_ref_slot(uint32_t addr, bool has_ref, const uint16_t *gain, const uint16_t *bias,
-                                              int c, float2 (&r2)[4]) {
-    if (!has_ref) {
-#pragma unroll
-        for (int i = 0; i < 4; i++) r2[i] = make_float2(0.f, 0.f);
-        return;
-    }
+__device__ __forceinline__ void load_ref_slot(uint32_t addr, const uint16_t *gain, const uint16_t *bias, int c,
+                                              u64 (&r2)[4]) {
     uint4 w = lds128(addr);
-    r2[0] = bf16x2_to_f2(w.x);
-    r2[1] = bf16x2_to_f2(w.y);
-    r2[2] = bf16x2_to_f2(w.z);
-    r2[3] = bf16x2_to_f2(w.w);
+    const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
     if (gain) {
         uint4 gw = __ldg(reinterpret_cast<const uint4 *>(gain + c));
         uint4 bw = __ldg(reinterpret_cast<const uint4 *>(bias + c));
@@ -153,36 +199,45 @@ __device__ __forceinline__ void load_ref_slot(uint32_t addr, bool has_ref, const
         for (int i = 0; i < 4; i++) {
             float g0 = half_bits_to_float(gws[i] & 0xffff), g1 = half_bits_to_float(gws[i] >> 16);
             float b0 = half_bits_to_float(bws[i] & 0xffff), b1 = half_bits_to_float(bws[i] >> 16);
-            r2[i].x = bf16_round(__fmaf_rn(g0, r2[i].x, b0));
-            r2[i].y = bf16_round(__fmaf_rn(g1, r2[i].y, b1));
+            float r0 = __uint_as_float(ws[i] << 16), r1 = __uint_as_float(ws[i] & 0xffff0000u);
+            r2[i] = pack2(bf16_round(__fmaf_rn(g0, r0, b0)), bf16_round(__fmaf_rn(g1, r1, b1)));
         }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; i++) r2[i] = bf16x2_to_p(ws[i]);
     }
 }
 
-// thread 0: start the copies of iteration `it` (token t) into its stage
-__device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ctrl, uint32_t smem_base, int stage0,
-                                                  int stage_bytes, int x_off, int r_off, int stage, long long t,
-                                                  const void *first_src, uint32_t first_bytes) {
-    long long row = p.ref_row ? (long long)p.ref_row[t] : t;
-    if (!p.ref_base) row = -1;
-    if (row >= p.ref_rows) {
+// thread 0: reference row of token t (-1 = coded directly); flags rows beyond the buffer
+__device__ __forceinline__ int resolve_row(const CodecParams &p, int raw_row) {
+    if (!p.ref_base || raw_row < 0) return -1;
+    if (raw_row >= p.ref_rows) {
         if (p.status) atomicOr(p.status, RAC_STATUS_REF_RANGE);
-        row = -1;
+        return -1;
     }
-    if (row < 0) row = -1;
-    ctrl->row[stage] = (int)row;
-    uint32_t bar = smem_u32(&ctrl->bar[stage]);
-    uint32_t base = smem_base + stage0 + stage * stage_bytes;
-    uint32_t row_bytes = 2u * (uint32_t)p.d;
+    return raw_row;
+}
+// thread 0: start the copies of one token into a stage: `first` (X row or record) and, if any, its reference row
+__device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ctrl, uint32_t stage_addr, uint32_t r_off,
+                                                  int stage, int row, const void *first_src, uint32_t first_bytes) {
+    ctrl->row[stage] = row;
+    const uint32_t bar = smem_u32(&ctrl->bar[stage]);
+    const uint32_t row_bytes = 2u * (uint32_t)p.d;
     mbar_arrive_expect_tx(bar, first_bytes + (row >= 0 ? row_bytes : 0u));
-    bulk_load(base + x_off, first_src, first_bytes, bar);
-    if (row >= 0) bulk_load(base + r_off, p.ref_base + row * (long long)p.d, row_bytes, bar);
+    bulk_load(stage_addr, first_src, first_bytes, bar);
+    if (row >= 0) bulk_load(stage_addr + r_off, p.ref_base + (long long)row * p.d, row_bytes, bar);
 }
 
 // ------------------------------------------------------------------------------------------------
 // encode / calibrate
 // ------------------------------------------------------------------------------------------------
 // MODE 0: encode.  MODE 1: accumulate e^2 per channel for the step tables.
+//
+// Per token: (1) every thread pulls its 32 channels of X and of the reference row out of the stage,
+// (2) Eq. 6 statistics: in-thread sums with packed binary32 adds / fmas, then log2(lanes per group) shuffles,
+// (3) wire coefficients, residual, scaling, rounding by the magic-number add, packing, all per thread,
+// (4) with outliers: the residuals overwrite the thread's own slab of the stage (same bytes: 2+2 per
+//     channel in, 4 out) so that the selection can look at other threads' values.
 template <int BITS, bool TOPK, int MODE>
 __global__ void __launch_bounds__(256) encode_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -198,10 +253,10 @@ __global__ void __launch_bounds__(256) encode_kernel(const CodecParams p) {
     const int S = p.stages;
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     constexpr uint32_t cmask = (1u << BITS) - 1u;
+    const uint32_t row_bytes = 2u * (uint32_t)d;
 
     if (tid == 0) {
         for (int s = 0; s < S; s++) mbar_init(smem_u32(&ctrl->bar[s]), 1);
-        ctrl->abort = 0;
         ctrl->n_hot = 0;
         ctrl->n_cand = 0;
         mbar_init_fence();
@@ -216,292 +271,322 @@ __global__ void __launch_bounds__(256) encode_kernel(const CodecParams p) {
     }
     __syncthreads();
 
-    const long long first = blockIdx.x, stride = gridDim.x;
-    const long long n_my = (p.T > first) ? (p.T - first + stride - 1) / stride : 0;
-    const uint32_t row_bytes = 2u * (uint32_t)d;
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
 
+    // thread 0 keeps the reference row of the next token to issue one iteration ahead of its use
+    int next_raw = 0;
+    auto raw_row_of = [&](int k) -> int {  // raw ref_row entry of this CTA's k-th token
+        long long t = first + (long long)k * stride;
+        return p.ref_row ? p.ref_row[t] : (int)t;
+    };
     if (tid == 0) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
-            long long t = first + k * stride;
-            issue_token_loads(p, ctrl, sbase, L.stage0, L.stage_bytes, 0, 2 * d, k, t, p.X + t * (long long)d, row_bytes);
+            long long t = first + (long long)k * stride;
+            issue_token_loads(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, row_bytes, k, resolve_row(p, raw_row_of(k)),
+                              p.X + t * d, row_bytes);
         }
+        if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
     }
     int cnt_ref = 0, cnt_dir = 0;  // calibrate: tokens per table row (thread 0 only)
 
-    for (long long it = 0; it < n_my; it++) {
-        const long long t = first + it * stride;
-        const int stage = (int)(it % S);
-        const uint32_t parity = (uint32_t)((it / S) & 1);
-        if (tid == 0 && it + S - 1 < n_my) {
-            long long k = it + S - 1;
-            long long tk = first + k * stride;
-            issue_token_loads(p, ctrl, sbase, L.stage0, L.stage_bytes, 0, 2 * d, (int)(k % S), tk, p.X + tk * (long long)d,
-                              row_bytes);
-        }
-        if (!mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity)) {
-            ctrl->abort = 1;
-            if (p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
-        }
-        const int row = ctrl->row[stage];
-        const bool has_ref = row >= 0;
-        const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
-        const uint32_t rs = xs + 2 * d;
-        unsigned char *rec = smem + L.rec0 + (int)(it % kRecBufs) * p.rec;
+    // byte offsets of the four 16-byte pieces of this thread's slab, in slot order
+    uint32_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
+    // the shuffles of step (2) run under `valid`: name exactly the lanes that take part (a group's lanes are
+    // always all valid or all invalid, so every partner is in the mask)
+    const unsigned int group_mask = __ballot_sync(0xffffffffu, valid);
 
-        // ---- load the slab: 4 slots of 8 channels, slot j holds piece (j + rot) & 3
-        float2 x2[16], r2[16];
+    int stage = 0, rbuf = 0, issue_stage = S - 1;
+    bool aborted = false;
+    uint32_t parity = 0;
+    for (int it = 0; it < n_my; it++) {
+        const long long t = first + (long long)it * stride;
+        if (tid == 0 && it + S - 1 < n_my) {
+            const int k = it + S - 1;
+            const long long tk = first + (long long)k * stride;
+            issue_token_loads(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, row_bytes, issue_stage,
+                              resolve_row(p, next_raw), p.X + tk * d, row_bytes);
+            if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
+        }
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
+        if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
+        const bool has_ref = ctrl->row[stage] >= 0;
+        const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
+        const uint32_t rs = xs + row_bytes;
+        unsigned char *rec = smem + L.rec0 + rbuf * p.rec;
+        float cmax[4] = {0.f, 0.f, 0.f, 0.f};
+
+        if (valid) {
+            // ---- (1) the slab: 4 slots of 8 channels, slot j holds piece (j + rot) & 3
+            u64 x2[16], r2[16];
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            const int q = (j + rot) & 3;
-            const int c = tid * 32 + q * 8;
-            if (valid) {
-                uint4 w = lds128(xs + 2 * c);
-                x2[4 * j + 0] = bf16x2_to_f2(w.x);
-                x2[4 * j + 1] = bf16x2_to_f2(w.y);
-                x2[4 * j + 2] = bf16x2_to_f2(w.z);
-                x2[4 * j + 3] = bf16x2_to_f2(w.w);
-                float2 rr[4];
-                load_ref_slot(rs + 2 * c, has_ref, p.gain, p.bias, c, rr);
+            for (int j = 0; j < 4; j++) {
+                uint4 w = lds128(xs + off[j]);
+                x2[4 * j + 0] = bf16x2_to_p(w.x);
+                x2[4 * j + 1] = bf16x2_to_p(w.y);
+                x2[4 * j + 2] = bf16x2_to_p(w.z);
+                x2[4 * j + 3] = bf16x2_to_p(w.w);
+            }
+            if (has_ref) {
 #pragma unroll
-                for (int i = 0; i < 4; i++) r2[4 * j + i] = rr[i];
+                for (int j = 0; j < 4; j++) {
+                    u64 rr[4];
+                    load_ref_slot(rs + off[j], p.gain, p.bias, (int)(off[j] >> 1), rr);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[4 * j + i] = rr[i];
+                }
             } else {
 #pragma unroll
-                for (int i = 0; i < 4; i++) { x2[4 * j + i] = make_float2(0.f, 0.f); r2[4 * j + i] = make_float2(0.f, 0.f); }
+                for (int i = 0; i < 16; i++) r2[i] = 0ull;
             }
-        }
 
-        // ---- Eq. 6: centred sums over the group (this thread's 32 channels, then the group's lanes)
-        float2 sr2 = make_float2(0.f, 0.f), sh2 = make_float2(0.f, 0.f);
+            // ---- (2) Eq. 6: centred sums over the group
+            u64 sr2 = 0ull, sh2 = 0ull;
 #pragma unroll
-        for (int i = 0; i < 16; i++) { sr2 = add2(sr2, r2[i]); sh2 = add2(sh2, x2[i]); }
-        float sr = sr2.x + sr2.y, sh = sh2.x + sh2.y;
-        for (int o = p.lpg >> 1; o > 0; o >>= 1) {
-            sr += __shfl_xor_sync(0xffffffffu, sr, o);
-            sh += __shfl_xor_sync(0xffffffffu, sh, o);
-        }
-        if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
-            if (p.status) atomicOr(p.status, RAC_STATUS_NONFINITE);
-        }
-        const float rbar = sr * p.inv_group, hbar = sh * p.inv_group;
-        const float2 rbar2 = make_float2(rbar, rbar), hbar2 = make_float2(hbar, hbar);
-        float2 sxx2 = make_float2(0.f, 0.f), sxy2 = make_float2(0.f, 0.f);
+            for (int i = 0; i < 16; i++) { sr2 = padd(sr2, r2[i]); sh2 = padd(sh2, x2[i]); }
+            float sr, sr_hi, sh, sh_hi;
+            unpack2(sr2, sr, sr_hi);
+            unpack2(sh2, sh, sh_hi);
+            sr += sr_hi;
+            sh += sh_hi;
+            for (int o = p.lpg >> 1; o > 0; o >>= 1) {
+                sr += __shfl_xor_sync(group_mask, sr, o);
+                sh += __shfl_xor_sync(group_mask, sh, o);
+            }
+            if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
+                if (p.status) atomicOr(p.status, RAC_STATUS_NONFINITE);
+            }
+            const float rbar = sr * p.inv_group, hbar = sh * p.inv_group;
+            const u64 rbar2 = pack2(rbar, rbar), hbar2 = pack2(hbar, hbar);
+            u64 sxx2 = 0ull, sxy2 = 0ull;
 #pragma unroll
-        for (int i = 0; i < 16; i++) {
-            float2 dr = sub2(r2[i], rbar2), dh = sub2(x2[i], hbar2);
-            sxx2 = fma2(dr, dr, sxx2);
-            sxy2 = fma2(dr, dh, sxy2);
-        }
-        float sxx = sxx2.x + sxx2.y, sxy = sxy2.x + sxy2.y;
-        for (int o = p.lpg >> 1; o > 0; o >>= 1) {
-            sxx += __shfl_xor_sync(0xffffffffu, sxx, o);
-            sxy += __shfl_xor_sync(0xffffffffu, sxy, o);
-        }
-        // zero-variance rule, then wire rounding to binary16
-        float a_star = 0.f, b_star = hbar;
-        if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {
-            a_star = __fdiv_rn(sxy, sxx);
-            b_star = __fmaf_rn(-a_star, rbar, hbar);
-        }
-        const uint32_t a16 = float_to_half_bits_sat(a_star), b16 = float_to_half_bits_sat(b_star);
-        const float a = half_bits_to_float(a16), b = half_bits_to_float(b16);
-        const float2 a2 = make_float2(a, a), b2 = make_float2(b, b);
+            for (int i = 0; i < 16; i++) {
+                u64 dr = psub(r2[i], rbar2), dh = psub(x2[i], hbar2);
+                sxx2 = pfma(dr, dr, sxx2);
+                sxy2 = pfma(dr, dh, sxy2);
+            }
+            float sxx, sxx_hi, sxy, sxy_hi;
+            unpack2(sxx2, sxx, sxx_hi);
+            unpack2(sxy2, sxy, sxy_hi);
+            sxx += sxx_hi;
+            sxy += sxy_hi;
+            for (int o = p.lpg >> 1; o > 0; o >>= 1) {
+                sxx += __shfl_xor_sync(group_mask, sxx, o);
+                sxy += __shfl_xor_sync(group_mask, sxy, o);
+            }
+            // zero-variance rule, then wire rounding to binary16
+            float a_star = 0.f, b_star = hbar;
+            if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {
+                a_star = __fdiv_rn(sxy, sxx);
+                b_star = __fmaf_rn(-a_star, rbar, hbar);
+            }
+            const uint32_t a16 = float_to_half_bits_sat(a_star), b16 = float_to_half_bits_sat(b_star);
+            const float a = half_bits_to_float(a16), b = half_bits_to_float(b16);
+            const u64 a2 = pack2(a, a), b2 = pack2(b, b);
 
-        if (CALIB) {
-            // ---- accumulate e^2 of the thread's own channels (row 0: referenced, row 1: direct)
-            float4 *acc = reinterpret_cast<float4 *>(smem + L.es0) + (has_ref ? 0 : 8 * nt);
-            if (valid) {
+            if (CALIB) {
+                // ---- accumulate e^2 of the thread's own channels (row 0: referenced, row 1: direct)
+                float4 *acc = reinterpret_cast<float4 *>(smem + L.es0) + (has_ref ? 0 : 8 * nt);
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const int q = (j + rot) & 3;
 #pragma unroll
                     for (int hh = 0; hh < 2; hh++) {
-                        float2 e0 = sub2(x2[4 * j + 2 * hh], fma2(a2, r2[4 * j + 2 * hh], b2));
-                        float2 e1 = sub2(x2[4 * j + 2 * hh + 1], fma2(a2, r2[4 * j + 2 * hh + 1], b2));
+                        float e0, e1, e2, e3;
+                        unpack2(psub(x2[4 * j + 2 * hh], pfma(a2, r2[4 * j + 2 * hh], b2)), e0, e1);
+                        unpack2(psub(x2[4 * j + 2 * hh + 1], pfma(a2, r2[4 * j + 2 * hh + 1], b2)), e2, e3);
                         float4 v = acc[(2 * q + hh) * nt + tid];
-                        v.x = __fmaf_rn(e0.x, e0.x, v.x);
-                        v.y = __fmaf_rn(e0.y, e0.y, v.y);
-                        v.z = __fmaf_rn(e1.x, e1.x, v.z);
-                        v.w = __fmaf_rn(e1.y, e1.y, v.w);
+                        v.x = __fmaf_rn(e0, e0, v.x);
+                        v.y = __fmaf_rn(e1, e1, v.y);
+                        v.z = __fmaf_rn(e2, e2, v.z);
+                        v.w = __fmaf_rn(e3, e3, v.w);
                         acc[(2 * q + hh) * nt + tid] = v;
                     }
                 }
-            }
-            if (tid == 0) { if (has_ref) cnt_ref++; else cnt_dir++; }
-            __syncthreads();
-            if (ctrl->abort) break;
-            continue;
-        }
-
-        // ---- Eq. 7 residual, Eq. 8 quantisation with the static table, packing
-        if (valid && (lane & (p.lpg - 1)) == 0)
-            reinterpret_cast<uint32_t *>(rec)[(tid * 32) / (32 * p.lpg)] = a16 | (b16 << 16);
-        const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
-        uint32_t words[4];
-        float cm[4];
-#pragma unroll
-        for (int j = 0; j < 4; j++) {
-            const int q = (j + rot) & 3;
-            const int c = tid * 32 + q * 8;
-            float4 iv0 = make_float4(0.f, 0.f, 0.f, 0.f), iv1 = iv0;
-            if (valid) {
-                iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
-                iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
-            }
-            const float2 inv2[4] = {make_float2(iv0.x, iv0.y), make_float2(iv0.z, iv0.w), make_float2(iv1.x, iv1.y),
-                                    make_float2(iv1.z, iv1.w)};
-            uint32_t w = 0;
-            float m = 0.f;
-            float2 e2[4];
-#pragma unroll
-            for (int i = 0; i < 4; i++) {
-                e2[i] = sub2(x2[4 * j + i], fma2(a2, r2[4 * j + i], b2));
-                float2 v = mul2(e2[i], inv2[i]);
-                float t0 = fminf(fmaxf(v.x, -qmax), qmax), t1 = fminf(fmaxf(v.y, -qmax), qmax);
-                float2 tt = add2(make_float2(t0, t1), make_float2(kMagic, kMagic));
-                w |= (__float_as_uint(tt.x) & cmask) << (BITS * (2 * i));
-                w |= (__float_as_uint(tt.y) & cmask) << (BITS * (2 * i + 1));
-                if (TOPK) m = fmaxf(m, fmaxf(fabsf(e2[i].x), fabsf(e2[i].y)));
-            }
-            words[j] = w;
-            cm[j] = m;
-            if (TOPK && valid) {
-                float4 *es = reinterpret_cast<float4 *>(smem + L.es0);
-                es[(2 * q) * nt + tid] = make_float4(e2[0].x, e2[0].y, e2[1].x, e2[1].y);
-                es[(2 * q + 1) * nt + tid] = make_float4(e2[2].x, e2[2].y, e2[3].x, e2[3].y);
-            }
-        }
-        rot_right4(words, rot);  // words[q] is now the code word of piece q
-        if (valid) {
-            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + 4 * p.J) + tid * BITS;
-            if (BITS == 4) {
-                cw[0] = words[0]; cw[1] = words[1]; cw[2] = words[2]; cw[3] = words[3];
-            } else if (BITS == 3) {
-                cw[0] = words[0] | (words[1] << 24);
-                cw[1] = (words[1] >> 8) | (words[2] << 16);
-                cw[2] = (words[2] >> 16) | (words[3] << 8);
             } else {
-                cw[0] = words[0] | (words[1] << 16);
-                cw[1] = words[2] | (words[3] << 16);
-            }
-        }
-
-        if (TOPK) {
-            // ---- outlier split: the k largest |e| of the token, ties to the lower channel.
-            // Threshold: every warp contributes its c-th largest lane maximum, c = ceil(k / warps); the
-            // minimum of those has at least k elements at or above it.
-            unsigned int lm = valid ? __float_as_uint(fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]))) : 0u;
-            const int cth = (p.topk + nwarps - 1) / nwarps;
-            unsigned int v = lm, m = 0;
-            for (int r = 0; r < cth; r++) {
-                m = __reduce_max_sync(0xffffffffu, v);
-                if (r + 1 < cth) {
-                    unsigned int bal = __ballot_sync(0xffffffffu, v == m);
-                    if (lane == __ffs(bal) - 1) v = 0u;
-                }
-            }
-            if (lane == 0) ctrl->wtau[warp] = m;
-            __syncthreads();  // S1
-            unsigned int tau = 0xffffffffu;
-            for (int w = 0; w < nwarps; w++) tau = min(tau, ctrl->wtau[w]);
-            unsigned short *hot = reinterpret_cast<unsigned short *>(smem + L.hot0);
-            if (valid) {
-                rot_right4(reinterpret_cast<uint32_t(&)[4]>(cm), rot);  // cm[q]: maximum of piece q
+                // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
+                if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = a16 | (b16 << 16);
+                const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
+                const u64 magic2 = pack2(kMagic, kMagic);
+                uint32_t words[4];
 #pragma unroll
-                for (int q = 0; q < 4; q++) {
-                    if (__float_as_uint(cm[q]) >= tau) {
-                        int pos = atomicAdd(&ctrl->n_hot, 1);
-                        hot[pos] = (unsigned short)((tid << 2) | q);
+                for (int j = 0; j < 4; j++) {
+                    const int c = (int)(off[j] >> 1);
+                    const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
+                    const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
+                    const u64 inv2[4] = {pack2(iv0.x, iv0.y), pack2(iv0.z, iv0.w), pack2(iv1.x, iv1.y), pack2(iv1.z, iv1.w)};
+                    uint32_t bits8[8];
+                    float ev[8];
+                    float m = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 4; i++) {
+                        const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                        float v0, v1, t0, t1;
+                        unpack2(pmul(e, inv2[i]), v0, v1);
+                        t0 = fminf(fmaxf(v0, -qmax), qmax);
+                        t1 = fminf(fmaxf(v1, -qmax), qmax);
+                        unpack2(padd(pack2(t0, t1), magic2), t0, t1);
+                        bits8[2 * i] = __float_as_uint(t0);
+                        bits8[2 * i + 1] = __float_as_uint(t1);
+                        if (TOPK) {
+                            unpack2(e, ev[2 * i], ev[2 * i + 1]);
+                            m = fmaxf(m, fmaxf(fabsf(ev[2 * i]), fabsf(ev[2 * i + 1])));
+                        }
+                    }
+                    words[j] = pack8<BITS>(bits8);
+                    if (TOPK) {
+                        // (4) residuals of piece q go to float4 slots 2q, 2q+1 of the thread's 8 (0-3: X slab, 4-7: R slab)
+                        cmax[j] = m;
+                        const uint32_t q = (off[j] >> 4) & 3u;
+                        const uint32_t base = (q < 2 ? xs : rs) + (uint32_t)tid * 64u + (q & 1u) * 32u;
+                        sts128(base, make_uint4(__float_as_uint(ev[0]), __float_as_uint(ev[1]), __float_as_uint(ev[2]),
+                                                __float_as_uint(ev[3])));
+                        sts128(base + 16, make_uint4(__float_as_uint(ev[4]), __float_as_uint(ev[5]), __float_as_uint(ev[6]),
+                                                     __float_as_uint(ev[7])));
                     }
                 }
-            }
-            __syncthreads();  // S2
-            const int nh = ctrl->n_hot;
-            const float *esf = reinterpret_cast<const float *>(smem + L.es0);
-            unsigned long long *cand = reinterpret_cast<unsigned long long *>(smem + L.cand0);
-            unsigned short *crank = reinterpret_cast<unsigned short *>(smem + L.crank0);
-            for (int x = tid; x < nh * 8; x += nt) {
-                int h = hot[x >> 3], ht = h >> 2, hq = h & 3, i = x & 7;
-                float e = esf[(((2 * hq + (i >> 2)) * nt) + ht) * 4 + (i & 3)];
-                unsigned int key = __float_as_uint(e) & 0x7fffffffu;
-                if (key >= tau) {
-                    int c = ht * 32 + hq * 8 + i;
-                    int pos = atomicAdd(&ctrl->n_cand, 1);
-                    if (pos < kCandCap) cand[pos] = ((unsigned long long)key << 16) | (unsigned long long)(0xffff - c);
+                rot_right4(words, rot);  // words[q] is now the code word of piece q
+                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + 4 * p.J) + tid * BITS;
+                if (BITS == 4) {
+                    cw[0] = words[0]; cw[1] = words[1]; cw[2] = words[2]; cw[3] = words[3];
+                } else if (BITS == 3) {
+                    cw[0] = words[0] | (words[1] << 24);
+                    cw[1] = (words[1] >> 8) | (words[2] << 16);
+                    cw[2] = (words[2] >> 16) | (words[3] << 8);
+                } else {
+                    cw[0] = words[0] | (words[1] << 16);
+                    cw[1] = words[2] | (words[3] << 16);
                 }
             }
-            __syncthreads();  // S3
-            const int nc = ctrl->n_cand;
-            const int k = p.topk;
-            unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
-            unsigned short *oval = oidx + k;
-            uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
-            unsigned long long *sel = reinterpret_cast<unsigned long long *>(smem + L.sel0);
-            if (nc <= kCandCap) {
-                // rank by counting: candidate x is the (rank)-th largest
-                for (int x = tid; x < nc; x += nt) {
-                    unsigned long long mine = cand[x];
-                    int rk = 0;
-                    for (int y = 0; y < nc; y++) rk += (cand[y] > mine) ? 1 : 0;
-                    crank[x] = (unsigned short)rk;
-                    if (rk < k) sel[rk] = mine;
+        }
+
+        if (CALIB) {
+            if (tid == 0) { if (has_ref) cnt_ref++; else cnt_dir++; }
+            if (__syncthreads_or(timed_out)) { aborted = true; break; }  // one vote: every thread leaves together
+        } else {
+            if (TOPK) {
+                // ---- outlier split: the k largest |e| of the token, ties to the lower channel.
+                // Threshold: every warp contributes its c-th largest lane maximum, c = ceil(k / warps); the
+                // minimum of those has at least k elements at or above it.
+                unsigned int lm = __float_as_uint(fmaxf(fmaxf(cmax[0], cmax[1]), fmaxf(cmax[2], cmax[3])));
+                const int cth = (p.topk + nwarps - 1) / nwarps;
+                unsigned int v = lm, m = 0;
+                for (int r = 0; r < cth; r++) {
+                    m = __reduce_max_sync(0xffffffffu, v);
+                    if (r + 1 < cth) {
+                        unsigned int bal = __ballot_sync(0xffffffffu, v == m);
+                        if (lane == __ffs(bal) - 1) v = 0u;
+                    }
                 }
-            } else {
-                // rare: more candidates than the list holds (many equal magnitudes).  k rounds of a
-                // block-wide maximum over all residuals, each strictly below the previous pick.
-                unsigned long long prev = ~0ull;
-                for (int n = 0; n < k; n++) {
-                    unsigned long long best = 0ull;
-                    if (valid) {
-                        for (int f = 0; f < 8; f++) {
-                            for (int cc = 0; cc < 4; cc++) {
-                                float e = esf[((f * nt) + tid) * 4 + cc];
-                                int c = tid * 32 + f * 4 + cc;
-                                unsigned long long comp =
-                                    ((unsigned long long)(__float_as_uint(e) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
-                                // every composite is > 0 except |e| == 0 at channel 65535, which d <= 8192 excludes
+                if (lane == 0) ctrl->wtau[warp] = m;
+                __syncthreads();  // S1
+                unsigned int tau = 0xffffffffu;
+                for (int w = 0; w < nwarps; w++) tau = min(tau, ctrl->wtau[w]);
+                unsigned short *hot = reinterpret_cast<unsigned short *>(smem + L.hot0);
+                if (valid) {
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        if (__float_as_uint(cmax[j]) >= tau) {
+                            int pos = atomicAdd(&ctrl->n_hot, 1);
+                            hot[pos] = (unsigned short)((tid << 2) | ((off[j] >> 4) & 3u));
+                        }
+                    }
+                }
+                __syncthreads();  // S2
+                const int nh = ctrl->n_hot;
+                const unsigned char *xsp = smem + L.stage0 + stage * L.stage_bytes;
+                // residual of channel c, as stored in step (4)
+                auto e_of = [&](int c) -> float {
+                    const int th = c >> 5, f = (c >> 2) & 7;
+                    return *reinterpret_cast<const float *>(xsp + (f < 4 ? 0 : row_bytes) + th * 64 + (f & 3) * 16 + (c & 3) * 4);
+                };
+                unsigned long long *cand = reinterpret_cast<unsigned long long *>(smem + L.cand0);
+                unsigned short *crank = reinterpret_cast<unsigned short *>(smem + L.crank0);
+                for (int x = tid; x < nh * 8; x += nt) {
+                    const int h = hot[x >> 3];
+                    const int c = (h >> 2) * 32 + (h & 3) * 8 + (x & 7);
+                    const unsigned int key = __float_as_uint(e_of(c)) & 0x7fffffffu;
+                    if (key >= tau) {
+                        int pos = atomicAdd(&ctrl->n_cand, 1);
+                        if (pos < kCandCap) cand[pos] = ((unsigned long long)key << 16) | (unsigned long long)(0xffff - c);
+                    }
+                }
+                __syncthreads();  // S3
+                const int nc = ctrl->n_cand;
+                const int k = p.topk;
+                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                unsigned short *oval = oidx + k;
+                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
+                unsigned long long *sel = reinterpret_cast<unsigned long long *>(smem + L.sel0);
+                if (nc <= kCandCap) {
+                    // rank by counting: candidate x is the (rank)-th largest
+                    for (int x = tid; x < nc; x += nt) {
+                        const unsigned long long mine = cand[x];
+                        int rk = 0;
+                        for (int y = 0; y < nc; y++) rk += (cand[y] > mine) ? 1 : 0;
+                        crank[x] = (unsigned short)rk;
+                        if (rk < k) sel[rk] = mine;
+                    }
+                } else {
+                    // rare: more candidates than the list holds (many equal magnitudes).  k rounds of a
+                    // block-wide maximum over all residuals, each strictly below the previous pick.
+                    unsigned long long prev = ~0ull;
+                    for (int n = 0; n < k; n++) {
+                        unsigned long long best = 0ull;
+                        if (valid) {
+                            for (int cc = 0; cc < 32; cc++) {
+                                const int c = tid * 32 + cc;
+                                const unsigned long long comp =
+                                    ((unsigned long long)(__float_as_uint(e_of(c)) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
+                                // a composite is 0 only for |e| == 0 at channel 65535, which d <= 8192 excludes
                                 if (comp < prev && comp > best) best = comp;
                             }
                         }
+                        for (int o = 16; o > 0; o >>= 1) {
+                            unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+                            best = other > best ? other : best;
+                        }
+                        if (lane == 0) ctrl->red[warp] = best;
+                        __syncthreads();
+                        best = 0ull;
+                        for (int w = 0; w < nwarps; w++) best = ctrl->red[w] > best ? ctrl->red[w] : best;
+                        if (tid == 0) sel[n] = best;
+                        prev = best;
+                        __syncthreads();
                     }
-                    for (int o = 16; o > 0; o >>= 1) {
-                        unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-                        best = other > best ? other : best;
-                    }
-                    if (lane == 0) ctrl->red[warp] = best;
-                    __syncthreads();
-                    best = 0ull;
-                    for (int w = 0; w < nwarps; w++) best = ctrl->red[w] > best ? ctrl->red[w] : best;
-                    if (tid == 0) sel[n] = best;
-                    prev = best;
-                    __syncthreads();
                 }
+                __syncthreads();  // S4
+                if (tid < k) {
+                    const unsigned long long mine = sel[tid];
+                    const int c = 0xffff - (int)(mine & 0xffffull);
+                    if (c < d) {
+                        int pos = 0;
+                        for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
+                        oidx[pos] = (unsigned short)c;
+                        oval[pos] = (unsigned short)float_to_half_bits_sat(e_of(c));
+                        // E^d = E - O: the dense code at an outlier position is zero
+                        const int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
+                        atomicAnd(&codes32[wd], ~(cmask << sh));
+                        if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
+                    }
+                }
+                if (tid == 0) { ctrl->n_hot = 0; ctrl->n_cand = 0; }
             }
-            __syncthreads();  // S4
-            if (tid < k) {
-                unsigned long long mine = sel[tid];
-                int c = 0xffff - (int)(mine & 0xffffull);
-                int pos = 0;
-                for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
-                float e = esf[((((c & 31) >> 2) * nt) + (c >> 5)) * 4 + (c & 3)];
-                oidx[pos] = (unsigned short)c;
-                oval[pos] = (unsigned short)float_to_half_bits_sat(e);
-                // E^d = E - O: the dense code at an outlier position is zero
-                int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
-                atomicAnd(&codes32[wd], ~(cmask << sh));
-                if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
-            }
-            if (tid == 0) { ctrl->n_hot = 0; ctrl->n_cand = 0; }
-        }
 
-        // ---- record complete: hand it to the copy engine
-        fence_async_smem();
-        __syncthreads();  // A
-        if (ctrl->abort) break;
-        if (tid == 0) {
-            bulk_store(p.payload + t * (long long)p.rec, smem_u32(rec), (uint32_t)p.rec);
-            bulk_commit();
-            bulk_wait_read<1>();  // the record buffer written two iterations from now is free again
+            // ---- record complete: hand it to the copy engine
+            fence_async_smem();
+            if (__syncthreads_or(timed_out)) { aborted = true; break; }  // A; one vote: every thread leaves together
+            if (tid == 0) {
+                bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                bulk_commit();
+                bulk_wait_read<1>();  // the record buffer written two iterations from now is free again
+            }
         }
+        if (++stage == S) { stage = 0; parity ^= 1u; }
+        if (++issue_stage == S) issue_stage = 0;
+        if (++rbuf == kRecBufs) rbuf = 0;
     }
 
     if (CALIB) {
@@ -523,7 +608,7 @@ __global__ void __launch_bounds__(256) encode_kernel(const CodecParams p) {
     }
     if (tid == 0) {
         bulk_wait_all();
-        if (ctrl->abort) {
+        if (aborted) {
             // give copies that may still be in flight a bounded chance to land before the CTA retires
             for (int s = 0; s < S; s++) {
                 mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
@@ -565,10 +650,15 @@ __global__ void calib_finalize_kernel(const float *partial, int nblocks, int d, 
 // ------------------------------------------------------------------------------------------------
 // reconstruct (receiver and sender)
 // ------------------------------------------------------------------------------------------------
+// Per token: record and reference row arrive in a stage; every thread dequantises its 32 channels
+// (code -> binary32 through the 2^23 trick, times the step), adds the aligned reference, rounds to bf16
+// into an output row in shared memory, patches the outliers it owns, and the row leaves as one bulk store.
+// The step table row of referenced tokens lives in registers for the whole kernel (a thread always owns
+// the same channels); direct tokens read row 1 through L1.
 template <int BITS, int KT>
 __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    const int tid = threadIdx.x, nt = blockDim.x;
+    const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int rot = (lane >> 1) & 3;
     const int d = p.d;
@@ -579,84 +669,78 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     const int S = p.stages;
     constexpr uint32_t cmask = (1u << BITS) - 1u;
     constexpr uint32_t H = 1u << (BITS - 1);
-    // H replicated into the 8 fields of a code word, and 1 in every field
+    // 1 in every one of the 8 fields of a code word, and H in every field
     constexpr uint32_t ones = (BITS == 4) ? 0x11111111u : (BITS == 3) ? 0x00249249u : 0x00005555u;
     constexpr uint32_t highs = ones << (BITS - 1);
     constexpr float kBase = 8388608.0f + (float)H;  // 2^23 + H
+    const uint32_t row_bytes = 2u * (uint32_t)d;
 
     if (tid == 0) {
         for (int s = 0; s < S; s++) mbar_init(smem_u32(&ctrl->bar[s]), 1);
-        ctrl->abort = 0;
         mbar_init_fence();
     }
     __syncthreads();
 
-    const long long first = blockIdx.x, stride = gridDim.x;
-    const long long n_my = (p.T > first) ? (p.T - first + stride - 1) / stride : 0;
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
 
+    int next_raw = 0;
+    auto raw_row_of = [&](int k) -> int {
+        long long t = first + (long long)k * stride;
+        return p.ref_row ? p.ref_row[t] : (int)t;
+    };
     if (tid == 0) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
-            long long t = first + k * stride;
-            issue_token_loads(p, ctrl, sbase, L.stage0, L.stage_bytes, 0, L.rec_pad, k, t, p.payload + t * (long long)p.rec,
-                              (uint32_t)p.rec);
+            long long t = first + (long long)k * stride;
+            issue_token_loads(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row(p, raw_row_of(k)),
+                              p.payload + t * p.rec, (uint32_t)p.rec);
         }
+        if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
     }
 
-    for (long long it = 0; it < n_my; it++) {
-        const long long t = first + it * stride;
-        const int stage = (int)(it % S);
-        const uint32_t parity = (uint32_t)((it / S) & 1);
+    uint32_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
+    // step table, row 0, in slot order
+    u64 st0[16];
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+        if (valid) {
+            s0 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1)));
+            s1 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1) + 4));
+        }
+        st0[4 * j + 0] = pack2(s0.x, s0.y);
+        st0[4 * j + 1] = pack2(s0.z, s0.w);
+        st0[4 * j + 2] = pack2(s1.x, s1.y);
+        st0[4 * j + 3] = pack2(s1.z, s1.w);
+    }
+    const u64 base2 = pack2(kBase, kBase);
+
+    int stage = 0, obuf = 0, issue_stage = S - 1;
+    bool aborted = false;
+    uint32_t parity = 0;
+    for (int it = 0; it < n_my; it++) {
+        const long long t = first + (long long)it * stride;
         if (tid == 0 && it + S - 1 < n_my) {
-            long long k = it + S - 1;
-            long long tk = first + k * stride;
-            issue_token_loads(p, ctrl, sbase, L.stage0, L.stage_bytes, 0, L.rec_pad, (int)(k % S), tk,
-                              p.payload + tk * (long long)p.rec, (uint32_t)p.rec);
+            const int k = it + S - 1;
+            const long long tk = first + (long long)k * stride;
+            issue_token_loads(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
+                              resolve_row(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
+            if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
-        if (!mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity)) {
-            ctrl->abort = 1;
-            if (p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
-        }
-        const int row = ctrl->row[stage];
-        const bool has_ref = row >= 0;
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
+        if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
+        const bool has_ref = ctrl->row[stage] >= 0;
         const unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = sbase + L.stage0 + stage * L.stage_bytes + L.rec_pad;
-        unsigned char *ob = smem + L.out0 + (int)(it % kRecBufs) * 2 * d;
+        unsigned char *ob = smem + L.out0 + obuf * (int)row_bytes;
         const uint32_t obs = smem_u32(ob);
-        const float *step_tab = p.step + (has_ref ? 0 : d);
-
-        // outliers owned by this thread: value to write after the dense pass
-        unsigned int own_mask = 0;
-        unsigned short pv[KT > 0 ? KT : 1];
-        if (KT > 0) {
-            const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
-            const unsigned short *oval = oidx + p.topk;
-#pragma unroll
-            for (int n = 0; n < KT; n++) {
-                pv[n] = 0;
-                if (n < p.topk) {
-                    int c = oidx[n];
-                    if (c >= d) {
-                        if (tid == 0 && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
-                    } else if ((c >> 5) == tid) {
-                        float r = 0.f;
-                        if (has_ref) {
-                            r = __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(rec + L.rec_pad + 2 * c)) << 16);
-                            if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
-                        }
-                        uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[c / (32 * p.lpg)];
-                        float rt = __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16));
-                        float xh = __fadd_rn(rt, half_bits_to_float(oval[n]));
-                        pv[n] = __bfloat16_as_ushort(__float2bfloat16_rn(xh));
-                        own_mask |= 1u << n;
-                    }
-                }
-            }
-        }
 
         if (valid) {
-            const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[(tid * 32) / (32 * p.lpg)];
+            const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
             const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
-            const float2 a2 = make_float2(a, a), b2 = make_float2(b, b);
+            const u64 a2 = pack2(a, a), b2 = pack2(b, b);
             // code words of the four pieces, in piece order, then rotated into slot order
             const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + 4 * p.J) + tid * BITS;
             uint32_t words[4];
@@ -683,48 +767,74 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             rot_left4(words, rot);
 #pragma unroll
             for (int j = 0; j < 4; j++) {
-                const int q = (j + rot) & 3;
-                const int c = tid * 32 + q * 8;
-                float2 r2[4];
-                load_ref_slot(rs + 2 * c, has_ref, p.gain, p.bias, c, r2);
-                float4 s0 = __ldg(reinterpret_cast<const float4 *>(step_tab + c));
-                float4 s1 = __ldg(reinterpret_cast<const float4 *>(step_tab + c + 4));
-                const float2 st2[4] = {make_float2(s0.x, s0.y), make_float2(s0.z, s0.w), make_float2(s1.x, s1.y),
-                                       make_float2(s1.z, s1.w)};
+                const int c = (int)(off[j] >> 1);
+                u64 r2[4], st2[4];
+                if (has_ref) {
+                    load_ref_slot(rs + off[j], p.gain, p.bias, c, r2);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) st2[i] = st0[4 * j + i];
+                } else {
+                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c));
+                    const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c + 4));
+                    st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[i] = 0ull;
+                }
                 const uint32_t w = words[j];
                 uint32_t o[4];
 #pragma unroll
                 for (int i = 0; i < 4; i++) {
                     // exact integer -> binary32 without a convert: 2^23 + (code + H), minus (2^23 + H)
-                    float q0 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i))) & cmask));
-                    float q1 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i + 1))) & cmask));
-                    float2 qf = sub2(make_float2(q0, q1), make_float2(kBase, kBase));
-                    float2 eh = mul2(qf, st2[i]);
-                    float2 rt = fma2(a2, r2[i], b2);
-                    float2 xh = add2(rt, eh);
-                    o[i] = f2_to_bf16x2(xh.x, xh.y);
+                    const float q0 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i))) & cmask));
+                    const float q1 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i + 1))) & cmask));
+                    const u64 eh = pmul(psub(pack2(q0, q1), base2), st2[i]);
+                    float x0, x1;
+                    unpack2(padd(pfma(a2, r2[i], b2), eh), x0, x1);
+                    o[i] = f2_to_bf16x2(x0, x1);
                 }
-                sts128(obs + 2 * c, make_uint4(o[0], o[1], o[2], o[3]));
+                sts128(obs + off[j], make_uint4(o[0], o[1], o[2], o[3]));
+            }
+            if (KT > 0) {
+                // outliers whose channel this thread owns replace what the dense pass wrote
+                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                const unsigned short *oval = oidx + p.topk;
+#pragma unroll
+                for (int n = 0; n < KT; n++) {
+                    if (n < p.topk) {
+                        const int c = oidx[n];
+                        if ((c >> 5) == tid) {
+                            float r = 0.f;
+                            if (has_ref) {
+                                r = __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(rec + L.rec_pad + 2 * c)) << 16);
+                                if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                            }
+                            const float xh = __fadd_rn(__fmaf_rn(a, r, b), half_bits_to_float(oval[n]));
+                            reinterpret_cast<unsigned short *>(ob)[c] = __bfloat16_as_ushort(__float2bfloat16_rn(xh));
+                        }
+                    }
+                }
             }
         }
-        if (KT > 0) {
+        if (KT > 0 && tid == 0) {
             const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
-#pragma unroll
-            for (int n = 0; n < KT; n++)
-                if (own_mask & (1u << n)) reinterpret_cast<unsigned short *>(ob)[oidx[n]] = pv[n];
+            bool bad = false;
+            for (int n = 0; n < p.topk; n++) bad |= oidx[n] >= d;
+            if (bad && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
         }
         fence_async_smem();
-        __syncthreads();
-        if (ctrl->abort) break;
+        if (__syncthreads_or(timed_out)) { aborted = true; break; }  // one vote: every thread leaves together
         if (tid == 0) {
-            bulk_store(p.X_hat + t * (long long)d, obs, 2u * (uint32_t)d);
+            bulk_store(p.X_hat + t * d, obs, row_bytes);
             bulk_commit();
             bulk_wait_read<1>();
         }
+        if (++stage == S) { stage = 0; parity ^= 1u; }
+        if (++issue_stage == S) issue_stage = 0;
+        if (++obuf == kRecBufs) obuf = 0;
     }
     if (tid == 0) {
         bulk_wait_all();
-        if (ctrl->abort) {
+        if (aborted) {
             for (int s = 0; s < S; s++) {
                 mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
                 mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
@@ -793,6 +903,8 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     p->d = g.d;
     p->J = g.J;
     p->lpg = g.lpg;
+    p->lpg_shift = 0;
+    while ((1 << p->lpg_shift) < g.lpg) p->lpg_shift++;
     p->topk = g.topk;
     p->rec = g.rec;
     p->code_bytes = g.code_bytes;
