@@ -12,6 +12,7 @@
 // pieces (piece (j + lane/2) mod 4 in step j), which makes the 128-bit accesses bank-conflict free
 // on a plain linear row.
 #include <math.h>
+#include <stdlib.h>
 
 #include "rac_common.cuh"
 
@@ -184,6 +185,16 @@ __device__ __forceinline__ uint32_t pack8(const uint32_t (&b)[8]) {
     }
 }
 
+// Two signed integers saturated to BITS-bit two's complement and packed below the bits of c
+// (d = c << 2*BITS | sat(hi) << BITS | sat(lo)); BITS is 4 or 2.
+template <int BITS>
+__device__ __forceinline__ uint32_t sat_pack2(int hi, int lo, uint32_t c) {
+    uint32_t d;
+    if (BITS == 4) asm("cvt.pack.sat.s4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(lo), "r"(c));
+    else asm("cvt.pack.sat.s2.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(lo), "r"(c));
+    return d;
+}
+
 // reference values of one slot (8 channels starting at channel c) from shared memory, with the optional
 // per-channel transform r <- bf16(gain*r + bias)
 __device__ __forceinline__ void load_ref_slot(uint32_t addr, const uint16_t *gain, const uint16_t *bias, int c,
@@ -239,7 +250,7 @@ __device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ct
 // (4) with outliers: the residuals overwrite the thread's own slab of the stage (same bytes: 2+2 per
 //     channel in, 4 out) so that the selection can look at other threads' values.
 template <int BITS, bool TOPK, int MODE>
-__global__ void __launch_bounds__(256) encode_kernel(const CodecParams p) {
+__global__ void __launch_bounds__(256, 2) encode_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
@@ -342,39 +353,49 @@ __global__ void __launch_bounds__(256) encode_kernel(const CodecParams p) {
                 for (int i = 0; i < 16; i++) r2[i] = 0ull;
             }
 
-            // ---- (2) Eq. 6: centred sums over the group
-            u64 sr2 = 0ull, sh2 = 0ull;
+            // ---- (2) Eq. 6: centred sums over the group (two accumulators per sum keep the adders busy)
+            u64 sra = 0ull, srb = 0ull, sha = 0ull, shb = 0ull;
 #pragma unroll
-            for (int i = 0; i < 16; i++) { sr2 = padd(sr2, r2[i]); sh2 = padd(sh2, x2[i]); }
+            for (int i = 0; i < 16; i += 2) {
+                sra = padd(sra, r2[i]); srb = padd(srb, r2[i + 1]);
+                sha = padd(sha, x2[i]); shb = padd(shb, x2[i + 1]);
+            }
             float sr, sr_hi, sh, sh_hi;
-            unpack2(sr2, sr, sr_hi);
-            unpack2(sh2, sh, sh_hi);
+            unpack2(padd(sra, srb), sr, sr_hi);
+            unpack2(padd(sha, shb), sh, sh_hi);
             sr += sr_hi;
             sh += sh_hi;
-            for (int o = p.lpg >> 1; o > 0; o >>= 1) {
-                sr += __shfl_xor_sync(group_mask, sr, o);
-                sh += __shfl_xor_sync(group_mask, sh, o);
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                if (p.lpg > o) {
+                    sr += __shfl_xor_sync(group_mask, sr, o);
+                    sh += __shfl_xor_sync(group_mask, sh, o);
+                }
             }
             if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
                 if (p.status) atomicOr(p.status, RAC_STATUS_NONFINITE);
             }
             const float rbar = sr * p.inv_group, hbar = sh * p.inv_group;
             const u64 rbar2 = pack2(rbar, rbar), hbar2 = pack2(hbar, hbar);
-            u64 sxx2 = 0ull, sxy2 = 0ull;
+            u64 sxxa = 0ull, sxxb = 0ull, sxya = 0ull, sxyb = 0ull;
 #pragma unroll
-            for (int i = 0; i < 16; i++) {
-                u64 dr = psub(r2[i], rbar2), dh = psub(x2[i], hbar2);
-                sxx2 = pfma(dr, dr, sxx2);
-                sxy2 = pfma(dr, dh, sxy2);
+            for (int i = 0; i < 16; i += 2) {
+                u64 dr0 = psub(r2[i], rbar2), dh0 = psub(x2[i], hbar2);
+                u64 dr1 = psub(r2[i + 1], rbar2), dh1 = psub(x2[i + 1], hbar2);
+                sxxa = pfma(dr0, dr0, sxxa); sxya = pfma(dr0, dh0, sxya);
+                sxxb = pfma(dr1, dr1, sxxb); sxyb = pfma(dr1, dh1, sxyb);
             }
             float sxx, sxx_hi, sxy, sxy_hi;
-            unpack2(sxx2, sxx, sxx_hi);
-            unpack2(sxy2, sxy, sxy_hi);
+            unpack2(padd(sxxa, sxxb), sxx, sxx_hi);
+            unpack2(padd(sxya, sxyb), sxy, sxy_hi);
             sxx += sxx_hi;
             sxy += sxy_hi;
-            for (int o = p.lpg >> 1; o > 0; o >>= 1) {
-                sxx += __shfl_xor_sync(group_mask, sxx, o);
-                sxy += __shfl_xor_sync(group_mask, sxy, o);
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                if (p.lpg > o) {
+                    sxx += __shfl_xor_sync(group_mask, sxx, o);
+                    sxy += __shfl_xor_sync(group_mask, sxy, o);
+                }
             }
             // zero-variance rule, then wire rounding to binary16
             float a_star = 0.f, b_star = hbar;
@@ -417,25 +438,44 @@ __global__ void __launch_bounds__(256) encode_kernel(const CodecParams p) {
                     const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
                     const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
                     const u64 inv2[4] = {pack2(iv0.x, iv0.y), pack2(iv0.z, iv0.w), pack2(iv1.x, iv1.y), pack2(iv1.z, iv1.w)};
-                    uint32_t bits8[8];
                     float ev[8];
-                    float m = 0.f;
+                    float m0 = 0.f, m1 = 0.f;
+                    uint32_t w = 0;
+                    if (BITS == 3) {
+                        uint32_t bits8[8];
 #pragma unroll
-                    for (int i = 0; i < 4; i++) {
-                        const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
-                        float v0, v1, t0, t1;
-                        unpack2(pmul(e, inv2[i]), v0, v1);
-                        t0 = fminf(fmaxf(v0, -qmax), qmax);
-                        t1 = fminf(fmaxf(v1, -qmax), qmax);
-                        unpack2(padd(pack2(t0, t1), magic2), t0, t1);
-                        bits8[2 * i] = __float_as_uint(t0);
-                        bits8[2 * i + 1] = __float_as_uint(t1);
-                        if (TOPK) {
+                        for (int i = 0; i < 4; i++) {
+                            const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                            float v0, v1, t0, t1;
+                            unpack2(pmul(e, inv2[i]), v0, v1);
+                            t0 = fminf(fmaxf(v0, -qmax), qmax);
+                            t1 = fminf(fmaxf(v1, -qmax), qmax);
+                            unpack2(padd(pack2(t0, t1), magic2), t0, t1);
+                            bits8[2 * i] = __float_as_uint(t0);
+                            bits8[2 * i + 1] = __float_as_uint(t1);
                             unpack2(e, ev[2 * i], ev[2 * i + 1]);
-                            m = fmaxf(m, fmaxf(fabsf(ev[2 * i]), fabsf(ev[2 * i + 1])));
+                        }
+                        w = pack8<BITS>(bits8);
+                    } else {
+                        // 4- and 2-bit codes: clamp from below in binary32, round by the magic add, take the integer
+                        // out of the mantissa and let the saturating pack clamp from above (its range is
+                        // [-2^(BITS-1), 2^(BITS-1)-1], whose upper end is Qmax)
+#pragma unroll
+                        for (int i = 3; i >= 0; i--) {
+                            const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                            float v0, v1, t0, t1;
+                            unpack2(pmul(e, inv2[i]), v0, v1);
+                            unpack2(padd(pack2(fmaxf(v0, -qmax), fmaxf(v1, -qmax)), magic2), t0, t1);
+                            w = sat_pack2<BITS>((int)__float_as_uint(t1) - 0x4b400000, (int)__float_as_uint(t0) - 0x4b400000, w);
+                            unpack2(e, ev[2 * i], ev[2 * i + 1]);
                         }
                     }
-                    words[j] = pack8<BITS>(bits8);
+                    words[j] = w;
+                    if (TOPK) {
+                        m0 = fmaxf(fmaxf(fabsf(ev[0]), fabsf(ev[1])), fmaxf(fabsf(ev[2]), fabsf(ev[3])));
+                        m1 = fmaxf(fmaxf(fabsf(ev[4]), fabsf(ev[5])), fmaxf(fabsf(ev[6]), fabsf(ev[7])));
+                    }
+                    const float m = fmaxf(m0, m1);
                     if (TOPK) {
                         // (4) residuals of piece q go to float4 slots 2q, 2q+1 of the thread's 8 (0-3: X slab, 4-7: R slab)
                         cmax[j] = m;
@@ -912,12 +952,18 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     return RAC_OK;
 }
 
-static int pick_stages(int d) { return d <= 4096 ? 3 : 2; }
+// Ring depth.  RAC_STAGES (2..4) overrides the default for tuning runs.
+static int pick_stages(int d, int dflt) {
+    const char *e = getenv("RAC_STAGES");
+    if (e && e[0] >= '2' && e[0] <= '4' && e[1] == 0) return e[0] - '0';
+    (void)d;
+    return dflt;
+}
 
 template <int MODE>
 static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
     const bool topk = g.topk > 0 && MODE == 0;
-    p.stages = pick_stages(g.d);
+    p.stages = pick_stages(g.d, g.d <= 4096 ? 3 : 2);
     EncSmem L = enc_smem_layout(g.d, g.rec, p.stages, g.nthreads, topk, MODE == 1);
 #define RAC_ENC(B, K) launch_persistent(encode_kernel<B, K, MODE>, p, g.nthreads, L.total, max_ctas, stream)
     switch (g.bits) {
@@ -930,7 +976,7 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
 }
 
 static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream) {
-    p.stages = 3;
+    p.stages = pick_stages(g.d, 2);
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
 #define RAC_DEC(B, K) launch_persistent(decode_kernel<B, K>, p, g.nthreads, L.total, p.T, stream)
@@ -1059,7 +1105,7 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, cons
     p.calib_partial = static_cast<float *>(workspace);
     // every CTA of the fixed grid writes its partials, also when it has no token
     {
-        p.stages = pick_stages(g.d);
+        p.stages = pick_stages(g.d, g.d <= 4096 ? 3 : 2);
         EncSmem L = enc_smem_layout(g.d, g.rec, p.stages, g.nthreads, false, true);
         DeviceInfo di;
         rc = device_info(&di);
