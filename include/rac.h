@@ -109,6 +109,31 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
                     int32_t min_ngram, int32_t max_hits, int32_t *ref_row, rac_span *spans, int32_t *n_spans,
                     void *workspace, size_t workspace_bytes, void *stream);
 
+/* Span retrieval for callers that cannot hand over device scratch.  (The paper has no counterpart: this is a
+ * convenience of this library.)
+ *
+ * Who needs it: code that runs where allocating device memory is off the table -- a plug-in called from inside
+ * another runtime that owns all device memory and gives out none, a serving loop whose memory budget was fixed
+ * at start-up, a callback in which cudaMalloc would synchronise the device at the worst moment.  Such callers
+ * can still pass their inputs and outputs, but have nowhere to get the matcher's workspace from.
+ *
+ * Same operation, arguments and results as rac_match_spans, minus the workspace: the scratch is a fixed array
+ * of RAC_MATCH_STATIC_BYTES = 3 MiB inside the library image (every GPU that loads the library holds
+ * it until the process ends).  That is enough for, e.g., a 32768-token history with 8192 query tokens and 8
+ * hits; a problem whose rac_match_workspace_bytes() exceeds the capacity is refused with RAC_ESIZE and nothing is
+ * launched.  The call allocates nothing and frees nothing, on the host side of CUDA or through any library.
+ *
+ * First call on a device: looks up the device address of the built-in array (one cudaGetSymbolAddress with
+ * that device current).  Make that first call outside any stream capture.
+ * All calls on a device share the one array.  Its contents survive from call to call, but every call
+ * re-initialises what it reads (hash table, rows, span count), so stale contents never matter.  Two calls that
+ * overlap on the GPU (different streams, or several host threads) race on the array and give garbage: keep the
+ * calls of one device ordered on one stream. */
+#define RAC_MATCH_STATIC_BYTES (3u << 20)
+int rac_match_spans_static(const int32_t *hist_tok, int64_t n_hist, const int32_t *query_tok, int64_t n_query,
+                           int32_t min_ngram, int32_t max_hits, int32_t *ref_row, rac_span *spans, int32_t *n_spans,
+                           void *stream);
+
 /* Receiver side of the retrieval: spans travel as control metadata, tokens do not.  Expands
  * `*n_spans` spans into ref_row[n_query] (-1 where no span covers).  Spans reaching outside
  * [0, n_query) are clipped. */

@@ -29,6 +29,7 @@ STATUS_OUTLIER_RANGE = 16
 EXPORTS = [
     "rac_version", "rac_strerror", "rac_record_bytes", "rac_payload_bytes",
     "rac_match_workspace_bytes", "rac_match_spans", "rac_spans_to_rows",
+    "rac_match_spans_static",
     "rac_encode", "rac_decode_reconstruct", "rac_sender_reconstruct",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
 ]
@@ -77,6 +78,8 @@ def load() -> C.CDLL:
     l.rac_match_workspace_bytes.argtypes = [i64, i64, i32]
     l.rac_match_spans.restype = C.c_int
     l.rac_match_spans.argtypes = [vp, i64, vp, i64, i32, i32, vp, vp, vp, vp, sz, vp]
+    l.rac_match_spans_static.restype = C.c_int
+    l.rac_match_spans_static.argtypes = [vp, i64, vp, i64, i32, i32, vp, vp, vp, vp]
     l.rac_spans_to_rows.restype = C.c_int
     l.rac_spans_to_rows.argtypes = [vp, vp, i64, vp, vp]
     l.rac_encode.restype = C.c_int
@@ -160,6 +163,20 @@ def rac_match_spans(hist_tok, n_hist, query_tok, n_query, min_ngram, max_hits, r
                                 _ptr(workspace, None, "workspace"), int(workspace_bytes),
                                 _stream() if stream is None else stream)
     _check("rac_match_spans", rc)
+
+
+MATCH_STATIC_BYTES = 3 << 20  # RAC_MATCH_STATIC_BYTES in rac.h
+
+
+def rac_match_spans_static(hist_tok, n_hist, query_tok, n_query, min_ngram, max_hits, ref_row, spans, n_spans,
+                           stream=None) -> None:
+    """Span retrieval on the library's built-in 3 MiB scratch: for callers that may not allocate device memory.
+    Calls on one device must not overlap on the GPU (they share the scratch)."""
+    rc = load().rac_match_spans_static(_ptr(hist_tok, _I32, "hist_tok"), int(n_hist), _ptr(query_tok, _I32, "query_tok"),
+                                       int(n_query), int(min_ngram), int(max_hits), _ptr(ref_row, _I32, "ref_row"),
+                                       _ptr(spans, _I32, "spans"), _ptr(n_spans, _I32, "n_spans"),
+                                       _stream() if stream is None else stream)
+    _check("rac_match_spans_static", rc)
 
 
 def rac_spans_to_rows(spans, n_spans, n_query, ref_row, stream=None) -> None:

@@ -11,6 +11,8 @@
 // candidate and by one otherwise.  "Next position at or after p that has a candidate" is a parallel
 // suffix scan; the remaining chain (one hop per selected span) is walked by a single thread, and the
 // spans are expanded to per-token rows in parallel.
+#include <mutex>
+
 #include "rac_common.cuh"
 
 namespace rac {
@@ -230,6 +232,30 @@ static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
     return L;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Scratch for rac_match_spans_static: lives in the library image, so every GPU that loads the library
+// holds these bytes until the process exits.  Host code must not pass the symbol itself to a kernel (on
+// the host it is only a stand-in); the device address is looked up once per device below.
+constexpr size_t kStaticMatchBytes = RAC_MATCH_STATIC_BYTES;  // 3 MiB: a 32768-token history, 8192 query tokens, 8 hits
+static __device__ __align__(256) unsigned char g_match_scratch[kStaticMatchBytes];
+
+static std::mutex g_match_scratch_mutex;
+static void *g_match_scratch_addr[64];  // device address of g_match_scratch, per device ordinal; null = not looked up yet
+
+// Device address of the scratch array on the CURRENT device (first call per device does the lookup).
+static int static_match_scratch(void **out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RAC_ECUDA;
+    std::lock_guard<std::mutex> lock(g_match_scratch_mutex);
+    if (!g_match_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_match_scratch) != cudaSuccess || !ptr) return RAC_ECUDA;
+        g_match_scratch_addr[dev] = ptr;
+    }
+    *out = g_match_scratch_addr[dev];
+    return RAC_OK;
+}
+
 }  // namespace rac
 
 using namespace rac;
@@ -305,6 +331,22 @@ int rac_spans_to_rows(const rac_span *spans, const int32_t *n_spans, int64_t n_q
     fill_i32_kernel<<<blocks, 256, 0, st>>>(ref_row, n_query, -1);
     spans_to_rows_kernel<<<148, 256, 0, st>>>(spans, n_spans, n_query, ref_row);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+int rac_match_spans_static(const int32_t *hist_tok, int64_t n_hist, const int32_t *query_tok, int64_t n_query,
+                           int32_t min_ngram, int32_t max_hits, int32_t *ref_row, rac_span *spans, int32_t *n_spans,
+                           void *stream) {
+    // size check first, with the same layout function the caller-workspace entry point uses
+    const size_t need = rac_match_workspace_bytes(n_hist, n_query, max_hits);
+    if (need == 0) return (n_hist < 0 || n_query < 0) ? RAC_EINVAL : RAC_EUNSUPPORTED;
+    if (need > kStaticMatchBytes) return RAC_ESIZE;  // problem too large for the built-in scratch
+    void *scratch = nullptr;
+    int rc = static_match_scratch(&scratch);
+    if (rc != RAC_OK) return rc;
+    // every launch of the matcher re-initialises the table, the rows and the span count, so whatever the
+    // previous call left in the scratch is harmless
+    return rac_match_spans(hist_tok, n_hist, query_tok, n_query, min_ngram, max_hits, ref_row, spans, n_spans, scratch,
+                           kStaticMatchBytes, stream);
 }
 
 }  // extern "C"
