@@ -118,7 +118,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------- workload
 class RoundTrip:
     """Device buffers and the ordered C-ABI calls of one step."""
-    LAUNCHES_PER_STEP = (4 + WORKLOAD["max_hits"]) + 2 + 3  # matcher kernels + 2 encodes + 3 reconstructions
+    LAUNCHES_PER_STEP = (4 + WORKLOAD["max_hits"]) + 2 * 2 + 3  # matcher kernels + 2 encodes (2 launches each) + 3 reconstructions
 
     def __init__(self, wl, seed, dev):
         import numpy as np
@@ -146,6 +146,8 @@ class RoundTrip:
         self.n_spans = z(1, dt=torch.int32)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.pay_up, self.pay_dn = z(T * self.rec), z(T * self.rec)
+        self.ews_bytes = rac.rac_encode_workspace_bytes(self.cfg, T)
+        self.ews = z(self.ews_bytes)
         self.Xs, self.Xh, self.Yh = (z(T, d, dt=torch.bfloat16) for _ in range(3))
         self.step_up, self.inv_up = z(2, d, dt=torch.float32), z(2, d, dt=torch.float32)
         self.step_dn, self.inv_dn = z(2, d, dt=torch.float32), z(2, d, dt=torch.float32)
@@ -174,7 +176,7 @@ class RoundTrip:
     def encode_up(self):
         w = self.wl
         self.rac.rac_encode(self.cfg, self.X, w["T"], self.Hs, w["n_hist"], self.ref_row, None, None, self.step_up,
-                            self.inv_up, self.pay_up, self.pay_up.numel(), self.status)
+                            self.inv_up, self.pay_up, self.pay_up.numel(), self.ews, self.ews_bytes, self.status)
 
     def sender_up(self):
         w = self.wl
@@ -189,7 +191,7 @@ class RoundTrip:
     def encode_dn(self):
         w = self.wl
         self.rac.rac_encode(self.cfg, self.Y, w["T"], self.Xh, w["T"], None, None, None, self.step_dn, self.inv_dn,
-                            self.pay_dn, self.pay_dn.numel(), self.status)
+                            self.pay_dn, self.pay_dn.numel(), self.ews, self.ews_bytes, self.status)
 
     def decode_dn(self):
         w = self.wl

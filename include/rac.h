@@ -154,13 +154,19 @@ int rac_spans_to_rows(const rac_span *spans, const int32_t *n_spans, int64_t n_q
  *   step, inv_step  float[2,d]   quantiser step and its reciprocal per channel; row 0 for tokens with a
  *                                reference, row 1 for direct tokens; step 0 means "code 0"
  *   payload   >= T*record bytes, 16-byte aligned; payload_cap is its capacity
+ *   workspace >= rac_encode_workspace_bytes(cfg, T) bytes of scratch, 16-byte aligned (0 bytes, and NULL
+ *             allowed, when cfg->topk == 0).  With outliers the call is two launches: the streaming pass leaves
+ *             the largest |e| of every 32-channel slab here (4*d/32 bytes per token) and the outlier pass reads it.
+ * The encoder reads only inv_step on the device: keep inv_step[c] == 0 wherever step[c] == 0 ("code 0").
  * The per-group fit is taken in binary32 on the device; its result, rounded to binary16, is what both
  * ends use, so any rounding difference against a binary64 fit shows up only in `coef`. */
+size_t rac_encode_workspace_bytes(const rac_codec_cfg *cfg, int64_t T);
 int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T,
                const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
                const void *ref_gain, const void *ref_bias,
                const float *step, const float *inv_step,
-               void *payload, size_t payload_cap, uint32_t *dev_status, void *stream);
+               void *payload, size_t payload_cap, void *workspace, size_t workspace_bytes,
+               uint32_t *dev_status, void *stream);
 
 /* Receiver reconstruction (Eq. 9): X_hat = bf16( (alpha*r + beta) + e_hat ), e_hat = code*step or the
  * stored binary16 outlier.  Arguments as rac_encode.  X_hat bf16[T,d] must not overlap payload.  X_hat

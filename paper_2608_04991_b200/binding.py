@@ -30,7 +30,7 @@ EXPORTS = [
     "rac_version", "rac_strerror", "rac_record_bytes", "rac_payload_bytes",
     "rac_match_workspace_bytes", "rac_match_spans", "rac_spans_to_rows",
     "rac_match_spans_static",
-    "rac_encode", "rac_decode_reconstruct", "rac_sender_reconstruct",
+    "rac_encode_workspace_bytes", "rac_encode", "rac_decode_reconstruct", "rac_sender_reconstruct",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
 ]
 
@@ -83,7 +83,9 @@ def load() -> C.CDLL:
     l.rac_spans_to_rows.restype = C.c_int
     l.rac_spans_to_rows.argtypes = [vp, vp, i64, vp, vp]
     l.rac_encode.restype = C.c_int
-    l.rac_encode.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    l.rac_encode_workspace_bytes.restype = sz
+    l.rac_encode_workspace_bytes.argtypes = [cfgp, i64]
+    l.rac_encode.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp]
     for name in ("rac_decode_reconstruct", "rac_sender_reconstruct"):
         f = getattr(l, name)
         f.restype = C.c_int
@@ -150,6 +152,10 @@ def rac_match_workspace_bytes(n_hist: int, n_query: int, max_hits: int) -> int:
     return int(load().rac_match_workspace_bytes(int(n_hist), int(n_query), int(max_hits)))
 
 
+def rac_encode_workspace_bytes(cfg: CodecCfg, T: int) -> int:
+    return int(load().rac_encode_workspace_bytes(C.byref(cfg), int(T)))
+
+
 def rac_calibrate_workspace_bytes(cfg: CodecCfg) -> int:
     return int(load().rac_calibrate_workspace_bytes(C.byref(cfg)))
 
@@ -186,11 +192,12 @@ def rac_spans_to_rows(spans, n_spans, n_query, ref_row, stream=None) -> None:
 
 
 def rac_encode(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload, payload_cap,
-               dev_status, stream=None) -> None:
+               workspace, workspace_bytes, dev_status, stream=None) -> None:
     rc = load().rac_encode(C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(ref_base, _BF16, "ref_base"), int(ref_rows),
                            _ptr(ref_row, _I32, "ref_row"), _ptr(ref_gain, _F16, "ref_gain"),
                            _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"), _ptr(inv_step, _F32, "inv_step"),
-                           _ptr(payload, _U8, "payload"), int(payload_cap), _ptr(dev_status, _I32, "dev_status"),
+                           _ptr(payload, _U8, "payload"), int(payload_cap), _ptr(workspace, None, "workspace"),
+                           int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"),
                            _stream() if stream is None else stream)
     _check("rac_encode", rc)
 

@@ -60,6 +60,7 @@ struct CodecParams {
     uint8_t *payload;          // encode out / decode in
     uint16_t *X_hat;           // decode out
     float *calib_partial;      // calibrate out: [grid][2][d] sums of e^2, then [grid][2] token counts
+    float *tmax;               // encode with outliers: [T][d/32] largest |e| per thread slab (caller workspace)
     uint32_t *status;
     long long T;
     long long ref_rows;
@@ -658,6 +659,423 @@ __global__ void __launch_bounds__(256, 2) encode_kernel(const CodecParams p) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// encode
+// ------------------------------------------------------------------------------------------------
+// Two launches.  (1) The streaming pass (this kernel): statistics, coefficients, residual, codes; every
+// warp of the CTA works on its 1024 channels of the token and ends with ONE arrival on the stage's `done`
+// mbarrier -- there is no CTA barrier in the loop.  Handing the finished record to the copy engine and
+// refilling the stage is the duty of warp (i mod warps) for token i; the other warps are already in the
+// next token and only ever wait for data (`full`).  With outliers, every thread also writes the largest
+// |e| of its 32 channels to the caller's workspace.  (2) outlier_kernel picks the k largest |e| per token
+// from those maxima with one warp per token -- thousands of tokens in flight, so the serial selection
+// (threshold, candidates, ranking) costs latency nobody waits for -- and patches the records in place.
+struct WsCtrl {
+    unsigned long long full[kMaxStages];
+    unsigned long long done[kMaxStages];
+    int row[kMaxStages];
+    int abort;
+};
+
+struct WsSmem {
+    int stage0, stage_bytes, rec_off, total;
+};
+__host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages) {
+    WsSmem s;
+    s.stage0 = align_up((int)sizeof(WsCtrl), 128);
+    s.rec_off = 4 * d;  // after X row + R row
+    s.stage_bytes = align_up(s.rec_off + rec, 128);
+    s.total = s.stage0 + stages * s.stage_bytes;
+    return s;
+}
+
+template <int BITS, bool TOPK, int MINB>
+__global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int rot = (lane >> 1) & 3;
+    const int d = p.d;
+    const bool valid = tid * 32 < d;
+    const WsSmem L = ws_smem_layout(d, p.rec, p.stages);
+    WsCtrl *ctrl = reinterpret_cast<WsCtrl *>(smem);
+    const uint32_t sbase = smem_u32(smem);
+    const int S = p.stages;
+    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
+    const uint32_t row_bytes = 2u * (uint32_t)d;
+
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+    auto raw_row_of = [&](int k) -> int {  // raw ref_row entry of this CTA's k-th token
+        long long t = first + (long long)k * stride;
+        return p.ref_row ? p.ref_row[t] : (int)t;
+    };
+    // one lane: start the copies of this CTA's k-th token into stage s
+    auto issue = [&](int k, int s, int raw_row) {
+        const long long t = first + (long long)k * stride;
+        const int row = resolve_row(p, raw_row);
+        ctrl->row[s] = row;
+        const uint32_t bar = smem_u32(&ctrl->full[s]);
+        const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
+        mbar_arrive_expect_tx(bar, row_bytes + (row >= 0 ? row_bytes : 0u));
+        bulk_load(base, p.X + t * d, row_bytes, bar);
+        if (row >= 0) bulk_load(base + row_bytes, p.ref_base + (long long)row * d, row_bytes, bar);
+    };
+
+    if (tid == 0) {
+        for (int s = 0; s < S; s++) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->done[s]), nwarps);
+        }
+        ctrl->abort = 0;
+        mbar_init_fence();
+    }
+    {
+        // padding words of the records are written once and never touched again
+        const int raw = 4 * p.J + p.code_bytes + 4 * p.topk;
+        for (int s = 0; s < S; s++)
+            for (int o = raw + 4 * tid; o < p.rec; o += 4 * nt)
+                *reinterpret_cast<uint32_t *>(smem + L.stage0 + s * L.stage_bytes + L.rec_off + o) = 0u;
+    }
+    __syncthreads();
+    if (tid == 0)
+        for (int k = 0; k < S && k < n_my; k++) issue(k, k, raw_row_of(k));
+
+    uint32_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
+    const unsigned int group_mask = __ballot_sync(0xffffffffu, valid);
+    const u64 magic2 = pack2(kMagic, kMagic);
+
+    int stage = 0, duty = 0;  // duty: the warp whose turn the tail of this token is
+    uint32_t parity = 0;
+    bool timed_out = false;
+    for (int it = 0; it < n_my; it++) {
+        if (*reinterpret_cast<volatile int *>(&ctrl->abort)) break;
+        unsigned char *stg = smem + L.stage0 + stage * L.stage_bytes;
+        const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
+        const uint32_t rs = xs + row_bytes;
+        unsigned char *rec = stg + L.rec_off;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
+        const bool has_ref = ctrl->row[stage] >= 0;
+
+        if (valid) {
+            // ---- (1) the slab: 4 slots of 8 channels, slot j holds piece (j + rot) & 3
+            u64 x2[16], r2[16];
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                uint4 w = lds128(xs + off[j]);
+                x2[4 * j + 0] = bf16x2_to_p(w.x);
+                x2[4 * j + 1] = bf16x2_to_p(w.y);
+                x2[4 * j + 2] = bf16x2_to_p(w.z);
+                x2[4 * j + 3] = bf16x2_to_p(w.w);
+            }
+            if (has_ref) {
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    u64 rr[4];
+                    load_ref_slot(rs + off[j], p.gain, p.bias, (int)(off[j] >> 1), rr);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[4 * j + i] = rr[i];
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; i++) r2[i] = 0ull;
+            }
+            // ---- (2) Eq. 6: centred sums over the group (two accumulators per sum keep the adders busy)
+            u64 sra = 0ull, srb = 0ull, sha = 0ull, shb = 0ull;
+#pragma unroll
+            for (int i = 0; i < 16; i += 2) {
+                sra = padd(sra, r2[i]); srb = padd(srb, r2[i + 1]);
+                sha = padd(sha, x2[i]); shb = padd(shb, x2[i + 1]);
+            }
+            float sr, sr_hi, sh, sh_hi;
+            unpack2(padd(sra, srb), sr, sr_hi);
+            unpack2(padd(sha, shb), sh, sh_hi);
+            sr += sr_hi;
+            sh += sh_hi;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                if (p.lpg > o) {
+                    sr += __shfl_xor_sync(group_mask, sr, o);
+                    sh += __shfl_xor_sync(group_mask, sh, o);
+                }
+            }
+            if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
+                if (p.status) atomicOr(p.status, RAC_STATUS_NONFINITE);
+            }
+            const float rbar = sr * p.inv_group, hbar = sh * p.inv_group;
+            const u64 rbar2 = pack2(rbar, rbar), hbar2 = pack2(hbar, hbar);
+            u64 sxxa = 0ull, sxxb = 0ull, sxya = 0ull, sxyb = 0ull;
+#pragma unroll
+            for (int i = 0; i < 16; i += 2) {
+                u64 dr0 = psub(r2[i], rbar2), dh0 = psub(x2[i], hbar2);
+                u64 dr1 = psub(r2[i + 1], rbar2), dh1 = psub(x2[i + 1], hbar2);
+                sxxa = pfma(dr0, dr0, sxxa); sxya = pfma(dr0, dh0, sxya);
+                sxxb = pfma(dr1, dr1, sxxb); sxyb = pfma(dr1, dh1, sxyb);
+            }
+            float sxx, sxx_hi, sxy, sxy_hi;
+            unpack2(padd(sxxa, sxxb), sxx, sxx_hi);
+            unpack2(padd(sxya, sxyb), sxy, sxy_hi);
+            sxx += sxx_hi;
+            sxy += sxy_hi;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                if (p.lpg > o) {
+                    sxx += __shfl_xor_sync(group_mask, sxx, o);
+                    sxy += __shfl_xor_sync(group_mask, sxy, o);
+                }
+            }
+            // zero-variance rule, then wire rounding to binary16
+            float a_star = 0.f, b_star = hbar;
+            if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {
+                a_star = __fdiv_rn(sxy, sxx);
+                b_star = __fmaf_rn(-a_star, rbar, hbar);
+            }
+            const uint32_t a16 = float_to_half_bits_sat(a_star), b16 = float_to_half_bits_sat(b_star);
+            const float a = half_bits_to_float(a16), b = half_bits_to_float(b16);
+            const u64 a2 = pack2(a, a), b2 = pack2(b, b);
+
+            // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
+            if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = a16 | (b16 << 16);
+            const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
+            uint32_t words[4];
+            float tmax = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                const int c = (int)(off[j] >> 1);
+                const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
+                const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
+                const u64 inv2[4] = {pack2(iv0.x, iv0.y), pack2(iv0.z, iv0.w), pack2(iv1.x, iv1.y), pack2(iv1.z, iv1.w)};
+                float ev[8];
+                uint32_t w = 0;
+                if (BITS == 3) {
+                    uint32_t bits8[8];
+#pragma unroll
+                    for (int i = 0; i < 4; i++) {
+                        const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                        float v0, v1, t0, t1;
+                        unpack2(pmul(e, inv2[i]), v0, v1);
+                        t0 = fminf(fmaxf(v0, -qmax), qmax);
+                        t1 = fminf(fmaxf(v1, -qmax), qmax);
+                        unpack2(padd(pack2(t0, t1), magic2), t0, t1);
+                        bits8[2 * i] = __float_as_uint(t0);
+                        bits8[2 * i + 1] = __float_as_uint(t1);
+                        unpack2(e, ev[2 * i], ev[2 * i + 1]);
+                    }
+                    w = pack8<BITS>(bits8);
+                } else {
+                    // 4- and 2-bit codes: clamp from below in binary32, round by the magic add, take the integer
+                    // out of the mantissa and let the saturating pack clamp from above (its range is
+                    // [-2^(BITS-1), 2^(BITS-1)-1], whose upper end is Qmax)
+#pragma unroll
+                    for (int i = 3; i >= 0; i--) {
+                        const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                        float v0, v1, t0, t1;
+                        unpack2(pmul(e, inv2[i]), v0, v1);
+                        unpack2(padd(pack2(fmaxf(v0, -qmax), fmaxf(v1, -qmax)), magic2), t0, t1);
+                        w = sat_pack2<BITS>((int)__float_as_uint(t1) - 0x4b400000, (int)__float_as_uint(t0) - 0x4b400000, w);
+                        unpack2(e, ev[2 * i], ev[2 * i + 1]);
+                    }
+                }
+                words[j] = w;
+                if (TOPK) {
+                    const float m0 = fmaxf(fmaxf(fabsf(ev[0]), fabsf(ev[1])), fmaxf(fabsf(ev[2]), fabsf(ev[3])));
+                    const float m1 = fmaxf(fmaxf(fabsf(ev[4]), fabsf(ev[5])), fmaxf(fabsf(ev[6]), fabsf(ev[7])));
+                    tmax = fmaxf(tmax, fmaxf(m0, m1));
+                }
+            }
+            rot_right4(words, rot);  // words[q] is now the code word of piece q
+            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + 4 * p.J) + tid * BITS;
+            if (BITS == 4) {
+                cw[0] = words[0]; cw[1] = words[1]; cw[2] = words[2]; cw[3] = words[3];
+            } else if (BITS == 3) {
+                cw[0] = words[0] | (words[1] << 24);
+                cw[1] = (words[1] >> 8) | (words[2] << 16);
+                cw[2] = (words[2] >> 16) | (words[3] << 8);
+            } else {
+                cw[0] = words[0] | (words[1] << 16);
+                cw[1] = words[2] | (words[3] << 16);
+            }
+            // (4) the largest |e| of this thread's 32 channels, for the outlier pass
+            if (TOPK) p.tmax[(first + (long long)it * stride) * (d >> 5) + tid] = tmax;
+        }
+        // this warp's share of the token is in shared memory: one arrival per warp
+        fence_async_smem();  // the record bytes written above will be read by the copy engine
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&ctrl->done[stage])) : "memory");
+
+        if (warp == duty) {
+            // ---- this warp's turn: hand the record over and refill the stage; the others have moved on
+            const int k_next = it + S;
+            int raw_next = 0;
+            if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);  // in flight while the tail runs
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
+            // ---- record complete: hand it to the copy engine, then refill the stage
+            if (lane == 0) {
+                const long long t = first + (long long)it * stride;
+                bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                bulk_commit();
+                if (k_next < n_my) {
+                    bulk_wait_read<0>();  // the record must have left before the next token may write it
+                    issue(k_next, stage, raw_next);
+                }
+            }
+            __syncwarp();
+        }
+        if (++stage == S) { stage = 0; parity ^= 1u; }
+        if (++duty == nwarps) duty = 0;
+    }
+    if (timed_out) {
+        ctrl->abort = 1;
+        if (p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
+    }
+    __syncthreads();
+    if (lane == 0) bulk_wait_all();  // every lane that stored records waits for its own copies
+    if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
+        // give copies that may still be in flight a bounded chance to land before the CTA retires
+        for (int s = 0; s < S; s++) {
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// encode, second launch: outlier split (the k largest |e| per token, ties to the lower channel)
+// ------------------------------------------------------------------------------------------------
+// One warp per token.  Input: the per-thread maxima the streaming pass left in the workspace (one value per
+// 32 channels).  (a) Threshold: the k-th largest of the 32 per-lane maxima (lane l covers slabs l, l+32,
+// ...): the k largest come from k different lanes, each with an element at least that large, so at least k
+// elements reach it.  (b) Only slabs whose maximum reaches the threshold can hold one of the k largest:
+// their residuals are recomputed from X, the reference row and the wire coefficients in the record (the
+// same binary32 operations as in the streaming pass, so the same bits); elements at or above the threshold
+// become candidates.  (c) Candidates are ranked exactly by counting (magnitude bits, then lower channel).
+// (d) The winners, in channel order, go into the record's outlier fields and their dense codes are cleared
+// (E^d = E - O).  More candidates than the list holds (many equal magnitudes) falls back to k rounds of a
+// maximum over the whole token.
+constexpr int kOutWarps = 8;       // warps (tokens in flight) per CTA
+constexpr int kOutCap = 128;       // candidate list per warp
+
+template <int BITS>
+__global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecParams p) {
+    __shared__ unsigned long long s_cand[kOutWarps][kOutCap];
+    __shared__ float s_cande[kOutWarps][kOutCap];
+    __shared__ unsigned long long s_sel[kOutWarps][16];
+    __shared__ float s_sele[kOutWarps][16];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int d = p.d, nth = d >> 5, k = p.topk;
+    constexpr uint32_t cmask = (1u << BITS) - 1u;
+    unsigned long long *cand = s_cand[warp];
+    float *cande = s_cande[warp];
+    unsigned long long *sel = s_sel[warp];
+    float *sele = s_sele[warp];
+    const long long wstride = (long long)gridDim.x * kOutWarps;
+
+    for (long long t = (long long)blockIdx.x * kOutWarps + warp; t < p.T; t += wstride) {
+        // reference row of the token, by the same rules as the streaming pass
+        long long row = p.ref_row ? (long long)p.ref_row[t] : t;
+        if (!p.ref_base || row < 0 || row >= p.ref_rows) row = -1;
+        const uint16_t *xrow = p.X + t * d;
+        const uint16_t *rrow = row >= 0 ? p.ref_base + row * d : nullptr;
+        unsigned char *rec = p.payload + t * p.rec;
+        const uint32_t *coef = reinterpret_cast<const uint32_t *>(rec);
+        // residual of channel c, exactly as the streaming pass computed it
+        auto residual = [&](int c) -> float {
+            const float h = __uint_as_float((uint32_t)xrow[c] << 16);
+            float r = 0.f;
+            if (rrow) {
+                r = __uint_as_float((uint32_t)rrow[c] << 16);
+                if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+            }
+            const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
+            return __fsub_rn(h, __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16)));
+        };
+
+        // (a) threshold
+        const float *tm = p.tmax + t * nth;
+        unsigned int v = 0u;
+        for (int th = lane; th < nth; th += 32) v = max(v, __float_as_uint(tm[th]));
+        unsigned int tau = 0u, vv = v;
+        for (int r = 0; r < k; r++) {
+            tau = __reduce_max_sync(0xffffffffu, vv);
+            if (r + 1 < k) {
+                const unsigned int bal = __ballot_sync(0xffffffffu, vv == tau);
+                if (lane == __ffs(bal) - 1) vv = 0u;
+            }
+        }
+        // (b) candidates from the slabs that reach the threshold
+        int n = 0;  // warp-uniform count
+        for (int base = 0; base < nth; base += 32) {
+            const int th = base + lane;
+            unsigned int hot = __ballot_sync(0xffffffffu, th < nth && __float_as_uint(tm[th]) >= tau);
+            while (hot) {
+                const int slab = base + __ffs(hot) - 1;
+                hot &= hot - 1;
+                const int c = slab * 32 + lane;
+                const float e = residual(c);
+                const unsigned int key = __float_as_uint(e) & 0x7fffffffu;
+                const unsigned int is = __ballot_sync(0xffffffffu, key >= tau);
+                if (key >= tau) {
+                    const int pos = n + __popc(is & ((1u << lane) - 1u));
+                    if (pos < kOutCap) {
+                        cand[pos] = ((unsigned long long)key << 16) | (unsigned long long)(0xffff - c);
+                        cande[pos] = e;
+                    }
+                }
+                n += __popc(is);
+            }
+        }
+        __syncwarp();
+        // (c) exact ranking
+        if (n <= kOutCap) {
+            for (int x = lane; x < n; x += 32) {
+                const unsigned long long mine = cand[x];
+                int rk = 0;
+                for (int y = 0; y < n; y++) rk += (cand[y] > mine) ? 1 : 0;
+                if (rk < k) { sel[rk] = mine; sele[rk] = cande[x]; }
+            }
+        } else {
+            unsigned long long prev = ~0ull;
+            for (int r = 0; r < k; r++) {
+                unsigned long long best = 0ull;
+                float beste = 0.f;
+                for (int c = lane; c < d; c += 32) {
+                    const float e = residual(c);
+                    const unsigned long long comp =
+                        ((unsigned long long)(__float_as_uint(e) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
+                    // a composite is 0 only for |e| == 0 at channel 65535, which d <= 8192 excludes
+                    if (comp < prev && comp > best) { best = comp; beste = e; }
+                }
+                for (int o = 16; o > 0; o >>= 1) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+                    const float othere = __shfl_xor_sync(0xffffffffu, beste, o);
+                    if (other > best) { best = other; beste = othere; }
+                }
+                if (lane == 0) { sel[r] = best; sele[r] = beste; }
+                prev = best;
+            }
+        }
+        __syncwarp();
+        // (d) outlier fields in channel order, dense codes at those channels cleared
+        if (lane < k) {
+            const int c = 0xffff - (int)(sel[lane] & 0xffffull);
+            if (c < d) {
+                int pos = 0;
+                for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
+                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                oidx[pos] = (unsigned short)c;
+                oidx[k + pos] = (unsigned short)float_to_half_bits_sat(sele[lane]);
+                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
+                const int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
+                atomicAnd(&codes32[wd], ~(cmask << sh));
+                if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
+            }
+        }
+        __syncwarp();
+    }
+}
+
 // step tables from the per-CTA partial sums (fixed summation order -> deterministic)
 __global__ void calib_finalize_kernel(const float *partial, int nblocks, int d, int bits, float clip_sigmas, float *step,
                                       float *inv_step) {
@@ -960,19 +1378,35 @@ static int pick_stages(int d, int dflt) {
     return dflt;
 }
 
-template <int MODE>
+// Encode: the streaming kernel, then (with outliers) the selection kernel.  Variant 4 of the streaming kernel
+// caps registers at 96 so that four 160-thread CTAs fit on an SM.
 static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
-    const bool topk = g.topk > 0 && MODE == 0;
-    p.stages = pick_stages(g.d, g.d <= 4096 ? 3 : 2);
-    EncSmem L = enc_smem_layout(g.d, g.rec, p.stages, g.nthreads, topk, MODE == 1);
-#define RAC_ENC(B, K) launch_persistent(encode_kernel<B, K, MODE>, p, g.nthreads, L.total, max_ctas, stream)
+    const bool topk = g.topk > 0;
+    p.stages = pick_stages(g.d, 2);
+    WsSmem L = ws_smem_layout(g.d, g.rec, p.stages);
+    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !getenv("RAC_ENC_WIDE");
+    int rc = RAC_EUNSUPPORTED;
+#define RAC_ENC(B, K)                                                                                              \
+    (tight ? launch_persistent(encode_ws_kernel<B, K, 4>, p, g.nthreads, L.total, max_ctas, stream)               \
+           : launch_persistent(encode_ws_kernel<B, K, 2>, p, g.nthreads, L.total, max_ctas, stream))
     switch (g.bits) {
-        case 4: return topk ? RAC_ENC(4, true) : RAC_ENC(4, false);
-        case 3: return topk ? RAC_ENC(3, true) : RAC_ENC(3, false);
-        case 2: return topk ? RAC_ENC(2, true) : RAC_ENC(2, false);
+        case 4: rc = topk ? RAC_ENC(4, true) : RAC_ENC(4, false); break;
+        case 3: rc = topk ? RAC_ENC(3, true) : RAC_ENC(3, false); break;
+        case 2: rc = topk ? RAC_ENC(2, true) : RAC_ENC(2, false); break;
     }
 #undef RAC_ENC
-    return RAC_EUNSUPPORTED;
+    if (rc != RAC_OK || !topk) return rc;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != RAC_OK) return rc;
+    long long blocks = (p.T + kOutWarps - 1) / kOutWarps;
+    if (blocks > (long long)di.sms * 8) blocks = (long long)di.sms * 8;
+    switch (g.bits) {
+        case 4: outlier_kernel<4><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); break;
+        case 3: outlier_kernel<3><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); break;
+        case 2: outlier_kernel<2><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); break;
+    }
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
 static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream) {
@@ -1048,9 +1482,17 @@ size_t rac_payload_bytes(const rac_codec_cfg *cfg, int64_t T) {
     return rac_record_bytes(cfg) * (size_t)T;
 }
 
+size_t rac_encode_workspace_bytes(const rac_codec_cfg *cfg, int64_t T) {
+    Geometry g;
+    if (make_geometry(cfg, &g) != RAC_OK || T < 0) return 0;
+    if (g.topk == 0) return 0;
+    return ((size_t)T * (size_t)(g.d / 32) * sizeof(float) + 15) / 16 * 16;
+}
+
 int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
                const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
-               const float *inv_step, void *payload, size_t payload_cap, uint32_t *dev_status, void *stream) {
+               const float *inv_step, void *payload, size_t payload_cap, void *workspace, size_t workspace_bytes,
+               uint32_t *dev_status, void *stream) {
     Geometry g;
     int rc = make_geometry(cfg, &g);
     if (rc != RAC_OK) return rc;
@@ -1061,11 +1503,18 @@ int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *r
     if (!X || !payload || !step || !inv_step) return RAC_EINVAL;
     if (!aligned16(X) || !aligned16(payload) || !aligned16(step) || !aligned16(inv_step)) return RAC_EALIGN;
     if (payload_cap < (size_t)g.rec * (size_t)T) return RAC_ESIZE;
+    const size_t need = rac_encode_workspace_bytes(cfg, T);
+    if (need > 0) {
+        if (!workspace) return RAC_EINVAL;
+        if (!aligned16(workspace)) return RAC_EALIGN;
+        if (workspace_bytes < need) return RAC_ESIZE;
+    }
     p.X = static_cast<const uint16_t *>(X);
     p.payload = static_cast<uint8_t *>(payload);
     p.step = step;
     p.inv_step = inv_step;
-    return launch_encode<0>(g, p, T, static_cast<cudaStream_t>(stream));
+    p.tmax = static_cast<float *>(workspace);
+    return launch_encode(g, p, T, static_cast<cudaStream_t>(stream));
 }
 
 int rac_decode_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_t T, const void *ref_base,

@@ -116,8 +116,13 @@ def gpu_encode(cfg, X, ref_base, ref_row, gain, bias, step, inv_step, pad=64):
     buf = torch.full((T * rec + 2 * pad,), 0xA5, dtype=torch.uint8, device=dev)
     payload = buf[pad:pad + T * rec]
     status = torch.zeros(1, dtype=torch.int32, device=dev)
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    wsbuf = torch.full((nws + 2 * pad,), 0x5A, dtype=torch.uint8, device=dev)  # dirty scratch, canaries around it
+    ws = wsbuf[pad:pad + nws] if nws else None
     rac.rac_encode(cfg, X, T, ref_base, 0 if ref_base is None else ref_base.shape[0], ref_row, gain, bias,
-                   step, inv_step, payload, T * rec, status)
+                   step, inv_step, payload, T * rec, ws, nws, status)
+    torch.cuda.synchronize()
+    assert torch.all(wsbuf[:pad] == 0x5A) and torch.all(wsbuf[pad + nws:] == 0x5A), "encode wrote outside its workspace"
     torch.cuda.synchronize()
     host = buf.cpu().numpy()
     assert np.all(host[:pad] == 0xA5) and np.all(host[pad + T * rec:] == 0xA5), "encode wrote outside the payload"

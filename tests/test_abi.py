@@ -25,7 +25,7 @@ def declared_symbols():
 
 def test_every_declared_symbol_is_exported(rac):
     names = declared_symbols()
-    assert len(names) >= 13
+    assert len(names) >= 14
     lib = rac.load()
     for n in names:
         assert hasattr(lib, n), f"{n} declared in rac.h but not exported by librac.so"
@@ -52,13 +52,14 @@ def test_host_side_rejections_happen_before_any_launch(rac):
     bad = rac.CodecCfg(4096, 96, 4, 8)
     A = 0x10000  # a 16-byte aligned fake address: never dereferenced because the call is rejected first
     args = dict(X=A, T=16, ref_base=A, ref_rows=16, ref_row=None, ref_gain=None, ref_bias=None, step=A, inv_step=A,
-                payload=A, payload_cap=16 * 2208, dev_status=None, stream=0)
+                payload=A, payload_cap=16 * 2208, workspace=A, workspace_bytes=16 * 128 * 4, dev_status=None,
+                stream=0)
 
     def enc(c=cfg, **kw):
         a = dict(args, **kw)
         return lib.rac_encode(C.byref(c), a["X"], a["T"], a["ref_base"], a["ref_rows"], a["ref_row"], a["ref_gain"],
-                              a["ref_bias"], a["step"], a["inv_step"], a["payload"], a["payload_cap"], a["dev_status"],
-                              a["stream"])
+                              a["ref_bias"], a["step"], a["inv_step"], a["payload"], a["payload_cap"], a["workspace"],
+                              a["workspace_bytes"], a["dev_status"], a["stream"])
     assert enc(c=bad) == -1                      # d % group
     assert enc(c=rac.CodecCfg(4100, 4100 // 4, 4, 0)) in (-1, -4)
     assert enc(T=-1) == -1
@@ -66,6 +67,9 @@ def test_host_side_rejections_happen_before_any_launch(rac):
     assert enc(X=A + 2) == -2                    # misaligned
     assert enc(payload=A + 8) == -2
     assert enc(payload_cap=16 * 2208 - 1) == -3
+    assert enc(workspace_bytes=16 * 128 * 4 - 1) == -3   # outliers need 4*d/32 bytes of scratch per token
+    assert enc(workspace=None) == -1
+    assert enc(workspace=A + 4) == -2
     assert enc(ref_rows=8) == -1                 # identity rows need ref_rows >= T
     assert enc(ref_gain=A) == -1                 # gain without bias
     assert enc(T=0, X=None, payload=None) == 0   # nothing to do

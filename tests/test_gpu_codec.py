@@ -221,7 +221,7 @@ def test_zero_tokens_is_a_no_op(env):
     t = torch.zeros(16, dtype=torch.uint8, device=env.dev)
     f = torch.zeros((2, 4096), dtype=torch.float32, device=env.dev)
     x = torch.zeros((0, 4096), dtype=torch.bfloat16, device=env.dev)
-    env.rac.rac_encode(cfg, x, 0, None, 0, None, None, None, f, f, t, 0, None)
+    env.rac.rac_encode(cfg, x, 0, None, 0, None, None, None, f, f, t, 0, None, 0, None)
     env.rac.rac_decode_reconstruct(cfg, t, 0, None, 0, None, None, None, f, x, None)
     torch.cuda.synchronize()
 
@@ -299,7 +299,9 @@ def test_long_context_sampled(env):
     rac.rac_calibrate_steps(cfg, X[:4096], 4096, Hs, H, ref_row[:4096].contiguous(), None, None, 3.0, step, inv, ws, nb, status)
     rec = rac.rac_record_bytes(cfg)
     payload = torch.empty(T * rec, dtype=torch.uint8, device=env.dev)
-    rac.rac_encode(cfg, X, T, Hs, H, ref_row, None, None, step, inv, payload, payload.numel(), status)
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    ews = torch.empty(nws, dtype=torch.uint8, device=env.dev)
+    rac.rac_encode(cfg, X, T, Hs, H, ref_row, None, None, step, inv, payload, payload.numel(), ews, nws, status)
     xh = torch.empty_like(X)
     rac.rac_decode_reconstruct(cfg, payload, T, Hs, H, ref_row, None, None, step, xh, status)
     torch.cuda.synchronize()
