@@ -956,11 +956,13 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 // maximum over the whole token.
 constexpr int kOutWarps = 8;       // warps (tokens in flight) per CTA
 constexpr int kOutCap = 128;       // candidate list per warp
+constexpr int kOutHot = 256;       // slab list per warp (d <= 8192 has at most 256 slabs)
 
 template <int BITS>
 __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecParams p) {
     __shared__ unsigned long long s_cand[kOutWarps][kOutCap];
     __shared__ float s_cande[kOutWarps][kOutCap];
+    __shared__ unsigned short s_hot[kOutWarps][kOutHot];
     __shared__ unsigned long long s_sel[kOutWarps][16];
     __shared__ float s_sele[kOutWarps][16];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -968,9 +970,11 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
     constexpr uint32_t cmask = (1u << BITS) - 1u;
     unsigned long long *cand = s_cand[warp];
     float *cande = s_cande[warp];
+    unsigned short *hot = s_hot[warp];
     unsigned long long *sel = s_sel[warp];
     float *sele = s_sele[warp];
     const long long wstride = (long long)gridDim.x * kOutWarps;
+    const unsigned int lt_mask = (1u << lane) - 1u;
 
     for (long long t = (long long)blockIdx.x * kOutWarps + warp; t < p.T; t += wstride) {
         // reference row of the token, by the same rules as the streaming pass
@@ -980,51 +984,93 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
         const uint16_t *rrow = row >= 0 ? p.ref_base + row * d : nullptr;
         unsigned char *rec = p.payload + t * p.rec;
         const uint32_t *coef = reinterpret_cast<const uint32_t *>(rec);
-        // residual of channel c, exactly as the streaming pass computed it
-        auto residual = [&](int c) -> float {
-            const float h = __uint_as_float((uint32_t)xrow[c] << 16);
+        // residual from the stored bits of x and r, exactly as the streaming pass computed it
+        auto residual_of = [&](uint32_t xb, uint32_t rb, int c, uint32_t cf) -> float {
+            const float h = __uint_as_float(xb << 16);
             float r = 0.f;
             if (rrow) {
-                r = __uint_as_float((uint32_t)rrow[c] << 16);
+                r = __uint_as_float(rb << 16);
                 if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
             }
-            const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
             return __fsub_rn(h, __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16)));
         };
+        auto residual = [&](int c) -> float {
+            return residual_of(xrow[c], rrow ? rrow[c] : 0u, c, coef[c >> (5 + p.lpg_shift)]);
+        };
 
-        // (a) threshold
+        // (a) threshold; the slabs that reach it, in slab order
         const float *tm = p.tmax + t * nth;
+        unsigned int tv[8];
         unsigned int v = 0u;
-        for (int th = lane; th < nth; th += 32) v = max(v, __float_as_uint(tm[th]));
-        unsigned int tau = 0u, vv = v;
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            const int th = lane + 32 * i;
+            tv[i] = th < nth ? __float_as_uint(tm[th]) : 0u;
+            v = max(v, tv[i]);
+        }
+        unsigned int tau = 0u;
         for (int r = 0; r < k; r++) {
-            tau = __reduce_max_sync(0xffffffffu, vv);
+            tau = __reduce_max_sync(0xffffffffu, v);
             if (r + 1 < k) {
-                const unsigned int bal = __ballot_sync(0xffffffffu, vv == tau);
-                if (lane == __ffs(bal) - 1) vv = 0u;
+                const unsigned int bal = __ballot_sync(0xffffffffu, v == tau);
+                if (lane == __ffs(bal) - 1) v = 0u;
             }
         }
-        // (b) candidates from the slabs that reach the threshold
+        int nh = 0;
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            const bool is_hot = (lane + 32 * i) < nth && tv[i] >= tau;
+            const unsigned int bal = __ballot_sync(0xffffffffu, is_hot);
+            if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(lane + 32 * i);
+            nh += __popc(bal);
+        }
+        __syncwarp();
+        // (b) candidates: eight slabs per round, a lane takes 8 consecutive channels of one slab, so that the
+        // loads of a round are all in flight together
         int n = 0;  // warp-uniform count
-        for (int base = 0; base < nth; base += 32) {
-            const int th = base + lane;
-            unsigned int hot = __ballot_sync(0xffffffffu, th < nth && __float_as_uint(tm[th]) >= tau);
-            while (hot) {
-                const int slab = base + __ffs(hot) - 1;
-                hot &= hot - 1;
-                const int c = slab * 32 + lane;
-                const float e = residual(c);
-                const unsigned int key = __float_as_uint(e) & 0x7fffffffu;
-                const unsigned int is = __ballot_sync(0xffffffffu, key >= tau);
-                if (key >= tau) {
-                    const int pos = n + __popc(is & ((1u << lane) - 1u));
-                    if (pos < kOutCap) {
-                        cand[pos] = ((unsigned long long)key << 16) | (unsigned long long)(0xffff - c);
-                        cande[pos] = e;
+        for (int base = 0; base < nh; base += 8) {
+            const int hi = base + (lane >> 2);
+            const bool act = hi < nh;
+            const int c0 = act ? (int)hot[hi] * 32 + (lane & 3) * 8 : 0;
+            uint4 xw = make_uint4(0u, 0u, 0u, 0u), rw = xw;
+            uint32_t cf = 0u;
+            if (act) {
+                xw = __ldg(reinterpret_cast<const uint4 *>(xrow + c0));
+                if (rrow) rw = __ldg(reinterpret_cast<const uint4 *>(rrow + c0));
+                cf = coef[c0 >> (5 + p.lpg_shift)];
+            }
+            const uint32_t xs[4] = {xw.x, xw.y, xw.z, xw.w}, rs[4] = {rw.x, rw.y, rw.z, rw.w};
+            float e[8];
+            int cnt = 0;
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const uint32_t xb = (i & 1) ? (xs[i >> 1] >> 16) : (xs[i >> 1] & 0xffffu);
+                const uint32_t rb = (i & 1) ? (rs[i >> 1] >> 16) : (rs[i >> 1] & 0xffffu);
+                e[i] = residual_of(xb, rb, c0 + i, cf);
+                cnt += (act && (__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? 1 : 0;
+            }
+            // exclusive prefix of the per-lane counts
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            int pos = n + incl - cnt;
+            if (act) {
+#pragma unroll
+                for (int i = 0; i < 8; i++) {
+                    const unsigned int key = __float_as_uint(e[i]) & 0x7fffffffu;
+                    if (key >= tau) {
+                        if (pos < kOutCap) {
+                            cand[pos] = ((unsigned long long)key << 16) | (unsigned long long)(0xffff - (c0 + i));
+                            cande[pos] = e[i];
+                        }
+                        pos++;
                     }
                 }
-                n += __popc(is);
             }
+            n += __shfl_sync(0xffffffffu, incl, 31);
         }
         __syncwarp();
         // (c) exact ranking
