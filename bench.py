@@ -412,7 +412,8 @@ def main():
         enc_ms = stage_ms[1] + stage_ms[4]
         dec_ms = stage_ms[2] + stage_ms[3] + stage_ms[5]
         if enc_ms >= dec_ms:
-            dom, dom_bytes, dom_ms, dom_n = "encode_kernel<4,topk>", rt.bytes_of("encode_up") + rt.bytes_of("encode_dn"), enc_ms, 2
+            dom, dom_bytes, dom_ms, dom_n = ("rac_encode (encode_ws_kernel<4,true> + outlier_kernel<4>)",
+                                             rt.bytes_of("encode_up") + rt.bytes_of("encode_dn"), enc_ms, 2)
         else:
             dom, dom_bytes, dom_ms, dom_n = ("decode_kernel<4,8>", rt.bytes_of("sender_up") + rt.bytes_of("decode_up")
                                              + rt.bytes_of("decode_dn"), dec_ms, 3)

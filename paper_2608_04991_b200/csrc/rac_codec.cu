@@ -1000,13 +1000,17 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
 
         // (a) threshold; the slabs that reach it, in slab order
         const float *tm = p.tmax + t * nth;
+        const int ni = (nth + 31) >> 5;  // values per lane, at most 8
         unsigned int tv[8];
         unsigned int v = 0u;
 #pragma unroll
         for (int i = 0; i < 8; i++) {
-            const int th = lane + 32 * i;
-            tv[i] = th < nth ? __float_as_uint(tm[th]) : 0u;
-            v = max(v, tv[i]);
+            tv[i] = 0u;
+            if (i < ni) {
+                const int th = lane + 32 * i;
+                if (th < nth) tv[i] = __float_as_uint(tm[th]);
+                v = max(v, tv[i]);
+            }
         }
         unsigned int tau = 0u;
         for (int r = 0; r < k; r++) {
@@ -1019,10 +1023,13 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
         int nh = 0;
 #pragma unroll
         for (int i = 0; i < 8; i++) {
-            const bool is_hot = (lane + 32 * i) < nth && tv[i] >= tau;
-            const unsigned int bal = __ballot_sync(0xffffffffu, is_hot);
-            if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(lane + 32 * i);
-            nh += __popc(bal);
+            if (i < ni) {
+                // a slab beyond the width has tv == 0 and can only pass when tau == 0; keep it out
+                const bool is_hot = tv[i] >= tau && (lane + 32 * i) < nth;
+                const unsigned int bal = __ballot_sync(0xffffffffu, is_hot);
+                if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(lane + 32 * i);
+                nh += __popc(bal);
+            }
         }
         __syncwarp();
         // (b) candidates: eight slabs per round, a lane takes 8 consecutive channels of one slab, so that the
@@ -1040,15 +1047,30 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
                 cf = coef[c0 >> (5 + p.lpg_shift)];
             }
             const uint32_t xs[4] = {xw.x, xw.y, xw.z, xw.w}, rs[4] = {rw.x, rw.y, rw.z, rw.w};
+            const float ca = half_bits_to_float(cf & 0xffff), cb = half_bits_to_float(cf >> 16);
             float e[8];
+            if (rrow && p.gain) {
+#pragma unroll
+                for (int i = 0; i < 8; i++) {
+                    const uint32_t xb = (i & 1) ? (xs[i >> 1] & 0xffff0000u) : (xs[i >> 1] << 16);
+                    const uint32_t rb = (i & 1) ? (rs[i >> 1] & 0xffff0000u) : (rs[i >> 1] << 16);
+                    const float r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c0 + i]), __uint_as_float(rb),
+                                                         half_bits_to_float(p.bias[c0 + i])));
+                    e[i] = __fsub_rn(__uint_as_float(xb), __fmaf_rn(ca, r, cb));
+                }
+            } else {
+                // without a reference rw is zero, which is the zero reference of a directly coded token
+#pragma unroll
+                for (int i = 0; i < 8; i++) {
+                    const uint32_t xb = (i & 1) ? (xs[i >> 1] & 0xffff0000u) : (xs[i >> 1] << 16);
+                    const uint32_t rb = (i & 1) ? (rs[i >> 1] & 0xffff0000u) : (rs[i >> 1] << 16);
+                    e[i] = __fsub_rn(__uint_as_float(xb), __fmaf_rn(ca, __uint_as_float(rb), cb));
+                }
+            }
             int cnt = 0;
 #pragma unroll
-            for (int i = 0; i < 8; i++) {
-                const uint32_t xb = (i & 1) ? (xs[i >> 1] >> 16) : (xs[i >> 1] & 0xffffu);
-                const uint32_t rb = (i & 1) ? (rs[i >> 1] >> 16) : (rs[i >> 1] & 0xffffu);
-                e[i] = residual_of(xb, rb, c0 + i, cf);
-                cnt += (act && (__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? 1 : 0;
-            }
+            for (int i = 0; i < 8; i++) cnt += ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? 1 : 0;
+            if (!act) cnt = 0;
             // exclusive prefix of the per-lane counts
             int incl = cnt;
 #pragma unroll
