@@ -112,10 +112,16 @@ __global__ void match_query_kernel(MatchParams p) {
 }
 
 // Single CTA.  (1) hop[p] = (s, s + len(s)) with s the first position >= p that has a candidate (n_query
-// if none); (2) one thread follows the chain from 0 and lists the spans; (3) all threads expand them.
-__global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p) {
+// if none); (2) one thread follows the chain from 0 and lists the positions it visits; (3) all threads turn
+// them into spans and rows.  The chain is the serial part of Eq. 3 (one dependent read per selected span);
+// to make each read a shared-memory access instead of a trip to L2, the jump lengths of a window of
+// positions are staged as 16-bit deltas (65535 = "look it up in global memory") before the walk enters it.
+constexpr int kWalkWindow = 96 * 1024;  // positions per window: 192 KiB of shared memory
+
+__global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p, int window) {
+    extern __shared__ unsigned short s_delta[];
     __shared__ int warp_first[32];
-    __shared__ int s_nspans;
+    __shared__ int s_nspans, s_pos;
     const int N = p.n_query;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     // contiguous range of whole 32-position tiles per warp
@@ -132,55 +138,83 @@ __global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p) {
         if (b) { first = tl * 32 + __ffs(b) - 1; break; }
     }
     if (lane == 0) warp_first[warp] = first;
+    if (tid == 0) { s_pos = 0; s_nspans = 0; }
     __syncthreads();
     // first candidate position after this warp's range
     int carry = N;
     for (int w = nwarps - 1; w > warp; w--) carry = min(carry, warp_first[w]);
     int carry_next = carry < N ? carry + p.best[carry].x : N;
 
-    // pass B: tiles backwards, carrying the next candidate position
-    for (int tl = t_hi - 1; tl >= t_lo; tl--) {
-        int i = tl * 32 + lane;
-        int len = i < N ? p.best[i].x : 0;
-        unsigned int b = __ballot_sync(0xffffffffu, len > 0);
-        unsigned int at_or_after = b >> lane;
-        int s = carry, nx = carry_next;
-        const int src = at_or_after ? lane + __ffs(at_or_after) - 1 : lane;
-        const int len_src = __shfl_sync(0xffffffffu, len, src);  // one convergent shuffle for all lanes
-        if (at_or_after) {
-            s = tl * 32 + src;
-            nx = s + len_src;
+    // pass B: tiles backwards, carrying the next candidate position; four tiles' loads in flight at a time
+    for (int tg = t_hi - 1; tg >= t_lo; tg -= 4) {
+        int lens[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const int i = (tg - u) * 32 + lane;
+            lens[u] = (tg - u >= t_lo && i < N) ? p.best[i].x : 0;
         }
-        if (i < N) p.hop[i] = make_int2(s, nx);
-        if (b) {
-            int f = __ffs(b) - 1;
-            carry = tl * 32 + f;
-            carry_next = carry + __shfl_sync(0xffffffffu, len, f);
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const int tl = tg - u;
+            if (tl < t_lo) break;
+            const int i = tl * 32 + lane;
+            const int len = lens[u];
+            unsigned int b = __ballot_sync(0xffffffffu, len > 0);
+            unsigned int at_or_after = b >> lane;
+            int s = carry, nx = carry_next;
+            const int src = at_or_after ? lane + __ffs(at_or_after) - 1 : lane;
+            const int len_src = __shfl_sync(0xffffffffu, len, src);  // one convergent shuffle for all lanes
+            if (at_or_after) {
+                s = tl * 32 + src;
+                nx = s + len_src;
+            }
+            if (i < N) p.hop[i] = make_int2(s, nx);
+            if (b) {
+                int f = __ffs(b) - 1;
+                carry = tl * 32 + f;
+                carry_next = carry + __shfl_sync(0xffffffffu, len, f);
+            }
         }
     }
     __syncthreads();
 
-    // (2) the serial part of Eq. 3: one dependent load per selected span
-    if (tid == 0) {
-        int n = 0, pos = 0;
-        while (pos < N) {
-            int2 h = p.hop[pos];
-            if (h.x >= N) break;
-            p.spans_ws[n].q_start = h.x;
-            p.spans_ws[n].len = h.y - h.x;
-            n++;
-            pos = h.y;
+    // (2) the chain, window by window; spans_ws[n].q_start keeps the n-th visited position
+    while (true) {
+        const int wbeg = s_pos;
+        if (wbeg >= N) break;
+        const int wend = min(N, wbeg + window);
+        for (int i = wbeg + tid; i < wend; i += blockDim.x) {
+            const int dlt = p.hop[i].y - i;
+            s_delta[i - wbeg] = (unsigned short)(dlt < 65535 ? dlt : 65535);
         }
+        __syncthreads();
+        if (tid == 0) {
+            int n = s_nspans, pos = wbeg;
+            while (pos < wend) {
+                p.spans_ws[n++].q_start = pos;
+                const int dlt = s_delta[pos - wbeg];
+                pos = dlt == 65535 ? p.hop[pos].y : pos + dlt;
+            }
+            s_nspans = n;
+            s_pos = pos;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        // the last visited position may have no candidate at or after it: then it starts no span
+        int n = s_nspans;
+        if (n > 0 && p.hop[p.spans_ws[n - 1].q_start].x >= N) n--;
         s_nspans = n;
         *p.n_spans = n;
     }
     __syncthreads();
 
-    // (3) history starts and per-token rows
+    // (3) spans and per-token rows
     const int ns = s_nspans;
     for (int sidx = warp; sidx < ns; sidx += nwarps) {
-        int q0 = p.spans_ws[sidx].q_start, len = p.spans_ws[sidx].len;
-        int h0 = p.best[q0].y;
+        const int2 h = p.hop[p.spans_ws[sidx].q_start];
+        const int q0 = h.x, len = h.y - h.x;
+        const int h0 = p.best[q0].y;
         if (lane == 0 && p.spans_out) {
             p.spans_out[sidx].q_start = q0;
             p.spans_out[sidx].h_start = h0;
@@ -315,7 +349,13 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     }
     if (n_query > 0) {
         match_query_kernel<<<(int)((n_query + tb - 1) / tb), tb, 0, st>>>(p);
-        match_select_kernel<<<1, 1024, 0, st>>>(p);
+        // shared-memory window of the chain walk (16-bit deltas)
+        int window = n_query < kWalkWindow ? (int)n_query : kWalkWindow;
+        size_t dyn = ((size_t)window * 2 + 15) / 16 * 16;
+        if (dyn > 48 * 1024 &&
+            cudaFuncSetAttribute(match_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+            return RAC_ECUDA;
+        match_select_kernel<<<1, 1024, dyn, st>>>(p, window);
     }
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
