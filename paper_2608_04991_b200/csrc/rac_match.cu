@@ -209,18 +209,21 @@ __global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p, int w
     }
     __syncthreads();
 
-    // (3) spans and per-token rows
+    // (3) spans (one thread each: the three dependent lookups of different spans overlap), then per-token rows
     const int ns = s_nspans;
-    for (int sidx = warp; sidx < ns; sidx += nwarps) {
+    for (int sidx = tid; sidx < ns; sidx += blockDim.x) {
         const int2 h = p.hop[p.spans_ws[sidx].q_start];
-        const int q0 = h.x, len = h.y - h.x;
-        const int h0 = p.best[q0].y;
-        if (lane == 0 && p.spans_out) {
-            p.spans_out[sidx].q_start = q0;
-            p.spans_out[sidx].h_start = h0;
-            p.spans_out[sidx].len = len;
-        }
-        for (int m = lane; m < len; m += 32) p.ref_row[q0 + m] = h0 + m;
+        rac_span sp;
+        sp.q_start = h.x;
+        sp.len = h.y - h.x;
+        sp.h_start = p.best[h.x].y;
+        p.spans_ws[sidx] = sp;
+        if (p.spans_out) p.spans_out[sidx] = sp;
+    }
+    __syncthreads();
+    for (int sidx = warp; sidx < ns; sidx += nwarps) {
+        const rac_span sp = p.spans_ws[sidx];
+        for (int m = lane; m < sp.len; m += 32) p.ref_row[sp.q_start + m] = sp.h_start + m;
     }
 }
 
