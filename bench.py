@@ -4,7 +4,7 @@
 One "step" is one pass of the whole hot path over the long-context round trip
 (T = 131072 tokens, d = 5120, group 128, 4-bit, top-8 outliers, 131072-token history):
 
-    span match -> uplink encode -> sender reconstruct -> receiver reconstruct
+    span match -> uplink encode + sender-side reconstruction (one call) -> receiver reconstruct
                -> downlink encode (reference = reconstructed uplink) -> receiver reconstruct
 
 `value` is GB/s of bf16 activations through the codec (both directions, 2 * 2*T*d bytes per step)
@@ -118,7 +118,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------- workload
 class RoundTrip:
     """Device buffers and the ordered C-ABI calls of one step."""
-    LAUNCHES_PER_STEP = (4 + WORKLOAD["max_hits"]) + 2 * 2 + 3  # matcher kernels + 2 encodes (2 launches each) + 3 reconstructions
+    LAUNCHES_PER_STEP = (4 + WORKLOAD["max_hits"]) + 2 * 2 + 2  # matcher kernels + 2 encodes (2 launches each) + 2 reconstructions
 
     def __init__(self, wl, seed, dev):
         import numpy as np
@@ -178,10 +178,12 @@ class RoundTrip:
         self.rac.rac_encode(self.cfg, self.X, w["T"], self.Hs, w["n_hist"], self.ref_row, None, None, self.step_up,
                             self.inv_up, self.pay_up, self.pay_up.numel(), self.ews, self.ews_bytes, self.status)
 
-    def sender_up(self):
+    def encode_sender_up(self):
+        """Uplink encode that also leaves the sender-side x_hat (the next reference) in Xs."""
         w = self.wl
-        self.rac.rac_sender_reconstruct(self.cfg, self.pay_up, w["T"], self.Hs, w["n_hist"], self.ref_row, None, None,
-                                        self.step_up, self.Xs, self.status)
+        self.rac.rac_encode_reconstruct(self.cfg, self.X, w["T"], self.Hs, w["n_hist"], self.ref_row, None, None,
+                                        self.step_up, self.inv_up, self.pay_up, self.pay_up.numel(), self.Xs, self.ews,
+                                        self.ews_bytes, self.status)
 
     def decode_up(self):
         w = self.wl
@@ -198,7 +200,7 @@ class RoundTrip:
         self.rac.rac_decode_reconstruct(self.cfg, self.pay_dn, w["T"], self.Xh, w["T"], None, None, None, self.step_dn,
                                         self.Yh, self.status)
 
-    STAGES = ["match", "encode_up", "sender_up", "decode_up", "encode_dn", "decode_dn"]
+    STAGES = ["match", "encode_sender_up", "decode_up", "encode_dn", "decode_dn"]
 
     def step(self, events=None):
         for i, name in enumerate(self.STAGES):
@@ -215,9 +217,11 @@ class RoundTrip:
         refd = self.coverage
         if name == "encode_up":
             return T * (2 * d + 2 * d * refd + rec + 4)
+        if name == "encode_sender_up":
+            return T * (2 * d + 2 * d * refd + rec + 4 + 2 * d)
         if name == "encode_dn":
             return T * (2 * d + 2 * d + rec)
-        if name in ("sender_up", "decode_up"):
+        if name == "decode_up":
             return T * (rec + 2 * d * refd + 2 * d + 4)
         if name == "decode_dn":
             return T * (rec + 2 * d + 2 * d)
@@ -409,14 +413,15 @@ def main():
         per = {n: {"ms": stage_ms[i], "GB/s_algorithmic": (rt.bytes_of(n) / (stage_ms[i] * 1e-3) / 1e9) if rt.bytes_of(n) else None,
                    "GB/s_activations_in": 2 * wl["T"] * wl["d"] / (stage_ms[i] * 1e-3) / 1e9 if n != "match" else None}
                for i, n in enumerate(names)}
-        enc_ms = stage_ms[1] + stage_ms[4]
-        dec_ms = stage_ms[2] + stage_ms[3] + stage_ms[5]
+        ix = {n: i for i, n in enumerate(names)}
+        enc_ms = stage_ms[ix["encode_sender_up"]] + stage_ms[ix["encode_dn"]]
+        dec_ms = stage_ms[ix["decode_up"]] + stage_ms[ix["decode_dn"]]
         if enc_ms >= dec_ms:
-            dom, dom_bytes, dom_ms, dom_n = ("rac_encode (encode_ws_kernel<4,true> + outlier_kernel<4>)",
-                                             rt.bytes_of("encode_up") + rt.bytes_of("encode_dn"), enc_ms, 2)
+            dom, dom_bytes, dom_ms, dom_n = ("rac_encode[_reconstruct] (encode_ws_kernel<4,true,*> + outlier_kernel<4>)",
+                                             rt.bytes_of("encode_sender_up") + rt.bytes_of("encode_dn"), enc_ms, 2)
         else:
-            dom, dom_bytes, dom_ms, dom_n = ("decode_kernel<4,8>", rt.bytes_of("sender_up") + rt.bytes_of("decode_up")
-                                             + rt.bytes_of("decode_dn"), dec_ms, 3)
+            dom, dom_bytes, dom_ms, dom_n = ("decode_kernel<4,8>", rt.bytes_of("decode_up") + rt.bytes_of("decode_dn"),
+                                             dec_ms, 2)
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None, "peak_source": peak_src, "launches_per_step": dom_n,

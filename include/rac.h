@@ -168,6 +168,20 @@ int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T,
                void *payload, size_t payload_cap, void *workspace, size_t workspace_bytes,
                uint32_t *dev_status, void *stream);
 
+/* Encode and sender-side reconstruction in one pass (Sec. IV-C: "the sender applies the same wire-format
+ * reconstruction as the receiver"; here it reuses the residuals and codes the encoder already holds instead of
+ * decoding its own payload again).  Arguments as rac_encode plus
+ *   X_hat  bf16[T,d] out: bit-identical to what rac_decode_reconstruct / rac_sender_reconstruct produce from
+ *          `payload` with the same reference and step table.  Must not overlap X, the reference rows in use, or
+ *          payload.
+ * Both tables are read here (inv_step for the codes, step for x_hat). */
+int rac_encode_reconstruct(const rac_codec_cfg *cfg, const void *X, int64_t T,
+                           const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                           const void *ref_gain, const void *ref_bias,
+                           const float *step, const float *inv_step,
+                           void *payload, size_t payload_cap, void *X_hat, void *workspace, size_t workspace_bytes,
+                           uint32_t *dev_status, void *stream);
+
 /* Receiver reconstruction (Eq. 9): X_hat = bf16( (alpha*r + beta) + e_hat ), e_hat = code*step or the
  * stored binary16 outlier.  Arguments as rac_encode.  X_hat bf16[T,d] must not overlap payload.  X_hat
  * may be the very buffer that ref_base points to ONLY with ref_row == NULL (token t reads row t and

@@ -30,7 +30,8 @@ EXPORTS = [
     "rac_version", "rac_strerror", "rac_record_bytes", "rac_payload_bytes",
     "rac_match_workspace_bytes", "rac_match_spans", "rac_spans_to_rows",
     "rac_match_spans_static",
-    "rac_encode_workspace_bytes", "rac_encode", "rac_decode_reconstruct", "rac_sender_reconstruct",
+    "rac_encode_workspace_bytes", "rac_encode", "rac_encode_reconstruct", "rac_decode_reconstruct",
+    "rac_sender_reconstruct",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
 ]
 
@@ -86,6 +87,8 @@ def load() -> C.CDLL:
     l.rac_encode_workspace_bytes.restype = sz
     l.rac_encode_workspace_bytes.argtypes = [cfgp, i64]
     l.rac_encode.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp]
+    l.rac_encode_reconstruct.restype = C.c_int
+    l.rac_encode_reconstruct.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp, vp, sz, vp, vp]
     for name in ("rac_decode_reconstruct", "rac_sender_reconstruct"):
         f = getattr(l, name)
         f.restype = C.c_int
@@ -200,6 +203,18 @@ def rac_encode(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step,
                            int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"),
                            _stream() if stream is None else stream)
     _check("rac_encode", rc)
+
+
+def rac_encode_reconstruct(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload,
+                           payload_cap, X_hat, workspace, workspace_bytes, dev_status, stream=None) -> None:
+    rc = load().rac_encode_reconstruct(C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(ref_base, _BF16, "ref_base"),
+                                       int(ref_rows), _ptr(ref_row, _I32, "ref_row"), _ptr(ref_gain, _F16, "ref_gain"),
+                                       _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"),
+                                       _ptr(inv_step, _F32, "inv_step"), _ptr(payload, _U8, "payload"), int(payload_cap),
+                                       _ptr(X_hat, _BF16, "X_hat"), _ptr(workspace, None, "workspace"),
+                                       int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"),
+                                       _stream() if stream is None else stream)
+    _check("rac_encode_reconstruct", rc)
 
 
 def _reconstruct(fn, cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, X_hat, dev_status, stream):

@@ -689,7 +689,7 @@ __host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages) {
     return s;
 }
 
-template <int BITS, bool TOPK, int MINB>
+template <int BITS, bool TOPK, bool XHAT, int MINB>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -839,6 +839,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
             if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = a16 | (b16 << 16);
             const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
+            const float *step_tab = p.step + (has_ref ? 0 : d);
             uint32_t words[4];
             float tmax = 0.f;
 #pragma unroll
@@ -847,21 +848,36 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                 const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
                 const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
                 const u64 inv2[4] = {pack2(iv0.x, iv0.y), pack2(iv0.z, iv0.w), pack2(iv1.x, iv1.y), pack2(iv1.z, iv1.w)};
+                u64 st2[4] = {0ull, 0ull, 0ull, 0ull};
+                if (XHAT) {
+                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(step_tab + c));
+                    const float4 s1 = __ldg(reinterpret_cast<const float4 *>(step_tab + c + 4));
+                    st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
+                }
                 float ev[8];
+                uint32_t xh[4];
                 uint32_t w = 0;
                 if (BITS == 3) {
                     uint32_t bits8[8];
 #pragma unroll
                     for (int i = 0; i < 4; i++) {
-                        const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                        const u64 rt = pfma(a2, r2[4 * j + i], b2);
+                        const u64 e = psub(x2[4 * j + i], rt);
                         float v0, v1, t0, t1;
                         unpack2(pmul(e, inv2[i]), v0, v1);
                         t0 = fminf(fmaxf(v0, -qmax), qmax);
                         t1 = fminf(fmaxf(v1, -qmax), qmax);
-                        unpack2(padd(pack2(t0, t1), magic2), t0, t1);
+                        const u64 tt = padd(pack2(t0, t1), magic2);
+                        unpack2(tt, t0, t1);
                         bits8[2 * i] = __float_as_uint(t0);
                         bits8[2 * i + 1] = __float_as_uint(t1);
                         unpack2(e, ev[2 * i], ev[2 * i + 1]);
+                        if (XHAT) {
+                            // Eq. 9 with the code just chosen: x_hat = bf16((alpha*r + beta) + q*step)
+                            float x0, x1;
+                            unpack2(padd(rt, pmul(psub(tt, magic2), st2[i])), x0, x1);
+                            xh[i] = f2_to_bf16x2(x0, x1);
+                        }
                     }
                     w = pack8<BITS>(bits8);
                 } else {
@@ -870,15 +886,27 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                     // [-2^(BITS-1), 2^(BITS-1)-1], whose upper end is Qmax)
 #pragma unroll
                     for (int i = 3; i >= 0; i--) {
-                        const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                        const u64 rt = pfma(a2, r2[4 * j + i], b2);
+                        const u64 e = psub(x2[4 * j + i], rt);
                         float v0, v1, t0, t1;
                         unpack2(pmul(e, inv2[i]), v0, v1);
-                        unpack2(padd(pack2(fmaxf(v0, -qmax), fmaxf(v1, -qmax)), magic2), t0, t1);
+                        v0 = fmaxf(v0, -qmax);
+                        v1 = fmaxf(v1, -qmax);
+                        if (XHAT) { v0 = fminf(v0, qmax); v1 = fminf(v1, qmax); }  // the float is used again below
+                        const u64 tt = padd(pack2(v0, v1), magic2);
+                        unpack2(tt, t0, t1);
                         w = sat_pack2<BITS>((int)__float_as_uint(t1) - 0x4b400000, (int)__float_as_uint(t0) - 0x4b400000, w);
                         unpack2(e, ev[2 * i], ev[2 * i + 1]);
+                        if (XHAT) {
+                            float x0, x1;
+                            unpack2(padd(rt, pmul(psub(tt, magic2), st2[i])), x0, x1);
+                            xh[i] = f2_to_bf16x2(x0, x1);
+                        }
                     }
                 }
                 words[j] = w;
+                // sender-side reconstruction: the thread's own slab of the X row now carries x_hat
+                if (XHAT) sts128(xs + off[j], make_uint4(xh[0], xh[1], xh[2], xh[3]));
                 if (TOPK) {
                     const float m0 = fmaxf(fmaxf(fabsf(ev[0]), fabsf(ev[1])), fmaxf(fabsf(ev[2]), fabsf(ev[3])));
                     const float m1 = fmaxf(fmaxf(fabsf(ev[4]), fabsf(ev[5])), fmaxf(fabsf(ev[6]), fabsf(ev[7])));
@@ -901,7 +929,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             if (TOPK) p.tmax[(first + (long long)it * stride) * (d >> 5) + tid] = tmax;
         }
         // this warp's share of the token is in shared memory: one arrival per warp
-        fence_async_smem();  // the record bytes written above will be read by the copy engine
+        fence_async_smem();  // the record (and x_hat) bytes written above will be read by the copy engine
         __syncwarp();
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&ctrl->done[stage])) : "memory");
 
@@ -915,6 +943,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             if (lane == 0) {
                 const long long t = first + (long long)it * stride;
                 bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                if (XHAT) bulk_store(p.X_hat + t * d, xs, row_bytes);
                 bulk_commit();
                 if (k_next < n_my) {
                     bulk_wait_read<0>();  // the record must have left before the next token may write it
@@ -1132,8 +1161,20 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
                 int pos = 0;
                 for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
                 unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                const uint32_t hv = float_to_half_bits_sat(sele[lane]);
                 oidx[pos] = (unsigned short)c;
-                oidx[k + pos] = (unsigned short)float_to_half_bits_sat(sele[lane]);
+                oidx[k + pos] = (unsigned short)hv;
+                if (p.X_hat) {
+                    // the sender-side reconstruction of an outlier channel: (alpha*r + beta) + the binary16 value
+                    float r = 0.f;
+                    if (rrow) {
+                        r = __uint_as_float((uint32_t)rrow[c] << 16);
+                        if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                    }
+                    const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
+                    const float rt = __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16));
+                    p.X_hat[t * d + c] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(rt, half_bits_to_float(hv))));
+                }
                 uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
                 const int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
                 atomicAnd(&codes32[wd], ~(cmask << sh));
@@ -1452,16 +1493,20 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     const bool topk = g.topk > 0;
     p.stages = pick_stages(g.d, 2);
     WsSmem L = ws_smem_layout(g.d, g.rec, p.stages);
-    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !getenv("RAC_ENC_WIDE");
+    // With x_hat the kernel reads both step tables every token; at four CTAs per SM the shared-memory carve-out
+    // leaves too little L1 for them, so that variant runs three CTAs per SM at 128 registers.
+    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
     int rc = RAC_EUNSUPPORTED;
-#define RAC_ENC(B, K)                                                                                              \
-    (tight ? launch_persistent(encode_ws_kernel<B, K, 4>, p, g.nthreads, L.total, max_ctas, stream)               \
-           : launch_persistent(encode_ws_kernel<B, K, 2>, p, g.nthreads, L.total, max_ctas, stream))
+#define RAC_ENC2(B, K, X)                                                                                          \
+    (tight ? launch_persistent(encode_ws_kernel<B, K, X, 4>, p, g.nthreads, L.total, max_ctas, stream)            \
+           : launch_persistent(encode_ws_kernel<B, K, X, 2>, p, g.nthreads, L.total, max_ctas, stream))
+#define RAC_ENC(B, K) (p.X_hat ? RAC_ENC2(B, K, true) : RAC_ENC2(B, K, false))
     switch (g.bits) {
         case 4: rc = topk ? RAC_ENC(4, true) : RAC_ENC(4, false); break;
         case 3: rc = topk ? RAC_ENC(3, true) : RAC_ENC(3, false); break;
         case 2: rc = topk ? RAC_ENC(2, true) : RAC_ENC(2, false); break;
     }
+#undef RAC_ENC2
 #undef RAC_ENC
     if (rc != RAC_OK || !topk) return rc;
     DeviceInfo di;
@@ -1557,10 +1602,10 @@ size_t rac_encode_workspace_bytes(const rac_codec_cfg *cfg, int64_t T) {
     return ((size_t)T * (size_t)(g.d / 32) * sizeof(float) + 15) / 16 * 16;
 }
 
-int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
-               const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
-               const float *inv_step, void *payload, size_t payload_cap, void *workspace, size_t workspace_bytes,
-               uint32_t *dev_status, void *stream) {
+static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+                       const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
+                       const float *inv_step, void *payload, size_t payload_cap, void *X_hat, void *workspace,
+                       size_t workspace_bytes, uint32_t *dev_status, void *stream) {
     Geometry g;
     int rc = make_geometry(cfg, &g);
     if (rc != RAC_OK) return rc;
@@ -1570,6 +1615,7 @@ int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *r
     if (T == 0) return RAC_OK;
     if (!X || !payload || !step || !inv_step) return RAC_EINVAL;
     if (!aligned16(X) || !aligned16(payload) || !aligned16(step) || !aligned16(inv_step)) return RAC_EALIGN;
+    if (X_hat && !aligned16(X_hat)) return RAC_EALIGN;
     if (payload_cap < (size_t)g.rec * (size_t)T) return RAC_ESIZE;
     const size_t need = rac_encode_workspace_bytes(cfg, T);
     if (need > 0) {
@@ -1579,10 +1625,28 @@ int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *r
     }
     p.X = static_cast<const uint16_t *>(X);
     p.payload = static_cast<uint8_t *>(payload);
+    p.X_hat = static_cast<uint16_t *>(X_hat);
     p.step = step;
     p.inv_step = inv_step;
     p.tmax = static_cast<float *>(workspace);
     return launch_encode(g, p, T, static_cast<cudaStream_t>(stream));
+}
+
+int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+               const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
+               const float *inv_step, void *payload, size_t payload_cap, void *workspace, size_t workspace_bytes,
+               uint32_t *dev_status, void *stream) {
+    return encode_impl(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload, payload_cap,
+                       nullptr, workspace, workspace_bytes, dev_status, stream);
+}
+
+int rac_encode_reconstruct(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+                           const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
+                           const float *inv_step, void *payload, size_t payload_cap, void *X_hat, void *workspace,
+                           size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+    if (T > 0 && !X_hat) return RAC_EINVAL;
+    return encode_impl(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload, payload_cap,
+                       X_hat, workspace, workspace_bytes, dev_status, stream);
 }
 
 int rac_decode_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_t T, const void *ref_base,

@@ -129,6 +129,23 @@ def gpu_encode(cfg, X, ref_base, ref_row, gain, bias, step, inv_step, pad=64):
     return host[pad:pad + T * rec].copy(), int(status.item())
 
 
+def gpu_encode_reconstruct(cfg, X, ref_base, ref_row, gain, bias, step, inv_step):
+    """rac_encode_reconstruct: returns (payload numpy, X_hat tensor, status)."""
+    dev = X.device
+    T = X.shape[0]
+    rec = rac.rac_record_bytes(cfg)
+    payload = torch.full((T * rec,), 0xA5, dtype=torch.uint8, device=dev)
+    buf = torch.full((T + 2, cfg.d), -7.0, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev) if nws else None
+    rac.rac_encode_reconstruct(cfg, X, T, ref_base, 0 if ref_base is None else ref_base.shape[0], ref_row, gain, bias,
+                               step, inv_step, payload, T * rec, buf[1:T + 1], ws, nws, status)
+    torch.cuda.synchronize()
+    assert torch.all(buf[0] == -7.0) and torch.all(buf[T + 1] == -7.0), "encode_reconstruct wrote outside X_hat"
+    return payload.cpu().numpy(), buf[1:T + 1], int(status.item())
+
+
 def gpu_decode(cfg, payload_np, T, ref_base, ref_row, gain, bias, step, dev, fn=None, pad_rows=1):
     fn = fn or rac.rac_decode_reconstruct
     d = cfg.d
@@ -162,6 +179,11 @@ def round_trip_case(cfg, X, ref_base=None, ref_row=None, gain=None, bias=None, s
     assert st == 0, f"decode status {st}"
     xs, st = gpu_decode(cfg, pay, T, ref_base, ref_row, gain, bias, step_d, dev, fn=rac.rac_sender_reconstruct)
     assert torch.equal(xr, xs), "sender and receiver reconstructions differ"
+    # the fused encode + sender reconstruction: same payload bytes, same x_hat bits
+    pay_f, xs_f, st = gpu_encode_reconstruct(cfg, X, ref_base, ref_row, gain, bias, step_d, inv_d)
+    assert st == 0, f"encode_reconstruct status {st}"
+    assert np.array_equal(pay_f, pay), "rac_encode_reconstruct payload differs from rac_encode"
+    assert torch.equal(xs_f, xr), "fused sender reconstruction differs from the receiver's"
     o_x = oracle.reconstruct(d, g, bits, k, pay, T, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step,
                              nthreads=oracle.max_threads())
     assert np.array_equal(o_x, synth.bf16_bits(xr)), "device reconstruction differs from the oracle's"
