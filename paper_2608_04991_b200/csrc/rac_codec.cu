@@ -1,16 +1,21 @@
-// RAC codec kernels for sm_100a: encode (Sec. IV-C, Eq. 6-8 + packing), reconstruct (Eq. 9), and the
-// residual-RMS pass behind the step tables.
+// RAC codec kernels for sm_100a: encode (Sec. IV-C, Eq. 6-8 + packing, outlier split), reconstruct (Eq. 9),
+// and the residual-RMS pass behind the step tables.
 //
-// Shape of every kernel: persistent CTAs, one token per CTA iteration, one thread per 32 consecutive
-// channels.  Rows travel between HBM and shared memory only as 1-D bulk copies (TMA without a tensor
-// map): a ring of stages is filled ahead by thread 0 and signalled through mbarriers, finished records
-// and rows leave through bulk stores.  The arithmetic that decides integers (residual, scaling,
-// rounding) is binary32 with one rounding per operation, written with explicit intrinsics / PTX so the
-// compiler cannot contract or reorder it.
+// Shape of the streaming kernels: persistent CTAs, one token per CTA iteration, one thread per 32
+// consecutive channels.  Rows travel between HBM and shared memory only as 1-D bulk copies (TMA without a
+// tensor map): a ring of stages is filled ahead and signalled through mbarriers, finished records and rows
+// leave through bulk stores.  Every wait on an mbarrier is bounded; a copy that never lands ends the kernel
+// with a status bit instead of a hang.  The arithmetic that decides integers (residual, scaling, rounding)
+// is binary32 with one rounding per operation, written with explicit intrinsics / PTX so the compiler
+// cannot contract or reorder it.
 //
 // Shared-memory reads of a thread's 64-byte slab go through a per-lane rotation of the four 16-byte
 // pieces (piece (j + lane/2) mod 4 in step j), which makes the 128-bit accesses bank-conflict free
 // on a plain linear row.
+//
+// Kernels: encode_ws_kernel (streaming pass of encode, optionally also the sender-side x_hat),
+// outlier_kernel (second launch of encode: the k largest |e| per token), decode_kernel (receiver and sender
+// reconstruction), calib_kernel + calib_finalize_kernel (step tables).
 #include <math.h>
 #include <stdlib.h>
 
@@ -71,36 +76,25 @@ struct CodecParams {
 
 constexpr int kMaxStages = 4;
 constexpr int kRecBufs = 3;
-constexpr int kCandCap = 256;
 constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer (ties to even) in the low mantissa bits
 
 // control block at the start of dynamic shared memory
 struct Ctrl {
     unsigned long long bar[kMaxStages];
     int row[kMaxStages];        // reference row of the token in each stage, -1 = direct
-    unsigned int wtau[8];
-    unsigned long long red[8];
-    int n_hot, n_cand, abort, pad;
 };
 
 __host__ __device__ inline int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
-struct EncSmem {
-    int ctrl, stage0, stage_bytes, rec0, es0, hot0, cand0, crank0, sel0, total;
+struct EncSmem {  // calibration kernel
+    int stage0, stage_bytes, acc0, total;
 };
-__host__ __device__ inline EncSmem enc_smem_layout(int d, int rec, int stages, int nthreads, bool topk, bool calib) {
+__host__ __device__ inline EncSmem enc_smem_layout(int d, int stages, int nthreads) {
     EncSmem s;
-    s.ctrl = 0;
     s.stage0 = align_up((int)sizeof(Ctrl), 128);
     s.stage_bytes = 4 * d;  // X row + R row
-    s.rec0 = s.stage0 + stages * s.stage_bytes;
-    s.es0 = align_up(s.rec0 + (calib ? 0 : kRecBufs * rec), 16);
-    int es_bytes = calib ? 2 * nthreads * 32 * 4 : 0;  // calibration accumulators (residuals reuse the stage)
-    s.hot0 = s.es0 + es_bytes;
-    s.cand0 = align_up(s.hot0 + (topk ? nthreads * 4 * 2 : 0), 16);
-    s.crank0 = s.cand0 + (topk ? kCandCap * 8 : 0);
-    s.sel0 = align_up(s.crank0 + (topk ? kCandCap * 2 : 0), 16);
-    s.total = s.sel0 + (topk ? 16 * 8 : 0);
+    s.acc0 = s.stage0 + stages * s.stage_bytes;   // e^2 accumulators: 2 table rows x 32 floats per thread
+    s.total = s.acc0 + 2 * nthreads * 32 * 4;
     return s;
 }
 
@@ -240,53 +234,97 @@ __device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ct
     if (row >= 0) bulk_load(stage_addr + r_off, p.ref_base + (long long)row * p.d, row_bytes, bar);
 }
 
+// Eq. 6 for the group this thread belongs to: centred two-pass sums over the thread's 32 channels (packed
+// binary32, two accumulators per sum), butterflies over the group's lanes, the zero-variance rule, and wire
+// rounding of (alpha, beta) to binary16.  Returns the wire coefficients splatted for packed arithmetic; a16/b16
+// are their bit patterns.
+__device__ __forceinline__ void fit_group(const u64 (&x2)[16], const u64 (&r2)[16], bool has_ref, int lpg, float inv_group,
+                                          unsigned int group_mask, uint32_t *status, u64 &a2, u64 &b2,
+                                          uint32_t *coef_word = nullptr) {
+    u64 sra = 0ull, srb = 0ull, sha = 0ull, shb = 0ull;
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        sra = padd(sra, r2[i]); srb = padd(srb, r2[i + 1]);
+        sha = padd(sha, x2[i]); shb = padd(shb, x2[i + 1]);
+    }
+    float sr, sr_hi, sh, sh_hi;
+    unpack2(padd(sra, srb), sr, sr_hi);
+    unpack2(padd(sha, shb), sh, sh_hi);
+    sr += sr_hi;
+    sh += sh_hi;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        if (lpg > o) {
+            sr += __shfl_xor_sync(group_mask, sr, o);
+            sh += __shfl_xor_sync(group_mask, sh, o);
+        }
+    }
+    if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
+        if (status) atomicOr(status, RAC_STATUS_NONFINITE);
+    }
+    const float rbar = sr * inv_group, hbar = sh * inv_group;
+    const u64 rbar2 = pack2(rbar, rbar), hbar2 = pack2(hbar, hbar);
+    u64 sxxa = 0ull, sxxb = 0ull, sxya = 0ull, sxyb = 0ull;
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        u64 dr0 = psub(r2[i], rbar2), dh0 = psub(x2[i], hbar2);
+        u64 dr1 = psub(r2[i + 1], rbar2), dh1 = psub(x2[i + 1], hbar2);
+        sxxa = pfma(dr0, dr0, sxxa); sxya = pfma(dr0, dh0, sxya);
+        sxxb = pfma(dr1, dr1, sxxb); sxyb = pfma(dr1, dh1, sxyb);
+    }
+    float sxx, sxx_hi, sxy, sxy_hi;
+    unpack2(padd(sxxa, sxxb), sxx, sxx_hi);
+    unpack2(padd(sxya, sxyb), sxy, sxy_hi);
+    sxx += sxx_hi;
+    sxy += sxy_hi;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        if (lpg > o) {
+            sxx += __shfl_xor_sync(group_mask, sxx, o);
+            sxy += __shfl_xor_sync(group_mask, sxy, o);
+        }
+    }
+    // zero-variance rule, then wire rounding to binary16
+    float a_star = 0.f, b_star = hbar;
+    if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {
+        a_star = __fdiv_rn(sxy, sxx);
+        b_star = __fmaf_rn(-a_star, rbar, hbar);
+    }
+    const uint32_t a16 = float_to_half_bits_sat(a_star), b16 = float_to_half_bits_sat(b_star);
+    const float a = half_bits_to_float(a16), b = half_bits_to_float(b16);
+    a2 = pack2(a, a);
+    b2 = pack2(b, b);
+    if (coef_word) *coef_word = a16 | (b16 << 16);
+}
+
 // ------------------------------------------------------------------------------------------------
-// encode / calibrate
+// calibration pass: per-channel sums of e^2 (the residual of Eq. 7 with wire coefficients)
 // ------------------------------------------------------------------------------------------------
-// MODE 0: encode.  MODE 1: accumulate e^2 per channel for the step tables.
-//
-// Per token: (1) every thread pulls its 32 channels of X and of the reference row out of the stage,
-// (2) Eq. 6 statistics: in-thread sums with packed binary32 adds / fmas, then log2(lanes per group) shuffles,
-// (3) wire coefficients, residual, scaling, rounding by the magic-number add, packing, all per thread,
-// (4) with outliers: the residuals overwrite the thread's own slab of the stage (same bytes: 2+2 per
-//     channel in, 4 out) so that the selection can look at other threads' values.
-template <int BITS, bool TOPK, int MODE>
-__global__ void __launch_bounds__(256, 2) encode_kernel(const CodecParams p) {
+// Same front end as the encoder (slab loads, Eq. 6 statistics, wire coefficients); instead of codes, every
+// thread accumulates e^2 of its own 32 channels in shared memory, separately for tokens with a reference
+// (row 0) and tokens coded directly (row 1).  One CTA barrier per token; the grid is fixed.
+__global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
-    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int lane = tid & 31;
     const int rot = (lane >> 1) & 3;
     const int d = p.d;
     const bool valid = tid * 32 < d;
-    constexpr bool CALIB = (MODE == 1);
-    const EncSmem L = enc_smem_layout(d, p.rec, p.stages, nt, TOPK, CALIB);
+    const EncSmem L = enc_smem_layout(d, p.stages, nt);
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
     const int S = p.stages;
-    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
-    constexpr uint32_t cmask = (1u << BITS) - 1u;
     const uint32_t row_bytes = 2u * (uint32_t)d;
 
     if (tid == 0) {
         for (int s = 0; s < S; s++) mbar_init(smem_u32(&ctrl->bar[s]), 1);
-        ctrl->n_hot = 0;
-        ctrl->n_cand = 0;
         mbar_init_fence();
     }
-    if (!CALIB) {
-        // padding words of the record buffers are written once and never touched again
-        int raw = 4 * p.J + p.code_bytes + 4 * p.topk;
-        for (int b = 0; b < kRecBufs; b++)
-            for (int o = raw + 4 * tid; o < p.rec; o += 4 * nt) *reinterpret_cast<uint32_t *>(smem + L.rec0 + b * p.rec + o) = 0u;
-    } else {
-        for (int o = tid; o < 2 * nt * 32; o += nt) reinterpret_cast<float *>(smem + L.es0)[o] = 0.f;
-    }
+    for (int o = tid; o < 2 * nt * 32; o += nt) reinterpret_cast<float *>(smem + L.acc0)[o] = 0.f;
     __syncthreads();
 
     const int first = blockIdx.x, stride = gridDim.x;
     const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
-
-    // thread 0 keeps the reference row of the next token to issue one iteration ahead of its use
     int next_raw = 0;
     auto raw_row_of = [&](int k) -> int {  // raw ref_row entry of this CTA's k-th token
         long long t = first + (long long)k * stride;
@@ -300,21 +338,16 @@ __global__ void __launch_bounds__(256, 2) encode_kernel(const CodecParams p) {
         }
         if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
     }
-    int cnt_ref = 0, cnt_dir = 0;  // calibrate: tokens per table row (thread 0 only)
-
-    // byte offsets of the four 16-byte pieces of this thread's slab, in slot order
+    int cnt_ref = 0, cnt_dir = 0;  // tokens per table row (thread 0 only)
     uint32_t off[4];
 #pragma unroll
     for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
-    // the shuffles of step (2) run under `valid`: name exactly the lanes that take part (a group's lanes are
-    // always all valid or all invalid, so every partner is in the mask)
     const unsigned int group_mask = __ballot_sync(0xffffffffu, valid);
 
-    int stage = 0, rbuf = 0, issue_stage = S - 1;
+    int stage = 0, issue_stage = S - 1;
     bool aborted = false;
     uint32_t parity = 0;
     for (int it = 0; it < n_my; it++) {
-        const long long t = first + (long long)it * stride;
         if (tid == 0 && it + S - 1 < n_my) {
             const int k = it + S - 1;
             const long long tk = first + (long long)k * stride;
@@ -327,11 +360,8 @@ __global__ void __launch_bounds__(256, 2) encode_kernel(const CodecParams p) {
         const bool has_ref = ctrl->row[stage] >= 0;
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
-        unsigned char *rec = smem + L.rec0 + rbuf * p.rec;
-        float cmax[4] = {0.f, 0.f, 0.f, 0.f};
 
         if (valid) {
-            // ---- (1) the slab: 4 slots of 8 channels, slot j holds piece (j + rot) & 3
             u64 x2[16], r2[16];
 #pragma unroll
             for (int j = 0; j < 4; j++) {
@@ -353,302 +383,46 @@ __global__ void __launch_bounds__(256, 2) encode_kernel(const CodecParams p) {
 #pragma unroll
                 for (int i = 0; i < 16; i++) r2[i] = 0ull;
             }
-
-            // ---- (2) Eq. 6: centred sums over the group (two accumulators per sum keep the adders busy)
-            u64 sra = 0ull, srb = 0ull, sha = 0ull, shb = 0ull;
+            u64 a2, b2;
+            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2);
+            float4 *acc = reinterpret_cast<float4 *>(smem + L.acc0) + (has_ref ? 0 : 8 * nt);
 #pragma unroll
-            for (int i = 0; i < 16; i += 2) {
-                sra = padd(sra, r2[i]); srb = padd(srb, r2[i + 1]);
-                sha = padd(sha, x2[i]); shb = padd(shb, x2[i + 1]);
-            }
-            float sr, sr_hi, sh, sh_hi;
-            unpack2(padd(sra, srb), sr, sr_hi);
-            unpack2(padd(sha, shb), sh, sh_hi);
-            sr += sr_hi;
-            sh += sh_hi;
+            for (int j = 0; j < 4; j++) {
+                const int q = (j + rot) & 3;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                if (p.lpg > o) {
-                    sr += __shfl_xor_sync(group_mask, sr, o);
-                    sh += __shfl_xor_sync(group_mask, sh, o);
-                }
-            }
-            if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
-                if (p.status) atomicOr(p.status, RAC_STATUS_NONFINITE);
-            }
-            const float rbar = sr * p.inv_group, hbar = sh * p.inv_group;
-            const u64 rbar2 = pack2(rbar, rbar), hbar2 = pack2(hbar, hbar);
-            u64 sxxa = 0ull, sxxb = 0ull, sxya = 0ull, sxyb = 0ull;
-#pragma unroll
-            for (int i = 0; i < 16; i += 2) {
-                u64 dr0 = psub(r2[i], rbar2), dh0 = psub(x2[i], hbar2);
-                u64 dr1 = psub(r2[i + 1], rbar2), dh1 = psub(x2[i + 1], hbar2);
-                sxxa = pfma(dr0, dr0, sxxa); sxya = pfma(dr0, dh0, sxya);
-                sxxb = pfma(dr1, dr1, sxxb); sxyb = pfma(dr1, dh1, sxyb);
-            }
-            float sxx, sxx_hi, sxy, sxy_hi;
-            unpack2(padd(sxxa, sxxb), sxx, sxx_hi);
-            unpack2(padd(sxya, sxyb), sxy, sxy_hi);
-            sxx += sxx_hi;
-            sxy += sxy_hi;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                if (p.lpg > o) {
-                    sxx += __shfl_xor_sync(group_mask, sxx, o);
-                    sxy += __shfl_xor_sync(group_mask, sxy, o);
-                }
-            }
-            // zero-variance rule, then wire rounding to binary16
-            float a_star = 0.f, b_star = hbar;
-            if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {
-                a_star = __fdiv_rn(sxy, sxx);
-                b_star = __fmaf_rn(-a_star, rbar, hbar);
-            }
-            const uint32_t a16 = float_to_half_bits_sat(a_star), b16 = float_to_half_bits_sat(b_star);
-            const float a = half_bits_to_float(a16), b = half_bits_to_float(b16);
-            const u64 a2 = pack2(a, a), b2 = pack2(b, b);
-
-            if (CALIB) {
-                // ---- accumulate e^2 of the thread's own channels (row 0: referenced, row 1: direct)
-                float4 *acc = reinterpret_cast<float4 *>(smem + L.es0) + (has_ref ? 0 : 8 * nt);
-#pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    const int q = (j + rot) & 3;
-#pragma unroll
-                    for (int hh = 0; hh < 2; hh++) {
-                        float e0, e1, e2, e3;
-                        unpack2(psub(x2[4 * j + 2 * hh], pfma(a2, r2[4 * j + 2 * hh], b2)), e0, e1);
-                        unpack2(psub(x2[4 * j + 2 * hh + 1], pfma(a2, r2[4 * j + 2 * hh + 1], b2)), e2, e3);
-                        float4 v = acc[(2 * q + hh) * nt + tid];
-                        v.x = __fmaf_rn(e0, e0, v.x);
-                        v.y = __fmaf_rn(e1, e1, v.y);
-                        v.z = __fmaf_rn(e2, e2, v.z);
-                        v.w = __fmaf_rn(e3, e3, v.w);
-                        acc[(2 * q + hh) * nt + tid] = v;
-                    }
-                }
-            } else {
-                // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
-                if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = a16 | (b16 << 16);
-                const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
-                const u64 magic2 = pack2(kMagic, kMagic);
-                uint32_t words[4];
-#pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    const int c = (int)(off[j] >> 1);
-                    const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
-                    const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
-                    const u64 inv2[4] = {pack2(iv0.x, iv0.y), pack2(iv0.z, iv0.w), pack2(iv1.x, iv1.y), pack2(iv1.z, iv1.w)};
-                    float ev[8];
-                    float m0 = 0.f, m1 = 0.f;
-                    uint32_t w = 0;
-                    if (BITS == 3) {
-                        uint32_t bits8[8];
-#pragma unroll
-                        for (int i = 0; i < 4; i++) {
-                            const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
-                            float v0, v1, t0, t1;
-                            unpack2(pmul(e, inv2[i]), v0, v1);
-                            t0 = fminf(fmaxf(v0, -qmax), qmax);
-                            t1 = fminf(fmaxf(v1, -qmax), qmax);
-                            unpack2(padd(pack2(t0, t1), magic2), t0, t1);
-                            bits8[2 * i] = __float_as_uint(t0);
-                            bits8[2 * i + 1] = __float_as_uint(t1);
-                            unpack2(e, ev[2 * i], ev[2 * i + 1]);
-                        }
-                        w = pack8<BITS>(bits8);
-                    } else {
-                        // 4- and 2-bit codes: clamp from below in binary32, round by the magic add, take the integer
-                        // out of the mantissa and let the saturating pack clamp from above (its range is
-                        // [-2^(BITS-1), 2^(BITS-1)-1], whose upper end is Qmax)
-#pragma unroll
-                        for (int i = 3; i >= 0; i--) {
-                            const u64 e = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
-                            float v0, v1, t0, t1;
-                            unpack2(pmul(e, inv2[i]), v0, v1);
-                            unpack2(padd(pack2(fmaxf(v0, -qmax), fmaxf(v1, -qmax)), magic2), t0, t1);
-                            w = sat_pack2<BITS>((int)__float_as_uint(t1) - 0x4b400000, (int)__float_as_uint(t0) - 0x4b400000, w);
-                            unpack2(e, ev[2 * i], ev[2 * i + 1]);
-                        }
-                    }
-                    words[j] = w;
-                    if (TOPK) {
-                        m0 = fmaxf(fmaxf(fabsf(ev[0]), fabsf(ev[1])), fmaxf(fabsf(ev[2]), fabsf(ev[3])));
-                        m1 = fmaxf(fmaxf(fabsf(ev[4]), fabsf(ev[5])), fmaxf(fabsf(ev[6]), fabsf(ev[7])));
-                    }
-                    const float m = fmaxf(m0, m1);
-                    if (TOPK) {
-                        // (4) residuals of piece q go to float4 slots 2q, 2q+1 of the thread's 8 (0-3: X slab, 4-7: R slab)
-                        cmax[j] = m;
-                        const uint32_t q = (off[j] >> 4) & 3u;
-                        const uint32_t base = (q < 2 ? xs : rs) + (uint32_t)tid * 64u + (q & 1u) * 32u;
-                        sts128(base, make_uint4(__float_as_uint(ev[0]), __float_as_uint(ev[1]), __float_as_uint(ev[2]),
-                                                __float_as_uint(ev[3])));
-                        sts128(base + 16, make_uint4(__float_as_uint(ev[4]), __float_as_uint(ev[5]), __float_as_uint(ev[6]),
-                                                     __float_as_uint(ev[7])));
-                    }
-                }
-                rot_right4(words, rot);  // words[q] is now the code word of piece q
-                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + 4 * p.J) + tid * BITS;
-                if (BITS == 4) {
-                    cw[0] = words[0]; cw[1] = words[1]; cw[2] = words[2]; cw[3] = words[3];
-                } else if (BITS == 3) {
-                    cw[0] = words[0] | (words[1] << 24);
-                    cw[1] = (words[1] >> 8) | (words[2] << 16);
-                    cw[2] = (words[2] >> 16) | (words[3] << 8);
-                } else {
-                    cw[0] = words[0] | (words[1] << 16);
-                    cw[1] = words[2] | (words[3] << 16);
+                for (int hh = 0; hh < 2; hh++) {
+                    float e0, e1, e2, e3;
+                    unpack2(psub(x2[4 * j + 2 * hh], pfma(a2, r2[4 * j + 2 * hh], b2)), e0, e1);
+                    unpack2(psub(x2[4 * j + 2 * hh + 1], pfma(a2, r2[4 * j + 2 * hh + 1], b2)), e2, e3);
+                    float4 v = acc[(2 * q + hh) * nt + tid];
+                    v.x = __fmaf_rn(e0, e0, v.x);
+                    v.y = __fmaf_rn(e1, e1, v.y);
+                    v.z = __fmaf_rn(e2, e2, v.z);
+                    v.w = __fmaf_rn(e3, e3, v.w);
+                    acc[(2 * q + hh) * nt + tid] = v;
                 }
             }
         }
-
-        if (CALIB) {
-            if (tid == 0) { if (has_ref) cnt_ref++; else cnt_dir++; }
-            if (__syncthreads_or(timed_out)) { aborted = true; break; }  // one vote: every thread leaves together
-        } else {
-            if (TOPK) {
-                // ---- outlier split: the k largest |e| of the token, ties to the lower channel.
-                // Threshold: every warp contributes its c-th largest lane maximum, c = ceil(k / warps); the
-                // minimum of those has at least k elements at or above it.
-                unsigned int lm = __float_as_uint(fmaxf(fmaxf(cmax[0], cmax[1]), fmaxf(cmax[2], cmax[3])));
-                const int cth = (p.topk + nwarps - 1) / nwarps;
-                unsigned int v = lm, m = 0;
-                for (int r = 0; r < cth; r++) {
-                    m = __reduce_max_sync(0xffffffffu, v);
-                    if (r + 1 < cth) {
-                        unsigned int bal = __ballot_sync(0xffffffffu, v == m);
-                        if (lane == __ffs(bal) - 1) v = 0u;
-                    }
-                }
-                if (lane == 0) ctrl->wtau[warp] = m;
-                __syncthreads();  // S1
-                unsigned int tau = 0xffffffffu;
-                for (int w = 0; w < nwarps; w++) tau = min(tau, ctrl->wtau[w]);
-                unsigned short *hot = reinterpret_cast<unsigned short *>(smem + L.hot0);
-                if (valid) {
-#pragma unroll
-                    for (int j = 0; j < 4; j++) {
-                        if (__float_as_uint(cmax[j]) >= tau) {
-                            int pos = atomicAdd(&ctrl->n_hot, 1);
-                            hot[pos] = (unsigned short)((tid << 2) | ((off[j] >> 4) & 3u));
-                        }
-                    }
-                }
-                __syncthreads();  // S2
-                const int nh = ctrl->n_hot;
-                const unsigned char *xsp = smem + L.stage0 + stage * L.stage_bytes;
-                // residual of channel c, as stored in step (4)
-                auto e_of = [&](int c) -> float {
-                    const int th = c >> 5, f = (c >> 2) & 7;
-                    return *reinterpret_cast<const float *>(xsp + (f < 4 ? 0 : row_bytes) + th * 64 + (f & 3) * 16 + (c & 3) * 4);
-                };
-                unsigned long long *cand = reinterpret_cast<unsigned long long *>(smem + L.cand0);
-                unsigned short *crank = reinterpret_cast<unsigned short *>(smem + L.crank0);
-                for (int x = tid; x < nh * 8; x += nt) {
-                    const int h = hot[x >> 3];
-                    const int c = (h >> 2) * 32 + (h & 3) * 8 + (x & 7);
-                    const unsigned int key = __float_as_uint(e_of(c)) & 0x7fffffffu;
-                    if (key >= tau) {
-                        int pos = atomicAdd(&ctrl->n_cand, 1);
-                        if (pos < kCandCap) cand[pos] = ((unsigned long long)key << 16) | (unsigned long long)(0xffff - c);
-                    }
-                }
-                __syncthreads();  // S3
-                const int nc = ctrl->n_cand;
-                const int k = p.topk;
-                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
-                unsigned short *oval = oidx + k;
-                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
-                unsigned long long *sel = reinterpret_cast<unsigned long long *>(smem + L.sel0);
-                if (nc <= kCandCap) {
-                    // rank by counting: candidate x is the (rank)-th largest
-                    for (int x = tid; x < nc; x += nt) {
-                        const unsigned long long mine = cand[x];
-                        int rk = 0;
-                        for (int y = 0; y < nc; y++) rk += (cand[y] > mine) ? 1 : 0;
-                        crank[x] = (unsigned short)rk;
-                        if (rk < k) sel[rk] = mine;
-                    }
-                } else {
-                    // rare: more candidates than the list holds (many equal magnitudes).  k rounds of a
-                    // block-wide maximum over all residuals, each strictly below the previous pick.
-                    unsigned long long prev = ~0ull;
-                    for (int n = 0; n < k; n++) {
-                        unsigned long long best = 0ull;
-                        if (valid) {
-                            for (int cc = 0; cc < 32; cc++) {
-                                const int c = tid * 32 + cc;
-                                const unsigned long long comp =
-                                    ((unsigned long long)(__float_as_uint(e_of(c)) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
-                                // a composite is 0 only for |e| == 0 at channel 65535, which d <= 8192 excludes
-                                if (comp < prev && comp > best) best = comp;
-                            }
-                        }
-                        for (int o = 16; o > 0; o >>= 1) {
-                            unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-                            best = other > best ? other : best;
-                        }
-                        if (lane == 0) ctrl->red[warp] = best;
-                        __syncthreads();
-                        best = 0ull;
-                        for (int w = 0; w < nwarps; w++) best = ctrl->red[w] > best ? ctrl->red[w] : best;
-                        if (tid == 0) sel[n] = best;
-                        prev = best;
-                        __syncthreads();
-                    }
-                }
-                __syncthreads();  // S4
-                if (tid < k) {
-                    const unsigned long long mine = sel[tid];
-                    const int c = 0xffff - (int)(mine & 0xffffull);
-                    if (c < d) {
-                        int pos = 0;
-                        for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
-                        oidx[pos] = (unsigned short)c;
-                        oval[pos] = (unsigned short)float_to_half_bits_sat(e_of(c));
-                        // E^d = E - O: the dense code at an outlier position is zero
-                        const int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
-                        atomicAnd(&codes32[wd], ~(cmask << sh));
-                        if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
-                    }
-                }
-                if (tid == 0) { ctrl->n_hot = 0; ctrl->n_cand = 0; }
-            }
-
-            // ---- record complete: hand it to the copy engine
-            fence_async_smem();
-            if (__syncthreads_or(timed_out)) { aborted = true; break; }  // A; one vote: every thread leaves together
-            if (tid == 0) {
-                bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
-                bulk_commit();
-                bulk_wait_read<1>();  // the record buffer written two iterations from now is free again
-            }
-        }
+        if (tid == 0) { if (has_ref) cnt_ref++; else cnt_dir++; }
+        if (__syncthreads_or(timed_out)) { aborted = true; break; }  // one vote: every thread leaves together
         if (++stage == S) { stage = 0; parity ^= 1u; }
         if (++issue_stage == S) issue_stage = 0;
-        if (++rbuf == kRecBufs) rbuf = 0;
     }
 
-    if (CALIB) {
-        __syncthreads();
-        // partial sums of this CTA, channel order, then its token counts
-        float *out = p.calib_partial + (long long)blockIdx.x * 2 * d;
-        const float *acc = reinterpret_cast<const float *>(smem + L.es0);
-        if (valid) {
-            for (int rrow = 0; rrow < 2; rrow++)
-                for (int f = 0; f < 8; f++)
-                    for (int cc = 0; cc < 4; cc++)
-                        out[rrow * d + tid * 32 + f * 4 + cc] = acc[rrow * nt * 32 + ((f * nt) + tid) * 4 + cc];
-        }
-        if (tid == 0) {
-            int *cnt = reinterpret_cast<int *>(p.calib_partial + (long long)gridDim.x * 2 * d) + 2 * blockIdx.x;
-            cnt[0] = cnt_ref;
-            cnt[1] = cnt_dir;
-        }
+    __syncthreads();
+    // partial sums of this CTA, channel order, then its token counts
+    float *out = p.calib_partial + (long long)blockIdx.x * 2 * d;
+    const float *acc = reinterpret_cast<const float *>(smem + L.acc0);
+    if (valid) {
+        for (int rrow = 0; rrow < 2; rrow++)
+            for (int f = 0; f < 8; f++)
+                for (int cc = 0; cc < 4; cc++)
+                    out[rrow * d + tid * 32 + f * 4 + cc] = acc[rrow * nt * 32 + ((f * nt) + tid) * 4 + cc];
     }
     if (tid == 0) {
-        bulk_wait_all();
+        int *cnt = reinterpret_cast<int *>(p.calib_partial + (long long)gridDim.x * 2 * d) + 2 * blockIdx.x;
+        cnt[0] = cnt_ref;
+        cnt[1] = cnt_dir;
         if (aborted) {
             // give copies that may still be in flight a bounded chance to land before the CTA retires
             for (int s = 0; s < S; s++) {
@@ -782,62 +556,13 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 #pragma unroll
                 for (int i = 0; i < 16; i++) r2[i] = 0ull;
             }
-            // ---- (2) Eq. 6: centred sums over the group (two accumulators per sum keep the adders busy)
-            u64 sra = 0ull, srb = 0ull, sha = 0ull, shb = 0ull;
-#pragma unroll
-            for (int i = 0; i < 16; i += 2) {
-                sra = padd(sra, r2[i]); srb = padd(srb, r2[i + 1]);
-                sha = padd(sha, x2[i]); shb = padd(shb, x2[i + 1]);
-            }
-            float sr, sr_hi, sh, sh_hi;
-            unpack2(padd(sra, srb), sr, sr_hi);
-            unpack2(padd(sha, shb), sh, sh_hi);
-            sr += sr_hi;
-            sh += sh_hi;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                if (p.lpg > o) {
-                    sr += __shfl_xor_sync(group_mask, sr, o);
-                    sh += __shfl_xor_sync(group_mask, sh, o);
-                }
-            }
-            if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
-                if (p.status) atomicOr(p.status, RAC_STATUS_NONFINITE);
-            }
-            const float rbar = sr * p.inv_group, hbar = sh * p.inv_group;
-            const u64 rbar2 = pack2(rbar, rbar), hbar2 = pack2(hbar, hbar);
-            u64 sxxa = 0ull, sxxb = 0ull, sxya = 0ull, sxyb = 0ull;
-#pragma unroll
-            for (int i = 0; i < 16; i += 2) {
-                u64 dr0 = psub(r2[i], rbar2), dh0 = psub(x2[i], hbar2);
-                u64 dr1 = psub(r2[i + 1], rbar2), dh1 = psub(x2[i + 1], hbar2);
-                sxxa = pfma(dr0, dr0, sxxa); sxya = pfma(dr0, dh0, sxya);
-                sxxb = pfma(dr1, dr1, sxxb); sxyb = pfma(dr1, dh1, sxyb);
-            }
-            float sxx, sxx_hi, sxy, sxy_hi;
-            unpack2(padd(sxxa, sxxb), sxx, sxx_hi);
-            unpack2(padd(sxya, sxyb), sxy, sxy_hi);
-            sxx += sxx_hi;
-            sxy += sxy_hi;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                if (p.lpg > o) {
-                    sxx += __shfl_xor_sync(group_mask, sxx, o);
-                    sxy += __shfl_xor_sync(group_mask, sxy, o);
-                }
-            }
-            // zero-variance rule, then wire rounding to binary16
-            float a_star = 0.f, b_star = hbar;
-            if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {
-                a_star = __fdiv_rn(sxy, sxx);
-                b_star = __fmaf_rn(-a_star, rbar, hbar);
-            }
-            const uint32_t a16 = float_to_half_bits_sat(a_star), b16 = float_to_half_bits_sat(b_star);
-            const float a = half_bits_to_float(a16), b = half_bits_to_float(b16);
-            const u64 a2 = pack2(a, a), b2 = pack2(b, b);
+            // ---- (2) Eq. 6 and wire rounding
+            u64 a2, b2;
+            uint32_t coef_word;
+            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
 
             // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
-            if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = a16 | (b16 << 16);
+            if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
             const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
             const float *step_tab = p.step + (has_ref ? 0 : d);
             uint32_t words[4];
@@ -1686,15 +1411,14 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, cons
     p.calib_partial = static_cast<float *>(workspace);
     // every CTA of the fixed grid writes its partials, also when it has no token
     {
-        p.stages = pick_stages(g.d, g.d <= 4096 ? 3 : 2);
-        EncSmem L = enc_smem_layout(g.d, g.rec, p.stages, g.nthreads, false, true);
+        p.stages = pick_stages(g.d, 2);
+        EncSmem L = enc_smem_layout(g.d, p.stages, g.nthreads);
         DeviceInfo di;
         rc = device_info(&di);
         if (rc != RAC_OK) return rc;
         if (L.total > di.max_smem_optin) return RAC_EUNSUPPORTED;
-        auto kern = encode_kernel<4, false, 1>;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return RAC_ECUDA;
-        kern<<<kCalibGrid, g.nthreads, L.total, st>>>(p);
+        if (cudaFuncSetAttribute(calib_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return RAC_ECUDA;
+        calib_kernel<<<kCalibGrid, g.nthreads, L.total, st>>>(p);
         if (cudaGetLastError() != cudaSuccess) return RAC_ECUDA;
     }
     int n = 2 * g.d;
