@@ -457,8 +457,8 @@ struct WsSmem {
 __host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages) {
     WsSmem s;
     s.stage0 = align_up((int)sizeof(WsCtrl), 128);
-    s.rec_off = 4 * d;  // after X row + R row
-    s.stage_bytes = align_up(s.rec_off + rec, 128);
+    s.rec_off = 4 * d;  // after X row + R row: two record slots, used alternately (by the stage's parity)
+    s.stage_bytes = align_up(s.rec_off + 2 * rec, 128);
     s.total = s.stage0 + stages * s.stage_bytes;
     return s;
 }
@@ -507,9 +507,9 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     {
         // padding words of the records are written once and never touched again
         const int raw = 4 * p.J + p.code_bytes + 4 * p.topk;
-        for (int s = 0; s < S; s++)
+        for (int s = 0; s < 2 * S; s++)
             for (int o = raw + 4 * tid; o < p.rec; o += 4 * nt)
-                *reinterpret_cast<uint32_t *>(smem + L.stage0 + s * L.stage_bytes + L.rec_off + o) = 0u;
+                *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * p.rec + o) = 0u;
     }
     __syncthreads();
     if (tid == 0)
@@ -529,7 +529,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         unsigned char *stg = smem + L.stage0 + stage * L.stage_bytes;
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
-        unsigned char *rec = stg + L.rec_off;
+        unsigned char *rec = stg + L.rec_off + parity * p.rec;
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
@@ -664,15 +664,24 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             int raw_next = 0;
             if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);  // in flight while the tail runs
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
-            // ---- record complete: hand it to the copy engine, then refill the stage
+            // ---- refill the stage, then hand the record to the copy engine.  The record sits in the slot of the
+            // stage's current parity; the stage's next token writes the other slot, and the one after that
+            // cannot start before this warp has arrived for the token in between, which it does only after the
+            // wait below.  So the refill need not wait for the record to leave.  (With x_hat the X row itself
+            // is the source of a store and must have been read before new data may land on it.)
             if (lane == 0) {
                 const long long t = first + (long long)it * stride;
-                bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
-                if (XHAT) bulk_store(p.X_hat + t * d, xs, row_bytes);
-                bulk_commit();
-                if (k_next < n_my) {
-                    bulk_wait_read<0>();  // the record must have left before the next token may write it
-                    issue(k_next, stage, raw_next);
+                if (XHAT) {
+                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_store(p.X_hat + t * d, xs, row_bytes);
+                    bulk_commit();
+                    bulk_wait_read<0>();
+                    if (k_next < n_my) issue(k_next, stage, raw_next);
+                } else {
+                    if (k_next < n_my) issue(k_next, stage, raw_next);
+                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_commit();
+                    bulk_wait_read<0>();
                 }
             }
             __syncwarp();
