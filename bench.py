@@ -31,6 +31,12 @@ if ROOT not in sys.path:
 METRIC = "codec GB/s of bf16 activations (encode+decode round trip)"
 UNIT = "GB/s"
 WORKLOAD = dict(T=131072, d=5120, group=128, bits=4, topk=8, n_hist=131072, min_ngram=4, max_hits=8, gap_max=112)
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one rac_encode[_reconstruct] call (streaming kernel +
+# outlier kernel) from the ncu capture of the SMALL case (profiles/codec_kernels_small_case_T16384_d5120.md);
+# traffic is proportional to tokens, so a launch of T tokens moves T/16384 times as much.
+NCU_SMALL_CASE_TRAFFIC = {"encode_sender_up": 267.80e6 + 179.96e6 + 53.34e6 + 1.63e6,
+                          "encode_dn": 335.61e6 + 44.24e6 + 59.43e6 + 0.45e6,
+                          "decode_up": 141.50e6 + 117.24e6, "decode_dn": 212.93e6 + 125.28e6}
 SMALL = dict(T=16384, d=5120, group=128, bits=4, topk=8, n_hist=16384, min_ngram=4, max_hits=8, gap_max=112)
 
 
@@ -423,8 +429,10 @@ def main():
             dom, dom_bytes, dom_ms, dom_n = ("decode_kernel<4,8>", rt.bytes_of("decode_up") + rt.bytes_of("decode_dn"),
                                              dec_ms, 2)
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+        dom_stages = ("encode_sender_up", "encode_dn") if enc_ms >= dec_ms else ("decode_up", "decode_dn")
+        traffic = sum(NCU_SMALL_CASE_TRAFFIC[n] for n in dom_stages) / len(dom_stages) * (wl["T"] / 16384.0)
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": None, "peak_source": peak_src, "launches_per_step": dom_n,
+                    "traffic": traffic, "traffic_source": "ncu small case (T=16384) scaled by tokens, bytes per call", "peak_source": peak_src, "launches_per_step": dom_n,
                     "algorithmic_bytes_per_launch": dom_bytes / dom_n, "avg_launch_ms": dom_ms / dom_n,
                     "frac_of_nominal_8TBps": achieved / 8000.0}
         cpu = None
