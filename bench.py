@@ -49,6 +49,7 @@ def parse_args():
     ap.add_argument("--small", action="store_true", help="a small case of the same path (for profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode-steps", action="store_true", help="skip the decode-step latency extra")
     return ap.parse_args()
 
 
@@ -235,6 +236,81 @@ class RoundTrip:
 
     def activation_bytes_per_step(self):
         return 2 * 2 * self.wl["T"] * self.wl["d"]
+
+
+# --------------------------------------------------------------------------------------------- decode-step latency
+def decode_step_latency(dev, n_steps=64, reps=20):
+    """Config 2 (64 sequences x 1 token, d=3584, 3-bit, group 128, no outliers, per-channel gain/bias reference,
+    x_hat fed back): microseconds per step of the sender call (encode + x_hat in one launch, in place) and of the
+    receiver call, launched eagerly and replayed from a CUDA graph of `n_steps` dependent steps."""
+    import torch
+    from paper_2608_04991_b200 import binding as rac
+    from paper_2608_04991_b200 import synth
+    B, d, g, bits = 64, 3584, 128, 3
+    cfg = rac.CodecCfg(d, g, bits, 0)
+    gen = synth.generator(synth.BASE_SEED + 2, dev)
+    scale = synth.channel_scale(d, 2, dev)
+    gain, bias = synth.predictor_gain_bias(d, 2, dev)
+    xs = [synth.activations(B, d, scale, gen)]
+    for _ in range(n_steps):
+        xs.append(synth.random_walk_step(xs[-1], gen))
+    step = torch.empty((2, d), dtype=torch.float32, device=dev)
+    inv = torch.empty_like(step)
+    nb = rac.rac_calibrate_workspace_bytes(cfg)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rac.rac_calibrate_steps(cfg, xs[1], B, xs[0], B, None, gain, bias, 3.0, step, inv, ws, nb, status)
+    rec = rac.rac_record_bytes(cfg)
+    pays = [torch.empty(B * rec, dtype=torch.uint8, device=dev) for _ in range(n_steps)]
+    send_state, recv_state = xs[0].clone(), xs[0].clone()      # the first step travels raw
+
+    def sender():
+        for t in range(n_steps):
+            rac.rac_encode_reconstruct(cfg, xs[t + 1], B, send_state, B, None, gain, bias, step, inv, pays[t],
+                                       pays[t].numel(), send_state, None, 0, status)
+
+    def receiver():
+        for t in range(n_steps):
+            rac.rac_decode_reconstruct(cfg, pays[t], B, recv_state, B, None, gain, bias, step, recv_state, status)
+
+    out = {}
+    for name, fn, state in (("sender_encode_plus_xhat", sender, send_state), ("receiver_reconstruct", receiver, recv_state)):
+        fn()                                                    # warm-up (also does the one-time function set-up)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        eager = e0.elapsed_time(e1) * 1e3 / (reps * n_steps)
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = {"us_per_step_eager": eager, "us_per_step_cuda_graph": e0.elapsed_time(e1) * 1e3 / (reps * n_steps)}
+    # one clean chain from the common first state: both ends must arrive at the same state
+    send_state.copy_(xs[0])
+    recv_state.copy_(xs[0])
+    sender()
+    receiver()
+    torch.cuda.synchronize()
+    if int(status.item()):
+        raise SystemExit(f"decode-step latency: device status {int(status.item())}")
+    if not torch.equal(send_state, recv_state):
+        raise SystemExit("decode-step latency: sender and receiver states differ")
+    out["config"] = {"sequences": B, "d": d, "bits": bits, "group": g, "steps_per_graph": n_steps}
+    return out
 
 
 # --------------------------------------------------------------------------------------------- CPU oracle legs
@@ -454,6 +530,7 @@ def main():
             "roofline": roofline,
             "cpu_baseline": cpu,
             "stages": per,
+            "decode_steps": None if args.no_decode_steps else decode_step_latency(dev),
         }
         print(json.dumps(line))
     if world > 1:

@@ -172,8 +172,9 @@ int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T,
  * reconstruction as the receiver"; here it reuses the residuals and codes the encoder already holds instead of
  * decoding its own payload again).  Arguments as rac_encode plus
  *   X_hat  bf16[T,d] out: bit-identical to what rac_decode_reconstruct / rac_sender_reconstruct produce from
- *          `payload` with the same reference and step table.  Must not overlap X, the reference rows in use, or
- *          payload.
+ *          `payload` with the same reference and step table.  Must not overlap X or payload.  It may be the very
+ *          buffer that ref_base points to ONLY with ref_row == NULL (token t reads row t and writes row t; each
+ *          row is read completely before it is written), which is how a decode loop keeps its state in place.
  * Both tables are read here (inv_step for the codes, step for x_hat). */
 int rac_encode_reconstruct(const rac_codec_cfg *cfg, const void *X, int64_t T,
                            const void *ref_base, int64_t ref_rows, const int32_t *ref_row,

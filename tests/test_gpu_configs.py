@@ -140,9 +140,17 @@ def test_config2_decode_steps_closed_loop(env):
     for t in range(1, steps + 1):
         x = s.random_walk_step(x, gen)
         prev_bits = s.bf16_bits(x_hat)      # the device's previous reconstruction: both sides start here
+        if t <= 64:
+            # the one-launch sender (encode + x_hat, state updated in place) must give the same bytes and state
+            fused_state = x_hat.clone()
+            fused_pay = torch.empty_like(payload)
+            rac.rac_encode_reconstruct(cfg, x, B, fused_state, B, None, gain, bias, step_d, inv_d, fused_pay,
+                                       fused_pay.numel(), fused_state, None, 0, status)
         rac.rac_encode(cfg, x, B, x_hat, B, None, gain, bias, step_d, inv_d, payload, payload.numel(), None, 0, status)
         rac.rac_sender_reconstruct(cfg, payload, B, x_hat, B, None, gain, bias, step_d, x_hat, status)  # in place
         torch.cuda.synchronize()
+        if t <= 64:
+            assert torch.equal(fused_pay, payload) and torch.equal(fused_state, x_hat), f"step {t}: fused sender differs"
         pay = payload.cpu().numpy()
         xb = s.bf16_bits(x)
         rep = env.P.compare_encode(cfg, pay, xb, prev_bits, None, gb, bb, step, inv)
