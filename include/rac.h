@@ -156,7 +156,8 @@ int rac_spans_to_rows(const rac_span *spans, const int32_t *n_spans, int64_t n_q
  *   payload   >= T*record bytes, 16-byte aligned; payload_cap is its capacity
  *   workspace >= rac_encode_workspace_bytes(cfg, T) bytes of scratch, 16-byte aligned (0 bytes, and NULL
  *             allowed, when cfg->topk == 0).  With outliers the call is two launches: the streaming pass leaves
- *             the largest |e| of every 32-channel slab here (4*d/32 bytes per token) and the outlier pass reads it.
+ *             the largest |e| of every 32-channel slab here (4*d/32 bytes per token, rows padded to 16 bytes) and the
+ *             outlier pass reads it.
  * The encoder reads only inv_step on the device: keep inv_step[c] == 0 wherever step[c] == 0 ("code 0").
  * The per-group fit is taken in binary32 on the device; its result, rounded to binary16, is what both
  * ends use, so any rounding difference against a binary64 fit shows up only in `coef`. */

@@ -452,13 +452,15 @@ struct WsCtrl {
 };
 
 struct WsSmem {
-    int stage0, stage_bytes, rec_off, total;
+    int stage0, stage_bytes, rec_off, tm_off, tm_bytes, total;
 };
-__host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages) {
+__host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages, bool topk) {
     WsSmem s;
     s.stage0 = align_up((int)sizeof(WsCtrl), 128);
     s.rec_off = 4 * d;  // after X row + R row: two record slots, used alternately (by the stage's parity)
-    s.stage_bytes = align_up(s.rec_off + 2 * rec, 128);
+    s.tm_off = s.rec_off + 2 * rec;  // two slots of per-slab maxima (outliers only), same alternation
+    s.tm_bytes = topk ? align_up((d / 32) * 4, 16) : 0;
+    s.stage_bytes = align_up(s.tm_off + 2 * s.tm_bytes, 128);
     s.total = s.stage0 + stages * s.stage_bytes;
     return s;
 }
@@ -471,7 +473,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     const int rot = (lane >> 1) & 3;
     const int d = p.d;
     const bool valid = tid * 32 < d;
-    const WsSmem L = ws_smem_layout(d, p.rec, p.stages);
+    const WsSmem L = ws_smem_layout(d, p.rec, p.stages, TOPK);
     WsCtrl *ctrl = reinterpret_cast<WsCtrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
     const int S = p.stages;
@@ -651,7 +653,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                 cw[1] = words[2] | (words[3] << 16);
             }
             // (4) the largest |e| of this thread's 32 channels, for the outlier pass
-            if (TOPK) p.tmax[(first + (long long)it * stride) * (d >> 5) + tid] = tmax;
+            if (TOPK) reinterpret_cast<float *>(stg + L.tm_off + parity * L.tm_bytes)[tid] = tmax;
         }
         // this warp's share of the token is in shared memory: one arrival per warp
         fence_async_smem();  // the record (and x_hat) bytes written above will be read by the copy engine
@@ -671,6 +673,8 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             // is the source of a store and must have been read before new data may land on it.)
             if (lane == 0) {
                 const long long t = first + (long long)it * stride;
+                if (TOPK)  // the slab maxima travel like the record: one bulk copy from this parity's slot
+                    bulk_store(p.tmax + t * (L.tm_bytes >> 2), xs + L.tm_off + parity * L.tm_bytes, (uint32_t)L.tm_bytes);
                 if (XHAT) {
                     bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
                     bulk_store(p.X_hat + t * d, xs, row_bytes);
@@ -762,7 +766,7 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
         };
 
         // (a) threshold; the slabs that reach it, in slab order
-        const float *tm = p.tmax + t * nth;
+        const float *tm = p.tmax + t * ((nth + 3) & ~3);  // rows are padded to 16 bytes
         const int ni = (nth + 31) >> 5;  // values per lane, at most 8
         unsigned int tv[8];
         unsigned int v = 0u;
@@ -1226,7 +1230,7 @@ static int pick_stages(int d, int dflt) {
 static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
     const bool topk = g.topk > 0;
     p.stages = pick_stages(g.d, 2);
-    WsSmem L = ws_smem_layout(g.d, g.rec, p.stages);
+    WsSmem L = ws_smem_layout(g.d, g.rec, p.stages, topk);
     // With x_hat the kernel reads both step tables every token; at four CTAs per SM the shared-memory carve-out
     // leaves too little L1 for them, so that variant runs three CTAs per SM at 128 registers.
     const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
@@ -1333,7 +1337,7 @@ size_t rac_encode_workspace_bytes(const rac_codec_cfg *cfg, int64_t T) {
     Geometry g;
     if (make_geometry(cfg, &g) != RAC_OK || T < 0) return 0;
     if (g.topk == 0) return 0;
-    return ((size_t)T * (size_t)(g.d / 32) * sizeof(float) + 15) / 16 * 16;
+    return (size_t)T * (size_t)(((g.d / 32) * 4 + 15) / 16 * 16);  // one 16-byte padded row of slab maxima per token
 }
 
 static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
