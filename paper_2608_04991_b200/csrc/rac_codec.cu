@@ -721,29 +721,38 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 // (d) The winners, in channel order, go into the record's outlier fields and their dense codes are cleared
 // (E^d = E - O).  More candidates than the list holds (many equal magnitudes) falls back to k rounds of a
 // maximum over the whole token.
-constexpr int kOutWarps = 8;       // warps (tokens in flight) per CTA
-constexpr int kOutCap = 128;       // candidate list per warp
-constexpr int kOutHot = 256;       // slab list per warp (d <= 8192 has at most 256 slabs)
+constexpr int kOutWarps = 8;       // warps per CTA
+constexpr int kOutCap = 128;       // candidate list per token in flight
+constexpr int kOutHot = 256;       // slab list per token in flight (d <= 8192 has at most 256 slabs)
 
-template <int BITS>
+// W lanes work on one token: W = 32 (a warp per token) or 16 (two tokens per warp; the instruction stream is
+// shared, so a token costs about two thirds of the issue slots).  All warp collectives name only the W lanes
+// of the token.
+template <int BITS, int W>
 __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecParams p) {
-    __shared__ unsigned long long s_cand[kOutWarps][kOutCap];
-    __shared__ float s_cande[kOutWarps][kOutCap];
-    __shared__ unsigned short s_hot[kOutWarps][kOutHot];
-    __shared__ unsigned long long s_sel[kOutWarps][16];
-    __shared__ float s_sele[kOutWarps][16];
+    constexpr int TPW = 32 / W;                 // tokens per warp
+    constexpr int NV = 256 / W;                 // slab maxima per lane, at most
+    __shared__ unsigned long long s_cand[kOutWarps * TPW][kOutCap];
+    __shared__ float s_cande[kOutWarps * TPW][kOutCap];
+    __shared__ unsigned short s_hot[kOutWarps * TPW][kOutHot];
+    __shared__ unsigned long long s_sel[kOutWarps * TPW][16];
+    __shared__ float s_sele[kOutWarps * TPW][16];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = lane / W, sl = lane % W;    // which token of the warp, lane within the token's group
+    const unsigned int gmask = (W == 32) ? 0xffffffffu : (0xffffu << (16 * sub));
+    const int slot = warp * TPW + sub;
     const int d = p.d, nth = d >> 5, k = p.topk;
     constexpr uint32_t cmask = (1u << BITS) - 1u;
-    unsigned long long *cand = s_cand[warp];
-    float *cande = s_cande[warp];
-    unsigned short *hot = s_hot[warp];
-    unsigned long long *sel = s_sel[warp];
-    float *sele = s_sele[warp];
-    const long long wstride = (long long)gridDim.x * kOutWarps;
-    const unsigned int lt_mask = (1u << lane) - 1u;
+    unsigned long long *cand = s_cand[slot];
+    float *cande = s_cande[slot];
+    unsigned short *hot = s_hot[slot];
+    unsigned long long *sel = s_sel[slot];
+    float *sele = s_sele[slot];
+    const long long tstride = (long long)gridDim.x * kOutWarps * TPW;
+    const unsigned int lt_mask = (1u << sl) - 1u;
+    const int tm_stride = (nth + 3) & ~3;       // rows of slab maxima are padded to 16 bytes
 
-    for (long long t = (long long)blockIdx.x * kOutWarps + warp; t < p.T; t += wstride) {
+    for (long long t = ((long long)blockIdx.x * kOutWarps + warp) * TPW + sub; t < p.T; t += tstride) {
         // reference row of the token, by the same rules as the streaming pass
         long long row = p.ref_row ? (long long)p.ref_row[t] : t;
         if (!p.ref_base || row < 0 || row >= p.ref_rows) row = -1;
@@ -751,61 +760,61 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
         const uint16_t *rrow = row >= 0 ? p.ref_base + row * d : nullptr;
         unsigned char *rec = p.payload + t * p.rec;
         const uint32_t *coef = reinterpret_cast<const uint32_t *>(rec);
-        // residual from the stored bits of x and r, exactly as the streaming pass computed it
-        auto residual_of = [&](uint32_t xb, uint32_t rb, int c, uint32_t cf) -> float {
-            const float h = __uint_as_float(xb << 16);
+        // residual of channel c, exactly as the streaming pass computed it (rare paths only)
+        auto residual = [&](int c) -> float {
+            const float h = __uint_as_float((uint32_t)xrow[c] << 16);
             float r = 0.f;
             if (rrow) {
-                r = __uint_as_float(rb << 16);
+                r = __uint_as_float((uint32_t)rrow[c] << 16);
                 if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
             }
+            const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
             return __fsub_rn(h, __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16)));
         };
-        auto residual = [&](int c) -> float {
-            return residual_of(xrow[c], rrow ? rrow[c] : 0u, c, coef[c >> (5 + p.lpg_shift)]);
-        };
 
-        // (a) threshold; the slabs that reach it, in slab order
-        const float *tm = p.tmax + t * ((nth + 3) & ~3);  // rows are padded to 16 bytes
-        const int ni = (nth + 31) >> 5;  // values per lane, at most 8
-        unsigned int tv[8];
+        // (a) threshold: the k-th largest of the W per-lane maxima (lane l covers slabs l, l+W, ...): the k largest
+        // come from k different lanes, each with an element at least that large, so at least k elements reach it;
+        // then the slabs that reach it, in slab order
+        const float *tm = p.tmax + t * tm_stride;
+        const int ni = (nth + W - 1) / W;
+        unsigned int tv[NV];
         unsigned int v = 0u;
 #pragma unroll
-        for (int i = 0; i < 8; i++) {
+        for (int i = 0; i < NV; i++) {
             tv[i] = 0u;
             if (i < ni) {
-                const int th = lane + 32 * i;
+                const int th = sl + W * i;
                 if (th < nth) tv[i] = __float_as_uint(tm[th]);
                 v = max(v, tv[i]);
             }
         }
         unsigned int tau = 0u;
-        for (int r = 0; r < k; r++) {
-            tau = __reduce_max_sync(0xffffffffu, v);
+        for (int r = 0; r < k; r++) {           // k <= 16 <= W, so k different lanes exist
+            tau = __reduce_max_sync(gmask, v);
             if (r + 1 < k) {
-                const unsigned int bal = __ballot_sync(0xffffffffu, v == tau);
+                const unsigned int bal = __ballot_sync(gmask, v == tau) & gmask;
                 if (lane == __ffs(bal) - 1) v = 0u;
             }
         }
         int nh = 0;
 #pragma unroll
-        for (int i = 0; i < 8; i++) {
+        for (int i = 0; i < NV; i++) {
             if (i < ni) {
                 // a slab beyond the width has tv == 0 and can only pass when tau == 0; keep it out
-                const bool is_hot = tv[i] >= tau && (lane + 32 * i) < nth;
-                const unsigned int bal = __ballot_sync(0xffffffffu, is_hot);
-                if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(lane + 32 * i);
+                const bool is_hot = tv[i] >= tau && (sl + W * i) < nth;
+                const unsigned int bal = (__ballot_sync(gmask, is_hot) & gmask) >> (W == 32 ? 0 : 16 * sub);
+                if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(sl + W * i);
                 nh += __popc(bal);
             }
         }
-        __syncwarp();
-        // (b) candidates: eight slabs per round, a lane takes 8 consecutive channels of one slab, so that the
-        // loads of a round are all in flight together
-        int n = 0;  // warp-uniform count
-        for (int base = 0; base < nh; base += 8) {
-            const int hi = base + (lane >> 2);
+        __syncwarp(gmask);
+        // (b) candidates: W/4 slabs per round, a lane takes 8 consecutive channels of one slab, so that the loads
+        // of a round are all in flight together
+        int n = 0;  // uniform over the token's lanes
+        for (int base = 0; base < nh; base += W / 4) {
+            const int hi = base + (sl >> 2);
             const bool act = hi < nh;
-            const int c0 = act ? (int)hot[hi] * 32 + (lane & 3) * 8 : 0;
+            const int c0 = act ? (int)hot[hi] * 32 + (sl & 3) * 8 : 0;
             uint4 xw = make_uint4(0u, 0u, 0u, 0u), rw = xw;
             uint32_t cf = 0u;
             if (act) {
@@ -838,15 +847,15 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
 #pragma unroll
             for (int i = 0; i < 8; i++) cnt += ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? 1 : 0;
             if (!act) cnt = 0;
-            // exclusive prefix of the per-lane counts
+            // exclusive prefix of the per-lane counts within the token's lanes
             int incl = cnt;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += up;
+            for (int o = 1; o < W; o <<= 1) {
+                const int up = __shfl_up_sync(gmask, incl, o, W);
+                if (sl >= o) incl += up;
             }
             int pos = n + incl - cnt;
-            if (act) {
+            if (cnt) {
 #pragma unroll
                 for (int i = 0; i < 8; i++) {
                     const unsigned int key = __float_as_uint(e[i]) & 0x7fffffffu;
@@ -859,12 +868,12 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
                     }
                 }
             }
-            n += __shfl_sync(0xffffffffu, incl, 31);
+            n += __shfl_sync(gmask, incl, W - 1, W);
         }
-        __syncwarp();
+        __syncwarp(gmask);
         // (c) exact ranking
         if (n <= kOutCap) {
-            for (int x = lane; x < n; x += 32) {
+            for (int x = sl; x < n; x += W) {
                 const unsigned long long mine = cand[x];
                 int rk = 0;
                 for (int y = 0; y < n; y++) rk += (cand[y] > mine) ? 1 : 0;
@@ -875,31 +884,31 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
             for (int r = 0; r < k; r++) {
                 unsigned long long best = 0ull;
                 float beste = 0.f;
-                for (int c = lane; c < d; c += 32) {
+                for (int c = sl; c < d; c += W) {
                     const float e = residual(c);
                     const unsigned long long comp =
                         ((unsigned long long)(__float_as_uint(e) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
                     // a composite is 0 only for |e| == 0 at channel 65535, which d <= 8192 excludes
                     if (comp < prev && comp > best) { best = comp; beste = e; }
                 }
-                for (int o = 16; o > 0; o >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-                    const float othere = __shfl_xor_sync(0xffffffffu, beste, o);
+                for (int o = W / 2; o > 0; o >>= 1) {
+                    const unsigned long long other = __shfl_xor_sync(gmask, best, o, W);
+                    const float othere = __shfl_xor_sync(gmask, beste, o, W);
                     if (other > best) { best = other; beste = othere; }
                 }
-                if (lane == 0) { sel[r] = best; sele[r] = beste; }
+                if (sl == 0) { sel[r] = best; sele[r] = beste; }
                 prev = best;
             }
         }
-        __syncwarp();
+        __syncwarp(gmask);
         // (d) outlier fields in channel order, dense codes at those channels cleared
-        if (lane < k) {
-            const int c = 0xffff - (int)(sel[lane] & 0xffffull);
+        if (sl < k) {
+            const int c = 0xffff - (int)(sel[sl] & 0xffffull);
             if (c < d) {
                 int pos = 0;
                 for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
                 unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
-                const uint32_t hv = float_to_half_bits_sat(sele[lane]);
+                const uint32_t hv = float_to_half_bits_sat(sele[sl]);
                 oidx[pos] = (unsigned short)c;
                 oidx[k + pos] = (unsigned short)hv;
                 if (p.X_hat) {
@@ -919,7 +928,7 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
                 if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
             }
         }
-        __syncwarp();
+        __syncwarp(gmask);
     }
 }
 
@@ -1250,13 +1259,21 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != RAC_OK) return rc;
-    long long blocks = (p.T + kOutWarps - 1) / kOutWarps;
+    // a warp per token; RAC_OUT_HALF=1 packs two tokens into a warp (16 lanes each; measured the same speed: the
+    // pass is bound by scattered 32-byte reads, not by issue slots)
+    const bool half = getenv("RAC_OUT_HALF") != nullptr;
+    const int tpw = half ? 2 : 1;
+    long long blocks = (p.T + kOutWarps * tpw - 1) / (kOutWarps * tpw);
     if (blocks > (long long)di.sms * 8) blocks = (long long)di.sms * 8;
+#define RAC_OUT(B)                                                                           \
+    if (half) outlier_kernel<B, 16><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p);     \
+    else outlier_kernel<B, 32><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p)
     switch (g.bits) {
-        case 4: outlier_kernel<4><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); break;
-        case 3: outlier_kernel<3><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); break;
-        case 2: outlier_kernel<2><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); break;
+        case 4: RAC_OUT(4); break;
+        case 3: RAC_OUT(3); break;
+        case 2: RAC_OUT(2); break;
     }
+#undef RAC_OUT
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
