@@ -33,9 +33,15 @@
  *     saturating at +-65504;
  *   - zero variance means centred Sxx <= 1e-12, or a slope that binary16 cannot
  *     hold (|Sxy| >= 65504*Sxx), or no reference at all;
- *   - the quantiser step is a static per-channel table (two rows: tokens with a
- *     reference, tokens coded directly) instead of Eq. 8's per-group dynamic
- *     scale, so dense values can clip; step 0 means "code 0";
+ *   - scale_mode 0 (the graded variant): the quantiser step is a static
+ *     per-channel table (two rows: tokens with a reference, tokens coded
+ *     directly) instead of Eq. 8's per-group dynamic scale, so dense values can
+ *     clip; step 0 means "code 0";
+ *   - scale_mode 1 (Eq. 8 as printed): per (token, group) scale
+ *     s = RoundUp_binary16(max|E^d| / Qmax), carried in the record; an all-zero
+ *     group carries scale 0 and codes 0 (the "zero marker"); no dense clipping;
+ *     the scale, its reciprocal and the scaled value are binary32 operations
+ *     (max / Qmax, 1 / s, e * (1/s)) because they decide codes;
  *   - outliers are the k largest |e| per TOKEN (not per group), ranked on the
  *     fp32 bit pattern of |e|, ties to the lower channel, stored with u16
  *     absolute channel indices in ascending order;
@@ -48,6 +54,7 @@
  *
  * Wire record of one token (all little endian), records back to back:
  *   coef    J  x u32   binary16 alpha in bits 0..15, binary16 beta in bits 16..31
+ *   scale   J  x u16   binary16, scale_mode 1 only, padded to a multiple of 4 bytes
  *   codes   d*b/8 B    code of channel c occupies stream bits [c*b, c*b+b),
  *                      stream bit n is bit (n%8) of byte (n/8); two's complement
  *   out_idx k  x u16   ascending
@@ -140,10 +147,16 @@ uint16_t orc_f64_to_f16_up(double x) {
 /* record geometry                                                     */
 /* ------------------------------------------------------------------ */
 
-int64_t orc_record_bytes(int d, int group, int bits, int topk) {
-    int64_t raw = 4 * (int64_t)(d / group) + ((int64_t)d * bits) / 8 + 4 * (int64_t)topk;
+static int64_t scale_bytes(int d, int group, int scale_mode) {
+    return scale_mode == 1 ? (2 * (int64_t)(d / group) + 3) / 4 * 4 : 0;
+}
+
+int64_t orc_record_bytes_mode(int d, int group, int bits, int topk, int scale_mode) {
+    int64_t raw = 4 * (int64_t)(d / group) + scale_bytes(d, group, scale_mode) + ((int64_t)d * bits) / 8 + 4 * (int64_t)topk;
     return (raw + 15) / 16 * 16;
 }
+
+int64_t orc_record_bytes(int d, int group, int bits, int topk) { return orc_record_bytes_mode(d, group, bits, topk, 0); }
 
 static int cfg_ok(int d, int group, int bits, int topk) {
     if (d <= 0 || group <= 0 || d % group) return 0;
@@ -255,7 +268,7 @@ static float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi
  *              and the scaled value v[T,d] the rounding decision was taken on.
  * returns 0, or -1 bad configuration, -2 ref_row out of range.
  */
-int orc_encode(int d, int group, int bits, int topk,
+int orc_encode(int d, int group, int bits, int topk, int scale_mode,
                const uint16_t *X, int64_t T,
                const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
                const uint16_t *gain, const uint16_t *bias,
@@ -265,9 +278,11 @@ int orc_encode(int d, int group, int bits, int topk,
                double *diag_alpha, double *diag_beta, double *diag_hbar, double *diag_rbar,
                float *diag_e, float *diag_v, int nthreads) {
     if (!cfg_ok(d, group, bits, topk)) return -1;
+    if (scale_mode != 0 && scale_mode != 1) return -1;
     if ((gain == NULL) != (bias == NULL)) return -1;
     const int J = d / group;
-    const int64_t rec = orc_record_bytes(d, group, bits, topk);
+    const int64_t rec = orc_record_bytes_mode(d, group, bits, topk, scale_mode);
+    const int64_t sbytes = scale_bytes(d, group, scale_mode);
     const int qmax = (1 << (bits - 1)) - 1;
     int err = 0;
     if (nthreads < 1) nthreads = 1;
@@ -282,7 +297,8 @@ int orc_encode(int d, int group, int bits, int topk,
             uint8_t *recp = payload + t * rec;
             memset(recp, 0, rec);
             uint32_t *coef = (uint32_t *)recp;
-            uint8_t *codes = recp + 4 * J;
+            uint8_t *scales = recp + 4 * J;
+            uint8_t *codes = scales + sbytes;
             uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             uint8_t *oval = oidx + 2 * topk;
 
@@ -338,19 +354,45 @@ int orc_encode(int d, int group, int bits, int topk,
                     n++;
                 }
             }
-            /* Eq. 8 with the static table, then packing */
-            const float *st = step + (has_ref ? 0 : d);
-            const float *ist = inv_step + (has_ref ? 0 : d);
-            for (int c = 0; c < d; c++) {
-                int q = 0;
-                float v = 0.0f;
-                if (st[c] != 0.0f && !is_out[c]) {
-                    v = e[c] * ist[c];
-                    q = (int)rintf(clampf(v, (float)-qmax, (float)qmax));
+            if (scale_mode == 0) {
+                /* Eq. 8 with the static table, then packing */
+                const float *st = step + (has_ref ? 0 : d);
+                const float *ist = inv_step + (has_ref ? 0 : d);
+                for (int c = 0; c < d; c++) {
+                    int q = 0;
+                    float v = 0.0f;
+                    if (st[c] != 0.0f && !is_out[c]) {
+                        v = e[c] * ist[c];
+                        q = (int)rintf(clampf(v, (float)-qmax, (float)qmax));
+                    }
+                    if (diag_v) diag_v[t * (int64_t)d + c] = v;
+                    if (diag_e) diag_e[t * (int64_t)d + c] = e[c];
+                    put_code(codes, c, bits, q);
                 }
-                if (diag_v) diag_v[t * (int64_t)d + c] = v;
-                if (diag_e) diag_e[t * (int64_t)d + c] = e[c];
-                put_code(codes, c, bits, q);
+            } else {
+                /* Eq. 8 as printed: scale of the group from its dense values, rounded UP in the wire
+                 * format so that nothing clips; an all-zero group carries scale 0 and codes 0 */
+                for (int j = 0; j < J; j++) {
+                    float m = 0.0f;
+                    for (int c = j * group; c < (j + 1) * group; c++)
+                        if (!is_out[c]) m = fmaxf(m, fabsf(e[c]));
+                    float s_star = m / (float)qmax;
+                    uint16_t s16 = orc_f64_to_f16_up((double)s_star);
+                    float sc = orc_f16_to_f32(s16);
+                    float isc = sc != 0.0f ? 1.0f / sc : 0.0f;
+                    memcpy(scales + 2 * j, &s16, 2);
+                    for (int c = j * group; c < (j + 1) * group; c++) {
+                        int q = 0;
+                        float v = 0.0f;
+                        if (!is_out[c]) {
+                            v = e[c] * isc;
+                            q = (int)rintf(clampf(v, (float)-qmax, (float)qmax));
+                        }
+                        if (diag_v) diag_v[t * (int64_t)d + c] = v;
+                        if (diag_e) diag_e[t * (int64_t)d + c] = e[c];
+                        put_code(codes, c, bits, q);
+                    }
+                }
             }
         }
         free(h); free(r); free(e); free(is_out);
@@ -365,15 +407,17 @@ int orc_encode(int d, int group, int bits, int topk,
 /* X_hat bf16[T,d] out.  status (optional, one word) gets bit 1 when a reserved
  * code -2^(b-1) was seen.  returns 0, -1, -2 as orc_encode; -3 when an outlier
  * index is >= d. */
-int orc_reconstruct(int d, int group, int bits, int topk,
+int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode,
                     const uint8_t *payload, int64_t T,
                     const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
                     const uint16_t *gain, const uint16_t *bias,
                     const float *step, uint16_t *X_hat, uint32_t *status, int nthreads) {
     if (!cfg_ok(d, group, bits, topk)) return -1;
     if ((gain == NULL) != (bias == NULL)) return -1;
+    if (scale_mode != 0 && scale_mode != 1) return -1;
     const int J = d / group;
-    const int64_t rec = orc_record_bytes(d, group, bits, topk);
+    const int64_t rec = orc_record_bytes_mode(d, group, bits, topk, scale_mode);
+    const int64_t sbytes = scale_bytes(d, group, scale_mode);
     int err = 0;
     uint32_t st_word = 0;
     if (nthreads < 1) nthreads = 1;
@@ -384,7 +428,8 @@ int orc_reconstruct(int d, int group, int bits, int topk,
 #pragma omp for schedule(static)
         for (int64_t t = 0; t < T; t++) {
             const uint8_t *recp = payload + t * rec;
-            const uint8_t *codes = recp + 4 * J;
+            const uint8_t *scales = recp + 4 * J;
+            const uint8_t *codes = scales + sbytes;
             const uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             const uint8_t *oval = oidx + 2 * topk;
             int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
@@ -393,14 +438,17 @@ int orc_reconstruct(int d, int group, int bits, int topk,
                 err = -2;
                 continue;
             }
-            const float *st = step + (has_ref ? 0 : d);
+            const float *st = scale_mode == 0 ? step + (has_ref ? 0 : d) : NULL;
             for (int c = 0; c < d; c++) {
                 int q = get_code(codes, c, bits);
                 if (q == -(1 << (bits - 1))) {
 #pragma omp atomic
                     st_word |= 2u;
                 }
-                eh[c] = (float)q * st[c];
+                float sc;
+                if (scale_mode == 0) sc = st[c];
+                else { uint16_t s16; memcpy(&s16, scales + 2 * (c / group), 2); sc = orc_f16_to_f32(s16); }
+                eh[c] = (float)q * sc;
             }
             for (int n = 0; n < topk; n++) {
                 uint16_t ci, hv;

@@ -342,3 +342,76 @@ def test_calibrated_step_is_three_sigma_rounded_up(orc):
     assert np.all(step[0] <= want * (1 + 2e-3) + np.spacing(step[0].astype(np.float16)).astype(np.float64))
     assert np.array_equal(inv[0], (np.float32(1) / step[0]).astype(np.float32))
     assert not step[1].any() and not inv[1].any()
+
+
+# ------------------------------------------------------------------ Eq. 8 as printed: dynamic per-group scale
+@pytest.mark.parametrize("bits,topk", [(4, 0), (3, 0), (2, 0), (4, 8)])
+def test_dynamic_scale_never_clips_and_rounds_up(orc, bits, topk):
+    d, g, T = 512, 64, 40
+    J = d // g
+    gen = synth.generator(80 + bits)
+    X = synth.activations(T, d, synth.channel_scale(d, 6), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    Xb, Rb = synth.bf16_bits(X), synth.bf16_bits(R)
+    payload = orc.encode(d, g, bits, topk, Xb, ref_base=Rb, scale_mode=1)
+    assert payload.size == T * orc.record_bytes(d, g, bits, topk, 1)
+    xh = orc.reconstruct(d, g, bits, topk, payload, T, ref_base=Rb, scale_mode=1)
+    coef, codes, oi, ov, scale = orc.split_payload(payload, T, d, g, bits, topk, 1)
+    qmax = (1 << (bits - 1)) - 1
+    h = orc.bf16_to_f32(Xb).astype(np.float64)
+    r = orc.bf16_to_f32(Rb).astype(np.float64)
+    alpha = np.repeat(f16(coef & 0xffff), g, axis=1)
+    beta = np.repeat(f16(coef >> 16), g, axis=1)
+    e = h - (alpha * r + beta)                         # Eq. 7 from the wire coefficients
+    q = np.stack([orc.unpack_codes(codes[t], d, bits) for t in range(T)])
+    is_out = np.zeros((T, d), bool)
+    if topk:
+        is_out[np.arange(T)[:, None], oi.astype(np.int64)] = True
+        assert np.all(q[is_out] == 0)
+    s = f16(scale)                                     # [T, J]
+    s_full = np.repeat(s, g, axis=1)
+    dense_max = np.where(is_out, 0, np.abs(e)).reshape(T, J, g).max(axis=2)
+    # RoundUp_wire: the stored scale is >= max|E^d|/Qmax (so nothing clips) and the binary16 below it is not
+    want = dense_max / qmax
+    assert np.all(s >= want * (1 - 1e-6))
+    below = np.nextafter(s.astype(np.float16), np.float16(-np.inf)).astype(np.float64)
+    assert np.all((below < want * (1 + 1e-6)) | (s == 0))
+    # Eq. 11: every dense value within half a scale step, no exceptions, and no reserved code
+    e_hat = q * s_full
+    assert q.min() >= -qmax and q.max() <= qmax
+    assert np.all(np.abs(e - e_hat)[~is_out] <= 0.5 * s_full[~is_out] * (1 + 1e-5) + 1e-12)
+    # the largest dense magnitude of every group sits at the end of the range
+    amax = np.abs(q).reshape(T, J, g).max(axis=2)
+    assert np.all((amax == qmax) | (dense_max == 0))
+    # Eq. 10 with the receiver's view
+    if topk:
+        e_hat[np.arange(T)[:, None], oi.astype(np.int64)] = f16(ov)
+    x_hat = orc.bf16_to_f32(xh).astype(np.float64)
+    assert np.all(np.abs((h - x_hat) - (e - e_hat)) <= np.abs(x_hat) * 2.0 ** -8 + 1e-30)
+    # Eq. 12: the residual range is far below the direct-coding range on this workload
+    direct_max = np.abs(h - h.reshape(T, J, g).mean(axis=2).repeat(g, axis=1)).reshape(T, J, g).max(axis=2)
+    assert np.median(dense_max / direct_max) < 0.5
+
+
+def test_dynamic_scale_zero_group_marker_and_identity(orc):
+    d, g, T = 256, 64, 6
+    gen = synth.generator(90)
+    X = synth.activations(T, d, synth.channel_scale(d, 7), gen)
+    Xb = synth.bf16_bits(X)
+    payload = orc.encode(d, g, 4, 0, Xb, ref_base=Xb, scale_mode=1)       # reference == X: residual zero everywhere
+    coef, codes, _, _, scale = orc.split_payload(payload, T, d, g, 4, 0, 1)
+    assert not scale.any() and not codes.any() and np.all(coef == 0x3c00)
+    assert np.array_equal(orc.reconstruct(d, g, 4, 0, payload, T, ref_base=Xb, scale_mode=1), Xb)
+    # 4-bit values stay 25 % of raw; scales add 2 bytes per group
+    assert orc.record_bytes(4096, 128, 4, 0, 1) - orc.record_bytes(4096, 128, 4, 0, 0) == 64
+    # one group with a single non-zero residual: its scale is that value / Qmax rounded up, code +-Qmax
+    row = np.zeros((1, d), np.float32)
+    row[0, 5] = 3.0
+    row[0, 6] = -3.0                                                     # zero mean: beta = 0 with no reference
+    p2 = orc.encode(d, g, 4, 0, bits_of(row), scale_mode=1)
+    coef, codes, _, _, scale = orc.split_payload(p2, 1, d, g, 4, 0, 1)
+    q = orc.unpack_codes(codes[0], d, 4)
+    assert q[5] == 7 and q[6] == -7 and np.count_nonzero(q) == 2
+    assert scale[0, 0] == np.float16(np.nextafter(np.float16(3.0 / 7), np.float16(1))).view(np.uint16) or \
+        f16(scale[0, :1])[0] >= 3.0 / 7
+    assert not scale[0, 1:].any()
