@@ -26,6 +26,7 @@
  *
  * Wire record of one token (little endian), records back to back in `payload`:
  *     coef    J x u32      binary16 alpha in bits 0..15, binary16 beta in 16..31,  J = d/group
+ *     scale   J x u16      binary16 group scales, scale_mode 1 only, padded to a multiple of 4 bytes
  *     codes   d*bits/8 B   code of channel c in stream bits [c*bits, c*bits+bits); stream bit n is
  *                          bit n%8 of byte n/8; two's complement; -2^(bits-1) is never produced
  *     out_idx topk x u16   channel indices, ascending
@@ -65,7 +66,10 @@ extern "C" {
  *   bits    code width: 2, 3 or 4            (Qmax = 2^(bits-1) - 1, Eq. 8a)
  *   topk    outliers per token kept as binary16, 0..16 (Sec. IV-C "Outlier Metadata"; per token here)
  *   coef_fmt   0 = binary16 pair (the only format)
- *   scale_mode 0 = static per-channel step table (the only mode)
+ *   scale_mode 0 = static per-channel step table `step`/`inv_step` (calibrated clip; dense values may clip)
+ *              1 = Eq. 8 as printed: per (token, group) scale s = RoundUp_binary16(max|E| / Qmax) carried in the
+ *                  record (J x u16 after `coef`, padded to 4 bytes), scale 0 = all-zero group; nothing clips;
+ *                  `step` and `inv_step` are not read and may be NULL; only with topk == 0
  *   flags   must be 0 */
 typedef struct {
     int32_t d, group, bits, topk, coef_fmt, scale_mode, flags;

@@ -31,7 +31,11 @@ static bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     if (!cfg) return RAC_EINVAL;
     if (cfg->d <= 0 || cfg->group <= 0 || cfg->topk < 0 || cfg->bits <= 0) return RAC_EINVAL;
-    if (cfg->coef_fmt != 0 || cfg->scale_mode != 0 || cfg->flags != 0) return RAC_EUNSUPPORTED;
+    if (cfg->coef_fmt != 0 || cfg->flags != 0) return RAC_EUNSUPPORTED;
+    if (cfg->scale_mode != 0 && cfg->scale_mode != 1) return RAC_EUNSUPPORTED;
+    // Eq. 8 takes the scale from the dense values, i.e. after the outliers are known; the outlier pass runs
+    // after the streaming pass here, so the per-group scale is offered without outliers only
+    if (cfg->scale_mode == 1 && cfg->topk != 0) return RAC_EUNSUPPORTED;
     if (cfg->d % cfg->group) return RAC_EINVAL;
     if (cfg->d % 32 || cfg->d > 8192) return RAC_EUNSUPPORTED;
     if (!is_pow2(cfg->group) || cfg->group < 32 || cfg->group > 1024) return RAC_EUNSUPPORTED;
@@ -45,7 +49,9 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     g->lpg = cfg->group / 32;
     g->nthreads = ((cfg->d / 32) + 31) / 32 * 32;
     g->code_bytes = cfg->d * cfg->bits / 8;
-    int raw = 4 * g->J + g->code_bytes + 4 * cfg->topk;
+    g->scale_mode = cfg->scale_mode;
+    g->codes_off = 4 * g->J + (cfg->scale_mode == 1 ? (2 * g->J + 3) / 4 * 4 : 0);
+    int raw = g->codes_off + g->code_bytes + 4 * cfg->topk;
     g->rec = (raw + 15) / 16 * 16;
     return RAC_OK;
 }
@@ -70,7 +76,7 @@ struct CodecParams {
     long long T;
     long long ref_rows;
     // geometry
-    int d, J, lpg, lpg_shift, topk, rec, code_bytes, stages;
+    int d, J, lpg, lpg_shift, topk, rec, code_bytes, codes_off, stages;
     float inv_group;
 };
 
@@ -465,7 +471,9 @@ __host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages, boo
     return s;
 }
 
-template <int BITS, bool TOPK, bool XHAT, int MINB>
+// DYN: Eq. 8 as printed -- the scale of a group is the largest dense |e| of the group over Qmax, rounded up to
+// binary16 and written into the record; no step table is read.
+template <int BITS, bool TOPK, bool XHAT, bool DYN, int MINB>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -508,10 +516,15 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     }
     {
         // padding words of the records are written once and never touched again
-        const int raw = 4 * p.J + p.code_bytes + 4 * p.topk;
+        const int raw = p.codes_off + p.code_bytes + 4 * p.topk;
         for (int s = 0; s < 2 * S; s++)
             for (int o = raw + 4 * tid; o < p.rec; o += 4 * nt)
                 *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * p.rec + o) = 0u;
+        // an odd number of binary16 scales leaves two bytes of padding before the codes: zero that word once
+        if (DYN && tid == 0 && (p.J & 1))
+            for (int s = 0; s < 2 * S; s++)
+                *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * p.rec +
+                                              p.codes_off - 4) = 0u;
     }
     __syncthreads();
     if (tid == 0)
@@ -565,21 +578,52 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 
             // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
             if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
-            const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
-            const float *step_tab = p.step + (has_ref ? 0 : d);
+            const float *inv_tab = DYN ? nullptr : p.inv_step + (has_ref ? 0 : d);
+            const float *step_tab = DYN ? nullptr : p.step + (has_ref ? 0 : d);
+            u64 dyn_inv2 = 0ull, dyn_s2 = 0ull;
+            if (DYN) {
+                // largest |e| of the group (this thread's 32 channels, then the group's lanes), in binary32
+                float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 16; i++) {
+                    float e0, e1;
+                    unpack2(psub(x2[i], pfma(a2, r2[i], b2)), e0, e1);
+                    m0 = fmaxf(m0, fabsf(e0));
+                    m1 = fmaxf(m1, fabsf(e1));
+                }
+                float m = fmaxf(m0, m1);
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1)
+                    if (p.lpg > o) m = fmaxf(m, __shfl_xor_sync(group_mask, m, o));
+                // s = RoundUp_binary16(m / Qmax): round to nearest, then one step up if that fell short
+                const float s_star = __fdiv_rn(m, qmax);
+                uint32_t s16 = float_to_half_bits_sat(s_star);
+                if (half_bits_to_float(s16) < s_star && s16 < 0x7bffu) s16++;
+                const float sc = half_bits_to_float(s16);
+                const float isc = sc != 0.f ? __fdiv_rn(1.0f, sc) : 0.f;
+                dyn_inv2 = pack2(isc, isc);
+                dyn_s2 = pack2(sc, sc);
+                if ((lane & (p.lpg - 1)) == 0)
+                    reinterpret_cast<unsigned short *>(rec + 4 * p.J)[tid >> p.lpg_shift] = (unsigned short)s16;
+            }
             uint32_t words[4];
             float tmax = 0.f;
 #pragma unroll
             for (int j = 0; j < 4; j++) {
                 const int c = (int)(off[j] >> 1);
-                const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
-                const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
-                const u64 inv2[4] = {pack2(iv0.x, iv0.y), pack2(iv0.z, iv0.w), pack2(iv1.x, iv1.y), pack2(iv1.z, iv1.w)};
-                u64 st2[4] = {0ull, 0ull, 0ull, 0ull};
-                if (XHAT) {
-                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(step_tab + c));
-                    const float4 s1 = __ldg(reinterpret_cast<const float4 *>(step_tab + c + 4));
-                    st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
+                u64 inv2[4], st2[4] = {0ull, 0ull, 0ull, 0ull};
+                if (DYN) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) { inv2[i] = dyn_inv2; st2[i] = dyn_s2; }
+                } else {
+                    const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
+                    const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
+                    inv2[0] = pack2(iv0.x, iv0.y); inv2[1] = pack2(iv0.z, iv0.w); inv2[2] = pack2(iv1.x, iv1.y); inv2[3] = pack2(iv1.z, iv1.w);
+                    if (XHAT) {
+                        const float4 s0 = __ldg(reinterpret_cast<const float4 *>(step_tab + c));
+                        const float4 s1 = __ldg(reinterpret_cast<const float4 *>(step_tab + c + 4));
+                        st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
+                    }
                 }
                 float ev[8];
                 uint32_t xh[4];
@@ -641,7 +685,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                 }
             }
             rot_right4(words, rot);  // words[q] is now the code word of piece q
-            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + 4 * p.J) + tid * BITS;
+            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + p.codes_off) + tid * BITS;
             if (BITS == 4) {
                 cw[0] = words[0]; cw[1] = words[1]; cw[2] = words[2]; cw[3] = words[3];
             } else if (BITS == 3) {
@@ -907,7 +951,7 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
             if (c < d) {
                 int pos = 0;
                 for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
-                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + p.codes_off + p.code_bytes);
                 const uint32_t hv = float_to_half_bits_sat(sele[sl]);
                 oidx[pos] = (unsigned short)c;
                 oidx[k + pos] = (unsigned short)hv;
@@ -922,7 +966,7 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
                     const float rt = __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16));
                     p.X_hat[t * d + c] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(rt, half_bits_to_float(hv))));
                 }
-                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
+                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + p.codes_off);
                 const int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
                 atomicAnd(&codes32[wd], ~(cmask << sh));
                 if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
@@ -969,7 +1013,8 @@ __global__ void calib_finalize_kernel(const float *partial, int nblocks, int d, 
 // into an output row in shared memory, patches the outliers it owns, and the row leaves as one bulk store.
 // The step table row of referenced tokens lives in registers for the whole kernel (a thread always owns
 // the same channels); direct tokens read row 1 through L1.
-template <int BITS, int KT>
+// DYN: the step of a channel is its group's binary16 scale from the record (Eq. 8 as printed), not a table.
+template <int BITS, int KT, bool DYN>
 __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x;
@@ -1020,7 +1065,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
 #pragma unroll
     for (int j = 0; j < 4; j++) {
         float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
-        if (valid) {
+        if (valid && !DYN) {
             s0 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1)));
             s1 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1) + 4));
         }
@@ -1055,8 +1100,13 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
             const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
             const u64 a2 = pack2(a, a), b2 = pack2(b, b);
+            u64 dyn_s2 = 0ull;
+            if (DYN) {
+                const float sc = half_bits_to_float(reinterpret_cast<const unsigned short *>(rec + 4 * p.J)[tid >> p.lpg_shift]);
+                dyn_s2 = pack2(sc, sc);
+            }
             // code words of the four pieces, in piece order, then rotated into slot order
-            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + 4 * p.J) + tid * BITS;
+            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + p.codes_off) + tid * BITS;
             uint32_t words[4];
             if (BITS == 4) {
                 words[0] = cw[0]; words[1] = cw[1]; words[2] = cw[2]; words[3] = cw[3];
@@ -1085,14 +1135,20 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
                 u64 r2[4], st2[4];
                 if (has_ref) {
                     load_ref_slot(rs + off[j], p.gain, p.bias, c, r2);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[i] = 0ull;
+                }
+                if (DYN) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) st2[i] = dyn_s2;
+                } else if (has_ref) {
 #pragma unroll
                     for (int i = 0; i < 4; i++) st2[i] = st0[4 * j + i];
                 } else {
                     const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c));
                     const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c + 4));
                     st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
-#pragma unroll
-                    for (int i = 0; i < 4; i++) r2[i] = 0ull;
                 }
                 const uint32_t w = words[j];
                 uint32_t o[4];
@@ -1110,7 +1166,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             }
             if (KT > 0) {
                 // outliers whose channel this thread owns replace what the dense pass wrote
-                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + p.codes_off + p.code_bytes);
                 const unsigned short *oval = oidx + p.topk;
 #pragma unroll
                 for (int n = 0; n < KT; n++) {
@@ -1130,7 +1186,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             }
         }
         if (KT > 0 && tid == 0) {
-            const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
+            const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + p.codes_off + p.code_bytes);
             bool bad = false;
             for (int n = 0; n < p.topk; n++) bad |= oidx[n] >= d;
             if (bad && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
@@ -1222,6 +1278,7 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     p->topk = g.topk;
     p->rec = g.rec;
     p->code_bytes = g.code_bytes;
+    p->codes_off = g.codes_off;
     p->inv_group = 1.0f / (float)g.group;
     return RAC_OK;
 }
@@ -1242,17 +1299,19 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     WsSmem L = ws_smem_layout(g.d, g.rec, p.stages, topk);
     // With x_hat the kernel reads both step tables every token; at four CTAs per SM the shared-memory carve-out
     // leaves too little L1 for them, so that variant runs three CTAs per SM at 128 registers.
-    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
+    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && (!p.X_hat || g.scale_mode == 1) && !getenv("RAC_ENC_WIDE");
     int rc = RAC_EUNSUPPORTED;
-#define RAC_ENC2(B, K, X)                                                                                          \
-    (tight ? launch_persistent(encode_ws_kernel<B, K, X, 4>, p, g.nthreads, L.total, max_ctas, stream)            \
-           : launch_persistent(encode_ws_kernel<B, K, X, 2>, p, g.nthreads, L.total, max_ctas, stream))
+#define RAC_ENC3(B, K, X, D)                                                                                       \
+    (tight ? launch_persistent(encode_ws_kernel<B, K, X, D, 4>, p, g.nthreads, L.total, max_ctas, stream)         \
+           : launch_persistent(encode_ws_kernel<B, K, X, D, 2>, p, g.nthreads, L.total, max_ctas, stream))
+#define RAC_ENC2(B, K, X) (g.scale_mode == 1 ? RAC_ENC3(B, false, X, true) : RAC_ENC3(B, K, X, false))
 #define RAC_ENC(B, K) (p.X_hat ? RAC_ENC2(B, K, true) : RAC_ENC2(B, K, false))
     switch (g.bits) {
         case 4: rc = topk ? RAC_ENC(4, true) : RAC_ENC(4, false); break;
         case 3: rc = topk ? RAC_ENC(3, true) : RAC_ENC(3, false); break;
         case 2: rc = topk ? RAC_ENC(2, true) : RAC_ENC(2, false); break;
     }
+#undef RAC_ENC3
 #undef RAC_ENC2
 #undef RAC_ENC
     if (rc != RAC_OK || !topk) return rc;
@@ -1281,7 +1340,9 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
     p.stages = pick_stages(g.d, 2);
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
-#define RAC_DEC(B, K) launch_persistent(decode_kernel<B, K>, p, g.nthreads, L.total, p.T, stream)
+#define RAC_DEC(B, K)                                                                                  \
+    (g.scale_mode == 1 ? launch_persistent(decode_kernel<B, K, true>, p, g.nthreads, L.total, p.T, stream) \
+                       : launch_persistent(decode_kernel<B, K, false>, p, g.nthreads, L.total, p.T, stream))
     switch (g.bits * 100 + kt) {
         case 400: return RAC_DEC(4, 0);
         case 408: return RAC_DEC(4, 8);
@@ -1309,8 +1370,8 @@ static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64
     rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, gain, bias, dev_status);
     if (rc != RAC_OK) return rc;
     if (T == 0) return RAC_OK;
-    if (!payload || !X_hat || !step) return RAC_EINVAL;
-    if (!aligned16(payload) || !aligned16(X_hat) || !aligned16(step)) return RAC_EALIGN;
+    if (!payload || !X_hat || (!step && g.scale_mode == 0)) return RAC_EINVAL;
+    if (!aligned16(payload) || !aligned16(X_hat) || (step && !aligned16(step))) return RAC_EALIGN;
     p.payload = const_cast<uint8_t *>(static_cast<const uint8_t *>(payload));
     p.X_hat = static_cast<uint16_t *>(X_hat);
     p.step = step;
@@ -1368,8 +1429,9 @@ static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const
     rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, dev_status);
     if (rc != RAC_OK) return rc;
     if (T == 0) return RAC_OK;
-    if (!X || !payload || !step || !inv_step) return RAC_EINVAL;
-    if (!aligned16(X) || !aligned16(payload) || !aligned16(step) || !aligned16(inv_step)) return RAC_EALIGN;
+    if (!X || !payload) return RAC_EINVAL;
+    if (g.scale_mode == 0 && (!step || !inv_step)) return RAC_EINVAL;   // the static tables; mode 1 reads neither
+    if (!aligned16(X) || !aligned16(payload) || (step && !aligned16(step)) || (inv_step && !aligned16(inv_step))) return RAC_EALIGN;
     if (X_hat && !aligned16(X_hat)) return RAC_EALIGN;
     if (payload_cap < (size_t)g.rec * (size_t)T) return RAC_ESIZE;
     const size_t need = rac_encode_workspace_bytes(cfg, T);

@@ -142,6 +142,8 @@ struct Geometry {
     int lpg;        // lanes per group (group / 32)
     int nthreads;   // threads per CTA: one per 32 channels, rounded up to whole warps
     int code_bytes; // d*bits/8
+    int scale_mode; // 0: static per-channel step table, 1: per-group binary16 scale in the record (Eq. 8)
+    int codes_off;  // byte offset of the codes in a record: 4*J, plus the scales (2*J padded to 4) in mode 1
     int rec;        // record stride in bytes
 };
 int make_geometry(const rac_codec_cfg *cfg, Geometry *g);  // RAC_OK or an error

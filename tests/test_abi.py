@@ -40,6 +40,9 @@ def test_record_geometry_matches_the_wire_format(rac, orc):
         cfg = rac.CodecCfg(d, g, b, k)
         assert rac.rac_record_bytes(cfg) == orc.record_bytes(d, g, b, k)
         assert rac.rac_payload_bytes(cfg, 1000) == 1000 * orc.record_bytes(d, g, b, k)
+    for d, g, b in [(4096, 128, 4), (3584, 128, 3), (2080, 32, 4), (96, 32, 2)]:   # per-group scales in the record
+        assert rac.rac_record_bytes(rac.CodecCfg(d, g, b, 0, scale_mode=1)) == orc.record_bytes(d, g, b, 0, 1)
+    assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 4, 0, scale_mode=1)) == 2176 + 64
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 100, 4, 0)) == 0   # group does not divide d
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 5, 0)) == 0   # unsupported width
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 4, 17)) == 0

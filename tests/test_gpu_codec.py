@@ -334,3 +334,39 @@ def test_long_context_sampled(env):
         total += err.numel()
     frac_within = within / total
     assert frac_within > 0.98  # the rest is clipping by the static table (3 sigma) on direct and referenced tokens
+
+
+# --------------------------------------------------------------------------- Eq. 8 as printed: per-group scale in the record
+@pytest.mark.parametrize("d,g,bits,T", [
+    (4096, 128, 4, 257), (4096, 64, 3, 64), (3584, 128, 4, 64), (5120, 128, 2, 95), (96, 32, 4, 9), (2080, 32, 4, 33),
+])
+def test_dynamic_group_scale_matches_oracle(env, d, g, bits, T):
+    """scale_mode 1: no step table; the scale of each (token, group) travels in the record.  Same protocol as the
+    static mode; on top, nothing may clip (Eq. 11): every element within half a scale step."""
+    X, R, _, _ = prefill_inputs(env, T, d, g, seed=2000 + d + bits)
+    cfg = env.rac.CodecCfg(d, g, bits, 0, scale_mode=1)
+    assert env.rac.rac_record_bytes(cfg) == env.orc.record_bytes(d, g, bits, 0, 1)
+    rep, pay, xr = env.P.round_trip_case(cfg, X, ref_base=R)
+    print(rep)
+    coef, codes, _, _, scale = env.orc.split_payload(pay, T, d, g, bits, 0, 1)
+    s = scale.view(np.float16).astype(np.float64).repeat(g, axis=1)
+    h = X.float().cpu().numpy().astype(np.float64)
+    xh = xr.float().cpu().numpy().astype(np.float64)
+    # half a scale step from the quantiser, plus the bf16 rounding of the reconstruction (relative to ITS magnitude)
+    assert np.all(np.abs(h - xh) <= 0.5 * s * (1 + 1e-5) + 2.0 ** -8 * np.maximum(np.abs(h), np.abs(xh)) + 1e-12)
+    # direct tokens and the gain/bias reference go through the same path
+    rows = np.arange(T, dtype=np.int32)
+    rows[::3] = -1
+    env.P.round_trip_case(cfg, X, ref_base=R, ref_row=torch.from_numpy(rows).to(env.dev))
+
+
+def test_dynamic_group_scale_identity_and_rejections(env):
+    d, g, T = 1024, 128, 5
+    s = env.synth
+    X = s.activations(T, d, s.channel_scale(d, 33, env.dev), s.generator(33, env.dev))
+    cfg = env.rac.CodecCfg(d, g, 4, 0, scale_mode=1)
+    rep, pay, xr = env.P.round_trip_case(cfg, X, ref_base=X)
+    coef, codes, _, _, scale = env.orc.split_payload(pay, T, d, g, 4, 0, 1)
+    assert not scale.any() and not codes.any() and torch.equal(xr, X)        # zero-group marker everywhere
+    assert env.rac.rac_record_bytes(env.rac.CodecCfg(d, g, 4, 8, scale_mode=1)) == 0   # outliers: not in this mode
+    assert env.rac.rac_record_bytes(env.rac.CodecCfg(d, g, 4, 0, scale_mode=2)) == 0
