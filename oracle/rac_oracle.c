@@ -42,6 +42,13 @@
  *     group carries scale 0 and codes 0 (the "zero marker"); no dense clipping;
  *     the scale, its reciprocal and the scaled value are binary32 operations
  *     (max / Qmax, 1 / s, e * (1/s)) because they decide codes;
+ *   - still scale_mode 1, the rest of the quantiser family of Sec. IV-C: the
+ *     quantisation group g_q may differ from the alignment group g_a (g_q = d
+ *     is the decode mode: one scale per token), the code width may be 8, and
+ *     the outlier mask may pick the k_g largest |e| of every quantisation
+ *     group (ranked like the per-token form, ties to the lower channel),
+ *     serialised as one-byte in-group offsets in ascending order plus binary16
+ *     values, which needs g_q <= 256;
  *   - outliers are the k largest |e| per TOKEN (not per group), ranked on the
  *     fp32 bit pattern of |e|, ties to the lower channel, stored with u16
  *     absolute channel indices in ascending order;
@@ -59,6 +66,9 @@
  *                      stream bit n is bit (n%8) of byte (n/8); two's complement
  *   out_idx k  x u16   ascending
  *   out_val k  x u16   binary16
+ *   grp_off Jq*kg x u8 in-group offsets of the per-group outliers, ascending
+ *                      within a group, padded to a multiple of 2 bytes
+ *   grp_val Jq*kg x u16 binary16                     (Jq = d/g_q, scale has Jq entries)
  *   padding to a multiple of 16 bytes (zero)
  *
  * Parity status: the LS fit, residual identity, quantiser bounds, packing,
@@ -147,13 +157,21 @@ uint16_t orc_f64_to_f16_up(double x) {
 /* record geometry                                                     */
 /* ------------------------------------------------------------------ */
 
-static int64_t scale_bytes(int d, int group, int scale_mode) {
-    return scale_mode == 1 ? (2 * (int64_t)(d / group) + 3) / 4 * 4 : 0;
+static int64_t scale_bytes(int d, int qgroup, int scale_mode) {
+    return scale_mode == 1 ? (2 * (int64_t)(d / qgroup) + 3) / 4 * 4 : 0;
+}
+
+/* qgroup 0 means "same as group"; topk_group outliers per quantisation group */
+int64_t orc_record_bytes_ext(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group) {
+    if (qgroup == 0) qgroup = group;
+    int64_t ng = (int64_t)(d / qgroup) * topk_group;
+    int64_t raw = 4 * (int64_t)(d / group) + scale_bytes(d, qgroup, scale_mode) + ((int64_t)d * bits) / 8 + 4 * (int64_t)topk +
+                  (ng + 1) / 2 * 2 + 2 * ng;
+    return (raw + 15) / 16 * 16;
 }
 
 int64_t orc_record_bytes_mode(int d, int group, int bits, int topk, int scale_mode) {
-    int64_t raw = 4 * (int64_t)(d / group) + scale_bytes(d, group, scale_mode) + ((int64_t)d * bits) / 8 + 4 * (int64_t)topk;
-    return (raw + 15) / 16 * 16;
+    return orc_record_bytes_ext(d, group, bits, topk, scale_mode, 0, 0);
 }
 
 int64_t orc_record_bytes(int d, int group, int bits, int topk) { return orc_record_bytes_mode(d, group, bits, topk, 0); }
@@ -163,6 +181,17 @@ static int cfg_ok(int d, int group, int bits, int topk) {
     if (bits < 2 || bits > 8) return 0;
     if (((int64_t)d * bits) % 8) return 0;
     if (topk < 0 || topk > d || d > 65536) return 0;
+    return 1;
+}
+
+/* the quantisation group and the per-group outliers exist in scale_mode 1 only */
+static int qcfg_ok(int d, int group, int topk, int scale_mode, int qgroup, int topk_group) {
+    if (scale_mode != 0 && scale_mode != 1) return 0;
+    if (qgroup < 0 || topk_group < 0) return 0;
+    if (scale_mode == 0) return (qgroup == 0 || qgroup == group) && topk_group == 0;
+    if (qgroup == 0) qgroup = group;
+    if (d % qgroup) return 0;
+    if (topk_group && (topk || qgroup > 256 || topk_group > qgroup)) return 0;
     return 1;
 }
 
@@ -268,7 +297,7 @@ static float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi
  *              and the scaled value v[T,d] the rounding decision was taken on.
  * returns 0, or -1 bad configuration, -2 ref_row out of range.
  */
-int orc_encode(int d, int group, int bits, int topk, int scale_mode,
+int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group,
                const uint16_t *X, int64_t T,
                const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
                const uint16_t *gain, const uint16_t *bias,
@@ -278,11 +307,12 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode,
                double *diag_alpha, double *diag_beta, double *diag_hbar, double *diag_rbar,
                float *diag_e, float *diag_v, int nthreads) {
     if (!cfg_ok(d, group, bits, topk)) return -1;
-    if (scale_mode != 0 && scale_mode != 1) return -1;
+    if (!qcfg_ok(d, group, topk, scale_mode, qgroup, topk_group)) return -1;
     if ((gain == NULL) != (bias == NULL)) return -1;
-    const int J = d / group;
-    const int64_t rec = orc_record_bytes_mode(d, group, bits, topk, scale_mode);
-    const int64_t sbytes = scale_bytes(d, group, scale_mode);
+    if (qgroup == 0) qgroup = group;
+    const int J = d / group, Jq = d / qgroup;
+    const int64_t rec = orc_record_bytes_ext(d, group, bits, topk, scale_mode, qgroup, topk_group);
+    const int64_t sbytes = scale_bytes(d, qgroup, scale_mode);
     const int qmax = (1 << (bits - 1)) - 1;
     int err = 0;
     if (nthreads < 1) nthreads = 1;
@@ -301,6 +331,8 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode,
             uint8_t *codes = scales + sbytes;
             uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             uint8_t *oval = oidx + 2 * topk;
+            uint8_t *goff = oval + 2 * topk;
+            uint8_t *gval = goff + ((int64_t)Jq * topk_group + 1) / 2 * 2;
 
             for (int c = 0; c < d; c++) h[c] = orc_bf16_to_f32(X[t * (int64_t)d + c]);
             int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
@@ -354,6 +386,27 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode,
                     n++;
                 }
             }
+            /* per-group form of the mask (Sec. IV-C, "Outlier Metadata"): the k_g largest |e| of every
+             * quantisation group, in-group offsets in ascending order, values as binary16 */
+            for (int j = 0; j < Jq && topk_group; j++) {
+                for (int n = 0; n < topk_group; n++) {
+                    int best = -1; uint32_t bestkey = 0;
+                    for (int c = j * qgroup; c < (j + 1) * qgroup; c++) {
+                        if (is_out[c]) continue;
+                        uint32_t key = f32_to_bits(e[c]) & 0x7fffffffu;
+                        if (best < 0 || key > bestkey) { best = c; bestkey = key; }
+                    }
+                    is_out[best] = 1;
+                }
+                int n = 0;
+                for (int c = j * qgroup; c < (j + 1) * qgroup; c++) {
+                    if (!is_out[c]) continue;
+                    uint16_t hv = orc_f64_to_f16((double)clampf(e[c], -65504.0f, 65504.0f));
+                    goff[j * topk_group + n] = (uint8_t)(c - j * qgroup);
+                    memcpy(gval + 2 * (j * topk_group + n), &hv, 2);
+                    n++;
+                }
+            }
             if (scale_mode == 0) {
                 /* Eq. 8 with the static table, then packing */
                 const float *st = step + (has_ref ? 0 : d);
@@ -372,16 +425,16 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode,
             } else {
                 /* Eq. 8 as printed: scale of the group from its dense values, rounded UP in the wire
                  * format so that nothing clips; an all-zero group carries scale 0 and codes 0 */
-                for (int j = 0; j < J; j++) {
+                for (int j = 0; j < Jq; j++) {
                     float m = 0.0f;
-                    for (int c = j * group; c < (j + 1) * group; c++)
+                    for (int c = j * qgroup; c < (j + 1) * qgroup; c++)
                         if (!is_out[c]) m = fmaxf(m, fabsf(e[c]));
                     float s_star = m / (float)qmax;
                     uint16_t s16 = orc_f64_to_f16_up((double)s_star);
                     float sc = orc_f16_to_f32(s16);
                     float isc = sc != 0.0f ? 1.0f / sc : 0.0f;
                     memcpy(scales + 2 * j, &s16, 2);
-                    for (int c = j * group; c < (j + 1) * group; c++) {
+                    for (int c = j * qgroup; c < (j + 1) * qgroup; c++) {
                         int q = 0;
                         float v = 0.0f;
                         if (!is_out[c]) {
@@ -407,17 +460,18 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode,
 /* X_hat bf16[T,d] out.  status (optional, one word) gets bit 1 when a reserved
  * code -2^(b-1) was seen.  returns 0, -1, -2 as orc_encode; -3 when an outlier
  * index is >= d. */
-int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode,
+int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group,
                     const uint8_t *payload, int64_t T,
                     const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
                     const uint16_t *gain, const uint16_t *bias,
                     const float *step, uint16_t *X_hat, uint32_t *status, int nthreads) {
     if (!cfg_ok(d, group, bits, topk)) return -1;
     if ((gain == NULL) != (bias == NULL)) return -1;
-    if (scale_mode != 0 && scale_mode != 1) return -1;
-    const int J = d / group;
-    const int64_t rec = orc_record_bytes_mode(d, group, bits, topk, scale_mode);
-    const int64_t sbytes = scale_bytes(d, group, scale_mode);
+    if (!qcfg_ok(d, group, topk, scale_mode, qgroup, topk_group)) return -1;
+    if (qgroup == 0) qgroup = group;
+    const int J = d / group, Jq = d / qgroup;
+    const int64_t rec = orc_record_bytes_ext(d, group, bits, topk, scale_mode, qgroup, topk_group);
+    const int64_t sbytes = scale_bytes(d, qgroup, scale_mode);
     int err = 0;
     uint32_t st_word = 0;
     if (nthreads < 1) nthreads = 1;
@@ -432,6 +486,8 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode,
             const uint8_t *codes = scales + sbytes;
             const uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             const uint8_t *oval = oidx + 2 * topk;
+            const uint8_t *goff = oval + 2 * topk;
+            const uint8_t *gval = goff + ((int64_t)Jq * topk_group + 1) / 2 * 2;
             int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
             if (has_ref < 0) {
 #pragma omp atomic write
@@ -447,7 +503,7 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode,
                 }
                 float sc;
                 if (scale_mode == 0) sc = st[c];
-                else { uint16_t s16; memcpy(&s16, scales + 2 * (c / group), 2); sc = orc_f16_to_f32(s16); }
+                else { uint16_t s16; memcpy(&s16, scales + 2 * (c / qgroup), 2); sc = orc_f16_to_f32(s16); }
                 eh[c] = (float)q * sc;
             }
             for (int n = 0; n < topk; n++) {
@@ -460,6 +516,17 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode,
                     continue;
                 }
                 eh[ci] = orc_f16_to_f32(hv);
+            }
+            for (int n = 0; n < Jq * topk_group; n++) {
+                uint16_t hv;
+                int o = goff[n];
+                memcpy(&hv, gval + 2 * n, 2);
+                if (o >= qgroup) {
+#pragma omp atomic write
+                    err = -3;
+                    continue;
+                }
+                eh[(n / topk_group) * qgroup + o] = orc_f16_to_f32(hv);
             }
             for (int j = 0; j < J; j++) {
                 uint32_t w;

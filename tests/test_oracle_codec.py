@@ -415,3 +415,118 @@ def test_dynamic_scale_zero_group_marker_and_identity(orc):
     assert scale[0, 0] == np.float16(np.nextafter(np.float16(3.0 / 7), np.float16(1))).view(np.uint16) or \
         f16(scale[0, :1])[0] >= 3.0 / 7
     assert not scale[0, 1:].any()
+
+
+# ------------------------------------------------------------------ the rest of the quantiser family (Sec. IV-C)
+def test_family_record_by_hand(orc):
+    """One token worked by hand: d = 8, one alignment group, no reference, zero-mean values (so beta = 0 and
+    e = x), quantisation groups of 4, one outlier per group, 4-bit codes."""
+    x = np.array([[8, -8, 1, -1, 0.5, -0.5, 0, 0]], np.float32)
+    pay = orc.encode(8, 8, 4, 0, bits_of(x), scale_mode=1, qgroup=4, topk_group=1)
+    # group 0: |8| ties with |-8| -> the lower channel (offset 0) is the outlier, 8.0 = 0x4800; the dense maximum
+    # is still 8: scale = RoundUp16(8/7 = 1.142857..) = 1171 * 2^-10 = 0x3c93; codes 0, -7, round(1/1.1436) = 1, -1.
+    # group 1: outlier offset 0, 0.5 = 0x3800; scale = RoundUp16(0.5/7) = 1171 * 2^-14 = 0x2c93; codes 0, -7, 0, 0.
+    want = bytes([0, 0, 0, 0,                   # alpha = 0, beta = 0
+                  0x93, 0x3c, 0x93, 0x2c,       # two scales
+                  0x90, 0xf1, 0x90, 0x00,       # codes, two per byte, low nibble first
+                  0, 0,                         # in-group offsets
+                  0x00, 0x48, 0x00, 0x38])      # outlier values
+    assert pay.size == 32 and pay.tobytes() == want + bytes(32 - len(want))
+    xh = orc.reconstruct(8, 8, 4, 0, pay, 1, scale_mode=1, qgroup=4, topk_group=1)
+    s0, s1 = 1171 * 2.0 ** -10, 1171 * 2.0 ** -14
+    exact = np.array([8, -7 * s0, s0, -s0, 0.5, -7 * s1, 0, 0])
+    assert np.array_equal(xh[0], bits_of(exact.astype(np.float32)[None])[0])
+
+
+@pytest.mark.parametrize("bits,g,qg,kg", [
+    (4, 64, 64, 1), (4, 64, 64, 2), (8, 64, 64, 1), (4, 128, 32, 4), (4, 32, 128, 2), (3, 64, 256, 3),
+    (8, 64, 0, 0), (8, 64, 512, 0), (4, 64, 512, 0), (2, 128, 512, 0), (4, 128, 16, 1),
+])
+def test_family_outliers_per_group_and_token_scale(orc, bits, g, qg, kg):
+    d, T = 512, 24
+    q_g = qg or g
+    Jq = d // q_g
+    gen = synth.generator(300 + bits + q_g + kg)
+    X = synth.activations(T, d, synth.channel_scale(d, 8), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    Xb, Rb = synth.bf16_bits(X), synth.bf16_bits(R)
+    kw = dict(scale_mode=1, qgroup=qg, topk_group=kg)
+    pay = orc.encode(d, g, bits, 0, Xb, ref_base=Rb, **kw)
+    # record size from the layout, typed out
+    ng = Jq * kg
+    raw = 4 * (d // g) + (2 * Jq + 3) // 4 * 4 + d * bits // 8 + (ng + 1) // 2 * 2 + 2 * ng
+    assert orc.record_bytes(d, g, bits, 0, 1, qg, kg) == (raw + 15) // 16 * 16 == pay.size // T
+    parts = orc.split_payload(pay, T, d, g, bits, 0, 1, qg, kg)
+    coef, codes, scale = parts[0], parts[1], parts[4]
+    assert scale.shape == (T, Jq)
+    qmax = (1 << (bits - 1)) - 1
+    h = orc.bf16_to_f32(Xb).astype(np.float64)
+    r = orc.bf16_to_f32(Rb).astype(np.float64)
+    e = h - (np.repeat(f16(coef & 0xffff), g, axis=1) * r + np.repeat(f16(coef >> 16), g, axis=1))
+    e32 = e.astype(np.float32)   # the residual is a binary32 value: ranking uses its bits
+    q = np.stack([orc.unpack_codes(codes[t], d, bits) for t in range(T)])
+    is_out = np.zeros((T, d), bool)
+    e_hat_out = np.zeros((T, d))
+    if kg:
+        goff, gval = parts[5], parts[6]
+        eg = np.abs(e32).reshape(T, Jq, q_g)
+        # brute force: stable sort by decreasing magnitude keeps the lower channel first among equals
+        order = np.argsort(-eg, axis=2, kind="stable")[:, :, :kg]
+        want_off = np.sort(order, axis=2)
+        assert np.array_equal(goff.astype(np.int64), want_off)
+        chan = want_off + (np.arange(Jq) * q_g)[None, :, None]
+        tt = np.arange(T)[:, None, None]
+        is_out[tt, chan] = True
+        want_val = e32[tt, chan].astype(np.float16)      # numpy's own round-to-nearest-even conversion
+        assert np.array_equal(gval, want_val.view(np.uint16))
+        e_hat_out[tt, chan] = want_val.astype(np.float64)
+        assert np.all(q[is_out] == 0)
+    s = f16(scale)
+    s_full = np.repeat(s, q_g, axis=1)
+    dense_max = np.where(is_out, 0, np.abs(e)).reshape(T, Jq, q_g).max(axis=2)
+    want = dense_max / qmax
+    assert np.all(s >= want * (1 - 1e-6))
+    below = np.nextafter(s.astype(np.float16), np.float16(-np.inf)).astype(np.float64)
+    assert np.all((below < want * (1 + 1e-6)) | (s == 0))
+    e_hat = q * s_full
+    assert q.min() >= -qmax and q.max() <= qmax
+    assert np.all(np.abs(e - e_hat)[~is_out] <= 0.5 * s_full[~is_out] * (1 + 1e-5) + 1e-12)
+    assert np.all((np.abs(q).reshape(T, Jq, q_g).max(axis=2) == qmax) | (dense_max == 0))
+    # Eq. 10 / Eq. 9 with the outliers restored
+    e_hat = np.where(is_out, e_hat_out, e_hat)
+    xh = orc.bf16_to_f32(orc.reconstruct(d, g, bits, 0, pay, T, ref_base=Rb, **kw)).astype(np.float64)
+    assert np.all(np.abs((h - xh) - (e - e_hat)) <= np.abs(xh) * 2.0 ** -8 + 1e-30)
+    # taking outliers out can only lower a group's scale
+    if kg:
+        s_plain = f16(orc.split_payload(orc.encode(d, g, bits, 0, Xb, ref_base=Rb, scale_mode=1, qgroup=qg),
+                                        T, d, g, bits, 0, 1, qg, 0)[4])
+        assert np.all(s <= s_plain) and np.mean(s < s_plain) > 0.5
+
+
+def test_family_token_scale_is_the_token_maximum_and_rejections(orc):
+    d, g, T = 256, 64, 5
+    gen = synth.generator(77)
+    X = synth.activations(T, d, synth.channel_scale(d, 9), gen)
+    Xb = synth.bf16_bits(X)
+    pay = orc.encode(d, g, 8, 0, Xb, scale_mode=1, qgroup=d)
+    coef, codes, _, _, scale = orc.split_payload(pay, T, d, g, 8, 0, 1, d, 0)
+    assert scale.shape == (T, 1)
+    q = np.stack([orc.unpack_codes(codes[t], d, 8) for t in range(T)])
+    assert np.all(np.abs(q).max(axis=1) == 127)          # one scale per token: exactly the token's largest |e| is at the end
+    assert np.array_equal(codes.view(np.int8).astype(np.int32), q)   # 8-bit codes are plain signed bytes
+    orc.encode(d, g, 4, 0, Xb, scale_mode=1, qgroup=d, topk_group=1)        # offsets are one byte: g_q = 256 still fits
+    with pytest.raises(ValueError):
+        orc.encode(512, g, 4, 0, np.zeros((1, 512), np.uint16), scale_mode=1, qgroup=512, topk_group=1)
+    with pytest.raises(ValueError):
+        orc.encode(d, g, 4, 2, Xb, scale_mode=1, topk_group=1)              # one outlier rule at a time
+    with pytest.raises(ValueError):
+        orc.encode(d, g, 4, 0, Xb, step=flat_tables(d, 0.1)[0], inv_step=flat_tables(d, 0.1)[1], qgroup=32)   # static table: g_q = g_a
+    with pytest.raises(ValueError):
+        orc.reconstruct(d, g, 4, 0, _bad_offset_payload(orc, d, g), 1, scale_mode=1, qgroup=32, topk_group=1)
+
+
+def _bad_offset_payload(orc, d, g):
+    pay = orc.encode(d, g, 4, 0, np.zeros((1, d), np.uint16), scale_mode=1, qgroup=32, topk_group=1)
+    J, Jq = d // g, d // 32
+    pay[4 * J + 2 * Jq + d // 2] = 32      # first in-group offset: 32 is outside a group of 32
+    return pay
