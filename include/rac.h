@@ -26,11 +26,15 @@
  *
  * Wire record of one token (little endian), records back to back in `payload`:
  *     coef    J x u32      binary16 alpha in bits 0..15, binary16 beta in 16..31,  J = d/group
- *     scale   J x u16      binary16 group scales, scale_mode 1 only, padded to a multiple of 4 bytes
+ *     scale   Jq x u16     binary16 scales of the quantisation groups, scale_mode 1 only (Jq = d/qgroup),
+ *                          padded to a multiple of 4 bytes
  *     codes   d*bits/8 B   code of channel c in stream bits [c*bits, c*bits+bits); stream bit n is
  *                          bit n%8 of byte n/8; two's complement; -2^(bits-1) is never produced
  *     out_idx topk x u16   channel indices, ascending
  *     out_val topk x u16   binary16 residuals of those channels (their dense code is 0)
+ *     grp_off Jq*topk_group x u8   in-group offsets of the per-group outliers, ascending within a group,
+ *                          padded to a multiple of 2 bytes (scale_mode 1 only)
+ *     grp_val Jq*topk_group x u16  binary16 residuals of those channels (their dense code is 0)
  *     zero padding to a multiple of 16 bytes
  * rac_record_bytes() gives the stride.  A token range is a contiguous byte range.
  */
@@ -59,20 +63,25 @@ extern "C" {
                                          stopped early and its outputs are incomplete                        */
 #define RAC_STATUS_OUTLIER_RANGE 16u  /* decode met an outlier index >= d and ignored that outlier            */
 
-/* Codec configuration (Sec. IV-C: calibration picks (g_a, g_q, q, k) per phase and direction; here
- * g_a == g_q == group).
+/* Codec configuration (Sec. IV-C: calibration picks (g_a, g_q, q, k) per phase and direction).
  *   d       hidden width; multiple of 32, <= 8192
- *   group   channels per alignment/quantisation group; power of two, 32..1024, divides d
- *   bits    code width: 2, 3 or 4            (Qmax = 2^(bits-1) - 1, Eq. 8a)
- *   topk    outliers per token kept as binary16, 0..16 (Sec. IV-C "Outlier Metadata"; per token here)
+ *   group   g_a, channels per alignment group; power of two, 32..1024, divides d
+ *   bits    code width q: 2, 3 or 4; also 8 in scale_mode 1     (Qmax = 2^(bits-1) - 1, Eq. 8a)
+ *   topk    outliers per TOKEN kept as binary16, 0..16 (u16 channel index); scale_mode 0 only
  *   coef_fmt   0 = binary16 pair (the only format)
- *   scale_mode 0 = static per-channel step table `step`/`inv_step` (calibrated clip; dense values may clip)
- *              1 = Eq. 8 as printed: per (token, group) scale s = RoundUp_binary16(max|E| / Qmax) carried in the
- *                  record (J x u16 after `coef`, padded to 4 bytes), scale 0 = all-zero group; nothing clips;
- *                  `step` and `inv_step` are not read and may be NULL; only with topk == 0
- *   flags   must be 0 */
+ *   scale_mode 0 = static per-channel step table `step`/`inv_step` (calibrated clip; dense values may clip);
+ *                  g_q == g_a, `qgroup` 0 or == group, `topk_group` 0
+ *              1 = Eq. 8 as printed: per quantisation group the scale s = RoundUp_binary16(max|E^d| / Qmax) is
+ *                  carried in the record, scale 0 = all-zero group; nothing clips; `step` and `inv_step` are
+ *                  not read and may be NULL
+ *   flags   must be 0
+ *   qgroup  g_q, channels per quantisation group (scale_mode 1): 0 = same as `group`; a power of two 32..1024
+ *           that divides d; or d itself (the paper's decode mode: one scale per token)
+ *   topk_group  k_g, outliers per quantisation group (Sec. IV-C "Outlier Metadata"), 0..4, scale_mode 1 with
+ *           qgroup <= 256: the k_g largest |e| of every group (ties to the lower channel) leave the dense base
+ *           before its scale is taken; one-byte in-group offsets in ascending order + binary16 values */
 typedef struct {
-    int32_t d, group, bits, topk, coef_fmt, scale_mode, flags;
+    int32_t d, group, bits, topk, coef_fmt, scale_mode, flags, qgroup, topk_group;
 } rac_codec_cfg;
 
 /* One selected span (Eq. 3): query[q_start .. q_start+len) == history[h_start .. h_start+len). */

@@ -44,14 +44,16 @@ class RacError(RuntimeError):
 
 class CodecCfg(C.Structure):
     """Mirror of ``rac_codec_cfg``."""
-    _fields_ = [(n, C.c_int32) for n in ("d", "group", "bits", "topk", "coef_fmt", "scale_mode", "flags")]
+    _fields_ = [(n, C.c_int32) for n in ("d", "group", "bits", "topk", "coef_fmt", "scale_mode", "flags",
+                                         "qgroup", "topk_group")]
 
-    def __init__(self, d: int, group: int, bits: int, topk: int = 0, scale_mode: int = 0):
-        super().__init__(d, group, bits, topk, 0, scale_mode, 0)
+    def __init__(self, d: int, group: int, bits: int, topk: int = 0, scale_mode: int = 0, qgroup: int = 0,
+                 topk_group: int = 0):
+        super().__init__(d, group, bits, topk, 0, scale_mode, 0, qgroup, topk_group)
 
     def __repr__(self):
         return (f"CodecCfg(d={self.d}, group={self.group}, bits={self.bits}, topk={self.topk}, "
-                f"scale_mode={self.scale_mode})")
+                f"scale_mode={self.scale_mode}, qgroup={self.qgroup}, topk_group={self.topk_group})")
 
 
 _lib: Optional[C.CDLL] = None

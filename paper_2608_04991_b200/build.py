@@ -8,11 +8,11 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librac.so")
-SOURCES = ["rac_codec.cu", "rac_match.cu"]
-HEADERS = ["rac_common.cuh", os.path.join("..", "..", "include", "rac.h")]
+SOURCES = ["rac_codec.cu", "rac_codec_dyn.cu", "rac_match.cu"]
+HEADERS = ["rac_common.cuh", "rac_codec_dev.cuh", os.path.join("..", "..", "include", "rac.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "--use_fast_math=false" if False else "-Xptxas", "-v",
+    "-Xcompiler", "-fPIC", "-shared", "--threads", "0", "-Xptxas", "-v",
 ]
 
 

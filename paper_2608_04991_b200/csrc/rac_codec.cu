@@ -16,10 +16,7 @@
 // Kernels: encode_ws_kernel (streaming pass of encode, optionally also the sender-side x_hat),
 // outlier_kernel (second launch of encode: the k largest |e| per token), decode_kernel (receiver and sender
 // reconstruction), calib_kernel + calib_finalize_kernel (step tables).
-#include <math.h>
-#include <stdlib.h>
-
-#include "rac_common.cuh"
+#include "rac_codec_dev.cuh"
 
 namespace rac {
 
@@ -31,16 +28,33 @@ static bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     if (!cfg) return RAC_EINVAL;
     if (cfg->d <= 0 || cfg->group <= 0 || cfg->topk < 0 || cfg->bits <= 0) return RAC_EINVAL;
+    if (cfg->qgroup < 0 || cfg->topk_group < 0) return RAC_EINVAL;
     if (cfg->coef_fmt != 0 || cfg->flags != 0) return RAC_EUNSUPPORTED;
     if (cfg->scale_mode != 0 && cfg->scale_mode != 1) return RAC_EUNSUPPORTED;
-    // Eq. 8 takes the scale from the dense values, i.e. after the outliers are known; the outlier pass runs
-    // after the streaming pass here, so the per-group scale is offered without outliers only
-    if (cfg->scale_mode == 1 && cfg->topk != 0) return RAC_EUNSUPPORTED;
     if (cfg->d % cfg->group) return RAC_EINVAL;
     if (cfg->d % 32 || cfg->d > 8192) return RAC_EUNSUPPORTED;
     if (!is_pow2(cfg->group) || cfg->group < 32 || cfg->group > 1024) return RAC_EUNSUPPORTED;
-    if (cfg->bits < 2 || cfg->bits > 4) return RAC_EUNSUPPORTED;
     if (cfg->topk > 16 || cfg->topk > cfg->d) return RAC_EUNSUPPORTED;
+    int qgroup = cfg->qgroup ? cfg->qgroup : cfg->group;
+    int lpq = 0;
+    if (cfg->scale_mode == 0) {
+        // the static table: one grouping, per-token outliers, 2..4 bits
+        if (qgroup != cfg->group || cfg->topk_group != 0) return RAC_EUNSUPPORTED;
+        if (cfg->bits < 2 || cfg->bits > 4) return RAC_EUNSUPPORTED;
+        lpq = cfg->group / 32;
+    } else {
+        // Eq. 8 takes the scale from the dense values, i.e. after the outliers are known.  The per-token
+        // selection runs as a second launch, after the codes exist, so this mode offers the paper's own
+        // per-group outliers (picked inside the streaming pass) and not the per-token ones.
+        if (cfg->topk != 0) return RAC_EUNSUPPORTED;
+        if (cfg->bits != 2 && cfg->bits != 3 && cfg->bits != 4 && cfg->bits != 8) return RAC_EUNSUPPORTED;
+        if (cfg->d % qgroup) return RAC_EINVAL;
+        if (is_pow2(qgroup) && qgroup >= 32 && qgroup <= 1024) lpq = qgroup / 32;
+        else if (qgroup == cfg->d) lpq = 0;   // one scale per token, exchanged through shared memory
+        else return RAC_EUNSUPPORTED;
+        if (cfg->topk_group > 4) return RAC_EUNSUPPORTED;
+        if (cfg->topk_group > 0 && (lpq == 0 || qgroup > 256)) return RAC_EUNSUPPORTED;   // one-byte offsets
+    }
     g->d = cfg->d;
     g->group = cfg->group;
     g->bits = cfg->bits;
@@ -50,257 +64,17 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     g->nthreads = ((cfg->d / 32) + 31) / 32 * 32;
     g->code_bytes = cfg->d * cfg->bits / 8;
     g->scale_mode = cfg->scale_mode;
-    g->codes_off = 4 * g->J + (cfg->scale_mode == 1 ? (2 * g->J + 3) / 4 * 4 : 0);
-    int raw = g->codes_off + g->code_bytes + 4 * cfg->topk;
+    g->qgroup = qgroup;
+    g->Jq = cfg->d / qgroup;
+    g->lpq = lpq;
+    g->topk_group = cfg->topk_group;
+    g->codes_off = 4 * g->J + (cfg->scale_mode == 1 ? (2 * g->Jq + 3) / 4 * 4 : 0);
+    const int ng = g->Jq * g->topk_group;
+    g->goff_off = g->codes_off + g->code_bytes + 4 * cfg->topk;
+    g->gval_off = g->goff_off + (ng + 1) / 2 * 2;
+    const int raw = g->gval_off + 2 * ng;
     g->rec = (raw + 15) / 16 * 16;
     return RAC_OK;
-}
-
-// ------------------------------------------------------------------------------------------------
-// kernel parameters
-// ------------------------------------------------------------------------------------------------
-struct CodecParams {
-    // tensors
-    const uint16_t *X;         // encode / calibrate input, bf16[T,d]
-    const uint16_t *ref_base;  // bf16[ref_rows,d] or null
-    const int32_t *ref_row;    // int32[T] or null
-    const uint16_t *gain;      // binary16[d] or null
-    const uint16_t *bias;
-    const float *step;         // [2,d]
-    const float *inv_step;     // [2,d]
-    uint8_t *payload;          // encode out / decode in
-    uint16_t *X_hat;           // decode out
-    float *calib_partial;      // calibrate out: [grid][2][d] sums of e^2, then [grid][2] token counts
-    float *tmax;               // encode with outliers: [T][d/32] largest |e| per thread slab (caller workspace)
-    uint32_t *status;
-    long long T;
-    long long ref_rows;
-    // geometry
-    int d, J, lpg, lpg_shift, topk, rec, code_bytes, codes_off, stages;
-    float inv_group;
-};
-
-constexpr int kMaxStages = 4;
-constexpr int kRecBufs = 3;
-constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer (ties to even) in the low mantissa bits
-
-// control block at the start of dynamic shared memory
-struct Ctrl {
-    unsigned long long bar[kMaxStages];
-    int row[kMaxStages];        // reference row of the token in each stage, -1 = direct
-};
-
-__host__ __device__ inline int align_up(int v, int a) { return (v + a - 1) / a * a; }
-
-struct EncSmem {  // calibration kernel
-    int stage0, stage_bytes, acc0, total;
-};
-__host__ __device__ inline EncSmem enc_smem_layout(int d, int stages, int nthreads) {
-    EncSmem s;
-    s.stage0 = align_up((int)sizeof(Ctrl), 128);
-    s.stage_bytes = 4 * d;  // X row + R row
-    s.acc0 = s.stage0 + stages * s.stage_bytes;   // e^2 accumulators: 2 table rows x 32 floats per thread
-    s.total = s.acc0 + 2 * nthreads * 32 * 4;
-    return s;
-}
-
-struct DecSmem {
-    int ctrl, stage0, stage_bytes, rec_pad, out0, total;
-};
-__host__ __device__ inline DecSmem dec_smem_layout(int d, int rec, int stages) {
-    DecSmem s;
-    s.ctrl = 0;
-    s.stage0 = align_up((int)sizeof(Ctrl), 128);
-    s.rec_pad = align_up(rec, 128);
-    s.stage_bytes = s.rec_pad + 2 * d;
-    s.out0 = s.stage0 + stages * s.stage_bytes;
-    s.total = s.out0 + kRecBufs * 2 * d;
-    return s;
-}
-
-// ------------------------------------------------------------------------------------------------
-// device helpers
-// ------------------------------------------------------------------------------------------------
-typedef unsigned long long u64;
-
-__device__ __forceinline__ u64 pack2(float lo, float hi) {
-    u64 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(u64 v, float &lo, float &hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ u64 pfma(u64 a, u64 b, u64 c) {
-    u64 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ u64 padd(u64 a, u64 b) {
-    u64 d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ u64 psub(u64 a, u64 b) {
-    u64 d;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ u64 pmul(u64 a, u64 b) {
-    u64 d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-// a 32-bit word of two bf16 -> packed (even channel, odd channel) binary32, exact
-__device__ __forceinline__ u64 bf16x2_to_p(uint32_t w) {
-    return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
-// bits of a where m is set, bits of b elsewhere
-__device__ __forceinline__ uint32_t bitsel(uint32_t a, uint32_t b, uint32_t m) { return (a & m) | (b & ~m); }
-
-// rotate the four entries right by rot (new[j] = old[(j - rot) & 3])
-__device__ __forceinline__ void rot_right4(uint32_t (&w)[4], int rot) {
-    if (rot & 1) { uint32_t t = w[3]; w[3] = w[2]; w[2] = w[1]; w[1] = w[0]; w[0] = t; }
-    if (rot & 2) { uint32_t t = w[0]; w[0] = w[2]; w[2] = t; t = w[1]; w[1] = w[3]; w[3] = t; }
-}
-// rotate left by rot (new[j] = old[(j + rot) & 3])
-__device__ __forceinline__ void rot_left4(uint32_t (&w)[4], int rot) {
-    if (rot & 1) { uint32_t t = w[0]; w[0] = w[1]; w[1] = w[2]; w[2] = w[3]; w[3] = t; }
-    if (rot & 2) { uint32_t t = w[0]; w[0] = w[2]; w[2] = t; t = w[1]; w[1] = w[3]; w[3] = t; }
-}
-
-// low BITS bits of eight integers -> one word, element 0 in the lowest field
-template <int BITS>
-__device__ __forceinline__ uint32_t pack8(const uint32_t (&b)[8]) {
-    if (BITS == 4) {
-        uint32_t b01 = bitsel(b[0], b[1] << 4, 0x0fu), b23 = bitsel(b[2], b[3] << 4, 0x0fu);
-        uint32_t b45 = bitsel(b[4], b[5] << 4, 0x0fu), b67 = bitsel(b[6], b[7] << 4, 0x0fu);
-        return __byte_perm(__byte_perm(b01, b23, 0x0040), __byte_perm(b45, b67, 0x0040), 0x5410);
-    } else {
-        constexpr uint32_t m1 = (1u << BITS) - 1u, m2 = (1u << (2 * BITS)) - 1u, m4 = (1u << (4 * BITS)) - 1u;
-        constexpr uint32_t m8 = (BITS * 8 == 32) ? 0xffffffffu : ((1u << (BITS * 8 % 32)) - 1u);
-        uint32_t p0 = bitsel(b[0], b[1] << BITS, m1), p1 = bitsel(b[2], b[3] << BITS, m1);
-        uint32_t p2 = bitsel(b[4], b[5] << BITS, m1), p3 = bitsel(b[6], b[7] << BITS, m1);
-        uint32_t q0 = bitsel(p0, p1 << (2 * BITS), m2), q1 = bitsel(p2, p3 << (2 * BITS), m2);
-        return bitsel(q0, q1 << (4 * BITS), m4) & m8;
-    }
-}
-
-// Two signed integers saturated to BITS-bit two's complement and packed below the bits of c
-// (d = c << 2*BITS | sat(hi) << BITS | sat(lo)); BITS is 4 or 2.
-template <int BITS>
-__device__ __forceinline__ uint32_t sat_pack2(int hi, int lo, uint32_t c) {
-    uint32_t d;
-    if (BITS == 4) asm("cvt.pack.sat.s4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(lo), "r"(c));
-    else asm("cvt.pack.sat.s2.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(lo), "r"(c));
-    return d;
-}
-
-// reference values of one slot (8 channels starting at channel c) from shared memory, with the optional
-// per-channel transform r <- bf16(gain*r + bias)
-__device__ __forceinline__ void load_ref_slot(uint32_t addr, const uint16_t *gain, const uint16_t *bias, int c,
-                                              u64 (&r2)[4]) {
-    uint4 w = lds128(addr);
-    const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
-    if (gain) {
-        uint4 gw = __ldg(reinterpret_cast<const uint4 *>(gain + c));
-        uint4 bw = __ldg(reinterpret_cast<const uint4 *>(bias + c));
-        const uint32_t gws[4] = {gw.x, gw.y, gw.z, gw.w};
-        const uint32_t bws[4] = {bw.x, bw.y, bw.z, bw.w};
-#pragma unroll
-        for (int i = 0; i < 4; i++) {
-            float g0 = half_bits_to_float(gws[i] & 0xffff), g1 = half_bits_to_float(gws[i] >> 16);
-            float b0 = half_bits_to_float(bws[i] & 0xffff), b1 = half_bits_to_float(bws[i] >> 16);
-            float r0 = __uint_as_float(ws[i] << 16), r1 = __uint_as_float(ws[i] & 0xffff0000u);
-            r2[i] = pack2(bf16_round(__fmaf_rn(g0, r0, b0)), bf16_round(__fmaf_rn(g1, r1, b1)));
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 4; i++) r2[i] = bf16x2_to_p(ws[i]);
-    }
-}
-
-// thread 0: reference row of token t (-1 = coded directly); flags rows beyond the buffer
-__device__ __forceinline__ int resolve_row(const CodecParams &p, int raw_row) {
-    if (!p.ref_base || raw_row < 0) return -1;
-    if (raw_row >= p.ref_rows) {
-        if (p.status) atomicOr(p.status, RAC_STATUS_REF_RANGE);
-        return -1;
-    }
-    return raw_row;
-}
-// thread 0: start the copies of one token into a stage: `first` (X row or record) and, if any, its reference row
-__device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ctrl, uint32_t stage_addr, uint32_t r_off,
-                                                  int stage, int row, const void *first_src, uint32_t first_bytes) {
-    ctrl->row[stage] = row;
-    const uint32_t bar = smem_u32(&ctrl->bar[stage]);
-    const uint32_t row_bytes = 2u * (uint32_t)p.d;
-    mbar_arrive_expect_tx(bar, first_bytes + (row >= 0 ? row_bytes : 0u));
-    bulk_load(stage_addr, first_src, first_bytes, bar);
-    if (row >= 0) bulk_load(stage_addr + r_off, p.ref_base + (long long)row * p.d, row_bytes, bar);
-}
-
-// Eq. 6 for the group this thread belongs to: centred two-pass sums over the thread's 32 channels (packed
-// binary32, two accumulators per sum), butterflies over the group's lanes, the zero-variance rule, and wire
-// rounding of (alpha, beta) to binary16.  Returns the wire coefficients splatted for packed arithmetic; a16/b16
-// are their bit patterns.
-__device__ __forceinline__ void fit_group(const u64 (&x2)[16], const u64 (&r2)[16], bool has_ref, int lpg, float inv_group,
-                                          unsigned int group_mask, uint32_t *status, u64 &a2, u64 &b2,
-                                          uint32_t *coef_word = nullptr) {
-    u64 sra = 0ull, srb = 0ull, sha = 0ull, shb = 0ull;
-#pragma unroll
-    for (int i = 0; i < 16; i += 2) {
-        sra = padd(sra, r2[i]); srb = padd(srb, r2[i + 1]);
-        sha = padd(sha, x2[i]); shb = padd(shb, x2[i + 1]);
-    }
-    float sr, sr_hi, sh, sh_hi;
-    unpack2(padd(sra, srb), sr, sr_hi);
-    unpack2(padd(sha, shb), sh, sh_hi);
-    sr += sr_hi;
-    sh += sh_hi;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        if (lpg > o) {
-            sr += __shfl_xor_sync(group_mask, sr, o);
-            sh += __shfl_xor_sync(group_mask, sh, o);
-        }
-    }
-    if (!(fabsf(sr) <= 3.0e38f) || !(fabsf(sh) <= 3.0e38f)) {
-        if (status) atomicOr(status, RAC_STATUS_NONFINITE);
-    }
-    const float rbar = sr * inv_group, hbar = sh * inv_group;
-    const u64 rbar2 = pack2(rbar, rbar), hbar2 = pack2(hbar, hbar);
-    u64 sxxa = 0ull, sxxb = 0ull, sxya = 0ull, sxyb = 0ull;
-#pragma unroll
-    for (int i = 0; i < 16; i += 2) {
-        u64 dr0 = psub(r2[i], rbar2), dh0 = psub(x2[i], hbar2);
-        u64 dr1 = psub(r2[i + 1], rbar2), dh1 = psub(x2[i + 1], hbar2);
-        sxxa = pfma(dr0, dr0, sxxa); sxya = pfma(dr0, dh0, sxya);
-        sxxb = pfma(dr1, dr1, sxxb); sxyb = pfma(dr1, dh1, sxyb);
-    }
-    float sxx, sxx_hi, sxy, sxy_hi;
-    unpack2(padd(sxxa, sxxb), sxx, sxx_hi);
-    unpack2(padd(sxya, sxyb), sxy, sxy_hi);
-    sxx += sxx_hi;
-    sxy += sxy_hi;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        if (lpg > o) {
-            sxx += __shfl_xor_sync(group_mask, sxx, o);
-            sxy += __shfl_xor_sync(group_mask, sxy, o);
-        }
-    }
-    // zero-variance rule, then wire rounding to binary16
-    float a_star = 0.f, b_star = hbar;
-    if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {
-        a_star = __fdiv_rn(sxy, sxx);
-        b_star = __fmaf_rn(-a_star, rbar, hbar);
-    }
-    const uint32_t a16 = float_to_half_bits_sat(a_star), b16 = float_to_half_bits_sat(b_star);
-    const float a = half_bits_to_float(a16), b = half_bits_to_float(b16);
-    a2 = pack2(a, a);
-    b2 = pack2(b, b);
-    if (coef_word) *coef_word = a16 | (b16 << 16);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -471,9 +245,7 @@ __host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages, boo
     return s;
 }
 
-// DYN: Eq. 8 as printed -- the scale of a group is the largest dense |e| of the group over Qmax, rounded up to
-// binary16 and written into the record; no step table is read.
-template <int BITS, bool TOPK, bool XHAT, bool DYN, int MINB>
+template <int BITS, bool TOPK, bool XHAT, int MINB>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -516,15 +288,10 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     }
     {
         // padding words of the records are written once and never touched again
-        const int raw = p.codes_off + p.code_bytes + 4 * p.topk;
+        const int raw = 4 * p.J + p.code_bytes + 4 * p.topk;
         for (int s = 0; s < 2 * S; s++)
             for (int o = raw + 4 * tid; o < p.rec; o += 4 * nt)
                 *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * p.rec + o) = 0u;
-        // an odd number of binary16 scales leaves two bytes of padding before the codes: zero that word once
-        if (DYN && tid == 0 && (p.J & 1))
-            for (int s = 0; s < 2 * S; s++)
-                *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * p.rec +
-                                              p.codes_off - 4) = 0u;
     }
     __syncthreads();
     if (tid == 0)
@@ -578,52 +345,21 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 
             // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
             if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
-            const float *inv_tab = DYN ? nullptr : p.inv_step + (has_ref ? 0 : d);
-            const float *step_tab = DYN ? nullptr : p.step + (has_ref ? 0 : d);
-            u64 dyn_inv2 = 0ull, dyn_s2 = 0ull;
-            if (DYN) {
-                // largest |e| of the group (this thread's 32 channels, then the group's lanes), in binary32
-                float m0 = 0.f, m1 = 0.f;
-#pragma unroll
-                for (int i = 0; i < 16; i++) {
-                    float e0, e1;
-                    unpack2(psub(x2[i], pfma(a2, r2[i], b2)), e0, e1);
-                    m0 = fmaxf(m0, fabsf(e0));
-                    m1 = fmaxf(m1, fabsf(e1));
-                }
-                float m = fmaxf(m0, m1);
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1)
-                    if (p.lpg > o) m = fmaxf(m, __shfl_xor_sync(group_mask, m, o));
-                // s = RoundUp_binary16(m / Qmax): round to nearest, then one step up if that fell short
-                const float s_star = __fdiv_rn(m, qmax);
-                uint32_t s16 = float_to_half_bits_sat(s_star);
-                if (half_bits_to_float(s16) < s_star && s16 < 0x7bffu) s16++;
-                const float sc = half_bits_to_float(s16);
-                const float isc = sc != 0.f ? __fdiv_rn(1.0f, sc) : 0.f;
-                dyn_inv2 = pack2(isc, isc);
-                dyn_s2 = pack2(sc, sc);
-                if ((lane & (p.lpg - 1)) == 0)
-                    reinterpret_cast<unsigned short *>(rec + 4 * p.J)[tid >> p.lpg_shift] = (unsigned short)s16;
-            }
+            const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
+            const float *step_tab = p.step + (has_ref ? 0 : d);
             uint32_t words[4];
             float tmax = 0.f;
 #pragma unroll
             for (int j = 0; j < 4; j++) {
                 const int c = (int)(off[j] >> 1);
-                u64 inv2[4], st2[4] = {0ull, 0ull, 0ull, 0ull};
-                if (DYN) {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) { inv2[i] = dyn_inv2; st2[i] = dyn_s2; }
-                } else {
-                    const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
-                    const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
-                    inv2[0] = pack2(iv0.x, iv0.y); inv2[1] = pack2(iv0.z, iv0.w); inv2[2] = pack2(iv1.x, iv1.y); inv2[3] = pack2(iv1.z, iv1.w);
-                    if (XHAT) {
-                        const float4 s0 = __ldg(reinterpret_cast<const float4 *>(step_tab + c));
-                        const float4 s1 = __ldg(reinterpret_cast<const float4 *>(step_tab + c + 4));
-                        st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
-                    }
+                const float4 iv0 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c));
+                const float4 iv1 = __ldg(reinterpret_cast<const float4 *>(inv_tab + c + 4));
+                const u64 inv2[4] = {pack2(iv0.x, iv0.y), pack2(iv0.z, iv0.w), pack2(iv1.x, iv1.y), pack2(iv1.z, iv1.w)};
+                u64 st2[4] = {0ull, 0ull, 0ull, 0ull};
+                if (XHAT) {
+                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(step_tab + c));
+                    const float4 s1 = __ldg(reinterpret_cast<const float4 *>(step_tab + c + 4));
+                    st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
                 }
                 float ev[8];
                 uint32_t xh[4];
@@ -685,7 +421,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                 }
             }
             rot_right4(words, rot);  // words[q] is now the code word of piece q
-            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + p.codes_off) + tid * BITS;
+            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + 4 * p.J) + tid * BITS;
             if (BITS == 4) {
                 cw[0] = words[0]; cw[1] = words[1]; cw[2] = words[2]; cw[3] = words[3];
             } else if (BITS == 3) {
@@ -951,7 +687,7 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
             if (c < d) {
                 int pos = 0;
                 for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
-                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + p.codes_off + p.code_bytes);
+                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
                 const uint32_t hv = float_to_half_bits_sat(sele[sl]);
                 oidx[pos] = (unsigned short)c;
                 oidx[k + pos] = (unsigned short)hv;
@@ -966,7 +702,7 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
                     const float rt = __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16));
                     p.X_hat[t * d + c] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(rt, half_bits_to_float(hv))));
                 }
-                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + p.codes_off);
+                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
                 const int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
                 atomicAnd(&codes32[wd], ~(cmask << sh));
                 if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
@@ -1013,8 +749,7 @@ __global__ void calib_finalize_kernel(const float *partial, int nblocks, int d, 
 // into an output row in shared memory, patches the outliers it owns, and the row leaves as one bulk store.
 // The step table row of referenced tokens lives in registers for the whole kernel (a thread always owns
 // the same channels); direct tokens read row 1 through L1.
-// DYN: the step of a channel is its group's binary16 scale from the record (Eq. 8 as printed), not a table.
-template <int BITS, int KT, bool DYN>
+template <int BITS, int KT>
 __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x;
@@ -1065,7 +800,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
 #pragma unroll
     for (int j = 0; j < 4; j++) {
         float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
-        if (valid && !DYN) {
+        if (valid) {
             s0 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1)));
             s1 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1) + 4));
         }
@@ -1100,13 +835,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
             const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
             const u64 a2 = pack2(a, a), b2 = pack2(b, b);
-            u64 dyn_s2 = 0ull;
-            if (DYN) {
-                const float sc = half_bits_to_float(reinterpret_cast<const unsigned short *>(rec + 4 * p.J)[tid >> p.lpg_shift]);
-                dyn_s2 = pack2(sc, sc);
-            }
             // code words of the four pieces, in piece order, then rotated into slot order
-            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + p.codes_off) + tid * BITS;
+            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + 4 * p.J) + tid * BITS;
             uint32_t words[4];
             if (BITS == 4) {
                 words[0] = cw[0]; words[1] = cw[1]; words[2] = cw[2]; words[3] = cw[3];
@@ -1135,20 +865,14 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
                 u64 r2[4], st2[4];
                 if (has_ref) {
                     load_ref_slot(rs + off[j], p.gain, p.bias, c, r2);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) r2[i] = 0ull;
-                }
-                if (DYN) {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) st2[i] = dyn_s2;
-                } else if (has_ref) {
 #pragma unroll
                     for (int i = 0; i < 4; i++) st2[i] = st0[4 * j + i];
                 } else {
                     const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c));
                     const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c + 4));
                     st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[i] = 0ull;
                 }
                 const uint32_t w = words[j];
                 uint32_t o[4];
@@ -1166,7 +890,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             }
             if (KT > 0) {
                 // outliers whose channel this thread owns replace what the dense pass wrote
-                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + p.codes_off + p.code_bytes);
+                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
                 const unsigned short *oval = oidx + p.topk;
 #pragma unroll
                 for (int n = 0; n < KT; n++) {
@@ -1186,7 +910,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             }
         }
         if (KT > 0 && tid == 0) {
-            const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + p.codes_off + p.code_bytes);
+            const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
             bool bad = false;
             for (int n = 0; n < p.topk; n++) bad |= oidx[n] >= d;
             if (bad && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
@@ -1216,44 +940,6 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
 // ------------------------------------------------------------------------------------------------
 // host side: launch plumbing
 // ------------------------------------------------------------------------------------------------
-struct DeviceInfo {
-    int sms = 0;
-    int max_smem_optin = 0;
-};
-static int device_info(DeviceInfo *out) {
-    static DeviceInfo cache[64];
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RAC_ECUDA;
-    if (cache[dev].sms == 0) {
-        int sms = 0, smem = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RAC_ECUDA;
-        if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return RAC_ECUDA;
-        cache[dev].max_smem_optin = smem;
-        cache[dev].sms = sms;
-    }
-    *out = cache[dev];
-    return RAC_OK;
-}
-
-template <typename K>
-static int launch_persistent(K kernel, const CodecParams &p, int nthreads, int smem_bytes, long long max_ctas,
-                             cudaStream_t stream) {
-    DeviceInfo di;
-    int rc = device_info(&di);
-    if (rc != RAC_OK) return rc;
-    if (smem_bytes > di.max_smem_optin) return RAC_EUNSUPPORTED;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return RAC_ECUDA;
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, nthreads, smem_bytes) != cudaSuccess || occ < 1)
-        return RAC_ECUDA;
-    long long grid = (long long)di.sms * occ;
-    if (grid > max_ctas) grid = max_ctas;
-    if (grid < 1) grid = 1;
-    kernel<<<(unsigned)grid, nthreads, smem_bytes, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
-}
-
-static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int fill_common(const Geometry &g, CodecParams *p, long long T, const void *ref_base, long long ref_rows,
                        const int32_t *ref_row, const void *gain, const void *bias, uint32_t *status) {
@@ -1278,40 +964,38 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     p->topk = g.topk;
     p->rec = g.rec;
     p->code_bytes = g.code_bytes;
-    p->codes_off = g.codes_off;
     p->inv_group = 1.0f / (float)g.group;
+    p->Jq = g.Jq;
+    p->lpq = g.lpq;
+    p->lpq_shift = 0;
+    while ((1 << p->lpq_shift) < g.lpq) p->lpq_shift++;
+    p->kg = g.topk_group;
+    p->codes_off = g.codes_off;
+    p->goff_off = g.goff_off;
+    p->gval_off = g.gval_off;
     return RAC_OK;
-}
-
-// Ring depth.  RAC_STAGES (2..4) overrides the default for tuning runs.
-static int pick_stages(int d, int dflt) {
-    const char *e = getenv("RAC_STAGES");
-    if (e && e[0] >= '2' && e[0] <= '4' && e[1] == 0) return e[0] - '0';
-    (void)d;
-    return dflt;
 }
 
 // Encode: the streaming kernel, then (with outliers) the selection kernel.  Variant 4 of the streaming kernel
 // caps registers at 96 so that four 160-thread CTAs fit on an SM.
 static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
+    if (g.scale_mode == 1) return launch_encode_dyn(g, p, max_ctas, stream);
     const bool topk = g.topk > 0;
     p.stages = pick_stages(g.d, 2);
     WsSmem L = ws_smem_layout(g.d, g.rec, p.stages, topk);
     // With x_hat the kernel reads both step tables every token; at four CTAs per SM the shared-memory carve-out
     // leaves too little L1 for them, so that variant runs three CTAs per SM at 128 registers.
-    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && (!p.X_hat || g.scale_mode == 1) && !getenv("RAC_ENC_WIDE");
+    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
     int rc = RAC_EUNSUPPORTED;
-#define RAC_ENC3(B, K, X, D)                                                                                       \
-    (tight ? launch_persistent(encode_ws_kernel<B, K, X, D, 4>, p, g.nthreads, L.total, max_ctas, stream)         \
-           : launch_persistent(encode_ws_kernel<B, K, X, D, 2>, p, g.nthreads, L.total, max_ctas, stream))
-#define RAC_ENC2(B, K, X) (g.scale_mode == 1 ? RAC_ENC3(B, false, X, true) : RAC_ENC3(B, K, X, false))
+#define RAC_ENC2(B, K, X)                                                                                          \
+    (tight ? launch_persistent(encode_ws_kernel<B, K, X, 4>, p, g.nthreads, L.total, max_ctas, stream)            \
+           : launch_persistent(encode_ws_kernel<B, K, X, 2>, p, g.nthreads, L.total, max_ctas, stream))
 #define RAC_ENC(B, K) (p.X_hat ? RAC_ENC2(B, K, true) : RAC_ENC2(B, K, false))
     switch (g.bits) {
         case 4: rc = topk ? RAC_ENC(4, true) : RAC_ENC(4, false); break;
         case 3: rc = topk ? RAC_ENC(3, true) : RAC_ENC(3, false); break;
         case 2: rc = topk ? RAC_ENC(2, true) : RAC_ENC(2, false); break;
     }
-#undef RAC_ENC3
 #undef RAC_ENC2
 #undef RAC_ENC
     if (rc != RAC_OK || !topk) return rc;
@@ -1337,12 +1021,11 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
 }
 
 static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream) {
+    if (g.scale_mode == 1) return launch_decode_dyn(g, p, stream);
     p.stages = pick_stages(g.d, 2);
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
-#define RAC_DEC(B, K)                                                                                  \
-    (g.scale_mode == 1 ? launch_persistent(decode_kernel<B, K, true>, p, g.nthreads, L.total, p.T, stream) \
-                       : launch_persistent(decode_kernel<B, K, false>, p, g.nthreads, L.total, p.T, stream))
+#define RAC_DEC(B, K) launch_persistent(decode_kernel<B, K>, p, g.nthreads, L.total, p.T, stream)
     switch (g.bits * 100 + kt) {
         case 400: return RAC_DEC(4, 0);
         case 408: return RAC_DEC(4, 8);
@@ -1370,7 +1053,7 @@ static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64
     rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, gain, bias, dev_status);
     if (rc != RAC_OK) return rc;
     if (T == 0) return RAC_OK;
-    if (!payload || !X_hat || (!step && g.scale_mode == 0)) return RAC_EINVAL;
+    if (!payload || !X_hat || (!step && g.scale_mode == 0)) return RAC_EINVAL;   // mode 1 reads no table
     if (!aligned16(payload) || !aligned16(X_hat) || (step && !aligned16(step))) return RAC_EALIGN;
     p.payload = const_cast<uint8_t *>(static_cast<const uint8_t *>(payload));
     p.X_hat = static_cast<uint16_t *>(X_hat);
@@ -1494,6 +1177,7 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, cons
     CodecParams p = {};
     rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, dev_status);
     if (rc != RAC_OK) return rc;
+    if (g.scale_mode != 0) return RAC_EUNSUPPORTED;   // the tables belong to the static quantiser only
     if (!step || !inv_step || !workspace || !(clip_sigmas > 0.f)) return RAC_EINVAL;
     if (T > 0 && !X) return RAC_EINVAL;
     if (!aligned16(X) || !aligned16(workspace) || !aligned16(step) || !aligned16(inv_step)) return RAC_EALIGN;

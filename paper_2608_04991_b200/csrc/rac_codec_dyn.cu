@@ -1,0 +1,592 @@
+// RAC codec kernels for sm_100a, the quantiser family of Sec. IV-C as printed (scale_mode 1):
+//   * Eq. 8: per quantisation group the scale s = RoundUp_binary16(max|E^d| / Qmax) travels in the record, an
+//     all-zero group carries scale 0 ("zero marker") and skips the division, nothing clips;
+//   * the quantisation group g_q may differ from the alignment group g_a; g_q = d is the decode mode of the
+//     paper (one scale per token);
+//   * code widths 2, 3, 4 and 8;
+//   * the outlier mask of "Outlier Metadata": the k_g largest |e| of every quantisation group leave the dense
+//     base (E^d = E - O) BEFORE the scale is taken, and travel as one-byte in-group offsets (ascending) plus
+//     binary16 values.
+//
+// Same streaming shape as the static-table kernels: persistent CTAs, a token per CTA iteration, a thread per 32
+// channels, rows in and records out as 1-D bulk copies, bounded mbarrier waits, no CTA barrier in the loop; the
+// finished record is handed over by a rotating duty warp.  Because the outliers are picked per GROUP, the
+// selection fits into the streaming pass: a group is 1 to 8 lanes of one warp, so k_g rounds of "largest
+// magnitude of the group, lowest channel among equals" need only warp shuffles.  The token-wide scale is the
+// one place where warps must meet: they exchange their maxima through shared memory and a third mbarrier.
+#include "rac_codec_dev.cuh"
+
+namespace rac {
+
+struct DynCtrl {
+    unsigned long long full[kMaxStages];    // data of the stage has landed
+    unsigned long long done[kMaxStages];    // every warp has finished its share of the token in the stage
+    unsigned long long tokmax[kMaxStages];  // every warp has published its largest |e| of the token
+    int row[kMaxStages];
+    int abort;
+    float wmax[kMaxStages][8];
+};
+
+struct DynSmem {
+    int stage0, stage_bytes, rec_off, total;
+};
+__host__ __device__ inline DynSmem dyn_smem_layout(int d, int rec, int stages) {
+    DynSmem s;
+    s.stage0 = align_up((int)sizeof(DynCtrl), 128);
+    s.rec_off = 4 * d;  // after X row + R row: two record slots, used alternately (by the stage's parity)
+    s.stage_bytes = align_up(s.rec_off + 2 * rec, 128);
+    s.total = s.stage0 + stages * s.stage_bytes;
+    return s;
+}
+
+__device__ __forceinline__ uint32_t rotl32(uint32_t v, int n) { return __funnelshift_l(v, v, n); }
+__device__ __forceinline__ uint32_t rotr32(uint32_t v, int n) { return __funnelshift_r(v, v, n); }
+
+// codes of the 8 channels of one slot -> BITS bytes (one word, or two for 8-bit codes)
+template <int BITS>
+__device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, uint32_t &w1) {
+    // t[i]: binary32 bit pattern of (code + 1.5*2^23): the low mantissa bits hold the code in two's complement
+    if constexpr (BITS == 8) {
+        w0 = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
+        w1 = __byte_perm(__byte_perm(t[4], t[5], 0x0040), __byte_perm(t[6], t[7], 0x0040), 0x5410);
+    } else {
+        w0 = pack8<BITS>(t);
+        w1 = 0;
+    }
+}
+
+template <int BITS, bool XHAT, bool KG>
+__global__ void __launch_bounds__(256, 2) encode_dyn_kernel(const CodecParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int rot = (lane >> 1) & 3;
+    const int d = p.d;
+    const bool valid = tid * 32 < d;
+    const bool qtok = p.lpq == 0;
+    const DynSmem L = dyn_smem_layout(d, p.rec, p.stages);
+    DynCtrl *ctrl = reinterpret_cast<DynCtrl *>(smem);
+    const uint32_t sbase = smem_u32(smem);
+    const int S = p.stages;
+    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
+    constexpr int WPT = BITS;  // code words per thread (32 channels)
+    const uint32_t row_bytes = 2u * (uint32_t)d;
+
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+    auto raw_row_of = [&](int k) -> int {
+        long long t = first + (long long)k * stride;
+        return p.ref_row ? p.ref_row[t] : (int)t;
+    };
+    auto issue = [&](int k, int s, int raw_row) {
+        const long long t = first + (long long)k * stride;
+        const int row = resolve_row(p, raw_row);
+        ctrl->row[s] = row;
+        const uint32_t bar = smem_u32(&ctrl->full[s]);
+        const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
+        mbar_arrive_expect_tx(bar, row_bytes + (row >= 0 ? row_bytes : 0u));
+        bulk_load(base, p.X + t * d, row_bytes, bar);
+        if (row >= 0) bulk_load(base + row_bytes, p.ref_base + (long long)row * d, row_bytes, bar);
+    };
+
+    if (tid == 0) {
+        for (int s = 0; s < S; s++) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->done[s]), nwarps);
+            mbar_init(smem_u32(&ctrl->tokmax[s]), nwarps);
+        }
+        ctrl->abort = 0;
+        mbar_init_fence();
+    }
+    // padding bytes of the record slots are zero from here on: every field is rewritten per token, the gaps never
+    for (int s = 0; s < S; s++)
+        for (int o = 4 * tid; o < 2 * p.rec; o += 4 * nt)
+            *reinterpret_cast<uint32_t *>(smem + L.stage0 + s * L.stage_bytes + L.rec_off + o) = 0u;
+    __syncthreads();
+    if (tid == 0)
+        for (int k = 0; k < S && k < n_my; k++) issue(k, k, raw_row_of(k));
+
+    uint32_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
+    const unsigned int group_mask = __ballot_sync(0xffffffffu, valid);
+    const u64 magic2 = pack2(kMagic, kMagic);
+    const int qbase = lane & ~(p.lpq - 1);              // first lane of this lane's quantisation group (lpq > 0)
+    const uint32_t qlanes = p.lpq >= 32 ? 0xffffffffu : ((1u << p.lpq) - 1u);
+    const int jq = qtok ? 0 : (tid >> p.lpq_shift);     // quantisation group of this thread
+
+    int stage = 0, duty = 0;
+    uint32_t parity = 0;
+    bool timed_out = false;
+    for (int it = 0; it < n_my; it++) {
+        if (*reinterpret_cast<volatile int *>(&ctrl->abort)) break;
+        unsigned char *stg = smem + L.stage0 + stage * L.stage_bytes;
+        const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
+        const uint32_t rs = xs + row_bytes;
+        unsigned char *rec = stg + L.rec_off + parity * p.rec;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
+        const bool has_ref = ctrl->row[stage] >= 0;
+
+        float e[32];       // Eq. 7 residual of this thread's channels, slot order: e[8j + k] is channel 8*((j+rot)&3) + k
+        u64 r2[16];        // aligned-reference inputs, kept for the sender-side reconstruction
+        u64 a2 = 0ull, b2 = 0ull;
+        uint32_t sel[4] = {0u, 0u, 0u, 0u};   // per round: in-group offset | binary16 value << 16 (same in every lane of the group)
+        uint32_t own = 0;                      // rounds whose outlier lives in this thread
+        float m = 0.f;
+        if (valid) {
+            u64 x2[16];
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                uint4 w = lds128(xs + off[j]);
+                x2[4 * j + 0] = bf16x2_to_p(w.x);
+                x2[4 * j + 1] = bf16x2_to_p(w.y);
+                x2[4 * j + 2] = bf16x2_to_p(w.z);
+                x2[4 * j + 3] = bf16x2_to_p(w.w);
+            }
+            if (has_ref) {
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    u64 rr[4];
+                    load_ref_slot(rs + off[j], p.gain, p.bias, (int)(off[j] >> 1), rr);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[4 * j + i] = rr[i];
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; i++) r2[i] = 0ull;
+            }
+            uint32_t coef_word;
+            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
+            if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
+#pragma unroll
+            for (int i = 0; i < 16; i++) unpack2(psub(x2[i], pfma(a2, r2[i], b2)), e[2 * i], e[2 * i + 1]);
+
+            // ---- outlier mask: k_g rounds of (largest |e| of the group, lowest channel among equals)
+            if (KG) {
+                uint32_t taken = 0;  // slot order
+#pragma unroll
+                for (int n = 0; n < 4; n++) {
+                    if (n < p.kg) {
+                        float gm = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; i++) gm = fmaxf(gm, fabsf(e[i]));   // taken elements are 0 by now
+#pragma unroll
+                        for (int o = 1; o < 8; o <<= 1)
+                            if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
+                        uint32_t eq = 0;
+#pragma unroll
+                        for (int i = 0; i < 32; i++) eq |= (fabsf(e[i]) == gm) ? (1u << i) : 0u;
+                        eq &= ~taken;                                // a taken element ties only when the maximum is 0
+                        const uint32_t eqc = rotl32(eq, 8 * rot);    // channel order within the slab
+                        const uint32_t gb = (__ballot_sync(group_mask, eqc != 0u) >> qbase) & qlanes;
+                        const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);
+                        const bool mine = lane == owner && eqc != 0u;
+                        const int cl = eqc ? __ffs(eqc) - 1 : 0;     // channel within the slab
+                        const uint32_t hit = mine ? rotr32(1u << cl, 8 * rot) : 0u;
+                        float val = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; i++) {
+                            const bool h = (hit >> i) & 1u;
+                            val = h ? e[i] : val;
+                            e[i] = h ? 0.f : e[i];                   // E^d = E - O
+                        }
+                        taken |= hit;
+                        const uint32_t word = (uint32_t)((lane - qbase) * 32 + cl) | (float_to_half_bits_sat(val) << 16);
+                        sel[n] = __shfl_sync(group_mask, word, owner);
+                        if (mine) own |= 1u << n;
+                    }
+                }
+                if ((lane & (p.lpq - 1)) == 0) {
+                    // the group's first lane serialises them in ascending offset order
+                    unsigned char *go = rec + p.goff_off + jq * p.kg;
+                    unsigned short *gv = reinterpret_cast<unsigned short *>(rec + p.gval_off) + jq * p.kg;
+#pragma unroll
+                    for (int n = 0; n < 4; n++) {
+                        if (n < p.kg) {
+                            int rank = 0;
+#pragma unroll
+                            for (int q = 0; q < 4; q++)
+                                if (q < p.kg && (sel[q] & 0xffffu) < (sel[n] & 0xffffu)) rank++;
+                            go[rank] = (unsigned char)(sel[n] & 0xffu);
+                            gv[rank] = (unsigned short)(sel[n] >> 16);
+                        }
+                    }
+                }
+            }
+            // ---- largest dense magnitude of this thread, then of its group
+#pragma unroll
+            for (int i = 0; i < 32; i++) m = fmaxf(m, fabsf(e[i]));
+            if (!qtok) {
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1)
+                    if (p.lpq > o) m = fmaxf(m, __shfl_xor_sync(group_mask, m, o));
+            }
+        }
+        if (qtok) {
+            // one scale per token: the warps meet once
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            if (lane == 0) {
+                ctrl->wmax[stage][warp] = m;
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&ctrl->tokmax[stage])) : "memory");
+            }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->tokmax[stage]), parity))) { timed_out = true; break; }
+            for (int w = 0; w < nwarps; w++) m = fmaxf(m, *reinterpret_cast<volatile float *>(&ctrl->wmax[stage][w]));
+        }
+
+        if (valid) {
+            // ---- Eq. 8: s = RoundUp_binary16(m / Qmax): round to nearest, then one step up if that fell short
+            const float s_star = __fdiv_rn(m, qmax);
+            uint32_t s16 = float_to_half_bits_sat(s_star);
+            if (half_bits_to_float(s16) < s_star && s16 < 0x7bffu) s16++;
+            const float sc = half_bits_to_float(s16);
+            const float isc = sc != 0.f ? __fdiv_rn(1.0f, sc) : 0.f;   // zero marker: no division, codes 0
+            const u64 inv2 = pack2(isc, isc), s2 = pack2(sc, sc);
+            if (qtok ? tid == 0 : (lane & (p.lpq - 1)) == 0)
+                reinterpret_cast<unsigned short *>(rec + 4 * p.J)[jq] = (unsigned short)s16;
+
+            uint32_t words[4][2];
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                uint32_t t8[8], xh[4];
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    float v0, v1;
+                    unpack2(pmul(pack2(e[8 * j + 2 * i], e[8 * j + 2 * i + 1]), inv2), v0, v1);
+                    v0 = fminf(fmaxf(v0, -qmax), qmax);
+                    v1 = fminf(fmaxf(v1, -qmax), qmax);
+                    const u64 tt = padd(pack2(v0, v1), magic2);
+                    float t0, t1;
+                    unpack2(tt, t0, t1);
+                    t8[2 * i] = __float_as_uint(t0);
+                    t8[2 * i + 1] = __float_as_uint(t1);
+                    if (XHAT) {
+                        // Eq. 9 with the code just chosen: x_hat = bf16((alpha*r + beta) + q*s)
+                        float x0, x1;
+                        unpack2(padd(pfma(a2, r2[4 * j + i], b2), pmul(psub(tt, magic2), s2)), x0, x1);
+                        xh[i] = f2_to_bf16x2(x0, x1);
+                    }
+                }
+                pack_slot<BITS>(t8, words[j][0], words[j][1]);
+                if (XHAT) sts128(xs + off[j], make_uint4(xh[0], xh[1], xh[2], xh[3]));
+            }
+            // slot order -> piece order (words[q] becomes the code word(s) of piece q)
+            {
+                uint32_t lo[4] = {words[0][0], words[1][0], words[2][0], words[3][0]};
+                rot_right4(lo, rot);
+                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + p.codes_off) + tid * WPT;
+                if (BITS == 8) {
+                    uint32_t hi[4] = {words[0][1], words[1][1], words[2][1], words[3][1]};
+                    rot_right4(hi, rot);
+#pragma unroll
+                    for (int q = 0; q < 4; q++) { cw[2 * q] = lo[q]; cw[2 * q + 1] = hi[q]; }
+                } else if (BITS == 4) {
+                    cw[0] = lo[0]; cw[1] = lo[1]; cw[2] = lo[2]; cw[3] = lo[3];
+                } else if (BITS == 3) {
+                    cw[0] = lo[0] | (lo[1] << 24);
+                    cw[1] = (lo[1] >> 8) | (lo[2] << 16);
+                    cw[2] = (lo[2] >> 16) | (lo[3] << 8);
+                } else {
+                    cw[0] = lo[0] | (lo[1] << 16);
+                    cw[1] = lo[2] | (lo[3] << 16);
+                }
+            }
+            if (KG && XHAT && own) {
+                // the outliers this thread owns: x_hat = bf16((alpha*r + beta) + binary16 value)
+                float a, b, unused;
+                unpack2(a2, a, unused);
+                unpack2(b2, b, unused);
+#pragma unroll
+                for (int n = 0; n < 4; n++) {
+                    if ((own >> n) & 1u) {
+                        const int c = jq * (p.lpq * 32) + (int)(sel[n] & 0xffffu);
+                        float r = 0.f;
+                        if (has_ref) {
+                            r = __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(stg + row_bytes + 2 * c)) << 16);
+                            if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                        }
+                        const float x = __fadd_rn(__fmaf_rn(a, r, b), half_bits_to_float(sel[n] >> 16));
+                        reinterpret_cast<unsigned short *>(stg)[c] = __bfloat16_as_ushort(__float2bfloat16_rn(x));
+                    }
+                }
+            }
+        }
+        // this warp's share of the token is in shared memory: one arrival per warp
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&ctrl->done[stage])) : "memory");
+
+        if (warp == duty) {
+            const int k_next = it + S;
+            int raw_next = 0;
+            if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
+            // The record sits in the slot of the stage's current parity; the stage's next token writes the other
+            // slot, and the one after that cannot start before this warp has arrived for the token in between.
+            // With x_hat the X row itself is the source of a store and must have been read before the refill.
+            if (lane == 0) {
+                const long long t = first + (long long)it * stride;
+                if (XHAT) {
+                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_store(p.X_hat + t * d, xs, row_bytes);
+                    bulk_commit();
+                    bulk_wait_read<0>();
+                    if (k_next < n_my) issue(k_next, stage, raw_next);
+                } else {
+                    if (k_next < n_my) issue(k_next, stage, raw_next);
+                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_commit();
+                    bulk_wait_read<0>();
+                }
+            }
+            __syncwarp();
+        }
+        if (++stage == S) { stage = 0; parity ^= 1u; }
+        if (++duty == nwarps) duty = 0;
+    }
+    if (timed_out) {
+        ctrl->abort = 1;
+        if (p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
+    }
+    __syncthreads();
+    if (lane == 0) bulk_wait_all();
+    if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
+        for (int s = 0; s < S; s++) {
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// reconstruct (receiver and sender), Eq. 9 with the record's own scales
+// ------------------------------------------------------------------------------------------------
+// Same shape as the static-table reconstruction: record and reference row arrive in a stage, every thread
+// dequantises its 32 channels (code -> binary32 through the 2^23 trick, times its group's scale), adds the
+// aligned reference, rounds to bf16 into an output row in shared memory; then the per-group outliers replace
+// what the dense pass wrote, and the row leaves as one bulk store.
+template <int BITS, bool KG>
+__global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int rot = (lane >> 1) & 3;
+    const int d = p.d;
+    const bool valid = tid * 32 < d;
+    const DecSmem L = dec_smem_layout(d, p.rec, p.stages);
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
+    const uint32_t sbase = smem_u32(smem);
+    const int S = p.stages;
+    constexpr int WPT = BITS;                     // code words per thread
+    constexpr int WPP = BITS == 8 ? 2 : 1;        // code words per piece of 8 channels
+    constexpr int FPW = 8 / WPP;                  // fields per word
+    constexpr uint32_t cmask = (BITS == 8) ? 0xffu : ((1u << BITS) - 1u);
+    constexpr uint32_t H = 1u << (BITS - 1);
+    constexpr uint32_t ones = (BITS == 8) ? 0x01010101u : (BITS == 4) ? 0x11111111u : (BITS == 3) ? 0x00249249u : 0x00005555u;
+    constexpr uint32_t highs = ones << (BITS - 1);
+    constexpr float kBase = 8388608.0f + (float)H;  // 2^23 + H
+    const uint32_t row_bytes = 2u * (uint32_t)d;
+    const int jq = p.lpq == 0 ? 0 : (tid >> p.lpq_shift);
+
+    if (tid == 0) {
+        for (int s = 0; s < S; s++) mbar_init(smem_u32(&ctrl->bar[s]), 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+
+    int next_raw = 0;
+    auto raw_row_of = [&](int k) -> int {
+        long long t = first + (long long)k * stride;
+        return p.ref_row ? p.ref_row[t] : (int)t;
+    };
+    if (tid == 0) {
+        for (int k = 0; k < S - 1 && k < n_my; k++) {
+            long long t = first + (long long)k * stride;
+            issue_token_loads(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row(p, raw_row_of(k)),
+                              p.payload + t * p.rec, (uint32_t)p.rec);
+        }
+        if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
+    }
+
+    uint32_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
+    const u64 base2 = pack2(kBase, kBase);
+
+    int stage = 0, obuf = 0, issue_stage = S - 1;
+    bool aborted = false;
+    uint32_t parity = 0;
+    for (int it = 0; it < n_my; it++) {
+        const long long t = first + (long long)it * stride;
+        if (tid == 0 && it + S - 1 < n_my) {
+            const int k = it + S - 1;
+            const long long tk = first + (long long)k * stride;
+            issue_token_loads(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
+                              resolve_row(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
+            if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
+        }
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
+        if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
+        const bool has_ref = ctrl->row[stage] >= 0;
+        const unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
+        const uint32_t rs = sbase + L.stage0 + stage * L.stage_bytes + L.rec_pad;
+        unsigned char *ob = smem + L.out0 + obuf * (int)row_bytes;
+        const uint32_t obs = smem_u32(ob);
+
+        if (valid) {
+            const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
+            const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
+            const u64 a2 = pack2(a, a), b2 = pack2(b, b);
+            const float sc = half_bits_to_float(reinterpret_cast<const unsigned short *>(rec + 4 * p.J)[jq]);
+            const u64 s2 = pack2(sc, sc);
+            // code words of the four pieces, in piece order, then rotated into slot order
+            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + p.codes_off) + tid * WPT;
+            uint32_t lo[4], hi[4] = {0u, 0u, 0u, 0u};
+            if (BITS == 8) {
+#pragma unroll
+                for (int q = 0; q < 4; q++) { lo[q] = cw[2 * q]; hi[q] = cw[2 * q + 1]; }
+            } else if (BITS == 4) {
+                lo[0] = cw[0]; lo[1] = cw[1]; lo[2] = cw[2]; lo[3] = cw[3];
+            } else if (BITS == 3) {
+                uint32_t w0 = cw[0], w1 = cw[1], w2 = cw[2];
+                lo[0] = w0 & 0xffffffu;
+                lo[1] = (w0 >> 24) | ((w1 & 0xffffu) << 8);
+                lo[2] = (w1 >> 16) | ((w2 & 0xffu) << 16);
+                lo[3] = w2 >> 8;
+            } else {
+                uint32_t w0 = cw[0], w1 = cw[1];
+                lo[0] = w0 & 0xffffu; lo[1] = w0 >> 16; lo[2] = w1 & 0xffffu; lo[3] = w1 >> 16;
+            }
+            uint32_t reserved = 0;
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                uint32_t v = lo[q] ^ highs;  // field == 0  <=>  code == -2^(BITS-1)
+                reserved |= (v - ones) & ~v & highs;
+                lo[q] = v;                   // fields now hold code + H (offset binary)
+                if (BITS == 8) {
+                    v = hi[q] ^ highs;
+                    reserved |= (v - ones) & ~v & highs;
+                    hi[q] = v;
+                }
+            }
+            if (reserved && p.status) atomicOr(p.status, RAC_STATUS_RESERVED_CODE);
+            rot_left4(lo, rot);
+            if (BITS == 8) rot_left4(hi, rot);
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                const int c = (int)(off[j] >> 1);
+                u64 r2[4];
+                if (has_ref) {
+                    load_ref_slot(rs + off[j], p.gain, p.bias, c, r2);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[i] = 0ull;
+                }
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    // exact integer -> binary32 without a convert: 2^23 + (code + H), minus (2^23 + H)
+                    const int f0 = 2 * i, f1 = 2 * i + 1;
+                    const uint32_t w0 = (f0 < FPW) ? lo[j] : hi[j];
+                    const uint32_t w1 = (f1 < FPW) ? lo[j] : hi[j];
+                    const float q0 = __uint_as_float(0x4b000000u | ((w0 >> (BITS * (f0 % FPW))) & cmask));
+                    const float q1 = __uint_as_float(0x4b000000u | ((w1 >> (BITS * (f1 % FPW))) & cmask));
+                    const u64 eh = pmul(psub(pack2(q0, q1), base2), s2);
+                    float x0, x1;
+                    unpack2(padd(pfma(a2, r2[i], b2), eh), x0, x1);
+                    o[i] = f2_to_bf16x2(x0, x1);
+                }
+                sts128(obs + off[j], make_uint4(o[0], o[1], o[2], o[3]));
+            }
+            if (KG) {
+                // outliers of this thread's group that fall into its own 32 channels, in record order
+                const unsigned char *go = rec + p.goff_off + jq * p.kg;
+                const unsigned short *gv = reinterpret_cast<const unsigned short *>(rec + p.gval_off) + jq * p.kg;
+                const int qsize = p.lpq * 32;
+                bool bad = false;
+#pragma unroll
+                for (int n = 0; n < 4; n++) {
+                    if (n < p.kg) {
+                        const int o = go[n];
+                        if (o >= qsize) {
+                            bad = true;
+                        } else if ((o >> 5) == (tid & (p.lpq - 1))) {
+                            const int c = jq * qsize + o;
+                            float r = 0.f;
+                            if (has_ref) {
+                                r = __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(rec + L.rec_pad + 2 * c)) << 16);
+                                if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                            }
+                            const float xh = __fadd_rn(__fmaf_rn(a, r, b), half_bits_to_float(gv[n]));
+                            reinterpret_cast<unsigned short *>(ob)[c] = __bfloat16_as_ushort(__float2bfloat16_rn(xh));
+                        }
+                    }
+                }
+                if (bad && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
+            }
+        }
+        fence_async_smem();
+        if (__syncthreads_or(timed_out)) { aborted = true; break; }  // one vote: every thread leaves together
+        if (tid == 0) {
+            bulk_store(p.X_hat + t * d, obs, row_bytes);
+            bulk_commit();
+            bulk_wait_read<1>();
+        }
+        if (++stage == S) { stage = 0; parity ^= 1u; }
+        if (++issue_stage == S) issue_stage = 0;
+        if (++obuf == kRecBufs) obuf = 0;
+    }
+    if (tid == 0) {
+        bulk_wait_all();
+        if (aborted) {
+            for (int s = 0; s < S; s++) {
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+int launch_encode_dyn(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
+    p.stages = pick_stages(g.d, 2);
+    const DynSmem L = dyn_smem_layout(g.d, g.rec, p.stages);
+    const bool kg = g.topk_group > 0;
+#define RAC_DYN_ENC2(B, X) \
+    (kg ? launch_persistent(encode_dyn_kernel<B, X, true>, p, g.nthreads, L.total, max_ctas, stream) \
+        : launch_persistent(encode_dyn_kernel<B, X, false>, p, g.nthreads, L.total, max_ctas, stream))
+#define RAC_DYN_ENC(B) (p.X_hat ? RAC_DYN_ENC2(B, true) : RAC_DYN_ENC2(B, false))
+    switch (g.bits) {
+        case 8: return RAC_DYN_ENC(8);
+        case 4: return RAC_DYN_ENC(4);
+        case 3: return RAC_DYN_ENC(3);
+        case 2: return RAC_DYN_ENC(2);
+    }
+#undef RAC_DYN_ENC
+#undef RAC_DYN_ENC2
+    return RAC_EUNSUPPORTED;
+}
+
+int launch_decode_dyn(const Geometry &g, CodecParams &p, cudaStream_t stream) {
+    p.stages = pick_stages(g.d, 2);
+    const DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
+    const bool kg = g.topk_group > 0;
+#define RAC_DYN_DEC(B) \
+    (kg ? launch_persistent(decode_dyn_kernel<B, true>, p, g.nthreads, L.total, p.T, stream) \
+        : launch_persistent(decode_dyn_kernel<B, false>, p, g.nthreads, L.total, p.T, stream))
+    switch (g.bits) {
+        case 8: return RAC_DYN_DEC(8);
+        case 4: return RAC_DYN_DEC(4);
+        case 3: return RAC_DYN_DEC(3);
+        case 2: return RAC_DYN_DEC(2);
+    }
+#undef RAC_DYN_DEC
+    return RAC_EUNSUPPORTED;
+}
+
+}  // namespace rac

@@ -138,12 +138,18 @@ __device__ __forceinline__ uint32_t float_to_half_bits_sat(float v) {
 // ---------------------------------------------------------------------------------------------
 struct Geometry {
     int d, group, bits, topk;
-    int J;          // groups per token
-    int lpg;        // lanes per group (group / 32)
+    int J;          // alignment groups per token
+    int lpg;        // lanes per alignment group (group / 32)
     int nthreads;   // threads per CTA: one per 32 channels, rounded up to whole warps
     int code_bytes; // d*bits/8
-    int scale_mode; // 0: static per-channel step table, 1: per-group binary16 scale in the record (Eq. 8)
-    int codes_off;  // byte offset of the codes in a record: 4*J, plus the scales (2*J padded to 4) in mode 1
+    int scale_mode; // 0: static per-channel step table, 1: binary16 scales in the record (Eq. 8)
+    int qgroup;     // channels per quantisation group (scale_mode 1; == group in mode 0)
+    int Jq;         // quantisation groups per token
+    int lpq;        // lanes per quantisation group, 0 when the group is the whole token and d/32 is no power of two <= 32
+    int topk_group; // outliers per quantisation group (scale_mode 1)
+    int codes_off;  // byte offset of the codes in a record: 4*J, plus the scales (2*Jq padded to 4) in mode 1
+    int goff_off;   // byte offset of the per-group outlier offsets (Jq*topk_group bytes, padded to 2)
+    int gval_off;   // byte offset of the per-group outlier values (Jq*topk_group binary16)
     int rec;        // record stride in bytes
 };
 int make_geometry(const rac_codec_cfg *cfg, Geometry *g);  // RAC_OK or an error

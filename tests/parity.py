@@ -64,13 +64,15 @@ def _check_flips(name, gpu16, orc16, exact, window_abs):
 
 def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None, gain=None, bias=None,
                    step=None, inv_step=None) -> EncodeReport:
-    d, g, bits, k, sm = cfg.d, cfg.group, cfg.bits, cfg.topk, cfg.scale_mode
+    d, g, bits, k = cfg.d, cfg.group, cfg.bits, cfg.topk
+    mode = (cfg.scale_mode, cfg.qgroup, cfg.topk_group)
+    mk = dict(scale_mode=cfg.scale_mode, qgroup=cfg.qgroup, topk_group=cfg.topk_group)
     T = Xb.size // d
     nthr = oracle.max_threads()
     o_payload, dg = oracle.encode(d, g, bits, k, Xb, ref_base=ref_base, ref_row=ref_row, gain=gain, bias=bias,
-                                  step=step, inv_step=inv_step, diag=True, nthreads=nthr, scale_mode=sm)
-    g_coef = oracle.split_payload(gpu_payload, T, d, g, bits, k, sm)[0]
-    o_coef = oracle.split_payload(o_payload, T, d, g, bits, k, sm)[0]
+                                  step=step, inv_step=inv_step, diag=True, nthreads=nthr, **mk)
+    g_coef = oracle.split_payload(gpu_payload, T, d, g, bits, k, *mode)[0]
+    o_coef = oracle.split_payload(o_payload, T, d, g, bits, k, *mode)[0]
     ga, gb = (g_coef & 0xffff).astype(np.uint16), (g_coef >> 16).astype(np.uint16)
     oa, ob = (o_coef & 0xffff).astype(np.uint16), (o_coef >> 16).astype(np.uint16)
     # 1e-3 relative (with the floor of one binary16 subnormal, and for beta the cancellation in hbar - alpha*rbar)
@@ -88,9 +90,9 @@ def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None
         _check_flips("beta", gb[mb], ob[mb], b_exact[mb], cancel[mb])
     # stage 2: same coefficients -> everything else bit-identical
     forced = oracle.encode(d, g, bits, k, Xb, ref_base=ref_base, ref_row=ref_row, gain=gain, bias=bias,
-                           step=step, inv_step=inv_step, forced_coef=g_coef.reshape(-1).copy(), nthreads=nthr, scale_mode=sm)
+                           step=step, inv_step=inv_step, forced_coef=g_coef.reshape(-1).copy(), nthreads=nthr, **mk)
     if not np.array_equal(forced, gpu_payload):
-        rec = oracle.record_bytes(d, g, bits, k, sm)
+        rec = oracle.record_bytes(d, g, bits, k, *mode)
         bad = np.flatnonzero((forced.reshape(T, rec) != gpu_payload.reshape(T, rec)).any(axis=1))
         t = int(bad[0])
         off = np.flatnonzero(forced.reshape(T, rec)[t] != gpu_payload.reshape(T, rec)[t])
@@ -163,7 +165,9 @@ def round_trip_case(cfg, X, ref_base=None, ref_row=None, gain=None, bias=None, s
     """Full protocol on one input set (torch CUDA tensors; step tables numpy float32[2,d]).
     Returns (EncodeReport, gpu payload numpy, X_hat tensor)."""
     dev = X.device
-    d, g, bits, k, sm = cfg.d, cfg.group, cfg.bits, cfg.topk, cfg.scale_mode
+    d, g, bits, k = cfg.d, cfg.group, cfg.bits, cfg.topk
+    mode = (cfg.scale_mode, cfg.qgroup, cfg.topk_group)
+    mk = dict(scale_mode=cfg.scale_mode, qgroup=cfg.qgroup, topk_group=cfg.topk_group)
     T = X.shape[0]
     step_d, inv_d = to_dev(step, dev), to_dev(inv_step, dev)
     Xb = synth.bf16_bits(X)
@@ -185,14 +189,14 @@ def round_trip_case(cfg, X, ref_base=None, ref_row=None, gain=None, bias=None, s
     assert np.array_equal(pay_f, pay), "rac_encode_reconstruct payload differs from rac_encode"
     assert torch.equal(xs_f, xr), "fused sender reconstruction differs from the receiver's"
     o_x = oracle.reconstruct(d, g, bits, k, pay, T, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step,
-                             nthreads=oracle.max_threads(), scale_mode=sm)
+                             nthreads=oracle.max_threads(), **mk)
     assert np.array_equal(o_x, synth.bf16_bits(xr)), "device reconstruction differs from the oracle's"
     # and the device's decode of the ORACLE's own payload
     o_pay = oracle.encode(d, g, bits, k, Xb, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step, inv_step=inv_step,
-                          nthreads=oracle.max_threads(), scale_mode=sm)
+                          nthreads=oracle.max_threads(), **mk)
     xo, st = gpu_decode(cfg, o_pay, T, ref_base, ref_row, gain, bias, step_d, dev)
     o_xo = oracle.reconstruct(d, g, bits, k, o_pay, T, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step,
-                              nthreads=oracle.max_threads(), scale_mode=sm)
+                              nthreads=oracle.max_threads(), **mk)
     assert st == 0 and np.array_equal(o_xo, synth.bf16_bits(xo)), "device decode of the oracle payload differs"
     # spec tolerance on the end-to-end activations where no coefficient flipped (implied by the above,
     # stated explicitly): abs 2e-2 / rel 1e-2

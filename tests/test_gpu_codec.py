@@ -370,3 +370,74 @@ def test_dynamic_group_scale_identity_and_rejections(env):
     assert not scale.any() and not codes.any() and torch.equal(xr, X)        # zero-group marker everywhere
     assert env.rac.rac_record_bytes(env.rac.CodecCfg(d, g, 4, 8, scale_mode=1)) == 0   # outliers: not in this mode
     assert env.rac.rac_record_bytes(env.rac.CodecCfg(d, g, 4, 0, scale_mode=2)) == 0
+
+
+# --------------------------------------------------------------------------- the rest of the quantiser family (Sec. IV-C)
+@pytest.mark.parametrize("d,g,bits,qg,kg,T", [
+    (4096, 128, 4, 0, 1, 150),      # one outlier per group of 128
+    (4096, 128, 4, 0, 2, 65),
+    (4096, 128, 8, 0, 1, 65),       # 8-bit codes
+    (4096, 128, 8, 0, 0, 65),
+    (4096, 64, 3, 64, 4, 40),       # four rounds, groups of two lanes
+    (5120, 128, 4, 32, 1, 95),      # quantisation groups of one lane inside alignment groups of four
+    (5120, 128, 2, 256, 3, 50),     # quantisation groups of eight lanes spanning two alignment groups
+    (3584, 128, 4, 3584, 0, 64),    # decode mode: one scale per token, d/32 not a power of two
+    (3584, 128, 8, 3584, 0, 64),
+    (4096, 128, 3, 4096, 0, 33),
+    (1024, 128, 4, 1024, 0, 20),    # one scale per token inside one warp
+    (8192, 256, 8, 0, 2, 21),       # widest token, eight warps
+    (96, 32, 4, 32, 2, 9),          # a single partly filled warp
+    (96, 32, 8, 96, 0, 9),
+    (2080, 32, 4, 0, 1, 33),        # odd group counts: padding after scales and after offsets
+])
+def test_family_matches_oracle(env, d, g, bits, qg, kg, T):
+    X, R, _, _ = prefill_inputs(env, T, d, g, seed=3000 + d + bits + qg + kg)
+    cfg = env.rac.CodecCfg(d, g, bits, 0, scale_mode=1, qgroup=qg, topk_group=kg)
+    assert env.rac.rac_record_bytes(cfg) == env.orc.record_bytes(d, g, bits, 0, 1, qg, kg)
+    rep, pay, xr = env.P.round_trip_case(cfg, X, ref_base=R)
+    print(rep)
+    # direct tokens mixed in, and the gain/bias reference
+    rows = np.arange(T, dtype=np.int32)
+    rows[1::3] = -1
+    env.P.round_trip_case(cfg, X, ref_base=R, ref_row=torch.from_numpy(rows).to(env.dev))
+    gain, bias = env.synth.predictor_gain_bias(d, 5, env.dev)
+    env.P.round_trip_case(cfg, X, ref_base=R, gain=gain, bias=bias)
+
+
+def test_family_ties_zero_groups_and_bad_offsets(env):
+    d, g, T = 1024, 128, 12
+    s = env.synth
+    X = s.activations(T, d, s.channel_scale(d, 34, env.dev), s.generator(34, env.dev))
+    # reference == X: every residual is zero, every |e| ties: the outliers are the k_g lowest offsets, scales 0
+    cfg = env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=64, topk_group=3)
+    rep, pay, xr = env.P.round_trip_case(cfg, X, ref_base=X)
+    parts = env.orc.split_payload(pay, T, d, g, 4, 0, 1, 64, 3)
+    assert not parts[4].any() and not parts[1].any() and not parts[6].any()
+    assert np.array_equal(parts[5], np.tile(np.arange(3, dtype=np.uint8), (T, d // 64, 1)))
+    assert torch.equal(xr, X)
+    # a coarse grid of values: many equal magnitudes inside every group
+    rng = np.random.default_rng(35)
+    vals = (rng.integers(-6, 7, size=(T, d)) / 2).astype(np.float32)
+    Xg = torch.from_numpy(vals).to(torch.bfloat16).to(env.dev)
+    for kg in (1, 4):
+        env.P.round_trip_case(env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=128, topk_group=kg), Xg, ref_base=None)
+    # an offset outside its group: flagged, ignored, nothing else disturbed
+    cfg = env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=32, topk_group=1)
+    pay, st = env.P.gpu_encode(cfg, X, None, None, None, None, None, None)
+    good, st0 = env.P.gpu_decode(cfg, pay, T, None, None, None, None, None, env.dev)
+    bad = pay.copy().reshape(T, -1)
+    goff = 4 * (d // g) + 2 * (d // 32) + d // 2
+    keep = bad[3, goff + 5]
+    bad[3, goff + 5] = 40
+    xb, st1 = env.P.gpu_decode(cfg, bad.reshape(-1), T, None, None, None, None, None, env.dev)
+    assert st0 == 0 and st1 == 16
+    diff = (xb != good).nonzero().cpu().numpy()
+    assert len(diff) == 1 and diff[0][0] == 3 and diff[0][1] == 5 * 32 + keep   # only the outlier that was dropped
+    # configurations this build has no kernel for
+    for bad_cfg in [env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=512, topk_group=1),   # one-byte offsets
+                    env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, topk_group=5),
+                    env.rac.CodecCfg(d, g, 8, 0),                                           # 8 bits: Eq. 8 family only
+                    env.rac.CodecCfg(d, g, 4, 0, qgroup=64),                                # static table: g_q = g_a
+                    env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=96),
+                    env.rac.CodecCfg(d, g, 5, 0, scale_mode=1)]:
+        assert env.rac.rac_record_bytes(bad_cfg) == 0
