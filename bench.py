@@ -50,6 +50,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode-steps", action="store_true", help="skip the decode-step latency extra")
+    ap.add_argument("--no-family", action="store_true", help="skip the Eq. 8 quantiser-family extra")
     return ap.parse_args()
 
 
@@ -236,6 +237,50 @@ class RoundTrip:
 
     def activation_bytes_per_step(self):
         return 2 * 2 * self.wl["T"] * self.wl["d"]
+
+
+# --------------------------------------------------------------------------------------------- the paper's quantiser family
+def paper_family(dev, T, d, g=128, reps=10):
+    """Eq. 8 as printed (scale_mode 1) on the benchmark's shape: encode and reconstruct of a few members of the
+    family (per-group scales, k_g outliers per group, 8-bit codes, one scale per token), each timed alone with
+    CUDA events over `reps` launches after 3 warm-ups; GB/s over the algorithmic bytes (X + reference + record,
+    resp. record + reference + x_hat).  Inputs are larger than L2."""
+    import torch
+    from paper_2608_04991_b200 import binding as rac
+    from paper_2608_04991_b200 import synth
+    gen = synth.generator(synth.BASE_SEED + 9, dev)
+    X = synth.activations(T, d, synth.channel_scale(d, 9, dev), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    xh = torch.empty_like(X)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = []
+    for name, bits, qg, kg in (("4-bit, scale per group", 4, 0, 0), ("4-bit, 1 outlier per group", 4, 0, 1),
+                               ("4-bit, 2 outliers per group", 4, 0, 2), ("8-bit, scale per group", 8, 0, 0),
+                               ("4-bit, one scale per token", 4, d, 0)):
+        cfg = rac.CodecCfg(d, g, bits, 0, scale_mode=1, qgroup=qg, topk_group=kg)
+        rec = rac.rac_record_bytes(cfg)
+        pay = torch.empty(T * rec, dtype=torch.uint8, device=dev)
+        enc = lambda: rac.rac_encode(cfg, X, T, R, T, None, None, None, None, None, pay, pay.numel(), None, 0, status)
+        dec = lambda: rac.rac_decode_reconstruct(cfg, pay, T, R, T, None, None, None, None, xh, status)
+        row = {"member": name, "record_bytes": rec, "payload_over_raw": rec / (2.0 * d)}
+        for key, fn in (("encode", enc), ("reconstruct", dec)):
+            for _ in range(3):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            row[key + "_ms"] = ms
+            row[key + "_GBps"] = T * (4 * d + rec) / (ms * 1e-3) / 1e9
+        out.append(row)
+        del pay
+    if int(status.item()) != 0:
+        raise RuntimeError(f"paper_family: device status {int(status.item())}")
+    return out
 
 
 # --------------------------------------------------------------------------------------------- decode-step latency
@@ -568,6 +613,7 @@ def main():
             "cpu_baseline": cpu,
             "stages": per,
             "decode_steps": None if args.no_decode_steps else decode_step_latency(dev),
+            "paper_family": None if args.no_family else paper_family(dev, wl["T"], wl["d"]),
         }
         print(json.dumps(line))
     if world > 1:

@@ -42,6 +42,24 @@ __host__ __device__ inline DynSmem dyn_smem_layout(int d, int rec, int stages) {
 __device__ __forceinline__ uint32_t rotl32(uint32_t v, int n) { return __funnelshift_l(v, v, n); }
 __device__ __forceinline__ uint32_t rotr32(uint32_t v, int n) { return __funnelshift_r(v, v, n); }
 
+// largest magnitude of 8 values, leaving out those whose bit is set in `skip` (three-input maxima)
+__device__ __forceinline__ float abs_max8(const float (&e)[8], uint32_t skip) {
+    float v[8];
+#pragma unroll
+    for (int k = 0; k < 8; k++) v[k] = ((skip >> k) & 1u) ? 0.f : fabsf(e[k]);
+    float m0 = 0.f, m1 = 0.f;
+    asm("max.f32 %0, %0, %1, %2;" : "+f"(m0) : "f"(v[0]), "f"(v[1]));
+    asm("max.f32 %0, %0, %1, %2;" : "+f"(m1) : "f"(v[2]), "f"(v[3]));
+    asm("max.f32 %0, %0, %1, %2;" : "+f"(m0) : "f"(v[4]), "f"(v[5]));
+    asm("max.f32 %0, %0, %1, %2;" : "+f"(m1) : "f"(v[6]), "f"(v[7]));
+    return fmaxf(m0, m1);
+}
+// rotate the four entries right by rot (new[j] = old[(j - rot) & 3])
+__device__ __forceinline__ void rot_right4f(float (&w)[4], int rot) {
+    if (rot & 1) { float t = w[3]; w[3] = w[2]; w[2] = w[1]; w[1] = w[0]; w[0] = t; }
+    if (rot & 2) { float t = w[0]; w[0] = w[2]; w[2] = t; t = w[1]; w[1] = w[3]; w[3] = t; }
+}
+
 // codes of the 8 channels of one slot -> BITS bytes (one word, or two for 8-bit codes)
 template <int BITS>
 __device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, uint32_t &w1) {
@@ -55,8 +73,9 @@ __device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, 
     }
 }
 
-template <int BITS, bool XHAT, bool KG>
-__global__ void __launch_bounds__(256, 2) encode_dyn_kernel(const CodecParams p) {
+// MINB = 4 caps registers at 96 so that four 160-thread CTAs (d = 5120) fit on an SM.
+template <int BITS, bool XHAT, bool KG, int MINB>
+__global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
@@ -127,7 +146,7 @@ __global__ void __launch_bounds__(256, 2) encode_dyn_kernel(const CodecParams p)
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
-        float e[32];       // Eq. 7 residual of this thread's channels, slot order: e[8j + k] is channel 8*((j+rot)&3) + k
+        u64 e2[16];        // Eq. 7 residual of this thread's channels, packed pairs in slot order
         u64 r2[16];        // aligned-reference inputs, kept for the sender-side reconstruction
         u64 a2 = 0ull, b2 = 0ull;
         uint32_t sel[4] = {0u, 0u, 0u, 0u};   // per round: in-group offset | binary16 value << 16 (same in every lane of the group)
@@ -158,42 +177,68 @@ __global__ void __launch_bounds__(256, 2) encode_dyn_kernel(const CodecParams p)
             uint32_t coef_word;
             fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
             if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
+            // residual, and the largest magnitude of each slot of 8 channels
+            float sm[4];
 #pragma unroll
-            for (int i = 0; i < 16; i++) unpack2(psub(x2[i], pfma(a2, r2[i], b2)), e[2 * i], e[2 * i + 1]);
+            for (int j = 0; j < 4; j++) {
+                float ev[8];
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    e2[4 * j + i] = psub(x2[4 * j + i], pfma(a2, r2[4 * j + i], b2));
+                    unpack2(e2[4 * j + i], ev[2 * i], ev[2 * i + 1]);
+                }
+                sm[j] = abs_max8(ev, 0u);
+            }
 
-            // ---- outlier mask: k_g rounds of (largest |e| of the group, lowest channel among equals)
+            // ---- outlier mask: k_g rounds of (largest |e| of the group, lowest channel among equals).  The
+            // registers are left alone: the thread that holds the round's maximum finds the element by reading its
+            // piece of the rows in shared memory again (same operations, same bits), removes it from that slot's
+            // maximum, and the codes and x_hat of the outliers are patched after the dense pass.
             if (KG) {
-                uint32_t taken = 0;  // slot order
+                uint32_t taken = 0;  // channel order within the slab
 #pragma unroll
                 for (int n = 0; n < 4; n++) {
                     if (n < p.kg) {
-                        float gm = 0.f;
-#pragma unroll
-                        for (int i = 0; i < 32; i++) gm = fmaxf(gm, fabsf(e[i]));   // taken elements are 0 by now
+                        const float mloc = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
+                        float gm = mloc;
 #pragma unroll
                         for (int o = 1; o < 8; o <<= 1)
                             if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
-                        uint32_t eq = 0;
+                        const uint32_t gb = (__ballot_sync(group_mask, mloc == gm) >> qbase) & qlanes;
+                        const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);   // gb == 0 only with NaNs around
+                        uint32_t word = 0;
+                        if (lane == owner) {
+                            // lowest piece whose maximum is the round's maximum; piece q sits in slot (q - rot) & 3
+                            float sp[4] = {sm[0], sm[1], sm[2], sm[3]};
+                            rot_right4f(sp, rot);
+                            const int q = sp[0] == gm ? 0 : sp[1] == gm ? 1 : sp[2] == gm ? 2 : 3;
+                            const uint32_t pa = (uint32_t)(tid * 64 + q * 16);
+                            const uint4 xw = lds128(xs + pa);
+                            const uint32_t xws[4] = {xw.x, xw.y, xw.z, xw.w};
+                            u64 rr[4] = {0ull, 0ull, 0ull, 0ull};
+                            if (has_ref) load_ref_slot(rs + pa, p.gain, p.bias, (int)(pa >> 1), rr);
+                            float ev[8];
 #pragma unroll
-                        for (int i = 0; i < 32; i++) eq |= (fabsf(e[i]) == gm) ? (1u << i) : 0u;
-                        eq &= ~taken;                                // a taken element ties only when the maximum is 0
-                        const uint32_t eqc = rotl32(eq, 8 * rot);    // channel order within the slab
-                        const uint32_t gb = (__ballot_sync(group_mask, eqc != 0u) >> qbase) & qlanes;
-                        const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);
-                        const bool mine = lane == owner && eqc != 0u;
-                        const int cl = eqc ? __ffs(eqc) - 1 : 0;     // channel within the slab
-                        const uint32_t hit = mine ? rotr32(1u << cl, 8 * rot) : 0u;
-                        float val = 0.f;
+                            for (int i = 0; i < 4; i++) unpack2(psub(bf16x2_to_p(xws[i]), pfma(a2, rr[i], b2)), ev[2 * i], ev[2 * i + 1]);
+                            uint32_t tq = (taken >> (8 * q)) & 0xffu;
+                            uint32_t eq = 0;
 #pragma unroll
-                        for (int i = 0; i < 32; i++) {
-                            const bool h = (hit >> i) & 1u;
-                            val = h ? e[i] : val;
-                            e[i] = h ? 0.f : e[i];                   // E^d = E - O
+                            for (int k = 0; k < 8; k++) eq |= (fabsf(ev[k]) == gm) ? (1u << k) : 0u;
+                            eq &= ~tq;
+                            const int k = eq ? __ffs(eq) - 1 : 0;
+                            float val = ev[0];
+#pragma unroll
+                            for (int kk = 1; kk < 8; kk++) val = (kk == k) ? ev[kk] : val;
+                            tq |= 1u << k;
+                            taken |= 1u << (8 * q + k);
+                            const float nm = abs_max8(ev, tq);          // E^d = E - O for this slot's maximum
+                            const int js = (q - rot) & 3;
+#pragma unroll
+                            for (int j = 0; j < 4; j++) sm[j] = (j == js) ? nm : sm[j];
+                            word = (uint32_t)((lane - qbase) * 32 + 8 * q + k) | (float_to_half_bits_sat(val) << 16);
+                            own |= 1u << n;
                         }
-                        taken |= hit;
-                        const uint32_t word = (uint32_t)((lane - qbase) * 32 + cl) | (float_to_half_bits_sat(val) << 16);
                         sel[n] = __shfl_sync(group_mask, word, owner);
-                        if (mine) own |= 1u << n;
                     }
                 }
                 if ((lane & (p.lpq - 1)) == 0) {
@@ -214,8 +259,7 @@ __global__ void __launch_bounds__(256, 2) encode_dyn_kernel(const CodecParams p)
                 }
             }
             // ---- largest dense magnitude of this thread, then of its group
-#pragma unroll
-            for (int i = 0; i < 32; i++) m = fmaxf(m, fabsf(e[i]));
+            m = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
             if (!qtok) {
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1)
@@ -252,7 +296,7 @@ __global__ void __launch_bounds__(256, 2) encode_dyn_kernel(const CodecParams p)
 #pragma unroll
                 for (int i = 0; i < 4; i++) {
                     float v0, v1;
-                    unpack2(pmul(pack2(e[8 * j + 2 * i], e[8 * j + 2 * i + 1]), inv2), v0, v1);
+                    unpack2(pmul(e2[4 * j + i], inv2), v0, v1);
                     v0 = fminf(fmaxf(v0, -qmax), qmax);
                     v1 = fminf(fmaxf(v1, -qmax), qmax);
                     const u64 tt = padd(pack2(v0, v1), magic2);
@@ -291,22 +335,30 @@ __global__ void __launch_bounds__(256, 2) encode_dyn_kernel(const CodecParams p)
                     cw[1] = lo[2] | (lo[3] << 16);
                 }
             }
-            if (KG && XHAT && own) {
-                // the outliers this thread owns: x_hat = bf16((alpha*r + beta) + binary16 value)
+            if (KG && own) {
+                // the outliers this thread owns: dense code 0 (E^d = E - O), and on the sender side
+                // x_hat = bf16((alpha*r + beta) + binary16 value)
                 float a, b, unused;
                 unpack2(a2, a, unused);
                 unpack2(b2, b, unused);
+                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + p.codes_off) + tid * WPT;
 #pragma unroll
                 for (int n = 0; n < 4; n++) {
                     if ((own >> n) & 1u) {
                         const int c = jq * (p.lpq * 32) + (int)(sel[n] & 0xffffu);
-                        float r = 0.f;
-                        if (has_ref) {
-                            r = __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(stg + row_bytes + 2 * c)) << 16);
-                            if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                        const int bp = (c & 31) * BITS, w = bp >> 5, sh = bp & 31;
+                        const unsigned long long mk = (unsigned long long)((1u << BITS) - 1u) << sh;
+                        cw[w] &= ~(uint32_t)mk;
+                        if (BITS == 3 && sh > 29) cw[w + 1] &= ~(uint32_t)(mk >> 32);
+                        if (XHAT) {
+                            float r = 0.f;
+                            if (has_ref) {
+                                r = __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(stg + row_bytes + 2 * c)) << 16);
+                                if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                            }
+                            const float x = __fadd_rn(__fmaf_rn(a, r, b), half_bits_to_float(sel[n] >> 16));
+                            reinterpret_cast<unsigned short *>(stg)[c] = __bfloat16_as_ushort(__float2bfloat16_rn(x));
                         }
-                        const float x = __fadd_rn(__fmaf_rn(a, r, b), half_bits_to_float(sel[n] >> 16));
-                        reinterpret_cast<unsigned short *>(stg)[c] = __bfloat16_as_ushort(__float2bfloat16_rn(x));
                     }
                 }
             }
@@ -557,9 +609,12 @@ int launch_encode_dyn(const Geometry &g, CodecParams &p, long long max_ctas, cud
     p.stages = pick_stages(g.d, 2);
     const DynSmem L = dyn_smem_layout(g.d, g.rec, p.stages);
     const bool kg = g.topk_group > 0;
+    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
 #define RAC_DYN_ENC2(B, X) \
-    (kg ? launch_persistent(encode_dyn_kernel<B, X, true>, p, g.nthreads, L.total, max_ctas, stream) \
-        : launch_persistent(encode_dyn_kernel<B, X, false>, p, g.nthreads, L.total, max_ctas, stream))
+    (kg ? (tight && B != 8 ? launch_persistent(encode_dyn_kernel<B, X, true, 4>, p, g.nthreads, L.total, max_ctas, stream) \
+                 : launch_persistent(encode_dyn_kernel<B, X, true, 2>, p, g.nthreads, L.total, max_ctas, stream)) \
+        : tight ? launch_persistent(encode_dyn_kernel<B, X, false, 4>, p, g.nthreads, L.total, max_ctas, stream) \
+                : launch_persistent(encode_dyn_kernel<B, X, false, 2>, p, g.nthreads, L.total, max_ctas, stream))
 #define RAC_DYN_ENC(B) (p.X_hat ? RAC_DYN_ENC2(B, true) : RAC_DYN_ENC2(B, false))
     switch (g.bits) {
         case 8: return RAC_DYN_ENC(8);
