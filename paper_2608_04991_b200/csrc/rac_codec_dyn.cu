@@ -74,7 +74,8 @@ __device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, 
 }
 
 // MINB = 4 caps registers at 96 so that four 160-thread CTAs (d = 5120) fit on an SM.
-template <int BITS, bool XHAT, bool KG, int MINB>
+// KG: rounds compiled in (0, 1, 2 or 4; p.kg <= KG is the number taken).
+template <int BITS, bool XHAT, int KG, int MINB>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -197,7 +198,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             if (KG) {
                 uint32_t taken = 0;  // channel order within the slab
 #pragma unroll
-                for (int n = 0; n < 4; n++) {
+                for (int n = 0; n < KG; n++) {
                     if (n < p.kg) {
                         const float mloc = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
                         float gm = mloc;
@@ -246,11 +247,11 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                     unsigned char *go = rec + p.goff_off + jq * p.kg;
                     unsigned short *gv = reinterpret_cast<unsigned short *>(rec + p.gval_off) + jq * p.kg;
 #pragma unroll
-                    for (int n = 0; n < 4; n++) {
+                    for (int n = 0; n < KG; n++) {
                         if (n < p.kg) {
                             int rank = 0;
 #pragma unroll
-                            for (int q = 0; q < 4; q++)
+                            for (int q = 0; q < KG; q++)
                                 if (q < p.kg && (sel[q] & 0xffffu) < (sel[n] & 0xffffu)) rank++;
                             go[rank] = (unsigned char)(sel[n] & 0xffu);
                             gv[rank] = (unsigned short)(sel[n] >> 16);
@@ -343,7 +344,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                 unpack2(b2, b, unused);
                 uint32_t *cw = reinterpret_cast<uint32_t *>(rec + p.codes_off) + tid * WPT;
 #pragma unroll
-                for (int n = 0; n < 4; n++) {
+                for (int n = 0; n < KG; n++) {
                     if ((own >> n) & 1u) {
                         const int c = jq * (p.lpq * 32) + (int)(sel[n] & 0xffffu);
                         const int bp = (c & 31) * BITS, w = bp >> 5, sh = bp & 31;
@@ -605,25 +606,41 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
+// The 96-register variant (four 160-thread CTAs per SM) exists where it does not spill: without x_hat, and with
+// outliers only below 8-bit codes.
+template <int B, bool X, int K>
+static int launch_encode_variant(bool tight, const Geometry &g, CodecParams &p, int smem, long long max_ctas, cudaStream_t stream) {
+    if constexpr (!X && (K == 0 || B != 8)) {
+        if (tight) return launch_persistent(encode_dyn_kernel<B, X, K, 4>, p, g.nthreads, smem, max_ctas, stream);
+    }
+    return launch_persistent(encode_dyn_kernel<B, X, K, 2>, p, g.nthreads, smem, max_ctas, stream);
+}
+
+template <int B>
+static int launch_encode_bits(const Geometry &g, CodecParams &p, int smem, long long max_ctas, cudaStream_t stream) {
+    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !getenv("RAC_ENC_WIDE");
+    const int k = g.topk_group;
+    if (p.X_hat) {
+        return k == 0 ? launch_encode_variant<B, true, 0>(tight, g, p, smem, max_ctas, stream)
+             : k == 1 ? launch_encode_variant<B, true, 1>(tight, g, p, smem, max_ctas, stream)
+             : k == 2 ? launch_encode_variant<B, true, 2>(tight, g, p, smem, max_ctas, stream)
+                      : launch_encode_variant<B, true, 4>(tight, g, p, smem, max_ctas, stream);
+    }
+    return k == 0 ? launch_encode_variant<B, false, 0>(tight, g, p, smem, max_ctas, stream)
+         : k == 1 ? launch_encode_variant<B, false, 1>(tight, g, p, smem, max_ctas, stream)
+         : k == 2 ? launch_encode_variant<B, false, 2>(tight, g, p, smem, max_ctas, stream)
+                  : launch_encode_variant<B, false, 4>(tight, g, p, smem, max_ctas, stream);
+}
+
 int launch_encode_dyn(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
     p.stages = pick_stages(g.d, 2);
     const DynSmem L = dyn_smem_layout(g.d, g.rec, p.stages);
-    const bool kg = g.topk_group > 0;
-    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
-#define RAC_DYN_ENC2(B, X) \
-    (kg ? (tight && B != 8 ? launch_persistent(encode_dyn_kernel<B, X, true, 4>, p, g.nthreads, L.total, max_ctas, stream) \
-                 : launch_persistent(encode_dyn_kernel<B, X, true, 2>, p, g.nthreads, L.total, max_ctas, stream)) \
-        : tight ? launch_persistent(encode_dyn_kernel<B, X, false, 4>, p, g.nthreads, L.total, max_ctas, stream) \
-                : launch_persistent(encode_dyn_kernel<B, X, false, 2>, p, g.nthreads, L.total, max_ctas, stream))
-#define RAC_DYN_ENC(B) (p.X_hat ? RAC_DYN_ENC2(B, true) : RAC_DYN_ENC2(B, false))
     switch (g.bits) {
-        case 8: return RAC_DYN_ENC(8);
-        case 4: return RAC_DYN_ENC(4);
-        case 3: return RAC_DYN_ENC(3);
-        case 2: return RAC_DYN_ENC(2);
+        case 8: return launch_encode_bits<8>(g, p, L.total, max_ctas, stream);
+        case 4: return launch_encode_bits<4>(g, p, L.total, max_ctas, stream);
+        case 3: return launch_encode_bits<3>(g, p, L.total, max_ctas, stream);
+        case 2: return launch_encode_bits<2>(g, p, L.total, max_ctas, stream);
     }
-#undef RAC_DYN_ENC
-#undef RAC_DYN_ENC2
     return RAC_EUNSUPPORTED;
 }
 
