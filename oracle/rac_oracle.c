@@ -12,7 +12,10 @@
  *                        every hit extended to its longest exact match, at most
  *                        K most recent hits per distinct window, selection by
  *                        lexargmax(length, recency), scan advances by the span
- *                        length or by one.
+ *                        length or by one.  orc_match_spans_req: the history as a
+ *                        list of earlier requests (candidates stay inside one
+ *                        request) and the intra-sequence references of uncovered
+ *                        repeated tokens.
  *   orc_encode           Sec. IV-C: grouped affine fit (Eq. 6) with the
  *                        zero-variance rule, wire rounding of the coefficients,
  *                        aligned reference and residual (Eq. 7), outlier split
@@ -632,28 +635,53 @@ static int cmp_hist_query(const int32_t *hist, int32_t p, const int32_t *query, 
 }
 
 /*
- * ref_row  int32[n_query] out: history row of every covered query position, -1 otherwise
+ * The history is the concatenation of n_req earlier requests: request r holds the
+ * tokens [req_off[r], req_off[r+1]) (req_off[0] = 0, req_off[n_req] = n_hist;
+ * req_off NULL = one request).  A candidate (r, j, L) lies inside ONE request: its
+ * window and its extension stop at the request's end.  Recency is the position in
+ * the concatenation (a later request is more recent; inside a request the later
+ * start).
+ *
+ * ref_row  int32[n_query] out: history row of every covered query position, -1 otherwise;
+ *          with `intra`, an uncovered position whose token occurred earlier in the
+ *          query gets n_hist + (position of the FIRST occurrence of that token in the
+ *          query): the "intra-sequence reference" of Sec. IV-B.1.  The first
+ *          occurrence itself never gets one, so such references never chain.
  * spans    int32[3*cap]  out (q_start, h_start, len), cap >= n_query/w + 1; may be NULL
  * n_spans  out
  * max_hits K: only the K largest history starts of each distinct window are
  *          candidates; 0 = all of them.
  * Not thread safe (qsort comparator state).
  */
-int orc_match_spans(const int32_t *hist, int64_t n_hist, const int32_t *query, int64_t n_query,
-                    int w, int max_hits, int32_t *ref_row, int32_t *spans, int32_t *n_spans) {
+int orc_match_spans_req(const int32_t *hist, int64_t n_hist, const int32_t *req_off, int32_t n_req,
+                        const int32_t *query, int64_t n_query, int w, int max_hits, int intra,
+                        int32_t *ref_row, int32_t *spans, int32_t *n_spans) {
     if (w < 1 || max_hits < 0) return -1;
+    if (req_off) {
+        if (n_req < 0 || req_off[0] != 0 || req_off[n_req] != n_hist) return -1;
+        for (int32_t r = 0; r < n_req; r++) if (req_off[r] > req_off[r + 1]) return -1;
+    }
     for (int64_t i = 0; i < n_query; i++) ref_row[i] = -1;
     *n_spans = 0;
-    int64_t nwin = n_hist - w + 1;
-    if (nwin <= 0) return 0;
-    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)nwin);
-    for (int64_t j = 0; j < nwin; j++) order[j] = (int32_t)j;
+    /* end of the request that holds each history position */
+    int32_t *end_of = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_hist > 0 ? n_hist : 1));
+    if (req_off) {
+        for (int32_t r = 0; r < n_req; r++)
+            for (int32_t j = req_off[r]; j < req_off[r + 1]; j++) end_of[j] = req_off[r + 1];
+    } else {
+        for (int64_t j = 0; j < n_hist; j++) end_of[j] = (int32_t)n_hist;
+    }
+    /* windows that lie inside one request, sorted by content then position */
+    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_hist > 0 ? n_hist : 1));
+    int64_t nwin = 0;
+    for (int64_t j = 0; j + w <= n_hist; j++)
+        if (j + w <= end_of[j]) order[nwin++] = (int32_t)j;
     g_sort_tok = hist; g_sort_w = w;
     qsort(order, (size_t)nwin, sizeof(int32_t), cmp_window_pos);
 
     int64_t i = 0;
     int32_t ns = 0;
-    while (i < n_query) {
+    while (i < n_query && nwin > 0) {
         if (i + w > n_query) { i++; continue; }
         /* equal range of the query window in the sorted window list */
         int64_t lo = 0, hi = nwin;
@@ -675,7 +703,7 @@ int orc_match_spans(const int32_t *hist, int64_t n_hist, const int32_t *query, i
         for (int64_t k = from; k < last; k++) {
             int32_t j = order[k];
             int64_t L = w;
-            while (i + L < n_query && j + L < n_hist && query[i + L] == hist[j + L]) L++;
+            while (i + L < n_query && j + L < end_of[j] && query[i + L] == hist[j + L]) L++;
             if (L > bestL || (L == bestL && j > bestj)) { bestL = L; bestj = j; }
         }
         if (spans) { spans[3 * ns] = (int32_t)i; spans[3 * ns + 1] = bestj; spans[3 * ns + 2] = (int32_t)bestL; }
@@ -684,8 +712,22 @@ int orc_match_spans(const int32_t *hist, int64_t n_hist, const int32_t *query, i
         i += bestL;
     }
     *n_spans = ns;
-    free(order);
+    if (intra) {
+        /* plain quadratic scan: the first occurrence of every uncovered position's token */
+        for (int64_t q = 0; q < n_query; q++) {
+            if (ref_row[q] >= 0) continue;
+            for (int64_t f = 0; f < q; f++) {
+                if (query[f] == query[q]) { ref_row[q] = (int32_t)(n_hist + f); break; }
+            }
+        }
+    }
+    free(order); free(end_of);
     return 0;
+}
+
+int orc_match_spans(const int32_t *hist, int64_t n_hist, const int32_t *query, int64_t n_query,
+                    int w, int max_hits, int32_t *ref_row, int32_t *spans, int32_t *n_spans) {
+    return orc_match_spans_req(hist, n_hist, NULL, 1, query, n_query, w, max_hits, 0, ref_row, spans, n_spans);
 }
 
 int orc_max_threads(void) {

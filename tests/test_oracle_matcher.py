@@ -161,3 +161,106 @@ def test_cap_changes_result_only_for_frequent_windows(orc):
     assert sp8.tolist()[0] == [0, last, 4]
     b_rr, b_sp = brute_force(hist, query, 4, 8)
     assert np.array_equal(sp8, b_sp)
+
+
+# ------------------------------------------------------------------ earlier requests and intra-sequence references
+def brute_force_requests(reqs, query, w, K, intra):
+    """The definition per request: candidate (r, j, L) with query[i:i+L] == reqs[r][j:j+L], L >= w maximal inside
+    request r; recency = (r, j); the K most recent hits per distinct window; longest, then most recent."""
+    N = len(query)
+    off = np.concatenate([[0], np.cumsum([len(r) for r in reqs])]).astype(np.int64)
+    ref_row = np.full(N, -1, np.int32)
+    spans = []
+    i = 0
+    while i < N:
+        hits = []   # (r, j) of every request window equal to the query window at i
+        if i + w <= N:
+            for r, req in enumerate(reqs):
+                for j in range(len(req) - w + 1):
+                    if list(req[j:j + w]) == list(query[i:i + w]):
+                        hits.append((r, j))
+        if K > 0:
+            hits = sorted(hits)[-K:]
+        if not hits:
+            i += 1
+            continue
+        best = None
+        for r, j in hits:
+            L = w
+            while i + L < N and j + L < len(reqs[r]) and query[i + L] == reqs[r][j + L]:
+                L += 1
+            key = (L, r, j)
+            if best is None or key > best:
+                best = key
+        L, r, j = best
+        spans.append((i, int(off[r]) + j, L))
+        ref_row[i:i + L] = np.arange(off[r] + j, off[r] + j + L)
+        i += L
+    if intra:
+        first = {}
+        for q in range(N):
+            t = int(query[q])
+            if ref_row[q] < 0 and t in first:
+                ref_row[q] = off[-1] + first[t]
+            first.setdefault(t, q)
+    return ref_row, np.array(spans, np.int32).reshape(-1, 3), off.astype(np.int32)
+
+
+@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("K", [0, 1, 3])
+def test_requests_match_brute_force(orc, seed, K):
+    rng = np.random.default_rng(500 + seed)
+    vocab = [2, 3, 6][seed % 3]
+    w = [1, 2, 3, 4][seed % 4]
+    reqs = [rng.integers(0, vocab, int(rng.integers(0, 25))).astype(np.int32) for _ in range(int(rng.integers(1, 6)))]
+    N = int(rng.integers(1, 50))
+    query = rng.integers(0, vocab, N).astype(np.int32)
+    if seed % 2 and len(reqs) > 1 and len(reqs[0]) + len(reqs[1]) >= 6:
+        # plant the JOIN of two requests: a match across the boundary must be cut at it
+        joined = np.concatenate([reqs[0], reqs[1]])
+        L = min(N, len(joined))
+        query[:L] = joined[:L]
+    brr, bsp, off = brute_force_requests(reqs, query, w, K, intra=bool(seed % 2))
+    hist = np.concatenate(reqs + [np.zeros(0, np.int32)]).astype(np.int32)
+    rr, sp = orc.match_spans_req(hist, off, query, w=w, max_hits=K, intra=bool(seed % 2))
+    assert np.array_equal(rr, brr)
+    assert np.array_equal(sp, bsp)
+
+
+def test_request_boundaries_cut_matches_and_one_request_is_the_flat_matcher(orc):
+    a = np.arange(100, 120, dtype=np.int32)
+    b = np.arange(120, 140, dtype=np.int32)
+    hist = np.concatenate([a, b])
+    query = np.arange(110, 130, dtype=np.int32)          # straddles the boundary at 120
+    rr_flat, sp_flat = orc.match_spans(hist, query, w=4)
+    assert sp_flat.tolist() == [[0, 10, 20]]
+    rr, sp = orc.match_spans_req(hist, [0, 20, 40], query, w=4)
+    assert sp.tolist() == [[0, 10, 10], [10, 20, 10]]    # cut at the end of the first request
+    assert np.array_equal(rr, rr_flat)                   # the rows happen to be the same; the spans are not
+    # a window that straddles the boundary is no candidate at all
+    rr, sp = orc.match_spans_req(hist, [0, 20, 40], np.arange(118, 122, dtype=np.int32), w=4)
+    assert len(sp) == 0 and np.all(rr == -1)
+    # one request == the flat form
+    rng = np.random.default_rng(9)
+    h = rng.integers(0, 4, 300).astype(np.int32)
+    q = rng.integers(0, 4, 200).astype(np.int32)
+    r1, s1 = orc.match_spans(h, q, w=3, max_hits=2)
+    r2, s2 = orc.match_spans_req(h, [0, 300], q, w=3, max_hits=2)
+    r3, s3 = orc.match_spans_req(h, None, q, w=3, max_hits=2)
+    assert np.array_equal(r1, r2) and np.array_equal(s1, s2) and np.array_equal(r1, r3) and np.array_equal(s1, s3)
+
+
+def test_intra_sequence_references_point_at_first_occurrences_and_never_chain(orc):
+    hist = np.arange(1000, 1040, dtype=np.int32)
+    query = np.array([7, 8, 7, 9, 8, 7, 1000, 1001, 1002, 1003, 7, 1001], np.int32)
+    rr, sp = orc.match_spans_req(hist, None, query, w=4, intra=True)
+    n = hist.size
+    #           7   8   7      9   8      7      span of four            7      1001 (first seen inside the span)
+    want = [-1, -1, n + 0, -1, n + 1, n + 0, 0, 1, 2, 3, n + 0, n + 7]
+    assert rr.tolist() == want and sp.tolist() == [[6, 0, 4]]
+    intra = rr >= n
+    targets = rr[intra] - n
+    assert np.all(rr[targets] < n)                        # a referenced position is never itself intra-referenced
+    assert np.all(query[targets] == query[intra]) and np.all(targets < np.flatnonzero(intra))
+    rr0, _ = orc.match_spans_req(hist, None, query, w=4, intra=False)
+    assert np.array_equal(np.where(intra, -1, rr), rr0)
