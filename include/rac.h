@@ -147,6 +147,47 @@ int rac_match_spans_static(const int32_t *hist_tok, int64_t n_hist, const int32_
                            int32_t min_ngram, int32_t max_hits, int32_t *ref_row, rac_span *spans, int32_t *n_spans,
                            void *stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Span retrieval over a growing history of earlier requests (Sec. IV-B.1: the windows of "earlier requests"
+ * are indexed, a candidate (r, j, L) lies inside one request r, recency breaks ties) with an index that
+ * persists between prompts, plus the intra-sequence references of the same passage.
+ *
+ * The history is the concatenation of the requests seen so far; row j of the history state buffer belongs to
+ * token j of that concatenation.  The index lives in caller memory (`index`, rac_index_bytes() bytes, 16-byte
+ * aligned) and holds the hash table, the `max_hits` most recent starts of every distinct window, and the end of
+ * the request of every history position.
+ *
+ *   rac_index_reset    empties the index.
+ *   rac_index_append   adds ONE request: the tokens hist_tok[n_before .. n_after).  hist_tok is the device buffer
+ *                      of the whole concatenation (tokens below n_before as at earlier calls: the index verifies
+ *                      keys against them).  Windows lie inside the request; a request shorter than min_ngram adds
+ *                      no window.  n_before must be the n_after of the previous append (0 after a reset); the
+ *                      library keeps no host state and cannot check this.  n_after <= capacity.
+ *                      Appending requests one by one gives the same index as any other split into calls with the
+ *                      same request boundaries: contents do not depend on thread timing.
+ *   rac_index_query    the selection of Eq. 3 for one prompt against the indexed history: like rac_match_spans,
+ *                      except that a match ends at the end of its request.  With intra != 0, every position that no
+ *                      span covers and whose token occurred EARLIER in the prompt gets
+ *                      ref_row = n_hist + (position of the first occurrence of that token in the prompt): a
+ *                      reference to the reconstruction of that earlier token of the same prompt.  First occurrences
+ *                      never get such a reference, so they never chain: all tokens with ref_row < n_hist can be
+ *                      coded first and the others second (rac_encode_rows / rac_decode_rows below).
+ *                      workspace >= rac_index_query_workspace_bytes(n_query) bytes, scratch.
+ * All three are asynchronous on `stream`; calls on one index must be ordered. */
+typedef struct {
+    int64_t capacity;      /* history tokens the index can hold, 1 .. 2^30 - 1 */
+    int32_t min_ngram;     /* w, 1..32 */
+    int32_t max_hits;      /* K, 1..16 */
+} rac_index_cfg;
+size_t rac_index_bytes(const rac_index_cfg *cfg);
+int rac_index_reset(const rac_index_cfg *cfg, void *index, size_t index_bytes, void *stream);
+int rac_index_append(const rac_index_cfg *cfg, void *index, size_t index_bytes, const int32_t *hist_tok,
+                     int64_t n_before, int64_t n_after, void *stream);
+size_t rac_index_query_workspace_bytes(int64_t n_query);
+int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_bytes, const int32_t *hist_tok,
+                    int64_t n_hist, const int32_t *query_tok, int64_t n_query, int32_t intra, int32_t *ref_row,
+                    rac_span *spans, int32_t *n_spans, void *workspace, size_t workspace_bytes, void *stream);
+
 /* Receiver side of the retrieval: spans travel as control metadata, tokens do not.  Expands
  * `*n_spans` spans into ref_row[n_query] (-1 where no span covers).  Spans reaching outside
  * [0, n_query) are clipped. */

@@ -30,6 +30,7 @@ EXPORTS = [
     "rac_version", "rac_strerror", "rac_record_bytes", "rac_payload_bytes",
     "rac_match_workspace_bytes", "rac_match_spans", "rac_spans_to_rows",
     "rac_match_spans_static",
+    "rac_index_bytes", "rac_index_reset", "rac_index_append", "rac_index_query_workspace_bytes", "rac_index_query",
     "rac_encode_workspace_bytes", "rac_encode", "rac_encode_reconstruct", "rac_decode_reconstruct",
     "rac_sender_reconstruct",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
@@ -54,6 +55,14 @@ class CodecCfg(C.Structure):
     def __repr__(self):
         return (f"CodecCfg(d={self.d}, group={self.group}, bits={self.bits}, topk={self.topk}, "
                 f"scale_mode={self.scale_mode}, qgroup={self.qgroup}, topk_group={self.topk_group})")
+
+
+class IndexCfg(C.Structure):
+    """Mirror of ``rac_index_cfg``."""
+    _fields_ = [("capacity", C.c_int64), ("min_ngram", C.c_int32), ("max_hits", C.c_int32)]
+
+    def __init__(self, capacity: int, min_ngram: int = 4, max_hits: int = 8):
+        super().__init__(capacity, min_ngram, max_hits)
 
 
 _lib: Optional[C.CDLL] = None
@@ -84,6 +93,17 @@ def load() -> C.CDLL:
     l.rac_match_spans.argtypes = [vp, i64, vp, i64, i32, i32, vp, vp, vp, vp, sz, vp]
     l.rac_match_spans_static.restype = C.c_int
     l.rac_match_spans_static.argtypes = [vp, i64, vp, i64, i32, i32, vp, vp, vp, vp]
+    icfgp = C.POINTER(IndexCfg)
+    l.rac_index_bytes.restype = sz
+    l.rac_index_bytes.argtypes = [icfgp]
+    l.rac_index_reset.restype = C.c_int
+    l.rac_index_reset.argtypes = [icfgp, vp, sz, vp]
+    l.rac_index_append.restype = C.c_int
+    l.rac_index_append.argtypes = [icfgp, vp, sz, vp, i64, i64, vp]
+    l.rac_index_query_workspace_bytes.restype = sz
+    l.rac_index_query_workspace_bytes.argtypes = [i64]
+    l.rac_index_query.restype = C.c_int
+    l.rac_index_query.argtypes = [icfgp, vp, sz, vp, i64, vp, i64, i32, vp, vp, vp, vp, sz, vp]
     l.rac_spans_to_rows.restype = C.c_int
     l.rac_spans_to_rows.argtypes = [vp, vp, i64, vp, vp]
     l.rac_encode.restype = C.c_int
@@ -189,6 +209,38 @@ def rac_match_spans_static(hist_tok, n_hist, query_tok, n_query, min_ngram, max_
                                        _ptr(spans, _I32, "spans"), _ptr(n_spans, _I32, "n_spans"),
                                        _stream() if stream is None else stream)
     _check("rac_match_spans_static", rc)
+
+
+def rac_index_bytes(cfg: IndexCfg) -> int:
+    return int(load().rac_index_bytes(C.byref(cfg)))
+
+
+def rac_index_query_workspace_bytes(n_query: int) -> int:
+    return int(load().rac_index_query_workspace_bytes(int(n_query)))
+
+
+def rac_index_reset(cfg, index, index_bytes, stream=None) -> None:
+    rc = load().rac_index_reset(C.byref(cfg), _ptr(index, None, "index"), int(index_bytes),
+                                _stream() if stream is None else stream)
+    _check("rac_index_reset", rc)
+
+
+def rac_index_append(cfg, index, index_bytes, hist_tok, n_before, n_after, stream=None) -> None:
+    rc = load().rac_index_append(C.byref(cfg), _ptr(index, None, "index"), int(index_bytes),
+                                 _ptr(hist_tok, _I32, "hist_tok"), int(n_before), int(n_after),
+                                 _stream() if stream is None else stream)
+    _check("rac_index_append", rc)
+
+
+def rac_index_query(cfg, index, index_bytes, hist_tok, n_hist, query_tok, n_query, intra, ref_row, spans, n_spans,
+                    workspace, workspace_bytes, stream=None) -> None:
+    rc = load().rac_index_query(C.byref(cfg), _ptr(index, None, "index"), int(index_bytes),
+                                _ptr(hist_tok, _I32, "hist_tok"), int(n_hist), _ptr(query_tok, _I32, "query_tok"),
+                                int(n_query), int(bool(intra)), _ptr(ref_row, _I32, "ref_row"),
+                                _ptr(spans, _I32, "spans"), _ptr(n_spans, _I32, "n_spans"),
+                                _ptr(workspace, None, "workspace"), int(workspace_bytes),
+                                _stream() if stream is None else stream)
+    _check("rac_index_query", rc)
 
 
 def rac_spans_to_rows(spans, n_spans, n_query, ref_row, stream=None) -> None:

@@ -32,6 +32,7 @@ struct MatchParams {
     rac_span *spans_ws;    // [N/w + 1]
     int n_hist, n_query, nwin, w, K;
     unsigned int mask;     // M - 1
+    const int32_t *end_of; // [n_hist] end of the request that holds each history position; null = one request
 };
 
 __device__ __forceinline__ unsigned int window_hash(const int32_t *tok, int w) {
@@ -103,7 +104,8 @@ __global__ void match_query_kernel(MatchParams p) {
                 int j = lst[r];
                 if (j < 0) break;
                 int L = p.w;
-                while (i + L < p.n_query && j + L < p.n_hist && p.query[i + L] == p.hist[j + L]) L++;
+                const int hend = p.end_of ? p.end_of[j] : p.n_hist;   // a match stays inside its request
+                while (i + L < p.n_query && j + L < hend && p.query[i + L] == p.hist[j + L]) L++;
                 if (L > bestL || (L == bestL && j > bestj)) { bestL = L; bestj = j; }
             }
         }
@@ -247,6 +249,104 @@ __global__ void fill_i32_kernel(int32_t *dst, long long n, int32_t v) {
     for (; i < n; i += stride) dst[i] = v;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Persistent index over a growing list of requests
+// ---------------------------------------------------------------------------------------------
+struct IndexParams {
+    const int32_t *hist;
+    int32_t *rep;       // [M]
+    int32_t *top;       // [M*K]
+    int32_t *end_of;    // [capacity]
+    int32_t *slot_of;   // [capacity]  slot of the window starting at each history position (append scratch)
+    int32_t *cnt;       // [M]         windows of the request being appended, per slot; zero between calls
+    int a, b;           // the request: tokens [a, b)
+    int w, K;
+    unsigned int mask;
+};
+
+// (1) every position of the request learns its end; every window of the request finds or claims its slot and
+// is counted there
+__global__ void index_append_insert_kernel(IndexParams p) {
+    const int j = p.a + blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= p.b) return;
+    p.end_of[j] = p.b;
+    if (j + p.w > p.b) return;  // the window would leave the request
+    const int32_t *win = p.hist + j;
+    unsigned int s = window_hash(win, p.w) & p.mask;
+    int slot = -1;
+    for (unsigned int probe = 0; probe <= p.mask; probe++) {
+        int cur = atomicCAS(&p.rep[s], -1, j);
+        if (cur == -1 || cur == j || same_window(p.hist + cur, win, p.w)) { slot = (int)s; break; }
+        s = (s + 1) & p.mask;
+    }
+    p.slot_of[j] = slot;
+    if (slot >= 0) atomicAdd(&p.cnt[slot], 1);
+}
+
+// (2) one thread per touched slot (the one that takes the count away) makes room at the head of the slot's
+// list: the request's starts are larger than everything already there
+__global__ void index_append_shift_kernel(IndexParams p) {
+    const int j = p.a + blockIdx.x * blockDim.x + threadIdx.x;
+    if (j + p.w > p.b) return;
+    const int slot = p.slot_of[j];
+    if (slot < 0) return;
+    const int c = atomicExch(&p.cnt[slot], 0);
+    if (c == 0) return;
+    int32_t *lst = p.top + (long long)slot * p.K;
+    const int sh = c < p.K ? c : p.K;
+    for (int r = p.K - 1; r >= sh; r--) lst[r] = lst[r - sh];
+    for (int r = 0; r < sh; r++) lst[r] = -1;
+}
+
+// (3) round r: the largest start of the request's windows below the one found in round r-1.  Entries behind the
+// request's own are older, hence smaller, and are never touched: no start of the request is below its smallest.
+__global__ void index_append_round_kernel(IndexParams p, int r) {
+    const int j = p.a + blockIdx.x * blockDim.x + threadIdx.x;
+    if (j + p.w > p.b) return;
+    const int slot = p.slot_of[j];
+    if (slot < 0) return;
+    int32_t *lst = p.top + (long long)slot * p.K;
+    if (r == 0 || j < lst[r - 1]) atomicMax(&lst[r], j);
+}
+
+// Intra-sequence references: first occurrence of every token of the prompt (a hash table keyed by a position
+// whose token is the key, verified by comparing tokens), then the uncovered positions look theirs up.
+__global__ void intra_insert_kernel(const int32_t *query, int n, int32_t *trep, int32_t *tfirst, unsigned int mask) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t tok = query[i];
+    unsigned int s = window_hash(&tok, 1) & mask;
+    for (unsigned int probe = 0; probe <= mask; probe++) {
+        int cur = atomicCAS(&trep[s], -1, i);
+        if (cur == -1 || cur == i || query[cur] == tok) { atomicMin(&tfirst[s], i); return; }
+        s = (s + 1) & mask;
+    }
+}
+__global__ void intra_assign_kernel(const int32_t *query, int n, const int32_t *trep, const int32_t *tfirst,
+                                    unsigned int mask, int n_hist, int32_t *ref_row) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n || ref_row[i] >= 0) return;
+    const int32_t tok = query[i];
+    unsigned int s = window_hash(&tok, 1) & mask;
+    for (unsigned int probe = 0; probe <= mask; probe++) {
+        int cur = trep[s];
+        if (cur < 0) return;
+        if (query[cur] == tok) {
+            const int f = tfirst[s];
+            if (f < i) ref_row[i] = n_hist + f;
+            return;
+        }
+        s = (s + 1) & mask;
+    }
+}
+
+__global__ void fill2_i32_kernel(int32_t *a, long long na, int32_t va, int32_t *b, long long nb, int32_t vb) {
+    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long k = i; k < na; k += stride) a[k] = va;
+    for (long long k = i; k < nb; k += stride) b[k] = vb;
+}
+
 static size_t align16(size_t v) { return (v + 15) / 16 * 16; }
 
 struct MatchLayout {
@@ -320,6 +420,7 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char *ws = static_cast<unsigned char *>(workspace);
     MatchParams p;
+    p.end_of = nullptr;
     p.hist = hist_tok;
     p.query = query_tok;
     p.ref_row = ref_row;
@@ -390,6 +491,170 @@ int rac_match_spans_static(const int32_t *hist_tok, int64_t n_hist, const int32_
     // previous call left in the scratch is harmless
     return rac_match_spans(hist_tok, n_hist, query_tok, n_query, min_ngram, max_hits, ref_row, spans, n_spans, scratch,
                            kStaticMatchBytes, stream);
+}
+
+}  // extern "C"
+
+// ---- persistent index ------------------------------------------------------------------------
+namespace {
+struct IndexLayout {
+    size_t rep, top, cnt, end_of, slot_of, total;
+    unsigned int M;
+};
+bool index_cfg_ok(const rac_index_cfg *c) {
+    return c && c->capacity >= 1 && c->capacity < (1ll << 30) && c->min_ngram >= 1 && c->min_ngram <= 32 &&
+           c->max_hits >= 1 && c->max_hits <= 16;
+}
+IndexLayout index_layout(const rac_index_cfg *c) {
+    IndexLayout L;
+    unsigned long long M = 1024;
+    while (M < 2ull * (unsigned long long)c->capacity) M <<= 1;
+    L.M = (unsigned int)M;
+    size_t o = 0;
+    L.rep = o;      o += (size_t)M * 4;                        // rep and top contiguous: one fill with -1
+    L.top = o;      o = align16(o + (size_t)M * c->max_hits * 4);
+    L.cnt = o;      o = align16(o + (size_t)M * 4);
+    L.end_of = o;   o = align16(o + (size_t)c->capacity * 4);
+    L.slot_of = o;  o = align16(o + (size_t)c->capacity * 4);
+    L.total = o;
+    return L;
+}
+struct QueryLayout {
+    size_t best, hop, spans, trep, tfirst, total;
+    unsigned int Mq;
+};
+QueryLayout query_layout(long long n_query) {
+    QueryLayout L;
+    const size_t n = (size_t)(n_query > 0 ? n_query : 1);
+    unsigned long long M = 1024;
+    while (M < 2ull * n) M <<= 1;
+    L.Mq = (unsigned int)M;
+    size_t o = 0;
+    L.best = o;    o = align16(o + n * 8);
+    L.hop = o;     o = align16(o + n * 8);
+    L.spans = o;   o = align16(o + (n + 1) * sizeof(rac_span));
+    L.trep = o;    o = align16(o + (size_t)M * 4);
+    L.tfirst = o;  o = align16(o + (size_t)M * 4);
+    L.total = o;
+    return L;
+}
+int grid_for(long long n, int tb) {
+    long long b = (n + tb - 1) / tb;
+    if (b > 148 * 16) b = 148 * 16;
+    return (int)(b < 1 ? 1 : b);
+}
+}  // namespace
+
+extern "C" {
+
+size_t rac_index_bytes(const rac_index_cfg *cfg) { return index_cfg_ok(cfg) ? index_layout(cfg).total : 0; }
+
+int rac_index_reset(const rac_index_cfg *cfg, void *index, size_t index_bytes, void *stream) {
+    if (!index_cfg_ok(cfg)) return cfg ? RAC_EUNSUPPORTED : RAC_EINVAL;
+    if (!index) return RAC_EINVAL;
+    if (reinterpret_cast<uintptr_t>(index) & 15u) return RAC_EALIGN;
+    const IndexLayout L = index_layout(cfg);
+    if (index_bytes < L.total) return RAC_ESIZE;
+    unsigned char *ix = static_cast<unsigned char *>(index);
+    const long long table = (long long)L.M * (1 + cfg->max_hits);
+    fill2_i32_kernel<<<grid_for(table, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<int32_t *>(ix + L.rep), table, -1, reinterpret_cast<int32_t *>(ix + L.cnt), (long long)L.M, 0);
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+int rac_index_append(const rac_index_cfg *cfg, void *index, size_t index_bytes, const int32_t *hist_tok,
+                     int64_t n_before, int64_t n_after, void *stream) {
+    if (!index_cfg_ok(cfg)) return cfg ? RAC_EUNSUPPORTED : RAC_EINVAL;
+    if (!index || n_before < 0 || n_after < n_before) return RAC_EINVAL;
+    if (n_after > cfg->capacity) return RAC_ESIZE;
+    if (reinterpret_cast<uintptr_t>(index) & 15u) return RAC_EALIGN;
+    const IndexLayout L = index_layout(cfg);
+    if (index_bytes < L.total) return RAC_ESIZE;
+    if (n_after == n_before) return RAC_OK;
+    if (!hist_tok) return RAC_EINVAL;
+    unsigned char *ix = static_cast<unsigned char *>(index);
+    IndexParams p;
+    p.hist = hist_tok;
+    p.rep = reinterpret_cast<int32_t *>(ix + L.rep);
+    p.top = reinterpret_cast<int32_t *>(ix + L.top);
+    p.cnt = reinterpret_cast<int32_t *>(ix + L.cnt);
+    p.end_of = reinterpret_cast<int32_t *>(ix + L.end_of);
+    p.slot_of = reinterpret_cast<int32_t *>(ix + L.slot_of);
+    p.a = (int)n_before;
+    p.b = (int)n_after;
+    p.w = cfg->min_ngram;
+    p.K = cfg->max_hits;
+    p.mask = L.M - 1;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int tb = 256;
+    const int nb = (int)((n_after - n_before + tb - 1) / tb);
+    index_append_insert_kernel<<<nb, tb, 0, st>>>(p);
+    if (n_after - n_before >= cfg->min_ngram) {
+        index_append_shift_kernel<<<nb, tb, 0, st>>>(p);
+        for (int r = 0; r < cfg->max_hits; r++) index_append_round_kernel<<<nb, tb, 0, st>>>(p, r);
+    }
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+size_t rac_index_query_workspace_bytes(int64_t n_query) {
+    if (n_query < 0 || n_query >= (1ll << 30)) return 0;
+    return query_layout(n_query).total;
+}
+
+int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_bytes, const int32_t *hist_tok,
+                    int64_t n_hist, const int32_t *query_tok, int64_t n_query, int32_t intra, int32_t *ref_row,
+                    rac_span *spans, int32_t *n_spans, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!index_cfg_ok(cfg)) return cfg ? RAC_EUNSUPPORTED : RAC_EINVAL;
+    if (!index || !n_spans || n_hist < 0 || n_query < 0 || !workspace) return RAC_EINVAL;
+    if (n_hist > cfg->capacity) return RAC_ESIZE;
+    if (n_query >= (1ll << 30) || n_hist + n_query >= (1ll << 31)) return RAC_EUNSUPPORTED;
+    if ((n_hist > 0 && !hist_tok) || (n_query > 0 && (!query_tok || !ref_row))) return RAC_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(index) & 15u) || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return RAC_EALIGN;
+    const IndexLayout L = index_layout(cfg);
+    if (index_bytes < L.total) return RAC_ESIZE;
+    const QueryLayout Q = query_layout(n_query);
+    if (workspace_bytes < Q.total) return RAC_ESIZE;
+    const unsigned char *ix = static_cast<const unsigned char *>(index);
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    MatchParams p;
+    p.hist = hist_tok;
+    p.query = query_tok;
+    p.ref_row = ref_row;
+    p.spans_out = spans;
+    p.n_spans = n_spans;
+    p.rep = const_cast<int32_t *>(reinterpret_cast<const int32_t *>(ix + L.rep));
+    p.top = const_cast<int32_t *>(reinterpret_cast<const int32_t *>(ix + L.top));
+    p.slot_of = nullptr;
+    p.best = reinterpret_cast<int2 *>(ws + Q.best);
+    p.hop = reinterpret_cast<int2 *>(ws + Q.hop);
+    p.spans_ws = reinterpret_cast<rac_span *>(ws + Q.spans);
+    p.n_hist = (int)n_hist;
+    p.n_query = (int)n_query;
+    p.nwin = (int)(n_hist - cfg->min_ngram + 1 > 0 ? n_hist - cfg->min_ngram + 1 : 0);
+    p.w = cfg->min_ngram;
+    p.K = cfg->max_hits;
+    p.mask = L.M - 1;
+    p.end_of = reinterpret_cast<const int32_t *>(ix + L.end_of);
+    const int tb = 256;
+    // rows to -1, span count to 0, and (for the intra-sequence pass) the token table to empty
+    int32_t *trep = reinterpret_cast<int32_t *>(ws + Q.trep), *tfirst = reinterpret_cast<int32_t *>(ws + Q.tfirst);
+    fill2_i32_kernel<<<grid_for(n_query > 1 ? n_query : 1, tb), tb, 0, st>>>(ref_row, n_query, -1, n_spans, 1, 0);
+    if (n_query == 0) return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+    match_query_kernel<<<(int)((n_query + tb - 1) / tb), tb, 0, st>>>(p);
+    const int window = n_query < kWalkWindow ? (int)n_query : kWalkWindow;
+    const size_t dyn = ((size_t)window * 2 + 15) / 16 * 16;
+    if (dyn > 48 * 1024 &&
+        cudaFuncSetAttribute(match_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+        return RAC_ECUDA;
+    match_select_kernel<<<1, 1024, dyn, st>>>(p, window);
+    if (intra) {
+        fill2_i32_kernel<<<grid_for(Q.Mq, tb), tb, 0, st>>>(trep, (long long)Q.Mq, -1, tfirst, (long long)Q.Mq, 0x7fffffff);
+        const int nb = (int)((n_query + tb - 1) / tb);
+        intra_insert_kernel<<<nb, tb, 0, st>>>(query_tok, (int)n_query, trep, tfirst, Q.Mq - 1);
+        intra_assign_kernel<<<nb, tb, 0, st>>>(query_tok, (int)n_query, trep, tfirst, Q.Mq - 1, (int)n_hist, ref_row);
+    }
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
 }  // extern "C"

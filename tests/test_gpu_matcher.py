@@ -123,3 +123,125 @@ def test_spans_to_rows(env):
     torch.cuda.synchronize()
     o = out.cpu().numpy()
     assert np.all(o[:4090] == -1) and o[4090:].tolist() == list(range(10, 16))
+
+
+# --------------------------------------------------------------------------- persistent index over earlier requests
+class GpuIndex:
+    """Drives rac_index_* the way a serving loop would: one append per finished request, one query per prompt."""
+
+    def __init__(self, env, capacity, w, K):
+        self.env, self.rac, self.dev = env, env.rac, env.dev
+        self.cfg = env.rac.IndexCfg(capacity, w, K)
+        self.nb = env.rac.rac_index_bytes(self.cfg)
+        self.mem = torch.full((self.nb + 32,), 0x5A, dtype=torch.uint8, device=env.dev)   # dirty, canary behind
+        self.hist = torch.zeros(capacity, dtype=torch.int32, device=env.dev)
+        self.n = 0
+        self.w = w
+        env.rac.rac_index_reset(self.cfg, self.mem[:self.nb], self.nb)
+
+    def append(self, req):
+        req = np.ascontiguousarray(req, np.int32)
+        if req.size:
+            self.hist[self.n:self.n + req.size] = torch.from_numpy(req).to(self.dev)
+        self.rac.rac_index_append(self.cfg, self.mem[:self.nb], self.nb, self.hist, self.n, self.n + req.size)
+        self.n += req.size
+
+    def query(self, query, intra=False):
+        q = torch.from_numpy(np.ascontiguousarray(query, np.int32)).to(self.dev)
+        N = q.numel()
+        nws = self.rac.rac_index_query_workspace_bytes(N)
+        ws = torch.full((nws + 32,), 0xA5, dtype=torch.uint8, device=self.dev)
+        rows = torch.full((N + 8,), 12345, dtype=torch.int32, device=self.dev)
+        cap = N // self.w + 1
+        spans = torch.full((cap + 2, 3), 777, dtype=torch.int32, device=self.dev)
+        n_spans = torch.full((1,), -5, dtype=torch.int32, device=self.dev)
+        self.rac.rac_index_query(self.cfg, self.mem[:self.nb], self.nb, self.hist, self.n, q if N else None, N, intra,
+                                 rows[:N] if N else None, spans[:cap], n_spans, ws[:nws], nws)
+        torch.cuda.synchronize()
+        assert torch.all(rows[N:] == 12345) and torch.all(spans[cap:] == 777) and torch.all(ws[nws:] == 0xA5)
+        assert torch.all(self.mem[self.nb:] == 0x5A)
+        ns = int(n_spans.item())
+        return rows[:N].cpu().numpy(), spans[:ns].cpu().numpy()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_index_appended_request_by_request_matches_oracle(env, seed):
+    rng = np.random.default_rng(700 + seed)
+    vocab = [2, 3, 6, 40][seed % 4]
+    w = [1, 2, 3, 4, 5][seed % 5]
+    K = [1, 2, 8, 16][seed % 4]
+    ix = GpuIndex(env, 4096, w, K)
+    reqs, off = [], [0]
+    for step in range(7):
+        # a prompt is matched against what has been appended so far, then becomes a request itself
+        N = int(rng.integers(1, 300))
+        query = rng.integers(0, vocab, N).astype(np.int32)
+        if reqs and step % 2:
+            src = np.concatenate(reqs)                  # copy across request joins: matches must be cut there
+            L = min(N, src.size, 60)
+            a = int(rng.integers(0, src.size - L + 1))
+            query[:L] = src[a:a + L]
+        hist = np.concatenate(reqs) if reqs else np.zeros(0, np.int32)
+        for intra in (False, True):
+            rr, sp = ix.query(query, intra=intra)
+            o_rr, o_sp = env.orc.match_spans_req(hist, np.array(off, np.int32), query, w=w, max_hits=K, intra=intra)
+            assert np.array_equal(sp, o_sp), f"step {step}"
+            assert np.array_equal(rr, o_rr), f"step {step} intra {intra}"
+        ix.append(query)
+        reqs.append(query)
+        off.append(off[-1] + N)
+    # short and empty requests add no window but keep the bookkeeping right
+    ix.append(np.zeros(0, np.int32))
+    ix.append(np.arange(max(w - 1, 0), dtype=np.int32))
+    reqs.append(np.arange(max(w - 1, 0), dtype=np.int32))
+    off += [off[-1], off[-1] + max(w - 1, 0)]
+    query = np.concatenate(reqs)[-50:]
+    rr, sp = ix.query(query)
+    o_rr, o_sp = env.orc.match_spans_req(np.concatenate(reqs), np.array(off, np.int32), query, w=w, max_hits=K)
+    assert np.array_equal(sp, o_sp) and np.array_equal(rr, o_rr)
+
+
+def test_index_one_request_equals_the_one_shot_matcher_and_reset(env):
+    s = env.synth
+    wl = s.span_workload(20000, 3000, seed=5, gap_max=120)
+    hist, query = wl.hist.astype(np.int32), wl.query.astype(np.int32)
+    ix = GpuIndex(env, 20000, 4, 8)
+    ix.append(hist)
+    rr, sp = ix.query(query)
+    rr1, sp1, _ = gpu_match(env, hist, query, 4, 8)
+    assert np.array_equal(rr, rr1) and np.array_equal(sp, sp1) and len(sp) > 3
+    # the same history in 50 requests: only matches that cross a boundary change
+    ix2 = GpuIndex(env, 20000, 4, 8)
+    bounds = np.linspace(0, 20000, 51).astype(np.int32)
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        ix2.append(hist[a:b])
+    rr2, sp2 = ix2.query(query, intra=True)
+    o_rr, o_sp = env.orc.match_spans_req(hist, bounds, query, w=4, max_hits=8, intra=True)
+    assert np.array_equal(rr2, o_rr) and np.array_equal(sp2, o_sp)
+    assert (o_rr >= 20000).sum() > 0
+    # reset: nothing matches any more
+    env.rac.rac_index_reset(ix2.cfg, ix2.mem[:ix2.nb], ix2.nb)
+    ix2.n = 0
+    rr3, sp3 = ix2.query(query)
+    assert len(sp3) == 0 and np.all(rr3 == -1)
+
+
+def test_index_argument_checks(env):
+    rac = env.rac
+    assert rac.rac_index_bytes(rac.IndexCfg(0, 4, 8)) == 0
+    assert rac.rac_index_bytes(rac.IndexCfg(100, 0, 8)) == 0
+    assert rac.rac_index_bytes(rac.IndexCfg(100, 4, 17)) == 0
+    cfg = rac.IndexCfg(100, 4, 8)
+    nb = rac.rac_index_bytes(cfg)
+    mem = torch.zeros(nb, dtype=torch.uint8, device=env.dev)
+    tok = torch.zeros(200, dtype=torch.int32, device=env.dev)
+    rac.rac_index_reset(cfg, mem, nb)
+    for fn, args, code in [
+        (rac.rac_index_reset, (cfg, mem, nb - 16), -3),
+        (rac.rac_index_append, (cfg, mem, nb, tok, 0, 101), -3),        # beyond the capacity
+        (rac.rac_index_append, (cfg, mem, nb, tok, 10, 5), -1),
+        (rac.rac_index_append, (cfg, mem[1:], nb - 1, tok, 0, 5), -2),
+    ]:
+        with pytest.raises(rac.RacError) as e:
+            fn(*args)
+        assert e.value.code == code
