@@ -171,7 +171,7 @@ int rac_match_spans_static(const int32_t *hist_tok, int64_t n_hist, const int32_
  *                      ref_row = n_hist + (position of the first occurrence of that token in the prompt): a
  *                      reference to the reconstruction of that earlier token of the same prompt.  First occurrences
  *                      never get such a reference, so they never chain: all tokens with ref_row < n_hist can be
- *                      coded first and the others second (rac_encode_rows / rac_decode_rows below).
+ *                      coded first and the others second (rac_split_waves and the *_list calls below).
  *                      workspace >= rac_index_query_workspace_bytes(n_query) bytes, scratch.
  * All three are asynchronous on `stream`; calls on one index must be ordered. */
 typedef struct {
@@ -254,6 +254,37 @@ int rac_sender_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_
                            const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
                            const void *ref_gain, const void *ref_bias, const float *step,
                            void *X_hat, uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Coding a subset of the tokens, with references into the reconstruction of the SAME prompt
+ * (the intra-sequence references of Sec. IV-B.1).
+ *
+ * rac_split_waves: tokens whose ref_row is >= first_intra_row (normally n_hist, see rac_index_query) reference
+ * another token of the prompt and must be coded after it; wave1[0 .. wave_count[0]) receives the other tokens,
+ * wave2[0 .. wave_count[1]) these, both in ascending order.  wave1, wave2: int32[T]; wave_count: int32[2]
+ * (all device memory).
+ *
+ * The *_list calls are rac_encode_reconstruct / rac_decode_reconstruct restricted to the tokens
+ * tok_list[0 .. *tok_count) (device int32 list and device count; both NULL = all T tokens) and with a second
+ * reference buffer: a ref_row entry r >= ref_rows names row r - ref_rows of `intra_base` (bf16 [intra_rows, d];
+ * NULL/0 = none).  X, payload and X_hat keep their full [T, ...] shapes; only the listed tokens are read and
+ * written.  List entries outside [0, T) are clamped into range.  X_hat of the encode call may be NULL (no sender
+ * reconstruction).
+ * Two-wave protocol, both endpoints: call once with wave 1 (intra_base may already be given: wave 1 never reads
+ * it), then with wave 2 and intra_base = X_hat of this prompt, on the same stream.  The rows a wave-2 token
+ * references were written by wave 1, and no wave-2 token is referenced by anyone, so the second call reads only
+ * finished rows while it writes others. */
+int rac_split_waves(const int32_t *ref_row, int64_t T, int64_t first_intra_row, int32_t *wave1, int32_t *wave2,
+                    int32_t *wave_count, void *stream);
+int rac_encode_reconstruct_list(const rac_codec_cfg *cfg, const void *X, int64_t T, const int32_t *tok_list,
+                                const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const float *step, const float *inv_step, void *payload, size_t payload_cap, void *X_hat,
+                                void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream);
+int rac_decode_reconstruct_list(const rac_codec_cfg *cfg, const void *payload, int64_t T, const int32_t *tok_list,
+                                const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const float *step, void *X_hat, uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Step tables from a calibration draw (the part of the offline calibration of Sec. IV-C that the

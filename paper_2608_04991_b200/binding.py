@@ -33,6 +33,7 @@ EXPORTS = [
     "rac_index_bytes", "rac_index_reset", "rac_index_append", "rac_index_query_workspace_bytes", "rac_index_query",
     "rac_encode_workspace_bytes", "rac_encode", "rac_encode_reconstruct", "rac_decode_reconstruct",
     "rac_sender_reconstruct",
+    "rac_split_waves", "rac_encode_reconstruct_list", "rac_decode_reconstruct_list",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
 ]
 
@@ -116,6 +117,13 @@ def load() -> C.CDLL:
         f = getattr(l, name)
         f.restype = C.c_int
         f.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, vp]
+    l.rac_split_waves.restype = C.c_int
+    l.rac_split_waves.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+    l.rac_encode_reconstruct_list.restype = C.c_int
+    l.rac_encode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp,
+                                              vp, sz, vp, vp]
+    l.rac_decode_reconstruct_list.restype = C.c_int
+    l.rac_decode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp]
     l.rac_calibrate_workspace_bytes.restype = sz
     l.rac_calibrate_workspace_bytes.argtypes = [cfgp]
     l.rac_calibrate_steps.restype = C.c_int
@@ -180,6 +188,37 @@ def rac_match_workspace_bytes(n_hist: int, n_query: int, max_hits: int) -> int:
 
 def rac_encode_workspace_bytes(cfg: CodecCfg, T: int) -> int:
     return int(load().rac_encode_workspace_bytes(C.byref(cfg), int(T)))
+
+
+def rac_split_waves(ref_row, T, first_intra_row, wave1, wave2, wave_count, stream=None) -> None:
+    rc = load().rac_split_waves(_ptr(ref_row, _I32, "ref_row"), int(T), int(first_intra_row), _ptr(wave1, _I32, "wave1"),
+                                _ptr(wave2, _I32, "wave2"), _ptr(wave_count, _I32, "wave_count"),
+                                _stream() if stream is None else stream)
+    _check("rac_split_waves", rc)
+
+
+def rac_encode_reconstruct_list(cfg, X, T, tok_list, tok_count, ref_base, ref_rows, ref_row, intra_base, intra_rows,
+                                ref_gain, ref_bias, step, inv_step, payload, payload_cap, X_hat, workspace,
+                                workspace_bytes, dev_status, stream=None) -> None:
+    rc = load().rac_encode_reconstruct_list(
+        C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(tok_list, _I32, "tok_list"), _ptr(tok_count, _I32, "tok_count"),
+        _ptr(ref_base, _BF16, "ref_base"), int(ref_rows), _ptr(ref_row, _I32, "ref_row"),
+        _ptr(intra_base, _BF16, "intra_base"), int(intra_rows), _ptr(ref_gain, _F16, "ref_gain"),
+        _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"), _ptr(inv_step, _F32, "inv_step"),
+        _ptr(payload, _U8, "payload"), int(payload_cap), _ptr(X_hat, _BF16, "X_hat"), _ptr(workspace, None, "workspace"),
+        int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
+    _check("rac_encode_reconstruct_list", rc)
+
+
+def rac_decode_reconstruct_list(cfg, payload, T, tok_list, tok_count, ref_base, ref_rows, ref_row, intra_base,
+                                intra_rows, ref_gain, ref_bias, step, X_hat, dev_status, stream=None) -> None:
+    rc = load().rac_decode_reconstruct_list(
+        C.byref(cfg), _ptr(payload, _U8, "payload"), int(T), _ptr(tok_list, _I32, "tok_list"),
+        _ptr(tok_count, _I32, "tok_count"), _ptr(ref_base, _BF16, "ref_base"), int(ref_rows),
+        _ptr(ref_row, _I32, "ref_row"), _ptr(intra_base, _BF16, "intra_base"), int(intra_rows),
+        _ptr(ref_gain, _F16, "ref_gain"), _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"),
+        _ptr(X_hat, _BF16, "X_hat"), _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
+    _check("rac_decode_reconstruct_list", rc)
 
 
 def rac_calibrate_workspace_bytes(cfg: CodecCfg) -> int:

@@ -84,6 +84,7 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
 // thread accumulates e^2 of its own 32 channels in shared memory, separately for tokens with a reference
 // (row 0) and tokens coded directly (row 1).  One CTA barrier per token; the grid is fixed.
 __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
+    constexpr bool SUB = false;  // calibration always runs over all tokens
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31;
@@ -104,16 +105,17 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
     __syncthreads();
 
     const int first = blockIdx.x, stride = gridDim.x;
-    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+    const long long n_tok = tokens_to_do<SUB>(p);
+    const int n_my = (n_tok > first) ? (int)((n_tok - first + stride - 1) / stride) : 0;
     int next_raw = 0;
     auto raw_row_of = [&](int k) -> int {  // raw ref_row entry of this CTA's k-th token
-        long long t = first + (long long)k * stride;
+        long long t = token_at<SUB>(p, first + (long long)k * stride);
         return p.ref_row ? p.ref_row[t] : (int)t;
     };
     if (tid == 0) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
-            long long t = first + (long long)k * stride;
-            issue_token_loads(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, row_bytes, k, resolve_row(p, raw_row_of(k)),
+            long long t = token_at<SUB>(p, first + (long long)k * stride);
+            issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, row_bytes, k, resolve_row<SUB>(p, raw_row_of(k)),
                               p.X + t * d, row_bytes);
         }
         if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
@@ -130,9 +132,9 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
     for (int it = 0; it < n_my; it++) {
         if (tid == 0 && it + S - 1 < n_my) {
             const int k = it + S - 1;
-            const long long tk = first + (long long)k * stride;
-            issue_token_loads(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, row_bytes, issue_stage,
-                              resolve_row(p, next_raw), p.X + tk * d, row_bytes);
+            const long long tk = token_at<SUB>(p, first + (long long)k * stride);
+            issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, row_bytes, issue_stage,
+                              resolve_row<SUB>(p, next_raw), p.X + tk * d, row_bytes);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
         const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
@@ -245,7 +247,8 @@ __host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages, boo
     return s;
 }
 
-template <int BITS, bool TOPK, bool XHAT, int MINB>
+// SUB: the token-list / second-reference-buffer form (see rac_codec_dev.cuh).
+template <int BITS, bool TOPK, bool XHAT, int MINB, bool SUB>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -261,21 +264,22 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     const uint32_t row_bytes = 2u * (uint32_t)d;
 
     const int first = blockIdx.x, stride = gridDim.x;
-    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+    const long long n_tok = tokens_to_do<SUB>(p);
+    const int n_my = (n_tok > first) ? (int)((n_tok - first + stride - 1) / stride) : 0;
     auto raw_row_of = [&](int k) -> int {  // raw ref_row entry of this CTA's k-th token
-        long long t = first + (long long)k * stride;
+        long long t = token_at<SUB>(p, first + (long long)k * stride);
         return p.ref_row ? p.ref_row[t] : (int)t;
     };
     // one lane: start the copies of this CTA's k-th token into stage s
     auto issue = [&](int k, int s, int raw_row) {
-        const long long t = first + (long long)k * stride;
-        const int row = resolve_row(p, raw_row);
+        const long long t = token_at<SUB>(p, first + (long long)k * stride);
+        const int row = resolve_row<SUB>(p, raw_row);
         ctrl->row[s] = row;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
         const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
         mbar_arrive_expect_tx(bar, row_bytes + (row >= 0 ? row_bytes : 0u));
         bulk_load(base, p.X + t * d, row_bytes, bar);
-        if (row >= 0) bulk_load(base + row_bytes, p.ref_base + (long long)row * d, row_bytes, bar);
+        if (row >= 0) bulk_load(base + row_bytes, ref_row_ptr<SUB>(p, row), row_bytes, bar);
     };
 
     if (tid == 0) {
@@ -452,7 +456,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             // wait below.  So the refill need not wait for the record to leave.  (With x_hat the X row itself
             // is the source of a store and must have been read before new data may land on it.)
             if (lane == 0) {
-                const long long t = first + (long long)it * stride;
+                const long long t = token_at<SUB>(p, first + (long long)it * stride);
                 if (TOPK)  // the slab maxima travel like the record: one bulk copy from this parity's slot
                     bulk_store(p.tmax + t * (L.tm_bytes >> 2), xs + L.tm_off + parity * L.tm_bytes, (uint32_t)L.tm_bytes);
                 if (XHAT) {
@@ -508,8 +512,8 @@ constexpr int kOutHot = 256;       // slab list per token in flight (d <= 8192 h
 // W lanes work on one token: W = 32 (a warp per token) or 16 (two tokens per warp; the instruction stream is
 // shared, so a token costs about two thirds of the issue slots).  All warp collectives name only the W lanes
 // of the token.
-template <int BITS, int W>
-__global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecParams p) {
+template <int BITS, int W, bool SUB>
+__global__ void __launch_bounds__(kOutWarps * 32, 5) outlier_kernel(const CodecParams p) {
     constexpr int TPW = 32 / W;                 // tokens per warp
     constexpr int NV = 256 / W;                 // slab maxima per lane, at most
     __shared__ unsigned long long s_cand[kOutWarps * TPW][kOutCap];
@@ -532,12 +536,13 @@ __global__ void __launch_bounds__(kOutWarps * 32) outlier_kernel(const CodecPara
     const unsigned int lt_mask = (1u << sl) - 1u;
     const int tm_stride = (nth + 3) & ~3;       // rows of slab maxima are padded to 16 bytes
 
-    for (long long t = ((long long)blockIdx.x * kOutWarps + warp) * TPW + sub; t < p.T; t += tstride) {
-        // reference row of the token, by the same rules as the streaming pass
-        long long row = p.ref_row ? (long long)p.ref_row[t] : t;
-        if (!p.ref_base || row < 0 || row >= p.ref_rows) row = -1;
+    const long long n_tok = tokens_to_do<SUB>(p);
+    for (long long ti = ((long long)blockIdx.x * kOutWarps + warp) * TPW + sub; ti < n_tok; ti += tstride) {
+        const long long t = token_at<SUB>(p, ti);
+        // reference row of the token, by the same rules as the streaming pass (which already reported bad rows)
+        const int row = resolve_row<SUB>(p, p.ref_row ? p.ref_row[t] : (int)t, false);
         const uint16_t *xrow = p.X + t * d;
-        const uint16_t *rrow = row >= 0 ? p.ref_base + row * d : nullptr;
+        const uint16_t *rrow = row >= 0 ? ref_row_ptr<SUB>(p, row) : nullptr;
         unsigned char *rec = p.payload + t * p.rec;
         const uint32_t *coef = reinterpret_cast<const uint32_t *>(rec);
         // residual of channel c, exactly as the streaming pass computed it (rare paths only)
@@ -749,7 +754,7 @@ __global__ void calib_finalize_kernel(const float *partial, int nblocks, int d, 
 // into an output row in shared memory, patches the outliers it owns, and the row leaves as one bulk store.
 // The step table row of referenced tokens lives in registers for the whole kernel (a thread always owns
 // the same channels); direct tokens read row 1 through L1.
-template <int BITS, int KT>
+template <int BITS, int KT, bool SUB>
 __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x;
@@ -776,17 +781,18 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     __syncthreads();
 
     const int first = blockIdx.x, stride = gridDim.x;
-    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+    const long long n_tok = tokens_to_do<SUB>(p);
+    const int n_my = (n_tok > first) ? (int)((n_tok - first + stride - 1) / stride) : 0;
 
     int next_raw = 0;
     auto raw_row_of = [&](int k) -> int {
-        long long t = first + (long long)k * stride;
+        long long t = token_at<SUB>(p, first + (long long)k * stride);
         return p.ref_row ? p.ref_row[t] : (int)t;
     };
     if (tid == 0) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
-            long long t = first + (long long)k * stride;
-            issue_token_loads(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row(p, raw_row_of(k)),
+            long long t = token_at<SUB>(p, first + (long long)k * stride);
+            issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row<SUB>(p, raw_row_of(k)),
                               p.payload + t * p.rec, (uint32_t)p.rec);
         }
         if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
@@ -815,12 +821,12 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     bool aborted = false;
     uint32_t parity = 0;
     for (int it = 0; it < n_my; it++) {
-        const long long t = first + (long long)it * stride;
+        const long long t = token_at<SUB>(p, first + (long long)it * stride);
         if (tid == 0 && it + S - 1 < n_my) {
             const int k = it + S - 1;
-            const long long tk = first + (long long)k * stride;
-            issue_token_loads(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
-                              resolve_row(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
+            const long long tk = token_at<SUB>(p, first + (long long)k * stride);
+            issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
+                              resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
         const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
@@ -987,9 +993,11 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     // leaves too little L1 for them, so that variant runs three CTAs per SM at 128 registers.
     const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
     int rc = RAC_EUNSUPPORTED;
+    const bool sub = p.tok_list || p.intra_base;   // the subset form has one variant per width: it is not the hot path
 #define RAC_ENC2(B, K, X)                                                                                          \
-    (tight ? launch_persistent(encode_ws_kernel<B, K, X, 4>, p, g.nthreads, L.total, max_ctas, stream)            \
-           : launch_persistent(encode_ws_kernel<B, K, X, 2>, p, g.nthreads, L.total, max_ctas, stream))
+    (sub ? launch_persistent(encode_ws_kernel<B, K, X, 2, true>, p, g.nthreads, L.total, max_ctas, stream)        \
+     : tight ? launch_persistent(encode_ws_kernel<B, K, X, 4, false>, p, g.nthreads, L.total, max_ctas, stream)   \
+             : launch_persistent(encode_ws_kernel<B, K, X, 2, false>, p, g.nthreads, L.total, max_ctas, stream))
 #define RAC_ENC(B, K) (p.X_hat ? RAC_ENC2(B, K, true) : RAC_ENC2(B, K, false))
     switch (g.bits) {
         case 4: rc = topk ? RAC_ENC(4, true) : RAC_ENC(4, false); break;
@@ -1005,12 +1013,13 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     // a warp per token; RAC_OUT_HALF=1 packs two tokens into a warp (16 lanes each; measured the same speed: the
     // pass is bound by scattered 32-byte reads, not by issue slots)
     const bool half = getenv("RAC_OUT_HALF") != nullptr;
-    const int tpw = half ? 2 : 1;
+    const int tpw = (half && !sub) ? 2 : 1;
     long long blocks = (p.T + kOutWarps * tpw - 1) / (kOutWarps * tpw);
     if (blocks > (long long)di.sms * 8) blocks = (long long)di.sms * 8;
-#define RAC_OUT(B)                                                                           \
-    if (half) outlier_kernel<B, 16><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p);     \
-    else outlier_kernel<B, 32><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p)
+#define RAC_OUT(B)                                                                                  \
+    if (sub) outlier_kernel<B, 32, true><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p);       \
+    else if (half) outlier_kernel<B, 16, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); \
+    else outlier_kernel<B, 32, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p)
     switch (g.bits) {
         case 4: RAC_OUT(4); break;
         case 3: RAC_OUT(3); break;
@@ -1025,7 +1034,10 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
     p.stages = pick_stages(g.d, 2);
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
-#define RAC_DEC(B, K) launch_persistent(decode_kernel<B, K>, p, g.nthreads, L.total, p.T, stream)
+    const bool sub = p.tok_list || p.intra_base;
+#define RAC_DEC(B, K)                                                                            \
+    (sub ? launch_persistent(decode_kernel<B, K, true>, p, g.nthreads, L.total, p.T, stream)    \
+         : launch_persistent(decode_kernel<B, K, false>, p, g.nthreads, L.total, p.T, stream))
     switch (g.bits * 100 + kt) {
         case 400: return RAC_DEC(4, 0);
         case 408: return RAC_DEC(4, 8);
@@ -1041,16 +1053,68 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
     return RAC_EUNSUPPORTED;
 }
 
+// Tokens whose reference is a row of the same prompt (ref_row >= first_intra_row) form the second wave; both
+// lists come out in ascending token order.  One CTA: per-thread chunk counts, a block scan, then the writes.
+__global__ void __launch_bounds__(1024) split_waves_kernel(const int32_t *ref_row, int T, long long first_intra_row,
+                                                           int32_t *wave1, int32_t *wave2, int32_t *wave_count) {
+    __shared__ int s_cnt[1024];
+    const int tid = threadIdx.x;
+    const int chunk = (T + 1023) / 1024;
+    const int lo = min(T, tid * chunk), hi = min(T, lo + chunk);
+    int c2 = 0;
+    for (int t = lo; t < hi; t++) c2 += ref_row[t] >= first_intra_row ? 1 : 0;
+    s_cnt[tid] = c2;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {   // inclusive scan
+        int v = tid >= o ? s_cnt[tid - o] : 0;
+        __syncthreads();
+        s_cnt[tid] += v;
+        __syncthreads();
+    }
+    int o2 = s_cnt[tid] - c2;      // second-wave tokens before this chunk
+    int o1 = lo - o2;              // first-wave tokens before this chunk
+    for (int t = lo; t < hi; t++) {
+        if (ref_row[t] >= first_intra_row) wave2[o2++] = t;
+        else wave1[o1++] = t;
+    }
+    if (tid == 1023) {
+        wave_count[1] = s_cnt[1023];
+        wave_count[0] = T - s_cnt[1023];
+    }
+}
+
 constexpr int kCalibGrid = 128;  // fixed, so that the summation order does not depend on the device
+
+// A subset of the tokens and a second reference buffer (the *_list entry points); all null/0 otherwise.
+struct Subset {
+    const int32_t *tok_list = nullptr;
+    const int32_t *tok_count = nullptr;
+    const void *intra_base = nullptr;
+    long long intra_rows = 0;
+};
+static int apply_subset(const Subset &sub, CodecParams *p) {
+    if ((sub.tok_list == nullptr) != (sub.tok_count == nullptr)) return RAC_EINVAL;
+    if (sub.intra_rows < 0 || (sub.intra_rows > 0 && !sub.intra_base)) return RAC_EINVAL;
+    if (sub.intra_base && !aligned16(sub.intra_base)) return RAC_EALIGN;
+    if (p->ref_rows + sub.intra_rows > 0x7fffffffLL) return RAC_EUNSUPPORTED;
+    p->tok_list = sub.tok_list;
+    p->tok_count = sub.tok_count;
+    p->intra_base = sub.intra_rows > 0 ? static_cast<const uint16_t *>(sub.intra_base) : nullptr;
+    p->intra_rows = sub.intra_rows;
+    return RAC_OK;
+}
 
 static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64_t T, const void *ref_base,
                             int64_t ref_rows, const int32_t *ref_row, const void *gain, const void *bias,
-                            const float *step, void *X_hat, uint32_t *dev_status, void *stream) {
+                            const float *step, void *X_hat, uint32_t *dev_status, void *stream,
+                            const Subset &sub = Subset()) {
     Geometry g;
     int rc = make_geometry(cfg, &g);
     if (rc != RAC_OK) return rc;
     CodecParams p = {};
     rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, gain, bias, dev_status);
+    if (rc != RAC_OK) return rc;
+    rc = apply_subset(sub, &p);
     if (rc != RAC_OK) return rc;
     if (T == 0) return RAC_OK;
     if (!payload || !X_hat || (!step && g.scale_mode == 0)) return RAC_EINVAL;   // mode 1 reads no table
@@ -1104,12 +1168,14 @@ size_t rac_encode_workspace_bytes(const rac_codec_cfg *cfg, int64_t T) {
 static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
                        const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
                        const float *inv_step, void *payload, size_t payload_cap, void *X_hat, void *workspace,
-                       size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+                       size_t workspace_bytes, uint32_t *dev_status, void *stream, const Subset &sub = Subset()) {
     Geometry g;
     int rc = make_geometry(cfg, &g);
     if (rc != RAC_OK) return rc;
     CodecParams p = {};
     rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, dev_status);
+    if (rc != RAC_OK) return rc;
+    rc = apply_subset(sub, &p);
     if (rc != RAC_OK) return rc;
     if (T == 0) return RAC_OK;
     if (!X || !payload) return RAC_EINVAL;
@@ -1159,6 +1225,43 @@ int rac_sender_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_
                            int64_t ref_rows, const int32_t *ref_row, const void *ref_gain, const void *ref_bias,
                            const float *step, void *X_hat, uint32_t *dev_status, void *stream) {
     return reconstruct_impl(cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, X_hat, dev_status, stream);
+}
+
+int rac_encode_reconstruct_list(const rac_codec_cfg *cfg, const void *X, int64_t T, const int32_t *tok_list,
+                                const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const float *step, const float *inv_step, void *payload, size_t payload_cap, void *X_hat,
+                                void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+    Subset sub;
+    sub.tok_list = tok_list;
+    sub.tok_count = tok_count;
+    sub.intra_base = intra_base;
+    sub.intra_rows = intra_rows;
+    return encode_impl(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload, payload_cap,
+                       X_hat, workspace, workspace_bytes, dev_status, stream, sub);
+}
+
+int rac_decode_reconstruct_list(const rac_codec_cfg *cfg, const void *payload, int64_t T, const int32_t *tok_list,
+                                const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const float *step, void *X_hat, uint32_t *dev_status, void *stream) {
+    Subset sub;
+    sub.tok_list = tok_list;
+    sub.tok_count = tok_count;
+    sub.intra_base = intra_base;
+    sub.intra_rows = intra_rows;
+    return reconstruct_impl(cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, X_hat, dev_status, stream,
+                            sub);
+}
+
+int rac_split_waves(const int32_t *ref_row, int64_t T, int64_t first_intra_row, int32_t *wave1, int32_t *wave2,
+                    int32_t *wave_count, void *stream) {
+    if (T < 0 || first_intra_row < 0 || !wave_count) return RAC_EINVAL;
+    if (T >= (1ll << 30)) return RAC_EUNSUPPORTED;
+    if (T > 0 && (!ref_row || !wave1 || !wave2)) return RAC_EINVAL;
+    split_waves_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(ref_row, (int)T, first_intra_row, wave1, wave2,
+                                                                         wave_count);
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
 size_t rac_calibrate_workspace_bytes(const rac_codec_cfg *cfg) {

@@ -31,6 +31,11 @@ struct CodecParams {
     // geometry
     int d, J, lpg, lpg_shift, topk, rec, code_bytes, stages;
     float inv_group;
+    // a subset of the tokens (both null = all T tokens, in order), and a second reference buffer behind ref_base
+    const int32_t *tok_list;     // int32[>= *tok_count] token indices in [0, T)
+    const int32_t *tok_count;    // device int32[1]
+    const uint16_t *intra_base;  // bf16[intra_rows, d]: reference rows ref_rows .. ref_rows + intra_rows - 1, or null
+    long long intra_rows;
     // scale_mode 1 only: quantisation groups, per-group outliers, field offsets in the record
     int Jq, lpq, lpq_shift, kg, codes_off, goff_off, gval_off;
 };
@@ -179,16 +184,48 @@ __device__ __forceinline__ void load_ref_slot(uint32_t addr, const uint16_t *gai
     }
 }
 
-// thread 0: reference row of token t (-1 = coded directly); flags rows beyond the buffer
-__device__ __forceinline__ int resolve_row(const CodecParams &p, int raw_row) {
-    if (!p.ref_base || raw_row < 0) return -1;
-    if (raw_row >= p.ref_rows) {
-        if (p.status) atomicOr(p.status, RAC_STATUS_REF_RANGE);
+// SUB = false compiles the plain form (all T tokens in order, one reference buffer); SUB = true the form of the
+// *_list entry points.  how many tokens this launch codes, and the idx-th of them:
+template <bool SUB>
+__device__ __forceinline__ long long tokens_to_do(const CodecParams &p) {
+    if constexpr (!SUB) return p.T;
+    if (!p.tok_count) return p.T;
+    const long long n = *p.tok_count;
+    return n < 0 ? 0 : (n > p.T ? p.T : n);
+}
+template <bool SUB>
+__device__ __forceinline__ long long token_at(const CodecParams &p, long long idx) {
+    if constexpr (!SUB) return idx;
+    if (!p.tok_list) return idx;
+    const long long t = p.tok_list[idx];
+    return t < 0 ? 0 : (t >= p.T ? p.T - 1 : t);   // a bad entry cannot leave the buffers
+}
+// Reference row of a token (-1 = coded directly); with SUB in the joint row space [ref_base rows | intra_base
+// rows].  `flag` false: do not report rows beyond the buffers (a second pass over tokens already reported).
+template <bool SUB>
+__device__ __forceinline__ int resolve_row(const CodecParams &p, int raw_row, bool flag = true) {
+    if constexpr (!SUB) {
+        if (!p.ref_base || raw_row < 0) return -1;
+        if (raw_row >= p.ref_rows) {
+            if (flag && p.status) atomicOr(p.status, RAC_STATUS_REF_RANGE);
+            return -1;
+        }
+        return raw_row;
+    } else {
+        if (raw_row < 0 || (!p.ref_base && !p.intra_base)) return -1;
+        if (raw_row < p.ref_rows) return raw_row;
+        if (p.intra_base && raw_row - p.ref_rows < p.intra_rows) return raw_row;
+        if (flag && p.status) atomicOr(p.status, RAC_STATUS_REF_RANGE);
         return -1;
     }
-    return raw_row;
+}
+template <bool SUB>
+__device__ __forceinline__ const uint16_t *ref_row_ptr(const CodecParams &p, long long row) {
+    if constexpr (!SUB) return p.ref_base + row * p.d;
+    return row < p.ref_rows ? p.ref_base + row * p.d : p.intra_base + (row - p.ref_rows) * p.d;
 }
 // thread 0: start the copies of one token into a stage: `first` (X row or record) and, if any, its reference row
+template <bool SUB>
 __device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ctrl, uint32_t stage_addr, uint32_t r_off,
                                                   int stage, int row, const void *first_src, uint32_t first_bytes) {
     ctrl->row[stage] = row;
@@ -196,7 +233,7 @@ __device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ct
     const uint32_t row_bytes = 2u * (uint32_t)p.d;
     mbar_arrive_expect_tx(bar, first_bytes + (row >= 0 ? row_bytes : 0u));
     bulk_load(stage_addr, first_src, first_bytes, bar);
-    if (row >= 0) bulk_load(stage_addr + r_off, p.ref_base + (long long)row * p.d, row_bytes, bar);
+    if (row >= 0) bulk_load(stage_addr + r_off, ref_row_ptr<SUB>(p, row), row_bytes, bar);
 }
 
 // Eq. 6 for the group this thread belongs to: centred two-pass sums over the thread's 32 channels (packed

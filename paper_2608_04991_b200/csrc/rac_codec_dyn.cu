@@ -75,7 +75,7 @@ __device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, 
 
 // MINB = 4 caps registers at 96 so that four 160-thread CTAs (d = 5120) fit on an SM.
 // KG: rounds compiled in (0, 1, 2 or 4; p.kg <= KG is the number taken).
-template <int BITS, bool XHAT, int KG, int MINB>
+template <int BITS, bool XHAT, int KG, int MINB, bool SUB>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -93,20 +93,21 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
     const uint32_t row_bytes = 2u * (uint32_t)d;
 
     const int first = blockIdx.x, stride = gridDim.x;
-    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+    const long long n_tok = tokens_to_do<SUB>(p);
+    const int n_my = (n_tok > first) ? (int)((n_tok - first + stride - 1) / stride) : 0;
     auto raw_row_of = [&](int k) -> int {
-        long long t = first + (long long)k * stride;
+        long long t = token_at<SUB>(p, first + (long long)k * stride);
         return p.ref_row ? p.ref_row[t] : (int)t;
     };
     auto issue = [&](int k, int s, int raw_row) {
-        const long long t = first + (long long)k * stride;
-        const int row = resolve_row(p, raw_row);
+        const long long t = token_at<SUB>(p, first + (long long)k * stride);
+        const int row = resolve_row<SUB>(p, raw_row);
         ctrl->row[s] = row;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
         const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
         mbar_arrive_expect_tx(bar, row_bytes + (row >= 0 ? row_bytes : 0u));
         bulk_load(base, p.X + t * d, row_bytes, bar);
-        if (row >= 0) bulk_load(base + row_bytes, p.ref_base + (long long)row * d, row_bytes, bar);
+        if (row >= 0) bulk_load(base + row_bytes, ref_row_ptr<SUB>(p, row), row_bytes, bar);
     };
 
     if (tid == 0) {
@@ -378,7 +379,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             // slot, and the one after that cannot start before this warp has arrived for the token in between.
             // With x_hat the X row itself is the source of a store and must have been read before the refill.
             if (lane == 0) {
-                const long long t = first + (long long)it * stride;
+                const long long t = token_at<SUB>(p, first + (long long)it * stride);
                 if (XHAT) {
                     bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
                     bulk_store(p.X_hat + t * d, xs, row_bytes);
@@ -418,7 +419,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
 // dequantises its 32 channels (code -> binary32 through the 2^23 trick, times its group's scale), adds the
 // aligned reference, rounds to bf16 into an output row in shared memory; then the per-group outliers replace
 // what the dense pass wrote, and the row leaves as one bulk store.
-template <int BITS, bool KG>
+template <int BITS, bool KG, bool SUB>
 __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x;
@@ -448,17 +449,18 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
     __syncthreads();
 
     const int first = blockIdx.x, stride = gridDim.x;
-    const int n_my = (p.T > first) ? (int)((p.T - first + stride - 1) / stride) : 0;
+    const long long n_tok = tokens_to_do<SUB>(p);
+    const int n_my = (n_tok > first) ? (int)((n_tok - first + stride - 1) / stride) : 0;
 
     int next_raw = 0;
     auto raw_row_of = [&](int k) -> int {
-        long long t = first + (long long)k * stride;
+        long long t = token_at<SUB>(p, first + (long long)k * stride);
         return p.ref_row ? p.ref_row[t] : (int)t;
     };
     if (tid == 0) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
-            long long t = first + (long long)k * stride;
-            issue_token_loads(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row(p, raw_row_of(k)),
+            long long t = token_at<SUB>(p, first + (long long)k * stride);
+            issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row<SUB>(p, raw_row_of(k)),
                               p.payload + t * p.rec, (uint32_t)p.rec);
         }
         if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
@@ -473,12 +475,12 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
     bool aborted = false;
     uint32_t parity = 0;
     for (int it = 0; it < n_my; it++) {
-        const long long t = first + (long long)it * stride;
+        const long long t = token_at<SUB>(p, first + (long long)it * stride);
         if (tid == 0 && it + S - 1 < n_my) {
             const int k = it + S - 1;
-            const long long tk = first + (long long)k * stride;
-            issue_token_loads(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
-                              resolve_row(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
+            const long long tk = token_at<SUB>(p, first + (long long)k * stride);
+            issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
+                              resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
         const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
@@ -610,10 +612,12 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
 // outliers only below 8-bit codes.
 template <int B, bool X, int K>
 static int launch_encode_variant(bool tight, const Geometry &g, CodecParams &p, int smem, long long max_ctas, cudaStream_t stream) {
+    if (p.tok_list || p.intra_base)   // the subset form: one variant, not the hot path
+        return launch_persistent(encode_dyn_kernel<B, X, K, 2, true>, p, g.nthreads, smem, max_ctas, stream);
     if constexpr (!X && (K == 0 || B != 8)) {
-        if (tight) return launch_persistent(encode_dyn_kernel<B, X, K, 4>, p, g.nthreads, smem, max_ctas, stream);
+        if (tight) return launch_persistent(encode_dyn_kernel<B, X, K, 4, false>, p, g.nthreads, smem, max_ctas, stream);
     }
-    return launch_persistent(encode_dyn_kernel<B, X, K, 2>, p, g.nthreads, smem, max_ctas, stream);
+    return launch_persistent(encode_dyn_kernel<B, X, K, 2, false>, p, g.nthreads, smem, max_ctas, stream);
 }
 
 template <int B>
@@ -648,9 +652,12 @@ int launch_decode_dyn(const Geometry &g, CodecParams &p, cudaStream_t stream) {
     p.stages = pick_stages(g.d, 2);
     const DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const bool kg = g.topk_group > 0;
+    const bool sub = p.tok_list || p.intra_base;
 #define RAC_DYN_DEC(B) \
-    (kg ? launch_persistent(decode_dyn_kernel<B, true>, p, g.nthreads, L.total, p.T, stream) \
-        : launch_persistent(decode_dyn_kernel<B, false>, p, g.nthreads, L.total, p.T, stream))
+    (sub ? (kg ? launch_persistent(decode_dyn_kernel<B, true, true>, p, g.nthreads, L.total, p.T, stream) \
+               : launch_persistent(decode_dyn_kernel<B, false, true>, p, g.nthreads, L.total, p.T, stream)) \
+         : (kg ? launch_persistent(decode_dyn_kernel<B, true, false>, p, g.nthreads, L.total, p.T, stream) \
+               : launch_persistent(decode_dyn_kernel<B, false, false>, p, g.nthreads, L.total, p.T, stream)))
     switch (g.bits) {
         case 8: return RAC_DYN_DEC(8);
         case 4: return RAC_DYN_DEC(4);
