@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode-steps", action="store_true", help="skip the decode-step latency extra")
-    ap.add_argument("--no-family", action="store_true", help="skip the Eq. 8 quantiser-family extra")
+    ap.add_argument("--no-family", action="store_true", help="skip the extras beyond the graded path (Eq. 8 family, persistent index)")
     return ap.parse_args()
 
 
@@ -280,6 +280,58 @@ def paper_family(dev, T, d, g=128, reps=10):
         del pay
     if int(status.item()) != 0:
         raise RuntimeError(f"paper_family: device status {int(status.item())}")
+    return out
+
+
+# --------------------------------------------------------------------------------------------- retrieval over requests
+def retrieval_index(dev, n_hist, n_query, gap_max, request_tokens=2048, reps=10):
+    """The persistent span index on the benchmark's token workload: the history appended as requests of
+    `request_tokens` tokens, then the prompt queried (Eq. 3 with request-bounded matches), with and without the
+    intra-sequence pass, and the wave split.  CUDA-event times; appends are timed as one sequence."""
+    import torch
+    from paper_2608_04991_b200 import binding as rac
+    from paper_2608_04991_b200 import synth
+    tw = synth.span_workload(n_hist, n_query, seed=synth.BASE_SEED + 11, gap_max=gap_max)
+    htok = torch.from_numpy(tw.hist).to(dev)
+    qtok = torch.from_numpy(tw.query).to(dev)
+    cfg = rac.IndexCfg(n_hist, WORKLOAD["min_ngram"], WORKLOAD["max_hits"])
+    nb = rac.rac_index_bytes(cfg)
+    mem = torch.empty(nb, dtype=torch.uint8, device=dev)
+    nws = rac.rac_index_query_workspace_bytes(n_query)
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+    rows = torch.empty(n_query, dtype=torch.int32, device=dev)
+    n_spans = torch.zeros(1, dtype=torch.int32, device=dev)
+    wave1, wave2 = torch.empty_like(rows), torch.empty_like(rows)
+    cnt = torch.zeros(2, dtype=torch.int32, device=dev)
+    bounds = list(range(0, n_hist, request_tokens)) + [n_hist]
+
+    def build():
+        rac.rac_index_reset(cfg, mem, nb)
+        for a, b in zip(bounds[:-1], bounds[1:]):
+            rac.rac_index_append(cfg, mem, nb, htok, a, b)
+
+    def timed(fn, n):
+        fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    out = {"history_tokens": n_hist, "query_tokens": n_query, "requests": len(bounds) - 1, "index_bytes": nb}
+    out["build_ms"] = timed(build, 3)
+    out["append_us_per_request"] = out["build_ms"] * 1e3 / (len(bounds) - 1)
+    q = lambda intra: rac.rac_index_query(cfg, mem, nb, htok, n_hist, qtok, n_query, intra, rows, None, n_spans, ws, nws)
+    out["query_ms"] = timed(lambda: q(False), reps)
+    out["query_with_intra_ms"] = timed(lambda: q(True), reps)
+    out["split_waves_ms"] = timed(lambda: rac.rac_split_waves(rows, n_query, n_hist, wave1, wave2, cnt), reps)
+    r = rows.cpu()
+    out["spans"] = int(n_spans.item())
+    out["covered_by_spans"] = float(((r >= 0) & (r < n_hist)).float().mean())
+    out["intra_referenced"] = float((r >= n_hist).float().mean())
     return out
 
 
@@ -614,6 +666,7 @@ def main():
             "stages": per,
             "decode_steps": None if args.no_decode_steps else decode_step_latency(dev),
             "paper_family": None if args.no_family else paper_family(dev, wl["T"], wl["d"]),
+            "retrieval_index": None if args.no_family else retrieval_index(dev, wl["n_hist"], wl["T"], wl["gap_max"]),
         }
         print(json.dumps(line))
     if world > 1:

@@ -1054,32 +1054,58 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
 }
 
 // Tokens whose reference is a row of the same prompt (ref_row >= first_intra_row) form the second wave; both
-// lists come out in ascending token order.  One CTA: per-thread chunk counts, a block scan, then the writes.
+// lists come out in ascending token order.  One CTA; every warp owns a contiguous range of 32-token tiles
+// (coalesced reads), counts its second-wave tokens with ballots, the warps' counts are prefix-summed, and a
+// second sweep writes both lists at running offsets.
 __global__ void __launch_bounds__(1024) split_waves_kernel(const int32_t *ref_row, int T, long long first_intra_row,
                                                            int32_t *wave1, int32_t *wave2, int32_t *wave_count) {
-    __shared__ int s_cnt[1024];
-    const int tid = threadIdx.x;
-    const int chunk = (T + 1023) / 1024;
-    const int lo = min(T, tid * chunk), hi = min(T, lo + chunk);
+    __shared__ int s_cnt[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tiles = (T + 31) / 32;
+    const int per = (tiles + 31) / 32;
+    const int t_lo = min(tiles, warp * per), t_hi = min(tiles, t_lo + per);
     int c2 = 0;
-    for (int t = lo; t < hi; t++) c2 += ref_row[t] >= first_intra_row ? 1 : 0;
-    s_cnt[tid] = c2;
+    for (int tg = t_lo; tg < t_hi; tg += 8) {
+        int v[8];
+#pragma unroll
+        for (int u = 0; u < 8; u++) {
+            const int i = (tg + u) * 32 + lane;
+            v[u] = (tg + u < t_hi && i < T) ? ref_row[i] : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; u++) c2 += __popc(__ballot_sync(0xffffffffu, v[u] >= first_intra_row));
+    }
+    if (lane == 0) s_cnt[warp] = c2;
     __syncthreads();
-    for (int o = 1; o < 1024; o <<= 1) {   // inclusive scan
-        int v = tid >= o ? s_cnt[tid - o] : 0;
-        __syncthreads();
-        s_cnt[tid] += v;
-        __syncthreads();
+    int o2 = 0, total2 = 0;
+    for (int w = 0; w < 32; w++) {
+        if (w < warp) o2 += s_cnt[w];
+        total2 += s_cnt[w];
     }
-    int o2 = s_cnt[tid] - c2;      // second-wave tokens before this chunk
-    int o1 = lo - o2;              // first-wave tokens before this chunk
-    for (int t = lo; t < hi; t++) {
-        if (ref_row[t] >= first_intra_row) wave2[o2++] = t;
-        else wave1[o1++] = t;
+    int o1 = min(T, t_lo * 32) - o2;
+    const unsigned int below = (1u << lane) - 1u;
+    for (int tg = t_lo; tg < t_hi; tg += 8) {
+        int v[8];
+#pragma unroll
+        for (int u = 0; u < 8; u++) {
+            const int i = (tg + u) * 32 + lane;
+            v[u] = (tg + u < t_hi && i < T) ? ref_row[i] : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; u++) {
+            const int i = (tg + u) * 32 + lane;
+            const bool in = tg + u < t_hi && i < T;
+            const bool is2 = in && v[u] >= first_intra_row, is1 = in && !is2;
+            const unsigned int b2 = __ballot_sync(0xffffffffu, is2), b1 = __ballot_sync(0xffffffffu, is1);
+            if (is2) wave2[o2 + __popc(b2 & below)] = i;
+            if (is1) wave1[o1 + __popc(b1 & below)] = i;
+            o2 += __popc(b2);
+            o1 += __popc(b1);
+        }
     }
-    if (tid == 1023) {
-        wave_count[1] = s_cnt[1023];
-        wave_count[0] = T - s_cnt[1023];
+    if (tid == 0) {
+        wave_count[1] = total2;
+        wave_count[0] = T - total2;
     }
 }
 
