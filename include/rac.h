@@ -302,6 +302,18 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T,
                         float *step, float *inv_step, void *workspace, size_t workspace_bytes,
                         uint32_t *dev_status, void *stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Reconstruction error of a sender-path run: the measurable half of the offline calibration of Sec. IV-C
+ * (there the sender's own reconstruction is run per candidate configuration, and quality is weighed against all
+ * the bytes of a record; the bytes are rac_record_bytes(), this call gives the error).
+ *   X, X_hat   bf16[T,d], d a multiple of 8
+ *   out        device double[3]: sum (x - x_hat)^2, sum x^2, max |x - x_hat|
+ *   workspace  >= rac_recon_error_workspace_bytes() bytes, 16-byte aligned scratch
+ * Sums are binary64 over a fixed partition in a fixed order: the result is the same on every run. */
+size_t rac_recon_error_workspace_bytes(void);
+int rac_recon_error(const void *X, const void *X_hat, int64_t T, int32_t d, double *out, void *workspace,
+                    size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

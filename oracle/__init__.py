@@ -309,3 +309,11 @@ def match_spans_req(hist: np.ndarray, req_off, query: np.ndarray, w: int = 4, ma
     if rc != 0:
         raise ValueError(f"orc_match_spans_req failed: {rc}")
     return ref_row, spans[: ns.value].copy()
+
+
+def recon_error(X_bits: np.ndarray, Xhat_bits: np.ndarray):
+    """Reconstruction error of a run, in float64: (sum (x - x_hat)^2, sum x^2, max |x - x_hat|)."""
+    x = bf16_to_f32(np.asarray(X_bits, np.uint16)).astype(np.float64)
+    y = bf16_to_f32(np.asarray(Xhat_bits, np.uint16)).astype(np.float64)
+    dlt = (x.astype(np.float32) - y.astype(np.float32)).astype(np.float64)   # the difference of two bf16 as binary32
+    return float((dlt * dlt).sum()), float((x * x).sum()), float(np.abs(dlt).max(initial=0.0))

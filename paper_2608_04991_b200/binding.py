@@ -35,6 +35,7 @@ EXPORTS = [
     "rac_sender_reconstruct",
     "rac_split_waves", "rac_encode_reconstruct_list", "rac_decode_reconstruct_list",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
+    "rac_recon_error_workspace_bytes", "rac_recon_error",
 ]
 
 
@@ -124,6 +125,10 @@ def load() -> C.CDLL:
                                               vp, sz, vp, vp]
     l.rac_decode_reconstruct_list.restype = C.c_int
     l.rac_decode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp]
+    l.rac_recon_error_workspace_bytes.restype = sz
+    l.rac_recon_error_workspace_bytes.argtypes = []
+    l.rac_recon_error.restype = C.c_int
+    l.rac_recon_error.argtypes = [vp, vp, i64, i32, vp, vp, sz, vp]
     l.rac_calibrate_workspace_bytes.restype = sz
     l.rac_calibrate_workspace_bytes.argtypes = [cfgp]
     l.rac_calibrate_steps.restype = C.c_int
@@ -219,6 +224,17 @@ def rac_decode_reconstruct_list(cfg, payload, T, tok_list, tok_count, ref_base, 
         _ptr(ref_gain, _F16, "ref_gain"), _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"),
         _ptr(X_hat, _BF16, "X_hat"), _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
     _check("rac_decode_reconstruct_list", rc)
+
+
+def rac_recon_error_workspace_bytes() -> int:
+    return int(load().rac_recon_error_workspace_bytes())
+
+
+def rac_recon_error(X, X_hat, T, d, out, workspace, workspace_bytes, stream=None) -> None:
+    rc = load().rac_recon_error(_ptr(X, _BF16, "X"), _ptr(X_hat, _BF16, "X_hat"), int(T), int(d), _ptr(out, None, "out"),
+                                _ptr(workspace, None, "workspace"), int(workspace_bytes),
+                                _stream() if stream is None else stream)
+    _check("rac_recon_error", rc)
 
 
 def rac_calibrate_workspace_bytes(cfg: CodecCfg) -> int:

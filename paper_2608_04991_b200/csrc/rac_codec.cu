@@ -1109,6 +1109,58 @@ __global__ void __launch_bounds__(1024) split_waves_kernel(const int32_t *ref_ro
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// reconstruction error of a sender-path run (input of the byte-cost side of calibration, Sec. IV-C)
+// ------------------------------------------------------------------------------------------------
+constexpr int kErrGrid = 592;     // fixed, so that the summation order does not depend on the device
+constexpr int kErrThreads = 256;
+
+// partial[b] = (sum (x - x_hat)^2, sum x^2, max |x - x_hat|) over the 8-element chunks b, b + grid, ...
+__global__ void __launch_bounds__(kErrThreads) recon_error_kernel(const uint4 *X, const uint4 *Xh, long long n8,
+                                                                  double *partial) {
+    double se = 0.0, sx = 0.0;
+    float mx = 0.f;
+    for (long long i = blockIdx.x * (long long)kErrThreads + threadIdx.x; i < n8; i += (long long)kErrGrid * kErrThreads) {
+        const uint4 a = X[i], b = Xh[i];
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            const float x0 = __uint_as_float(aw[k] << 16), x1 = __uint_as_float(aw[k] & 0xffff0000u);
+            const float y0 = __uint_as_float(bw[k] << 16), y1 = __uint_as_float(bw[k] & 0xffff0000u);
+            const float d0 = __fsub_rn(x0, y0), d1 = __fsub_rn(x1, y1);   // exact or one rounding: both are bf16
+            se += (double)d0 * (double)d0 + (double)d1 * (double)d1;
+            sx += (double)x0 * (double)x0 + (double)x1 * (double)x1;
+            mx = fmaxf(mx, fmaxf(fabsf(d0), fabsf(d1)));
+        }
+    }
+    __shared__ double s_se[kErrThreads], s_sx[kErrThreads];
+    __shared__ float s_mx[kErrThreads];
+    s_se[threadIdx.x] = se; s_sx[threadIdx.x] = sx; s_mx[threadIdx.x] = mx;
+    __syncthreads();
+    for (int o = kErrThreads / 2; o > 0; o >>= 1) {   // fixed tree: the same order on every run
+        if (threadIdx.x < o) {
+            s_se[threadIdx.x] += s_se[threadIdx.x + o];
+            s_sx[threadIdx.x] += s_sx[threadIdx.x + o];
+            s_mx[threadIdx.x] = fmaxf(s_mx[threadIdx.x], s_mx[threadIdx.x + o]);
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        partial[3 * blockIdx.x + 0] = s_se[0];
+        partial[3 * blockIdx.x + 1] = s_sx[0];
+        partial[3 * blockIdx.x + 2] = (double)s_mx[0];
+    }
+}
+__global__ void recon_error_finalize_kernel(const double *partial, double *out) {
+    double se = 0.0, sx = 0.0, mx = 0.0;
+    for (int b = 0; b < kErrGrid; b++) {
+        se += partial[3 * b];
+        sx += partial[3 * b + 1];
+        mx = fmax(mx, partial[3 * b + 2]);
+    }
+    out[0] = se; out[1] = sx; out[2] = mx;
+}
+
 constexpr int kCalibGrid = 128;  // fixed, so that the summation order does not depend on the device
 
 // A subset of the tokens and a second reference buffer (the *_list entry points); all null/0 otherwise.
@@ -1287,6 +1339,23 @@ int rac_split_waves(const int32_t *ref_row, int64_t T, int64_t first_intra_row, 
     if (T > 0 && (!ref_row || !wave1 || !wave2)) return RAC_EINVAL;
     split_waves_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(ref_row, (int)T, first_intra_row, wave1, wave2,
                                                                          wave_count);
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+size_t rac_recon_error_workspace_bytes(void) { return (size_t)kErrGrid * 3 * sizeof(double); }
+
+int rac_recon_error(const void *X, const void *X_hat, int64_t T, int32_t d, double *out, void *workspace,
+                    size_t workspace_bytes, void *stream) {
+    if (T < 0 || d <= 0 || !out || !workspace) return RAC_EINVAL;
+    if (d % 8) return RAC_EUNSUPPORTED;
+    if (T > 0 && (!X || !X_hat)) return RAC_EINVAL;
+    if (!aligned16(X) || !aligned16(X_hat) || !aligned16(workspace) || (reinterpret_cast<uintptr_t>(out) & 7u)) return RAC_EALIGN;
+    if (workspace_bytes < rac_recon_error_workspace_bytes()) return RAC_ESIZE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double *partial = static_cast<double *>(workspace);
+    recon_error_kernel<<<kErrGrid, kErrThreads, 0, st>>>(static_cast<const uint4 *>(X), static_cast<const uint4 *>(X_hat),
+                                                       (long long)T * d / 8, partial);
+    recon_error_finalize_kernel<<<1, 1, 0, st>>>(partial, out);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
