@@ -68,6 +68,11 @@ def _declare(l: C.CDLL) -> None:
     l.orc_record_bytes_mode.argtypes = [C.c_int] * 5
     l.orc_record_bytes_ext.restype = C.c_int64
     l.orc_record_bytes_ext.argtypes = [C.c_int] * 7
+    l.orc_record_bytes_full.restype = C.c_int64
+    l.orc_record_bytes_full.argtypes = [C.c_int] * 8
+    l.orc_fit_segments.restype = C.c_int
+    l.orc_fit_segments.argtypes = [C.c_int, C.c_int, _u16p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
+                                   _i32p, C.c_int32, _u32p, _f64p, _f64p, _f64p, _f64p]
     l.orc_pack_codes.restype = None
     l.orc_pack_codes.argtypes = [_i32p, C.c_int, C.c_int, _u8p]
     l.orc_unpack_codes.restype = None
@@ -75,11 +80,11 @@ def _declare(l: C.CDLL) -> None:
     l.orc_fit_group.restype = None
     l.orc_fit_group.argtypes = [_f32p, _f32p, C.c_int, C.c_int, _f64p, _f64p, _f64p, _f64p]
     l.orc_encode.restype = C.c_int
-    l.orc_encode.argtypes = [C.c_int] * 7 + [_u16p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
+    l.orc_encode.argtypes = [C.c_int] * 8 + [_u16p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
                                              _f32p, _f32p, _u32p, _u8p,
                                              _f64p, _f64p, _f64p, _f64p, _f32p, _f32p, C.c_int]
     l.orc_reconstruct.restype = C.c_int
-    l.orc_reconstruct.argtypes = [C.c_int] * 7 + [_u8p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
+    l.orc_reconstruct.argtypes = [C.c_int] * 8 + [_u32p, _u8p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
                                                   _f32p, _u16p, _u32p, C.c_int]
     l.orc_calibrate.restype = C.c_int
     l.orc_calibrate.argtypes = [C.c_int] * 3 + [_u16p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
@@ -145,30 +150,31 @@ def max_threads() -> int:
 
 # ---------------------------------------------------------------- geometry
 def record_bytes(d: int, group: int, bits: int, topk: int, scale_mode: int = 0, qgroup: int = 0,
-                 topk_group: int = 0) -> int:
-    return int(lib().orc_record_bytes_ext(d, group, bits, topk, scale_mode, qgroup, topk_group))
+                 topk_group: int = 0, coef_fmt: int = 0) -> int:
+    return int(lib().orc_record_bytes_full(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt))
 
 
 def split_payload(payload: np.ndarray, T: int, d: int, group: int, bits: int, topk: int, scale_mode: int = 0,
-                  qgroup: int = 0, topk_group: int = 0):
+                  qgroup: int = 0, topk_group: int = 0, coef_fmt: int = 0):
     """Views into a payload: coef u32[T,J], codes u8[T,d*b/8], out_idx u16[T,k], out_val u16[T,k];
     for scale_mode 1 also scale u16[T,Jq] as a fifth item, and with per-group outliers
     grp_off u8[T,Jq,kg] and grp_val u16[T,Jq,kg] as a sixth and seventh."""
     J = d // group
     qg = qgroup or group
     Jq = d // qg
-    rec = record_bytes(d, group, bits, topk, scale_mode, qgroup, topk_group)
+    rec = record_bytes(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt)
     p = payload.reshape(T, rec)
     nb = d * bits // 8
     sb = (2 * Jq + 3) // 4 * 4 if scale_mode == 1 else 0
-    o = 4 * J + sb
-    coef = np.ascontiguousarray(p[:, : 4 * J]).view(np.uint32)
+    cb = 0 if coef_fmt == 1 else 4 * J          # shared coefficients travel outside the record: coef comes back empty
+    o = cb + sb
+    coef = np.ascontiguousarray(p[:, : cb]).view(np.uint32)
     codes = np.ascontiguousarray(p[:, o: o + nb])
     oi = np.ascontiguousarray(p[:, o + nb: o + nb + 2 * topk]).view(np.uint16)
     ov = np.ascontiguousarray(p[:, o + nb + 2 * topk: o + nb + 4 * topk]).view(np.uint16)
     if scale_mode != 1:
         return coef, codes, oi, ov
-    scale = np.ascontiguousarray(p[:, 4 * J: 4 * J + 2 * Jq]).view(np.uint16)
+    scale = np.ascontiguousarray(p[:, cb: cb + 2 * Jq]).view(np.uint16)
     if not topk_group:
         return coef, codes, oi, ov, scale
     ng = Jq * topk_group
@@ -205,7 +211,8 @@ def fit_group(h: np.ndarray, r: np.ndarray, has_ref: bool = True):
 
 
 def encode(d, group, bits, topk, X, ref_base=None, ref_row=None, gain=None, bias=None,
-           step=None, inv_step=None, forced_coef=None, diag=False, nthreads=1, scale_mode=0, qgroup=0, topk_group=0):
+           step=None, inv_step=None, forced_coef=None, diag=False, nthreads=1, scale_mode=0, qgroup=0, topk_group=0,
+           coef_fmt=0):
     """Encode X (uint16 bf16 bits [T,d]).  Returns payload (uint8[T*rec]) and, with
     ``diag=True``, a dict of the unrounded fit and the binary32 residual / scaled value."""
     X = _chk(X, np.uint16)
@@ -221,13 +228,13 @@ def encode(d, group, bits, topk, X, ref_base=None, ref_row=None, gain=None, bias
     assert scale_mode == 1 or (step is not None and inv_step is not None), "scale_mode 0 needs the step tables"
     J = d // group
     forced_coef = _chk(forced_coef, np.uint32, T * J)
-    rec = record_bytes(d, group, bits, topk, scale_mode, qgroup, topk_group)
+    rec = record_bytes(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt)
     payload = np.zeros(T * rec, np.uint8)
     dg = {}
     if diag:
         dg = dict(alpha=np.zeros((T, J)), beta=np.zeros((T, J)), hbar=np.zeros((T, J)), rbar=np.zeros((T, J)),
                   e=np.zeros((T, d), np.float32), v=np.zeros((T, d), np.float32))
-    rc = lib().orc_encode(d, group, bits, topk, scale_mode, qgroup, topk_group, _p(X, _u16p), T, _p(ref_base, _u16p), ref_rows,
+    rc = lib().orc_encode(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt, _p(X, _u16p), T, _p(ref_base, _u16p), ref_rows,
                           _p(ref_row, _i32p), _p(gain, _u16p), _p(bias, _u16p),
                           _p(step, _f32p), _p(inv_step, _f32p), _p(forced_coef, _u32p), _p(payload, _u8p),
                           _p(dg.get("alpha"), _f64p), _p(dg.get("beta"), _f64p),
@@ -239,9 +246,12 @@ def encode(d, group, bits, topk, X, ref_base=None, ref_row=None, gain=None, bias
 
 
 def reconstruct(d, group, bits, topk, payload, T, ref_base=None, ref_row=None, gain=None, bias=None,
-                step=None, nthreads=1, return_status=False, scale_mode=0, qgroup=0, topk_group=0):
-    """Eq. 9.  Returns X_hat as uint16 bf16 bits [T,d]."""
-    rec = record_bytes(d, group, bits, topk, scale_mode, qgroup, topk_group)
+                step=None, nthreads=1, return_status=False, scale_mode=0, qgroup=0, topk_group=0, coef_fmt=0,
+                shared_coef=None):
+    """Eq. 9.  Returns X_hat as uint16 bf16 bits [T,d].  ``coef_fmt=1``: the records hold no coefficients;
+    ``shared_coef`` uint32[T,J] gives every token the words of its segment."""
+    rec = record_bytes(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt)
+    shared_coef = _chk(shared_coef, np.uint32, T * (d // group))
     payload = _chk(payload, np.uint8, T * rec)
     ref_base = _chk(ref_base, np.uint16)
     ref_rows = 0 if ref_base is None else ref_base.size // d
@@ -251,7 +261,7 @@ def reconstruct(d, group, bits, topk, payload, T, ref_base=None, ref_row=None, g
     step = _chk(step, np.float32, 2 * d)
     out = np.zeros((T, d), np.uint16)
     st = C.c_uint32(0)
-    rc = lib().orc_reconstruct(d, group, bits, topk, scale_mode, qgroup, topk_group, _p(payload, _u8p), T, _p(ref_base, _u16p), ref_rows,
+    rc = lib().orc_reconstruct(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt, _p(shared_coef, _u32p), _p(payload, _u8p), T, _p(ref_base, _u16p), ref_rows,
                                _p(ref_row, _i32p), _p(gain, _u16p), _p(bias, _u16p), _p(step, _f32p),
                                _p(out, _u16p), C.byref(st), int(nthreads))
     if rc != 0:
@@ -317,3 +327,29 @@ def recon_error(X_bits: np.ndarray, Xhat_bits: np.ndarray):
     y = bf16_to_f32(np.asarray(Xhat_bits, np.uint16)).astype(np.float64)
     dlt = (x.astype(np.float32) - y.astype(np.float32)).astype(np.float64)   # the difference of two bf16 as binary32
     return float((dlt * dlt).sum()), float((x * x).sum()), float(np.abs(dlt).max(initial=0.0))
+
+
+def fit_segments(d, group, X, seg_off, ref_base=None, ref_row=None, gain=None, bias=None, diag=False):
+    """Eq. 6 over several fitting positions: one wire coefficient word per (segment, group).
+    ``seg_off`` int32[n_seg+1].  Returns coef uint32[n_seg, J] (and the unrounded fit with ``diag``)."""
+    X = _chk(X, np.uint16)
+    T = X.size // d
+    ref_base = _chk(ref_base, np.uint16)
+    ref_rows = 0 if ref_base is None else ref_base.size // d
+    ref_row = _chk(ref_row, np.int32, T)
+    gain = _chk(gain, np.uint16, d)
+    bias = _chk(bias, np.uint16, d)
+    seg_off = _chk(np.asarray(seg_off, np.int32), np.int32)
+    n_seg = seg_off.size - 1
+    J = d // group
+    coef = np.zeros((n_seg, J), np.uint32)
+    dg = {}
+    if diag:
+        dg = dict(alpha=np.zeros((n_seg, J)), beta=np.zeros((n_seg, J)), hbar=np.zeros((n_seg, J)), rbar=np.zeros((n_seg, J)))
+    rc = lib().orc_fit_segments(d, group, _p(X, _u16p), T, _p(ref_base, _u16p), ref_rows, _p(ref_row, _i32p),
+                                _p(gain, _u16p), _p(bias, _u16p), _p(seg_off, _i32p), n_seg, _p(coef, _u32p),
+                                _p(dg.get("alpha"), _f64p), _p(dg.get("beta"), _f64p), _p(dg.get("hbar"), _f64p),
+                                _p(dg.get("rbar"), _f64p))
+    if rc != 0:
+        raise ValueError(f"orc_fit_segments failed: {rc}")
+    return (coef, dg) if diag else coef

@@ -164,13 +164,18 @@ static int64_t scale_bytes(int d, int qgroup, int scale_mode) {
     return scale_mode == 1 ? (2 * (int64_t)(d / qgroup) + 3) / 4 * 4 : 0;
 }
 
-/* qgroup 0 means "same as group"; topk_group outliers per quantisation group */
-int64_t orc_record_bytes_ext(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group) {
+/* qgroup 0 means "same as group"; topk_group outliers per quantisation group; coef_fmt 1: the coefficient
+ * pairs are shared by the tokens of a segment and travel outside the record */
+int64_t orc_record_bytes_full(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group, int coef_fmt) {
     if (qgroup == 0) qgroup = group;
     int64_t ng = (int64_t)(d / qgroup) * topk_group;
-    int64_t raw = 4 * (int64_t)(d / group) + scale_bytes(d, qgroup, scale_mode) + ((int64_t)d * bits) / 8 + 4 * (int64_t)topk +
-                  (ng + 1) / 2 * 2 + 2 * ng;
+    int64_t raw = (coef_fmt == 1 ? 0 : 4 * (int64_t)(d / group)) + scale_bytes(d, qgroup, scale_mode) + ((int64_t)d * bits) / 8 +
+                  4 * (int64_t)topk + (ng + 1) / 2 * 2 + 2 * ng;
     return (raw + 15) / 16 * 16;
+}
+
+int64_t orc_record_bytes_ext(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group) {
+    return orc_record_bytes_full(d, group, bits, topk, scale_mode, qgroup, topk_group, 0);
 }
 
 int64_t orc_record_bytes_mode(int d, int group, int bits, int topk, int scale_mode) {
@@ -279,6 +284,64 @@ void orc_fit_group(const float *h, const float *r, int g, int has_ref,
     if (rbar_out) *rbar_out = rbar;
 }
 
+/* Eq. 6 with several fitting positions: one (alpha, beta) per (segment, group), H_j and R_j being the
+ * [positions x g] slices of the segment's tokens (a token coded directly contributes r = 0).
+ * seg_off int32[n_seg+1], ascending, seg_off[0] = 0, seg_off[n_seg] = T.
+ * coef_out u32[n_seg*J] wire words; diag_* optional double[n_seg*J] (unrounded optimum and the two means).
+ * Centred two-pass sums in binary64 over all positions of the segment. */
+int orc_fit_segments(int d, int group, const uint16_t *X, int64_t T,
+                     const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                     const uint16_t *gain, const uint16_t *bias,
+                     const int32_t *seg_off, int32_t n_seg, uint32_t *coef_out,
+                     double *diag_alpha, double *diag_beta, double *diag_hbar, double *diag_rbar) {
+    if (d <= 0 || group <= 0 || d % group || n_seg < 0) return -1;
+    if ((gain == NULL) != (bias == NULL)) return -1;
+    if (n_seg > 0 && (seg_off[0] != 0 || seg_off[n_seg] != T)) return -1;
+    const int J = d / group;
+    float *r = (float *)malloc(sizeof(float) * d);
+    int err = 0;
+    for (int32_t k = 0; k < n_seg && !err; k++) {
+        const int64_t t0 = seg_off[k], t1 = seg_off[k + 1];
+        if (t1 < t0) { err = -1; break; }
+        for (int j = 0; j < J; j++) {
+            double sr = 0.0, sh = 0.0;
+            int any_ref = 0;
+            for (int64_t t = t0; t < t1; t++) {
+                int has = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
+                if (has < 0) { err = -2; break; }
+                any_ref |= has;
+                for (int c = j * group; c < (j + 1) * group; c++) {
+                    sr += (double)r[c];
+                    sh += (double)orc_bf16_to_f32(X[t * (int64_t)d + c]);
+                }
+            }
+            if (err) break;
+            const double n = (double)(t1 - t0) * group;
+            double rbar = n > 0 ? sr / n : 0.0, hbar = n > 0 ? sh / n : 0.0;
+            double sxx = 0.0, sxy = 0.0;
+            for (int64_t t = t0; t < t1; t++) {
+                resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
+                for (int c = j * group; c < (j + 1) * group; c++) {
+                    double dr = (double)r[c] - rbar;
+                    double dh = (double)orc_bf16_to_f32(X[t * (int64_t)d + c]) - hbar;
+                    sxx += dr * dr;
+                    sxy += dr * dh;
+                }
+            }
+            int degenerate = !any_ref || !(sxx > 1e-12) || !(fabs(sxy) < 65504.0 * sxx);
+            double as = 0.0, bs = hbar;
+            if (!degenerate) { as = sxy / sxx; bs = hbar - as * rbar; }
+            coef_out[(int64_t)k * J + j] = (uint32_t)orc_f64_to_f16(as) | ((uint32_t)orc_f64_to_f16(bs) << 16);
+            if (diag_alpha) diag_alpha[(int64_t)k * J + j] = as;
+            if (diag_beta) diag_beta[(int64_t)k * J + j] = bs;
+            if (diag_hbar) diag_hbar[(int64_t)k * J + j] = hbar;
+            if (diag_rbar) diag_rbar[(int64_t)k * J + j] = rbar;
+        }
+    }
+    free(r);
+    return err;
+}
+
 /* ------------------------------------------------------------------ */
 /* encode                                                              */
 /* ------------------------------------------------------------------ */
@@ -300,7 +363,7 @@ static float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi
  *              and the scaled value v[T,d] the rounding decision was taken on.
  * returns 0, or -1 bad configuration, -2 ref_row out of range.
  */
-int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group,
+int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group, int coef_fmt,
                const uint16_t *X, int64_t T,
                const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
                const uint16_t *gain, const uint16_t *bias,
@@ -312,10 +375,13 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
     if (!cfg_ok(d, group, bits, topk)) return -1;
     if (!qcfg_ok(d, group, topk, scale_mode, qgroup, topk_group)) return -1;
     if ((gain == NULL) != (bias == NULL)) return -1;
+    if (coef_fmt != 0 && coef_fmt != 1) return -1;
+    if (coef_fmt == 1 && !forced_coef) return -1;      /* shared coefficients come from outside */
     if (qgroup == 0) qgroup = group;
     const int J = d / group, Jq = d / qgroup;
-    const int64_t rec = orc_record_bytes_ext(d, group, bits, topk, scale_mode, qgroup, topk_group);
+    const int64_t rec = orc_record_bytes_full(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt);
     const int64_t sbytes = scale_bytes(d, qgroup, scale_mode);
+    const int64_t cbytes = coef_fmt == 1 ? 0 : 4 * (int64_t)J;
     const int qmax = (1 << (bits - 1)) - 1;
     int err = 0;
     if (nthreads < 1) nthreads = 1;
@@ -330,7 +396,7 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
             uint8_t *recp = payload + t * rec;
             memset(recp, 0, rec);
             uint32_t *coef = (uint32_t *)recp;
-            uint8_t *scales = recp + 4 * J;
+            uint8_t *scales = recp + cbytes;
             uint8_t *codes = scales + sbytes;
             uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             uint8_t *oval = oidx + 2 * topk;
@@ -356,7 +422,7 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
                     a16 = orc_f64_to_f16(as); b16 = orc_f64_to_f16(bs);
                 }
                 uint32_t w = (uint32_t)a16 | ((uint32_t)b16 << 16);
-                memcpy(&coef[j], &w, 4);
+                if (coef_fmt == 0) memcpy(&coef[j], &w, 4);
                 if (diag_alpha) diag_alpha[t * J + j] = as;
                 if (diag_beta) diag_beta[t * J + j] = bs;
                 if (diag_hbar) diag_hbar[t * J + j] = hb;
@@ -463,7 +529,8 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
 /* X_hat bf16[T,d] out.  status (optional, one word) gets bit 1 when a reserved
  * code -2^(b-1) was seen.  returns 0, -1, -2 as orc_encode; -3 when an outlier
  * index is >= d. */
-int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group,
+int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group, int coef_fmt,
+                    const uint32_t *shared_coef,
                     const uint8_t *payload, int64_t T,
                     const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
                     const uint16_t *gain, const uint16_t *bias,
@@ -471,10 +538,13 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qg
     if (!cfg_ok(d, group, bits, topk)) return -1;
     if ((gain == NULL) != (bias == NULL)) return -1;
     if (!qcfg_ok(d, group, topk, scale_mode, qgroup, topk_group)) return -1;
+    if (coef_fmt != 0 && coef_fmt != 1) return -1;
+    if (coef_fmt == 1 && !shared_coef) return -1;      /* u32[T,J]: the words of each token's segment */
     if (qgroup == 0) qgroup = group;
     const int J = d / group, Jq = d / qgroup;
-    const int64_t rec = orc_record_bytes_ext(d, group, bits, topk, scale_mode, qgroup, topk_group);
+    const int64_t rec = orc_record_bytes_full(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt);
     const int64_t sbytes = scale_bytes(d, qgroup, scale_mode);
+    const int64_t cbytes = coef_fmt == 1 ? 0 : 4 * (int64_t)J;
     int err = 0;
     uint32_t st_word = 0;
     if (nthreads < 1) nthreads = 1;
@@ -485,7 +555,7 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qg
 #pragma omp for schedule(static)
         for (int64_t t = 0; t < T; t++) {
             const uint8_t *recp = payload + t * rec;
-            const uint8_t *scales = recp + 4 * J;
+            const uint8_t *scales = recp + cbytes;
             const uint8_t *codes = scales + sbytes;
             const uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             const uint8_t *oval = oidx + 2 * topk;
@@ -533,7 +603,8 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qg
             }
             for (int j = 0; j < J; j++) {
                 uint32_t w;
-                memcpy(&w, recp + 4 * j, 4);
+                if (coef_fmt == 1) w = shared_coef[t * J + j];
+                else memcpy(&w, recp + 4 * j, 4);
                 float a = orc_f16_to_f32((uint16_t)(w & 0xffff));
                 float b = orc_f16_to_f32((uint16_t)(w >> 16));
                 for (int c = j * group; c < (j + 1) * group; c++) {

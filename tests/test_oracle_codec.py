@@ -530,3 +530,84 @@ def _bad_offset_payload(orc, d, g):
     J, Jq = d // g, d // 32
     pay[4 * J + 2 * Jq + d // 2] = 32      # first in-group offset: 32 is outside a group of 32
     return pay
+
+
+# ------------------------------------------------------------------ Eq. 6 over several fitting positions
+def test_segment_fit_matches_library_least_squares_and_single_token_case(orc):
+    d, g, T = 256, 64, 37
+    J = d // g
+    gen = synth.generator(410)
+    X = synth.activations(T, d, synth.channel_scale(d, 11), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    Xb, Rb = synth.bf16_bits(X), synth.bf16_bits(R)
+    seg_off = np.array([0, 1, 9, 9, 30, 37], np.int32)            # a single token, an empty segment, longer ones
+    coef, dg = orc.fit_segments(d, g, Xb, seg_off, ref_base=Rb, diag=True)
+    h = orc.bf16_to_f32(Xb).astype(np.float64)
+    r = orc.bf16_to_f32(Rb).astype(np.float64)
+    for k in range(len(seg_off) - 1):
+        t0, t1 = seg_off[k], seg_off[k + 1]
+        for j in range(J):
+            hh = h[t0:t1, j * g:(j + 1) * g].reshape(-1)
+            rr = r[t0:t1, j * g:(j + 1) * g].reshape(-1)
+            if hh.size == 0:
+                assert coef[k, j] == 0                            # nothing to fit: alpha = 0, beta = 0
+                continue
+            A = np.stack([rr, np.ones_like(rr)], axis=1)          # the Frobenius problem of Eq. 6, solved by numpy
+            (a, b), *_ = np.linalg.lstsq(A, hh, rcond=None)
+            assert abs(dg["alpha"][k, j] - a) <= 1e-9 * max(1.0, abs(a))
+            assert abs(dg["beta"][k, j] - b) <= 1e-9 * max(1.0, abs(b))
+            assert coef[k, j] & 0xffff == np.float16(dg["alpha"][k, j]).view(np.uint16)
+            assert coef[k, j] >> 16 == np.float16(dg["beta"][k, j]).view(np.uint16)
+    # a segment of one token is the per-token fit
+    per_tok = orc.split_payload(orc.encode(d, g, 4, 0, Xb[:1], ref_base=Rb[:1], scale_mode=1), 1, d, g, 4, 0, 1)[0]
+    assert np.array_equal(coef[0], per_tok[0])
+    # no reference at all: alpha = 0, beta = the mean over all positions of the segment
+    c2, d2 = orc.fit_segments(d, g, Xb, seg_off, diag=True)
+    assert not (c2 & 0x7fff).any()
+    assert np.allclose(d2["beta"][3], h[9:30].reshape(21, J, g).mean(axis=(0, 2)), rtol=0, atol=1e-12)
+    # a pooled fit is never better than per-token fits on its own tokens, and equal when one map generated them all
+    a_true, b_true = 1.25, -0.5
+    Rc = synth.activations(8, d, synth.channel_scale(d, 12), gen)
+    Xc = (a_true * Rc.float() + b_true)
+    cc, dc = orc.fit_segments(d, g, synth.bf16_bits(Xc.to(torch.bfloat16)), np.array([0, 8], np.int32),
+                              ref_base=synth.bf16_bits(Rc), diag=True)
+    assert np.allclose(dc["alpha"], a_true, atol=2e-3) and np.allclose(dc["beta"], b_true, atol=2e-2)
+
+
+@pytest.mark.parametrize("mode", [dict(scale_mode=0, bits=4, topk=8), dict(scale_mode=1, bits=4, topk=0, topk_group=1),
+                                  dict(scale_mode=1, bits=8, topk=0, qgroup=512)])
+def test_shared_coefficients_leave_the_record_and_round_trip(orc, mode):
+    d, g, T = 512, 64, 40
+    J = d // g
+    gen = synth.generator(420)
+    X = synth.activations(T, d, synth.channel_scale(d, 13), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    Xb, Rb = synth.bf16_bits(X), synth.bf16_bits(R)
+    bits, topk = mode["bits"], mode["topk"]
+    kw = {k: v for k, v in mode.items() if k not in ("bits", "topk")}
+    seg_off = np.array([0, 8, 8, 25, 40], np.int32)
+    coef = orc.fit_segments(d, g, Xb, seg_off, ref_base=Rb)
+    seg_of = np.repeat(np.arange(len(seg_off) - 1), np.diff(seg_off))
+    per_tok = np.ascontiguousarray(coef[seg_of])                  # uint32[T, J]
+    step = inv = None
+    if kw["scale_mode"] == 0:
+        step, inv = orc.calibrate(d, g, bits, Xb, ref_base=Rb)
+    # the record shrinks by exactly the coefficient words (up to the 16-byte padding)
+    r0 = orc.record_bytes(d, g, bits, topk, kw["scale_mode"], kw.get("qgroup", 0), kw.get("topk_group", 0))
+    r1 = orc.record_bytes(d, g, bits, topk, kw["scale_mode"], kw.get("qgroup", 0), kw.get("topk_group", 0), 1)
+    assert r0 - 4 * J - 15 <= r1 <= r0 - 4 * J + 15 and r1 % 16 == 0
+    pay1 = orc.encode(d, g, bits, topk, Xb, ref_base=Rb, step=step, inv_step=inv, forced_coef=per_tok.reshape(-1).copy(),
+                      coef_fmt=1, **kw)
+    pay0 = orc.encode(d, g, bits, topk, Xb, ref_base=Rb, step=step, inv_step=inv, forced_coef=per_tok.reshape(-1).copy(), **kw)
+    assert pay1.size == T * r1
+    # same coefficients, same everything else: the two layouts differ only by the missing words
+    body0 = pay0.reshape(T, r0)[:, 4 * J:]
+    body1 = pay1.reshape(T, r1)
+    n = min(body0.shape[1], body1.shape[1])
+    assert np.array_equal(body0[:, :n], body1[:, :n]) and not body1[:, n:].any() and not body0[:, n:].any()
+    assert np.array_equal(pay0.reshape(T, r0)[:, :4 * J].copy().view(np.uint32), per_tok)
+    x1 = orc.reconstruct(d, g, bits, topk, pay1, T, ref_base=Rb, step=step, coef_fmt=1, shared_coef=per_tok, **kw)
+    x0 = orc.reconstruct(d, g, bits, topk, pay0, T, ref_base=Rb, step=step, **kw)
+    assert np.array_equal(x0, x1)
+    with pytest.raises(ValueError):
+        orc.encode(d, g, bits, topk, Xb, ref_base=Rb, step=step, inv_step=inv, coef_fmt=1, **kw)   # nothing to share
