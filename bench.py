@@ -283,6 +283,53 @@ def paper_family(dev, T, d, g=128, reps=10):
     return out
 
 
+# --------------------------------------------------------------------------------------------- shared coefficients
+def shared_coefficients(dev, T, d, g=128, seg_tokens=64, reps=10):
+    """Eq. 6 over several fitting positions on the benchmark's shape: one coefficient pair per (segment of
+    `seg_tokens` tokens, group), records without coefficient words (4-bit codes, scale per group).  Times of the
+    fit (statistics pass + merge), of the encode and of the reconstruction with the shared words."""
+    import torch
+    from paper_2608_04991_b200 import binding as rac
+    from paper_2608_04991_b200 import synth
+    gen = synth.generator(synth.BASE_SEED + 13, dev)
+    X = synth.activations(T, d, synth.channel_scale(d, 13, dev), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    cfg = rac.CodecCfg(d, g, 4, 0, scale_mode=1, coef_fmt=1)
+    rec = rac.rac_record_bytes(cfg)
+    n_seg = (T + seg_tokens - 1) // seg_tokens
+    seg_off = torch.clamp(torch.arange(n_seg + 1, dtype=torch.int32, device=dev) * seg_tokens, max=T).to(torch.int32)
+    coef = torch.empty((n_seg, d // g), dtype=torch.int32, device=dev)
+    seg_of = torch.empty(T, dtype=torch.int32, device=dev)
+    nb = rac.rac_fit_segments_workspace_bytes(cfg, T)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    pay = torch.empty(T * rec, dtype=torch.uint8, device=dev)
+    xh = torch.empty_like(X)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    fit = lambda: rac.rac_fit_segments(cfg, X, T, R, T, None, None, None, seg_off, n_seg, coef, seg_of, ws, nb, status)
+    enc = lambda: rac.rac_encode_reconstruct_list(cfg, X, T, None, None, R, T, None, None, 0, None, None, None, None, pay,
+                                                  pay.numel(), None, None, 0, status, coef_seg=coef, seg_of=seg_of)
+    dec = lambda: rac.rac_decode_reconstruct_list(cfg, pay, T, None, None, R, T, None, None, 0, None, None, None, xh,
+                                                  status, coef_seg=coef, seg_of=seg_of)
+    out = {"segment_tokens": seg_tokens, "segments": n_seg, "record_bytes": rec, "payload_over_raw": rec / (2.0 * d),
+           "shared_words_bytes_per_token": 4.0 * (d // g) / seg_tokens}
+    for key, fn, nbytes in (("fit", fit, T * 4 * d), ("encode", enc, T * (4 * d + rec)), ("reconstruct", dec, T * (4 * d + rec))):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        out[key + "_ms"] = ms
+        out[key + "_GBps"] = nbytes / (ms * 1e-3) / 1e9
+    if int(status.item()) != 0:
+        raise RuntimeError(f"shared_coefficients: device status {int(status.item())}")
+    return out
+
+
 # --------------------------------------------------------------------------------------------- retrieval over requests
 def retrieval_index(dev, n_hist, n_query, gap_max, request_tokens=2048, reps=10):
     """The persistent span index on the benchmark's token workload: the history appended as requests of
@@ -667,6 +714,7 @@ def main():
             "decode_steps": None if args.no_decode_steps else decode_step_latency(dev),
             "paper_family": None if args.no_family else paper_family(dev, wl["T"], wl["d"]),
             "retrieval_index": None if args.no_family else retrieval_index(dev, wl["n_hist"], wl["T"], wl["gap_max"]),
+            "shared_coefficients": None if args.no_family else shared_coefficients(dev, wl["T"], wl["d"]),
         }
         print(json.dumps(line))
     if world > 1:

@@ -25,7 +25,8 @@
  *    boundaries (d is a multiple of 32, base pointers 16-byte aligned).
  *
  * Wire record of one token (little endian), records back to back in `payload`:
- *     coef    J x u32      binary16 alpha in bits 0..15, binary16 beta in 16..31,  J = d/group
+ *     coef    J x u32      binary16 alpha in bits 0..15, binary16 beta in 16..31,  J = d/group (absent with
+ *                          coef_fmt 1)
  *     scale   Jq x u16     binary16 scales of the quantisation groups, scale_mode 1 only (Jq = d/qgroup),
  *                          padded to a multiple of 4 bytes
  *     codes   d*bits/8 B   code of channel c in stream bits [c*bits, c*bits+bits); stream bit n is
@@ -68,7 +69,9 @@ extern "C" {
  *   group   g_a, channels per alignment group; power of two, 32..1024, divides d
  *   bits    code width q: 2, 3 or 4; also 8 in scale_mode 1     (Qmax = 2^(bits-1) - 1, Eq. 8a)
  *   topk    outliers per TOKEN kept as binary16, 0..16 (u16 channel index); scale_mode 0 only
- *   coef_fmt   0 = binary16 pair (the only format)
+ *   coef_fmt   0 = one binary16 pair per (token, group), in the record
+ *              1 = one binary16 pair per (segment, group), outside the record (scale_mode 1 only; see
+ *                  rac_fit_segments): the record then starts with the scales
  *   scale_mode 0 = static per-channel step table `step`/`inv_step` (calibrated clip; dense values may clip);
  *                  g_q == g_a, `qgroup` 0 or == group, `topk_group` 0
  *              1 = Eq. 8 as printed: per quantisation group the scale s = RoundUp_binary16(max|E^d| / Qmax) is
@@ -278,13 +281,39 @@ int rac_split_waves(const int32_t *ref_row, int64_t T, int64_t first_intra_row, 
                     int32_t *wave_count, void *stream);
 int rac_encode_reconstruct_list(const rac_codec_cfg *cfg, const void *X, int64_t T, const int32_t *tok_list,
                                 const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
-                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const void *intra_base, int64_t intra_rows, const uint32_t *coef_seg, const int32_t *seg_of,
+                                const void *ref_gain, const void *ref_bias,
                                 const float *step, const float *inv_step, void *payload, size_t payload_cap, void *X_hat,
                                 void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream);
 int rac_decode_reconstruct_list(const rac_codec_cfg *cfg, const void *payload, int64_t T, const int32_t *tok_list,
                                 const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
-                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const void *intra_base, int64_t intra_rows, const uint32_t *coef_seg, const int32_t *seg_of,
+                                const void *ref_gain, const void *ref_bias,
                                 const float *step, void *X_hat, uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Eq. 6 over several fitting positions: one coefficient pair per (segment of consecutive tokens, group)
+ * instead of one per (token, group).  H_j and R_j of Eq. 6 are then the [positions x group] slices of the
+ * segment; a token coded directly contributes r = 0.  The pairs are shared by the tokens of the segment and
+ * travel once per segment, outside the records: rac_codec_cfg.coef_fmt = 1 (scale_mode 1 only) gives records
+ * without coefficient words.
+ *
+ * rac_fit_segments
+ *   seg_off   device int32[n_seg + 1], ascending, seg_off[0] = 0, seg_off[n_seg] = T; equal neighbours = an
+ *             empty segment (its pairs come out as 0).  Spans of the retrieval and the gaps between them are the
+ *             natural segments.
+ *   coef_seg  device u32[n_seg, J] out: binary16 alpha | binary16 beta << 16, the zero-variance rule as for a
+ *             single token
+ *   seg_of    device int32[T] out: the segment of every token
+ *   workspace >= rac_fit_segments_workspace_bytes(cfg, T) bytes, 16-byte aligned scratch
+ * Sums are merged in binary64 in a fixed order: the same result on every run.
+ * Coding: pass coef_seg and seg_of to the *_list calls (with tok_list NULL for all tokens) together with
+ * coef_fmt = 1; with coef_fmt = 0 both must be NULL. */
+size_t rac_fit_segments_workspace_bytes(const rac_codec_cfg *cfg, int64_t T);
+int rac_fit_segments(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+                     const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const int32_t *seg_off,
+                     int64_t n_seg, uint32_t *coef_seg, int32_t *seg_of, void *workspace, size_t workspace_bytes,
+                     uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Step tables from a calibration draw (the part of the offline calibration of Sec. IV-C that the

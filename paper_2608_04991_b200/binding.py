@@ -34,6 +34,7 @@ EXPORTS = [
     "rac_encode_workspace_bytes", "rac_encode", "rac_encode_reconstruct", "rac_decode_reconstruct",
     "rac_sender_reconstruct",
     "rac_split_waves", "rac_encode_reconstruct_list", "rac_decode_reconstruct_list",
+    "rac_fit_segments_workspace_bytes", "rac_fit_segments",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
     "rac_recon_error_workspace_bytes", "rac_recon_error",
 ]
@@ -51,8 +52,8 @@ class CodecCfg(C.Structure):
                                          "qgroup", "topk_group")]
 
     def __init__(self, d: int, group: int, bits: int, topk: int = 0, scale_mode: int = 0, qgroup: int = 0,
-                 topk_group: int = 0):
-        super().__init__(d, group, bits, topk, 0, scale_mode, 0, qgroup, topk_group)
+                 topk_group: int = 0, coef_fmt: int = 0):
+        super().__init__(d, group, bits, topk, coef_fmt, scale_mode, 0, qgroup, topk_group)
 
     def __repr__(self):
         return (f"CodecCfg(d={self.d}, group={self.group}, bits={self.bits}, topk={self.topk}, "
@@ -121,10 +122,14 @@ def load() -> C.CDLL:
     l.rac_split_waves.restype = C.c_int
     l.rac_split_waves.argtypes = [vp, i64, i64, vp, vp, vp, vp]
     l.rac_encode_reconstruct_list.restype = C.c_int
-    l.rac_encode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp,
-                                              vp, sz, vp, vp]
+    l.rac_encode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, sz,
+                                              vp, vp, sz, vp, vp]
     l.rac_decode_reconstruct_list.restype = C.c_int
-    l.rac_decode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp]
+    l.rac_decode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp]
+    l.rac_fit_segments_workspace_bytes.restype = sz
+    l.rac_fit_segments_workspace_bytes.argtypes = [cfgp, i64]
+    l.rac_fit_segments.restype = C.c_int
+    l.rac_fit_segments.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp, vp]
     l.rac_recon_error_workspace_bytes.restype = sz
     l.rac_recon_error_workspace_bytes.argtypes = []
     l.rac_recon_error.restype = C.c_int
@@ -204,11 +209,12 @@ def rac_split_waves(ref_row, T, first_intra_row, wave1, wave2, wave_count, strea
 
 def rac_encode_reconstruct_list(cfg, X, T, tok_list, tok_count, ref_base, ref_rows, ref_row, intra_base, intra_rows,
                                 ref_gain, ref_bias, step, inv_step, payload, payload_cap, X_hat, workspace,
-                                workspace_bytes, dev_status, stream=None) -> None:
+                                workspace_bytes, dev_status, stream=None, coef_seg=None, seg_of=None) -> None:
     rc = load().rac_encode_reconstruct_list(
         C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(tok_list, _I32, "tok_list"), _ptr(tok_count, _I32, "tok_count"),
         _ptr(ref_base, _BF16, "ref_base"), int(ref_rows), _ptr(ref_row, _I32, "ref_row"),
-        _ptr(intra_base, _BF16, "intra_base"), int(intra_rows), _ptr(ref_gain, _F16, "ref_gain"),
+        _ptr(intra_base, _BF16, "intra_base"), int(intra_rows), _ptr(coef_seg, _I32, "coef_seg"),
+        _ptr(seg_of, _I32, "seg_of"), _ptr(ref_gain, _F16, "ref_gain"),
         _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"), _ptr(inv_step, _F32, "inv_step"),
         _ptr(payload, _U8, "payload"), int(payload_cap), _ptr(X_hat, _BF16, "X_hat"), _ptr(workspace, None, "workspace"),
         int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
@@ -216,14 +222,32 @@ def rac_encode_reconstruct_list(cfg, X, T, tok_list, tok_count, ref_base, ref_ro
 
 
 def rac_decode_reconstruct_list(cfg, payload, T, tok_list, tok_count, ref_base, ref_rows, ref_row, intra_base,
-                                intra_rows, ref_gain, ref_bias, step, X_hat, dev_status, stream=None) -> None:
+                                intra_rows, ref_gain, ref_bias, step, X_hat, dev_status, stream=None, coef_seg=None,
+                                seg_of=None) -> None:
     rc = load().rac_decode_reconstruct_list(
         C.byref(cfg), _ptr(payload, _U8, "payload"), int(T), _ptr(tok_list, _I32, "tok_list"),
         _ptr(tok_count, _I32, "tok_count"), _ptr(ref_base, _BF16, "ref_base"), int(ref_rows),
         _ptr(ref_row, _I32, "ref_row"), _ptr(intra_base, _BF16, "intra_base"), int(intra_rows),
+        _ptr(coef_seg, _I32, "coef_seg"), _ptr(seg_of, _I32, "seg_of"),
         _ptr(ref_gain, _F16, "ref_gain"), _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"),
         _ptr(X_hat, _BF16, "X_hat"), _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
     _check("rac_decode_reconstruct_list", rc)
+
+
+def rac_fit_segments_workspace_bytes(cfg: CodecCfg, T: int) -> int:
+    return int(load().rac_fit_segments_workspace_bytes(C.byref(cfg), int(T)))
+
+
+def rac_fit_segments(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, seg_off, n_seg, coef_seg, seg_of,
+                     workspace, workspace_bytes, dev_status, stream=None) -> None:
+    """Eq. 6 over several fitting positions; ``coef_seg`` is an int32 tensor [n_seg, J] holding the u32 words."""
+    rc = load().rac_fit_segments(C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(ref_base, _BF16, "ref_base"),
+                                 int(ref_rows), _ptr(ref_row, _I32, "ref_row"), _ptr(ref_gain, _F16, "ref_gain"),
+                                 _ptr(ref_bias, _F16, "ref_bias"), _ptr(seg_off, _I32, "seg_off"), int(n_seg),
+                                 _ptr(coef_seg, _I32, "coef_seg"), _ptr(seg_of, _I32, "seg_of"),
+                                 _ptr(workspace, None, "workspace"), int(workspace_bytes),
+                                 _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
+    _check("rac_fit_segments", rc)
 
 
 def rac_recon_error_workspace_bytes() -> int:

@@ -29,7 +29,8 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     if (!cfg) return RAC_EINVAL;
     if (cfg->d <= 0 || cfg->group <= 0 || cfg->topk < 0 || cfg->bits <= 0) return RAC_EINVAL;
     if (cfg->qgroup < 0 || cfg->topk_group < 0) return RAC_EINVAL;
-    if (cfg->coef_fmt != 0 || cfg->flags != 0) return RAC_EUNSUPPORTED;
+    if ((cfg->coef_fmt != 0 && cfg->coef_fmt != 1) || cfg->flags != 0) return RAC_EUNSUPPORTED;
+    if (cfg->coef_fmt == 1 && cfg->scale_mode != 1) return RAC_EUNSUPPORTED;   // shared coefficients: Eq. 8 family only
     if (cfg->scale_mode != 0 && cfg->scale_mode != 1) return RAC_EUNSUPPORTED;
     if (cfg->d % cfg->group) return RAC_EINVAL;
     if (cfg->d % 32 || cfg->d > 8192) return RAC_EUNSUPPORTED;
@@ -68,7 +69,9 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     g->Jq = cfg->d / qgroup;
     g->lpq = lpq;
     g->topk_group = cfg->topk_group;
-    g->codes_off = 4 * g->J + (cfg->scale_mode == 1 ? (2 * g->Jq + 3) / 4 * 4 : 0);
+    g->coef_fmt = cfg->coef_fmt;
+    g->scale_off = cfg->coef_fmt == 1 ? 0 : 4 * g->J;
+    g->codes_off = g->scale_off + (cfg->scale_mode == 1 ? (2 * g->Jq + 3) / 4 * 4 : 0);
     const int ng = g->Jq * g->topk_group;
     g->goff_off = g->codes_off + g->code_bytes + 4 * cfg->topk;
     g->gval_off = g->goff_off + (ng + 1) / 2 * 2;
@@ -83,8 +86,11 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
 // Same front end as the encoder (slab loads, Eq. 6 statistics, wire coefficients); instead of codes, every
 // thread accumulates e^2 of its own 32 channels in shared memory, separately for tokens with a reference
 // (row 0) and tokens coded directly (row 1).  One CTA barrier per token; the grid is fixed.
+// MOMENTS: the first pass of the segment fit instead -- the centred statistics of Eq. 6 of every (token, group)
+// go to p.moments and nothing is accumulated.
+template <bool MOMENTS>
 __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
-    constexpr bool SUB = false;  // calibration always runs over all tokens
+    constexpr bool SUB = false;  // always over all tokens
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31;
@@ -115,6 +121,7 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
     if (tid == 0) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
             long long t = token_at<SUB>(p, first + (long long)k * stride);
+            ctrl->tok[k] = t;
             issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, row_bytes, k, resolve_row<SUB>(p, raw_row_of(k)),
                               p.X + t * d, row_bytes);
         }
@@ -133,6 +140,7 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
         if (tid == 0 && it + S - 1 < n_my) {
             const int k = it + S - 1;
             const long long tk = token_at<SUB>(p, first + (long long)k * stride);
+            ctrl->tok[issue_stage] = tk;
             issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, row_bytes, issue_stage,
                               resolve_row<SUB>(p, next_raw), p.X + tk * d, row_bytes);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
@@ -140,6 +148,7 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
         const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
         if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
         const bool has_ref = ctrl->row[stage] >= 0;
+        const long long tok = ctrl->tok[stage];
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
 
@@ -166,10 +175,15 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
                 for (int i = 0; i < 16; i++) r2[i] = 0ull;
             }
             u64 a2, b2;
-            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2);
+            float4 st;
+            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, nullptr, &st);
+            if (MOMENTS) {
+                if (!timed_out && (lane & (p.lpg - 1)) == 0) p.moments[tok * p.J + (tid >> p.lpg_shift)] = st;
+            }
             float4 *acc = reinterpret_cast<float4 *>(smem + L.acc0) + (has_ref ? 0 : 8 * nt);
 #pragma unroll
             for (int j = 0; j < 4; j++) {
+                if (MOMENTS) break;
                 const int q = (j + rot) & 3;
 #pragma unroll
                 for (int hh = 0; hh < 2; hh++) {
@@ -192,6 +206,15 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
     }
 
     __syncthreads();
+    if (MOMENTS) {
+        if (tid == 0 && aborted) {
+            for (int s = 0; s < S; s++) {
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
+            }
+        }
+        return;
+    }
     // partial sums of this CTA, channel order, then its token counts
     float *out = p.calib_partial + (long long)blockIdx.x * 2 * d;
     const float *acc = reinterpret_cast<const float *>(smem + L.acc0);
@@ -976,6 +999,7 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     p->lpq_shift = 0;
     while ((1 << p->lpq_shift) < g.lpq) p->lpq_shift++;
     p->kg = g.topk_group;
+    p->scale_off = g.scale_off;
     p->codes_off = g.codes_off;
     p->goff_off = g.goff_off;
     p->gval_off = g.gval_off;
@@ -993,7 +1017,7 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     // leaves too little L1 for them, so that variant runs three CTAs per SM at 128 registers.
     const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
     int rc = RAC_EUNSUPPORTED;
-    const bool sub = p.tok_list || p.intra_base;   // the subset form has one variant per width: it is not the hot path
+    const bool sub = p.tok_list || p.intra_base || p.coef_ext;   // the subset form has one variant per width: it is not the hot path
 #define RAC_ENC2(B, K, X)                                                                                          \
     (sub ? launch_persistent(encode_ws_kernel<B, K, X, 2, true>, p, g.nthreads, L.total, max_ctas, stream)        \
      : tight ? launch_persistent(encode_ws_kernel<B, K, X, 4, false>, p, g.nthreads, L.total, max_ctas, stream)   \
@@ -1034,7 +1058,7 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
     p.stages = pick_stages(g.d, 2);
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
-    const bool sub = p.tok_list || p.intra_base;
+    const bool sub = p.tok_list || p.intra_base || p.coef_ext;
 #define RAC_DEC(B, K)                                                                            \
     (sub ? launch_persistent(decode_kernel<B, K, true>, p, g.nthreads, L.total, p.T, stream)    \
          : launch_persistent(decode_kernel<B, K, false>, p, g.nthreads, L.total, p.T, stream))
@@ -1110,6 +1134,78 @@ __global__ void __launch_bounds__(1024) split_waves_kernel(const int32_t *ref_ro
 }
 
 // ------------------------------------------------------------------------------------------------
+// Eq. 6 over several fitting positions: one coefficient pair per (segment of tokens, group)
+// ------------------------------------------------------------------------------------------------
+// Pass 1 (calib_kernel<true>) leaves the centred statistics of every (token, group).  Pass 2: one warp per
+// (segment, group) merges them with the pairwise update of means and centred sums, in binary64 and in a fixed
+// order (lane l takes tokens l, l+32, ... of the segment in order, then a shuffle tree), applies the
+// zero-variance rule and rounds to the wire format.
+struct Mom {
+    double n, mr, mh, sxx, sxy;
+};
+__device__ __forceinline__ Mom mom_merge(const Mom &a, const Mom &b) {
+    if (b.n == 0.0) return a;
+    if (a.n == 0.0) return b;
+    Mom o;
+    o.n = a.n + b.n;
+    const double dr = b.mr - a.mr, dh = b.mh - a.mh, w = b.n / o.n, f = a.n * w;
+    o.mr = a.mr + dr * w;
+    o.mh = a.mh + dh * w;
+    o.sxx = a.sxx + b.sxx + dr * dr * f;
+    o.sxy = a.sxy + b.sxy + dr * dh * f;
+    return o;
+}
+__global__ void __launch_bounds__(256) segment_fit_kernel(const float4 *moments, const int32_t *seg_off, long long n_seg,
+                                                          int J, int group, long long T, uint32_t *coef_seg) {
+    const long long wid = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (wid >= n_seg * J) return;
+    const long long k = wid / J;
+    const int j = (int)(wid - k * J);
+    long long t0 = seg_off[k], t1 = seg_off[k + 1];
+    t0 = t0 < 0 ? 0 : (t0 > T ? T : t0);
+    t1 = t1 < t0 ? t0 : (t1 > T ? T : t1);
+    Mom m = {0.0, 0.0, 0.0, 0.0, 0.0};
+    for (long long t = t0 + lane; t < t1; t += 32) {
+        const float4 s = moments[t * J + j];
+        const Mom one = {(double)group, (double)s.x, (double)s.y, (double)s.z, (double)s.w};
+        m = mom_merge(m, one);
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {   // lane l absorbs lane l + o: earlier tokens stay on the left
+        Mom b;
+        b.n = __shfl_down_sync(0xffffffffu, m.n, o);
+        b.mr = __shfl_down_sync(0xffffffffu, m.mr, o);
+        b.mh = __shfl_down_sync(0xffffffffu, m.mh, o);
+        b.sxx = __shfl_down_sync(0xffffffffu, m.sxx, o);
+        b.sxy = __shfl_down_sync(0xffffffffu, m.sxy, o);
+        if (lane + o < 32) m = mom_merge(m, b);
+    }
+    if (lane == 0) {
+        double a = 0.0, b = m.mh;
+        if (m.sxx > 1e-12 && fabs(m.sxy) < 65504.0 * m.sxx) {
+            a = m.sxy / m.sxx;
+            b = m.mh - a * m.mr;
+        }
+        a = fmin(fmax(a, -65504.0), 65504.0);
+        b = fmin(fmax(b, -65504.0), 65504.0);
+        const uint32_t a16 = __half_as_ushort(__double2half(a)), b16 = __half_as_ushort(__double2half(b));
+        coef_seg[k * J + j] = a16 | (b16 << 16);
+    }
+}
+// segment of every token: the last k with seg_off[k] <= t (empty segments have equal offsets and are skipped)
+__global__ void seg_of_kernel(const int32_t *seg_off, long long n_seg, long long T, int32_t *seg_of) {
+    const long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    long long lo = 0, hi = n_seg;   // invariant: seg_off[lo] <= t (seg_off[0] = 0), answer in [lo, hi)
+    while (hi - lo > 1) {
+        const long long mid = (lo + hi) >> 1;
+        if (seg_off[mid] <= t) lo = mid; else hi = mid;
+    }
+    seg_of[t] = (int32_t)lo;
+}
+
+// ------------------------------------------------------------------------------------------------
 // reconstruction error of a sender-path run (input of the byte-cost side of calibration, Sec. IV-C)
 // ------------------------------------------------------------------------------------------------
 constexpr int kErrGrid = 592;     // fixed, so that the summation order does not depend on the device
@@ -1169,6 +1265,8 @@ struct Subset {
     const int32_t *tok_count = nullptr;
     const void *intra_base = nullptr;
     long long intra_rows = 0;
+    const uint32_t *coef_seg = nullptr;
+    const int32_t *seg_of = nullptr;
 };
 static int apply_subset(const Subset &sub, CodecParams *p) {
     if ((sub.tok_list == nullptr) != (sub.tok_count == nullptr)) return RAC_EINVAL;
@@ -1179,6 +1277,8 @@ static int apply_subset(const Subset &sub, CodecParams *p) {
     p->tok_count = sub.tok_count;
     p->intra_base = sub.intra_rows > 0 ? static_cast<const uint16_t *>(sub.intra_base) : nullptr;
     p->intra_rows = sub.intra_rows;
+    p->coef_ext = sub.coef_seg;
+    p->seg_of = sub.seg_of;
     return RAC_OK;
 }
 
@@ -1194,6 +1294,7 @@ static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64
     if (rc != RAC_OK) return rc;
     rc = apply_subset(sub, &p);
     if (rc != RAC_OK) return rc;
+    if ((g.coef_fmt == 1) != (sub.coef_seg != nullptr) || (sub.coef_seg != nullptr) != (sub.seg_of != nullptr)) return RAC_EINVAL;
     if (T == 0) return RAC_OK;
     if (!payload || !X_hat || (!step && g.scale_mode == 0)) return RAC_EINVAL;   // mode 1 reads no table
     if (!aligned16(payload) || !aligned16(X_hat) || (step && !aligned16(step))) return RAC_EALIGN;
@@ -1255,6 +1356,7 @@ static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const
     if (rc != RAC_OK) return rc;
     rc = apply_subset(sub, &p);
     if (rc != RAC_OK) return rc;
+    if ((g.coef_fmt == 1) != (sub.coef_seg != nullptr) || (sub.coef_seg != nullptr) != (sub.seg_of != nullptr)) return RAC_EINVAL;
     if (T == 0) return RAC_OK;
     if (!X || !payload) return RAC_EINVAL;
     if (g.scale_mode == 0 && (!step || !inv_step)) return RAC_EINVAL;   // the static tables; mode 1 reads neither
@@ -1307,7 +1409,8 @@ int rac_sender_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_
 
 int rac_encode_reconstruct_list(const rac_codec_cfg *cfg, const void *X, int64_t T, const int32_t *tok_list,
                                 const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
-                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const void *intra_base, int64_t intra_rows, const uint32_t *coef_seg, const int32_t *seg_of,
+                                const void *ref_gain, const void *ref_bias,
                                 const float *step, const float *inv_step, void *payload, size_t payload_cap, void *X_hat,
                                 void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream) {
     Subset sub;
@@ -1315,19 +1418,24 @@ int rac_encode_reconstruct_list(const rac_codec_cfg *cfg, const void *X, int64_t
     sub.tok_count = tok_count;
     sub.intra_base = intra_base;
     sub.intra_rows = intra_rows;
+    sub.coef_seg = coef_seg;
+    sub.seg_of = seg_of;
     return encode_impl(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload, payload_cap,
                        X_hat, workspace, workspace_bytes, dev_status, stream, sub);
 }
 
 int rac_decode_reconstruct_list(const rac_codec_cfg *cfg, const void *payload, int64_t T, const int32_t *tok_list,
                                 const int32_t *tok_count, const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
-                                const void *intra_base, int64_t intra_rows, const void *ref_gain, const void *ref_bias,
+                                const void *intra_base, int64_t intra_rows, const uint32_t *coef_seg, const int32_t *seg_of,
+                                const void *ref_gain, const void *ref_bias,
                                 const float *step, void *X_hat, uint32_t *dev_status, void *stream) {
     Subset sub;
     sub.tok_list = tok_list;
     sub.tok_count = tok_count;
     sub.intra_base = intra_base;
     sub.intra_rows = intra_rows;
+    sub.coef_seg = coef_seg;
+    sub.seg_of = seg_of;
     return reconstruct_impl(cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, X_hat, dev_status, stream,
                             sub);
 }
@@ -1339,6 +1447,43 @@ int rac_split_waves(const int32_t *ref_row, int64_t T, int64_t first_intra_row, 
     if (T > 0 && (!ref_row || !wave1 || !wave2)) return RAC_EINVAL;
     split_waves_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(ref_row, (int)T, first_intra_row, wave1, wave2,
                                                                          wave_count);
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+size_t rac_fit_segments_workspace_bytes(const rac_codec_cfg *cfg, int64_t T) {
+    Geometry g;
+    if (make_geometry(cfg, &g) != RAC_OK || T < 0) return 0;
+    return ((size_t)T * (size_t)g.J * sizeof(float4) + 15) / 16 * 16 + 16;
+}
+
+int rac_fit_segments(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+                     const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const int32_t *seg_off,
+                     int64_t n_seg, uint32_t *coef_seg, int32_t *seg_of, void *workspace, size_t workspace_bytes,
+                     uint32_t *dev_status, void *stream) {
+    Geometry g;
+    int rc = make_geometry(cfg, &g);
+    if (rc != RAC_OK) return rc;
+    CodecParams p = {};
+    rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, dev_status);
+    if (rc != RAC_OK) return rc;
+    if (n_seg < 0 || n_seg >= (1ll << 30) || T >= (1ll << 31)) return RAC_EUNSUPPORTED;
+    if (n_seg == 0) return T == 0 ? RAC_OK : RAC_EINVAL;
+    if (!seg_off || !coef_seg || !workspace || (T > 0 && (!X || !seg_of))) return RAC_EINVAL;
+    if (!aligned16(X) || !aligned16(workspace)) return RAC_EALIGN;
+    if (workspace_bytes < rac_fit_segments_workspace_bytes(cfg, T)) return RAC_ESIZE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p.X = static_cast<const uint16_t *>(X);
+    p.moments = static_cast<float4 *>(workspace);
+    if (T > 0) {
+        p.stages = pick_stages(g.d, 2);
+        EncSmem L = enc_smem_layout(g.d, p.stages, g.nthreads);
+        rc = launch_persistent(calib_kernel<true>, p, g.nthreads, L.total, T, st);
+        if (rc != RAC_OK) return rc;
+        seg_of_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(seg_off, n_seg, T, seg_of);
+    }
+    const long long warps = n_seg * g.J;
+    segment_fit_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(p.moments, seg_off, n_seg, g.J, g.group, T,
+                                                                            coef_seg);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
@@ -1391,8 +1536,8 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, cons
         rc = device_info(&di);
         if (rc != RAC_OK) return rc;
         if (L.total > di.max_smem_optin) return RAC_EUNSUPPORTED;
-        if (cudaFuncSetAttribute(calib_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return RAC_ECUDA;
-        calib_kernel<<<kCalibGrid, g.nthreads, L.total, st>>>(p);
+        if (cudaFuncSetAttribute(calib_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return RAC_ECUDA;
+        calib_kernel<false><<<kCalibGrid, g.nthreads, L.total, st>>>(p);
         if (cudaGetLastError() != cudaSuccess) return RAC_ECUDA;
     }
     int n = 2 * g.d;

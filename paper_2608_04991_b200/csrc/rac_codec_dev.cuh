@@ -36,8 +36,12 @@ struct CodecParams {
     const int32_t *tok_count;    // device int32[1]
     const uint16_t *intra_base;  // bf16[intra_rows, d]: reference rows ref_rows .. ref_rows + intra_rows - 1, or null
     long long intra_rows;
+    // coefficient words shared by the tokens of a segment (Eq. 6 over several fitting positions), outside the record
+    const uint32_t *coef_ext;    // u32[n_seg, J] or null (coefficients in the record)
+    const int32_t *seg_of;       // int32[T] segment of each token
+    float4 *moments;             // segment fit, first pass out: (mean r, mean h, Sxx, Sxy) per (token, group)
     // scale_mode 1 only: quantisation groups, per-group outliers, field offsets in the record
-    int Jq, lpq, lpq_shift, kg, codes_off, goff_off, gval_off;
+    int Jq, lpq, lpq_shift, kg, scale_off, codes_off, goff_off, gval_off;
 };
 
 // scale_mode 1 (defined in rac_codec_dyn.cu)
@@ -52,6 +56,8 @@ constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an int
 struct Ctrl {
     unsigned long long bar[kMaxStages];
     int row[kMaxStages];        // reference row of the token in each stage, -1 = direct
+    int seg[kMaxStages];        // segment of the token in each stage (shared coefficients only)
+    long long tok[kMaxStages];  // the token in each stage (segment fit only)
 };
 
 __host__ __device__ inline int align_up(int v, int a) { return (v + a - 1) / a * a; }
@@ -227,8 +233,10 @@ __device__ __forceinline__ const uint16_t *ref_row_ptr(const CodecParams &p, lon
 // thread 0: start the copies of one token into a stage: `first` (X row or record) and, if any, its reference row
 template <bool SUB>
 __device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ctrl, uint32_t stage_addr, uint32_t r_off,
-                                                  int stage, int row, const void *first_src, uint32_t first_bytes) {
+                                                  int stage, int row, const void *first_src, uint32_t first_bytes,
+                                                  long long tok = 0) {
     ctrl->row[stage] = row;
+    if constexpr (SUB) ctrl->seg[stage] = p.seg_of ? p.seg_of[tok] : 0;
     const uint32_t bar = smem_u32(&ctrl->bar[stage]);
     const uint32_t row_bytes = 2u * (uint32_t)p.d;
     mbar_arrive_expect_tx(bar, first_bytes + (row >= 0 ? row_bytes : 0u));
@@ -242,7 +250,7 @@ __device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ct
 // are their bit patterns.
 __device__ __forceinline__ void fit_group(const u64 (&x2)[16], const u64 (&r2)[16], bool has_ref, int lpg, float inv_group,
                                           unsigned int group_mask, uint32_t *status, u64 &a2, u64 &b2,
-                                          uint32_t *coef_word = nullptr) {
+                                          uint32_t *coef_word = nullptr, float4 *stats = nullptr) {
     u64 sra = 0ull, srb = 0ull, sha = 0ull, shb = 0ull;
 #pragma unroll
     for (int i = 0; i < 16; i += 2) {
@@ -286,6 +294,7 @@ __device__ __forceinline__ void fit_group(const u64 (&x2)[16], const u64 (&r2)[1
             sxy += __shfl_xor_sync(group_mask, sxy, o);
         }
     }
+    if (stats) *stats = make_float4(rbar, hbar, sxx, sxy);
     // zero-variance rule, then wire rounding to binary16
     float a_star = 0.f, b_star = hbar;
     if (has_ref && sxx > 1e-12f && fabsf(sxy) < 65504.0f * sxx) {

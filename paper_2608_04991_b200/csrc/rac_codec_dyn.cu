@@ -23,6 +23,7 @@ struct DynCtrl {
     unsigned long long done[kMaxStages];    // every warp has finished its share of the token in the stage
     unsigned long long tokmax[kMaxStages];  // every warp has published its largest |e| of the token
     int row[kMaxStages];
+    int seg[kMaxStages];                    // segment of the token in each stage (shared coefficients only)
     int abort;
     float wmax[kMaxStages][8];
 };
@@ -103,6 +104,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
         const long long t = token_at<SUB>(p, first + (long long)k * stride);
         const int row = resolve_row<SUB>(p, raw_row);
         ctrl->row[s] = row;
+        if constexpr (SUB) ctrl->seg[s] = p.seg_of ? p.seg_of[t] : 0;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
         const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
         mbar_arrive_expect_tx(bar, row_bytes + (row >= 0 ? row_bytes : 0u));
@@ -176,9 +178,19 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
 #pragma unroll
                 for (int i = 0; i < 16; i++) r2[i] = 0ull;
             }
-            uint32_t coef_word;
-            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
-            if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
+            bool shared = false;
+            if constexpr (SUB) shared = p.coef_ext != nullptr;
+            if (shared) {
+                // Eq. 6 was solved over all positions of the token's segment beforehand: the words come from outside
+                const uint32_t cw = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> p.lpg_shift)];
+                const float a = half_bits_to_float(cw & 0xffffu), b = half_bits_to_float(cw >> 16);
+                a2 = pack2(a, a);
+                b2 = pack2(b, b);
+            } else {
+                uint32_t coef_word;
+                fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
+                if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
+            }
             // residual, and the largest magnitude of each slot of 8 channels
             float sm[4];
 #pragma unroll
@@ -289,7 +301,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             const float isc = sc != 0.f ? __fdiv_rn(1.0f, sc) : 0.f;   // zero marker: no division, codes 0
             const u64 inv2 = pack2(isc, isc), s2 = pack2(sc, sc);
             if (qtok ? tid == 0 : (lane & (p.lpq - 1)) == 0)
-                reinterpret_cast<unsigned short *>(rec + 4 * p.J)[jq] = (unsigned short)s16;
+                reinterpret_cast<unsigned short *>(rec + p.scale_off)[jq] = (unsigned short)s16;
 
             uint32_t words[4][2];
 #pragma unroll
@@ -461,7 +473,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
             long long t = token_at<SUB>(p, first + (long long)k * stride);
             issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row<SUB>(p, raw_row_of(k)),
-                              p.payload + t * p.rec, (uint32_t)p.rec);
+                              p.payload + t * p.rec, (uint32_t)p.rec, t);
         }
         if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
     }
@@ -480,7 +492,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
             const int k = it + S - 1;
             const long long tk = token_at<SUB>(p, first + (long long)k * stride);
             issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
-                              resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
+                              resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec, tk);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
         const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
@@ -492,10 +504,14 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
         const uint32_t obs = smem_u32(ob);
 
         if (valid) {
-            const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
+            uint32_t cf;
+            bool shared = false;
+            if constexpr (SUB) shared = p.coef_ext != nullptr;
+            if (shared) cf = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> p.lpg_shift)];
+            else cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
             const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
             const u64 a2 = pack2(a, a), b2 = pack2(b, b);
-            const float sc = half_bits_to_float(reinterpret_cast<const unsigned short *>(rec + 4 * p.J)[jq]);
+            const float sc = half_bits_to_float(reinterpret_cast<const unsigned short *>(rec + p.scale_off)[jq]);
             const u64 s2 = pack2(sc, sc);
             // code words of the four pieces, in piece order, then rotated into slot order
             const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + p.codes_off) + tid * WPT;
@@ -612,7 +628,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
 // outliers only below 8-bit codes.
 template <int B, bool X, int K>
 static int launch_encode_variant(bool tight, const Geometry &g, CodecParams &p, int smem, long long max_ctas, cudaStream_t stream) {
-    if (p.tok_list || p.intra_base)   // the subset form: one variant, not the hot path
+    if (p.tok_list || p.intra_base || p.coef_ext)   // the subset form: one variant, not the hot path
         return launch_persistent(encode_dyn_kernel<B, X, K, 2, true>, p, g.nthreads, smem, max_ctas, stream);
     if constexpr (!X && (K == 0 || B != 8)) {
         if (tight) return launch_persistent(encode_dyn_kernel<B, X, K, 4, false>, p, g.nthreads, smem, max_ctas, stream);
@@ -652,7 +668,7 @@ int launch_decode_dyn(const Geometry &g, CodecParams &p, cudaStream_t stream) {
     p.stages = pick_stages(g.d, 2);
     const DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const bool kg = g.topk_group > 0;
-    const bool sub = p.tok_list || p.intra_base;
+    const bool sub = p.tok_list || p.intra_base || p.coef_ext;
 #define RAC_DYN_DEC(B) \
     (sub ? (kg ? launch_persistent(decode_dyn_kernel<B, true, true>, p, g.nthreads, L.total, p.T, stream) \
                : launch_persistent(decode_dyn_kernel<B, false, true>, p, g.nthreads, L.total, p.T, stream)) \

@@ -147,7 +147,9 @@ struct Geometry {
     int Jq;         // quantisation groups per token
     int lpq;        // lanes per quantisation group, 0 when the group is the whole token and d/32 is no power of two <= 32
     int topk_group; // outliers per quantisation group (scale_mode 1)
-    int codes_off;  // byte offset of the codes in a record: 4*J, plus the scales (2*Jq padded to 4) in mode 1
+    int coef_fmt;   // 0: coefficient words in the record; 1: shared per segment, outside the record (scale_mode 1)
+    int scale_off;  // byte offset of the scales in a record: 4*J, or 0 when the record holds no coefficients
+    int codes_off;  // byte offset of the codes in a record: after the coefficient words and the scales
     int goff_off;   // byte offset of the per-group outlier offsets (Jq*topk_group bytes, padded to 2)
     int gval_off;   // byte offset of the per-group outlier values (Jq*topk_group binary16)
     int rec;        // record stride in bytes
