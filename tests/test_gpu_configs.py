@@ -262,3 +262,109 @@ def test_config4_long_context_round_trip(env):
         within += int((err <= bound).sum().item())
         total += err.numel()
     assert within / total > 0.98
+
+
+@pytest.mark.parametrize("member", [dict(bits=4, topk_group=1), dict(bits=8), dict(bits=4, qgroup=5120),
+                                    dict(bits=4, coef_fmt=1)])
+def test_config4_shape_with_the_eq8_family(env, member):
+    """The benchmark's shape (131072 x 5120, groups of 128) through the per-group-scale kernels, in the launch
+    configuration `bench.py` times for its `paper_family` / `shared_coefficients` extras: ~1000 sampled tokens
+    checked one by one against the oracle, sender x_hat == receiver x_hat on the whole tensor, and Eq. 11's
+    half-step bound (nothing clips) on every element."""
+    s, rac, orc, dev = env.synth, env.rac, env.orc, env.dev
+    d, g, T = 5120, 128, 131072
+    J = d // g
+    bits = member["bits"]
+    mk = dict(scale_mode=1, qgroup=member.get("qgroup", 0), topk_group=member.get("topk_group", 0))
+    shared = member.get("coef_fmt", 0) == 1
+    cfg = rac.CodecCfg(d, g, bits, 0, coef_fmt=int(shared), **mk)
+    gen = s.generator(s.BASE_SEED + 9, dev)
+    X = s.activations(T, d, s.channel_scale(d, 9, dev), gen)
+    R = s.affine_noisy_reference(X, g, gen)
+    rec = rac.rac_record_bytes(cfg)
+    pay = torch.empty(T * rec, dtype=torch.uint8, device=dev)
+    xs, xr = torch.empty_like(X), torch.empty_like(X)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    seg_tokens = 64
+    coef = seg_of = None
+    if shared:
+        n_seg = T // seg_tokens
+        seg_off = (torch.arange(n_seg + 1, dtype=torch.int32, device=dev) * seg_tokens).to(torch.int32)
+        coef = torch.empty((n_seg, J), dtype=torch.int32, device=dev)
+        seg_of = torch.empty(T, dtype=torch.int32, device=dev)
+        nb = rac.rac_fit_segments_workspace_bytes(cfg, T)
+        ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+        rac.rac_fit_segments(cfg, X, T, R, T, None, None, None, seg_off, n_seg, coef, seg_of, ws, nb, status)
+        rac.rac_encode_reconstruct_list(cfg, X, T, None, None, R, T, None, None, 0, None, None, None, None, pay,
+                                        pay.numel(), xs, None, 0, status, coef_seg=coef, seg_of=seg_of)
+        rac.rac_decode_reconstruct_list(cfg, pay, T, None, None, R, T, None, None, 0, None, None, None, xr, status,
+                                        coef_seg=coef, seg_of=seg_of)
+    else:
+        rac.rac_encode_reconstruct(cfg, X, T, R, T, None, None, None, None, None, pay, pay.numel(), xs, None, 0, status)
+        rac.rac_decode_reconstruct(cfg, pay, T, R, T, None, None, None, None, xr, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(xs, xr)
+    rng = np.random.default_rng(9)
+    if shared:   # whole segments, so that the oracle can redo the pooled fit of the sampled ones
+        segs = np.unique(np.concatenate([[0, n_seg - 1], rng.integers(0, n_seg, 14)]))
+        sample = (segs[:, None] * seg_tokens + np.arange(seg_tokens)[None, :]).reshape(-1)
+    else:
+        sample = np.unique(np.concatenate([np.arange(48), np.arange(T - 48, T), rng.integers(0, T, 900)]))
+    idx = torch.from_numpy(sample).to(dev)
+    p_s = pay.view(T, rec)[idx].cpu().numpy().reshape(-1)
+    Xb, Rb = s.bf16_bits(X[idx]), s.bf16_bits(R[idx])
+    if shared:
+        so = np.arange(len(segs) + 1, dtype=np.int32) * seg_tokens
+        o_coef = orc.fit_segments(d, g, Xb, so, ref_base=Rb)
+        g_coef = coef[torch.from_numpy(segs).to(dev)].cpu().numpy().view(np.uint32)
+        assert (g_coef != o_coef).sum() <= 3
+        per_tok = np.ascontiguousarray(np.repeat(g_coef, seg_tokens, axis=0))
+        o_pay = orc.encode(d, g, bits, 0, Xb, ref_base=Rb, forced_coef=per_tok.reshape(-1).copy(), coef_fmt=1,
+                           nthreads=orc.max_threads(), **mk)
+        assert np.array_equal(o_pay, p_s)
+        o_x = orc.reconstruct(d, g, bits, 0, p_s, sample.size, ref_base=Rb, coef_fmt=1, shared_coef=per_tok,
+                              nthreads=orc.max_threads(), **mk)
+    else:
+        rep = env.P.compare_encode(cfg, p_s, Xb, Rb, None, None, None, None, None)
+        print(member, rep)
+        o_x = orc.reconstruct(d, g, bits, 0, p_s, sample.size, ref_base=Rb, nthreads=orc.max_threads(), **mk)
+    assert np.array_equal(o_x, s.bf16_bits(xr[idx]))
+    # Eq. 11 on every element: half a scale step (the record's own scale) plus the bf16 rounding; outliers: binary16
+    scale_off = 0 if shared else 4 * J
+    qg = mk["qgroup"] or g
+    Jq = d // qg
+    for t0 in range(0, T, 16384):
+        sl = slice(t0, t0 + 16384)
+        sc = pay.view(T, rec)[sl, scale_off:scale_off + 2 * Jq].contiguous().view(torch.float16).float()
+        half_step = 0.5 * sc.repeat_interleave(qg, dim=1) * 1.00001
+        err = (X[sl].float() - xr[sl].float()).abs()
+        mag = torch.maximum(X[sl].float().abs(), xr[sl].float().abs())
+        assert bool((err <= half_step + 2.0 ** -8 * mag + 2.0 ** -10 * mag + 1e-12).all())
+
+
+def test_config4_tokens_through_the_persistent_index(env):
+    """The benchmark's token workload (131072-token history, 131072-token prompt) through the persistent index,
+    appended as 64 requests: spans, rows and intra-sequence references against the oracle, whole."""
+    s, rac, orc, dev = env.synth, env.rac, env.orc, env.dev
+    H = T = 131072
+    wl = s.span_workload(H, T, seed=s.BASE_SEED + 11, gap_max=112)
+    htok, qtok = torch.from_numpy(wl.hist).to(dev), torch.from_numpy(wl.query).to(dev)
+    cfg = rac.IndexCfg(H, 4, 8)
+    nb = rac.rac_index_bytes(cfg)
+    mem = torch.empty(nb, dtype=torch.uint8, device=dev)
+    rac.rac_index_reset(cfg, mem, nb)
+    bounds = np.arange(0, H + 1, 2048, dtype=np.int32)
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        rac.rac_index_append(cfg, mem, nb, htok, int(a), int(b))
+    nws = rac.rac_index_query_workspace_bytes(T)
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+    rows = torch.empty(T, dtype=torch.int32, device=dev)
+    spans = torch.empty((T // 4 + 1, 3), dtype=torch.int32, device=dev)
+    n_spans = torch.zeros(1, dtype=torch.int32, device=dev)
+    rac.rac_index_query(cfg, mem, nb, htok, H, qtok, T, True, rows, spans, n_spans, ws, nws)
+    torch.cuda.synchronize()
+    o_rr, o_sp = orc.match_spans_req(wl.hist, bounds, wl.query, w=4, max_hits=8, intra=True)
+    ns = int(n_spans.item())
+    assert ns == len(o_sp) and np.array_equal(spans[:ns].cpu().numpy(), o_sp)
+    assert np.array_equal(rows.cpu().numpy(), o_rr)
+    print(f"index, 64 requests: {ns} spans, covered {((o_rr >= 0) & (o_rr < H)).mean():.3f}, intra {(o_rr >= H).mean():.3f}")
