@@ -967,6 +967,201 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// reconstruct, streaming form: no CTA barrier in the loop
+// ------------------------------------------------------------------------------------------------
+// Same arithmetic as decode_kernel.  The output row is written IN PLACE over the token's reference row in the
+// stage (a thread reads its 64-byte slab of r and writes x_hat there), so a stage is record + one row; every warp
+// ends its share of a token with one arrival on the stage's `done` mbarrier and moves on, and the warp whose turn
+// it is (token i: warp i mod warps) waits for `done`, sends the row off as a bulk store, and refills the stage once
+// the store has read it.  Records without per-token outliers only: patching outliers needs the reference of
+// single channels after the row has been overwritten, and keeping those aside cost more than the barrier of
+// decode_kernel (measured), so records with outliers stay with that kernel.
+struct DwSmem {
+    int stage0, stage_bytes, rec_pad, total;
+};
+__host__ __device__ inline DwSmem dw_smem_layout(int d, int rec, int stages) {
+    DwSmem s;
+    s.stage0 = align_up((int)sizeof(WsCtrl), 128);
+    s.rec_pad = align_up(rec, 128);
+    s.stage_bytes = s.rec_pad + 2 * d;
+    s.total = s.stage0 + stages * s.stage_bytes;
+    return s;
+}
+
+template <int BITS, bool SUB>
+__global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int rot = (lane >> 1) & 3;
+    const int d = p.d;
+    const bool valid = tid * 32 < d;
+    const DwSmem L = dw_smem_layout(d, p.rec, p.stages);
+    WsCtrl *ctrl = reinterpret_cast<WsCtrl *>(smem);
+    const uint32_t sbase = smem_u32(smem);
+    const int S = p.stages;
+    constexpr uint32_t cmask = (1u << BITS) - 1u;
+    constexpr uint32_t H = 1u << (BITS - 1);
+    constexpr uint32_t ones = (BITS == 4) ? 0x11111111u : (BITS == 3) ? 0x00249249u : 0x00005555u;
+    constexpr uint32_t highs = ones << (BITS - 1);
+    constexpr float kBase = 8388608.0f + (float)H;  // 2^23 + H
+    const uint32_t row_bytes = 2u * (uint32_t)d;
+
+    const int first = blockIdx.x, stride = gridDim.x;
+    const long long n_tok = tokens_to_do<SUB>(p);
+    const int n_my = (n_tok > first) ? (int)((n_tok - first + stride - 1) / stride) : 0;
+    auto raw_row_of = [&](int k) -> int {
+        long long t = token_at<SUB>(p, first + (long long)k * stride);
+        return p.ref_row ? p.ref_row[t] : (int)t;
+    };
+    auto issue = [&](int k, int s, int raw_row) {
+        const long long t = token_at<SUB>(p, first + (long long)k * stride);
+        const int row = resolve_row<SUB>(p, raw_row);
+        ctrl->row[s] = row;
+        const uint32_t bar = smem_u32(&ctrl->full[s]);
+        const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
+        mbar_arrive_expect_tx(bar, (uint32_t)p.rec + (row >= 0 ? row_bytes : 0u));
+        bulk_load(base, p.payload + t * p.rec, (uint32_t)p.rec, bar);
+        if (row >= 0) bulk_load(base + L.rec_pad, ref_row_ptr<SUB>(p, row), row_bytes, bar);
+    };
+
+    if (tid == 0) {
+        for (int s = 0; s < S; s++) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->done[s]), nwarps);
+        }
+        ctrl->abort = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    if (tid == 0)
+        for (int k = 0; k < S && k < n_my; k++) issue(k, k, raw_row_of(k));
+
+    uint32_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
+    // step table, row 0, in slot order
+    u64 st0[16];
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+        if (valid) {
+            s0 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1)));
+            s1 = __ldg(reinterpret_cast<const float4 *>(p.step + (off[j] >> 1) + 4));
+        }
+        st0[4 * j + 0] = pack2(s0.x, s0.y);
+        st0[4 * j + 1] = pack2(s0.z, s0.w);
+        st0[4 * j + 2] = pack2(s1.x, s1.y);
+        st0[4 * j + 3] = pack2(s1.z, s1.w);
+    }
+    const u64 base2 = pack2(kBase, kBase);
+
+    int stage = 0, duty = 0;
+    uint32_t parity = 0;
+    bool timed_out = false;
+    for (int it = 0; it < n_my; it++) {
+        if (*reinterpret_cast<volatile int *>(&ctrl->abort)) break;
+        unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
+        const uint32_t rs = sbase + L.stage0 + stage * L.stage_bytes + L.rec_pad;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
+        const bool has_ref = ctrl->row[stage] >= 0;
+
+        if (valid) {
+            const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
+            const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
+            const u64 a2 = pack2(a, a), b2 = pack2(b, b);
+            // code words of the four pieces, in piece order, then rotated into slot order
+            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + 4 * p.J) + tid * BITS;
+            uint32_t words[4];
+            if (BITS == 4) {
+                words[0] = cw[0]; words[1] = cw[1]; words[2] = cw[2]; words[3] = cw[3];
+            } else if (BITS == 3) {
+                uint32_t w0 = cw[0], w1 = cw[1], w2 = cw[2];
+                words[0] = w0 & 0xffffffu;
+                words[1] = (w0 >> 24) | ((w1 & 0xffffu) << 8);
+                words[2] = (w1 >> 16) | ((w2 & 0xffu) << 16);
+                words[3] = w2 >> 8;
+            } else {
+                uint32_t w0 = cw[0], w1 = cw[1];
+                words[0] = w0 & 0xffffu; words[1] = w0 >> 16; words[2] = w1 & 0xffffu; words[3] = w1 >> 16;
+            }
+            uint32_t reserved = 0;
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                uint32_t v = words[q] ^ highs;  // field == 0  <=>  code == -2^(BITS-1)
+                reserved |= (v - ones) & ~v & highs;
+                words[q] = v;                   // fields now hold code + H (offset binary)
+            }
+            if (reserved && p.status) atomicOr(p.status, RAC_STATUS_RESERVED_CODE);
+            rot_left4(words, rot);
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                const int c = (int)(off[j] >> 1);
+                u64 r2[4], st2[4];
+                if (has_ref) {
+                    load_ref_slot(rs + off[j], p.gain, p.bias, c, r2);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) r2[i] = 0ull;
+                }
+                if (has_ref) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) st2[i] = st0[4 * j + i];
+                } else {
+                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c));
+                    const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c + 4));
+                    st2[0] = pack2(s0.x, s0.y); st2[1] = pack2(s0.z, s0.w); st2[2] = pack2(s1.x, s1.y); st2[3] = pack2(s1.z, s1.w);
+                }
+                const uint32_t w = words[j];
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    const float q0 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i))) & cmask));
+                    const float q1 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i + 1))) & cmask));
+                    const u64 eh = pmul(psub(pack2(q0, q1), base2), st2[i]);
+                    float x0, x1;
+                    unpack2(padd(pfma(a2, r2[i], b2), eh), x0, x1);
+                    o[i] = f2_to_bf16x2(x0, x1);
+                }
+                sts128(rs + off[j], make_uint4(o[0], o[1], o[2], o[3]));   // x_hat over the slab just read
+            }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&ctrl->done[stage])) : "memory");
+
+        if (warp == duty) {
+            const int k_next = it + S;
+            int raw_next = 0;
+            if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
+            if (lane == 0) {
+                const long long t = token_at<SUB>(p, first + (long long)it * stride);
+                bulk_store(p.X_hat + t * d, rs, row_bytes);
+                bulk_commit();
+                bulk_wait_read<0>();      // the row has been read: the stage may be refilled
+                if (k_next < n_my) issue(k_next, stage, raw_next);
+            }
+            __syncwarp();
+        }
+        if (++stage == S) { stage = 0; parity ^= 1u; }
+        if (++duty == nwarps) duty = 0;
+    }
+    if (timed_out) {
+        ctrl->abort = 1;
+        if (p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
+    }
+    __syncthreads();
+    if (lane == 0) bulk_wait_all();
+    if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
+        for (int s = 0; s < S; s++) {
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // host side: launch plumbing
 // ------------------------------------------------------------------------------------------------
 
@@ -1059,8 +1254,17 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;
+    // Without outliers the streaming form is the faster one (0.44-0.49 ms against 0.52 ms at 131072 x 5120; 0.37
+    // against 0.43 ms at 131072 x 4096).  With outliers it is not: their patching costs the streaming form more than
+    // the barrier costs the other (0.57 against 0.49 ms), so those keep the kernel with the CTA barrier, which is
+    // already at 94 % of the copy bandwidth there.  RAC_DEC_BARRIER=1 forces the barrier form everywhere.
+    const bool ws = kt == 0 && !sub && !getenv("RAC_DEC_BARRIER");
+    const int wstages = pick_stages(g.d, g.nthreads > 128 ? 3 : 2);
+    DwSmem LW = dw_smem_layout(g.d, g.rec, wstages);
+    if (ws) p.stages = wstages;
 #define RAC_DEC(B, K)                                                                            \
     (sub ? launch_persistent(decode_kernel<B, K, true>, p, g.nthreads, L.total, p.T, stream)    \
+     : ws ? launch_persistent(decode_ws_kernel<B, false>, p, g.nthreads, LW.total, p.T, stream) \
          : launch_persistent(decode_kernel<B, K, false>, p, g.nthreads, L.total, p.T, stream))
     switch (g.bits * 100 + kt) {
         case 400: return RAC_DEC(4, 0);
