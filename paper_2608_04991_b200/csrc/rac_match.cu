@@ -30,6 +30,8 @@ struct MatchParams {
     int2 *best;            // [N]      (length, history start) of the best candidate, length 0 = none
     int2 *hop;             // [N]      (next position >= p with a candidate, position after its span)
     rac_span *spans_ws;    // [N/w + 1]
+    int32_t *chunk_first;  // [ceil(N/1024)] first position with a candidate in each chunk of 1024 positions
+    unsigned short *delta16; // [N]    hop.y - position, 65535 = does not fit
     int n_hist, n_query, nwin, w, K;
     unsigned int mask;     // M - 1
     const int32_t *end_of; // [n_hist] end of the request that holds each history position; null = one request
@@ -113,71 +115,70 @@ __global__ void match_query_kernel(MatchParams p) {
     p.best[i] = make_int2(bestL, bestj);
 }
 
-// Single CTA.  (1) hop[p] = (s, s + len(s)) with s the first position >= p that has a candidate (n_query
-// if none); (2) one thread follows the chain from 0 and lists the positions it visits; (3) all threads turn
-// them into spans and rows.  The chain is the serial part of Eq. 3 (one dependent read per selected span);
-// to make each read a shared-memory access instead of a trip to L2, the jump lengths of a window of
-// positions are staged as 16-bit deltas (65535 = "look it up in global memory") before the walk enters it.
+// Selection.  (1) hop[p] = (s, s + len(s)) with s the first position >= p that has a candidate (n_query if
+// none): a suffix scan, done grid-wide in two launches -- first the first candidate of every chunk of 1024
+// positions, then every chunk completes its positions with the first candidate of the later chunks as carry --
+// which also leaves the jump lengths hop.y - p as 16-bit deltas (65535 = "look it up in hop").  (2) One thread
+// of a single CTA follows the chain from 0 and lists the positions it visits: the serial part of Eq. 3, one
+// dependent read per selected span; the deltas of a window of positions are staged in shared memory so that each
+// read is a shared-memory access instead of a trip to L2.  (3) A grid-wide kernel turns the visited positions into
+// spans and per-token rows.
 constexpr int kWalkWindow = 96 * 1024;  // positions per window: 192 KiB of shared memory
+constexpr int kHopChunk = 1024;         // positions per CTA of the suffix scan
+
+__global__ void __launch_bounds__(kHopChunk) match_chunk_first_kernel(MatchParams p) {
+    __shared__ int s_first;
+    const int i = blockIdx.x * kHopChunk + threadIdx.x;
+    if (threadIdx.x == 0) s_first = p.n_query;
+    __syncthreads();
+    const bool st = i < p.n_query && p.best[i].x > 0;
+    const unsigned int b = __ballot_sync(0xffffffffu, st);
+    if (b && (threadIdx.x & 31) == 0) atomicMin(&s_first, i + __ffs(b) - 1);
+    __syncthreads();
+    if (threadIdx.x == 0) p.chunk_first[blockIdx.x] = s_first;
+}
+
+__global__ void __launch_bounds__(kHopChunk) match_hop_kernel(MatchParams p, int nchunks) {
+    __shared__ int warp_first[kHopChunk / 32];
+    __shared__ int s_carry;
+    const int N = p.n_query;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int i = blockIdx.x * kHopChunk + tid;
+    const int len = i < N ? p.best[i].x : 0;
+    const unsigned int b = __ballot_sync(0xffffffffu, len > 0);
+    if (lane == 0) warp_first[warp] = b ? (i + __ffs(b) - 1) : N;
+    if (tid == 0) {
+        int c = N;   // first candidate of the later chunks
+        for (int k = blockIdx.x + 1; k < nchunks; k++) {
+            const int f = p.chunk_first[k];
+            if (f < N) { c = f; break; }
+        }
+        s_carry = c;
+    }
+    __syncthreads();
+    if (i >= N) return;
+    const unsigned int at_or_after = b >> lane;
+    int s;
+    if (at_or_after) {
+        s = i + __ffs(at_or_after) - 1;
+    } else {
+        s = s_carry;
+        for (int w = warp + 1; w < kHopChunk / 32; w++) {
+            if (warp_first[w] < N) { s = warp_first[w]; break; }
+        }
+    }
+    const int nx = s < N ? s + p.best[s].x : N;
+    p.hop[i] = make_int2(s, nx);
+    const int dlt = nx - i;
+    p.delta16[i] = (unsigned short)(dlt < 65535 ? dlt : 65535);
+}
 
 __global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p, int window) {
     extern __shared__ unsigned short s_delta[];
-    __shared__ int warp_first[32];
     __shared__ int s_nspans, s_pos;
     const int N = p.n_query;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    // contiguous range of whole 32-position tiles per warp
-    const int tiles = (N + 31) / 32;
-    const int tiles_per_warp = (tiles + nwarps - 1) / nwarps;
-    const int t_lo = warp * tiles_per_warp, t_hi = min(tiles, t_lo + tiles_per_warp);
-
-    // pass A: first position with a candidate in this warp's range
-    int first = N;
-    for (int tl = t_lo; tl < t_hi; tl++) {
-        int i = tl * 32 + lane;
-        bool st = i < N && p.best[i].x > 0;
-        unsigned int b = __ballot_sync(0xffffffffu, st);
-        if (b) { first = tl * 32 + __ffs(b) - 1; break; }
-    }
-    if (lane == 0) warp_first[warp] = first;
+    const int tid = threadIdx.x;
     if (tid == 0) { s_pos = 0; s_nspans = 0; }
-    __syncthreads();
-    // first candidate position after this warp's range
-    int carry = N;
-    for (int w = nwarps - 1; w > warp; w--) carry = min(carry, warp_first[w]);
-    int carry_next = carry < N ? carry + p.best[carry].x : N;
-
-    // pass B: tiles backwards, carrying the next candidate position; four tiles' loads in flight at a time
-    for (int tg = t_hi - 1; tg >= t_lo; tg -= 4) {
-        int lens[4];
-#pragma unroll
-        for (int u = 0; u < 4; u++) {
-            const int i = (tg - u) * 32 + lane;
-            lens[u] = (tg - u >= t_lo && i < N) ? p.best[i].x : 0;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; u++) {
-            const int tl = tg - u;
-            if (tl < t_lo) break;
-            const int i = tl * 32 + lane;
-            const int len = lens[u];
-            unsigned int b = __ballot_sync(0xffffffffu, len > 0);
-            unsigned int at_or_after = b >> lane;
-            int s = carry, nx = carry_next;
-            const int src = at_or_after ? lane + __ffs(at_or_after) - 1 : lane;
-            const int len_src = __shfl_sync(0xffffffffu, len, src);  // one convergent shuffle for all lanes
-            if (at_or_after) {
-                s = tl * 32 + src;
-                nx = s + len_src;
-            }
-            if (i < N) p.hop[i] = make_int2(s, nx);
-            if (b) {
-                int f = __ffs(b) - 1;
-                carry = tl * 32 + f;
-                carry_next = carry + __shfl_sync(0xffffffffu, len, f);
-            }
-        }
-    }
     __syncthreads();
 
     // (2) the chain, window by window; spans_ws[n].q_start keeps the n-th visited position
@@ -185,9 +186,15 @@ __global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p, int w
         const int wbeg = s_pos;
         if (wbeg >= N) break;
         const int wend = min(N, wbeg + window);
-        for (int i = wbeg + tid; i < wend; i += blockDim.x) {
-            const int dlt = p.hop[i].y - i;
-            s_delta[i - wbeg] = (unsigned short)(dlt < 65535 ? dlt : 65535);
+        // eight deltas per load where the window start allows it (the array itself is 16-byte aligned)
+        if ((wbeg & 7) == 0) {
+            const int n8 = (wend - wbeg) >> 3;
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.delta16 + wbeg);
+            uint4 *dst = reinterpret_cast<uint4 *>(s_delta);
+            for (int i = tid; i < n8; i += blockDim.x) dst[i] = src[i];
+            for (int i = wbeg + (n8 << 3) + tid; i < wend; i += blockDim.x) s_delta[i - wbeg] = p.delta16[i];
+        } else {
+            for (int i = wbeg + tid; i < wend; i += blockDim.x) s_delta[i - wbeg] = p.delta16[i];
         }
         __syncthreads();
         if (tid == 0) {
@@ -206,25 +213,22 @@ __global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p, int w
         // the last visited position may have no candidate at or after it: then it starts no span
         int n = s_nspans;
         if (n > 0 && p.hop[p.spans_ws[n - 1].q_start].x >= N) n--;
-        s_nspans = n;
         *p.n_spans = n;
     }
-    __syncthreads();
+}
 
-    // (3) spans (one thread each: the three dependent lookups of different spans overlap), then per-token rows
-    const int ns = s_nspans;
-    for (int sidx = tid; sidx < ns; sidx += blockDim.x) {
+// (3) grid-wide: every visited position becomes a span (three dependent lookups), which a warp expands to rows
+__global__ void match_expand_kernel(MatchParams p) {
+    const int ns = *p.n_spans;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    for (int sidx = gw; sidx < ns; sidx += warps) {
         const int2 h = p.hop[p.spans_ws[sidx].q_start];
         rac_span sp;
         sp.q_start = h.x;
         sp.len = h.y - h.x;
         sp.h_start = p.best[h.x].y;
-        p.spans_ws[sidx] = sp;
-        if (p.spans_out) p.spans_out[sidx] = sp;
-    }
-    __syncthreads();
-    for (int sidx = warp; sidx < ns; sidx += nwarps) {
-        const rac_span sp = p.spans_ws[sidx];
+        if (lane == 0 && p.spans_out) p.spans_out[sidx] = sp;
         for (int m = lane; m < sp.len; m += 32) p.ref_row[sp.q_start + m] = sp.h_start + m;
     }
 }
@@ -349,8 +353,25 @@ __global__ void fill2_i32_kernel(int32_t *a, long long na, int32_t va, int32_t *
 
 static size_t align16(size_t v) { return (v + 15) / 16 * 16; }
 
+// the four launches of the selection (suffix scan grid-wide, chain walk in one CTA, expansion grid-wide)
+static int launch_selection(const MatchParams &p, cudaStream_t st) {
+    const int nchunks = (p.n_query + kHopChunk - 1) / kHopChunk;
+    match_chunk_first_kernel<<<nchunks, kHopChunk, 0, st>>>(p);
+    match_hop_kernel<<<nchunks, kHopChunk, 0, st>>>(p, nchunks);
+    const int window = p.n_query < kWalkWindow ? p.n_query : kWalkWindow;
+    const size_t dyn = ((size_t)window * 2 + 15) / 16 * 16;
+    if (dyn > 48 * 1024 &&
+        cudaFuncSetAttribute(match_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+        return RAC_ECUDA;
+    match_select_kernel<<<1, 1024, dyn, st>>>(p, window);
+    match_expand_kernel<<<148, 256, 0, st>>>(p);
+    return RAC_OK;
+}
+
+
+
 struct MatchLayout {
-    size_t rep, top, slot_of, best, hop, spans, total;
+    size_t rep, top, slot_of, best, hop, spans, chunk_first, delta16, total;
     unsigned int M;
 };
 static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
@@ -365,6 +386,8 @@ static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
     L.best = o;     o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 8);
     L.hop = o;      o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 8);
     L.spans = o;    o = align16(o + (size_t)(n_query + 1) * sizeof(rac_span));
+    L.chunk_first = o; o = align16(o + ((size_t)(n_query > 0 ? n_query : 1) / kHopChunk + 1) * 4);
+    L.delta16 = o;  o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 2);
     L.total = o;
     return L;
 }
@@ -432,6 +455,8 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     p.best = reinterpret_cast<int2 *>(ws + L.best);
     p.hop = reinterpret_cast<int2 *>(ws + L.hop);
     p.spans_ws = reinterpret_cast<rac_span *>(ws + L.spans);
+    p.chunk_first = reinterpret_cast<int32_t *>(ws + L.chunk_first);
+    p.delta16 = reinterpret_cast<unsigned short *>(ws + L.delta16);
     p.n_hist = (int)n_hist;
     p.n_query = (int)n_query;
     p.nwin = (int)(n_hist - min_ngram + 1 > 0 ? n_hist - min_ngram + 1 : 0);
@@ -453,13 +478,7 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     }
     if (n_query > 0) {
         match_query_kernel<<<(int)((n_query + tb - 1) / tb), tb, 0, st>>>(p);
-        // shared-memory window of the chain walk (16-bit deltas)
-        int window = n_query < kWalkWindow ? (int)n_query : kWalkWindow;
-        size_t dyn = ((size_t)window * 2 + 15) / 16 * 16;
-        if (dyn > 48 * 1024 &&
-            cudaFuncSetAttribute(match_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
-            return RAC_ECUDA;
-        match_select_kernel<<<1, 1024, dyn, st>>>(p, window);
+        if (launch_selection(p, st) != RAC_OK) return RAC_ECUDA;
     }
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
@@ -520,7 +539,7 @@ IndexLayout index_layout(const rac_index_cfg *c) {
     return L;
 }
 struct QueryLayout {
-    size_t best, hop, spans, trep, tfirst, total;
+    size_t best, hop, spans, chunk_first, delta16, trep, tfirst, total;
     unsigned int Mq;
 };
 QueryLayout query_layout(long long n_query) {
@@ -533,6 +552,8 @@ QueryLayout query_layout(long long n_query) {
     L.best = o;    o = align16(o + n * 8);
     L.hop = o;     o = align16(o + n * 8);
     L.spans = o;   o = align16(o + (n + 1) * sizeof(rac_span));
+    L.chunk_first = o; o = align16(o + (n / kHopChunk + 1) * 4);
+    L.delta16 = o; o = align16(o + n * 2);
     L.trep = o;    o = align16(o + (size_t)M * 4);
     L.tfirst = o;  o = align16(o + (size_t)M * 4);
     L.total = o;
@@ -629,6 +650,8 @@ int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_by
     p.best = reinterpret_cast<int2 *>(ws + Q.best);
     p.hop = reinterpret_cast<int2 *>(ws + Q.hop);
     p.spans_ws = reinterpret_cast<rac_span *>(ws + Q.spans);
+    p.chunk_first = reinterpret_cast<int32_t *>(ws + Q.chunk_first);
+    p.delta16 = reinterpret_cast<unsigned short *>(ws + Q.delta16);
     p.n_hist = (int)n_hist;
     p.n_query = (int)n_query;
     p.nwin = (int)(n_hist - cfg->min_ngram + 1 > 0 ? n_hist - cfg->min_ngram + 1 : 0);
@@ -642,12 +665,7 @@ int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_by
     fill2_i32_kernel<<<grid_for(n_query > 1 ? n_query : 1, tb), tb, 0, st>>>(ref_row, n_query, -1, n_spans, 1, 0);
     if (n_query == 0) return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
     match_query_kernel<<<(int)((n_query + tb - 1) / tb), tb, 0, st>>>(p);
-    const int window = n_query < kWalkWindow ? (int)n_query : kWalkWindow;
-    const size_t dyn = ((size_t)window * 2 + 15) / 16 * 16;
-    if (dyn > 48 * 1024 &&
-        cudaFuncSetAttribute(match_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
-        return RAC_ECUDA;
-    match_select_kernel<<<1, 1024, dyn, st>>>(p, window);
+    if (launch_selection(p, st) != RAC_OK) return RAC_ECUDA;
     if (intra) {
         fill2_i32_kernel<<<grid_for(Q.Mq, tb), tb, 0, st>>>(trep, (long long)Q.Mq, -1, tfirst, (long long)Q.Mq, 0x7fffffff);
         const int nb = (int)((n_query + tb - 1) / tb);
