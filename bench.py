@@ -522,7 +522,7 @@ def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    smp = OracleSample(wl, seed=4, sample_tokens=1024)
+    smp = OracleSample(wl, seed=4, sample_tokens=4096)
     vals = []
     desc = None
     for i in range(args.warmup + args.steps):
@@ -694,7 +694,7 @@ def main():
                     "frac_of_nominal_8TBps": achieved / 8000.0}
         cpu = None
         if not args.no_cpu_baseline:
-            smp = OracleSample(wl, seed=4, sample_tokens=16384)
+            smp = OracleSample(wl, seed=4, sample_tokens=32768)
             gbs, desc = smp.run()
             cpu = {"value": gbs, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": desc}
         line = {
