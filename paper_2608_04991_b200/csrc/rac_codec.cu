@@ -536,7 +536,7 @@ constexpr int kOutHot = 256;       // slab list per token in flight (d <= 8192 h
 // shared, so a token costs about two thirds of the issue slots).  All warp collectives name only the W lanes
 // of the token.
 template <int BITS, int W, bool SUB>
-__global__ void __launch_bounds__(kOutWarps * 32, 5) outlier_kernel(const CodecParams p) {
+__global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecParams p) {
     constexpr int TPW = 32 / W;                 // tokens per warp
     constexpr int NV = 256 / W;                 // slab maxima per lane, at most
     __shared__ unsigned long long s_cand[kOutWarps * TPW][kOutCap];
@@ -560,8 +560,29 @@ __global__ void __launch_bounds__(kOutWarps * 32, 5) outlier_kernel(const CodecP
     const int tm_stride = (nth + 3) & ~3;       // rows of slab maxima are padded to 16 bytes
 
     const long long n_tok = tokens_to_do<SUB>(p);
-    for (long long ti = ((long long)blockIdx.x * kOutWarps + warp) * TPW + sub; ti < n_tok; ti += tstride) {
+    const int ni = (nth + W - 1) / W;
+    // slab maxima of a token, lane l taking slabs l, l+W, ...; loaded one token ahead so that the first trip to
+    // memory of a token overlaps the work on the one before
+    unsigned int tv[NV], tvn[NV];
+    auto load_maxima = [&](long long tix, unsigned int (&dst)[NV]) {
+        const long long tt = tix < n_tok ? token_at<SUB>(p, tix) : 0;
+        const float *tm = p.tmax + tt * tm_stride;
+#pragma unroll
+        for (int i = 0; i < NV; i++) {
+            dst[i] = 0u;
+            if (i < ni && tix < n_tok) {
+                const int th = sl + W * i;
+                if (th < nth) dst[i] = __float_as_uint(__ldg(tm + th));
+            }
+        }
+    };
+    const long long ti0 = ((long long)blockIdx.x * kOutWarps + warp) * TPW + sub;
+    load_maxima(ti0, tvn);
+    for (long long ti = ti0; ti < n_tok; ti += tstride) {
         const long long t = token_at<SUB>(p, ti);
+#pragma unroll
+        for (int i = 0; i < NV; i++) tv[i] = tvn[i];
+        load_maxima(ti + tstride, tvn);
         // reference row of the token, by the same rules as the streaming pass (which already reported bad rows)
         const int row = resolve_row<SUB>(p, p.ref_row ? p.ref_row[t] : (int)t, false);
         const uint16_t *xrow = p.X + t * d;
@@ -583,19 +604,10 @@ __global__ void __launch_bounds__(kOutWarps * 32, 5) outlier_kernel(const CodecP
         // (a) threshold: the k-th largest of the W per-lane maxima (lane l covers slabs l, l+W, ...): the k largest
         // come from k different lanes, each with an element at least that large, so at least k elements reach it;
         // then the slabs that reach it, in slab order
-        const float *tm = p.tmax + t * tm_stride;
-        const int ni = (nth + W - 1) / W;
-        unsigned int tv[NV];
         unsigned int v = 0u;
 #pragma unroll
-        for (int i = 0; i < NV; i++) {
-            tv[i] = 0u;
-            if (i < ni) {
-                const int th = sl + W * i;
-                if (th < nth) tv[i] = __float_as_uint(tm[th]);
-                v = max(v, tv[i]);
-            }
-        }
+        for (int i = 0; i < NV; i++)
+            if (i < ni) v = max(v, tv[i]);
         unsigned int tau = 0u;
         for (int r = 0; r < k; r++) {           // k <= 16 <= W, so k different lanes exist
             tau = __reduce_max_sync(gmask, v);
