@@ -628,26 +628,32 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
             }
         }
         __syncwarp(gmask);
-        // (b) candidates: W/4 slabs per round, a lane takes 8 consecutive channels of one slab, so that the loads
-        // of a round are all in flight together
+        // (b) candidates: W/2 slabs per round, a lane takes 16 consecutive channels of one slab, so that the loads
+        // of all hot slabs of a typical token (8 to 16) are in flight together
         int n = 0;  // uniform over the token's lanes
-        for (int base = 0; base < nh; base += W / 4) {
-            const int hi = base + (sl >> 2);
+        for (int base = 0; base < nh; base += W / 2) {
+            const int hi = base + (sl >> 1);
             const bool act = hi < nh;
-            const int c0 = act ? (int)hot[hi] * 32 + (sl & 3) * 8 : 0;
-            uint4 xw = make_uint4(0u, 0u, 0u, 0u), rw = xw;
+            const int c0 = act ? (int)hot[hi] * 32 + (sl & 1) * 16 : 0;
+            uint4 xw[2], rw[2];
+            xw[0] = xw[1] = rw[0] = rw[1] = make_uint4(0u, 0u, 0u, 0u);
             uint32_t cf = 0u;
             if (act) {
-                xw = __ldg(reinterpret_cast<const uint4 *>(xrow + c0));
-                if (rrow) rw = __ldg(reinterpret_cast<const uint4 *>(rrow + c0));
+                xw[0] = __ldg(reinterpret_cast<const uint4 *>(xrow + c0));
+                xw[1] = __ldg(reinterpret_cast<const uint4 *>(xrow + c0 + 8));
+                if (rrow) {
+                    rw[0] = __ldg(reinterpret_cast<const uint4 *>(rrow + c0));
+                    rw[1] = __ldg(reinterpret_cast<const uint4 *>(rrow + c0 + 8));
+                }
                 cf = coef[c0 >> (5 + p.lpg_shift)];
             }
-            const uint32_t xs[4] = {xw.x, xw.y, xw.z, xw.w}, rs[4] = {rw.x, rw.y, rw.z, rw.w};
+            const uint32_t xs[8] = {xw[0].x, xw[0].y, xw[0].z, xw[0].w, xw[1].x, xw[1].y, xw[1].z, xw[1].w};
+            const uint32_t rs[8] = {rw[0].x, rw[0].y, rw[0].z, rw[0].w, rw[1].x, rw[1].y, rw[1].z, rw[1].w};
             const float ca = half_bits_to_float(cf & 0xffff), cb = half_bits_to_float(cf >> 16);
-            float e[8];
+            float e[16];
             if (rrow && p.gain) {
 #pragma unroll
-                for (int i = 0; i < 8; i++) {
+                for (int i = 0; i < 16; i++) {
                     const uint32_t xb = (i & 1) ? (xs[i >> 1] & 0xffff0000u) : (xs[i >> 1] << 16);
                     const uint32_t rb = (i & 1) ? (rs[i >> 1] & 0xffff0000u) : (rs[i >> 1] << 16);
                     const float r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c0 + i]), __uint_as_float(rb),
@@ -657,7 +663,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
             } else {
                 // without a reference rw is zero, which is the zero reference of a directly coded token
 #pragma unroll
-                for (int i = 0; i < 8; i++) {
+                for (int i = 0; i < 16; i++) {
                     const uint32_t xb = (i & 1) ? (xs[i >> 1] & 0xffff0000u) : (xs[i >> 1] << 16);
                     const uint32_t rb = (i & 1) ? (rs[i >> 1] & 0xffff0000u) : (rs[i >> 1] << 16);
                     e[i] = __fsub_rn(__uint_as_float(xb), __fmaf_rn(ca, __uint_as_float(rb), cb));
@@ -665,7 +671,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
             }
             int cnt = 0;
 #pragma unroll
-            for (int i = 0; i < 8; i++) cnt += ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? 1 : 0;
+            for (int i = 0; i < 16; i++) cnt += ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? 1 : 0;
             if (!act) cnt = 0;
             // exclusive prefix of the per-lane counts within the token's lanes
             int incl = cnt;
@@ -677,7 +683,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
             int pos = n + incl - cnt;
             if (cnt) {
 #pragma unroll
-                for (int i = 0; i < 8; i++) {
+                for (int i = 0; i < 16; i++) {
                     const unsigned int key = __float_as_uint(e[i]) & 0x7fffffffu;
                     if (key >= tau) {
                         if (pos < kOutCap) {
