@@ -34,9 +34,9 @@ WORKLOAD = dict(T=131072, d=5120, group=128, bits=4, topk=8, n_hist=131072, min_
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one rac_encode[_reconstruct] call (streaming kernel +
 # outlier kernel) from the ncu capture of the SMALL case (profiles/codec_kernels_small_case_T16384_d5120.md);
 # traffic is proportional to tokens, so a launch of T tokens moves T/16384 times as much.
-NCU_SMALL_CASE_TRAFFIC = {"encode_sender_up": 267.80e6 + 179.96e6 + 53.34e6 + 1.63e6,
-                          "encode_dn": 335.61e6 + 44.24e6 + 59.43e6 + 0.45e6,
-                          "decode_up": 141.50e6 + 117.24e6, "decode_dn": 212.93e6 + 125.28e6}
+NCU_SMALL_CASE_TRAFFIC = {"encode_sender_up": 267.86e6 + 179.56e6 + 53.35e6 + 1.72e6,
+                          "encode_dn": 335.63e6 + 43.31e6 + 59.46e6 + 0.53e6,
+                          "decode_up": 141.17e6 + 117.74e6, "decode_dn": 212.96e6 + 125.12e6}
 SMALL = dict(T=16384, d=5120, group=128, bits=4, topk=8, n_hist=16384, min_ngram=4, max_hits=8, gap_max=112)
 
 
