@@ -669,10 +669,12 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
                     e[i] = __fsub_rn(__uint_as_float(xb), __fmaf_rn(ca, __uint_as_float(rb), cb));
                 }
             }
-            int cnt = 0;
+            // which of the lane's 16 elements reach the threshold
+            uint32_t m = 0u;
 #pragma unroll
-            for (int i = 0; i < 16; i++) cnt += ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? 1 : 0;
-            if (!act) cnt = 0;
+            for (int i = 0; i < 16; i++) m |= ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? (1u << i) : 0u;
+            if (!act) m = 0u;
+            const int cnt = __popc(m);
             // exclusive prefix of the per-lane counts within the token's lanes
             int incl = cnt;
 #pragma unroll
@@ -681,18 +683,23 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
                 if (sl >= o) incl += up;
             }
             int pos = n + incl - cnt;
-            if (cnt) {
+            // few lanes have any, and those mostly one: walk the set bits, fetching the element by a select tree
+            while (m) {
+                const int i = __ffs(m) - 1;
+                m &= m - 1u;
+                float s8[8], s4[4];
 #pragma unroll
-                for (int i = 0; i < 16; i++) {
-                    const unsigned int key = __float_as_uint(e[i]) & 0x7fffffffu;
-                    if (key >= tau) {
-                        if (pos < kOutCap) {
-                            cand[pos] = ((unsigned long long)key << 16) | (unsigned long long)(0xffff - (c0 + i));
-                            cande[pos] = e[i];
-                        }
-                        pos++;
-                    }
+                for (int j = 0; j < 8; j++) s8[j] = (i & 1) ? e[2 * j + 1] : e[2 * j];
+#pragma unroll
+                for (int j = 0; j < 4; j++) s4[j] = (i & 2) ? s8[2 * j + 1] : s8[2 * j];
+                const float s20 = (i & 4) ? s4[1] : s4[0], s21 = (i & 4) ? s4[3] : s4[2];
+                const float ei = (i & 8) ? s21 : s20;
+                if (pos < kOutCap) {
+                    cand[pos] = ((unsigned long long)(__float_as_uint(ei) & 0x7fffffffu) << 16) |
+                                (unsigned long long)(0xffff - (c0 + i));
+                    cande[pos] = ei;
                 }
+                pos++;
             }
             n += __shfl_sync(gmask, incl, W - 1, W);
         }
