@@ -565,15 +565,14 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
     // memory of a token overlaps the work on the one before
     unsigned int tv[NV], tvn[NV];
     auto load_maxima = [&](long long tix, unsigned int (&dst)[NV]) {
-        const long long tt = tix < n_tok ? token_at<SUB>(p, tix) : 0;
+        const bool live = tix < n_tok;
+        const long long tt = live ? token_at<SUB>(p, tix) : 0;
         const float *tm = p.tmax + tt * tm_stride;
+        const int lim = live ? nth : 0;     // slabs beyond the width (or beyond the last token) read as 0
 #pragma unroll
         for (int i = 0; i < NV; i++) {
-            dst[i] = 0u;
-            if (i < ni && tix < n_tok) {
-                const int th = sl + W * i;
-                if (th < nth) dst[i] = __float_as_uint(__ldg(tm + th));
-            }
+            const int th = sl + W * i;
+            dst[i] = th < lim ? __float_as_uint(__ldg(tm + th)) : 0u;
         }
     };
     const long long ti0 = ((long long)blockIdx.x * kOutWarps + warp) * TPW + sub;
@@ -606,8 +605,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
         // then the slabs that reach it, in slab order
         unsigned int v = 0u;
 #pragma unroll
-        for (int i = 0; i < NV; i++)
-            if (i < ni) v = max(v, tv[i]);
+        for (int i = 0; i < NV; i++) v = max(v, tv[i]);
         unsigned int tau = 0u;
         for (int r = 0; r < k; r++) {           // k <= 16 <= W, so k different lanes exist
             tau = __reduce_max_sync(gmask, v);
