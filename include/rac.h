@@ -309,6 +309,14 @@ int rac_decode_reconstruct_list(const rac_codec_cfg *cfg, const void *payload, i
  * Sums are merged in binary64 in a fixed order: the same result on every run.
  * Coding: pass coef_seg and seg_of to the *_list calls (with tok_list NULL for all tokens) together with
  * coef_fmt = 1; with coef_fmt = 0 both must be NULL. */
+/* The spans of a retrieval and the gaps between them as segments for rac_fit_segments, without a trip to the
+ * host: seg_off[0 .. *n_seg] receives the boundaries (0, starts and ends of the spans, T; empty pieces dropped),
+ * and seg_off[*n_seg + 1 .. max_seg] is filled with T, so that rac_fit_segments can be called with n_seg = max_seg
+ * (the surplus segments are empty).  seg_off: device int32[max_seg + 1]; n_seg: device int32[1].  Spans must be in
+ * query order and disjoint (as rac_match_spans / rac_index_query emit them).  At most (max_seg - 1) / 2 spans are
+ * used: size max_seg as 2 * (span capacity) + 1. */
+int rac_spans_to_segments(const rac_span *spans, const int32_t *n_spans, int64_t T, int64_t max_seg,
+                          int32_t *seg_off, int32_t *n_seg, void *stream);
 size_t rac_fit_segments_workspace_bytes(const rac_codec_cfg *cfg, int64_t T);
 int rac_fit_segments(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
                      const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const int32_t *seg_off,

@@ -353,3 +353,15 @@ def fit_segments(d, group, X, seg_off, ref_base=None, ref_row=None, gain=None, b
     if rc != 0:
         raise ValueError(f"orc_fit_segments failed: {rc}")
     return (coef, dg) if diag else coef
+
+
+def segments_from_spans(spans: np.ndarray, T: int) -> np.ndarray:
+    """Boundaries of the segmentation "spans and the gaps between them": int32[n_seg+1], empty pieces dropped."""
+    b = [0]
+    for q, _, ln in np.asarray(spans, np.int64).reshape(-1, 3):
+        for x in (q, q + ln):
+            if x > b[-1]:
+                b.append(int(x))
+    if b[-1] < T:
+        b.append(int(T))
+    return np.array(b, np.int32)

@@ -34,7 +34,7 @@ EXPORTS = [
     "rac_encode_workspace_bytes", "rac_encode", "rac_encode_reconstruct", "rac_decode_reconstruct",
     "rac_sender_reconstruct",
     "rac_split_waves", "rac_encode_reconstruct_list", "rac_decode_reconstruct_list",
-    "rac_fit_segments_workspace_bytes", "rac_fit_segments",
+    "rac_fit_segments_workspace_bytes", "rac_fit_segments", "rac_spans_to_segments",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
     "rac_recon_error_workspace_bytes", "rac_recon_error",
 ]
@@ -126,6 +126,8 @@ def load() -> C.CDLL:
                                               vp, vp, sz, vp, vp]
     l.rac_decode_reconstruct_list.restype = C.c_int
     l.rac_decode_reconstruct_list.argtypes = [cfgp, vp, i64, vp, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp]
+    l.rac_spans_to_segments.restype = C.c_int
+    l.rac_spans_to_segments.argtypes = [vp, vp, i64, i64, vp, vp, vp]
     l.rac_fit_segments_workspace_bytes.restype = sz
     l.rac_fit_segments_workspace_bytes.argtypes = [cfgp, i64]
     l.rac_fit_segments.restype = C.c_int
@@ -232,6 +234,13 @@ def rac_decode_reconstruct_list(cfg, payload, T, tok_list, tok_count, ref_base, 
         _ptr(ref_gain, _F16, "ref_gain"), _ptr(ref_bias, _F16, "ref_bias"), _ptr(step, _F32, "step"),
         _ptr(X_hat, _BF16, "X_hat"), _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
     _check("rac_decode_reconstruct_list", rc)
+
+
+def rac_spans_to_segments(spans, n_spans, T, max_seg, seg_off, n_seg, stream=None) -> None:
+    rc = load().rac_spans_to_segments(_ptr(spans, _I32, "spans"), _ptr(n_spans, _I32, "n_spans"), int(T), int(max_seg),
+                                      _ptr(seg_off, _I32, "seg_off"), _ptr(n_seg, _I32, "n_seg"),
+                                      _stream() if stream is None else stream)
+    _check("rac_spans_to_segments", rc)
 
 
 def rac_fit_segments_workspace_bytes(cfg: CodecCfg, T: int) -> int:

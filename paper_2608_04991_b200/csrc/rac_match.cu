@@ -247,6 +247,53 @@ __global__ void spans_to_rows_kernel(const rac_span *spans, const int32_t *n_spa
     }
 }
 
+// Spans and the gaps between them as segments: boundaries in ascending order, empty pieces dropped, the unused
+// tail of seg_off filled with T (empty segments).  One CTA; thread k looks at span k.
+__global__ void __launch_bounds__(1024) spans_to_segments_kernel(const rac_span *spans, const int32_t *n_spans, int T,
+                                                                 int max_seg, int32_t *seg_off, int32_t *n_seg) {
+    __shared__ int s_scan[1024];
+    __shared__ int s_base;
+    const int ns = min(*n_spans, (max_seg - 1) / 2);
+    const int tid = threadIdx.x;
+    if (tid == 0) { s_base = 1; seg_off[0] = 0; }   // boundary 0 always; every span adds its start (if a gap precedes) and its end
+    __syncthreads();
+    for (int k0 = 0; k0 < ns; k0 += 1024) {
+        const int k = k0 + tid;
+        int q0 = 0, q1 = 0, prev_end = 0, cnt = 0;
+        if (k < ns) {
+            q0 = spans[k].q_start;
+            q1 = q0 + spans[k].len;
+            prev_end = k > 0 ? spans[k - 1].q_start + spans[k - 1].len : 0;
+            cnt = (q0 > prev_end ? 1 : 0) + (q1 > q0 ? 1 : 0);   // boundaries q0 (new only after a gap) and q1
+        }
+        s_scan[tid] = cnt;
+        __syncthreads();
+        for (int o = 1; o < 1024; o <<= 1) {
+            const int v = tid >= o ? s_scan[tid - o] : 0;
+            __syncthreads();
+            s_scan[tid] += v;
+            __syncthreads();
+        }
+        int at = s_base + s_scan[tid] - cnt;
+        if (k < ns) {
+            if (q0 > prev_end) seg_off[at++] = q0;
+            if (q1 > q0) seg_off[at] = q1;
+        }
+        __syncthreads();
+        if (tid == 1023) s_base += s_scan[1023];
+        __syncthreads();
+    }
+    int nb = s_base;                      // boundaries written so far, the last one is the end of the last span
+    __syncthreads();
+    if (tid == 0) {
+        if (seg_off[nb - 1] < T) seg_off[nb++] = T;   // the gap behind the last span
+        *n_seg = nb - 1;
+        s_base = nb;
+    }
+    __syncthreads();
+    for (int i = s_base + tid; i <= max_seg; i += 1024) seg_off[i] = T;
+}
+
 __global__ void fill_i32_kernel(int32_t *dst, long long n, int32_t v) {
     long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     long long stride = (long long)gridDim.x * blockDim.x;
@@ -676,3 +723,13 @@ int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_by
 }
 
 }  // extern "C"
+
+extern "C" int rac_spans_to_segments(const rac_span *spans, const int32_t *n_spans, int64_t T, int64_t max_seg,
+                                     int32_t *seg_off, int32_t *n_seg, void *stream) {
+    if (!n_spans || !seg_off || !n_seg || T < 0 || max_seg < 1) return RAC_EINVAL;
+    if (T >= (1ll << 30) || max_seg >= (1ll << 30)) return RAC_EUNSUPPORTED;
+    if (!spans) return RAC_EINVAL;
+    spans_to_segments_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(spans, n_spans, (int)T, (int)max_seg, seg_off,
+                                                                               n_seg);
+    return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}

@@ -145,3 +145,49 @@ def test_one_long_segment_and_single_token_segments(env):
     o2 = orc.fit_segments(d, g, s.bf16_bits(X[:T2]), seg_off, ref_base=s.bf16_bits(R[:T2]))
     assert (c2.cpu().numpy().view(np.uint32) != o2).sum() <= 3
     assert np.array_equal(so2.cpu().numpy(), np.arange(T2))
+
+
+def test_spans_become_segments_on_the_device(env):
+    s, rac, orc, dev = env.synth, env.rac, env.orc, env.dev
+    for H, T, gap, seed in [(20000, 6000, 100, 3), (4000, 5000, 0, 4), (3000, 200, 2000, 5), (50, 40, 5, 6)]:
+        wl = s.span_workload(H, T, seed=seed, gap_max=gap)
+        htok, qtok = torch.from_numpy(wl.hist).to(dev), torch.from_numpy(wl.query).to(dev)
+        nb = rac.rac_match_workspace_bytes(H, T, 8)
+        ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+        rows = torch.empty(T, dtype=torch.int32, device=dev)
+        cap = T // 4 + 1
+        spans = torch.zeros((cap, 3), dtype=torch.int32, device=dev)
+        n_spans = torch.zeros(1, dtype=torch.int32, device=dev)
+        rac.rac_match_spans(htok, H, qtok, T, 4, 8, rows, spans, n_spans, ws, nb)
+        max_seg = 2 * cap + 1
+        seg_off = torch.full((max_seg + 3,), -9, dtype=torch.int32, device=dev)
+        n_seg = torch.full((1,), -9, dtype=torch.int32, device=dev)
+        rac.rac_spans_to_segments(spans, n_spans, T, max_seg, seg_off, n_seg)
+        torch.cuda.synchronize()
+        ns = int(n_spans.item())
+        want = orc.segments_from_spans(spans[:ns].cpu().numpy(), T)
+        got_n = int(n_seg.item())
+        assert got_n == len(want) - 1
+        assert np.array_equal(seg_off[:got_n + 1].cpu().numpy(), want)
+        assert torch.all(seg_off[got_n + 1:max_seg + 1] == T) and torch.all(seg_off[max_seg + 1:] == -9)
+        # every segment is a whole span or a whole gap
+        r = rows.cpu().numpy()
+        for a, b in zip(want[:-1], want[1:]):
+            assert (r[a:b] >= 0).all() or (r[a:b] < 0).all()
+    # and straight into the fit, without reading the count back: the surplus segments are empty
+    d, g = 256, 64
+    gen = s.generator(77, dev)
+    Hs = s.activations(H, d, s.channel_scale(d, 7, dev), gen)
+    X = s.affine_noisy_target(Hs, rows, g, gen, s.channel_scale(d, 7, dev))
+    cfg = rac.CodecCfg(d, g, 4, 0, scale_mode=1, coef_fmt=1)
+    coef = torch.full((max_seg, d // g), -1, dtype=torch.int32, device=dev)
+    seg_of = torch.empty(T, dtype=torch.int32, device=dev)
+    nbf = rac.rac_fit_segments_workspace_bytes(cfg, T)
+    wsf = torch.empty(nbf, dtype=torch.uint8, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    rac.rac_fit_segments(cfg, X, T, Hs, H, rows, None, None, seg_off, max_seg, coef, seg_of, wsf, nbf, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and not coef[got_n:].any()
+    o_coef = orc.fit_segments(d, g, s.bf16_bits(X), want, ref_base=s.bf16_bits(Hs), ref_row=r)
+    assert (coef[:got_n].cpu().numpy().view(np.uint32) != o_coef).sum() <= 2
+    assert np.array_equal(seg_of.cpu().numpy(), np.repeat(np.arange(got_n), np.diff(want)))
