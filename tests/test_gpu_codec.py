@@ -441,3 +441,41 @@ def test_family_ties_zero_groups_and_bad_offsets(env):
                     env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=96),
                     env.rac.CodecCfg(d, g, 5, 0, scale_mode=1)]:
         assert env.rac.rac_record_bytes(bad_cfg) == 0
+
+
+def test_family_random_configurations(env):
+    """Forty seeded random members of the Eq. 8 family on small shapes: widths, both groupings, outlier counts,
+    direct tokens, gathered rows and the gain/bias reference in random combination."""
+    rng = np.random.default_rng(4242)
+    s = env.synth
+    tried = 0
+    while tried < 40:
+        d = int(rng.choice([64, 96, 256, 512, 1024, 2080, 3584, 4096]))
+        g = int(rng.choice([32, 64, 128, 256]))
+        if d % g:
+            continue
+        bits = int(rng.choice([2, 3, 4, 8]))
+        qg = int(rng.choice([0, 32, 64, 128, 256, d]))
+        kg = int(rng.choice([0, 0, 1, 2, 3, 4]))
+        cfg = env.rac.CodecCfg(d, g, bits, 0, scale_mode=1, qgroup=qg, topk_group=kg)
+        if env.rac.rac_record_bytes(cfg) == 0:
+            assert env.orc.record_bytes(d, g, bits, 0, 1, qg, kg) == 0 or (qg or g) > 256 or d % (qg or g) or \
+                not ((qg or g) == d or ((qg or g) & ((qg or g) - 1)) == 0)
+            continue
+        tried += 1
+        T = int(rng.integers(1, 70))
+        X, R, _, _ = prefill_inputs(env, T, d, g, seed=int(rng.integers(1 << 30)))
+        kw = {}
+        mode = int(rng.integers(0, 4))
+        if mode == 1:      # some tokens coded directly
+            rows = np.arange(T, dtype=np.int32)
+            rows[rng.random(T) < 0.4] = -1
+            kw["ref_row"] = torch.from_numpy(rows).to(env.dev)
+        elif mode == 2:    # gathered rows
+            kw["ref_row"] = torch.from_numpy(rng.integers(0, T, T).astype(np.int32)).to(env.dev)
+        elif mode == 3:    # the per-channel transform of the reference
+            kw["gain"], kw["bias"] = s.predictor_gain_bias(d, int(rng.integers(100)), env.dev)
+        try:
+            env.P.round_trip_case(cfg, X, ref_base=R, **kw)
+        except AssertionError as e:
+            raise AssertionError(f"{cfg!r} T={T} mode={mode}: {e}") from e
