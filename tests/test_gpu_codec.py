@@ -479,3 +479,43 @@ def test_family_random_configurations(env):
             env.P.round_trip_case(cfg, X, ref_base=R, **kw)
         except AssertionError as e:
             raise AssertionError(f"{cfg!r} T={T} mode={mode}: {e}") from e
+
+
+def test_static_random_configurations(env):
+    """Thirty seeded random configurations of the static-table quantiser with per-token outliers on small shapes."""
+    rng = np.random.default_rng(2424)
+    s = env.synth
+    tried = 0
+    while tried < 30:
+        d = int(rng.choice([32, 96, 256, 512, 1024, 2080, 3584, 4096, 8192]))
+        g = int(rng.choice([32, 64, 128, 256, 1024]))
+        if d % g:
+            continue
+        bits = int(rng.choice([2, 3, 4]))
+        k = int(rng.choice([0, 1, 3, 8, 16]))
+        if k > d:
+            continue
+        tried += 1
+        T = int(rng.integers(1, 60))
+        X, R, cal, calr = prefill_inputs(env, T, d, g, seed=int(rng.integers(1 << 30)), cal_T=64)
+        kw = {}
+        mode = int(rng.integers(0, 4))
+        rows = None
+        if mode == 1:
+            rows = np.arange(T, dtype=np.int32)
+            rows[rng.random(T) < 0.4] = -1
+        elif mode == 2:
+            rows = rng.integers(0, T, T).astype(np.int32)
+        if rows is not None:
+            kw["ref_row"] = torch.from_numpy(rows).to(env.dev)
+        gb = {}
+        if mode == 3:
+            kw["gain"], kw["bias"] = s.predictor_gain_bias(d, int(rng.integers(100)), env.dev)
+            gb = dict(gain=s.f16_bits(kw["gain"]), bias=s.f16_bits(kw["bias"]))
+        step, inv = env.orc.calibrate(d, g, bits, s.bf16_bits(X), ref_base=s.bf16_bits(R), ref_row=rows, **gb)
+        # a table row without calibration tokens is all zero ("code 0"): legal, and part of what is being tested
+        cfg = env.rac.CodecCfg(d, g, bits, k)
+        try:
+            env.P.round_trip_case(cfg, X, ref_base=R, step=step, inv_step=inv, **kw)
+        except AssertionError as e:
+            raise AssertionError(f"{cfg!r} T={T} mode={mode}: {e}") from e
