@@ -14,8 +14,12 @@
 // on a plain linear row.
 //
 // Kernels: encode_ws_kernel (streaming pass of encode, optionally also the sender-side x_hat),
-// outlier_kernel (second launch of encode: the k largest |e| per token), decode_kernel (receiver and sender
-// reconstruction), calib_kernel + calib_finalize_kernel (step tables).
+// outlier_kernel (second launch of encode: the k largest |e| per token), decode_kernel and decode_ws_kernel
+// (receiver and sender reconstruction, with and without per-token outliers), calib_kernel +
+// calib_finalize_kernel (step tables; in its second form the statistics pass of the segment fit),
+// segment_fit_kernel + seg_of_kernel (Eq. 6 over several fitting positions), split_waves_kernel (tokens that
+// reference the same prompt go second), recon_error_kernel (error of a sender-path run).  The kernels of the
+// per-group-scale quantiser (Eq. 8 as printed) live in rac_codec_dyn.cu; this file holds the C ABI of both.
 #include "rac_codec_dev.cuh"
 
 namespace rac {
