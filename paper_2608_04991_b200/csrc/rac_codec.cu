@@ -996,26 +996,30 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
 // ------------------------------------------------------------------------------------------------
 // reconstruct, streaming form: no CTA barrier in the loop
 // ------------------------------------------------------------------------------------------------
-// Same arithmetic as decode_kernel.  The output row is written IN PLACE over the token's reference row in the
-// stage (a thread reads its 64-byte slab of r and writes x_hat there), so a stage is record + one row; every warp
-// ends its share of a token with one arrival on the stage's `done` mbarrier and moves on, and the warp whose turn
-// it is (token i: warp i mod warps) waits for `done`, sends the row off as a bulk store, and refills the stage once
-// the store has read it.  Records without per-token outliers only: patching outliers needs the reference of
-// single channels after the row has been overwritten, and keeping those aside cost more than the barrier of
-// decode_kernel (measured), so records with outliers stay with that kernel.
+// Same arithmetic as decode_kernel.  Every warp ends its share of a token with one arrival on the stage's `done`
+// mbarrier and moves on, and the warp whose turn it is (token i: warp i mod warps) waits for `done`, sends the
+// row off as a bulk store, and refills the stage once the store has read it.
+// Records without per-token outliers: the output row is written IN PLACE over the token's reference row in the
+// stage (a thread reads its 64-byte slab of r and writes x_hat there), so a stage is record + one row.
+// Records with outliers: the output row is a row of its own, so that the reference survives the dense pass; the
+// warp whose turn it is prepares the outliers while it waits for the others (lane n takes outlier n: aligned
+// reference of that channel + the stored binary16 value) and writes them over the dense results once every warp
+// has arrived.  No other thread looks at the outlier fields.  (A first version that let every thread test the
+// outlier list for channels it owns cost ~150 warp instructions per 32 channels and lost to the barrier form.)
 struct DwSmem {
     int stage0, stage_bytes, rec_pad, total;
 };
-__host__ __device__ inline DwSmem dw_smem_layout(int d, int rec, int stages) {
+__host__ __device__ inline DwSmem dw_smem_layout(int d, int rec, int stages, bool out_row) {
     DwSmem s;
     s.stage0 = align_up((int)sizeof(WsCtrl), 128);
     s.rec_pad = align_up(rec, 128);
-    s.stage_bytes = s.rec_pad + 2 * d;
+    s.stage_bytes = s.rec_pad + 2 * d + (out_row ? 2 * d : 0);   // record, reference row (, output row)
     s.total = s.stage0 + stages * s.stage_bytes;
     return s;
 }
 
-template <int BITS, bool SUB>
+// KT > 0: records with per-token outliers (the output row is a row of its own behind the reference row).
+template <int BITS, int KT, bool SUB>
 __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -1023,7 +1027,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
     const int rot = (lane >> 1) & 3;
     const int d = p.d;
     const bool valid = tid * 32 < d;
-    const DwSmem L = dw_smem_layout(d, p.rec, p.stages);
+    const DwSmem L = dw_smem_layout(d, p.rec, p.stages, KT > 0);
     WsCtrl *ctrl = reinterpret_cast<WsCtrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
     const int S = p.stages;
@@ -1090,6 +1094,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
         if (*reinterpret_cast<volatile int *>(&ctrl->abort)) break;
         unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = sbase + L.stage0 + stage * L.stage_bytes + L.rec_pad;
+        const uint32_t os = KT > 0 ? rs + row_bytes : rs;     // where x_hat goes: its own row, or over the reference
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
@@ -1150,7 +1155,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
                     unpack2(padd(pfma(a2, r2[i], b2), eh), x0, x1);
                     o[i] = f2_to_bf16x2(x0, x1);
                 }
-                sts128(rs + off[j], make_uint4(o[0], o[1], o[2], o[3]));   // x_hat over the slab just read
+                sts128(os + off[j], make_uint4(o[0], o[1], o[2], o[3]));
             }
         }
         fence_async_smem();
@@ -1161,10 +1166,41 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
             const int k_next = it + S;
             int raw_next = 0;
             if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);
+            // outliers: lane n prepares outlier n (Eq. 9: aligned reference + binary16 value) while the other warps
+            // are still busy; record and reference row do not change any more
+            int patch_c = -1;
+            unsigned short patch_x = 0;
+            if (KT > 0) {
+                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                const unsigned short *oval = oidx + p.topk;
+                const int c = lane < p.topk ? (int)oidx[lane] : -1;
+                const bool ok = c >= 0 && c < d;
+                if (ok) {
+                    const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[c >> (5 + p.lpg_shift)];
+                    float r = 0.f;
+                    if (has_ref) {
+                        r = __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(rec + L.rec_pad + 2 * c)) << 16);
+                        if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                    }
+                    const float xh = __fadd_rn(__fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16)),
+                                               half_bits_to_float(oval[lane]));
+                    patch_x = __bfloat16_as_ushort(__float2bfloat16_rn(xh));
+                }
+                // a malformed record may name a channel twice: the later entry wins, as in a serial pass
+                const unsigned int same = __match_any_sync(0xffffffffu, ok ? c : -1 - lane);
+                if (ok && (31 - __clz(same)) == lane) patch_c = c;
+                if (__any_sync(0xffffffffu, c >= d) && lane == 0 && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
+            }
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
+            if (KT > 0) {
+                if (patch_c >= 0)
+                    reinterpret_cast<unsigned short *>(rec + L.rec_pad + row_bytes)[patch_c] = patch_x;
+                fence_async_smem();
+                __syncwarp();
+            }
             if (lane == 0) {
                 const long long t = token_at<SUB>(p, first + (long long)it * stride);
-                bulk_store(p.X_hat + t * d, rs, row_bytes);
+                bulk_store(p.X_hat + t * d, os, row_bytes);
                 bulk_commit();
                 bulk_wait_read<0>();      // the row has been read: the stage may be refilled
                 if (k_next < n_my) issue(k_next, stage, raw_next);
@@ -1281,17 +1317,16 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;
-    // Without outliers the streaming form is the faster one (0.44-0.49 ms against 0.52 ms at 131072 x 5120; 0.37
-    // against 0.43 ms at 131072 x 4096).  With outliers it is not: their patching costs the streaming form more than
-    // the barrier costs the other (0.57 against 0.49 ms), so those keep the kernel with the CTA barrier, which is
-    // already at 94 % of the copy bandwidth there.  RAC_DEC_BARRIER=1 forces the barrier form everywhere.
-    const bool ws = kt == 0 && !sub && !getenv("RAC_DEC_BARRIER");
+    // The streaming form is the faster one (131072 x 5120: 0.444 against 0.517 ms without outliers, 0.451 against
+    // 0.491 ms with eight; 131072 x 4096: 0.37 against 0.43 and 0.40 against 0.46 ms).  The barrier form serves the
+    // token-list / second-reference-buffer calls, and everything under RAC_DEC_BARRIER=1.
+    const bool ws = !sub && !getenv("RAC_DEC_BARRIER");
     const int wstages = pick_stages(g.d, g.nthreads > 128 ? 3 : 2);
-    DwSmem LW = dw_smem_layout(g.d, g.rec, wstages);
+    DwSmem LW = dw_smem_layout(g.d, g.rec, wstages, kt > 0);
     if (ws) p.stages = wstages;
 #define RAC_DEC(B, K)                                                                            \
     (sub ? launch_persistent(decode_kernel<B, K, true>, p, g.nthreads, L.total, p.T, stream)    \
-     : ws ? launch_persistent(decode_ws_kernel<B, false>, p, g.nthreads, LW.total, p.T, stream) \
+     : ws ? launch_persistent(decode_ws_kernel<B, K, false>, p, g.nthreads, LW.total, p.T, stream) \
          : launch_persistent(decode_kernel<B, K, false>, p, g.nthreads, L.total, p.T, stream))
     switch (g.bits * 100 + kt) {
         case 400: return RAC_DEC(4, 0);
