@@ -34,9 +34,9 @@ WORKLOAD = dict(T=131072, d=5120, group=128, bits=4, topk=8, n_hist=131072, min_
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one rac_encode[_reconstruct] call (streaming kernel +
 # outlier kernel) from the ncu capture of the SMALL case (profiles/codec_kernels_small_case_T16384_d5120.md);
 # traffic is proportional to tokens, so a launch of T tokens moves T/16384 times as much.
-NCU_SMALL_CASE_TRAFFIC = {"encode_sender_up": 267.86e6 + 179.56e6 + 53.35e6 + 1.72e6,
-                          "encode_dn": 335.63e6 + 43.31e6 + 59.46e6 + 0.53e6,
-                          "decode_up": 141.17e6 + 117.74e6, "decode_dn": 212.96e6 + 125.12e6}
+NCU_SMALL_CASE_TRAFFIC = {"encode_sender_up": 267.66e6 + 179.89e6 + 53.39e6 + 1.70e6,
+                          "encode_dn": 335.63e6 + 43.53e6 + 59.44e6 + 0.51e6,
+                          "decode_up": 141.35e6 + 116.71e6, "decode_dn": 212.92e6 + 123.52e6}
 SMALL = dict(T=16384, d=5120, group=128, bits=4, topk=8, n_hist=16384, min_ngram=4, max_hits=8, gap_max=112)
 
 
@@ -683,7 +683,7 @@ def main():
             dom, dom_bytes, dom_ms, dom_n = ("rac_encode[_reconstruct] (encode_ws_kernel<4,true,*> + outlier_kernel<4>)",
                                              rt.bytes_of("encode_sender_up") + rt.bytes_of("encode_dn"), enc_ms, 2)
         else:
-            dom, dom_bytes, dom_ms, dom_n = ("decode_kernel<4,8>", rt.bytes_of("decode_up") + rt.bytes_of("decode_dn"),
+            dom, dom_bytes, dom_ms, dom_n = ("decode_ws_kernel<4,8>", rt.bytes_of("decode_up") + rt.bytes_of("decode_dn"),
                                              dec_ms, 2)
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
         dom_stages = ("encode_sender_up", "encode_dn") if enc_ms >= dec_ms else ("decode_up", "decode_dn")
