@@ -471,7 +471,9 @@ class OracleSample:
         self.orc, self.wl = oracle, wl
         T, d, g, bits = wl["T"], wl["d"], wl["group"], wl["bits"]
         self.S = S = min(sample_tokens, T)
-        self.cores = oracle.max_threads()
+        # every core this process may run on (a launcher may have set OMP_NUM_THREADS=1; the oracle takes its
+        # thread count as an argument, so that does not bind it)
+        self.cores = max(1, min(64, len(os.sched_getaffinity(0))))
         self.tw = tw = synth.span_workload(wl["n_hist"], T, seed=seed, gap_max=wl["gap_max"])
         rows, _ = oracle.match_spans(tw.hist, tw.query, wl["min_ngram"], wl["max_hits"])
         # activations only for the history rows the sample needs
