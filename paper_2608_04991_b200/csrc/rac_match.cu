@@ -107,7 +107,20 @@ __global__ void match_query_kernel(MatchParams p) {
                 if (j < 0) break;
                 int L = p.w;
                 const int hend = p.end_of ? p.end_of[j] : p.n_hist;   // a match stays inside its request
-                while (i + L < p.n_query && j + L < hend && p.query[i + L] == p.hist[j + L]) L++;
+                // four tokens per trip to memory: the loads of a trip are independent, and a long match is a chain
+                // of dependent trips
+                const int room = min(p.n_query - i, hend - j);            // L may grow up to this
+                while (L + 4 <= room) {
+                    const int32_t q0 = p.query[i + L], q1 = p.query[i + L + 1], q2 = p.query[i + L + 2], q3 = p.query[i + L + 3];
+                    const int32_t h0 = p.hist[j + L], h1 = p.hist[j + L + 1], h2 = p.hist[j + L + 2], h3 = p.hist[j + L + 3];
+                    if (q0 != h0) break;
+                    if (q1 != h1) { L += 1; goto extended; }
+                    if (q2 != h2) { L += 2; goto extended; }
+                    if (q3 != h3) { L += 3; goto extended; }
+                    L += 4;
+                }
+                while (L < room && p.query[i + L] == p.hist[j + L]) L++;
+            extended:;
                 if (L > bestL || (L == bestL && j > bestj)) { bestL = L; bestj = j; }
             }
         }
