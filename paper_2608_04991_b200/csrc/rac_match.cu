@@ -107,20 +107,21 @@ __global__ void match_query_kernel(MatchParams p) {
                 if (j < 0) break;
                 int L = p.w;
                 const int hend = p.end_of ? p.end_of[j] : p.n_hist;   // a match stays inside its request
-                // four tokens per trip to memory: the loads of a trip are independent, and a long match is a chain
+                // eight tokens per trip to memory: the loads of a trip are independent, and a long match is a chain
                 // of dependent trips
                 const int room = min(p.n_query - i, hend - j);            // L may grow up to this
-                while (L + 4 <= room) {
-                    const int32_t q0 = p.query[i + L], q1 = p.query[i + L + 1], q2 = p.query[i + L + 2], q3 = p.query[i + L + 3];
-                    const int32_t h0 = p.hist[j + L], h1 = p.hist[j + L + 1], h2 = p.hist[j + L + 2], h3 = p.hist[j + L + 3];
-                    if (q0 != h0) break;
-                    if (q1 != h1) { L += 1; goto extended; }
-                    if (q2 != h2) { L += 2; goto extended; }
-                    if (q3 != h3) { L += 3; goto extended; }
-                    L += 4;
+                bool open = true;
+                while (open && L + 8 <= room) {
+                    int32_t q[8], h[8];
+#pragma unroll
+                    for (int u = 0; u < 8; u++) { q[u] = p.query[i + L + u]; h[u] = p.hist[j + L + u]; }
+                    unsigned int ne = 0;
+#pragma unroll
+                    for (int u = 0; u < 8; u++) ne |= (q[u] != h[u]) ? (1u << u) : 0u;
+                    if (ne) { L += __ffs(ne) - 1; open = false; }
+                    else L += 8;
                 }
-                while (L < room && p.query[i + L] == p.hist[j + L]) L++;
-            extended:;
+                while (open && L < room && p.query[i + L] == p.hist[j + L]) L++;
                 if (L > bestL || (L == bestL && j > bestj)) { bestL = L; bestj = j; }
             }
         }
