@@ -31,7 +31,9 @@ struct MatchParams {
     int2 *hop;             // [N]      (next position >= p with a candidate, position after its span)
     rac_span *spans_ws;    // [N/w + 1]
     int32_t *chunk_first;  // [ceil(N/1024)] first position with a candidate in each chunk of 1024 positions
-    unsigned short *delta16; // [N]    hop.y - position, 65535 = does not fit
+    unsigned short *delta16; // [N]    jump4 - position, 65535 = does not fit
+    int32_t *jump2;        // [N]      position after the next two spans at or after each position (n_query if fewer)
+    int32_t *jump4;        // [N]      ... after the next four
     int n_hist, n_query, nwin, w, K;
     unsigned int mask;     // M - 1
     const int32_t *end_of; // [n_hist] end of the request that holds each history position; null = one request
@@ -183,7 +185,23 @@ __global__ void __launch_bounds__(kHopChunk) match_hop_kernel(MatchParams p, int
     }
     const int nx = s < N ? s + p.best[s].x : N;
     p.hop[i] = make_int2(s, nx);
-    const int dlt = nx - i;
+}
+
+// pointer doubling over "the position after the span at or after i": two spans, then four; the chain walk then
+// takes one dependent step per FOUR selected spans
+__global__ void match_jump2_kernel(MatchParams p) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.n_query) return;
+    const int a = p.hop[i].y;
+    p.jump2[i] = a < p.n_query ? p.hop[a].y : p.n_query;
+}
+__global__ void match_jump4_kernel(MatchParams p) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.n_query) return;
+    const int a = p.jump2[i];
+    const int b = a < p.n_query ? p.jump2[a] : p.n_query;
+    p.jump4[i] = b;
+    const int dlt = b - i;
     p.delta16[i] = (unsigned short)(dlt < 65535 ? dlt : 65535);
 }
 
@@ -214,9 +232,9 @@ __global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p, int w
         if (tid == 0) {
             int n = s_nspans, pos = wbeg;
             while (pos < wend) {
-                p.spans_ws[n++].q_start = pos;
+                p.spans_ws[n++].q_start = pos;          // start of a group of (up to) four spans
                 const int dlt = s_delta[pos - wbeg];
-                pos = dlt == 65535 ? p.hop[pos].y : pos + dlt;
+                pos = dlt == 65535 ? p.jump4[pos] : pos + dlt;
             }
             s_nspans = n;
             s_pos = pos;
@@ -224,26 +242,33 @@ __global__ void __launch_bounds__(1024) match_select_kernel(MatchParams p, int w
         __syncthreads();
     }
     if (tid == 0) {
-        // the last visited position may have no candidate at or after it: then it starts no span
-        int n = s_nspans;
-        if (n > 0 && p.hop[p.spans_ws[n - 1].q_start].x >= N) n--;
-        *p.n_spans = n;
+        p.chunk_first[0] = s_nspans;   // the suffix scan is done with this array: it now carries the group count
+        *p.n_spans = 0;                // the expansion of the last group sets the real count
     }
 }
 
-// (3) grid-wide: every visited position becomes a span (three dependent lookups), which a warp expands to rows
+// (3) grid-wide: a warp per group walks its (up to) four spans -- three dependent lookups each -- and expands them
+// to rows; only the last group can hold fewer than four, and its warp sets the span count
 __global__ void match_expand_kernel(MatchParams p) {
-    const int ns = *p.n_spans;
+    const int N = p.n_query;
+    const int ng = p.chunk_first[0];
     const int warps = (gridDim.x * blockDim.x) >> 5;
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    for (int sidx = gw; sidx < ns; sidx += warps) {
-        const int2 h = p.hop[p.spans_ws[sidx].q_start];
-        rac_span sp;
-        sp.q_start = h.x;
-        sp.len = h.y - h.x;
-        sp.h_start = p.best[h.x].y;
-        if (lane == 0 && p.spans_out) p.spans_out[sidx] = sp;
-        for (int m = lane; m < sp.len; m += 32) p.ref_row[sp.q_start + m] = sp.h_start + m;
+    for (int g = gw; g < ng; g += warps) {
+        int pos = p.spans_ws[g].q_start;
+        int m = 0;
+        for (; m < 4 && pos < N; m++) {
+            const int2 h = p.hop[pos];
+            if (h.x >= N) break;               // no candidate at or after pos: the chain ends
+            rac_span sp;
+            sp.q_start = h.x;
+            sp.len = h.y - h.x;
+            sp.h_start = p.best[h.x].y;
+            if (lane == 0 && p.spans_out) p.spans_out[4 * g + m] = sp;
+            for (int q = lane; q < sp.len; q += 32) p.ref_row[sp.q_start + q] = sp.h_start + q;
+            pos = h.y;
+        }
+        if (g == ng - 1 && lane == 0) *p.n_spans = 4 * g + m;
     }
 }
 
@@ -414,11 +439,14 @@ __global__ void fill2_i32_kernel(int32_t *a, long long na, int32_t va, int32_t *
 
 static size_t align16(size_t v) { return (v + 15) / 16 * 16; }
 
-// the four launches of the selection (suffix scan grid-wide, chain walk in one CTA, expansion grid-wide)
+// the six launches of the selection (suffix scan and pointer doubling grid-wide, chain walk in one CTA, expansion
+// grid-wide)
 static int launch_selection(const MatchParams &p, cudaStream_t st) {
     const int nchunks = (p.n_query + kHopChunk - 1) / kHopChunk;
     match_chunk_first_kernel<<<nchunks, kHopChunk, 0, st>>>(p);
     match_hop_kernel<<<nchunks, kHopChunk, 0, st>>>(p, nchunks);
+    match_jump2_kernel<<<(p.n_query + 255) / 256, 256, 0, st>>>(p);
+    match_jump4_kernel<<<(p.n_query + 255) / 256, 256, 0, st>>>(p);
     const int window = p.n_query < kWalkWindow ? p.n_query : kWalkWindow;
     const size_t dyn = ((size_t)window * 2 + 15) / 16 * 16;
     if (dyn > 48 * 1024 &&
@@ -432,7 +460,7 @@ static int launch_selection(const MatchParams &p, cudaStream_t st) {
 
 
 struct MatchLayout {
-    size_t rep, top, slot_of, best, hop, spans, chunk_first, delta16, total;
+    size_t rep, top, slot_of, best, hop, spans, chunk_first, delta16, jump2, jump4, total;
     unsigned int M;
 };
 static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
@@ -449,6 +477,8 @@ static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
     L.spans = o;    o = align16(o + (size_t)(n_query + 1) * sizeof(rac_span));
     L.chunk_first = o; o = align16(o + ((size_t)(n_query > 0 ? n_query : 1) / kHopChunk + 1) * 4);
     L.delta16 = o;  o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 2);
+    L.jump2 = o;    o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 4);
+    L.jump4 = o;    o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 4);
     L.total = o;
     return L;
 }
@@ -518,6 +548,8 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     p.spans_ws = reinterpret_cast<rac_span *>(ws + L.spans);
     p.chunk_first = reinterpret_cast<int32_t *>(ws + L.chunk_first);
     p.delta16 = reinterpret_cast<unsigned short *>(ws + L.delta16);
+    p.jump2 = reinterpret_cast<int32_t *>(ws + L.jump2);
+    p.jump4 = reinterpret_cast<int32_t *>(ws + L.jump4);
     p.n_hist = (int)n_hist;
     p.n_query = (int)n_query;
     p.nwin = (int)(n_hist - min_ngram + 1 > 0 ? n_hist - min_ngram + 1 : 0);
@@ -600,7 +632,7 @@ IndexLayout index_layout(const rac_index_cfg *c) {
     return L;
 }
 struct QueryLayout {
-    size_t best, hop, spans, chunk_first, delta16, trep, tfirst, total;
+    size_t best, hop, spans, chunk_first, delta16, jump2, jump4, trep, tfirst, total;
     unsigned int Mq;
 };
 QueryLayout query_layout(long long n_query) {
@@ -615,6 +647,8 @@ QueryLayout query_layout(long long n_query) {
     L.spans = o;   o = align16(o + (n + 1) * sizeof(rac_span));
     L.chunk_first = o; o = align16(o + (n / kHopChunk + 1) * 4);
     L.delta16 = o; o = align16(o + n * 2);
+    L.jump2 = o;   o = align16(o + n * 4);
+    L.jump4 = o;   o = align16(o + n * 4);
     L.trep = o;    o = align16(o + (size_t)M * 4);
     L.tfirst = o;  o = align16(o + (size_t)M * 4);
     L.total = o;
@@ -713,6 +747,8 @@ int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_by
     p.spans_ws = reinterpret_cast<rac_span *>(ws + Q.spans);
     p.chunk_first = reinterpret_cast<int32_t *>(ws + Q.chunk_first);
     p.delta16 = reinterpret_cast<unsigned short *>(ws + Q.delta16);
+    p.jump2 = reinterpret_cast<int32_t *>(ws + Q.jump2);
+    p.jump4 = reinterpret_cast<int32_t *>(ws + Q.jump4);
     p.n_hist = (int)n_hist;
     p.n_query = (int)n_query;
     p.nwin = (int)(n_hist - cfg->min_ngram + 1 > 0 ? n_hist - cfg->min_ngram + 1 : 0);
