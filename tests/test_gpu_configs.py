@@ -368,3 +368,60 @@ def test_config4_tokens_through_the_persistent_index(env):
     assert ns == len(o_sp) and np.array_equal(spans[:ns].cpu().numpy(), o_sp)
     assert np.array_equal(rows.cpu().numpy(), o_rr)
     print(f"index, 64 requests: {ns} spans, covered {((o_rr >= 0) & (o_rr < H)).mean():.3f}, intra {(o_rr >= H).mean():.3f}")
+
+
+def test_whole_step_replays_from_a_cuda_graph(env):
+    """Nothing on the path synchronises, allocates or reads a result back, so one step (retrieval, uplink encode with
+    the sender's reconstruction, receiver reconstruction, downlink encode, reconstruction) can be captured once and
+    replayed: the replay leaves the same bytes as the eager calls."""
+    s, rac, dev = env.synth, env.rac, env.dev
+    d, g, bits, k, T, H = 1024, 128, 4, 8, 3000, 8000
+    wl = s.span_workload(H, T, seed=31, gap_max=100)
+    hist, query = torch.from_numpy(wl.hist).to(dev), torch.from_numpy(wl.query).to(dev)
+    gen = s.generator(31, dev)
+    scale = s.channel_scale(d, 31, dev)
+    Hs = s.activations(H, d, scale, gen)
+    X = s.affine_noisy_target(Hs, torch.from_numpy(wl.planted_row), g, gen, scale)
+    Y = s.drifted_state(X, gen)
+    cfg = rac.CodecCfg(d, g, bits, k)
+    rec = rac.rac_record_bytes(cfg)
+    nb = rac.rac_match_workspace_bytes(H, T, 8)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    ews = torch.empty(nws, dtype=torch.uint8, device=dev)
+    step = torch.full((2, d), 0.05, dtype=torch.float32, device=dev)
+    inv = 1.0 / step
+    out = {n: torch.zeros(sz, dtype=dt, device=dev) for n, sz, dt in [
+        ("rows", T, torch.int32), ("n_spans", 1, torch.int32), ("pay_up", T * rec, torch.uint8),
+        ("pay_dn", T * rec, torch.uint8), ("status", 1, torch.int32)]}
+    xs, xr, yr = torch.zeros_like(X), torch.zeros_like(X), torch.zeros_like(X)
+
+    def one_step():
+        rac.rac_match_spans(hist, H, query, T, 4, 8, out["rows"], None, out["n_spans"], ws, nb)
+        rac.rac_encode_reconstruct(cfg, X, T, Hs, H, out["rows"], None, None, step, inv, out["pay_up"], T * rec, xs, ews,
+                                   nws, out["status"])
+        rac.rac_decode_reconstruct(cfg, out["pay_up"], T, Hs, H, out["rows"], None, None, step, xr, out["status"])
+        rac.rac_encode(cfg, Y, T, xr, T, None, None, None, step, inv, out["pay_dn"], T * rec, ews, nws, out["status"])
+        rac.rac_decode_reconstruct(cfg, out["pay_dn"], T, xr, T, None, None, None, step, yr, out["status"])
+
+    one_step()
+    torch.cuda.synchronize()
+    want = {n: t.clone() for n, t in out.items()}
+    want_x, want_y = xr.clone(), yr.clone()
+    assert int(out["status"].item()) == 0 and int(out["n_spans"].item()) > 3 and torch.equal(xs, xr)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            one_step()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        for t in list(out.values()) + [xs, xr, yr]:
+            t.fill_(7)
+        graph.replay()
+        torch.cuda.synchronize()
+        # the status word is only ever ORed into: it was filled with 7 above
+        for n in ("rows", "n_spans", "pay_up", "pay_dn"):
+            assert torch.equal(out[n], want[n]), n
+        assert torch.equal(xr, want_x) and torch.equal(yr, want_y) and torch.equal(xs, want_x)
