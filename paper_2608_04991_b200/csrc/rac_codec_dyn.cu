@@ -205,15 +205,48 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             }
 
             // ---- outlier mask: k_g rounds of (largest |e| of the group, lowest channel among equals).  The
-            // registers are left alone: the thread that holds the round's maximum finds the element by reading its
-            // piece of the rows in shared memory again (same operations, same bits), removes it from that slot's
-            // maximum, and the codes and x_hat of the outliers are patched after the dense pass.
+            // registers are left alone.  Every lane first finds ITS candidate -- the lowest channel that holds the
+            // lane's own maximum -- by reading that piece of the rows in shared memory again (same operations, same
+            // bits); none of this depends on the other lanes, so it overlaps the group's shuffles.  A round is then
+            // the group maximum, one ballot for the lowest lane that holds it, and that lane handing out its
+            // candidate; only the winner looks for a new candidate, and only if another round follows.  Codes and
+            // x_hat of the outliers are patched after the dense pass.
             if (KG) {
                 uint32_t taken = 0;  // channel order within the slab
+                float mloc, cval, cnm;
+                int cq, ck;
+                auto find = [&]() {
+                    mloc = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
+                    // lowest piece whose maximum is the lane's maximum; piece q sits in slot (q - rot) & 3
+                    float sp[4] = {sm[0], sm[1], sm[2], sm[3]};
+                    rot_right4f(sp, rot);
+                    const int q = sp[0] == mloc ? 0 : sp[1] == mloc ? 1 : sp[2] == mloc ? 2 : 3;
+                    const uint32_t pa = (uint32_t)(tid * 64 + q * 16);
+                    const uint4 xw = lds128(xs + pa);
+                    const uint32_t xws[4] = {xw.x, xw.y, xw.z, xw.w};
+                    u64 rr[4] = {0ull, 0ull, 0ull, 0ull};
+                    if (has_ref) load_ref_slot(rs + pa, p.gain, p.bias, (int)(pa >> 1), rr);
+                    float ev[8];
+#pragma unroll
+                    for (int i = 0; i < 4; i++) unpack2(psub(bf16x2_to_p(xws[i]), pfma(a2, rr[i], b2)), ev[2 * i], ev[2 * i + 1]);
+                    uint32_t tq = (taken >> (8 * q)) & 0xffu;
+                    uint32_t eq = 0;
+#pragma unroll
+                    for (int k = 0; k < 8; k++) eq |= (fabsf(ev[k]) == mloc) ? (1u << k) : 0u;
+                    eq &= ~tq;
+                    const int k = eq ? __ffs(eq) - 1 : 0;   // eq == 0 only with NaNs around
+                    float val = ev[0];
+#pragma unroll
+                    for (int kk = 1; kk < 8; kk++) val = (kk == k) ? ev[kk] : val;
+                    cnm = abs_max8(ev, tq | (1u << k));     // E^d = E - O for this slot's maximum
+                    cq = q;
+                    ck = k;
+                    cval = val;
+                };
+                find();
 #pragma unroll
                 for (int n = 0; n < KG; n++) {
                     if (n < p.kg) {
-                        const float mloc = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
                         float gm = mloc;
 #pragma unroll
                         for (int o = 1; o < 8; o <<= 1)
@@ -222,35 +255,13 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                         const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);   // gb == 0 only with NaNs around
                         uint32_t word = 0;
                         if (lane == owner) {
-                            // lowest piece whose maximum is the round's maximum; piece q sits in slot (q - rot) & 3
-                            float sp[4] = {sm[0], sm[1], sm[2], sm[3]};
-                            rot_right4f(sp, rot);
-                            const int q = sp[0] == gm ? 0 : sp[1] == gm ? 1 : sp[2] == gm ? 2 : 3;
-                            const uint32_t pa = (uint32_t)(tid * 64 + q * 16);
-                            const uint4 xw = lds128(xs + pa);
-                            const uint32_t xws[4] = {xw.x, xw.y, xw.z, xw.w};
-                            u64 rr[4] = {0ull, 0ull, 0ull, 0ull};
-                            if (has_ref) load_ref_slot(rs + pa, p.gain, p.bias, (int)(pa >> 1), rr);
-                            float ev[8];
-#pragma unroll
-                            for (int i = 0; i < 4; i++) unpack2(psub(bf16x2_to_p(xws[i]), pfma(a2, rr[i], b2)), ev[2 * i], ev[2 * i + 1]);
-                            uint32_t tq = (taken >> (8 * q)) & 0xffu;
-                            uint32_t eq = 0;
-#pragma unroll
-                            for (int k = 0; k < 8; k++) eq |= (fabsf(ev[k]) == gm) ? (1u << k) : 0u;
-                            eq &= ~tq;
-                            const int k = eq ? __ffs(eq) - 1 : 0;
-                            float val = ev[0];
-#pragma unroll
-                            for (int kk = 1; kk < 8; kk++) val = (kk == k) ? ev[kk] : val;
-                            tq |= 1u << k;
-                            taken |= 1u << (8 * q + k);
-                            const float nm = abs_max8(ev, tq);          // E^d = E - O for this slot's maximum
-                            const int js = (q - rot) & 3;
-#pragma unroll
-                            for (int j = 0; j < 4; j++) sm[j] = (j == js) ? nm : sm[j];
-                            word = (uint32_t)((lane - qbase) * 32 + 8 * q + k) | (float_to_half_bits_sat(val) << 16);
+                            word = (uint32_t)((lane - qbase) * 32 + 8 * cq + ck) | (float_to_half_bits_sat(cval) << 16);
                             own |= 1u << n;
+                            taken |= 1u << (8 * cq + ck);
+                            const int js = (cq - rot) & 3;
+#pragma unroll
+                            for (int j = 0; j < 4; j++) sm[j] = (j == js) ? cnm : sm[j];
+                            if (n + 1 < p.kg) find();
                         }
                         sel[n] = __shfl_sync(group_mask, word, owner);
                     }
