@@ -211,7 +211,12 @@ int rac_spans_to_rows(const rac_span *spans, const int32_t *n_spans, int64_t n_q
  *   ref_gain, ref_bias  binary16[d], both or neither: the reference row is first mapped per channel to
  *                                bf16(gain*r + bias) (stand-in for the decode predictor of Eq. 5)
  *   step, inv_step  float[2,d]   quantiser step and its reciprocal per channel; row 0 for tokens with a
- *                                reference, row 1 for direct tokens; step 0 means "code 0"
+ *                                reference, row 1 for direct tokens; step 0 means "code 0".  Steps are meant to
+ *                                be binary16-representable values held as float (what rac_calibrate_steps
+ *                                writes): code*step is then exact in binary32.  Every reconstruction in the
+ *                                library evaluates fma(code, step, alpha*r + beta), so sender and receiver agree
+ *                                bit for bit for ANY table; with a step that is not binary16-representable the
+ *                                result can differ in its last bf16 bit from (alpha*r + beta) + round(code*step).
  *   payload   >= T*record bytes, 16-byte aligned; payload_cap is its capacity
  *   workspace >= rac_encode_workspace_bytes(cfg, T) bytes of scratch, 16-byte aligned (0 bytes, and NULL
  *             allowed, when cfg->topk == 0).  With outliers the call is two launches: the streaming pass leaves

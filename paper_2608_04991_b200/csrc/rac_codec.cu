@@ -411,9 +411,10 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                         bits8[2 * i + 1] = __float_as_uint(t1);
                         unpack2(e, ev[2 * i], ev[2 * i + 1]);
                         if (XHAT) {
-                            // Eq. 9 with the code just chosen: x_hat = bf16((alpha*r + beta) + q*step)
+                            // Eq. 9 with the code just chosen: x_hat = bf16(fma(q, step, alpha*r + beta)); a binary16-valued
+                            // step makes q*step exact, so the fused form and (alpha*r + beta) + q*step are the same bits
                             float x0, x1;
-                            unpack2(padd(rt, pmul(psub(tt, magic2), st2[i])), x0, x1);
+                            unpack2(pfma(psub(tt, magic2), st2[i], rt), x0, x1);
                             xh[i] = f2_to_bf16x2(x0, x1);
                         }
                     }
@@ -437,7 +438,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                         unpack2(e, ev[2 * i], ev[2 * i + 1]);
                         if (XHAT) {
                             float x0, x1;
-                            unpack2(padd(rt, pmul(psub(tt, magic2), st2[i])), x0, x1);
+                            unpack2(pfma(psub(tt, magic2), st2[i], rt), x0, x1);
                             xh[i] = f2_to_bf16x2(x0, x1);
                         }
                     }
@@ -937,9 +938,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
                     // exact integer -> binary32 without a convert: 2^23 + (code + H), minus (2^23 + H)
                     const float q0 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i))) & cmask));
                     const float q1 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i + 1))) & cmask));
-                    const u64 eh = pmul(psub(pack2(q0, q1), base2), st2[i]);
                     float x0, x1;
-                    unpack2(padd(pfma(a2, r2[i], b2), eh), x0, x1);
+                    unpack2(pfma(psub(pack2(q0, q1), base2), st2[i], pfma(a2, r2[i], b2)), x0, x1);
                     o[i] = f2_to_bf16x2(x0, x1);
                 }
                 sts128(obs + off[j], make_uint4(o[0], o[1], o[2], o[3]));
@@ -1150,9 +1150,8 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
                 for (int i = 0; i < 4; i++) {
                     const float q0 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i))) & cmask));
                     const float q1 = __uint_as_float(0x4b000000u | ((w >> (BITS * (2 * i + 1))) & cmask));
-                    const u64 eh = pmul(psub(pack2(q0, q1), base2), st2[i]);
                     float x0, x1;
-                    unpack2(padd(pfma(a2, r2[i], b2), eh), x0, x1);
+                    unpack2(pfma(psub(pack2(q0, q1), base2), st2[i], pfma(a2, r2[i], b2)), x0, x1);
                     o[i] = f2_to_bf16x2(x0, x1);
                 }
                 sts128(os + off[j], make_uint4(o[0], o[1], o[2], o[3]));

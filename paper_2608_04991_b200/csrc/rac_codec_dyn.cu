@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                     if (XHAT) {
                         // Eq. 9 with the code just chosen: x_hat = bf16((alpha*r + beta) + q*s)
                         float x0, x1;
-                        unpack2(padd(pfma(a2, r2[4 * j + i], b2), pmul(psub(tt, magic2), s2)), x0, x1);
+                        unpack2(pfma(psub(tt, magic2), s2, pfma(a2, r2[4 * j + i], b2)), x0, x1);
                         xh[i] = f2_to_bf16x2(x0, x1);
                     }
                 }
@@ -576,9 +576,8 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
                     const uint32_t w1 = (f1 < FPW) ? lo[j] : hi[j];
                     const float q0 = __uint_as_float(0x4b000000u | ((w0 >> (BITS * (f0 % FPW))) & cmask));
                     const float q1 = __uint_as_float(0x4b000000u | ((w1 >> (BITS * (f1 % FPW))) & cmask));
-                    const u64 eh = pmul(psub(pack2(q0, q1), base2), s2);
                     float x0, x1;
-                    unpack2(padd(pfma(a2, r2[i], b2), eh), x0, x1);
+                    unpack2(pfma(psub(pack2(q0, q1), base2), s2, pfma(a2, r2[i], b2)), x0, x1);
                     o[i] = f2_to_bf16x2(x0, x1);
                 }
                 sts128(obs + off[j], make_uint4(o[0], o[1], o[2], o[3]));

@@ -172,6 +172,32 @@ def span_workload(n_hist: int, n_query: int, seed: int, gap_max: int = 176,
     return TokenWorkload(hist, query, planted, float((planted >= 0).mean()))
 
 
+def request_stream(n_req: int, tokens: int, seed: int, gap_max: int = 112, len_lo: int = 8,
+                   len_hi: int = 256) -> list:
+    """``n_req`` prompts of ``tokens`` ids each: the first is fresh Zipf text, every later one alternates fresh
+    gaps U{0..gap_max} with copies of spans U{len_lo..len_hi} taken from inside ONE earlier prompt (multi-turn
+    traffic: shared system prompts, quoted context).  Returns a list of int32 arrays."""
+    rng = np.random.default_rng([BASE_SEED, seed, 11])
+    out = [zipf_tokens(tokens, rng)]
+    for _ in range(1, n_req):
+        q = np.empty(tokens, np.int32)
+        i = 0
+        while i < tokens:
+            gap = min(int(rng.integers(0, gap_max + 1)), tokens - i)
+            if gap:
+                q[i:i + gap] = zipf_tokens(gap, rng)
+                i += gap
+            if i >= tokens:
+                break
+            src = out[int(rng.integers(0, len(out)))]
+            L = min(int(rng.integers(len_lo, len_hi + 1)), tokens - i, src.size)
+            j = int(rng.integers(0, src.size - L + 1))
+            q[i:i + L] = src[j:j + L]
+            i += L
+        out.append(q)
+    return out
+
+
 # ----------------------------------------------------------------- bit views
 def bf16_bits(x: torch.Tensor) -> np.ndarray:
     """bf16 tensor -> numpy uint16 bit patterns (host copy)."""

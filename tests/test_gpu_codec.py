@@ -519,3 +519,31 @@ def test_static_random_configurations(env):
             env.P.round_trip_case(cfg, X, ref_base=R, step=step, inv_step=inv, **kw)
         except AssertionError as e:
             raise AssertionError(f"{cfg!r} T={T} mode={mode}: {e}") from e
+
+
+@pytest.mark.parametrize("k", [0, 8])
+def test_tables_that_are_not_binary16_valued(env, k, monkeypatch):
+    """Steps that binary16 cannot hold make code*step inexact in binary32.  Every reconstruction in the library takes
+    fma(code, step, alpha*r + beta): the sender's pass, the streaming reconstruction and the one with a CTA barrier
+    give the same bits, and the two-rounding evaluation of the oracle is at most one bf16 step away, rarely."""
+    d, g, bits, T = 2048, 128, 4, 600
+    X, R, cal, calr = prefill_inputs(env, T, d, g, seed=61)
+    rng = np.random.default_rng(61)
+    step = (0.03 + 0.02 * rng.random((2, d))).astype(np.float32)        # 24 significant bits
+    assert np.any(step.astype(np.float16).astype(np.float32) != step)
+    inv = (np.float32(1) / step).astype(np.float32)
+    cfg = env.rac.CodecCfg(d, g, bits, k)
+    P, dev = env.P, env.dev
+    pay, xs, st = P.gpu_encode_reconstruct(cfg, X, R, None, None, None, P.to_dev(step, dev), P.to_dev(inv, dev))
+    assert st == 0
+    xr, st = P.gpu_decode(cfg, pay, T, R, None, None, None, P.to_dev(step, dev), dev)
+    assert st == 0 and torch.equal(xs, xr)
+    monkeypatch.setenv("RAC_DEC_BARRIER", "1")
+    xb, st = P.gpu_decode(cfg, pay, T, R, None, None, None, P.to_dev(step, dev), dev)
+    assert st == 0 and torch.equal(xb, xr)
+    o = env.orc.reconstruct(d, g, bits, k, pay, T, ref_base=env.synth.bf16_bits(R), step=step)
+    got = env.synth.bf16_bits(xr)
+    diff = got != o
+    assert diff.mean() < 1e-3
+    of, gf = env.orc.bf16_to_f32(o[diff]), env.orc.bf16_to_f32(got[diff])
+    assert np.all(np.abs(of - gf) <= np.maximum(np.abs(of), np.abs(gf)) * 2.0 ** -7)
