@@ -547,3 +547,65 @@ def test_tables_that_are_not_binary16_valued(env, k, monkeypatch):
     assert diff.mean() < 1e-3
     of, gf = env.orc.bf16_to_f32(o[diff]), env.orc.bf16_to_f32(got[diff])
     assert np.all(np.abs(of - gf) <= np.maximum(np.abs(of), np.abs(gf)) * 2.0 ** -7)
+
+
+def test_random_configurations_on_stressed_inputs(env):
+    """600 seeded random cases over both quantisers with inputs pushed off the comfortable range: magnitudes 1e-3 and
+    300 times the usual, a reference equal to the token, a constant reference row, an all-zero token, values on a
+    quarter grid (exact ties everywhere); identity, direct, gathered and transformed references; 1 to 400 tokens."""
+    s, rac, dev = env.synth, env.rac, env.dev
+    master = np.random.default_rng(777)
+    done = 0
+    while done < 600:
+        rng = np.random.default_rng(int(master.integers(1 << 40)))
+        fam = rng.random() < 0.55
+        d = int(rng.choice([32, 64, 96, 256, 512, 1024, 2080, 3584, 4096, 5120, 8192]))
+        g = int(rng.choice([32, 64, 128, 256, 1024]))
+        if d % g:
+            continue
+        T = int(rng.integers(1, 400 if d <= 2080 else 120))
+        if fam:
+            cfg = rac.CodecCfg(d, g, int(rng.choice([2, 3, 4, 8])), 0, scale_mode=1,
+                               qgroup=int(rng.choice([0, 32, 64, 128, 256, d])), topk_group=int(rng.choice([0, 0, 1, 2, 3, 4])))
+            if rac.rac_record_bytes(cfg) == 0:
+                continue
+        else:
+            k = int(rng.choice([0, 1, 3, 8, 16]))
+            if k > d:
+                continue
+            cfg = rac.CodecCfg(d, g, int(rng.choice([2, 3, 4])), k)
+        done += 1
+        X, R, _, _ = prefill_inputs(env, T, d, g, seed=int(rng.integers(1 << 30)), cal_T=8)
+        kind = int(rng.integers(0, 7))
+        if kind == 1:
+            X, R = (X.float() * 1e-3).to(torch.bfloat16), (R.float() * 1e-3).to(torch.bfloat16)
+        elif kind == 2:
+            X, R = (X.float() * 300).to(torch.bfloat16), (R.float() * 300).to(torch.bfloat16)
+        elif kind == 3:
+            R = X.clone()
+        elif kind == 4:
+            R[int(rng.integers(0, T))] = 1.5
+        elif kind == 5:
+            X[int(rng.integers(0, T))] = 0
+        elif kind == 6:
+            X = torch.round(X.float() * 4).div(4).to(torch.bfloat16)
+            R = torch.round(R.float() * 4).div(4).to(torch.bfloat16)
+        mode = int(rng.integers(0, 4))
+        kw, gb, rows = {}, {}, None
+        if mode == 1:
+            rows = np.arange(T, dtype=np.int32)
+            rows[rng.random(T) < 0.4] = -1
+        elif mode == 2:
+            rows = rng.integers(0, T, T).astype(np.int32)
+        if rows is not None:
+            kw["ref_row"] = torch.from_numpy(rows).to(dev)
+        if mode == 3:
+            kw["gain"], kw["bias"] = s.predictor_gain_bias(d, int(rng.integers(100)), dev)
+            gb = dict(gain=s.f16_bits(kw["gain"]), bias=s.f16_bits(kw["bias"]))
+        if not fam:
+            kw["step"], kw["inv_step"] = env.orc.calibrate(d, g, cfg.bits, s.bf16_bits(X), ref_base=s.bf16_bits(R),
+                                                           ref_row=rows, **gb)
+        try:
+            env.P.round_trip_case(cfg, X, ref_base=R, **kw)
+        except AssertionError as e:
+            raise AssertionError(f"{cfg!r} T={T} mode={mode} kind={kind}: {e}") from e

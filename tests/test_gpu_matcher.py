@@ -245,3 +245,71 @@ def test_index_argument_checks(env):
         with pytest.raises(rac.RacError) as e:
             fn(*args)
         assert e.value.code == code
+
+
+def _random_tokens(rng, n, vocab, hist=None):
+    q = rng.integers(0, vocab, n).astype(np.int32)
+    if hist is not None and hist.size and n:
+        for _ in range(int(rng.integers(0, 6))):       # planted copies of history spans
+            L = int(rng.integers(1, min(n, hist.size, 300) + 1))
+            i, j = int(rng.integers(0, n - L + 1)), int(rng.integers(0, hist.size - L + 1))
+            q[i:i + L] = hist[j:j + L]
+    if rng.random() < 0.1 and n:
+        q[:] = q[0]                                     # one token repeated
+    return q
+
+
+def test_random_sweep_one_shot_and_index(env):
+    """2000 seeded random cases, half through the one-shot matcher and half through the persistent index with
+    random request boundaries (empty and one-token requests included) and random use of intra-sequence references:
+    vocabularies from 1 to 32000 ids, windows 1..32, 1..16 hits, sizes from 0 to a few thousand."""
+    rac, orc, dev = env.rac, env.orc, env.dev
+    master = np.random.default_rng(4711)
+    for _ in range(2000):
+        rng = np.random.default_rng(int(master.integers(1 << 40)))
+        if rng.random() < 0.5:
+            vocab = int(rng.choice([1, 2, 3, 7, 50, 1000, 32000]))
+            w, K = int(rng.choice([1, 2, 3, 4, 4, 5, 8, 16, 32])), int(rng.choice([1, 2, 3, 8, 8, 16]))
+            H = int(rng.choice([0, 1, 3, int(rng.integers(0, 6000))]))
+            N = int(rng.choice([0, 1, 2, int(rng.integers(0, 4000))]))
+            hist = _random_tokens(rng, H, vocab)
+            query = _random_tokens(rng, N, vocab, hist)
+            rr, sp, ns = gpu_match(env, hist, query, w, K)
+            o_rr, o_sp = orc.match_spans(hist, query, w, K)
+            assert ns == len(o_sp) and np.array_equal(rr, o_rr) and np.array_equal(sp, o_sp.reshape(-1, 3)), \
+                dict(vocab=vocab, w=w, K=K, H=H, N=N)
+            continue
+        vocab = int(rng.choice([2, 3, 7, 50, 1000, 32000]))
+        w, K = int(rng.choice([1, 2, 3, 4, 4, 5, 8])), int(rng.choice([1, 2, 8, 8, 16]))
+        lens = [int(rng.choice([0, 1, 2, 3, int(rng.integers(0, 1500))])) for _ in range(int(rng.integers(1, 9)))]
+        H = sum(lens)
+        cap = H + int(rng.integers(0, 100)) + 1
+        icfg = rac.IndexCfg(cap, w, K)
+        nb = rac.rac_index_bytes(icfg)
+        imem = torch.full((nb,), 0x5A, dtype=torch.uint8, device=dev)
+        htok = torch.zeros(cap, dtype=torch.int32, device=dev)
+        rac.rac_index_reset(icfg, imem, nb)
+        hist, off = np.zeros(0, np.int32), [0]
+        for L in lens:
+            req = _random_tokens(rng, L, vocab, hist)
+            if L:
+                htok[hist.size:hist.size + L] = torch.from_numpy(req).to(dev)
+            rac.rac_index_append(icfg, imem, nb, htok, hist.size, hist.size + L)
+            hist = np.concatenate([hist, req])
+            off.append(hist.size)
+        N = int(rng.choice([0, 1, int(rng.integers(0, 3000))]))
+        intra = bool(rng.random() < 0.5)
+        query = _random_tokens(rng, N, vocab, hist)
+        q = torch.from_numpy(query).to(dev)
+        rows = torch.full((N + 8,), 12345, dtype=torch.int32, device=dev)
+        sp = torch.full((N // w + 3, 3), 777, dtype=torch.int32, device=dev)
+        ns = torch.full((1,), -5, dtype=torch.int32, device=dev)
+        nws = rac.rac_index_query_workspace_bytes(N)
+        ws = torch.full((max(nws, 16),), 0x5A, dtype=torch.uint8, device=dev)
+        rac.rac_index_query(icfg, imem, nb, htok, H, q if N else None, N, intra, rows[:N] if N else None,
+                            sp[:N // w + 1], ns, ws, nws)
+        o_rr, o_sp = orc.match_spans_req(hist, off, query, w, K, intra)
+        n = int(ns.item())
+        what = dict(vocab=vocab, w=w, K=K, lens=lens, N=N, intra=intra)
+        assert n == len(o_sp) and torch.all(rows[N:] == 12345), what
+        assert np.array_equal(rows[:N].cpu().numpy(), o_rr) and np.array_equal(sp[:n].cpu().numpy(), o_sp.reshape(-1, 3)), what
