@@ -1019,7 +1019,9 @@ __host__ __device__ inline DwSmem dw_smem_layout(int d, int rec, int stages, boo
 }
 
 // KT > 0: records with per-token outliers (the output row is a row of its own behind the reference row).
-template <int BITS, int KT, bool SUB>
+// ROW1: the call can contain directly coded tokens (a row list, or no reference at all); they take their steps
+// from row 1 of the table, which this form keeps in registers as well.
+template <int BITS, int KT, bool SUB, bool ROW1>
 __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -1085,6 +1087,27 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
         st0[4 * j + 2] = pack2(s1.x, s1.y);
         st0[4 * j + 3] = pack2(s1.z, s1.w);
     }
+    // Row 1 (directly coded tokens) as packed binary16 in 16 registers, when binary16 holds every entry of the row
+    // exactly -- which is how the calibration writes them.  Otherwise those tokens read the row from memory.
+    uint32_t sh1[16];
+    bool row1_exact = ROW1;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+        if (ROW1 && valid) {
+            s0 = __ldg(reinterpret_cast<const float4 *>(p.step + d + (off[j] >> 1)));
+            s1 = __ldg(reinterpret_cast<const float4 *>(p.step + d + (off[j] >> 1) + 4));
+        }
+        const float v[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            const __half2 h = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+            const float2 back = __half22float2(h);
+            row1_exact = row1_exact && back.x == v[2 * i] && back.y == v[2 * i + 1];
+            sh1[4 * j + i] = *reinterpret_cast<const uint32_t *>(&h);
+        }
+    }
+    if (ROW1) row1_exact = __syncthreads_and(row1_exact) != 0;
     const u64 base2 = pack2(kBase, kBase);
 
     int stage = 0, duty = 0;
@@ -1139,6 +1162,12 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
                 if (has_ref) {
 #pragma unroll
                     for (int i = 0; i < 4; i++) st2[i] = st0[4 * j + i];
+                } else if (ROW1 && row1_exact) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&sh1[4 * j + i]));
+                        st2[i] = pack2(f.x, f.y);
+                    }
                 } else {
                     const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c));
                     const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.step + d + c + 4));
@@ -1323,9 +1352,11 @@ static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream)
     const int wstages = pick_stages(g.d, g.nthreads > 128 ? 3 : 2);
     DwSmem LW = dw_smem_layout(g.d, g.rec, wstages, kt > 0);
     if (ws) p.stages = wstages;
+    const bool row1 = p.ref_row != nullptr || p.ref_base == nullptr;   // else every token has its reference row
 #define RAC_DEC(B, K)                                                                            \
     (sub ? launch_persistent(decode_kernel<B, K, true>, p, g.nthreads, L.total, p.T, stream)    \
-     : ws ? launch_persistent(decode_ws_kernel<B, K, false>, p, g.nthreads, LW.total, p.T, stream) \
+     : ws ? (row1 ? launch_persistent(decode_ws_kernel<B, K, false, true>, p, g.nthreads, LW.total, p.T, stream)   \
+                  : launch_persistent(decode_ws_kernel<B, K, false, false>, p, g.nthreads, LW.total, p.T, stream)) \
          : launch_persistent(decode_kernel<B, K, false>, p, g.nthreads, L.total, p.T, stream))
     switch (g.bits * 100 + kt) {
         case 400: return RAC_DEC(4, 0);

@@ -534,14 +534,31 @@ def test_tables_that_are_not_binary16_valued(env, k, monkeypatch):
     inv = (np.float32(1) / step).astype(np.float32)
     cfg = env.rac.CodecCfg(d, g, bits, k)
     P, dev = env.P, env.dev
-    pay, xs, st = P.gpu_encode_reconstruct(cfg, X, R, None, None, None, P.to_dev(step, dev), P.to_dev(inv, dev))
+    # a third of the tokens coded directly: they take row 1 of the table, which the streaming reconstruction keeps
+    # as packed binary16 only when that is exact -- here it is not, so it has to read the row from memory
+    rows_np = np.arange(T, dtype=np.int32)
+    rows_np[rng.random(T) < 0.33] = -1
+    rows = torch.from_numpy(rows_np).to(dev)
+    pay, xs, st = P.gpu_encode_reconstruct(cfg, X, R, rows, None, None, P.to_dev(step, dev), P.to_dev(inv, dev))
     assert st == 0
-    xr, st = P.gpu_decode(cfg, pay, T, R, None, None, None, P.to_dev(step, dev), dev)
+    xr, st = P.gpu_decode(cfg, pay, T, R, rows, None, None, P.to_dev(step, dev), dev)
     assert st == 0 and torch.equal(xs, xr)
     monkeypatch.setenv("RAC_DEC_BARRIER", "1")
-    xb, st = P.gpu_decode(cfg, pay, T, R, None, None, None, P.to_dev(step, dev), dev)
+    xb, st = P.gpu_decode(cfg, pay, T, R, rows, None, None, P.to_dev(step, dev), dev)
     assert st == 0 and torch.equal(xb, xr)
-    o = env.orc.reconstruct(d, g, bits, k, pay, T, ref_base=env.synth.bf16_bits(R), step=step)
+    monkeypatch.delenv("RAC_DEC_BARRIER")
+    # row 0 exact in binary16, row 1 not, and the other way round: the two rows are handled independently
+    for keep in (0, 1):
+        mixed = step.copy()
+        mixed[keep] = mixed[keep].astype(np.float16).astype(np.float32)
+        minv = (np.float32(1) / mixed).astype(np.float32)
+        pm, xm, st = P.gpu_encode_reconstruct(cfg, X, R, rows, None, None, P.to_dev(mixed, dev), P.to_dev(minv, dev))
+        xd, st2 = P.gpu_decode(cfg, pm, T, R, rows, None, None, P.to_dev(mixed, dev), dev)
+        assert st == 0 and st2 == 0 and torch.equal(xm, xd)
+        om = env.orc.reconstruct(d, g, bits, k, pm, T, ref_base=env.synth.bf16_bits(R), ref_row=rows_np, step=mixed)
+        exact_tokens = (rows_np >= 0) if keep == 0 else (rows_np < 0)
+        assert np.array_equal(env.synth.bf16_bits(xd)[exact_tokens], om[exact_tokens])
+    o = env.orc.reconstruct(d, g, bits, k, pay, T, ref_base=env.synth.bf16_bits(R), ref_row=rows_np, step=step)
     got = env.synth.bf16_bits(xr)
     diff = got != o
     assert diff.mean() < 1e-3
