@@ -99,6 +99,19 @@ const char *rac_strerror(int err);
 size_t rac_record_bytes(const rac_codec_cfg *cfg);
 size_t rac_payload_bytes(const rac_codec_cfg *cfg, int64_t T);
 
+/* Header of a serialised payload: 64 bytes that say how to read the T records behind them (the record format is
+ * this library's own: the paper fixes only two 4-bit values per byte, per-group scales and in-group offsets with
+ * binary16 values, Sec. IV-C).  HOST memory, host work only: nothing is launched.
+ *   bytes  0..3   "RACP"          4..5  version (1)      6..7  header size (64)
+ *          8..15  T (int64)       16..51  d, group, bits, topk, coef_fmt, scale_mode, flags, qgroup, topk_group
+ *                                         (int32 each, qgroup as given)
+ *         52..55  record bytes    56..59  sum of the fourteen 32-bit words before it, modulo 2^32    60..63  zero
+ * All little endian.  rac_header_write returns RAC_EINVAL for an invalid configuration or T < 0.  rac_header_parse
+ * returns RAC_EINVAL when magic, version, size, checksum or record size do not fit, and leaves the outputs alone. */
+#define RAC_HEADER_BYTES 64
+int rac_header_write(const rac_codec_cfg *cfg, int64_t T, void *header /* host, 64 bytes */);
+int rac_header_parse(const void *header /* host, 64 bytes */, rac_codec_cfg *cfg_out, int64_t *T_out);
+
 /* ---------------------------------------------------------------------------------------------
  * Span retrieval for prefill uplinks (Sec. IV-B.1, Eq. 3).
  *

@@ -27,7 +27,7 @@ STATUS_TIMEOUT = 8
 STATUS_OUTLIER_RANGE = 16
 
 EXPORTS = [
-    "rac_version", "rac_strerror", "rac_record_bytes", "rac_payload_bytes",
+    "rac_version", "rac_strerror", "rac_record_bytes", "rac_payload_bytes", "rac_header_write", "rac_header_parse",
     "rac_match_workspace_bytes", "rac_match_spans", "rac_spans_to_rows",
     "rac_match_spans_static",
     "rac_index_bytes", "rac_index_reset", "rac_index_append", "rac_index_query_workspace_bytes", "rac_index_query",
@@ -90,6 +90,10 @@ def load() -> C.CDLL:
     l.rac_record_bytes.argtypes = [cfgp]
     l.rac_payload_bytes.restype = sz
     l.rac_payload_bytes.argtypes = [cfgp, i64]
+    l.rac_header_write.restype = C.c_int
+    l.rac_header_write.argtypes = [cfgp, i64, vp]
+    l.rac_header_parse.restype = C.c_int
+    l.rac_header_parse.argtypes = [vp, cfgp, C.POINTER(i64)]
     l.rac_match_workspace_bytes.restype = sz
     l.rac_match_workspace_bytes.argtypes = [i64, i64, i32]
     l.rac_match_spans.restype = C.c_int
@@ -192,6 +196,26 @@ def rac_record_bytes(cfg: CodecCfg) -> int:
 
 def rac_payload_bytes(cfg: CodecCfg, T: int) -> int:
     return int(load().rac_payload_bytes(C.byref(cfg), int(T)))
+
+
+HEADER_BYTES = 64
+
+
+def rac_header_write(cfg: CodecCfg, T: int) -> bytes:
+    """The 64-byte header of a serialised payload of T records (host work only)."""
+    buf = C.create_string_buffer(HEADER_BYTES)
+    _check("rac_header_write", load().rac_header_write(C.byref(cfg), int(T), buf))
+    return buf.raw
+
+
+def rac_header_parse(header: bytes):
+    """(CodecCfg, T) of a header written by rac_header_write; raises RacError when it does not check out."""
+    if len(header) < HEADER_BYTES:
+        raise ValueError("a header is 64 bytes")
+    buf = C.create_string_buffer(bytes(header[:HEADER_BYTES]), HEADER_BYTES)
+    cfg, T = CodecCfg(64, 32, 4, 0), C.c_int64(0)
+    _check("rac_header_parse", load().rac_header_parse(buf, C.byref(cfg), C.byref(T)))
+    return cfg, int(T.value)
 
 
 def rac_match_workspace_bytes(n_hist: int, n_query: int, max_hits: int) -> int:

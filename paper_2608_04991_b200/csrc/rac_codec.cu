@@ -20,6 +20,8 @@
 // segment_fit_kernel + seg_of_kernel (Eq. 6 over several fitting positions), split_waves_kernel (tokens that
 // reference the same prompt go second), recon_error_kernel (error of a sender-path run).  The kernels of the
 // per-group-scale quantiser (Eq. 8 as printed) live in rac_codec_dyn.cu; this file holds the C ABI of both.
+#include <cstring>
+
 #include "rac_codec_dev.cuh"
 
 namespace rac {
@@ -1631,6 +1633,63 @@ size_t rac_record_bytes(const rac_codec_cfg *cfg) {
 size_t rac_payload_bytes(const rac_codec_cfg *cfg, int64_t T) {
     if (T < 0) return 0;
     return rac_record_bytes(cfg) * (size_t)T;
+}
+
+// ---- header of a serialised payload (host only)
+static uint32_t header_sum(const unsigned char *h) {
+    uint32_t sum = 0;
+    for (int i = 0; i < 14; i++) {
+        uint32_t w;
+        memcpy(&w, h + 4 * i, 4);
+        sum += w;
+    }
+    return sum;
+}
+
+int rac_header_write(const rac_codec_cfg *cfg, int64_t T, void *header) {
+    const size_t rec = rac_record_bytes(cfg);
+    if (!header || rec == 0 || T < 0) return RAC_EINVAL;
+    unsigned char h[RAC_HEADER_BYTES];
+    memset(h, 0, sizeof h);
+    memcpy(h, "RACP", 4);
+    const uint16_t version = 1, size = RAC_HEADER_BYTES;
+    memcpy(h + 4, &version, 2);
+    memcpy(h + 6, &size, 2);
+    memcpy(h + 8, &T, 8);
+    const int32_t f[9] = {cfg->d, cfg->group, cfg->bits, cfg->topk, cfg->coef_fmt, cfg->scale_mode, cfg->flags,
+                          cfg->qgroup, cfg->topk_group};
+    memcpy(h + 16, f, sizeof f);
+    const uint32_t rec32 = (uint32_t)rec;
+    memcpy(h + 52, &rec32, 4);
+    const uint32_t sum = header_sum(h);
+    memcpy(h + 56, &sum, 4);
+    memcpy(header, h, sizeof h);
+    return RAC_OK;
+}
+
+int rac_header_parse(const void *header, rac_codec_cfg *cfg_out, int64_t *T_out) {
+    if (!header || !cfg_out || !T_out) return RAC_EINVAL;
+    const unsigned char *h = static_cast<const unsigned char *>(header);
+    uint16_t version, size;
+    uint32_t rec32, sum, tail;
+    int64_t T;
+    int32_t f[9];
+    memcpy(&version, h + 4, 2);
+    memcpy(&size, h + 6, 2);
+    memcpy(&T, h + 8, 8);
+    memcpy(f, h + 16, sizeof f);
+    memcpy(&rec32, h + 52, 4);
+    memcpy(&sum, h + 56, 4);
+    memcpy(&tail, h + 60, 4);
+    if (memcmp(h, "RACP", 4) != 0 || version != 1 || size != RAC_HEADER_BYTES || tail != 0 || sum != header_sum(h)) return RAC_EINVAL;
+    rac_codec_cfg cfg;
+    cfg.d = f[0]; cfg.group = f[1]; cfg.bits = f[2]; cfg.topk = f[3]; cfg.coef_fmt = f[4]; cfg.scale_mode = f[5];
+    cfg.flags = f[6]; cfg.qgroup = f[7]; cfg.topk_group = f[8];
+    const size_t rec = rac_record_bytes(&cfg);
+    if (rec == 0 || rec != (size_t)rec32 || T < 0) return RAC_EINVAL;
+    *cfg_out = cfg;
+    *T_out = T;
+    return RAC_OK;
 }
 
 size_t rac_encode_workspace_bytes(const rac_codec_cfg *cfg, int64_t T) {

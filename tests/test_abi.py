@@ -98,3 +98,33 @@ def test_host_side_rejections_happen_before_any_launch(rac):
     assert rac.rac_strerror(-3) == "caller buffer too small"
     with pytest.raises(rac.RacError):
         rac._check("x", -1)
+
+
+def test_payload_header_round_trip_and_rejections(rac):
+    cfgs = [rac.CodecCfg(4096, 128, 4, 8), rac.CodecCfg(3584, 128, 3, 0),
+            rac.CodecCfg(5120, 128, 8, 0, scale_mode=1, qgroup=256, topk_group=2),
+            rac.CodecCfg(4096, 128, 4, 0, scale_mode=1, coef_fmt=1)]
+    for cfg in cfgs:
+        for T in (0, 1, 131072, 1 << 40):
+            h = rac.rac_header_write(cfg, T)
+            assert len(h) == rac.HEADER_BYTES == 64 and h[:4] == b"RACP"
+            got, gT = rac.rac_header_parse(h)
+            assert gT == T and bytes(got) == bytes(cfg)
+            assert int.from_bytes(h[52:56], "little") == rac.rac_record_bytes(cfg) and h[60:] == b"\0\0\0\0"
+    h = rac.rac_header_write(cfgs[0], 77)
+    for i in range(64):                                  # any single corrupted byte is noticed
+        bad = bytearray(h)
+        bad[i] ^= 0x10
+        with pytest.raises(rac.RacError) as e:
+            rac.rac_header_parse(bytes(bad))
+        assert e.value.code == -1
+    # a consistent checksum over an impossible configuration is still refused (record size is re-derived)
+    bad = bytearray(h)
+    bad[20:24] = (100).to_bytes(4, "little")             # group 100 does not divide 4096
+    bad[56:60] = (sum(int.from_bytes(bad[4 * i:4 * i + 4], "little") for i in range(14)) & 0xffffffff).to_bytes(4, "little")
+    with pytest.raises(rac.RacError):
+        rac.rac_header_parse(bytes(bad))
+    with pytest.raises(rac.RacError):
+        rac.rac_header_write(rac.CodecCfg(4096, 100, 4, 0), 5)
+    with pytest.raises(rac.RacError):
+        rac.rac_header_write(cfgs[0], -1)
