@@ -425,3 +425,53 @@ def test_whole_step_replays_from_a_cuda_graph(env):
         for n in ("rows", "n_spans", "pay_up", "pay_dn"):
             assert torch.equal(out[n], want[n]), n
         assert torch.equal(xr, want_x) and torch.equal(yr, want_y) and torch.equal(xs, want_x)
+
+
+@pytest.mark.parametrize("mode", ["static top-8", "Eq. 8, one outlier per group"])
+def test_buffers_beyond_four_gibibytes(env, mode):
+    """1.2 million tokens of 2048 channels: X, the reference and x_hat are 4.9 GB each, so token offsets pass 2^32
+    bytes and 2^31 elements, and the records of the last tokens lie beyond the first GiB of the payload.  The device
+    runs the whole size; the oracle checks the first, the last and 1500 random tokens one by one."""
+    s, rac, orc, dev, P = env.synth, env.rac, env.orc, env.dev, env.P
+    d, g, bits, T = 2048, 128, 4, 1_200_000
+    assert 2 * T * d > 2 ** 32 and T * d > 2 ** 31
+    gen = s.generator(91, dev)
+    scale = s.channel_scale(d, 91, dev)
+    X = s.activations(T, d, scale, gen)
+    R = s.affine_noisy_reference(X, g, gen)
+    if mode == "static top-8":
+        cfg, k, mk = rac.CodecCfg(d, g, bits, 8), 8, {}
+        step = torch.empty((2, d), dtype=torch.float32, device=dev)
+        inv = torch.empty_like(step)
+        nb = rac.rac_calibrate_workspace_bytes(cfg)
+        cws = torch.empty(nb, dtype=torch.uint8, device=dev)
+        st0 = torch.zeros(1, dtype=torch.int32, device=dev)
+        rac.rac_calibrate_steps(cfg, X[:2048], 2048, R, T, None, None, None, 3.0, step, inv, cws, nb, st0)
+        st_np, iv_np = step.cpu().numpy(), inv.cpu().numpy()
+    else:
+        cfg, k, mk = rac.CodecCfg(d, g, bits, 0, scale_mode=1, topk_group=1), 0, dict(scale_mode=1, topk_group=1)
+        step = inv = st_np = iv_np = None
+    rec = rac.rac_record_bytes(cfg)
+    assert T * rec > 2 ** 30
+    payload = torch.empty(T * rec, dtype=torch.uint8, device=dev)
+    xs = torch.empty_like(X)
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    ews = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rac.rac_encode_reconstruct(cfg, X, T, R, T, None, None, None, step, inv, payload, payload.numel(), xs, ews, nws, status)
+    xr = torch.empty_like(X)
+    rac.rac_decode_reconstruct(cfg, payload, T, R, T, None, None, None, step, xr, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for t0 in range(0, T, 200_000):                       # sender and receiver agree everywhere
+        assert torch.equal(xs[t0:t0 + 200_000], xr[t0:t0 + 200_000])
+    rng = np.random.default_rng(91)
+    sample = np.unique(np.concatenate([np.arange(32), np.arange(T - 32, T), rng.integers(0, T, 1500),
+                                       rng.integers(T - 100_000, T, 300)]))     # extra weight beyond 2^32 bytes
+    idx = torch.from_numpy(sample).to(dev)
+    pay_s = payload.view(T, rec)[idx].cpu().numpy().reshape(-1)
+    Xs, Rs = s.bf16_bits(X[idx]), s.bf16_bits(R[idx])
+    rep = P.compare_encode(cfg, pay_s, Xs, Rs, None, None, None, st_np, iv_np)
+    print(rep)
+    o_x = orc.reconstruct(d, g, bits, k, pay_s, sample.size, ref_base=Rs, step=st_np, nthreads=orc.max_threads(), **mk)
+    assert np.array_equal(o_x, s.bf16_bits(xr[idx]))
