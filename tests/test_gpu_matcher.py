@@ -313,3 +313,16 @@ def test_random_sweep_one_shot_and_index(env):
         what = dict(vocab=vocab, w=w, K=K, lens=lens, N=N, intra=intra)
         assert n == len(o_sp) and torch.all(rows[N:] == 12345), what
         assert np.array_equal(rows[:N].cpu().numpy(), o_rr) and np.array_equal(sp[:n].cpu().numpy(), o_sp.reshape(-1, 3)), what
+
+
+def test_two_million_token_history(env):
+    """History of 2^21 tokens, prompt of 2^19: sixteen times the benchmark's history; positions need 21 bits, the most
+    frequent windows occur hundreds of times (the K cap decides), the chain walk crosses its shared-memory window
+    several times.  Whole result against the oracle."""
+    s, orc = env.synth, env.orc
+    wl = s.span_workload(1 << 21, 1 << 19, seed=5, gap_max=112)
+    rr, sp, ns = gpu_match(env, wl.hist, wl.query, 4, 8)
+    o_rr, o_sp = orc.match_spans(wl.hist, wl.query, 4, 8)
+    assert ns == len(o_sp) > 5000
+    assert np.array_equal(rr, o_rr) and np.array_equal(sp, o_sp.reshape(-1, 3))
+    assert (rr >= 0).mean() > 0.7
