@@ -296,7 +296,10 @@ int rac_sender_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_
  * Two-wave protocol, both endpoints: call once with wave 1 (intra_base may already be given: wave 1 never reads
  * it), then with wave 2 and intra_base = X_hat of this prompt, on the same stream.  The rows a wave-2 token
  * references were written by wave 1, and no wave-2 token is referenced by anyone, so the second call reads only
- * finished rows while it writes others. */
+ * finished rows while it writes others.  That is a PRECONDITION on ref_row when it does not come from
+ * rac_index_query: an entry >= first_intra_row must name a token whose own entry is below first_intra_row.  A
+ * chain (a wave-2 token that references another wave-2 token) is not detected and makes the second call read a
+ * row while another CTA writes it. */
 int rac_split_waves(const int32_t *ref_row, int64_t T, int64_t first_intra_row, int32_t *wave1, int32_t *wave2,
                     int32_t *wave_count, void *stream);
 int rac_encode_reconstruct_list(const rac_codec_cfg *cfg, const void *X, int64_t T, const int32_t *tok_list,
