@@ -160,3 +160,83 @@ def test_list_argument_checks_and_bad_entries(env):
                                     None, 0, st)
     torch.cuda.synchronize()
     assert torch.equal(pay, before)
+
+
+def test_random_two_wave_cases(env):
+    """300 seeded random cases of the two-wave protocol with hand-made row lists: directly coded tokens, history
+    rows and references to first-wave tokens of the same prompt in random mix (no chains), both quantisers, widths
+    from 64 to 5120, references uncorrelated with the tokens (tiny slopes)."""
+    s, rac, orc, dev, P = env.synth, env.rac, env.orc, env.dev, env.P
+    master = np.random.default_rng(9090)
+    done = 0
+    while done < 300:
+        rng = np.random.default_rng(int(master.integers(1 << 40)))
+        d, g = int(rng.choice([64, 256, 1024, 2080, 4096, 5120])), int(rng.choice([32, 64, 128, 256]))
+        if d % g:
+            continue
+        if rng.random() < 0.5:
+            bits, kg, k = int(rng.choice([2, 3, 4, 8])), int(rng.choice([0, 1, 2])), 0
+            cfg, mk = rac.CodecCfg(d, g, bits, 0, scale_mode=1, topk_group=kg), dict(scale_mode=1, topk_group=kg)
+        else:
+            bits, k = int(rng.choice([2, 3, 4])), int(rng.choice([0, 3, 8]))
+            cfg, mk = rac.CodecCfg(d, g, bits, k), {}
+        if rac.rac_record_bytes(cfg) == 0:
+            continue
+        done += 1
+        n_hist, T = int(rng.integers(1, 300)), int(rng.integers(1, 250))
+        gen = s.generator(int(rng.integers(1 << 30)), dev)
+        scale = s.channel_scale(d, 5, dev)
+        Hs, X = s.activations(n_hist, d, scale, gen), s.activations(T, d, scale, gen)
+        rows = np.full(T, -1, np.int64)
+        kind = rng.random(T)
+        rows[kind < 0.4] = rng.integers(0, n_hist, int((kind < 0.4).sum()))
+        stay = np.flatnonzero(kind <= 0.75)                      # tokens of the first wave
+        for t in np.flatnonzero(kind > 0.75):
+            cand = stay[stay < t]
+            if cand.size:
+                rows[t] = n_hist + int(rng.choice(cand))
+        rows = rows.astype(np.int32)
+        w1, w2 = np.flatnonzero(rows < n_hist).astype(np.int32), np.flatnonzero(rows >= n_hist).astype(np.int32)
+        rows_d = torch.from_numpy(rows).to(dev)
+        Xb, Hb = s.bf16_bits(X), s.bf16_bits(Hs)
+        step = inv = step_d = inv_d = None
+        if cfg.scale_mode == 0:
+            step, inv = orc.calibrate(d, g, bits, Xb, ref_base=Hb, ref_row=np.where(rows < n_hist, rows, -1).astype(np.int32))
+            step_d, inv_d = P.to_dev(step, dev), P.to_dev(inv, dev)
+        rec = rac.rac_record_bytes(cfg)
+        wave1 = torch.full((T,), -9, dtype=torch.int32, device=dev)
+        wave2 = torch.full((T,), -9, dtype=torch.int32, device=dev)
+        cnt = torch.zeros(2, dtype=torch.int32, device=dev)
+        rac.rac_split_waves(rows_d, T, n_hist, wave1, wave2, cnt)
+        assert cnt.tolist() == [len(w1), len(w2)]
+        assert np.array_equal(wave1[:len(w1)].cpu().numpy(), w1) and np.array_equal(wave2[:len(w2)].cpu().numpy(), w2)
+        pay = torch.full((T * rec,), 0xA5, dtype=torch.uint8, device=dev)
+        xh = torch.full((T, d), -7.0, dtype=torch.bfloat16, device=dev)
+        st = torch.zeros(1, dtype=torch.int32, device=dev)
+        nws = rac.rac_encode_workspace_bytes(cfg, T)
+        ews = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
+        for lst, c in ((wave1, cnt[0:1]), (wave2, cnt[1:2])):
+            rac.rac_encode_reconstruct_list(cfg, X, T, lst, c, Hs, n_hist, rows_d, xh, T, None, None, step_d, inv_d, pay,
+                                            T * rec, xh, ews if nws else None, nws, st)
+        torch.cuda.synchronize()
+        what = f"{cfg!r} T={T} n_hist={n_hist}"
+        assert int(st.item()) == 0, what
+        pay_np, xh_bits = pay.cpu().numpy(), s.bf16_bits(xh)
+        try:
+            if len(w1):
+                P.compare_encode(cfg, records(pay_np, rec, w1), Xb[w1], Hb, rows[w1], None, None, step, inv)
+                o1 = orc.reconstruct(d, g, bits, k, records(pay_np, rec, w1), len(w1), ref_base=Hb, ref_row=rows[w1], step=step, **mk)
+                assert np.array_equal(o1, xh_bits[w1]), "first-wave reconstruction"
+            if len(w2):
+                joint = np.concatenate([Hb, xh_bits])
+                joint[n_hist + w2] = 0x7fc0                      # NaN where nothing may be read
+                P.compare_encode(cfg, records(pay_np, rec, w2), Xb[w2], joint, rows[w2], None, None, step, inv)
+                o2 = orc.reconstruct(d, g, bits, k, records(pay_np, rec, w2), len(w2), ref_base=joint, ref_row=rows[w2], step=step, **mk)
+                assert np.array_equal(o2, xh_bits[w2]), "second-wave reconstruction"
+        except AssertionError as e:
+            raise AssertionError(f"{what}: {e}") from e
+        xd = torch.full((T, d), 3.0, dtype=torch.bfloat16, device=dev)
+        for lst, c in ((wave1, cnt[0:1]), (wave2, cnt[1:2])):
+            rac.rac_decode_reconstruct_list(cfg, pay, T, lst, c, Hs, n_hist, rows_d, xd, T, None, None, step_d, xd, st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0 and torch.equal(xd, xh), what
