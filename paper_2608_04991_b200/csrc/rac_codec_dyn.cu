@@ -14,6 +14,8 @@
 // selection fits into the streaming pass: a group is 1 to 8 lanes of one warp, so k_g rounds of "largest
 // magnitude of the group, lowest channel among equals" need only warp shuffles.  The token-wide scale is the
 // one place where warps must meet: they exchange their maxima through shared memory and a third mbarrier.
+#include <type_traits>
+
 #include "rac_codec_dev.cuh"
 
 namespace rac {
@@ -314,31 +316,46 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             if (qtok ? tid == 0 : (lane & (p.lpq - 1)) == 0)
                 reinterpret_cast<unsigned short *>(rec + p.scale_off)[jq] = (unsigned short)s16;
 
+            // No dense value can leave [-Qmax, Qmax] (Eq. 11): s >= max|E^d| / Qmax by the round-up, and the two
+            // binary32 roundings of e * (1/s) add a few 2^-24 relative, far from the next half.  The exception is a
+            // scale that binary16 cannot hold (s stuck at 65504): then, and only then, the clamp does something.
+            // The channels of the outlier mask do exceed the range; their codes and x_hat are replaced below, and
+            // the packing keeps only the low bits of every field.  The magic add is written as v*1 + magic so that
+            // it stays a second rounding after the product (a plain add could be merged with the multiply).
+            const bool clamp = __any_sync(group_mask, s16 >= 0x7bffu);
+            const u64 one2 = pack2(1.0f, 1.0f);
             uint32_t words[4][2];
+            auto quantise = [&](auto clamp_tag) {
+                constexpr bool CLAMP = decltype(clamp_tag)::value;
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
-                uint32_t t8[8], xh[4];
+                for (int j = 0; j < 4; j++) {
+                    uint32_t t8[8], xh[4];
 #pragma unroll
-                for (int i = 0; i < 4; i++) {
-                    float v0, v1;
-                    unpack2(pmul(e2[4 * j + i], inv2), v0, v1);
-                    v0 = fminf(fmaxf(v0, -qmax), qmax);
-                    v1 = fminf(fmaxf(v1, -qmax), qmax);
-                    const u64 tt = padd(pack2(v0, v1), magic2);
-                    float t0, t1;
-                    unpack2(tt, t0, t1);
-                    t8[2 * i] = __float_as_uint(t0);
-                    t8[2 * i + 1] = __float_as_uint(t1);
-                    if (XHAT) {
-                        // Eq. 9 with the code just chosen: x_hat = bf16((alpha*r + beta) + q*s)
-                        float x0, x1;
-                        unpack2(pfma(psub(tt, magic2), s2, pfma(a2, r2[4 * j + i], b2)), x0, x1);
-                        xh[i] = f2_to_bf16x2(x0, x1);
+                    for (int i = 0; i < 4; i++) {
+                        u64 vv = pmul(e2[4 * j + i], inv2);
+                        if (CLAMP) {
+                            float v0, v1;
+                            unpack2(vv, v0, v1);
+                            vv = pack2(fminf(fmaxf(v0, -qmax), qmax), fminf(fmaxf(v1, -qmax), qmax));
+                        }
+                        const u64 tt = pfma(vv, one2, magic2);
+                        float t0, t1;
+                        unpack2(tt, t0, t1);
+                        t8[2 * i] = __float_as_uint(t0);
+                        t8[2 * i + 1] = __float_as_uint(t1);
+                        if (XHAT) {
+                            // Eq. 9 with the code just chosen: x_hat = bf16((alpha*r + beta) + q*s)
+                            float x0, x1;
+                            unpack2(pfma(psub(tt, magic2), s2, pfma(a2, r2[4 * j + i], b2)), x0, x1);
+                            xh[i] = f2_to_bf16x2(x0, x1);
+                        }
                     }
+                    pack_slot<BITS>(t8, words[j][0], words[j][1]);
+                    if (XHAT) sts128(xs + off[j], make_uint4(xh[0], xh[1], xh[2], xh[3]));
                 }
-                pack_slot<BITS>(t8, words[j][0], words[j][1]);
-                if (XHAT) sts128(xs + off[j], make_uint4(xh[0], xh[1], xh[2], xh[3]));
-            }
+            };
+            if (clamp) quantise(std::true_type{});
+            else quantise(std::false_type{});
             // slot order -> piece order (words[q] becomes the code word(s) of piece q)
             {
                 uint32_t lo[4] = {words[0][0], words[1][0], words[2][0], words[3][0]};

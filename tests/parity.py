@@ -53,8 +53,9 @@ def _check_flips(name, gpu16, orc16, exact, window_abs):
     [exact - W, exact + W] must reach the device value's binary16 rounding cell.
     gpu16: uint16 bit patterns of the mismatching entries; exact: binary64 optimum."""
     g = np.asarray(gpu16, np.uint16).view(np.float16)
-    below = np.nextafter(g, np.float16(-np.inf)).astype(np.float64)
-    above = np.nextafter(g, np.float16(np.inf)).astype(np.float64)
+    with np.errstate(over="ignore"):          # the neighbour of +-65504 is an infinity: fine as a cell border
+        below = np.nextafter(g, np.float16(-np.inf)).astype(np.float64)
+        above = np.nextafter(g, np.float16(np.inf)).astype(np.float64)
     gv = g.astype(np.float64)
     W = window_abs + ALPHA_WINDOW_ULP * np.maximum(above - gv, gv - below)
     lo_cell, hi_cell = (gv + below) / 2, (gv + above) / 2
@@ -97,9 +98,10 @@ def _eval_windows(Xb, d, g, tj, ref_base, ref_row, gain, bias, alpha):
 def _half_ulp16(bits16):
     g = np.asarray(bits16, np.uint16).view(np.float16)
     gv = g.astype(np.float64)
-    below = np.nextafter(g, np.float16(-np.inf)).astype(np.float64)
-    above = np.nextafter(g, np.float16(np.inf)).astype(np.float64)
-    return np.maximum(above - gv, gv - below) / 2
+    with np.errstate(over="ignore"):
+        below = np.nextafter(g, np.float16(-np.inf)).astype(np.float64)
+        above = np.nextafter(g, np.float16(np.inf)).astype(np.float64)
+    return np.maximum(np.where(np.isfinite(above), above - gv, 0), np.where(np.isfinite(below), gv - below, 0)) / 2
 
 
 def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None, gain=None, bias=None,

@@ -626,3 +626,23 @@ def test_random_configurations_on_stressed_inputs(env):
             env.P.round_trip_case(cfg, X, ref_base=R, **kw)
         except AssertionError as e:
             raise AssertionError(f"{cfg!r} T={T} mode={mode} kind={kind}: {e}") from e
+
+
+@pytest.mark.parametrize("bits,kg,qg", [(4, 0, 0), (4, 1, 0), (8, 2, 0), (3, 0, 1024), (2, 1, 64)])
+def test_scale_that_binary16_cannot_hold(env, bits, kg, qg):
+    """Eq. 8 rounds the scale up in binary16; beyond 65504 it cannot, the scale sticks there and the codes clip --
+    the one case in which the clamp of the Eq. 8 encoder does something (without it the kernel skips the clamp).
+    Magnitudes of 1e5..1e7 with half of the tokens coded directly put many groups there; the rest of the groups,
+    in the same warps, stay below."""
+    d, g, T = 1024, 128, 150
+    X, R, _, _ = prefill_inputs(env, T, d, g, seed=71)
+    mag = 6e4 * ((1 << (bits - 1)) - 1)            # about Qmax * 65504: the border runs through the data
+    X = (X.float() * mag).to(torch.bfloat16)
+    R = (R.float() * mag).to(torch.bfloat16)
+    rows = np.arange(T, dtype=np.int32)
+    rows[::2] = -1
+    cfg = env.rac.CodecCfg(d, g, bits, 0, scale_mode=1, qgroup=qg, topk_group=kg)
+    rep, pay, xh = env.P.round_trip_case(cfg, X, ref_base=R, ref_row=torch.from_numpy(rows).to(env.dev))
+    scales = env.orc.split_payload(pay, T, d, g, bits, 0, 1, qg, kg)[4]
+    sat = (np.asarray(scales).reshape(-1) == 0x7bff).mean()
+    assert 0.02 < sat < 0.98, sat           # saturated and ordinary groups side by side
