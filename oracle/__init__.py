@@ -82,7 +82,7 @@ def _declare(l: C.CDLL) -> None:
     l.orc_encode.restype = C.c_int
     l.orc_encode.argtypes = [C.c_int] * 8 + [_u16p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
                                              _f32p, _f32p, _u32p, _u8p,
-                                             _f64p, _f64p, _f64p, _f64p, _f32p, _f32p, C.c_int]
+                                             _f64p, _f64p, _f64p, _f64p, _f32p, _f32p, _f64p, C.c_int]
     l.orc_reconstruct.restype = C.c_int
     l.orc_reconstruct.argtypes = [C.c_int] * 8 + [_u32p, _u8p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
                                                   _f32p, _u16p, _u32p, C.c_int]
@@ -214,7 +214,9 @@ def encode(d, group, bits, topk, X, ref_base=None, ref_row=None, gain=None, bias
            step=None, inv_step=None, forced_coef=None, diag=False, nthreads=1, scale_mode=0, qgroup=0, topk_group=0,
            coef_fmt=0):
     """Encode X (uint16 bf16 bits [T,d]).  Returns payload (uint8[T*rec]) and, with
-    ``diag=True``, a dict of the unrounded fit and the binary32 residual / scaled value."""
+    ``diag=True``, a dict of the unrounded fit, the binary32 residual ``e``, the binary32 scaled
+    value ``v`` the codes were rounded from, and ``v_ideal`` = e / s with the quotient in binary64
+    (Eq. 8 as printed; decides nothing, tests count the codes that differ from its rounding)."""
     X = _chk(X, np.uint16)
     T = X.size // d
     assert X.size == T * d
@@ -231,15 +233,18 @@ def encode(d, group, bits, topk, X, ref_base=None, ref_row=None, gain=None, bias
     rec = record_bytes(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt)
     payload = np.zeros(T * rec, np.uint8)
     dg = {}
-    if diag:
-        dg = dict(alpha=np.zeros((T, J)), beta=np.zeros((T, J)), hbar=np.zeros((T, J)), rbar=np.zeros((T, J)),
-                  e=np.zeros((T, d), np.float32), v=np.zeros((T, d), np.float32))
+    if diag:    # diag="fit": only the per-group outputs (the per-channel ones are large)
+        dg = dict(alpha=np.zeros((T, J)), beta=np.zeros((T, J)), hbar=np.zeros((T, J)), rbar=np.zeros((T, J)))
+        if diag != "fit":
+            dg.update(e=np.zeros((T, d), np.float32), v=np.zeros((T, d), np.float32),
+                      v_ideal=np.zeros((T, d), np.float64))
     rc = lib().orc_encode(d, group, bits, topk, scale_mode, qgroup, topk_group, coef_fmt, _p(X, _u16p), T, _p(ref_base, _u16p), ref_rows,
                           _p(ref_row, _i32p), _p(gain, _u16p), _p(bias, _u16p),
                           _p(step, _f32p), _p(inv_step, _f32p), _p(forced_coef, _u32p), _p(payload, _u8p),
                           _p(dg.get("alpha"), _f64p), _p(dg.get("beta"), _f64p),
                           _p(dg.get("hbar"), _f64p), _p(dg.get("rbar"), _f64p),
-                          _p(dg.get("e"), _f32p), _p(dg.get("v"), _f32p), int(nthreads))
+                          _p(dg.get("e"), _f32p), _p(dg.get("v"), _f32p), _p(dg.get("v_ideal"), _f64p),
+                          int(nthreads))
     if rc != 0:
         raise ValueError(f"orc_encode failed: {rc}")
     return (payload, dg) if diag else payload

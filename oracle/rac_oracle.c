@@ -359,8 +359,13 @@ static float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi
  *              rounding flip from everything downstream of it)
  * payload      T*record bytes out
  * diag_*       optional outputs (NULL to skip): unrounded alpha, beta, the
- *              group means (double[T,J] each), the binary32 residual e[T,d]
- *              and the scaled value v[T,d] the rounding decision was taken on.
+ *              group means (double[T,J] each), the binary32 residual e[T,d],
+ *              the scaled value v[T,d] the rounding decision was taken on
+ *              (binary32, e times the reciprocal of the step or scale), and
+ *              v_ideal[T,d] = e / s as Eq. 8 prints it, the quotient taken in
+ *              binary64 -- a diagnostic that decides no code: tests count the
+ *              codes that differ from the rounding of this value (0 where the
+ *              channel is an outlier or its step / scale is 0).
  * returns 0, or -1 bad configuration, -2 ref_row out of range.
  */
 int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group, int coef_fmt,
@@ -371,7 +376,7 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
                const uint32_t *forced_coef,
                uint8_t *payload,
                double *diag_alpha, double *diag_beta, double *diag_hbar, double *diag_rbar,
-               float *diag_e, float *diag_v, int nthreads) {
+               float *diag_e, float *diag_v, double *diag_v_ideal, int nthreads) {
     if (!cfg_ok(d, group, bits, topk)) return -1;
     if (!qcfg_ok(d, group, topk, scale_mode, qgroup, topk_group)) return -1;
     if ((gain == NULL) != (bias == NULL)) return -1;
@@ -483,11 +488,14 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
                 for (int c = 0; c < d; c++) {
                     int q = 0;
                     float v = 0.0f;
+                    double v_ideal = 0.0;
                     if (st[c] != 0.0f && !is_out[c]) {
                         v = e[c] * ist[c];
                         q = (int)rintf(clampf(v, (float)-qmax, (float)qmax));
+                        v_ideal = (double)e[c] / (double)st[c];
                     }
                     if (diag_v) diag_v[t * (int64_t)d + c] = v;
+                    if (diag_v_ideal) diag_v_ideal[t * (int64_t)d + c] = v_ideal;
                     if (diag_e) diag_e[t * (int64_t)d + c] = e[c];
                     put_code(codes, c, bits, q);
                 }
@@ -506,11 +514,14 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
                     for (int c = j * qgroup; c < (j + 1) * qgroup; c++) {
                         int q = 0;
                         float v = 0.0f;
+                        double v_ideal = 0.0;
                         if (!is_out[c]) {
                             v = e[c] * isc;
                             q = (int)rintf(clampf(v, (float)-qmax, (float)qmax));
+                            if (sc != 0.0f) v_ideal = (double)e[c] / (double)sc;
                         }
                         if (diag_v) diag_v[t * (int64_t)d + c] = v;
+                        if (diag_v_ideal) diag_v_ideal[t * (int64_t)d + c] = v_ideal;
                         if (diag_e) diag_e[t * (int64_t)d + c] = e[c];
                         put_code(codes, c, bits, q);
                     }

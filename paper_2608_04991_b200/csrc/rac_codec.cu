@@ -526,49 +526,54 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 // encode, second launch: outlier split (the k largest |e| per token, ties to the lower channel)
 // ------------------------------------------------------------------------------------------------
 // One warp per token.  Input: the per-thread maxima the streaming pass left in the workspace (one value per
-// 32 channels).  (a) Threshold: the k-th largest of the 32 per-lane maxima (lane l covers slabs l, l+32,
-// ...): the k largest come from k different lanes, each with an element at least that large, so at least k
-// elements reach it.  (b) Only slabs whose maximum reaches the threshold can hold one of the k largest:
-// their residuals are recomputed from X, the reference row and the wire coefficients in the record (the
-// same binary32 operations as in the streaming pass, so the same bits); elements at or above the threshold
-// become candidates.  (c) Candidates are ranked exactly by counting (magnitude bits, then lower channel).
-// (d) The winners, in channel order, go into the record's outlier fields and their dense codes are cleared
-// (E^d = E - O).  More candidates than the list holds (many equal magnitudes) falls back to k rounds of a
-// maximum over the whole token.
+// 32-channel slab).  (a) Threshold tau = the k-th largest slab maximum (duplicates counted): the k largest maxima
+// belong to k different slabs, each with an element at least that large, so at least k elements reach tau, and
+// an element that reaches it can only sit in a slab whose maximum does.  Every lane sorts its few maxima once
+// (lane l holds slabs l, l+32, ...); then k rounds of one warp-wide maximum over the lanes' heads, the lowest
+// lane that holds it popping its head.  (b) The slabs that reach tau -- k of them unless maxima tie -- are
+// listed in slab order and their residuals recomputed from X, the reference row and the wire coefficients in
+// the record, four lanes per slab, eight channels per lane, with the same binary32 operations as the streaming
+// pass (so the same bits).  Elements at or above tau are candidates, collected in channel order.  (c) Exactly
+// k candidates (the common case: no slab holds two of the k largest, nothing ties with tau) are the answer as
+// they stand.  More: ranked exactly by counting (magnitude bits, then lower channel).  More than the list holds
+// (many equal magnitudes, e.g. an all-zero residual): k rounds of a maximum over the whole token.  (d) The
+// winners, in channel order, go into the record's outlier fields and their dense codes are cleared (E^d = E - O);
+// with the sender-side reconstruction those channels of x_hat are replaced too.
 constexpr int kOutWarps = 8;       // warps per CTA
 constexpr int kOutCap = 128;       // candidate list per token in flight
-constexpr int kOutHot = 256;       // slab list per token in flight (d <= 8192 has at most 256 slabs)
 
-// W lanes work on one token: W = 32 (a warp per token) or 16 (two tokens per warp; the instruction stream is
-// shared, so a token costs about two thirds of the issue slots).  All warp collectives name only the W lanes
-// of the token.
-template <int BITS, int W, bool SUB>
-__global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecParams p) {
-    constexpr int TPW = 32 / W;                 // tokens per warp
-    constexpr int NV = 256 / W;                 // slab maxima per lane, at most
-    __shared__ unsigned long long s_cand[kOutWarps * TPW][kOutCap];
-    __shared__ float s_cande[kOutWarps * TPW][kOutCap];
-    __shared__ unsigned short s_hot[kOutWarps * TPW][kOutHot];
-    __shared__ unsigned long long s_sel[kOutWarps * TPW][16];
-    __shared__ float s_sele[kOutWarps * TPW][16];
+// eight values by a run-time index, as a select tree (no local-memory array)
+__device__ __forceinline__ float pick8(const float (&v)[8], int i) {
+    const float a0 = (i & 1) ? v[1] : v[0], a1 = (i & 1) ? v[3] : v[2], a2 = (i & 1) ? v[5] : v[4], a3 = (i & 1) ? v[7] : v[6];
+    const float b0 = (i & 2) ? a1 : a0, b1 = (i & 2) ? a3 : a2;
+    return (i & 4) ? b1 : b0;
+}
+
+// NV: slab maxima per lane (d <= 32*32*NV).  bits: code width (only the clearing of the codes depends on it).
+template <int NV, bool SUB>
+__global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecParams p, const int bits) {
+    __shared__ unsigned long long s_cand[kOutWarps][kOutCap];
+    __shared__ float s_cande[kOutWarps][kOutCap];
+    __shared__ float s_candrt[kOutWarps][kOutCap];
+    __shared__ unsigned short s_hot[kOutWarps][32 * NV];
+    __shared__ unsigned long long s_sel[kOutWarps][16];
+    __shared__ float s_sele[kOutWarps][16];
+    __shared__ float s_selrt[kOutWarps][16];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int sub = lane / W, sl = lane % W;    // which token of the warp, lane within the token's group
-    const unsigned int gmask = (W == 32) ? 0xffffffffu : (0xffffu << (16 * sub));
-    const int slot = warp * TPW + sub;
     const int d = p.d, nth = d >> 5, k = p.topk;
-    constexpr uint32_t cmask = (1u << BITS) - 1u;
-    unsigned long long *cand = s_cand[slot];
-    float *cande = s_cande[slot];
-    unsigned short *hot = s_hot[slot];
-    unsigned long long *sel = s_sel[slot];
-    float *sele = s_sele[slot];
-    const long long tstride = (long long)gridDim.x * kOutWarps * TPW;
-    const unsigned int lt_mask = (1u << sl) - 1u;
+    const uint32_t cmask = (1u << bits) - 1u;
+    unsigned long long *cand = s_cand[warp];
+    float *cande = s_cande[warp], *candrt = s_candrt[warp];
+    unsigned short *hot = s_hot[warp];
+    unsigned long long *sel = s_sel[warp];
+    float *sele = s_sele[warp], *selrt = s_selrt[warp];
+    const long long tstride = (long long)gridDim.x * kOutWarps;
+    const unsigned int lt_mask = (1u << lane) - 1u;
     const int tm_stride = (nth + 3) & ~3;       // rows of slab maxima are padded to 16 bytes
+    const bool want_xhat = p.X_hat != nullptr;
 
     const long long n_tok = tokens_to_do<SUB>(p);
-    const int ni = (nth + W - 1) / W;
-    // slab maxima of a token, lane l taking slabs l, l+W, ...; loaded one token ahead so that the first trip to
+    // slab maxima of a token, lane l taking slabs l, l+32, ...; loaded one token ahead so that the first trip to
     // memory of a token overlaps the work on the one before
     unsigned int tv[NV], tvn[NV];
     auto load_maxima = [&](long long tix, unsigned int (&dst)[NV]) {
@@ -578,11 +583,11 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
         const int lim = live ? nth : 0;     // slabs beyond the width (or beyond the last token) read as 0
 #pragma unroll
         for (int i = 0; i < NV; i++) {
-            const int th = sl + W * i;
+            const int th = lane + 32 * i;
             dst[i] = th < lim ? __float_as_uint(__ldg(tm + th)) : 0u;
         }
     };
-    const long long ti0 = ((long long)blockIdx.x * kOutWarps + warp) * TPW + sub;
+    const long long ti0 = (long long)blockIdx.x * kOutWarps + warp;
     load_maxima(ti0, tvn);
     for (long long ti = ti0; ti < n_tok; ti += tstride) {
         const long long t = token_at<SUB>(p, ti);
@@ -595,178 +600,180 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
         const uint16_t *rrow = row >= 0 ? ref_row_ptr<SUB>(p, row) : nullptr;
         unsigned char *rec = p.payload + t * p.rec;
         const uint32_t *coef = reinterpret_cast<const uint32_t *>(rec);
-        // residual of channel c, exactly as the streaming pass computed it (rare paths only)
-        auto residual = [&](int c) -> float {
-            const float h = __uint_as_float((uint32_t)xrow[c] << 16);
-            float r = 0.f;
-            if (rrow) {
-                r = __uint_as_float((uint32_t)rrow[c] << 16);
-                if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
-            }
-            const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
-            return __fsub_rn(h, __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16)));
-        };
 
-        // (a) threshold: the k-th largest of the W per-lane maxima (lane l covers slabs l, l+W, ...): the k largest
-        // come from k different lanes, each with an element at least that large, so at least k elements reach it;
-        // then the slabs that reach it, in slab order
-        unsigned int v = 0u;
+        // (a) threshold: the k-th largest slab maximum.  Bit patterns of non-negative floats order like integers.
+        unsigned int sv[NV];
 #pragma unroll
-        for (int i = 0; i < NV; i++) v = max(v, tv[i]);
-        unsigned int tau = 0u;
-        for (int r = 0; r < k; r++) {           // k <= 16 <= W, so k different lanes exist
-            tau = __reduce_max_sync(gmask, v);
-            if (r + 1 < k) {
-                const unsigned int bal = __ballot_sync(gmask, v == tau) & gmask;
-                if (lane == __ffs(bal) - 1) v = 0u;
+        for (int i = 0; i < NV; i++) sv[i] = tv[i];
+#pragma unroll
+        for (int r = 0; r < NV; r++) {          // odd-even transposition sort, descending
+#pragma unroll
+            for (int i = r & 1; i + 1 < NV; i += 2) {
+                const unsigned int hi = max(sv[i], sv[i + 1]), lo = min(sv[i], sv[i + 1]);
+                sv[i] = hi; sv[i + 1] = lo;
             }
         }
+        unsigned int tau = 0u;
+        for (int r = 0; r < k; r++) {
+            tau = __reduce_max_sync(0xffffffffu, sv[0]);
+            if (r + 1 < k) {
+                const unsigned int bal = __ballot_sync(0xffffffffu, sv[0] == tau);
+                if (lane == __ffs(bal) - 1) {
+#pragma unroll
+                    for (int i = 0; i + 1 < NV; i++) sv[i] = sv[i + 1];
+                    sv[NV - 1] = 0u;
+                }
+            }
+        }
+        // the slabs that reach it, in slab order
         int nh = 0;
 #pragma unroll
         for (int i = 0; i < NV; i++) {
-            if (i < ni) {
-                // a slab beyond the width has tv == 0 and can only pass when tau == 0; keep it out
-                const bool is_hot = tv[i] >= tau && (sl + W * i) < nth;
-                const unsigned int bal = (__ballot_sync(gmask, is_hot) & gmask) >> (W == 32 ? 0 : 16 * sub);
-                if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(sl + W * i);
-                nh += __popc(bal);
-            }
+            const bool is_hot = tv[i] >= tau && (lane + 32 * i) < nth;   // a slab beyond the width passes only when tau == 0
+            const unsigned int bal = __ballot_sync(0xffffffffu, is_hot);
+            if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(lane + 32 * i);
+            nh += __popc(bal);
         }
-        __syncwarp(gmask);
-        // (b) candidates: W/2 slabs per round, a lane takes 16 consecutive channels of one slab, so that the loads
-        // of all hot slabs of a typical token (8 to 16) are in flight together
-        int n = 0;  // uniform over the token's lanes
-        for (int base = 0; base < nh; base += W / 2) {
-            const int hi = base + (sl >> 1);
+        __syncwarp();
+        // (b) candidates: eight slabs per round, four lanes per slab, eight channels per lane
+        int n = 0;  // uniform over the warp
+        for (int base = 0; base < nh; base += 8) {
+            const int hi = base + (lane >> 2);
             const bool act = hi < nh;
-            const int c0 = act ? (int)hot[hi] * 32 + (sl & 1) * 16 : 0;
-            uint4 xw[2], rw[2];
-            xw[0] = xw[1] = rw[0] = rw[1] = make_uint4(0u, 0u, 0u, 0u);
+            const int c0 = act ? (int)hot[hi] * 32 + (lane & 3) * 8 : 0;
+            uint4 xw = make_uint4(0u, 0u, 0u, 0u), rw = xw;
             uint32_t cf = 0u;
             if (act) {
-                xw[0] = __ldg(reinterpret_cast<const uint4 *>(xrow + c0));
-                xw[1] = __ldg(reinterpret_cast<const uint4 *>(xrow + c0 + 8));
-                if (rrow) {
-                    rw[0] = __ldg(reinterpret_cast<const uint4 *>(rrow + c0));
-                    rw[1] = __ldg(reinterpret_cast<const uint4 *>(rrow + c0 + 8));
-                }
+                xw = __ldg(reinterpret_cast<const uint4 *>(xrow + c0));
+                if (rrow) rw = __ldg(reinterpret_cast<const uint4 *>(rrow + c0));
                 cf = coef[c0 >> (5 + p.lpg_shift)];
             }
-            const uint32_t xs[8] = {xw[0].x, xw[0].y, xw[0].z, xw[0].w, xw[1].x, xw[1].y, xw[1].z, xw[1].w};
-            const uint32_t rs[8] = {rw[0].x, rw[0].y, rw[0].z, rw[0].w, rw[1].x, rw[1].y, rw[1].z, rw[1].w};
+            const uint32_t xs[4] = {xw.x, xw.y, xw.z, xw.w};
+            const uint32_t rs[4] = {rw.x, rw.y, rw.z, rw.w};
             const float ca = half_bits_to_float(cf & 0xffff), cb = half_bits_to_float(cf >> 16);
-            float e[16];
+            float e[8], rt[8];
             if (rrow && p.gain) {
 #pragma unroll
-                for (int i = 0; i < 16; i++) {
+                for (int i = 0; i < 8; i++) {
                     const uint32_t xb = (i & 1) ? (xs[i >> 1] & 0xffff0000u) : (xs[i >> 1] << 16);
                     const uint32_t rb = (i & 1) ? (rs[i >> 1] & 0xffff0000u) : (rs[i >> 1] << 16);
                     const float r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c0 + i]), __uint_as_float(rb),
                                                          half_bits_to_float(p.bias[c0 + i])));
-                    e[i] = __fsub_rn(__uint_as_float(xb), __fmaf_rn(ca, r, cb));
+                    rt[i] = __fmaf_rn(ca, r, cb);
+                    e[i] = __fsub_rn(__uint_as_float(xb), rt[i]);
                 }
             } else {
                 // without a reference rw is zero, which is the zero reference of a directly coded token
+                const u64 a2 = pack2(ca, ca), b2 = pack2(cb, cb);
 #pragma unroll
-                for (int i = 0; i < 16; i++) {
-                    const uint32_t xb = (i & 1) ? (xs[i >> 1] & 0xffff0000u) : (xs[i >> 1] << 16);
-                    const uint32_t rb = (i & 1) ? (rs[i >> 1] & 0xffff0000u) : (rs[i >> 1] << 16);
-                    e[i] = __fsub_rn(__uint_as_float(xb), __fmaf_rn(ca, __uint_as_float(rb), cb));
+                for (int i = 0; i < 4; i++) {
+                    const u64 rt2 = pfma(a2, bf16x2_to_p(rs[i]), b2);
+                    unpack2(rt2, rt[2 * i], rt[2 * i + 1]);
+                    unpack2(psub(bf16x2_to_p(xs[i]), rt2), e[2 * i], e[2 * i + 1]);
                 }
             }
-            // which of the lane's 16 elements reach the threshold
+            // which of the lane's eight elements reach the threshold
             uint32_t m = 0u;
 #pragma unroll
-            for (int i = 0; i < 16; i++) m |= ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? (1u << i) : 0u;
+            for (int i = 0; i < 8; i++) m |= ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? (1u << i) : 0u;
             if (!act) m = 0u;
             const int cnt = __popc(m);
-            // exclusive prefix of the per-lane counts within the token's lanes
+            // exclusive prefix of the per-lane counts: candidates come out in channel order
             int incl = cnt;
 #pragma unroll
-            for (int o = 1; o < W; o <<= 1) {
-                const int up = __shfl_up_sync(gmask, incl, o, W);
-                if (sl >= o) incl += up;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
             }
             int pos = n + incl - cnt;
-            // few lanes have any, and those mostly one: walk the set bits, fetching the element by a select tree
-            while (m) {
+            while (m) {     // few lanes have any, and those mostly one
                 const int i = __ffs(m) - 1;
                 m &= m - 1u;
-                float s8[8], s4[4];
-#pragma unroll
-                for (int j = 0; j < 8; j++) s8[j] = (i & 1) ? e[2 * j + 1] : e[2 * j];
-#pragma unroll
-                for (int j = 0; j < 4; j++) s4[j] = (i & 2) ? s8[2 * j + 1] : s8[2 * j];
-                const float s20 = (i & 4) ? s4[1] : s4[0], s21 = (i & 4) ? s4[3] : s4[2];
-                const float ei = (i & 8) ? s21 : s20;
+                const float ei = pick8(e, i);
                 if (pos < kOutCap) {
                     cand[pos] = ((unsigned long long)(__float_as_uint(ei) & 0x7fffffffu) << 16) |
                                 (unsigned long long)(0xffff - (c0 + i));
                     cande[pos] = ei;
+                    if (want_xhat) candrt[pos] = pick8(rt, i);
                 }
                 pos++;
             }
-            n += __shfl_sync(gmask, incl, W - 1, W);
+            n += __shfl_sync(0xffffffffu, incl, 31);
         }
-        __syncwarp(gmask);
-        // (c) exact ranking
-        if (n <= kOutCap) {
-            for (int x = sl; x < n; x += W) {
+        __syncwarp();
+        // (c) the k winners: sel[] in any order, or (exactly k candidates) the list itself, already in channel order
+        const unsigned long long *win = sel;
+        const float *wine = sele, *winrt = selrt;
+        bool ordered = false;
+        if (n == k) {
+            win = cand; wine = cande; winrt = candrt;
+            ordered = true;
+        } else if (n <= kOutCap) {
+            for (int x = lane; x < n; x += 32) {
                 const unsigned long long mine = cand[x];
                 int rk = 0;
                 for (int y = 0; y < n; y++) rk += (cand[y] > mine) ? 1 : 0;
-                if (rk < k) { sel[rk] = mine; sele[rk] = cande[x]; }
+                if (rk < k) { sel[rk] = mine; sele[rk] = cande[x]; selrt[rk] = candrt[x]; }
             }
         } else {
+            // residual of channel c and its aligned reference, exactly as the streaming pass computed them
+            auto residual = [&](int c, float &rt_out) -> float {
+                const float h = __uint_as_float((uint32_t)xrow[c] << 16);
+                float r = 0.f;
+                if (rrow) {
+                    r = __uint_as_float((uint32_t)rrow[c] << 16);
+                    if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+                }
+                const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
+                rt_out = __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16));
+                return __fsub_rn(h, rt_out);
+            };
             unsigned long long prev = ~0ull;
             for (int r = 0; r < k; r++) {
                 unsigned long long best = 0ull;
-                float beste = 0.f;
-                for (int c = sl; c < d; c += W) {
-                    const float e = residual(c);
+                float beste = 0.f, bestrt = 0.f;
+                for (int c = lane; c < d; c += 32) {
+                    float rtc;
+                    const float e = residual(c, rtc);
                     const unsigned long long comp =
                         ((unsigned long long)(__float_as_uint(e) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
                     // a composite is 0 only for |e| == 0 at channel 65535, which d <= 8192 excludes
-                    if (comp < prev && comp > best) { best = comp; beste = e; }
+                    if (comp < prev && comp > best) { best = comp; beste = e; bestrt = rtc; }
                 }
-                for (int o = W / 2; o > 0; o >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(gmask, best, o, W);
-                    const float othere = __shfl_xor_sync(gmask, beste, o, W);
-                    if (other > best) { best = other; beste = othere; }
+                for (int o = 16; o > 0; o >>= 1) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+                    const float othere = __shfl_xor_sync(0xffffffffu, beste, o);
+                    const float otherrt = __shfl_xor_sync(0xffffffffu, bestrt, o);
+                    if (other > best) { best = other; beste = othere; bestrt = otherrt; }
                 }
-                if (sl == 0) { sel[r] = best; sele[r] = beste; }
+                if (lane == 0) { sel[r] = best; sele[r] = beste; selrt[r] = bestrt; }
                 prev = best;
             }
         }
-        __syncwarp(gmask);
+        __syncwarp();
         // (d) outlier fields in channel order, dense codes at those channels cleared
-        if (sl < k) {
-            const int c = 0xffff - (int)(sel[sl] & 0xffffull);
+        if (lane < k) {
+            const int c = 0xffff - (int)(win[lane] & 0xffffull);
             if (c < d) {
-                int pos = 0;
-                for (int y = 0; y < k; y++) pos += ((0xffff - (int)(sel[y] & 0xffffull)) < c) ? 1 : 0;
+                int pos = lane;
+                if (!ordered) {
+                    pos = 0;
+                    for (int y = 0; y < k; y++) pos += ((0xffff - (int)(win[y] & 0xffffull)) < c) ? 1 : 0;
+                }
                 unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
-                const uint32_t hv = float_to_half_bits_sat(sele[sl]);
+                const uint32_t hv = float_to_half_bits_sat(wine[lane]);
                 oidx[pos] = (unsigned short)c;
                 oidx[k + pos] = (unsigned short)hv;
-                if (p.X_hat) {
-                    // the sender-side reconstruction of an outlier channel: (alpha*r + beta) + the binary16 value
-                    float r = 0.f;
-                    if (rrow) {
-                        r = __uint_as_float((uint32_t)rrow[c] << 16);
-                        if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
-                    }
-                    const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
-                    const float rt = __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16));
-                    p.X_hat[t * d + c] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(rt, half_bits_to_float(hv))));
-                }
+                // the sender-side reconstruction of an outlier channel: (alpha*r + beta) + the binary16 value
+                if (want_xhat)
+                    p.X_hat[t * d + c] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(winrt[lane], half_bits_to_float(hv))));
                 uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
-                const int bit = c * BITS, wd = bit >> 5, sh = bit & 31;
+                const int bit = c * bits, wd = bit >> 5, sh = bit & 31;
                 atomicAnd(&codes32[wd], ~(cmask << sh));
-                if (sh + BITS > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
+                if (sh + bits > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
             }
         }
-        __syncwarp(gmask);
+        __syncwarp();
     }
 }
 
@@ -1322,22 +1329,14 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != RAC_OK) return rc;
-    // a warp per token; RAC_OUT_HALF=1 packs two tokens into a warp (16 lanes each; measured the same speed: the
-    // pass is bound by scattered 32-byte reads, not by issue slots)
-    const bool half = getenv("RAC_OUT_HALF") != nullptr;
-    const int tpw = (half && !sub) ? 2 : 1;
-    long long blocks = (p.T + kOutWarps * tpw - 1) / (kOutWarps * tpw);
+    // a warp per token
+    long long blocks = (p.T + kOutWarps - 1) / kOutWarps;
     if (blocks > (long long)di.sms * 8) blocks = (long long)di.sms * 8;
-#define RAC_OUT(B)                                                                                  \
-    if (sub) outlier_kernel<B, 32, true><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p);       \
-    else if (half) outlier_kernel<B, 16, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p); \
-    else outlier_kernel<B, 32, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p)
-    switch (g.bits) {
-        case 4: RAC_OUT(4); break;
-        case 3: RAC_OUT(3); break;
-        case 2: RAC_OUT(2); break;
-    }
-#undef RAC_OUT
+    const int nth = g.d / 32;
+    if (sub) outlier_kernel<8, true><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
+    else if (nth <= 128) outlier_kernel<4, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
+    else if (nth <= 160) outlier_kernel<5, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
+    else outlier_kernel<8, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 

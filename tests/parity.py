@@ -35,16 +35,60 @@ def f16v(bits):
     return np.asarray(bits, np.uint16).view(np.float16).astype(np.float64)
 
 
+BOUNDARY_TOL = 1e-4
+
+
 @dataclass
 class EncodeReport:
     groups: int
     alpha_flips: int
     beta_flips: int
     tokens_with_flip: int
+    widened_alpha: int = 0      # coefficients outside the plain 1e-3 relative bound, inside it with the evaluation windows
+    widened_beta: int = 0
+    codes: int = 0              # dense codes compared with the rounding of e / s taken in binary64
+    boundary_codes: int = 0     # of those, the ones that differ (each within 1e-4 of a rounding boundary)
 
     def __str__(self):
         return (f"{self.groups} groups: alpha flips {self.alpha_flips}, beta flips {self.beta_flips}, "
-                f"tokens touched {self.tokens_with_flip}")
+                f"tokens touched {self.tokens_with_flip}; beyond plain 1e-3: alpha {self.widened_alpha}, "
+                f"beta {self.widened_beta}; boundary codes {self.boundary_codes} of {self.codes}")
+
+    def __add__(self, o):
+        return EncodeReport(*[a + b for a, b in zip(self.astuple(), o.astuple())])
+
+    def astuple(self):
+        return (self.groups, self.alpha_flips, self.beta_flips, self.tokens_with_flip, self.widened_alpha,
+                self.widened_beta, self.codes, self.boundary_codes)
+
+
+def unpack_codes_all(codes: np.ndarray, d: int, bits: int) -> np.ndarray:
+    """uint8[T, d*bits/8] -> int8[T, d]: code of channel c = stream bits [c*bits, c*bits+bits), least significant
+    bit first, two's complement (the record layout; written out here with numpy's bit unpacking)."""
+    T = codes.shape[0]
+    b = np.unpackbits(codes, axis=1, bitorder="little")[:, : d * bits].reshape(T, d, bits)
+    val = np.zeros((T, d), np.int16)
+    for i in range(bits):
+        val += b[:, :, i].astype(np.int16) << i
+    val -= (val >> (bits - 1)) << bits
+    return val.astype(np.int8)
+
+
+def count_boundary_codes(codes_u8, v_ideal, d, bits):
+    """Codes against Eq. 8c as printed, q = round(clip(e / s)) with the quotient in binary64: returns
+    (codes compared, codes that differ); every difference must sit within BOUNDARY_TOL of a rounding boundary."""
+    qmax = (1 << (bits - 1)) - 1
+    q = unpack_codes_all(codes_u8, d, bits)
+    q_ideal = np.rint(np.clip(v_ideal, -qmax, qmax)).astype(np.int8)
+    diff = q != q_ideal
+    n = int(diff.sum())
+    if n:
+        vi = np.abs(v_ideal[diff])
+        dist = np.abs(vi - np.floor(vi) - 0.5)
+        assert np.all(np.abs(q[diff].astype(np.int16) - q_ideal[diff]) == 1), "a code is more than one level away from round(e/s)"
+        assert np.all(dist < BOUNDARY_TOL), (f"{int((dist >= BOUNDARY_TOL).sum())} codes differ from round(e/s) away from a "
+                                            f"rounding boundary; worst distance {float(dist.max())!r}")
+    return q.size, n
 
 
 def _check_flips(name, gpu16, orc16, exact, window_abs):
@@ -112,7 +156,7 @@ def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None
     T = Xb.size // d
     nthr = oracle.max_threads()
     o_payload, dg = oracle.encode(d, g, bits, k, Xb, ref_base=ref_base, ref_row=ref_row, gain=gain, bias=bias,
-                                  step=step, inv_step=inv_step, diag=True, nthreads=nthr, **mk)
+                                  step=step, inv_step=inv_step, diag="fit", nthreads=nthr, **mk)
     g_coef = oracle.split_payload(gpu_payload, T, d, g, bits, k, *mode)[0]
     o_coef = oracle.split_payload(o_payload, T, d, g, bits, k, *mode)[0]
     ga, gb = (g_coef & 0xffff).astype(np.uint16), (g_coef >> 16).astype(np.uint16)
@@ -146,8 +190,9 @@ def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None
         wa, wm = _eval_windows(Xb, d, g, np.argwhere(mb), ref_base, ref_row, gain, bias, a_exact[mb])
         _check_flips("beta", gb[mb], ob[mb], b_exact[mb], cancel[mb] + wa * np.abs(dg["rbar"][mb]) + wm)
     # stage 2: same coefficients -> everything else bit-identical
-    forced = oracle.encode(d, g, bits, k, Xb, ref_base=ref_base, ref_row=ref_row, gain=gain, bias=bias,
-                           step=step, inv_step=inv_step, forced_coef=g_coef.reshape(-1).copy(), nthreads=nthr, **mk)
+    forced, dgf = oracle.encode(d, g, bits, k, Xb, ref_base=ref_base, ref_row=ref_row, gain=gain, bias=bias,
+                                step=step, inv_step=inv_step, forced_coef=g_coef.reshape(-1).copy(), diag=True,
+                                nthreads=nthr, **mk)
     if not np.array_equal(forced, gpu_payload):
         rec = oracle.record_bytes(d, g, bits, k, *mode)
         bad = np.flatnonzero((forced.reshape(T, rec) != gpu_payload.reshape(T, rec)).any(axis=1))
@@ -155,7 +200,12 @@ def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None
         off = np.flatnonzero(forced.reshape(T, rec)[t] != gpu_payload.reshape(T, rec)[t])
         raise AssertionError(f"payload differs from the oracle in {bad.size} tokens; first token {t}, "
                              f"byte offsets {off[:8].tolist()} of {rec} (coef {4 * (d // g)}, codes {d * bits // 8})")
-    return EncodeReport(ma.size, int(ma.sum()), int(mb.sum()), int((ma | mb).any(axis=1).sum()))
+    # Eq. 8c prints a division; both sides multiply by a binary32 reciprocal.  The device's codes (equal to the
+    # forced run's) against the rounding of the binary64 quotient: they may differ only next to a rounding boundary.
+    n_codes, n_boundary = count_boundary_codes(oracle.split_payload(gpu_payload, T, d, g, bits, k, *mode)[1],
+                                               dgf["v_ideal"], d, bits)
+    return EncodeReport(ma.size, int(ma.sum()), int(mb.sum()), int((ma | mb).any(axis=1).sum()),
+                        int(va.sum()), int(vb.sum()), n_codes, n_boundary)
 
 
 def to_dev(a, dev, dtype=None):
