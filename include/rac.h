@@ -253,6 +253,10 @@ int rac_encode(const rac_codec_cfg *cfg, const void *X, int64_t T,
  *          `payload` with the same reference and step table.  Must not overlap X or payload.  It may be the very
  *          buffer that ref_base points to ONLY with ref_row == NULL (token t reads row t and writes row t; each
  *          row is read completely before it is written), which is how a decode loop keeps its state in place.
+ *          With per-token outliers (topk > 0) the outliers are picked in a second launch that reads X and the
+ *          reference rows again, after x_hat has been written: there X_hat must not overlap X, the in-place form
+ *          above is refused (RAC_EUNSUPPORTED), and with a row list no token may reference a row that this call
+ *          writes (the two-wave protocol of the *_list calls keeps to that; it is not checked on the device).
  * Both tables are read here (inv_step for the codes, step for x_hat). */
 int rac_encode_reconstruct(const rac_codec_cfg *cfg, const void *X, int64_t T,
                            const void *ref_base, int64_t ref_rows, const int32_t *ref_row,

@@ -526,21 +526,23 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 // encode, second launch: outlier split (the k largest |e| per token, ties to the lower channel)
 // ------------------------------------------------------------------------------------------------
 // One warp per token.  Input: the per-thread maxima the streaming pass left in the workspace (one value per
-// 32-channel slab).  (a) Threshold tau = the k-th largest slab maximum (duplicates counted): the k largest maxima
-// belong to k different slabs, each with an element at least that large, so at least k elements reach tau, and
-// an element that reaches it can only sit in a slab whose maximum does.  Every lane sorts its few maxima once
-// (lane l holds slabs l, l+32, ...); then k rounds of one warp-wide maximum over the lanes' heads, the lowest
-// lane that holds it popping its head.  (b) The slabs that reach tau -- k of them unless maxima tie -- are
-// listed in slab order and their residuals recomputed from X, the reference row and the wire coefficients in
-// the record, four lanes per slab, eight channels per lane, with the same binary32 operations as the streaming
-// pass (so the same bits).  Elements at or above tau are candidates, collected in channel order.  (c) Exactly
-// k candidates (the common case: no slab holds two of the k largest, nothing ties with tau) are the answer as
-// they stand.  More: ranked exactly by counting (magnitude bits, then lower channel).  More than the list holds
-// (many equal magnitudes, e.g. an all-zero residual): k rounds of a maximum over the whole token.  (d) The
-// winners, in channel order, go into the record's outlier fields and their dense codes are cleared (E^d = E - O);
-// with the sender-side reconstruction those channels of x_hat are replaced too.
+// 32-channel slab); lane l holds the NV consecutive slabs NV*l .. NV*l+NV-1, so lane order is channel order.
+// (a) Threshold tau: every lane offers its two largest maxima (two different slabs); k-1 rounds of a warp-wide
+// maximum over the heads, the lowest lane that holds it moving on to its second value, then one more maximum.
+// The k values seen are maxima of k different slabs, so at least k elements reach tau, and an element that
+// reaches it can only sit in a slab whose maximum does.  tau is the exact k-th largest slab maximum unless one
+// lane holds three of the k largest, and then only lower: a few more slabs are looked at, the result is the same.
+// (b) The slabs that reach tau -- k of them unless maxima tie -- are listed in slab order and their residuals
+// recomputed from X, the reference row and the wire coefficients in the record, four lanes per slab, eight
+// channels per lane, with the same binary32 operations as the streaming pass (so the same bits).  Elements at or
+// above tau are candidates, collected in channel order, one per lane.  (c) While there are more than k, the
+// smallest goes (smallest magnitude; among equals the highest channel): the survivors are the k largest with
+// ties to the lower channel, still in channel order.  More than 32 candidates (many equal magnitudes, e.g. an
+// all-zero residual): k rounds of a maximum over the whole token instead.  (d) The winners go into the record's
+// outlier fields in channel order, their dense codes are cleared (E^d = E - O), and with the sender-side
+// reconstruction those channels of x_hat are replaced.
 constexpr int kOutWarps = 8;       // warps per CTA
-constexpr int kOutCap = 128;       // candidate list per token in flight
+constexpr int kOutCap = 32;        // candidates per token: one per lane
 
 // eight values by a run-time index, as a select tree (no local-memory array)
 __device__ __forceinline__ float pick8(const float (&v)[8], int i) {
@@ -549,110 +551,167 @@ __device__ __forceinline__ float pick8(const float (&v)[8], int i) {
     return (i & 4) ? b1 : b0;
 }
 
-// NV: slab maxima per lane (d <= 32*32*NV).  bits: code width (only the clearing of the codes depends on it).
-template <int NV, bool SUB>
-__global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecParams p, const int bits) {
-    __shared__ unsigned long long s_cand[kOutWarps][kOutCap];
-    __shared__ float s_cande[kOutWarps][kOutCap];
-    __shared__ float s_candrt[kOutWarps][kOutCap];
-    __shared__ unsigned short s_hot[kOutWarps][32 * NV];
-    __shared__ unsigned long long s_sel[kOutWarps][16];
-    __shared__ float s_sele[kOutWarps][16];
-    __shared__ float s_selrt[kOutWarps][16];
+// whole-token path: k rounds of a maximum over all d channels (rare).  Lane r returns the r-th winner:
+// channel, residual, aligned reference.
+__device__ __noinline__ void select_whole_token(int d, int k, int coef_shift, const uint16_t *xrow, const uint16_t *rrow,
+                                                const uint16_t *gain, const uint16_t *bias, const uint32_t *coef,
+                                                int lane, int *c_out, float *e_out, float *rt_out) {
+    unsigned long long prev = ~0ull, mine = 0ull;
+    float minee = 0.f, minert = 0.f;
+    for (int r = 0; r < k; r++) {
+        unsigned long long best = 0ull;
+        float beste = 0.f, bestrt = 0.f;
+        for (int c = lane; c < d; c += 32) {
+            const float h = __uint_as_float((uint32_t)xrow[c] << 16);
+            float rr = 0.f;
+            if (rrow) {
+                rr = __uint_as_float((uint32_t)rrow[c] << 16);
+                if (gain) rr = bf16_round(__fmaf_rn(half_bits_to_float(gain[c]), rr, half_bits_to_float(bias[c])));
+            }
+            const uint32_t cf = coef[c >> coef_shift];
+            const float rtc = __fmaf_rn(half_bits_to_float(cf & 0xffff), rr, half_bits_to_float(cf >> 16));
+            const float e = __fsub_rn(h, rtc);
+            const unsigned long long comp =
+                ((unsigned long long)(__float_as_uint(e) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
+            // a composite is 0 only for |e| == 0 at channel 65535, which d <= 8192 excludes
+            if (comp < prev && comp > best) { best = comp; beste = e; bestrt = rtc; }
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+            const float othere = __shfl_xor_sync(0xffffffffu, beste, o);
+            const float otherrt = __shfl_xor_sync(0xffffffffu, bestrt, o);
+            if (other > best) { best = other; beste = othere; bestrt = otherrt; }
+        }
+        if (lane == r) { mine = best; minee = beste; minert = bestrt; }
+        prev = best;
+    }
+    *c_out = 0xffff - (int)(mine & 0xffffull);
+    *e_out = minee;
+    *rt_out = minert;
+}
+
+// NV: slab maxima per lane (d <= 32*32*NV).  KT: the number of outliers when it is 8 (unrolled), else 0 = p.topk.
+// bits: code width (only the clearing of the codes depends on it).  A warp works on kOutPair tokens at a time, phase
+// by phase, so that their trips to memory (scattered 32-byte reads of X, the reference row and the record, which
+// bound this pass) overlap.
+constexpr int kOutPair = 2;
+
+template <int NV, int KT, bool SUB>
+__global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecParams p, const int bits) {
+    constexpr int U = kOutPair;
+    __shared__ float s_e[kOutWarps][U][kOutCap];
+    __shared__ float s_rt[kOutWarps][U][kOutCap];
+    __shared__ unsigned short s_c[kOutWarps][U][kOutCap];
+    __shared__ unsigned char s_hot[kOutWarps][U][32 * NV];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int d = p.d, nth = d >> 5, k = p.topk;
+    const int d = p.d, nth = d >> 5;
+    const int k = KT ? KT : p.topk;
     const uint32_t cmask = (1u << bits) - 1u;
-    unsigned long long *cand = s_cand[warp];
-    float *cande = s_cande[warp], *candrt = s_candrt[warp];
-    unsigned short *hot = s_hot[warp];
-    unsigned long long *sel = s_sel[warp];
-    float *sele = s_sele[warp], *selrt = s_selrt[warp];
-    const long long tstride = (long long)gridDim.x * kOutWarps;
+    const long long tstride = (long long)gridDim.x * kOutWarps * U;
     const unsigned int lt_mask = (1u << lane) - 1u;
     const int tm_stride = (nth + 3) & ~3;       // rows of slab maxima are padded to 16 bytes
     const bool want_xhat = p.X_hat != nullptr;
-
+    const int my0 = NV * lane;                  // first slab of this lane
+    const int my_n = min(NV, max(0, nth - my0));  // how many of its NV slabs exist
+    const int coef_shift = 5 + p.lpg_shift;
     const long long n_tok = tokens_to_do<SUB>(p);
-    // slab maxima of a token, lane l taking slabs l, l+32, ...; loaded one token ahead so that the first trip to
-    // memory of a token overlaps the work on the one before
-    unsigned int tv[NV], tvn[NV];
-    auto load_maxima = [&](long long tix, unsigned int (&dst)[NV]) {
-        const bool live = tix < n_tok;
-        const long long tt = live ? token_at<SUB>(p, tix) : 0;
-        const float *tm = p.tmax + tt * tm_stride;
-        const int lim = live ? nth : 0;     // slabs beyond the width (or beyond the last token) read as 0
-#pragma unroll
-        for (int i = 0; i < NV; i++) {
-            const int th = lane + 32 * i;
-            dst[i] = th < lim ? __float_as_uint(__ldg(tm + th)) : 0u;
-        }
-    };
-    const long long ti0 = (long long)blockIdx.x * kOutWarps + warp;
-    load_maxima(ti0, tvn);
-    for (long long ti = ti0; ti < n_tok; ti += tstride) {
-        const long long t = token_at<SUB>(p, ti);
-#pragma unroll
-        for (int i = 0; i < NV; i++) tv[i] = tvn[i];
-        load_maxima(ti + tstride, tvn);
-        // reference row of the token, by the same rules as the streaming pass (which already reported bad rows)
-        const int row = resolve_row<SUB>(p, p.ref_row ? p.ref_row[t] : (int)t, false);
-        const uint16_t *xrow = p.X + t * d;
-        const uint16_t *rrow = row >= 0 ? ref_row_ptr<SUB>(p, row) : nullptr;
-        unsigned char *rec = p.payload + t * p.rec;
-        const uint32_t *coef = reinterpret_cast<const uint32_t *>(rec);
 
-        // (a) threshold: the k-th largest slab maximum.  Bit patterns of non-negative floats order like integers.
-        unsigned int sv[NV];
+    for (long long ti0 = ((long long)blockIdx.x * kOutWarps + warp) * U; ti0 < n_tok; ti0 += tstride) {
+        long long t[U];
+        const uint16_t *xrow[U], *rrow[U];
+        unsigned char *rec[U];
+        unsigned int tau[U];
+        int nh[U], n[U];
+        bool live[U];
+        // ---- (a) slab maxima, threshold, and the slabs that reach it, in slab order
 #pragma unroll
-        for (int i = 0; i < NV; i++) sv[i] = tv[i];
+        for (int u = 0; u < U; u++) {
+            live[u] = ti0 + u < n_tok;
+            t[u] = live[u] ? token_at<SUB>(p, ti0 + u) : 0;
+            unsigned int tv[NV];
+            {
+                const float *tm = p.tmax + t[u] * tm_stride + my0;
+                const int lim = live[u] ? my_n : 0;
+                if (NV % 4 == 0) {
 #pragma unroll
-        for (int r = 0; r < NV; r++) {          // odd-even transposition sort, descending
+                    for (int j = 0; j < NV / 4; j++) {
+                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        if (4 * j < lim) v = __ldg(reinterpret_cast<const uint4 *>(tm) + j);   // rows are padded to 16 bytes
+                        tv[4 * j + 0] = 4 * j + 0 < lim ? v.x : 0u;
+                        tv[4 * j + 1] = 4 * j + 1 < lim ? v.y : 0u;
+                        tv[4 * j + 2] = 4 * j + 2 < lim ? v.z : 0u;
+                        tv[4 * j + 3] = 4 * j + 3 < lim ? v.w : 0u;
+                    }
+                } else {
 #pragma unroll
-            for (int i = r & 1; i + 1 < NV; i += 2) {
-                const unsigned int hi = max(sv[i], sv[i + 1]), lo = min(sv[i], sv[i + 1]);
-                sv[i] = hi; sv[i + 1] = lo;
-            }
-        }
-        unsigned int tau = 0u;
-        for (int r = 0; r < k; r++) {
-            tau = __reduce_max_sync(0xffffffffu, sv[0]);
-            if (r + 1 < k) {
-                const unsigned int bal = __ballot_sync(0xffffffffu, sv[0] == tau);
-                if (lane == __ffs(bal) - 1) {
-#pragma unroll
-                    for (int i = 0; i + 1 < NV; i++) sv[i] = sv[i + 1];
-                    sv[NV - 1] = 0u;
+                    for (int i = 0; i < NV; i++) tv[i] = i < lim ? __float_as_uint(__ldg(tm + i)) : 0u;
                 }
             }
-        }
-        // the slabs that reach it, in slab order
-        int nh = 0;
+            // reference row of the token, by the same rules as the streaming pass (which already reported bad rows)
+            const int row = live[u] ? resolve_row<SUB>(p, p.ref_row ? p.ref_row[t[u]] : (int)t[u], false) : -1;
+            xrow[u] = p.X + t[u] * d;
+            rrow[u] = row >= 0 ? ref_row_ptr<SUB>(p, row) : nullptr;
+            rec[u] = p.payload + t[u] * p.rec;
+            // threshold.  Bit patterns of non-negative floats order like integers.
+            unsigned int m1 = tv[0], m2 = 0u;
 #pragma unroll
-        for (int i = 0; i < NV; i++) {
-            const bool is_hot = tv[i] >= tau && (lane + 32 * i) < nth;   // a slab beyond the width passes only when tau == 0
-            const unsigned int bal = __ballot_sync(0xffffffffu, is_hot);
-            if (is_hot) hot[nh + __popc(bal & lt_mask)] = (unsigned short)(lane + 32 * i);
-            nh += __popc(bal);
+            for (int i = 1; i < NV; i++) {
+                m2 = max(m2, min(m1, tv[i]));
+                m1 = max(m1, tv[i]);
+            }
+#pragma unroll
+            for (int r = 1; r < k; r++) {
+                const unsigned int top = __reduce_max_sync(0xffffffffu, m1);
+                const unsigned int bal = __ballot_sync(0xffffffffu, m1 == top);
+                const bool pop = m1 == top && (bal & lt_mask) == 0u;
+                m1 = pop ? m2 : m1;
+                m2 = pop ? 0u : m2;
+            }
+            tau[u] = __reduce_max_sync(0xffffffffu, m1);
+            // tau == 0: fewer than k slabs hold anything but zeros, every element is a candidate: whole-token path
+            nh[u] = 0;
+            n[u] = live[u] ? kOutCap + 1 : 0;
+            if (tau[u] != 0u) {
+                unsigned int hm = 0u;
+#pragma unroll
+                for (int i = 0; i < NV; i++) hm |= (tv[i] >= tau[u]) ? (1u << i) : 0u;
+                int incl = __popc(hm);
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                    incl += lane >= o ? up : 0;
+                }
+                nh[u] = __shfl_sync(0xffffffffu, incl, 31);
+                int at = incl - __popc(hm);
+                while (hm) {
+                    s_hot[warp][u][at++] = (unsigned char)(my0 + __ffs(hm) - 1);
+                    hm &= hm - 1u;
+                }
+                n[u] = 0;
+            }
         }
         __syncwarp();
-        // (b) candidates: eight slabs per round, four lanes per slab, eight channels per lane
-        int n = 0;  // uniform over the warp
-        for (int base = 0; base < nh; base += 8) {
+        // ---- (b) candidates: eight slabs per round, four lanes per slab, eight channels per lane.  The first
+        // round of every token is loaded before any of them is used.
+        auto load_round = [&](int u, int base, int &c0, bool &act, uint4 &xw, uint4 &rw, uint32_t &cf) {
             const int hi = base + (lane >> 2);
-            const bool act = hi < nh;
-            const int c0 = act ? (int)hot[hi] * 32 + (lane & 3) * 8 : 0;
-            uint4 xw = make_uint4(0u, 0u, 0u, 0u), rw = xw;
-            uint32_t cf = 0u;
+            act = hi < nh[u];
+            c0 = act ? (int)s_hot[warp][u][hi] * 32 + (lane & 3) * 8 : 0;
+            xw = make_uint4(0u, 0u, 0u, 0u);
+            rw = xw;
+            cf = 0u;
             if (act) {
-                xw = __ldg(reinterpret_cast<const uint4 *>(xrow + c0));
-                if (rrow) rw = __ldg(reinterpret_cast<const uint4 *>(rrow + c0));
-                cf = coef[c0 >> (5 + p.lpg_shift)];
+                xw = __ldg(reinterpret_cast<const uint4 *>(xrow[u] + c0));
+                if (rrow[u]) rw = __ldg(reinterpret_cast<const uint4 *>(rrow[u] + c0));
+                cf = reinterpret_cast<const uint32_t *>(rec[u])[c0 >> coef_shift];
             }
+        };
+        auto use_round = [&](int u, int c0, bool act, const uint4 &xw, const uint4 &rw, uint32_t cf) {
             const uint32_t xs[4] = {xw.x, xw.y, xw.z, xw.w};
             const uint32_t rs[4] = {rw.x, rw.y, rw.z, rw.w};
             const float ca = half_bits_to_float(cf & 0xffff), cb = half_bits_to_float(cf >> 16);
             float e[8], rt[8];
-            if (rrow && p.gain) {
+            if (rrow[u] && p.gain) {
 #pragma unroll
                 for (int i = 0; i < 8; i++) {
                     const uint32_t xb = (i & 1) ? (xs[i >> 1] & 0xffff0000u) : (xs[i >> 1] << 16);
@@ -672,103 +731,104 @@ __global__ void __launch_bounds__(kOutWarps * 32, 4) outlier_kernel(const CodecP
                     unpack2(psub(bf16x2_to_p(xs[i]), rt2), e[2 * i], e[2 * i + 1]);
                 }
             }
-            // which of the lane's eight elements reach the threshold
+            // which of the lane's eight elements reach the threshold (tau > 0 here; for finite values the
+            // comparison of magnitudes is the comparison of their bit patterns)
+            const float tauf = __uint_as_float(tau[u]);
             uint32_t m = 0u;
 #pragma unroll
-            for (int i = 0; i < 8; i++) m |= ((__float_as_uint(e[i]) & 0x7fffffffu) >= tau) ? (1u << i) : 0u;
+            for (int i = 0; i < 8; i++) m |= (fabsf(e[i]) >= tauf) ? (1u << i) : 0u;
             if (!act) m = 0u;
             const int cnt = __popc(m);
-            // exclusive prefix of the per-lane counts: candidates come out in channel order
-            int incl = cnt;
+            // position of the lane's first candidate (candidates come out in channel order).  Almost always no
+            // lane has two, and a ballot does; otherwise a prefix sum over the lanes.
+            int pos, total;
+            if (!__any_sync(0xffffffffu, cnt > 1)) {
+                const unsigned int bal = __ballot_sync(0xffffffffu, cnt != 0);
+                pos = n[u] + __popc(bal & lt_mask);
+                total = __popc(bal);
+            } else {
+                int inc2 = cnt;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += up;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int up = __shfl_up_sync(0xffffffffu, inc2, o);
+                    inc2 += lane >= o ? up : 0;
+                }
+                pos = n[u] + inc2 - cnt;
+                total = __shfl_sync(0xffffffffu, inc2, 31);
             }
-            int pos = n + incl - cnt;
-            while (m) {     // few lanes have any, and those mostly one
+            while (m) {
                 const int i = __ffs(m) - 1;
                 m &= m - 1u;
-                const float ei = pick8(e, i);
                 if (pos < kOutCap) {
-                    cand[pos] = ((unsigned long long)(__float_as_uint(ei) & 0x7fffffffu) << 16) |
-                                (unsigned long long)(0xffff - (c0 + i));
-                    cande[pos] = ei;
-                    if (want_xhat) candrt[pos] = pick8(rt, i);
+                    s_e[warp][u][pos] = pick8(e, i);
+                    s_c[warp][u][pos] = (unsigned short)(c0 + i);
+                    if (want_xhat) s_rt[warp][u][pos] = pick8(rt, i);
                 }
                 pos++;
             }
-            n += __shfl_sync(0xffffffffu, incl, 31);
-        }
-        __syncwarp();
-        // (c) the k winners: sel[] in any order, or (exactly k candidates) the list itself, already in channel order
-        const unsigned long long *win = sel;
-        const float *wine = sele, *winrt = selrt;
-        bool ordered = false;
-        if (n == k) {
-            win = cand; wine = cande; winrt = candrt;
-            ordered = true;
-        } else if (n <= kOutCap) {
-            for (int x = lane; x < n; x += 32) {
-                const unsigned long long mine = cand[x];
-                int rk = 0;
-                for (int y = 0; y < n; y++) rk += (cand[y] > mine) ? 1 : 0;
-                if (rk < k) { sel[rk] = mine; sele[rk] = cande[x]; selrt[rk] = candrt[x]; }
-            }
-        } else {
-            // residual of channel c and its aligned reference, exactly as the streaming pass computed them
-            auto residual = [&](int c, float &rt_out) -> float {
-                const float h = __uint_as_float((uint32_t)xrow[c] << 16);
-                float r = 0.f;
-                if (rrow) {
-                    r = __uint_as_float((uint32_t)rrow[c] << 16);
-                    if (p.gain) r = bf16_round(__fmaf_rn(half_bits_to_float(p.gain[c]), r, half_bits_to_float(p.bias[c])));
+            n[u] += total;
+        };
+        {
+            int c0[U];
+            bool act[U];
+            uint4 xw[U], rw[U];
+            uint32_t cf[U];
+#pragma unroll
+            for (int u = 0; u < U; u++) load_round(u, 0, c0[u], act[u], xw[u], rw[u], cf[u]);
+#pragma unroll
+            for (int u = 0; u < U; u++) {
+                if (nh[u] > 0) use_round(u, c0[u], act[u], xw[u], rw[u], cf[u]);
+                for (int base = 8; base < nh[u] && n[u] <= kOutCap; base += 8) {
+                    load_round(u, base, c0[u], act[u], xw[u], rw[u], cf[u]);
+                    use_round(u, c0[u], act[u], xw[u], rw[u], cf[u]);
                 }
-                const uint32_t cf = coef[c >> (5 + p.lpg_shift)];
-                rt_out = __fmaf_rn(half_bits_to_float(cf & 0xffff), r, half_bits_to_float(cf >> 16));
-                return __fsub_rn(h, rt_out);
-            };
-            unsigned long long prev = ~0ull;
-            for (int r = 0; r < k; r++) {
-                unsigned long long best = 0ull;
-                float beste = 0.f, bestrt = 0.f;
-                for (int c = lane; c < d; c += 32) {
-                    float rtc;
-                    const float e = residual(c, rtc);
-                    const unsigned long long comp =
-                        ((unsigned long long)(__float_as_uint(e) & 0x7fffffffu) << 16) | (unsigned long long)(0xffff - c);
-                    // a composite is 0 only for |e| == 0 at channel 65535, which d <= 8192 excludes
-                    if (comp < prev && comp > best) { best = comp; beste = e; bestrt = rtc; }
-                }
-                for (int o = 16; o > 0; o >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-                    const float othere = __shfl_xor_sync(0xffffffffu, beste, o);
-                    const float otherrt = __shfl_xor_sync(0xffffffffu, bestrt, o);
-                    if (other > best) { best = other; beste = othere; bestrt = otherrt; }
-                }
-                if (lane == 0) { sel[r] = best; sele[r] = beste; selrt[r] = bestrt; }
-                prev = best;
             }
         }
         __syncwarp();
-        // (d) outlier fields in channel order, dense codes at those channels cleared
-        if (lane < k) {
-            const int c = 0xffff - (int)(win[lane] & 0xffffull);
-            if (c < d) {
-                int pos = lane;
-                if (!ordered) {
-                    pos = 0;
-                    for (int y = 0; y < k; y++) pos += ((0xffff - (int)(win[y] & 0xffffull)) < c) ? 1 : 0;
+        // ---- (c) one candidate per lane, in channel order; while there are too many the smallest goes
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+            if (!live[u]) continue;
+            bool won;
+            int wc = 0;
+            float we = 0.f, wrt = 0.f;
+            if (n[u] <= kOutCap) {
+                won = lane < n[u];
+                if (won) {
+                    wc = s_c[warp][u][lane];
+                    we = s_e[warp][u][lane];
+                    if (want_xhat) wrt = s_rt[warp][u][lane];
                 }
-                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec + 4 * p.J + p.code_bytes);
-                const uint32_t hv = float_to_half_bits_sat(wine[lane]);
-                oidx[pos] = (unsigned short)c;
+                unsigned int mag = won ? (__float_as_uint(we) & 0x7fffffffu) : 0xffffffffu;
+                for (int extra = n[u] - k; extra > 0; extra--) {
+                    const unsigned int low = __reduce_min_sync(0xffffffffu, mag);
+                    const unsigned int bal = __ballot_sync(0xffffffffu, mag == low);
+                    if (lane == 31 - __clz(bal)) { mag = 0xffffffffu; won = false; }   // among equals the highest channel
+                }
+            } else {
+                select_whole_token(d, k, coef_shift, xrow[u], rrow[u], p.gain, p.bias,
+                                   reinterpret_cast<const uint32_t *>(rec[u]), lane, &wc, &we, &wrt);
+                won = lane < k;
+            }
+            // ---- (d) outlier fields in channel order, dense codes at those channels cleared
+            int pos = __popc(__ballot_sync(0xffffffffu, won) & lt_mask);
+            if (n[u] > kOutCap) {   // the whole-token path returns its winners by rank, not by channel
+                pos = 0;
+                for (int y = 0; y < k; y++) {
+                    const int cy = __shfl_sync(0xffffffffu, wc, y);
+                    pos += cy < wc ? 1 : 0;
+                }
+            }
+            if (won) {
+                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec[u] + 4 * p.J + p.code_bytes);
+                const uint32_t hv = float_to_half_bits_sat(we);
+                oidx[pos] = (unsigned short)wc;
                 oidx[k + pos] = (unsigned short)hv;
                 // the sender-side reconstruction of an outlier channel: (alpha*r + beta) + the binary16 value
                 if (want_xhat)
-                    p.X_hat[t * d + c] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(winrt[lane], half_bits_to_float(hv))));
-                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec + 4 * p.J);
-                const int bit = c * bits, wd = bit >> 5, sh = bit & 31;
+                    p.X_hat[t[u] * d + wc] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(wrt, half_bits_to_float(hv))));
+                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec[u] + 4 * p.J);
+                const int bit = wc * bits, wd = bit >> 5, sh = bit & 31;
                 atomicAnd(&codes32[wd], ~(cmask << sh));
                 if (sh + bits > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
             }
@@ -1306,11 +1366,11 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
 static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
     if (g.scale_mode == 1) return launch_encode_dyn(g, p, max_ctas, stream);
     const bool topk = g.topk > 0;
-    p.stages = pick_stages(g.d, 2);
+    p.stages = 2;
     WsSmem L = ws_smem_layout(g.d, g.rec, p.stages, topk);
     // With x_hat the kernel reads both step tables every token; at four CTAs per SM the shared-memory carve-out
     // leaves too little L1 for them, so that variant runs three CTAs per SM at 128 registers.
-    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !p.X_hat && !getenv("RAC_ENC_WIDE");
+    const bool tight = g.nthreads > 96 && g.nthreads <= 160 && !p.X_hat;
     int rc = RAC_EUNSUPPORTED;
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;   // the subset form has one variant per width: it is not the hot path
 #define RAC_ENC2(B, K, X)                                                                                          \
@@ -1330,27 +1390,34 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     rc = device_info(&di);
     if (rc != RAC_OK) return rc;
     // a warp per token
-    long long blocks = (p.T + kOutWarps - 1) / kOutWarps;
-    if (blocks > (long long)di.sms * 8) blocks = (long long)di.sms * 8;
+    long long blocks = (p.T + kOutWarps * kOutPair - 1) / (kOutWarps * kOutPair);
+    if (blocks > (long long)di.sms * 3) blocks = (long long)di.sms * 3;   // three CTAs of 80 registers per SM
     const int nth = g.d / 32;
-    if (sub) outlier_kernel<8, true><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
-    else if (nth <= 128) outlier_kernel<4, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
-    else if (nth <= 160) outlier_kernel<5, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
-    else outlier_kernel<8, false><<<(unsigned)blocks, kOutWarps * 32, 0, stream>>>(p, g.bits);
+    const unsigned nb = (unsigned)blocks, nt = kOutWarps * 32;
+    if (sub) outlier_kernel<8, 0, true><<<nb, nt, 0, stream>>>(p, g.bits);
+    else if (g.topk == 8) {
+        if (nth <= 128) outlier_kernel<4, 8, false><<<nb, nt, 0, stream>>>(p, g.bits);
+        else if (nth <= 160) outlier_kernel<5, 8, false><<<nb, nt, 0, stream>>>(p, g.bits);
+        else outlier_kernel<8, 8, false><<<nb, nt, 0, stream>>>(p, g.bits);
+    } else {
+        if (nth <= 128) outlier_kernel<4, 0, false><<<nb, nt, 0, stream>>>(p, g.bits);
+        else if (nth <= 160) outlier_kernel<5, 0, false><<<nb, nt, 0, stream>>>(p, g.bits);
+        else outlier_kernel<8, 0, false><<<nb, nt, 0, stream>>>(p, g.bits);
+    }
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
 static int launch_decode(const Geometry &g, CodecParams &p, cudaStream_t stream) {
     if (g.scale_mode == 1) return launch_decode_dyn(g, p, stream);
-    p.stages = pick_stages(g.d, 2);
+    p.stages = 2;
     DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const int kt = g.topk == 0 ? 0 : (g.topk <= 8 ? 8 : 16);
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;
     // The streaming form is the faster one (131072 x 5120: 0.444 against 0.517 ms without outliers, 0.451 against
     // 0.491 ms with eight; 131072 x 4096: 0.37 against 0.43 and 0.40 against 0.46 ms).  The barrier form serves the
-    // token-list / second-reference-buffer calls, and everything under RAC_DEC_BARRIER=1.
-    const bool ws = !sub && !getenv("RAC_DEC_BARRIER");
-    const int wstages = pick_stages(g.d, g.nthreads > 128 ? 3 : 2);
+    // token-list / second-reference-buffer calls.
+    const bool ws = !sub;
+    const int wstages = (g.nthreads > 128 ? 3 : 2);
     DwSmem LW = dw_smem_layout(g.d, g.rec, wstages, kt > 0);
     if (ws) p.stages = wstages;
     const bool row1 = p.ref_row != nullptr || p.ref_base == nullptr;   // else every token has its reference row
@@ -1698,6 +1765,11 @@ size_t rac_encode_workspace_bytes(const rac_codec_cfg *cfg, int64_t T) {
     return (size_t)T * (size_t)(((g.d / 32) * 4 + 15) / 16 * 16);  // one 16-byte padded row of slab maxima per token
 }
 
+static bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return na > 0 && nb > 0 && a0 < b0 + nb && b0 < a0 + na;
+}
+
 static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
                        const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
                        const float *inv_step, void *payload, size_t payload_cap, void *X_hat, void *workspace,
@@ -1717,6 +1789,15 @@ static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const
     if (!aligned16(X) || !aligned16(payload) || (step && !aligned16(step)) || (inv_step && !aligned16(inv_step))) return RAC_EALIGN;
     if (X_hat && !aligned16(X_hat)) return RAC_EALIGN;
     if (payload_cap < (size_t)g.rec * (size_t)T) return RAC_ESIZE;
+    if (X_hat && g.topk > 0 && g.scale_mode == 0) {
+        // the outlier pass runs after the streaming pass has written x_hat and reads X and the reference rows
+        // again: a token's x_hat must not land on X, nor on a reference row that this call still reads.  With
+        // identity rows (ref_row == NULL) every token's reference row is the row it writes.
+        const size_t out_bytes = (size_t)T * (size_t)g.d * 2;
+        if (ranges_overlap(X_hat, out_bytes, X, out_bytes)) return RAC_EUNSUPPORTED;
+        if (ref_base && !ref_row && ranges_overlap(X_hat, out_bytes, ref_base, (size_t)ref_rows * (size_t)g.d * 2))
+            return RAC_EUNSUPPORTED;
+    }
     const size_t need = rac_encode_workspace_bytes(cfg, T);
     if (need > 0) {
         if (!workspace) return RAC_EINVAL;
@@ -1829,7 +1910,7 @@ int rac_fit_segments(const rac_codec_cfg *cfg, const void *X, int64_t T, const v
     p.X = static_cast<const uint16_t *>(X);
     p.moments = static_cast<float4 *>(workspace);
     if (T > 0) {
-        p.stages = pick_stages(g.d, 2);
+        p.stages = 2;
         EncSmem L = enc_smem_layout(g.d, p.stages, g.nthreads);
         rc = launch_persistent(calib_kernel<true>, p, g.nthreads, L.total, T, st);
         if (rc != RAC_OK) return rc;
@@ -1884,7 +1965,7 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, cons
     p.calib_partial = static_cast<float *>(workspace);
     // every CTA of the fixed grid writes its partials, also when it has no token
     {
-        p.stages = pick_stages(g.d, 2);
+        p.stages = 2;
         EncSmem L = enc_smem_layout(g.d, p.stages, g.nthreads);
         DeviceInfo di;
         rc = device_info(&di);

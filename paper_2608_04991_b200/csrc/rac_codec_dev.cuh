@@ -5,6 +5,11 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <utility>
+
 #include "rac_common.cuh"
 
 namespace rac {
@@ -315,10 +320,15 @@ struct DeviceInfo {
     int sms = 0;
     int max_smem_optin = 0;
 };
-static int device_info(DeviceInfo *out) {
+inline std::mutex &launch_mutex() {
+    static std::mutex m;
+    return m;
+}
+static int device_info(DeviceInfo *out, int *dev_out = nullptr) {
     static DeviceInfo cache[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RAC_ECUDA;
+    std::lock_guard<std::mutex> lock(launch_mutex());
     if (cache[dev].sms == 0) {
         int sms = 0, smem = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RAC_ECUDA;
@@ -327,6 +337,38 @@ static int device_info(DeviceInfo *out) {
         cache[dev].sms = sms;
     }
     *out = cache[dev];
+    if (dev_out) *dev_out = dev;
+    return RAC_OK;
+}
+
+// Resident CTAs per SM of one kernel at one block size and shared-memory size, looked up once per device.  The
+// kernel's shared-memory limit is an attribute of the kernel, not of a launch: it is only ever raised, so that a
+// launch with less shared memory between two larger ones leaves it where the larger ones need it.
+static int resident_ctas(const void *kernel, int dev, int nthreads, int smem_bytes, int *occ_out) {
+    struct Key {
+        const void *kernel;
+        int dev, nthreads, smem;
+        bool operator<(const Key &o) const {
+            return std::tie(kernel, dev, nthreads, smem) < std::tie(o.kernel, o.dev, o.nthreads, o.smem);
+        }
+    };
+    static std::map<Key, int> table;
+    static std::map<std::pair<const void *, int>, int> limit;   // (kernel, device) -> shared-memory limit set so far
+    const Key key{kernel, dev, nthreads, smem_bytes};
+    std::lock_guard<std::mutex> lock(launch_mutex());
+    auto it = table.find(key);
+    if (it == table.end()) {
+        int &lim = limit[std::make_pair(kernel, dev)];
+        if (smem_bytes > lim) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return RAC_ECUDA;
+            lim = smem_bytes;
+        }
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, nthreads, smem_bytes) != cudaSuccess || occ < 1)
+            return RAC_ECUDA;
+        it = table.emplace(key, occ).first;
+    }
+    *occ_out = it->second;
     return RAC_OK;
 }
 
@@ -334,13 +376,13 @@ template <typename K>
 static int launch_persistent(K kernel, const CodecParams &p, int nthreads, int smem_bytes, long long max_ctas,
                              cudaStream_t stream) {
     DeviceInfo di;
-    int rc = device_info(&di);
+    int dev = 0;
+    int rc = device_info(&di, &dev);
     if (rc != RAC_OK) return rc;
     if (smem_bytes > di.max_smem_optin) return RAC_EUNSUPPORTED;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return RAC_ECUDA;
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, nthreads, smem_bytes) != cudaSuccess || occ < 1)
-        return RAC_ECUDA;
+    rc = resident_ctas(reinterpret_cast<const void *>(kernel), dev, nthreads, smem_bytes, &occ);
+    if (rc != RAC_OK) return rc;
     long long grid = (long long)di.sms * occ;
     if (grid > max_ctas) grid = max_ctas;
     if (grid < 1) grid = 1;
@@ -349,13 +391,5 @@ static int launch_persistent(K kernel, const CodecParams &p, int nthreads, int s
 }
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-// Ring depth.  RAC_STAGES (2..4) overrides the default for tuning runs.
-static int pick_stages(int d, int dflt) {
-    const char *e = getenv("RAC_STAGES");
-    if (e && e[0] >= '2' && e[0] <= '4' && e[1] == 0) return e[0] - '0';
-    (void)d;
-    return dflt;
-}
 
 }  // namespace rac

@@ -665,7 +665,7 @@ static int launch_encode_variant(bool tight, const Geometry &g, CodecParams &p, 
 
 template <int B>
 static int launch_encode_bits(const Geometry &g, CodecParams &p, int smem, long long max_ctas, cudaStream_t stream) {
-    const bool tight = g.nthreads > 128 && g.nthreads <= 160 && !getenv("RAC_ENC_WIDE");
+    const bool tight = g.nthreads > 128 && g.nthreads <= 160;
     const int k = g.topk_group;
     if (p.X_hat) {
         return k == 0 ? launch_encode_variant<B, true, 0>(tight, g, p, smem, max_ctas, stream)
@@ -680,7 +680,7 @@ static int launch_encode_bits(const Geometry &g, CodecParams &p, int smem, long 
 }
 
 int launch_encode_dyn(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
-    p.stages = pick_stages(g.d, 2);
+    p.stages = 2;
     const DynSmem L = dyn_smem_layout(g.d, g.rec, p.stages);
     switch (g.bits) {
         case 8: return launch_encode_bits<8>(g, p, L.total, max_ctas, stream);
@@ -692,7 +692,7 @@ int launch_encode_dyn(const Geometry &g, CodecParams &p, long long max_ctas, cud
 }
 
 int launch_decode_dyn(const Geometry &g, CodecParams &p, cudaStream_t stream) {
-    p.stages = pick_stages(g.d, 2);
+    p.stages = 2;
     const DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const bool kg = g.topk_group > 0;
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;

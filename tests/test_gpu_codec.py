@@ -216,6 +216,40 @@ def test_in_place_identity_reconstruction(env):
     assert int(status.item()) == 0 and torch.equal(buf, out_of_place)
 
 
+def test_fused_sender_in_place_with_outliers_is_refused(env):
+    """With per-token outliers the sender-side x_hat may not overwrite the rows it was coded against (the outlier
+    launch reads them again after x_hat is written): the call is refused before anything runs, the buffers stay
+    untouched, and the out-of-place call on the same inputs matches the receiver and the oracle."""
+    d, g, bits, k, T = 2048, 128, 4, 8, 96
+    s, rac, dev = env.synth, env.rac, env.dev
+    gen = s.generator(18, dev)
+    prev = s.activations(T, d, s.channel_scale(d, 18, dev), gen)
+    X = s.random_walk_step(prev, gen)
+    step, inv = env.orc.calibrate(d, g, bits, s.bf16_bits(X), ref_base=s.bf16_bits(prev))
+    step_d, inv_d = env.P.to_dev(step, dev), env.P.to_dev(inv, dev)
+    cfg = rac.CodecCfg(d, g, bits, k)
+    rec = rac.rac_record_bytes(cfg)
+    pay = torch.full((T * rec,), 0xA5, dtype=torch.uint8, device=dev)
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    state = prev.clone()
+    with pytest.raises(Exception) as ei:
+        rac.rac_encode_reconstruct(cfg, X, T, state, T, None, None, None, step_d, inv_d, pay, pay.numel(), state, ws, nws, status)
+    assert "unsupported" in str(ei.value).lower()
+    xin = X.clone()
+    with pytest.raises(Exception):       # x_hat over X itself
+        rac.rac_encode_reconstruct(cfg, xin, T, prev, T, None, None, None, step_d, inv_d, pay, pay.numel(), xin, ws, nws, status)
+    torch.cuda.synchronize()
+    assert torch.equal(state, prev) and torch.equal(xin, X) and bool(torch.all(pay == 0xA5))
+    # out of place: same bytes as rac_encode, x_hat equal to the receiver's and the oracle's
+    pay_f, xs, st = env.P.gpu_encode_reconstruct(cfg, X, prev, None, None, None, step_d, inv_d)
+    xr, st2 = env.P.gpu_decode(cfg, pay_f, T, prev, None, None, None, step_d, dev)
+    assert st == 0 and st2 == 0 and torch.equal(xs, xr)
+    o_x = env.orc.reconstruct(d, g, bits, k, pay_f, T, ref_base=s.bf16_bits(prev), step=step)
+    assert np.array_equal(o_x, s.bf16_bits(xs))
+
+
 def test_zero_tokens_is_a_no_op(env):
     cfg = env.rac.CodecCfg(4096, 128, 4, 8)
     t = torch.zeros(16, dtype=torch.uint8, device=env.dev)
@@ -543,10 +577,15 @@ def test_tables_that_are_not_binary16_valued(env, k, monkeypatch):
     assert st == 0
     xr, st = P.gpu_decode(cfg, pay, T, R, rows, None, None, P.to_dev(step, dev), dev)
     assert st == 0 and torch.equal(xs, xr)
-    monkeypatch.setenv("RAC_DEC_BARRIER", "1")
-    xb, st = P.gpu_decode(cfg, pay, T, R, rows, None, None, P.to_dev(step, dev), dev)
-    assert st == 0 and torch.equal(xb, xr)
-    monkeypatch.delenv("RAC_DEC_BARRIER")
+    # the reconstruction kernel with a CTA barrier serves the token-list calls: all tokens through a list
+    toks = torch.arange(T, dtype=torch.int32, device=dev)
+    cnt = torch.tensor([T], dtype=torch.int32, device=dev)
+    xb = torch.empty_like(xr)
+    stt = torch.zeros(1, dtype=torch.int32, device=dev)
+    env.rac.rac_decode_reconstruct_list(cfg, torch.from_numpy(pay).to(dev), T, toks, cnt, R, T, rows, None, 0, None, None,
+                                        P.to_dev(step, dev), xb, stt)
+    torch.cuda.synchronize()
+    assert int(stt.item()) == 0 and torch.equal(xb, xr)
     # row 0 exact in binary16, row 1 not, and the other way round: the two rows are handled independently
     for keep in (0, 1):
         mixed = step.copy()
