@@ -208,6 +208,64 @@ def compare_encode(cfg, gpu_payload: np.ndarray, Xb, ref_base=None, ref_row=None
                         int(va.sum()), int(vb.sum()), n_codes, n_boundary)
 
 
+# Caps on what the protocol tolerates, as fractions of what was compared, so that a regression cannot hide inside
+# the tolerances.  Coefficient words that differ from the binary64 fit (each already checked to sit inside the
+# rounding window): the binary32 fit errs by ~1e-7 relative against a binary16 cell of ~1e-3, so ~1e-4 of the slopes
+# and (the intercept is a difference of two larger numbers) ~1e-3 of the intercepts land on the other side of a
+# rounding boundary (measured on B200: 0.7-1.2e-4 and 4e-4-3.1e-3 on the five configurations).  Entries that need the
+# evaluation windows on top of the plain 1e-3 relative bound: none on the configurations' generators; only crafted
+# inputs (uncorrelated references, groups whose values cancel) produce them.  Codes that differ from round(e/s): the
+# quotient within ~2^-22*Qmax of a boundary, measured 0-1.5e-6 of the codes at 2-4 bits, 1.3e-5 at 8 bits.
+CAP_ALPHA_FLIPS = 5e-4
+CAP_BETA_FLIPS = 5e-3
+CAP_WIDENED_ALPHA = 1e-4
+CAP_WIDENED_BETA = 1e-4
+CAP_BOUNDARY_CODES = 3e-5
+
+
+def assert_caps(rep: EncodeReport):
+    floor = 4     # small cases: a handful of entries is no rate
+    assert rep.alpha_flips <= max(floor, CAP_ALPHA_FLIPS * rep.groups), rep
+    assert rep.beta_flips <= max(floor, CAP_BETA_FLIPS * rep.groups), rep
+    assert rep.widened_alpha <= max(floor, CAP_WIDENED_ALPHA * rep.groups), rep
+    assert rep.widened_beta <= max(floor, CAP_WIDENED_BETA * rep.groups), rep
+    assert rep.boundary_codes <= max(floor, CAP_BOUNDARY_CODES * rep.codes), rep
+
+
+def compare_whole(cfg, payload_dev, X, X_hat, ref_base=None, ref_row=None, step=None, inv_step=None, chunk=16384):
+    """Every token of a large call against the oracle, in chunks the oracle finishes in seconds: the encode protocol
+    (compare_encode) on the device's records, and the oracle's reconstruction of those records against X_hat (the
+    device's reconstruction, or None).  ref_base: device tensor of reference rows or None; ref_row: numpy int32[T]
+    (entries < 0 = coded directly) or None for identity rows.  Returns the summed EncodeReport."""
+    d = cfg.d
+    T = X.shape[0]
+    rec = rac.rac_record_bytes(cfg)
+    mk = dict(scale_mode=cfg.scale_mode, qgroup=cfg.qgroup, topk_group=cfg.topk_group)
+    pay2 = payload_dev.view(T, rec)
+    total = None
+    for t0 in range(0, T, chunk):
+        t1 = min(T, t0 + chunk)
+        Xb = synth.bf16_bits(X[t0:t1])
+        Rb = rows = None
+        if ref_base is not None:
+            if ref_row is None:
+                Rb = synth.bf16_bits(ref_base[t0:t1])
+            else:      # gathered rows, made compact for the oracle
+                r = np.asarray(ref_row[t0:t1])
+                has = r >= 0
+                rows = np.where(has, np.cumsum(has) - 1, -1).astype(np.int32)
+                gathered = ref_base[torch.from_numpy(r[has].astype(np.int64)).to(ref_base.device)]
+                Rb = synth.bf16_bits(gathered) if has.any() else np.zeros((1, d), np.uint16)
+        pay = pay2[t0:t1].cpu().numpy().reshape(-1)
+        rep = compare_encode(cfg, pay, Xb, Rb, rows, None, None, step, inv_step)
+        total = rep if total is None else total + rep
+        if X_hat is not None:
+            o_x = oracle.reconstruct(d, cfg.group, cfg.bits, cfg.topk, pay, t1 - t0, ref_base=Rb, ref_row=rows, step=step,
+                                     nthreads=oracle.max_threads(), **mk)
+            assert np.array_equal(o_x, synth.bf16_bits(X_hat[t0:t1])), f"reconstruction differs in tokens {t0}..{t1}"
+    return total
+
+
 def to_dev(a, dev, dtype=None):
     if a is None:
         return None

@@ -310,12 +310,12 @@ def test_full_size_sweep_point(env, bits, g):
     step, inv = oracle_tables(env, d, g, bits, cal, calr)
     rep, _, _ = env.P.round_trip_case(env.rac.CodecCfg(d, g, bits, k), X, ref_base=R, step=step, inv_step=inv)
     print(rep)
-    assert rep.alpha_flips <= rep.groups * 5e-4 and rep.beta_flips <= rep.groups * 5e-3
+    env.P.assert_caps(rep)
 
 
-def test_long_context_sampled(env):
+def test_long_context_whole(env):
     """T=131072, d=5120, span-style gathered rows with 30 % direct tokens: the device runs the full size in
-    the launch configuration of the benchmark; the oracle checks a sample of tokens one by one."""
+    the launch configuration of the benchmark; the oracle checks every token, chunk by chunk."""
     d, g, bits, k, T, H = 5120, 128, 4, 8, 131072, 131072
     s, rac, orc = env.synth, env.rac, env.orc
     gen = s.generator(4, env.dev)
@@ -340,23 +340,11 @@ def test_long_context_sampled(env):
     rac.rac_decode_reconstruct(cfg, payload, T, Hs, H, ref_row, None, None, step, xh, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    # sample: first and last tokens, a stretch around a span boundary, and random ones
-    rng = np.random.default_rng(4)
-    sample = np.unique(np.concatenate([np.arange(64), np.arange(T - 64, T), rng.integers(0, T, 1900)]))
-    idx = torch.from_numpy(sample).to(env.dev)
-    rows = wl.planted_row[sample]
-    # the oracle gets the sampled tokens with their reference rows gathered into a compact buffer
-    has = rows >= 0
-    compact_rows = np.where(has, np.cumsum(has) - 1, -1).astype(np.int32)
-    Rc = Hs[torch.from_numpy(rows[has]).to(env.dev).long()]
-    Xs = X[idx]
-    pay_s = payload.view(T, rec)[idx].cpu().numpy().reshape(-1)
+    # every token against the oracle, in chunks (reference rows gathered into a compact buffer per chunk)
     st, iv = step.cpu().numpy(), inv.cpu().numpy()
-    rep = env.P.compare_encode(cfg, pay_s, s.bf16_bits(Xs), s.bf16_bits(Rc), compact_rows, None, None, st, iv)
+    rep = env.P.compare_whole(cfg, payload, X, xh, ref_base=Hs, ref_row=wl.planted_row, step=st, inv_step=iv)
     print(rep)
-    o_x = orc.reconstruct(d, g, bits, k, pay_s, sample.size, ref_base=s.bf16_bits(Rc), ref_row=compact_rows, step=st,
-                          nthreads=orc.max_threads())
-    assert np.array_equal(o_x, s.bf16_bits(xh[idx]))
+    env.P.assert_caps(rep)
     # properties that hold at any size: Eq. 10 bound on every element of the full tensor
     within, total = 0, 0
     for t0 in range(0, T, 16384):

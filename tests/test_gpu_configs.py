@@ -52,6 +52,7 @@ def test_config0_prefill_uplink_single_sequence(env):
     step, inv = env.orc.calibrate(d, g, 4, s.bf16_bits(cal), ref_base=s.bf16_bits(calr))
     rep, pay, xr = env.P.round_trip_case(env.rac.CodecCfg(d, g, 4, 0), X, ref_base=R, step=step, inv_step=inv)
     print("config 0:", rep)
+    env.P.assert_caps(rep)
     # the residual is coded: error about a step (3 sigma / 7), far below the activations
     err = (xr.float() - X.float()).abs()
     assert err.mean().item() < 0.02 and X.float().abs().mean().item() > 0.5
@@ -188,14 +189,14 @@ def test_config3_receiver_sweep(env, bits, g):
     step, inv = orc.calibrate(d, g, bits, s.bf16_bits(cal), ref_base=s.bf16_bits(calr))
     rep, _, _ = env.P.round_trip_case(env.rac.CodecCfg(d, g, bits, k), X, ref_base=R, step=step, inv_step=inv)
     print(f"config 3 b={bits} g={g}:", rep)
-    assert rep.alpha_flips <= rep.groups * 5e-4 and rep.beta_flips <= rep.groups * 5e-3
+    env.P.assert_caps(rep)
 
 
 def test_config4_long_context_round_trip(env):
     """T=131072, d=5120, group 128, 4-bit, top-8: span match (131072-token history, ~70 % coverage), uplink encode
     with the fused sender reconstruction, cloud reconstruct, downlink encode of Y = 1.05 * X_hat + N(0, 0.2)
     against X_hat, local reconstruct -- in the launch configuration of the benchmark; the oracle checks the
-    matcher whole and ~1500 sampled tokens of each direction one by one."""
+    matcher whole and every token of each direction against the oracle, chunk by chunk."""
     s, rac, orc, dev = env.synth, env.rac, env.orc, env.dev
     d, g, bits, k, T, H = 5120, 128, 4, 8, 131072, 131072
     cfg = rac.CodecCfg(d, g, bits, k)
@@ -235,24 +236,12 @@ def test_config4_long_context_round_trip(env):
     rac.rac_decode_reconstruct(cfg, pay_dn, T, Xh, T, None, None, None, step_dn, Yh, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    rng = np.random.default_rng(4)
-    sample = np.unique(np.concatenate([np.arange(48), np.arange(T - 48, T), rng.integers(0, T, 1400)]))
-    idx = torch.from_numpy(sample).to(dev)
-    # uplink sample: gathered references made compact for the oracle
-    rows = o_rows[sample]
-    has = rows >= 0
-    compact = np.where(has, np.cumsum(has) - 1, -1).astype(np.int32)
-    Rc = Hs[torch.from_numpy(rows[has]).to(dev).long()]
-    p_s = pay_up.view(T, rec)[idx].cpu().numpy().reshape(-1)
-    rep_up = env.P.compare_encode(cfg, p_s, s.bf16_bits(X[idx]), s.bf16_bits(Rc), compact, None, None, st_up, iv_up)
-    o_x = orc.reconstruct(d, g, bits, k, p_s, sample.size, ref_base=s.bf16_bits(Rc), ref_row=compact, step=st_up)
-    assert np.array_equal(o_x, s.bf16_bits(Xh[idx]))
-    # downlink sample: reference = the reconstructed uplink rows of the same tokens
-    p_s = pay_dn.view(T, rec)[idx].cpu().numpy().reshape(-1)
-    rep_dn = env.P.compare_encode(cfg, p_s, s.bf16_bits(Y[idx]), s.bf16_bits(Xh[idx]), None, None, None, st_dn, iv_dn)
-    o_y = orc.reconstruct(d, g, bits, k, p_s, sample.size, ref_base=s.bf16_bits(Xh[idx]), step=st_dn)
-    assert np.array_equal(o_y, s.bf16_bits(Yh[idx]))
+    # every token of both directions against the oracle, in chunks
+    rep_up = env.P.compare_whole(cfg, pay_up, X, Xh, ref_base=Hs, ref_row=o_rows, step=st_up, inv_step=iv_up)
+    rep_dn = env.P.compare_whole(cfg, pay_dn, Y, Yh, ref_base=Xh, ref_row=None, step=st_dn, inv_step=iv_dn)
     print("config 4 uplink:", rep_up, "| downlink:", rep_dn)
+    for rep in (rep_up, rep_dn):
+        env.P.assert_caps(rep)
     # Eq. 10 on every element of the downlink: inside the clip range the error is half a step plus the bf16 rounding
     within = total = 0
     for t0 in range(0, T, 16384):
@@ -268,8 +257,8 @@ def test_config4_long_context_round_trip(env):
                                     dict(bits=4, coef_fmt=1)])
 def test_config4_shape_with_the_eq8_family(env, member):
     """The benchmark's shape (131072 x 5120, groups of 128) through the per-group-scale kernels, in the launch
-    configuration `bench.py` times for its `paper_family` / `shared_coefficients` extras: ~1000 sampled tokens
-    checked one by one against the oracle, sender x_hat == receiver x_hat on the whole tensor, and Eq. 11's
+    configuration `bench.py` times for its `paper_family` / `shared_coefficients` extras: every token checked
+    against the oracle chunk by chunk, sender x_hat == receiver x_hat on the whole tensor, and Eq. 11's
     half-step bound (nothing clips) on every element."""
     s, rac, orc, dev = env.synth, env.rac, env.orc, env.dev
     d, g, T = 5120, 128, 131072
@@ -304,31 +293,32 @@ def test_config4_shape_with_the_eq8_family(env, member):
         rac.rac_decode_reconstruct(cfg, pay, T, R, T, None, None, None, None, xr, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and torch.equal(xs, xr)
-    rng = np.random.default_rng(9)
-    if shared:   # whole segments, so that the oracle can redo the pooled fit of the sampled ones
-        segs = np.unique(np.concatenate([[0, n_seg - 1], rng.integers(0, n_seg, 14)]))
-        sample = (segs[:, None] * seg_tokens + np.arange(seg_tokens)[None, :]).reshape(-1)
-    else:
-        sample = np.unique(np.concatenate([np.arange(48), np.arange(T - 48, T), rng.integers(0, T, 900)]))
-    idx = torch.from_numpy(sample).to(dev)
-    p_s = pay.view(T, rec)[idx].cpu().numpy().reshape(-1)
-    Xb, Rb = s.bf16_bits(X[idx]), s.bf16_bits(R[idx])
     if shared:
-        so = np.arange(len(segs) + 1, dtype=np.int32) * seg_tokens
-        o_coef = orc.fit_segments(d, g, Xb, so, ref_base=Rb)
-        g_coef = coef[torch.from_numpy(segs).to(dev)].cpu().numpy().view(np.uint32)
-        assert (g_coef != o_coef).sum() <= 3
-        per_tok = np.ascontiguousarray(np.repeat(g_coef, seg_tokens, axis=0))
-        o_pay = orc.encode(d, g, bits, 0, Xb, ref_base=Rb, forced_coef=per_tok.reshape(-1).copy(), coef_fmt=1,
-                           nthreads=orc.max_threads(), **mk)
-        assert np.array_equal(o_pay, p_s)
-        o_x = orc.reconstruct(d, g, bits, 0, p_s, sample.size, ref_base=Rb, coef_fmt=1, shared_coef=per_tok,
-                              nthreads=orc.max_threads(), **mk)
+        # every segment: the oracle redoes the pooled fit, then codes with the device's shared words, chunk by chunk
+        g_coef = coef.cpu().numpy().view(np.uint32)
+        flips = 0
+        chunk = 256 * seg_tokens
+        for t0 in range(0, T, chunk):
+            t1 = min(T, t0 + chunk)
+            k0, k1 = t0 // seg_tokens, t1 // seg_tokens
+            Xb, Rb = s.bf16_bits(X[t0:t1]), s.bf16_bits(R[t0:t1])
+            so = np.arange(k1 - k0 + 1, dtype=np.int32) * seg_tokens
+            o_coef = orc.fit_segments(d, g, Xb, so, ref_base=Rb)
+            flips += int((g_coef[k0:k1] != o_coef).sum())
+            per_tok = np.ascontiguousarray(np.repeat(g_coef[k0:k1], seg_tokens, axis=0))
+            p_s = pay.view(T, rec)[t0:t1].cpu().numpy().reshape(-1)
+            o_pay = orc.encode(d, g, bits, 0, Xb, ref_base=Rb, forced_coef=per_tok.reshape(-1).copy(), coef_fmt=1,
+                               nthreads=orc.max_threads(), **mk)
+            assert np.array_equal(o_pay, p_s)
+            o_x = orc.reconstruct(d, g, bits, 0, p_s, t1 - t0, ref_base=Rb, coef_fmt=1, shared_coef=per_tok,
+                                  nthreads=orc.max_threads(), **mk)
+            assert np.array_equal(o_x, s.bf16_bits(xr[t0:t1]))
+        print(member, f"shared words that differ from the binary64 pooled fit: {flips} of {g_coef.size}")
+        assert flips <= max(3, g_coef.size // 2000)
     else:
-        rep = env.P.compare_encode(cfg, p_s, Xb, Rb, None, None, None, None, None)
+        rep = env.P.compare_whole(cfg, pay, X, xr, ref_base=R, ref_row=None)
         print(member, rep)
-        o_x = orc.reconstruct(d, g, bits, 0, p_s, sample.size, ref_base=Rb, nthreads=orc.max_threads(), **mk)
-    assert np.array_equal(o_x, s.bf16_bits(xr[idx]))
+        env.P.assert_caps(rep)
     # Eq. 11 on every element: half a scale step (the record's own scale) plus the bf16 rounding; outliers: binary16
     scale_off = 0 if shared else 4 * J
     qg = mk["qgroup"] or g
