@@ -614,6 +614,8 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
     const int my0 = NV * lane;                  // first slab of this lane
     const int my_n = min(NV, max(0, nth - my0));  // how many of its NV slabs exist
     const int coef_shift = 5 + p.lpg_shift;
+    // everything this kernel reads was written by the streaming pass launched just before it
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const long long n_tok = tokens_to_do<SUB>(p);
 
     for (long long ti0 = ((long long)blockIdx.x * kOutWarps + warp) * U; ti0 < n_tok; ti0 += tstride) {
@@ -1361,6 +1363,23 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     return RAC_OK;
 }
 
+// Launch of a kernel that runs after the one before it on the stream, allowed to be set up while that one drains
+// (programmatic dependent launch): the kernel itself waits for its predecessor's memory before it reads anything.
+template <typename K, typename... Args>
+static void launch_after(K kernel, unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // Encode: the streaming kernel, then (with outliers) the selection kernel.  Variant 4 of the streaming kernel
 // caps registers at 96 so that four 160-thread CTAs fit on an SM.
 static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {
@@ -1390,19 +1409,26 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     rc = device_info(&di);
     if (rc != RAC_OK) return rc;
     // a warp per token
-    long long blocks = (p.T + kOutWarps * kOutPair - 1) / (kOutWarps * kOutPair);
-    if (blocks > (long long)di.sms * 3) blocks = (long long)di.sms * 3;   // three CTAs of 80 registers per SM
+    // three CTAs of 80 registers per SM; with more work than one round of them, every warp gets the same number of
+    // rounds (a grid of whole rounds, not a full grid with a ragged last round)
+    const long long per_cta = kOutWarps * kOutPair;
+    long long blocks = (p.T + per_cta - 1) / per_cta;
+    const long long resident = (long long)di.sms * 3;
+    if (blocks > resident) {
+        const long long rounds = (blocks + resident - 1) / resident;
+        blocks = (blocks + rounds - 1) / rounds;
+    }
     const int nth = g.d / 32;
     const unsigned nb = (unsigned)blocks, nt = kOutWarps * 32;
-    if (sub) outlier_kernel<8, 0, true><<<nb, nt, 0, stream>>>(p, g.bits);
+    if (sub) launch_after(outlier_kernel<8, 0, true>, nb, nt, stream, p, g.bits);
     else if (g.topk == 8) {
-        if (nth <= 128) outlier_kernel<4, 8, false><<<nb, nt, 0, stream>>>(p, g.bits);
-        else if (nth <= 160) outlier_kernel<5, 8, false><<<nb, nt, 0, stream>>>(p, g.bits);
-        else outlier_kernel<8, 8, false><<<nb, nt, 0, stream>>>(p, g.bits);
+        if (nth <= 128) launch_after(outlier_kernel<4, 8, false>, nb, nt, stream, p, g.bits);
+        else if (nth <= 160) launch_after(outlier_kernel<5, 8, false>, nb, nt, stream, p, g.bits);
+        else launch_after(outlier_kernel<8, 8, false>, nb, nt, stream, p, g.bits);
     } else {
-        if (nth <= 128) outlier_kernel<4, 0, false><<<nb, nt, 0, stream>>>(p, g.bits);
-        else if (nth <= 160) outlier_kernel<5, 0, false><<<nb, nt, 0, stream>>>(p, g.bits);
-        else outlier_kernel<8, 0, false><<<nb, nt, 0, stream>>>(p, g.bits);
+        if (nth <= 128) launch_after(outlier_kernel<4, 0, false>, nb, nt, stream, p, g.bits);
+        else if (nth <= 160) launch_after(outlier_kernel<5, 0, false>, nb, nt, stream, p, g.bits);
+        else launch_after(outlier_kernel<8, 0, false>, nb, nt, stream, p, g.bits);
     }
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
