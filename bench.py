@@ -46,6 +46,9 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="rac", choices=["rac", "reference"])
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every rank codes its own sequences; strong: the ranks share ONE tensor by token ranges "
+                         "and gather the payload byte ranges")
     ap.add_argument("--small", action="store_true", help="a small case of the same path (for profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -129,13 +132,14 @@ class RoundTrip:
     """Device buffers and the ordered C-ABI calls of one step."""
     LAUNCHES_PER_STEP = (9 + WORKLOAD["max_hits"]) + 2 * 2 + 2  # matcher kernels + 2 encodes (2 launches each) + 2 reconstructions
 
-    def __init__(self, wl, seed, dev):
+    def __init__(self, wl, seed, dev, token_range=None):
         import numpy as np
         import torch
         from paper_2608_04991_b200 import binding as rac
         from paper_2608_04991_b200 import synth
         self.rac, self.torch, self.wl, self.dev = rac, torch, wl, dev
         T, d, g = wl["T"], wl["d"], wl["group"]
+        self.a, self.b = 0, T
         self.cfg = rac.CodecCfg(d, g, wl["bits"], wl["topk"])
         self.rec = rac.rac_record_bytes(self.cfg)
         tw = synth.span_workload(wl["n_hist"], T, seed=seed, gap_max=wl["gap_max"])
@@ -175,6 +179,10 @@ class RoundTrip:
         torch.cuda.synchronize()
         self.coverage = float((self.ref_row >= 0).float().mean().item())
         self.np = np
+        # strong scaling: this rank codes tokens [a, b) of the one tensor (the set-up above ran over all of them, so
+        # every rank holds the same tables and the same downlink state)
+        self.a, self.b = (0, T) if token_range is None else token_range
+        self.shard_coverage = float((self.ref_row[self.a:self.b] >= 0).float().mean().item()) if self.b > self.a else 0.0
 
     # ---- the calls of one step, in order
     def match(self):
@@ -187,27 +195,28 @@ class RoundTrip:
         self.rac.rac_encode(self.cfg, self.X, w["T"], self.Hs, w["n_hist"], self.ref_row, None, None, self.step_up,
                             self.inv_up, self.pay_up, self.pay_up.numel(), self.ews, self.ews_bytes, self.status)
 
+    # the calls below work on this rank's token range [a, b) (all T tokens unless the run shards one tensor)
     def encode_sender_up(self):
         """Uplink encode that also leaves the sender-side x_hat (the next reference) in Xs."""
-        w = self.wl
-        self.rac.rac_encode_reconstruct(self.cfg, self.X, w["T"], self.Hs, w["n_hist"], self.ref_row, None, None,
-                                        self.step_up, self.inv_up, self.pay_up, self.pay_up.numel(), self.Xs, self.ews,
-                                        self.ews_bytes, self.status)
+        w, a, b, rec = self.wl, self.a, self.b, self.rec
+        self.rac.rac_encode_reconstruct(self.cfg, self.X[a:b], b - a, self.Hs, w["n_hist"], self.ref_row[a:b], None, None,
+                                        self.step_up, self.inv_up, self.pay_up[a * rec:b * rec], (b - a) * rec,
+                                        self.Xs[a:b], self.ews, self.ews_bytes, self.status)
 
     def decode_up(self):
-        w = self.wl
-        self.rac.rac_decode_reconstruct(self.cfg, self.pay_up, w["T"], self.Hs, w["n_hist"], self.ref_row, None, None,
-                                        self.step_up, self.Xh, self.status)
+        w, a, b, rec = self.wl, self.a, self.b, self.rec
+        self.rac.rac_decode_reconstruct(self.cfg, self.pay_up[a * rec:b * rec], b - a, self.Hs, w["n_hist"],
+                                        self.ref_row[a:b], None, None, self.step_up, self.Xh[a:b], self.status)
 
     def encode_dn(self):
-        w = self.wl
-        self.rac.rac_encode(self.cfg, self.Y, w["T"], self.Xh, w["T"], None, None, None, self.step_dn, self.inv_dn,
-                            self.pay_dn, self.pay_dn.numel(), self.ews, self.ews_bytes, self.status)
+        a, b, rec = self.a, self.b, self.rec
+        self.rac.rac_encode(self.cfg, self.Y[a:b], b - a, self.Xh[a:b], b - a, None, None, None, self.step_dn, self.inv_dn,
+                            self.pay_dn[a * rec:b * rec], (b - a) * rec, self.ews, self.ews_bytes, self.status)
 
     def decode_dn(self):
-        w = self.wl
-        self.rac.rac_decode_reconstruct(self.cfg, self.pay_dn, w["T"], self.Xh, w["T"], None, None, None, self.step_dn,
-                                        self.Yh, self.status)
+        a, b, rec = self.a, self.b, self.rec
+        self.rac.rac_decode_reconstruct(self.cfg, self.pay_dn[a * rec:b * rec], b - a, self.Xh[a:b], b - a, None, None, None,
+                                        self.step_dn, self.Yh[a:b], self.status)
 
     STAGES = ["match", "encode_sender_up", "decode_up", "encode_dn", "decode_dn"]
 
@@ -222,8 +231,8 @@ class RoundTrip:
     # ---- algorithmic bytes (what the method itself must move, per launch)
     def bytes_of(self, name):
         w = self.wl
-        T, d, rec = w["T"], w["d"], self.rec
-        refd = self.coverage
+        T, d, rec = self.b - self.a, w["d"], self.rec
+        refd = self.shard_coverage
         if name == "encode_up":
             return T * (2 * d + 2 * d * refd + rec + 4)
         if name == "encode_sender_up":
@@ -672,7 +681,21 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE {world}"
 
-    rt = RoundTrip(wl, seed=4 + rank, dev=dev)   # every rank codes its own sequences: no data-path collective
+    strong = args.scaling == "strong"
+    if strong:
+        # one tensor, the same on every rank; rank r codes the token range shard.token_range(T, r, world) against its
+        # own replica of the history states, and the payload byte ranges are gathered into every rank's own buffer
+        from paper_2608_04991_b200 import shard
+        rt = RoundTrip(wl, seed=4, dev=dev, token_range=shard.token_range(wl["T"], rank, world))
+        byte_ranges = [shard.payload_range(rt.rec, x, y) for x, y in shard.all_ranges(wl["T"], world)]
+
+        def exchange():
+            shard.all_gather_ranges(rt.pay_up, byte_ranges, rank)
+            shard.all_gather_ranges(rt.pay_dn, byte_ranges, rank)
+        rt.exchange = exchange
+        rt.STAGES = rt.STAGES + ["exchange"]
+    else:
+        rt = RoundTrip(wl, seed=4 + rank, dev=dev)   # every rank codes its own sequences: no data-path collective
     nst = len(rt.STAGES)
     steps, warm = args.steps, max(args.warmup, 3)
 
@@ -702,11 +725,25 @@ def main():
     total_ms = float(t.item())
     ms_per_step = total_ms / steps
     act = rt.activation_bytes_per_step()
-    value = world * act / (ms_per_step * 1e-3) / 1e9
+    value = (1 if strong else world) * act / (ms_per_step * 1e-3) / 1e9
+    strong_check = None
+    if strong:
+        # the gathered payloads against one rank coding the whole tensor (untimed)
+        got_up, got_dn = rt.pay_up.clone(), rt.pay_dn.clone()
+        mine = (rt.a, rt.b)
+        rt.a, rt.b = 0, wl["T"]
+        rt.encode_sender_up()
+        rt.decode_up()
+        rt.encode_dn()
+        torch.cuda.synchronize()
+        strong_check = bool(torch.equal(got_up, rt.pay_up) and torch.equal(got_dn, rt.pay_dn))
+        if not strong_check:
+            raise SystemExit(f"rank {rank}: the gathered payload differs from the single-rank payload")
+        rt.a, rt.b = mine
 
     # ---- end to end: inputs from pinned host memory, payloads and final activations back to the host
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not strong:     # the end-to-end number belongs to the default (weak) mode
         T, d = wl["T"], wl["d"]
         pin = lambda t_: torch.empty(t_.shape, dtype=t_.dtype, pin_memory=True).copy_(t_)
         hX, hY, hq = pin(rt.X), pin(rt.Y), pin(rt.query)
@@ -808,11 +845,12 @@ def main():
                    "one_thread": {"value": gbs1, "unit": UNIT, "cores": 1, "sample": desc1}}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None,
+            "strong_scaling_check": strong_check,
             "dtype": "f32", "data": "synthetic",
             "config": bench_config(wl, args.small),
             "workload_stats": {"record_bytes": rt.rec, "matched_coverage": rt.coverage, "planted_coverage": rt.planted_coverage,
-                               "tokens_per_s": world * wl["T"] / (ms_per_step * 1e-3)},
+                               "tokens_per_s": (1 if strong else world) * wl["T"] / (ms_per_step * 1e-3)},
             "clocks": sampler.summary(),
             "e2e": e2e,
             "gpu_launches": rt.LAUNCHES_PER_STEP * steps,

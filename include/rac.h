@@ -126,7 +126,11 @@ int rac_header_parse(const void *header /* host, 64 bytes */, rac_codec_cfg *cfg
  *   hist_tok   int32[n_hist]     history token ids (row j of the history state buffer belongs to token j)
  *   query_tok  int32[n_query]    tokens of the current prompt
  *   min_ngram  w, 1..32
- *   max_hits   K, 1..16
+ *   max_hits   K, 1..16; or 0 = no limit: every occurrence of a window is a candidate (the plain longest
+ *              match of the paper, the K-hit cap being a bucket policy).  The cost of a query position then
+ *              grows with the number of occurrences of its window times the length they match over, so a
+ *              history that repeats one token thousands of times is slow; keep the cap for token streams
+ *              you do not control.  The persistent index (rac_index_*) takes 1..16 only.
  *   ref_row    int32[n_query]    out: history row of every covered position, -1 elsewhere
  *   spans      rac_span[n_query/min_ngram + 1]  out, in query order; may be NULL
  *   n_spans    int32[1]          out (device)

@@ -37,6 +37,8 @@ struct MatchParams {
     int n_hist, n_query, nwin, w, K;
     unsigned int mask;     // M - 1
     const int32_t *end_of; // [n_hist] end of the request that holds each history position; null = one request
+    int32_t *next;         // [nwin]   unlimited hits (max_hits = 0) only: another start of the same window, -1 = none;
+                           //          top[slot] is then the head of the slot's chain (K = 1 entry per slot)
 };
 
 __device__ __forceinline__ unsigned int window_hash(const int32_t *tok, int w) {
@@ -76,6 +78,9 @@ __global__ void match_insert_kernel(MatchParams p) {
         s = (s + 1) & p.mask;
     }
     p.slot_of[j] = slot;  // the table has >= 2*nwin slots, so a slot is always found
+    // unlimited hits: every start of the window goes onto the slot's chain.  The order of a chain depends on which
+    // thread came first; the query looks at ALL of it and keeps lexargmax(length, start), so the result does not.
+    if (p.next && slot >= 0) p.next[j] = atomicExch(&p.top[slot], j);
 }
 
 // round r: the largest start of each window that is below the start found in round r-1
@@ -103,10 +108,8 @@ __global__ void match_query_kernel(MatchParams p) {
             s = (s + 1) & p.mask;
         }
         if (slot >= 0) {
-            const int32_t *lst = p.top + (long long)slot * p.K;
-            for (int r = 0; r < p.K; r++) {
-                int j = lst[r];
-                if (j < 0) break;
+            // candidate j: extend forward to the longest exact match, keep lexargmax(length, start)
+            auto consider = [&](int j) {
                 int L = p.w;
                 const int hend = p.end_of ? p.end_of[j] : p.n_hist;   // a match stays inside its request
                 // eight tokens per trip to memory: the loads of a trip are independent, and a long match is a chain
@@ -125,6 +128,21 @@ __global__ void match_query_kernel(MatchParams p) {
                 }
                 while (open && L < room && p.query[i + L] == p.hist[j + L]) L++;
                 if (L > bestL || (L == bestL && j > bestj)) { bestL = L; bestj = j; }
+            };
+            if (p.next) {
+                // every occurrence of the window (at most nwin of them: the walk is bounded by construction)
+                int j = p.top[slot];
+                for (int n = 0; j >= 0 && n < p.nwin; n++) {
+                    consider(j);
+                    j = p.next[j];
+                }
+            } else {
+                const int32_t *lst = p.top + (long long)slot * p.K;
+                for (int r = 0; r < p.K; r++) {
+                    const int j = lst[r];
+                    if (j < 0) break;
+                    consider(j);
+                }
             }
         }
     }
@@ -399,6 +417,56 @@ __global__ void index_append_round_kernel(IndexParams p, int r) {
     if (r == 0 || j < lst[r - 1]) atomicMax(&lst[r], j);
 }
 
+// The three steps above for a request small enough for ONE CTA, in one launch: the CTA's barriers stand where the
+// launch boundaries stood (every thread strides over the request's positions in every step).
+constexpr int kAppendFusedMax = 16384;   // tokens per request up to which the single-CTA form is used
+__global__ void __launch_bounds__(1024) index_append_fused_kernel(IndexParams p) {
+    const int n = p.b - p.a;
+    for (int o = threadIdx.x; o < n; o += blockDim.x) {
+        const int j = p.a + o;
+        p.end_of[j] = p.b;
+        if (j + p.w > p.b) continue;
+        const int32_t *win = p.hist + j;
+        unsigned int s = window_hash(win, p.w) & p.mask;
+        int slot = -1;
+        for (unsigned int probe = 0; probe <= p.mask; probe++) {
+            int cur = atomicCAS(&p.rep[s], -1, j);
+            if (cur == -1 || cur == j || same_window(p.hist + cur, win, p.w)) { slot = (int)s; break; }
+            s = (s + 1) & p.mask;
+        }
+        p.slot_of[j] = slot;
+        if (slot >= 0) atomicAdd(&p.cnt[slot], 1);
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < n; o += blockDim.x) {
+        const int j = p.a + o;
+        if (j + p.w > p.b) continue;
+        const int slot = p.slot_of[j];
+        if (slot < 0) continue;
+        const int c = atomicExch(&p.cnt[slot], 0);
+        if (c == 0) continue;
+        int32_t *lst = p.top + (long long)slot * p.K;
+        const int sh = c < p.K ? c : p.K;
+        for (int r = p.K - 1; r >= sh; r--) lst[r] = lst[r - sh];
+        for (int r = 0; r < sh; r++) lst[r] = -1;
+    }
+    for (int r = 0; r < p.K; r++) {
+        __syncthreads();
+        int any = 0;
+        for (int o = threadIdx.x; o < n; o += blockDim.x) {
+            const int j = p.a + o;
+            if (j + p.w > p.b) continue;
+            const int slot = p.slot_of[j];
+            if (slot < 0) continue;
+            int32_t *lst = p.top + (long long)slot * p.K;
+            if (r == 0 || j < lst[r - 1]) { atomicMax(&lst[r], j); any = 1; }
+        }
+        // a round in which no start was left to place is the last one that can change anything: most windows
+        // occur once in a request, so one or two rounds do
+        if (!__syncthreads_or(any)) break;
+    }
+}
+
 // Intra-sequence references: first occurrence of every token of the prompt (a hash table keyed by a position
 // whose token is the key, verified by comparing tokens), then the uncovered positions look theirs up.
 __global__ void intra_insert_kernel(const int32_t *query, int n, int32_t *trep, int32_t *tfirst, unsigned int mask) {
@@ -439,6 +507,21 @@ __global__ void fill2_i32_kernel(int32_t *a, long long na, int32_t va, int32_t *
 
 static size_t align16(size_t v) { return (v + 15) / 16 * 16; }
 
+// SMs of the current device (grids of the grid-stride kernels are sized from it); looked up once per device
+static int sm_count() {
+    static int cache[64];
+    static std::mutex m;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    std::lock_guard<std::mutex> lock(m);
+    if (cache[dev] == 0) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
+        cache[dev] = sms;
+    }
+    return cache[dev];
+}
+
 // the six launches of the selection (suffix scan and pointer doubling grid-wide, chain walk in one CTA, expansion
 // grid-wide)
 static int launch_selection(const MatchParams &p, cudaStream_t st) {
@@ -453,18 +536,21 @@ static int launch_selection(const MatchParams &p, cudaStream_t st) {
         cudaFuncSetAttribute(match_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
         return RAC_ECUDA;
     match_select_kernel<<<1, 1024, dyn, st>>>(p, window);
-    match_expand_kernel<<<148, 256, 0, st>>>(p);
+    match_expand_kernel<<<sm_count(), 256, 0, st>>>(p);
     return RAC_OK;
 }
 
 
 
 struct MatchLayout {
-    size_t rep, top, slot_of, best, hop, spans, chunk_first, delta16, jump2, jump4, total;
+    size_t rep, top, slot_of, best, hop, spans, chunk_first, delta16, jump2, jump4, next, total;
     unsigned int M;
 };
+// K = 0 (unlimited hits): one entry per slot (the head of its chain) and a chain link per history position
 static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
     MatchLayout L;
+    const bool chains = K == 0;
+    if (chains) K = 1;
     unsigned long long M = 1024;
     while (M < 2ull * (unsigned long long)(n_hist > 0 ? n_hist : 1)) M <<= 1;
     L.M = (unsigned int)M;
@@ -479,6 +565,7 @@ static MatchLayout match_layout(long long n_hist, long long n_query, int K) {
     L.delta16 = o;  o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 2);
     L.jump2 = o;    o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 4);
     L.jump4 = o;    o = align16(o + (size_t)(n_query > 0 ? n_query : 1) * 4);
+    L.next = o;     if (chains) o = align16(o + (size_t)(n_hist > 0 ? n_hist : 1) * 4);
     L.total = o;
     return L;
 }
@@ -514,7 +601,7 @@ using namespace rac;
 extern "C" {
 
 size_t rac_match_workspace_bytes(int64_t n_hist, int64_t n_query, int32_t max_hits) {
-    if (n_hist < 0 || n_query < 0 || max_hits < 1 || max_hits > 16) return 0;
+    if (n_hist < 0 || n_query < 0 || max_hits < 0 || max_hits > 16) return 0;
     if (n_hist >= (1ll << 30) || n_query >= (1ll << 30)) return 0;
     return match_layout(n_hist, n_query, max_hits).total;
 }
@@ -525,7 +612,7 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     if (n_hist < 0 || n_query < 0 || !n_spans) return RAC_EINVAL;
     if (n_hist >= (1ll << 30) || n_query >= (1ll << 30)) return RAC_EUNSUPPORTED;
     if (min_ngram < 1 || min_ngram > 32) return RAC_EUNSUPPORTED;
-    if (max_hits < 1 || max_hits > 16) return RAC_EUNSUPPORTED;
+    if (max_hits < 0 || max_hits > 16) return RAC_EUNSUPPORTED;
     if ((n_hist > 0 && !hist_tok) || (n_query > 0 && (!query_tok || !ref_row))) return RAC_EINVAL;
     if (!workspace) return RAC_EINVAL;
     if (reinterpret_cast<uintptr_t>(workspace) & 15u) return RAC_EALIGN;
@@ -554,20 +641,21 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     p.n_query = (int)n_query;
     p.nwin = (int)(n_hist - min_ngram + 1 > 0 ? n_hist - min_ngram + 1 : 0);
     p.w = min_ngram;
-    p.K = max_hits;
+    p.K = max_hits > 0 ? max_hits : 1;
+    p.next = max_hits == 0 ? reinterpret_cast<int32_t *>(ws + L.next) : nullptr;
     p.mask = L.M - 1;
 
-    const long long table_ints = (long long)L.M * (1 + max_hits);
+    const long long table_ints = (long long)L.M * (1 + p.K);
     const int tb = 256;
     long long work = table_ints > n_query ? table_ints : n_query;
     int init_blocks = (int)((work + tb - 1) / tb);
-    if (init_blocks > 148 * 8) init_blocks = 148 * 8;
+    if (init_blocks > sm_count() * 8) init_blocks = sm_count() * 8;
     if (init_blocks < 1) init_blocks = 1;
     match_init_kernel<<<init_blocks, tb, 0, st>>>(p, table_ints);
     if (p.nwin > 0 && n_query > 0) {
         int nb = (p.nwin + tb - 1) / tb;
         match_insert_kernel<<<nb, tb, 0, st>>>(p);
-        for (int r = 0; r < max_hits; r++) match_round_kernel<<<nb, tb, 0, st>>>(p, r);
+        for (int r = 0; r < max_hits; r++) match_round_kernel<<<nb, tb, 0, st>>>(p, r);   // none with chains
     }
     if (n_query > 0) {
         match_query_kernel<<<(int)((n_query + tb - 1) / tb), tb, 0, st>>>(p);
@@ -583,9 +671,9 @@ int rac_spans_to_rows(const rac_span *spans, const int32_t *n_spans, int64_t n_q
     if (n_query >= (1ll << 30)) return RAC_EUNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int blocks = (int)((n_query + 255) / 256);
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > sm_count() * 8) blocks = sm_count() * 8;
     fill_i32_kernel<<<blocks, 256, 0, st>>>(ref_row, n_query, -1);
-    spans_to_rows_kernel<<<148, 256, 0, st>>>(spans, n_spans, n_query, ref_row);
+    spans_to_rows_kernel<<<sm_count(), 256, 0, st>>>(spans, n_spans, n_query, ref_row);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
@@ -656,7 +744,7 @@ QueryLayout query_layout(long long n_query) {
 }
 int grid_for(long long n, int tb) {
     long long b = (n + tb - 1) / tb;
-    if (b > 148 * 16) b = 148 * 16;
+    if (b > (long long)sm_count() * 16) b = (long long)sm_count() * 16;
     return (int)(b < 1 ? 1 : b);
 }
 }  // namespace
@@ -704,6 +792,12 @@ int rac_index_append(const rac_index_cfg *cfg, void *index, size_t index_bytes, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int tb = 256;
     const int nb = (int)((n_after - n_before + tb - 1) / tb);
+    if (n_after - n_before <= kAppendFusedMax) {
+        // a request of ordinary size: one launch (the K + 2 launches below cost ~3 us each, which is all an append
+        // of a few thousand tokens costs)
+        index_append_fused_kernel<<<1, 1024, 0, st>>>(p);
+        return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+    }
     index_append_insert_kernel<<<nb, tb, 0, st>>>(p);
     if (n_after - n_before >= cfg->min_ngram) {
         index_append_shift_kernel<<<nb, tb, 0, st>>>(p);
@@ -755,6 +849,7 @@ int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_by
     p.w = cfg->min_ngram;
     p.K = cfg->max_hits;
     p.mask = L.M - 1;
+    p.next = nullptr;
     p.end_of = reinterpret_cast<const int32_t *>(ix + L.end_of);
     const int tb = 256;
     // rows to -1, span count to 0, and (for the intra-sequence pass) the token table to empty

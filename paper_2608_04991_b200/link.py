@@ -298,6 +298,9 @@ def _demo(argv=None) -> None:
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--group", type=int, default=128)
     ap.add_argument("--topk-group", type=int, default=1)
+    ap.add_argument("--check", action="store_true",
+                    help="fail (exit status 1) unless both ends hold the same reconstructed history at the end: their "
+                         "digests travel over the process group and are compared on both ranks")
     a = ap.parse_args(argv)
     rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
     if world != 2:
@@ -339,7 +342,10 @@ def _demo(argv=None) -> None:
                           "matched_fraction": st.matched_tokens / max(st.tokens, 1),
                           "references_in_step": int(both[0].item()) == int(both[1].item()),
                           "ms_total": t0.elapsed_time(t1)}))
+    in_step = int(both[0].item()) == int(both[1].item())
     dist.destroy_process_group()
+    if a.check and not in_step:
+        raise SystemExit(f"rank {rank}: sender and receiver histories differ")
 
 
 if __name__ == "__main__":

@@ -89,12 +89,14 @@ def test_host_side_rejections_happen_before_any_launch(rac):
     assert lib.rac_decode_reconstruct(C.byref(cfg), A, 4, A, 4, None, None, None, A, A + 4, None, 0) == -2
     # matcher
     assert rac.rac_match_workspace_bytes(1000, 100, 8) > 0
-    assert rac.rac_match_workspace_bytes(1000, 100, 0) == 0
+    # 0 = unlimited hits: one chain head per slot and a link per history position, less than any K-list
+    assert 0 < rac.rac_match_workspace_bytes(1000, 100, 0) < rac.rac_match_workspace_bytes(1000, 100, 1) + 4 * 1000 + 16
+    assert rac.rac_match_workspace_bytes(1000, 100, -1) == 0
     assert rac.rac_match_workspace_bytes(1000, 100, 17) == 0
     need = rac.rac_match_workspace_bytes(1000, 100, 8)
     m = lambda **kw: lib.rac_match_spans(kw.get("h", A), kw.get("nh", 1000), A, 100, kw.get("w", 4), kw.get("K", 8), A, None, A,
                                          kw.get("ws", A), kw.get("wsb", need), 0)
-    assert m(w=0) == -4 and m(K=0) == -4 and m(wsb=need - 1) == -3 and m(ws=A + 4) == -2 and m(h=None) == -1
+    assert m(w=0) == -4 and m(K=-1) == -4 and m(K=17) == -4 and m(wsb=need - 1) == -3 and m(ws=A + 4) == -2 and m(h=None) == -1
     assert rac.rac_strerror(-3) == "caller buffer too small"
     with pytest.raises(rac.RacError):
         rac._check("x", -1)

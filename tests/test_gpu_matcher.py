@@ -91,6 +91,49 @@ def test_frequent_window_cap(env):
     assert gpu_match(env, hist, query, 4, 12)[1].tolist() == [[0, 0, 9]]
 
 
+def test_unlimited_hits(env):
+    """max_hits = 0: every occurrence of a window is a candidate (Sec. IV-B.1's longest exact match without the
+    bucket cap).  Tiny random inputs, the adversarial token streams (one token everywhere: every position of the
+    history is a candidate of every query position), a window that occurs more often than any cap, and the two
+    workloads against the oracle's K = 0; at the long-context size the span list differs from the K = 8 one."""
+    orc = env.orc
+    rng = np.random.default_rng(77)
+    for trial in range(12):
+        vocab = [2, 3, 5, 50][trial % 4]
+        w = [1, 2, 3, 4, 6][trial % 5]
+        H, N = int(rng.integers(5, 400)), int(rng.integers(1, 300))
+        hist = rng.integers(0, vocab, H).astype(np.int32)
+        query = rng.integers(0, vocab, N).astype(np.int32)
+        rr, sp, _ = gpu_match(env, hist, query, w, 0)
+        o_rr, o_sp = orc.match_spans(hist, query, w, 0)
+        assert np.array_equal(rr, o_rr) and np.array_equal(sp, o_sp), (trial, H, N, w)
+    for hist, query, w in [(np.ones(700), np.ones(500), 4), (np.arange(500) % 7, np.arange(333) % 7, 4),
+                           (np.arange(64), np.arange(64), 4), (np.arange(3), np.arange(10), 4), (np.arange(0), np.arange(10), 4)]:
+        hist, query = hist.astype(np.int32), query.astype(np.int32)
+        rr, sp, _ = gpu_match(env, hist, query, w, 0)
+        o_rr, o_sp = orc.match_spans(hist, query, w, 0)
+        assert np.array_equal(rr, o_rr) and np.array_equal(sp, o_sp), (len(hist), len(query))
+    # a window with 20 occurrences, the OLDEST of which has the longest continuation: only K = 0 finds it
+    gram = np.array([1, 2, 3, 4], np.int32)
+    tail = np.array([50, 51, 52, 53, 54], np.int32)
+    parts = [gram, tail]
+    for _ in range(19):
+        parts += [rng.integers(100, 10000, 6).astype(np.int32), gram]
+    hist = np.concatenate(parts)
+    query = np.concatenate([gram, tail])
+    assert gpu_match(env, hist, query, 4, 0)[1].tolist() == [[0, 0, 9]]
+    assert gpu_match(env, hist, query, 4, 16)[1].tolist() != [[0, 0, 9]]
+    # the workloads
+    for n_hist, n_query, gap, seed in [(32768, 2048, 176, 1), (131072, 131072, 112, 4)]:
+        wl = env.synth.span_workload(n_hist, n_query, seed=seed, gap_max=gap)
+        rr, sp, ns = gpu_match(env, wl.hist, wl.query, 4, 0)
+        o_rr, o_sp = orc.match_spans(wl.hist, wl.query, 4, 0)
+        assert ns == len(o_sp) and np.array_equal(sp, o_sp) and np.array_equal(rr, o_rr)
+        o8_rr, o8_sp = orc.match_spans(wl.hist, wl.query, 4, 8)
+        print(f"{n_hist}/{n_query}: {ns} spans without a cap, {len(o8_sp)} with 8 hits, rows differ at "
+              f"{int((o8_rr != o_rr).sum())} positions")
+
+
 @pytest.mark.parametrize("n_hist,n_query,gap,seed", [(32768, 2048, 176, 1), (131072, 131072, 112, 4), (5000, 70001, 60, 9)])
 def test_workload_sizes(env, n_hist, n_query, gap, seed):
     wl = env.synth.span_workload(n_hist, n_query, seed=seed, gap_max=gap)

@@ -35,17 +35,20 @@ def _worker(rank, world, port, T, d, g, bits, k, out_dir):
     R = synth.affine_noisy_reference(X, g, gen)
     step = np.full((2, d), 0.02, np.float32)
     inv = (np.float32(1) / step).astype(np.float32)
-    a, b = shard.token_range(T, rank, world)
     rec = oracle.record_bytes(d, g, bits, k)
-    mine = oracle.encode(d, g, bits, k, synth.bf16_bits(X[a:b]), ref_base=synth.bf16_bits(R[a:b]), step=step, inv_step=inv)
-    assert mine.size == shard.payload_range(rec, a, b)[1] - shard.payload_range(rec, a, b)[0]
-    # exchange: every rank learns every shard (sizes differ by one record at most, so pad to the largest)
-    biggest = max(y - x for x, y in shard.all_ranges(T, world)) * rec
-    buf = torch.zeros(biggest, dtype=torch.uint8)
-    buf[: mine.size] = torch.from_numpy(mine)
-    got = [torch.zeros(biggest, dtype=torch.uint8) for _ in range(world)]
-    dist.all_gather(got, buf)
-    full = np.concatenate([got[r][: (y - x) * rec].numpy() for r, (x, y) in enumerate(shard.all_ranges(T, world))])
+    # the function the benchmark's strong-scaling mode uses: code the own token range into the own byte range of a
+    # full-length buffer, then exchange the byte ranges
+    payload = torch.zeros(T * rec, dtype=torch.uint8)
+
+    def encode_range(a, b):
+        mine = oracle.encode(d, g, bits, k, synth.bf16_bits(X[a:b]), ref_base=synth.bf16_bits(R[a:b]), step=step, inv_step=inv)
+        lo, hi = shard.payload_range(rec, a, b)
+        assert mine.size == hi - lo
+        payload[lo:hi] = torch.from_numpy(mine)
+
+    a, b = shard.sharded_encode(encode_range, T, rec, payload, rank, world)
+    assert (a, b) == shard.token_range(T, rank, world)
+    full = payload.numpy()
     # max-over-ranks reduction as the benchmark does for its timing
     t = torch.tensor([float(rank + 1)])
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
