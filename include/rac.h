@@ -269,6 +269,19 @@ int rac_encode_reconstruct(const rac_codec_cfg *cfg, const void *X, int64_t T,
                            void *payload, size_t payload_cap, void *X_hat, void *workspace, size_t workspace_bytes,
                            uint32_t *dev_status, void *stream);
 
+/* Self-test of the bounded waits (the paper has no counterpart: it is about this library's failure handling).
+ * Every wait of the streaming kernels on an mbarrier gives up after a fixed number of polls, sets
+ * RAC_STATUS_TIMEOUT in *dev_status and lets the kernel return normally, so that a copy that never lands cannot
+ * hang the GPU.  This call runs rac_encode (which = 0: `in` = X bf16[T,d], `out` = payload) or
+ * rac_decode_reconstruct (which = 1: `in` = payload, `out` = X_hat bf16[T,d], out_cap in bytes) on at most 1024
+ * tokens with identity rows, with every stage announcing 16 bytes more than its copies deliver and the poll limit
+ * lowered to 2048: no wait can complete, every CTA takes the give-up path (a few milliseconds).  Expected: RAC_OK
+ * from the call, RAC_STATUS_TIMEOUT in *dev_status, `out` unspecified, and the stream usable afterwards.  Nothing
+ * faults and nothing waits without a bound. */
+int rac_selftest_bounded_wait(const rac_codec_cfg *cfg, int32_t which, const void *in, int64_t T, const void *ref_base,
+                              int64_t ref_rows, const float *step, const float *inv_step, void *out, size_t out_cap,
+                              void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream);
+
 /* Receiver reconstruction (Eq. 9): X_hat = bf16( (alpha*r + beta) + e_hat ), e_hat = code*step or the
  * stored binary16 outlier.  Arguments as rac_encode.  X_hat bf16[T,d] must not overlap payload.  X_hat
  * may be the very buffer that ref_base points to ONLY with ref_row == NULL (token t reads row t and

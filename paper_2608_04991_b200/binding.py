@@ -37,6 +37,7 @@ EXPORTS = [
     "rac_fit_segments_workspace_bytes", "rac_fit_segments", "rac_spans_to_segments",
     "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
     "rac_recon_error_workspace_bytes", "rac_recon_error",
+    "rac_selftest_bounded_wait",
 ]
 
 
@@ -123,6 +124,8 @@ def load() -> C.CDLL:
         f = getattr(l, name)
         f.restype = C.c_int
         f.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, vp, vp]
+    l.rac_selftest_bounded_wait.restype = C.c_int
+    l.rac_selftest_bounded_wait.argtypes = [cfgp, i32, vp, i64, vp, i64, vp, vp, vp, sz, vp, sz, vp, vp]
     l.rac_split_waves.restype = C.c_int
     l.rac_split_waves.argtypes = [vp, i64, i64, vp, vp, vp, vp]
     l.rac_encode_reconstruct_list.restype = C.c_int
@@ -402,6 +405,17 @@ def rac_sender_reconstruct(cfg, payload, T, ref_base, ref_rows, ref_row, ref_gai
                            dev_status, stream=None) -> None:
     _reconstruct("rac_sender_reconstruct", cfg, payload, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step,
                  X_hat, dev_status, stream)
+
+
+def rac_selftest_bounded_wait(cfg, which, inp, T, ref_base, ref_rows, step, inv_step, out, out_cap, workspace,
+                              workspace_bytes, dev_status, stream=None) -> None:
+    """Runs the encode (which=0) or reconstruction (which=1) kernels with waits that cannot complete; see rac.h."""
+    rc = load().rac_selftest_bounded_wait(C.byref(cfg), int(which), _ptr(inp, None, "in"), int(T),
+                                          _ptr(ref_base, _BF16, "ref_base"), int(ref_rows), _ptr(step, _F32, "step"),
+                                          _ptr(inv_step, _F32, "inv_step"), _ptr(out, None, "out"), int(out_cap),
+                                          _ptr(workspace, None, "workspace"), int(workspace_bytes),
+                                          _ptr(dev_status, _I32, "dev_status"), _stream() if stream is None else stream)
+    _check("rac_selftest_bounded_wait", rc)
 
 
 def rac_calibrate_steps(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, clip_sigmas, step, inv_step,

@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
                               resolve_row<SUB>(p, next_raw), p.X + tk * d, row_bytes);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
-        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity, p.wait_polls);
         if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
         const bool has_ref = ctrl->row[stage] >= 0;
         const long long tok = ctrl->tok[stage];
@@ -215,8 +215,8 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
     if (MOMENTS) {
         if (tid == 0 && aborted) {
             for (int s = 0; s < S; s++) {
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0, p.wait_polls);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1, p.wait_polls);
             }
         }
         return;
@@ -237,8 +237,8 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
         if (aborted) {
             // give copies that may still be in flight a bounded chance to land before the CTA retires
             for (int s = 0; s < S; s++) {
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0, p.wait_polls);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1, p.wait_polls);
             }
         }
     }
@@ -306,7 +306,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         ctrl->row[s] = row;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
         const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
-        mbar_arrive_expect_tx(bar, row_bytes + (row >= 0 ? row_bytes : 0u));
+        mbar_arrive_expect_tx(bar, p.test_extra_tx + row_bytes + (row >= 0 ? row_bytes : 0u));
         bulk_load(base, p.X + t * d, row_bytes, bar);
         if (row >= 0) bulk_load(base + row_bytes, ref_row_ptr<SUB>(p, row), row_bytes, bar);
     };
@@ -345,7 +345,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
         unsigned char *rec = stg + L.rec_off + parity * p.rec;
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity, p.wait_polls))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
         if (valid) {
@@ -479,7 +479,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             const int k_next = it + S;
             int raw_next = 0;
             if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);  // in flight while the tail runs
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity, p.wait_polls))) { timed_out = true; break; }
             // ---- refill the stage, then hand the record to the copy engine.  The record sits in the slot of the
             // stage's current parity; the stage's next token writes the other slot, and the one after that
             // cannot start before this warp has arrived for the token in between, which it does only after the
@@ -516,8 +516,8 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
         // give copies that may still be in flight a bounded chance to land before the CTA retires
         for (int s = 0; s < S; s++) {
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0, p.wait_polls);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1, p.wait_polls);
         }
     }
 }
@@ -951,7 +951,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
                               resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
-        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity, p.wait_polls);
         if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
         const bool has_ref = ctrl->row[stage] >= 0;
         const unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
@@ -1057,8 +1057,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
         bulk_wait_all();
         if (aborted) {
             for (int s = 0; s < S; s++) {
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0, p.wait_polls);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1, p.wait_polls);
             }
         }
     }
@@ -1124,7 +1124,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
         ctrl->row[s] = row;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
         const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
-        mbar_arrive_expect_tx(bar, (uint32_t)p.rec + (row >= 0 ? row_bytes : 0u));
+        mbar_arrive_expect_tx(bar, p.test_extra_tx + (uint32_t)p.rec + (row >= 0 ? row_bytes : 0u));
         bulk_load(base, p.payload + t * p.rec, (uint32_t)p.rec, bar);
         if (row >= 0) bulk_load(base + L.rec_pad, ref_row_ptr<SUB>(p, row), row_bytes, bar);
     };
@@ -1189,7 +1189,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
         unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = sbase + L.stage0 + stage * L.stage_bytes + L.rec_pad;
         const uint32_t os = KT > 0 ? rs + row_bytes : rs;     // where x_hat goes: its own row, or over the reference
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity, p.wait_polls))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
         if (valid) {
@@ -1290,7 +1290,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
                 if (ok && (31 - __clz(same)) == lane) patch_c = c;
                 if (__any_sync(0xffffffffu, c >= d) && lane == 0 && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
             }
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity, p.wait_polls))) { timed_out = true; break; }
             if (KT > 0) {
                 if (patch_c >= 0)
                     reinterpret_cast<unsigned short *>(rec + L.rec_pad + row_bytes)[patch_c] = patch_x;
@@ -1317,8 +1317,8 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
     if (lane == 0) bulk_wait_all();
     if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
         for (int s = 0; s < S; s++) {
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0, p.wait_polls);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1, p.wait_polls);
         }
     }
 }
@@ -1360,6 +1360,8 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     p->codes_off = g.codes_off;
     p->goff_off = g.goff_off;
     p->gval_off = g.gval_off;
+    p->wait_polls = kWaitPolls;
+    p->test_extra_tx = 0;
     return RAC_OK;
 }
 
@@ -1672,10 +1674,15 @@ static int apply_subset(const Subset &sub, CodecParams *p) {
     return RAC_OK;
 }
 
+// test hook of rac_selftest_bounded_wait: a poll limit and bytes announced beyond what a stage's copies deliver
+struct WaitTest {
+    uint32_t polls, extra_tx;
+};
+
 static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64_t T, const void *ref_base,
                             int64_t ref_rows, const int32_t *ref_row, const void *gain, const void *bias,
                             const float *step, void *X_hat, uint32_t *dev_status, void *stream,
-                            const Subset &sub = Subset()) {
+                            const Subset &sub = Subset(), const WaitTest *wt = nullptr) {
     Geometry g;
     int rc = make_geometry(cfg, &g);
     if (rc != RAC_OK) return rc;
@@ -1691,6 +1698,7 @@ static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64
     p.payload = const_cast<uint8_t *>(static_cast<const uint8_t *>(payload));
     p.X_hat = static_cast<uint16_t *>(X_hat);
     p.step = step;
+    if (wt) { p.wait_polls = wt->polls; p.test_extra_tx = wt->extra_tx; }
     return launch_decode(g, p, static_cast<cudaStream_t>(stream));
 }
 
@@ -1799,7 +1807,8 @@ static bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb) {
 static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
                        const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const float *step,
                        const float *inv_step, void *payload, size_t payload_cap, void *X_hat, void *workspace,
-                       size_t workspace_bytes, uint32_t *dev_status, void *stream, const Subset &sub = Subset()) {
+                       size_t workspace_bytes, uint32_t *dev_status, void *stream, const Subset &sub = Subset(),
+                       const WaitTest *wt = nullptr) {
     Geometry g;
     int rc = make_geometry(cfg, &g);
     if (rc != RAC_OK) return rc;
@@ -1836,6 +1845,7 @@ static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const
     p.step = step;
     p.inv_step = inv_step;
     p.tmax = static_cast<float *>(workspace);
+    if (wt) { p.wait_polls = wt->polls; p.test_extra_tx = wt->extra_tx; }
     return launch_encode(g, p, T, static_cast<cudaStream_t>(stream));
 }
 
@@ -1854,6 +1864,23 @@ int rac_encode_reconstruct(const rac_codec_cfg *cfg, const void *X, int64_t T, c
     if (T > 0 && !X_hat) return RAC_EINVAL;
     return encode_impl(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, step, inv_step, payload, payload_cap,
                        X_hat, workspace, workspace_bytes, dev_status, stream);
+}
+
+int rac_selftest_bounded_wait(const rac_codec_cfg *cfg, int32_t which, const void *in, int64_t T, const void *ref_base,
+                              int64_t ref_rows, const float *step, const float *inv_step, void *out, size_t out_cap,
+                              void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream) {
+    if (T < 1 || T > 1024 || !dev_status) return RAC_EINVAL;
+    const WaitTest wt = {2048u, 16u};   // every stage announces 16 bytes that never come; a wait gives up after 2048 polls
+    if (which == 0)
+        return encode_impl(cfg, in, T, ref_base, ref_rows, nullptr, nullptr, nullptr, step, inv_step, out, out_cap, nullptr,
+                           workspace, workspace_bytes, dev_status, stream, Subset(), &wt);
+    if (which == 1) {
+        const size_t need = rac_record_bytes(cfg) ? (size_t)T * (size_t)cfg->d * 2 : 0;
+        if (need == 0 || out_cap < need) return need == 0 ? RAC_EINVAL : RAC_ESIZE;
+        return reconstruct_impl(cfg, in, T, ref_base, ref_rows, nullptr, nullptr, nullptr, step, out, dev_status, stream,
+                                Subset(), &wt);
+    }
+    return RAC_EINVAL;
 }
 
 int rac_decode_reconstruct(const rac_codec_cfg *cfg, const void *payload, int64_t T, const void *ref_base,

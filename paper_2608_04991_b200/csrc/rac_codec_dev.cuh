@@ -47,6 +47,9 @@ struct CodecParams {
     float4 *moments;             // segment fit, first pass out: (mean r, mean h, Sxx, Sxy) per (token, group)
     // scale_mode 1 only: quantisation groups, per-group outliers, field offsets in the record
     int Jq, lpq, lpq_shift, kg, scale_off, codes_off, goff_off, gval_off;
+    // bounded waits: polls before a wait on an mbarrier gives up (kWaitPolls), and -- only from rac_selftest_bounded_wait
+    // -- bytes announced on top of what the copies of a stage deliver, so that the wait cannot complete
+    uint32_t wait_polls, test_extra_tx;
 };
 
 // scale_mode 1 (defined in rac_codec_dyn.cu)
@@ -244,7 +247,7 @@ __device__ __forceinline__ void issue_token_loads(const CodecParams &p, Ctrl *ct
     if constexpr (SUB) ctrl->seg[stage] = p.seg_of ? p.seg_of[tok] : 0;
     const uint32_t bar = smem_u32(&ctrl->bar[stage]);
     const uint32_t row_bytes = 2u * (uint32_t)p.d;
-    mbar_arrive_expect_tx(bar, first_bytes + (row >= 0 ? row_bytes : 0u));
+    mbar_arrive_expect_tx(bar, p.test_extra_tx + first_bytes + (row >= 0 ? row_bytes : 0u));
     bulk_load(stage_addr, first_src, first_bytes, bar);
     if (row >= 0) bulk_load(stage_addr + r_off, ref_row_ptr<SUB>(p, row), row_bytes, bar);
 }

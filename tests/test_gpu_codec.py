@@ -250,6 +250,47 @@ def test_fused_sender_in_place_with_outliers_is_refused(env):
     assert np.array_equal(o_x, s.bf16_bits(xs))
 
 
+@pytest.mark.parametrize("d,bits,k,kg", [(5120, 4, 8, -1), (4096, 3, 0, -1), (96, 2, 0, -1), (5120, 4, 0, 1), (4096, 8, 0, 0)])
+def test_waits_that_cannot_complete_give_up_and_leave_the_stream_usable(env, d, bits, k, kg):
+    """The give-up path of the bounded waits, run on purpose in its safe form: every stage announces more bytes than
+    its copies deliver and the poll limit is lowered, so each CTA's wait runs out, the kernel sets RAC_STATUS_TIMEOUT
+    and returns.  Nothing faults, nothing spins without a bound; the next ordinary calls on the same stream give the
+    bits they always give."""
+    g, T = 32 if d == 96 else 128, 40
+    rac, P, dev = env.rac, env.P, env.dev
+    X, R, cal, calr = prefill_inputs(env, T, d, g, seed=91)
+    if kg < 0:      # the static table
+        step, inv = oracle_tables(env, d, g, bits, cal, calr)
+        step_d, inv_d = P.to_dev(step, dev), P.to_dev(inv, dev)
+        cfg = rac.CodecCfg(d, g, bits, k)
+    else:           # Eq. 8 as printed: scales in the record, kg outliers per group
+        step_d = inv_d = None
+        cfg = rac.CodecCfg(d, g, bits, 0, scale_mode=1, topk_group=kg)
+    rec = rac.rac_record_bytes(cfg)
+    good, st = P.gpu_encode(cfg, X, R, None, None, None, step_d, inv_d)
+    assert st == 0
+    good_x, st = P.gpu_decode(cfg, good, T, R, None, None, None, step_d, dev)
+    assert st == 0
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    ws = torch.zeros(max(nws, 16), dtype=torch.uint8, device=dev)
+    for which in (0, 1):
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        if which == 0:
+            out = torch.zeros(T * rec, dtype=torch.uint8, device=dev)
+            rac.rac_selftest_bounded_wait(cfg, 0, X, T, R, T, step_d, inv_d, out, out.numel(), ws if nws else None, nws, status)
+        else:
+            out = torch.zeros((T, d), dtype=torch.bfloat16, device=dev)
+            rac.rac_selftest_bounded_wait(cfg, 1, torch.from_numpy(good).to(dev), T, R, T, step_d, None, out,
+                                          out.numel() * 2, None, 0, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) & rac.STATUS_TIMEOUT, f"which={which}: status {int(status.item())}"
+        # the same stream, right afterwards: ordinary calls, ordinary results
+        again, st = P.gpu_encode(cfg, X, R, None, None, None, step_d, inv_d)
+        assert st == 0 and np.array_equal(again, good)
+        again_x, st = P.gpu_decode(cfg, good, T, R, None, None, None, step_d, dev)
+        assert st == 0 and torch.equal(again_x, good_x)
+
+
 def test_zero_tokens_is_a_no_op(env):
     cfg = env.rac.CodecCfg(4096, 128, 4, 8)
     t = torch.zeros(16, dtype=torch.uint8, device=env.dev)
