@@ -28,8 +28,7 @@
  *                        thing the codec needs as an input: a per-channel step
  *                        from the RMS of the aligned residual.
  *
- * Readings taken where the paper is silent (each is also listed in the design
- * notes of the repository):
+ * Readings taken where the paper is silent:
  *   - one fit per (token, group): the "fitting positions" of Eq. 6 are the
  *     channels of one group of one token;
  *   - Round_wire of the coefficients is IEEE binary16 round-to-nearest-even,

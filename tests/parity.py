@@ -363,7 +363,7 @@ def round_trip_case(cfg, X, ref_base=None, ref_row=None, gain=None, bias=None, s
     o_xo = oracle.reconstruct(d, g, bits, k, o_pay, T, ref_base=Rb, ref_row=rr, gain=gb, bias=bb, step=step,
                               nthreads=oracle.max_threads(), **mk)
     assert st == 0 and np.array_equal(o_xo, synth.bf16_bits(xo)), "device decode of the oracle payload differs"
-    # spec tolerance on the end-to-end activations where no coefficient flipped (implied by the above,
+    # the stated tolerance on the end-to-end activations where no coefficient flipped (implied by the above,
     # stated explicitly): abs 2e-2 / rel 1e-2
     a, b = synth.bf16_from_bits(o_xo).float(), xr.float().cpu()
     if rep.tokens_with_flip == 0:
