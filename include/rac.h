@@ -274,8 +274,8 @@ int rac_encode_reconstruct(const rac_codec_cfg *cfg, const void *X, int64_t T,
  * RAC_STATUS_TIMEOUT in *dev_status and lets the kernel return normally, so that a copy that never lands cannot
  * hang the GPU.  This call runs rac_encode (which = 0: `in` = X bf16[T,d], `out` = payload) or
  * rac_decode_reconstruct (which = 1: `in` = payload, `out` = X_hat bf16[T,d], out_cap in bytes) on at most 1024
- * tokens with identity rows, with every stage announcing 16 bytes more than its copies deliver and the poll limit
- * lowered to 2048: no wait can complete, every CTA takes the give-up path (a few milliseconds).  Expected: RAC_OK
+ * tokens with identity rows, with every stage announcing 16 bytes more than its copies deliver: no wait can
+ * complete, every CTA polls its limit out and takes the give-up path (well under a second per wait).  Expected: RAC_OK
  * from the call, RAC_STATUS_TIMEOUT in *dev_status, `out` unspecified, and the stream usable afterwards.  Nothing
  * faults and nothing waits without a bound. */
 int rac_selftest_bounded_wait(const rac_codec_cfg *cfg, int32_t which, const void *in, int64_t T, const void *ref_base,

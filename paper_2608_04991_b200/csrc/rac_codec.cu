@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
                               resolve_row<SUB>(p, next_raw), p.X + tk * d, row_bytes);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
-        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity, p.wait_polls);
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
         if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
         const bool has_ref = ctrl->row[stage] >= 0;
         const long long tok = ctrl->tok[stage];
@@ -215,8 +215,8 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
     if (MOMENTS) {
         if (tid == 0 && aborted) {
             for (int s = 0; s < S; s++) {
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0, p.wait_polls);
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1, p.wait_polls);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
             }
         }
         return;
@@ -237,8 +237,8 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
         if (aborted) {
             // give copies that may still be in flight a bounded chance to land before the CTA retires
             for (int s = 0; s < S; s++) {
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0, p.wait_polls);
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1, p.wait_polls);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
             }
         }
     }
@@ -277,7 +277,9 @@ __host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages, boo
 }
 
 // SUB: the token-list / second-reference-buffer form (see rac_codec_dev.cuh).
-template <int BITS, bool TOPK, bool XHAT, int MINB, bool SUB>
+// LPG: lanes per alignment group as a compile-time constant (4 = groups of 128 channels, 2 = groups of 64), or 0 to
+// read it from the parameters; the constant removes the uniform branches of the shuffle reductions.
+template <int BITS, bool TOPK, bool XHAT, int MINB, bool SUB, int LPG = 0>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -345,7 +347,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
         unsigned char *rec = stg + L.rec_off + parity * p.rec;
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity, p.wait_polls))) { timed_out = true; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
         if (valid) {
@@ -374,10 +376,12 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             // ---- (2) Eq. 6 and wire rounding
             u64 a2, b2;
             uint32_t coef_word;
-            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
+            constexpr int kShift = LPG == 4 ? 2 : 1;
+            const int lpg = LPG ? LPG : p.lpg, lpg_shift = LPG ? kShift : p.lpg_shift;
+            fit_group(x2, r2, has_ref, lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
 
             // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
-            if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
+            if ((lane & (lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> lpg_shift] = coef_word;
             const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
             const float *step_tab = p.step + (has_ref ? 0 : d);
             uint32_t words[4];
@@ -479,7 +483,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             const int k_next = it + S;
             int raw_next = 0;
             if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);  // in flight while the tail runs
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity, p.wait_polls))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
             // ---- refill the stage, then hand the record to the copy engine.  The record sits in the slot of the
             // stage's current parity; the stage's next token writes the other slot, and the one after that
             // cannot start before this warp has arrived for the token in between, which it does only after the
@@ -516,8 +520,8 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
         // give copies that may still be in flight a bounded chance to land before the CTA retires
         for (int s = 0; s < S; s++) {
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0, p.wait_polls);
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1, p.wait_polls);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
         }
     }
 }
@@ -951,7 +955,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
                               resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
-        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity, p.wait_polls);
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
         if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
         const bool has_ref = ctrl->row[stage] >= 0;
         const unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
@@ -1057,8 +1061,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
         bulk_wait_all();
         if (aborted) {
             for (int s = 0; s < S; s++) {
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0, p.wait_polls);
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1, p.wait_polls);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
             }
         }
     }
@@ -1189,7 +1193,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
         unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = sbase + L.stage0 + stage * L.stage_bytes + L.rec_pad;
         const uint32_t os = KT > 0 ? rs + row_bytes : rs;     // where x_hat goes: its own row, or over the reference
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity, p.wait_polls))) { timed_out = true; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
         if (valid) {
@@ -1290,7 +1294,7 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
                 if (ok && (31 - __clz(same)) == lane) patch_c = c;
                 if (__any_sync(0xffffffffu, c >= d) && lane == 0 && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
             }
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity, p.wait_polls))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
             if (KT > 0) {
                 if (patch_c >= 0)
                     reinterpret_cast<unsigned short *>(rec + L.rec_pad + row_bytes)[patch_c] = patch_x;
@@ -1317,8 +1321,8 @@ __global__ void __launch_bounds__(256, 2) decode_ws_kernel(const CodecParams p) 
     if (lane == 0) bulk_wait_all();
     if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
         for (int s = 0; s < S; s++) {
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0, p.wait_polls);
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1, p.wait_polls);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
         }
     }
 }
@@ -1360,7 +1364,6 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     p->codes_off = g.codes_off;
     p->goff_off = g.goff_off;
     p->gval_off = g.gval_off;
-    p->wait_polls = kWaitPolls;
     p->test_extra_tx = 0;
     return RAC_OK;
 }
@@ -1394,16 +1397,19 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     const bool tight = g.nthreads > 96 && g.nthreads <= 160 && !p.X_hat;
     int rc = RAC_EUNSUPPORTED;
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;   // the subset form has one variant per width: it is not the hot path
-#define RAC_ENC2(B, K, X)                                                                                          \
-    (sub ? launch_persistent(encode_ws_kernel<B, K, X, 2, true>, p, g.nthreads, L.total, max_ctas, stream)        \
-     : tight ? launch_persistent(encode_ws_kernel<B, K, X, 4, false>, p, g.nthreads, L.total, max_ctas, stream)   \
-             : launch_persistent(encode_ws_kernel<B, K, X, 2, false>, p, g.nthreads, L.total, max_ctas, stream))
+#define RAC_ENC3(B, K, X, G)                                                                                          \
+    (tight ? launch_persistent(encode_ws_kernel<B, K, X, 4, false, G>, p, g.nthreads, L.total, max_ctas, stream)   \
+           : launch_persistent(encode_ws_kernel<B, K, X, 2, false, G>, p, g.nthreads, L.total, max_ctas, stream))
+#define RAC_ENC2(B, K, X)                                                                                           \
+    (sub ? launch_persistent(encode_ws_kernel<B, K, X, 2, true, 0>, p, g.nthreads, L.total, max_ctas, stream)      \
+     : g.lpg == 4 ? RAC_ENC3(B, K, X, 4) : g.lpg == 2 ? RAC_ENC3(B, K, X, 2) : RAC_ENC3(B, K, X, 0))
 #define RAC_ENC(B, K) (p.X_hat ? RAC_ENC2(B, K, true) : RAC_ENC2(B, K, false))
     switch (g.bits) {
         case 4: rc = topk ? RAC_ENC(4, true) : RAC_ENC(4, false); break;
         case 3: rc = topk ? RAC_ENC(3, true) : RAC_ENC(3, false); break;
         case 2: rc = topk ? RAC_ENC(2, true) : RAC_ENC(2, false); break;
     }
+#undef RAC_ENC3
 #undef RAC_ENC2
 #undef RAC_ENC
     if (rc != RAC_OK || !topk) return rc;
@@ -1674,9 +1680,9 @@ static int apply_subset(const Subset &sub, CodecParams *p) {
     return RAC_OK;
 }
 
-// test hook of rac_selftest_bounded_wait: a poll limit and bytes announced beyond what a stage's copies deliver
+// test hook of rac_selftest_bounded_wait: bytes announced beyond what a stage's copies deliver
 struct WaitTest {
-    uint32_t polls, extra_tx;
+    uint32_t extra_tx;
 };
 
 static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64_t T, const void *ref_base,
@@ -1698,7 +1704,7 @@ static int reconstruct_impl(const rac_codec_cfg *cfg, const void *payload, int64
     p.payload = const_cast<uint8_t *>(static_cast<const uint8_t *>(payload));
     p.X_hat = static_cast<uint16_t *>(X_hat);
     p.step = step;
-    if (wt) { p.wait_polls = wt->polls; p.test_extra_tx = wt->extra_tx; }
+    if (wt) p.test_extra_tx = wt->extra_tx;
     return launch_decode(g, p, static_cast<cudaStream_t>(stream));
 }
 
@@ -1845,7 +1851,7 @@ static int encode_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const
     p.step = step;
     p.inv_step = inv_step;
     p.tmax = static_cast<float *>(workspace);
-    if (wt) { p.wait_polls = wt->polls; p.test_extra_tx = wt->extra_tx; }
+    if (wt) p.test_extra_tx = wt->extra_tx;
     return launch_encode(g, p, T, static_cast<cudaStream_t>(stream));
 }
 
@@ -1870,7 +1876,7 @@ int rac_selftest_bounded_wait(const rac_codec_cfg *cfg, int32_t which, const voi
                               int64_t ref_rows, const float *step, const float *inv_step, void *out, size_t out_cap,
                               void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream) {
     if (T < 1 || T > 1024 || !dev_status) return RAC_EINVAL;
-    const WaitTest wt = {2048u, 16u};   // every stage announces 16 bytes that never come; a wait gives up after 2048 polls
+    const WaitTest wt = {16u};   // every stage announces 16 bytes that never come
     if (which == 0)
         return encode_impl(cfg, in, T, ref_base, ref_rows, nullptr, nullptr, nullptr, step, inv_step, out, out_cap, nullptr,
                            workspace, workspace_bytes, dev_status, stream, Subset(), &wt);

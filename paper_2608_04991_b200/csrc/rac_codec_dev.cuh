@@ -47,9 +47,9 @@ struct CodecParams {
     float4 *moments;             // segment fit, first pass out: (mean r, mean h, Sxx, Sxy) per (token, group)
     // scale_mode 1 only: quantisation groups, per-group outliers, field offsets in the record
     int Jq, lpq, lpq_shift, kg, scale_off, codes_off, goff_off, gval_off;
-    // bounded waits: polls before a wait on an mbarrier gives up (kWaitPolls), and -- only from rac_selftest_bounded_wait
-    // -- bytes announced on top of what the copies of a stage deliver, so that the wait cannot complete
-    uint32_t wait_polls, test_extra_tx;
+    // only from rac_selftest_bounded_wait: bytes announced on top of what the copies of a stage deliver, so that the
+    // (bounded) wait for them cannot complete
+    uint32_t test_extra_tx;
 };
 
 // scale_mode 1 (defined in rac_codec_dyn.cu)

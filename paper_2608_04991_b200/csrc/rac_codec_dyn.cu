@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
         unsigned char *rec = stg + L.rec_off + parity * p.rec;
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity, p.wait_polls))) { timed_out = true; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
         u64 e2[16];        // Eq. 7 residual of this thread's channels, packed pairs in slot order
@@ -301,7 +301,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                 ctrl->wmax[stage][warp] = m;
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&ctrl->tokmax[stage])) : "memory");
             }
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->tokmax[stage]), parity, p.wait_polls))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->tokmax[stage]), parity))) { timed_out = true; break; }
             for (int w = 0; w < nwarps; w++) m = fmaxf(m, *reinterpret_cast<volatile float *>(&ctrl->wmax[stage][w]));
         }
 
@@ -414,7 +414,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             const int k_next = it + S;
             int raw_next = 0;
             if (lane == 0 && k_next < n_my) raw_next = raw_row_of(k_next);
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity, p.wait_polls))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->done[stage]), parity))) { timed_out = true; break; }
             // The record sits in the slot of the stage's current parity; the stage's next token writes the other
             // slot, and the one after that cannot start before this warp has arrived for the token in between.
             // With x_hat the X row itself is the source of a store and must have been read before the refill.
@@ -446,8 +446,8 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
     if (lane == 0) bulk_wait_all();
     if (tid == 0 && *reinterpret_cast<volatile int *>(&ctrl->abort)) {
         for (int s = 0; s < S; s++) {
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0, p.wait_polls);
-            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1, p.wait_polls);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 0);
+            mbar_wait_bounded(smem_u32(&ctrl->full[s]), 1);
         }
     }
 }
@@ -523,7 +523,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
                               resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec, tk);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
-        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity, p.wait_polls);
+        const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
         if (timed_out && p.status) atomicOr(p.status, RAC_STATUS_TIMEOUT);
         const bool has_ref = ctrl->row[stage] >= 0;
         const unsigned char *rec = smem + L.stage0 + stage * L.stage_bytes;
@@ -641,8 +641,8 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
         bulk_wait_all();
         if (aborted) {
             for (int s = 0; s < S; s++) {
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0, p.wait_polls);
-                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1, p.wait_polls);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 0);
+                mbar_wait_bounded(smem_u32(&ctrl->bar[s]), 1);
             }
         }
     }

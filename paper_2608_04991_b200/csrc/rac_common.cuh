@@ -42,9 +42,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: gives up after a fixed number of polls (well under a second) and reports it, so a copy
 // that never lands cannot hang the GPU.
-constexpr uint32_t kWaitPolls = 1u << 19;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t polls = kWaitPolls) {
-    for (uint32_t i = 0; i < polls; ++i) {
+constexpr uint32_t kWaitPolls = 1u << 16;   // ~0.2 s of polling; a copy normally lands within microseconds
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitPolls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
     }
     return false;
