@@ -32,11 +32,11 @@ METRIC = "codec GB/s of bf16 activations (encode+decode round trip)"
 UNIT = "GB/s"
 WORKLOAD = dict(T=131072, d=5120, group=128, bits=4, topk=8, n_hist=131072, min_ngram=4, max_hits=8, gap_max=112)
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one rac_encode[_reconstruct] call (streaming kernel +
-# outlier kernel) from the ncu capture of the SMALL case (profiles/codec_kernels_small_case_T16384_d5120.md);
+# outlier kernel) and of one reconstruction, from an ncu capture of the SMALL case (T = 16384, same d and record);
 # traffic is proportional to tokens, so a launch of T tokens moves T/16384 times as much.
-NCU_SMALL_CASE_TRAFFIC = {"encode_sender_up": 267.70e6 + 179.99e6 + 53.37e6 + 1.67e6,
-                          "encode_dn": 335.69e6 + 43.16e6 + 59.45e6 + 0.55e6,
-                          "decode_up": 141.29e6 + 116.54e6, "decode_dn": 212.92e6 + 122.74e6}
+NCU_SMALL_CASE_TRAFFIC = {"encode_sender_up": 267.85e6 + 180.01e6 + 51.13e6 + 1.67e6,
+                          "encode_dn": 335.62e6 + 44.00e6 + 56.33e6 + 0.49e6,
+                          "decode_up": 141.15e6 + 118.01e6, "decode_dn": 212.92e6 + 123.03e6}
 SMALL = dict(T=16384, d=5120, group=128, bits=4, topk=8, n_hist=16384, min_ngram=4, max_hits=8, gap_max=112)
 
 
