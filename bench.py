@@ -130,7 +130,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------- workload
 class RoundTrip:
     """Device buffers and the ordered C-ABI calls of one step."""
-    LAUNCHES_PER_STEP = (9 + WORKLOAD["max_hits"]) + 2 * 2 + 2  # matcher kernels + 2 encodes (2 launches each) + 2 reconstructions
+    LAUNCHES_PER_STEP = 9 + 2 * 2 + 2  # matcher kernels + 2 encodes (2 launches each) + 2 reconstructions
 
     def __init__(self, wl, seed, dev, token_range=None):
         import numpy as np

@@ -80,7 +80,7 @@ extern "C" {
  *   flags   must be 0
  *   qgroup  g_q, channels per quantisation group (scale_mode 1): 0 = same as `group`; a power of two 32..1024
  *           that divides d; or d itself (the paper's decode mode: one scale per token)
- *   topk_group  k_g, outliers per quantisation group (Sec. IV-C "Outlier Metadata"), 0..4, scale_mode 1 with
+ *   topk_group  k_g, outliers per quantisation group (Sec. IV-C "Outlier Metadata"), 0..8, scale_mode 1 with
  *           qgroup <= 256: the k_g largest |e| of every group (ties to the lower channel) leave the dense base
  *           before its scale is taken; one-byte in-group offsets in ascending order + binary16 values */
 typedef struct {

@@ -59,7 +59,7 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
         if (is_pow2(qgroup) && qgroup >= 32 && qgroup <= 1024) lpq = qgroup / 32;
         else if (qgroup == cfg->d) lpq = 0;   // one scale per token, exchanged through shared memory
         else return RAC_EUNSUPPORTED;
-        if (cfg->topk_group > 4) return RAC_EUNSUPPORTED;
+        if (cfg->topk_group > 8) return RAC_EUNSUPPORTED;
         if (cfg->topk_group > 0 && (lpq == 0 || qgroup > 256)) return RAC_EUNSUPPORTED;   // one-byte offsets
     }
     g->d = cfg->d;

@@ -77,7 +77,7 @@ __device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, 
 }
 
 // MINB = 4 caps registers at 96 so that four 160-thread CTAs (d = 5120) fit on an SM.
-// KG: rounds compiled in (0, 1, 2 or 4; p.kg <= KG is the number taken).
+// KG: rounds compiled in (0, 1, 2, 4 or 8; p.kg <= KG is the number taken).
 template <int BITS, bool XHAT, int KG, int MINB, bool SUB>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
         u64 e2[16];        // Eq. 7 residual of this thread's channels, packed pairs in slot order
         u64 r2[16];        // aligned-reference inputs, kept for the sender-side reconstruction
         u64 a2 = 0ull, b2 = 0ull;
-        uint32_t sel[4] = {0u, 0u, 0u, 0u};   // per round: in-group offset | binary16 value << 16 (same in every lane of the group)
+        uint32_t sel[KG > 4 ? 8 : 4] = {};   // per round: in-group offset | binary16 value << 16 (same in every lane of the group)
         uint32_t own = 0;                      // rounds whose outlier lives in this thread
         float m = 0.f;
         if (valid) {
@@ -606,7 +606,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
                 const int qsize = p.lpq * 32;
                 bool bad = false;
 #pragma unroll
-                for (int n = 0; n < 4; n++) {
+                for (int n = 0; n < 8; n++) {
                     if (n < p.kg) {
                         const int o = go[n];
                         if (o >= qsize) {
@@ -671,12 +671,14 @@ static int launch_encode_bits(const Geometry &g, CodecParams &p, int smem, long 
         return k == 0 ? launch_encode_variant<B, true, 0>(tight, g, p, smem, max_ctas, stream)
              : k == 1 ? launch_encode_variant<B, true, 1>(tight, g, p, smem, max_ctas, stream)
              : k == 2 ? launch_encode_variant<B, true, 2>(tight, g, p, smem, max_ctas, stream)
-                      : launch_encode_variant<B, true, 4>(tight, g, p, smem, max_ctas, stream);
+             : k <= 4 ? launch_encode_variant<B, true, 4>(tight, g, p, smem, max_ctas, stream)
+                      : launch_encode_variant<B, true, 8>(tight, g, p, smem, max_ctas, stream);
     }
     return k == 0 ? launch_encode_variant<B, false, 0>(tight, g, p, smem, max_ctas, stream)
          : k == 1 ? launch_encode_variant<B, false, 1>(tight, g, p, smem, max_ctas, stream)
          : k == 2 ? launch_encode_variant<B, false, 2>(tight, g, p, smem, max_ctas, stream)
-                  : launch_encode_variant<B, false, 4>(tight, g, p, smem, max_ctas, stream);
+         : k <= 4 ? launch_encode_variant<B, false, 4>(tight, g, p, smem, max_ctas, stream)
+                  : launch_encode_variant<B, false, 8>(tight, g, p, smem, max_ctas, stream);
 }
 
 int launch_encode_dyn(const Geometry &g, CodecParams &p, long long max_ctas, cudaStream_t stream) {

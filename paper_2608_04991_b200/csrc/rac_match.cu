@@ -2,9 +2,11 @@
 //
 // Index: an open-addressing hash table with one slot per DISTINCT w-token window of the history.  A slot
 // stores one representative start position (used to verify a key token by token, so hash collisions can
-// never change the result) and the K largest start positions of that window, found by K rounds of
-// atomicMax ("largest start below the previous round's").  Because every round is a maximum, the
-// table contents do not depend on the order in which threads run.
+// never change the result) and the K largest start positions of that window in descending order.  A start
+// enters its slot's list by a cascade of atomicMax: it is offered to entry 0, the smaller of (offered, found)
+// is carried to entry 1, and so on.  Every step keeps the pair it touches, so entry 0 ends as the largest
+// value ever offered, entry 1 as the largest of the rest, ...: the final lists do not depend on the order in
+// which threads run.
 // Query: one thread per query position looks its window up, extends each of the <= K candidates forward
 // to the longest exact match and keeps lexargmax(length, start).
 // Selection: the left-to-right scan of Eq. 3 visits a position, jumps by the span length if it has a
@@ -57,6 +59,17 @@ __device__ __forceinline__ bool same_window(const int32_t *a, const int32_t *b, 
     return true;
 }
 
+// Offers start j to a descending list of K entries (-1 = empty): atomicMax at entry r keeps the larger of
+// (offered, found) there and carries the smaller on to entry r + 1.  Whatever the interleaving with other
+// threads, the list ends as the K largest values ever offered, in descending order.
+__device__ __forceinline__ void cascade_insert(int32_t *lst, int K, int j) {
+    int v = j;
+    for (int r = 0; r < K && v >= 0; r++) {
+        const int old = atomicMax(&lst[r], v);
+        v = old < v ? old : v;
+    }
+}
+
 __global__ void match_init_kernel(MatchParams p, long long table_ints) {
     long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     long long stride = (long long)gridDim.x * blockDim.x;
@@ -78,19 +91,11 @@ __global__ void match_insert_kernel(MatchParams p) {
         s = (s + 1) & p.mask;
     }
     p.slot_of[j] = slot;  // the table has >= 2*nwin slots, so a slot is always found
+    if (slot < 0) return;
     // unlimited hits: every start of the window goes onto the slot's chain.  The order of a chain depends on which
     // thread came first; the query looks at ALL of it and keeps lexargmax(length, start), so the result does not.
-    if (p.next && slot >= 0) p.next[j] = atomicExch(&p.top[slot], j);
-}
-
-// round r: the largest start of each window that is below the start found in round r-1
-__global__ void match_round_kernel(MatchParams p, int r) {
-    int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= p.nwin) return;
-    int s = p.slot_of[j];
-    if (s < 0) return;
-    int32_t *lst = p.top + (long long)s * p.K;
-    if (r == 0 || j < lst[r - 1]) atomicMax(&lst[r], j);
+    if (p.next) p.next[j] = atomicExch(&p.top[slot], j);
+    else cascade_insert(p.top + (long long)slot * p.K, p.K, j);
 }
 
 __global__ void match_query_kernel(MatchParams p) {
@@ -372,9 +377,10 @@ struct IndexParams {
     unsigned int mask;
 };
 
-// (1) every position of the request learns its end; every window of the request finds or claims its slot and
-// is counted there
-__global__ void index_append_insert_kernel(IndexParams p) {
+// Appending a request: every position learns the end of its request; every window of the request finds or claims
+// its slot and enters the slot's list by the cascade.  The request's starts are larger than everything already
+// there, so the older entries move down (and the oldest fall off) as a by-product.  One launch, any request size.
+__global__ void index_append_kernel(IndexParams p) {
     const int j = p.a + blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= p.b) return;
     p.end_of[j] = p.b;
@@ -387,84 +393,7 @@ __global__ void index_append_insert_kernel(IndexParams p) {
         if (cur == -1 || cur == j || same_window(p.hist + cur, win, p.w)) { slot = (int)s; break; }
         s = (s + 1) & p.mask;
     }
-    p.slot_of[j] = slot;
-    if (slot >= 0) atomicAdd(&p.cnt[slot], 1);
-}
-
-// (2) one thread per touched slot (the one that takes the count away) makes room at the head of the slot's
-// list: the request's starts are larger than everything already there
-__global__ void index_append_shift_kernel(IndexParams p) {
-    const int j = p.a + blockIdx.x * blockDim.x + threadIdx.x;
-    if (j + p.w > p.b) return;
-    const int slot = p.slot_of[j];
-    if (slot < 0) return;
-    const int c = atomicExch(&p.cnt[slot], 0);
-    if (c == 0) return;
-    int32_t *lst = p.top + (long long)slot * p.K;
-    const int sh = c < p.K ? c : p.K;
-    for (int r = p.K - 1; r >= sh; r--) lst[r] = lst[r - sh];
-    for (int r = 0; r < sh; r++) lst[r] = -1;
-}
-
-// (3) round r: the largest start of the request's windows below the one found in round r-1.  Entries behind the
-// request's own are older, hence smaller, and are never touched: no start of the request is below its smallest.
-__global__ void index_append_round_kernel(IndexParams p, int r) {
-    const int j = p.a + blockIdx.x * blockDim.x + threadIdx.x;
-    if (j + p.w > p.b) return;
-    const int slot = p.slot_of[j];
-    if (slot < 0) return;
-    int32_t *lst = p.top + (long long)slot * p.K;
-    if (r == 0 || j < lst[r - 1]) atomicMax(&lst[r], j);
-}
-
-// The three steps above for a request small enough for ONE CTA, in one launch: the CTA's barriers stand where the
-// launch boundaries stood (every thread strides over the request's positions in every step).
-constexpr int kAppendFusedMax = 16384;   // tokens per request up to which the single-CTA form is used
-__global__ void __launch_bounds__(1024) index_append_fused_kernel(IndexParams p) {
-    const int n = p.b - p.a;
-    for (int o = threadIdx.x; o < n; o += blockDim.x) {
-        const int j = p.a + o;
-        p.end_of[j] = p.b;
-        if (j + p.w > p.b) continue;
-        const int32_t *win = p.hist + j;
-        unsigned int s = window_hash(win, p.w) & p.mask;
-        int slot = -1;
-        for (unsigned int probe = 0; probe <= p.mask; probe++) {
-            int cur = atomicCAS(&p.rep[s], -1, j);
-            if (cur == -1 || cur == j || same_window(p.hist + cur, win, p.w)) { slot = (int)s; break; }
-            s = (s + 1) & p.mask;
-        }
-        p.slot_of[j] = slot;
-        if (slot >= 0) atomicAdd(&p.cnt[slot], 1);
-    }
-    __syncthreads();
-    for (int o = threadIdx.x; o < n; o += blockDim.x) {
-        const int j = p.a + o;
-        if (j + p.w > p.b) continue;
-        const int slot = p.slot_of[j];
-        if (slot < 0) continue;
-        const int c = atomicExch(&p.cnt[slot], 0);
-        if (c == 0) continue;
-        int32_t *lst = p.top + (long long)slot * p.K;
-        const int sh = c < p.K ? c : p.K;
-        for (int r = p.K - 1; r >= sh; r--) lst[r] = lst[r - sh];
-        for (int r = 0; r < sh; r++) lst[r] = -1;
-    }
-    for (int r = 0; r < p.K; r++) {
-        __syncthreads();
-        int any = 0;
-        for (int o = threadIdx.x; o < n; o += blockDim.x) {
-            const int j = p.a + o;
-            if (j + p.w > p.b) continue;
-            const int slot = p.slot_of[j];
-            if (slot < 0) continue;
-            int32_t *lst = p.top + (long long)slot * p.K;
-            if (r == 0 || j < lst[r - 1]) { atomicMax(&lst[r], j); any = 1; }
-        }
-        // a round in which no start was left to place is the last one that can change anything: most windows
-        // occur once in a request, so one or two rounds do
-        if (!__syncthreads_or(any)) break;
-    }
+    if (slot >= 0) cascade_insert(p.top + (long long)slot * p.K, p.K, j);
 }
 
 // Intra-sequence references: first occurrence of every token of the prompt (a hash table keyed by a position
@@ -655,7 +584,6 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     if (p.nwin > 0 && n_query > 0) {
         int nb = (p.nwin + tb - 1) / tb;
         match_insert_kernel<<<nb, tb, 0, st>>>(p);
-        for (int r = 0; r < max_hits; r++) match_round_kernel<<<nb, tb, 0, st>>>(p, r);   // none with chains
     }
     if (n_query > 0) {
         match_query_kernel<<<(int)((n_query + tb - 1) / tb), tb, 0, st>>>(p);
@@ -792,17 +720,7 @@ int rac_index_append(const rac_index_cfg *cfg, void *index, size_t index_bytes, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int tb = 256;
     const int nb = (int)((n_after - n_before + tb - 1) / tb);
-    if (n_after - n_before <= kAppendFusedMax) {
-        // a request of ordinary size: one launch (the K + 2 launches below cost ~3 us each, which is all an append
-        // of a few thousand tokens costs)
-        index_append_fused_kernel<<<1, 1024, 0, st>>>(p);
-        return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
-    }
-    index_append_insert_kernel<<<nb, tb, 0, st>>>(p);
-    if (n_after - n_before >= cfg->min_ngram) {
-        index_append_shift_kernel<<<nb, tb, 0, st>>>(p);
-        for (int r = 0; r < cfg->max_hits; r++) index_append_round_kernel<<<nb, tb, 0, st>>>(p, r);
-    }
+    index_append_kernel<<<nb, tb, 0, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 

@@ -452,6 +452,9 @@ def test_dynamic_group_scale_identity_and_rejections(env):
     (96, 32, 4, 32, 2, 9),          # a single partly filled warp
     (96, 32, 8, 96, 0, 9),
     (2080, 32, 4, 0, 1, 33),        # odd group counts: padding after scales and after offsets
+    (4096, 128, 4, 0, 8, 70),       # eight outliers per group of 128
+    (5120, 128, 4, 256, 6, 41),     # six, groups of eight lanes
+    (4096, 64, 8, 32, 5, 23),       # five in groups of one lane, 8-bit codes
 ])
 def test_family_matches_oracle(env, d, g, bits, qg, kg, T):
     X, R, _, _ = prefill_inputs(env, T, d, g, seed=3000 + d + bits + qg + kg)
@@ -498,7 +501,7 @@ def test_family_ties_zero_groups_and_bad_offsets(env):
     assert len(diff) == 1 and diff[0][0] == 3 and diff[0][1] == 5 * 32 + keep   # only the outlier that was dropped
     # configurations this build has no kernel for
     for bad_cfg in [env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=512, topk_group=1),   # one-byte offsets
-                    env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, topk_group=5),
+                    env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, topk_group=9),
                     env.rac.CodecCfg(d, g, 8, 0),                                           # 8 bits: Eq. 8 family only
                     env.rac.CodecCfg(d, g, 4, 0, qgroup=64),                                # static table: g_q = g_a
                     env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=96),
@@ -519,7 +522,7 @@ def test_family_random_configurations(env):
             continue
         bits = int(rng.choice([2, 3, 4, 8]))
         qg = int(rng.choice([0, 32, 64, 128, 256, d]))
-        kg = int(rng.choice([0, 0, 1, 2, 3, 4]))
+        kg = int(rng.choice([0, 0, 1, 2, 3, 4, 6, 8]))
         cfg = env.rac.CodecCfg(d, g, bits, 0, scale_mode=1, qgroup=qg, topk_group=kg)
         if env.rac.rac_record_bytes(cfg) == 0:
             assert env.orc.record_bytes(d, g, bits, 0, 1, qg, kg) == 0 or (qg or g) > 256 or d % (qg or g) or \
@@ -651,7 +654,7 @@ def test_random_configurations_on_stressed_inputs(env):
         T = int(rng.integers(1, 400 if d <= 2080 else 120))
         if fam:
             cfg = rac.CodecCfg(d, g, int(rng.choice([2, 3, 4, 8])), 0, scale_mode=1,
-                               qgroup=int(rng.choice([0, 32, 64, 128, 256, d])), topk_group=int(rng.choice([0, 0, 1, 2, 3, 4])))
+                               qgroup=int(rng.choice([0, 32, 64, 128, 256, d])), topk_group=int(rng.choice([0, 0, 1, 2, 3, 4, 7, 8])))
             if rac.rac_record_bytes(cfg) == 0:
                 continue
         else:
