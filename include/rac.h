@@ -206,6 +206,17 @@ int rac_index_reset(const rac_index_cfg *cfg, void *index, size_t index_bytes, v
 int rac_index_append(const rac_index_cfg *cfg, void *index, size_t index_bytes, const int32_t *hist_tok,
                      int64_t n_before, int64_t n_after, void *stream);
 size_t rac_index_query_workspace_bytes(int64_t n_query);
+/* rac_index_query over a bounded history ("recent hits", Sec. IV-B.1): only windows that START at or after history
+ * position first_live (0 <= first_live <= n_hist) are candidates; a match still runs forward as far as it goes.
+ * Nothing is removed from the index: an old request is dropped by raising first_live past it, at no cost, and the
+ * state rows below first_live are never referenced again (the caller may reuse that part of its state buffer; the
+ * token buffer must stay readable, the index verifies keys against it).  The K most recent starts of a window that
+ * lie in the live part are exactly the leading entries of its list, so the result equals a rebuild from the live
+ * requests only.  rac_index_query is this call with first_live = 0. */
+int rac_index_query_live(const rac_index_cfg *cfg, const void *index, size_t index_bytes, const int32_t *hist_tok,
+                         int64_t n_hist, int64_t first_live, const int32_t *query_tok, int64_t n_query, int32_t intra,
+                         int32_t *ref_row, rac_span *spans, int32_t *n_spans, void *workspace, size_t workspace_bytes,
+                         void *stream);
 int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_bytes, const int32_t *hist_tok,
                     int64_t n_hist, const int32_t *query_tok, int64_t n_query, int32_t intra, int32_t *ref_row,
                     rac_span *spans, int32_t *n_spans, void *workspace, size_t workspace_bytes, void *stream);

@@ -94,6 +94,9 @@ def _declare(l: C.CDLL) -> None:
     l.orc_match_spans_req.restype = C.c_int
     l.orc_match_spans_req.argtypes = [_i32p, C.c_int64, _i32p, C.c_int32, _i32p, C.c_int64, C.c_int, C.c_int, C.c_int,
                                       _i32p, _i32p, _i32p]
+    l.orc_match_spans_live.restype = C.c_int
+    l.orc_match_spans_live.argtypes = [_i32p, C.c_int64, _i32p, C.c_int32, _i32p, C.c_int64, C.c_int, C.c_int, C.c_int,
+                                       C.c_int64, _i32p, _i32p, _i32p]
     l.orc_max_threads.restype = C.c_int
     l.orc_max_threads.argtypes = []
 
@@ -308,9 +311,11 @@ def match_spans(hist: np.ndarray, query: np.ndarray, w: int = 4, max_hits: int =
     return ref_row, spans[: ns.value].copy()
 
 
-def match_spans_req(hist: np.ndarray, req_off, query: np.ndarray, w: int = 4, max_hits: int = 8, intra: bool = False):
+def match_spans_req(hist: np.ndarray, req_off, query: np.ndarray, w: int = 4, max_hits: int = 8, intra: bool = False,
+                    first_live: int = 0):
     """Sec. IV-B.1 with the history as a list of earlier requests (``req_off`` int32[n_req+1], or None for one
-    request) and, with ``intra``, the intra-sequence references (rows >= len(hist)).  Returns (ref_row, spans)."""
+    request) and, with ``intra``, the intra-sequence references (rows >= len(hist)).  ``first_live``: only windows
+    that start at or after this history position are candidates.  Returns (ref_row, spans)."""
     hist = _chk(hist, np.int32)
     query = _chk(query, np.int32)
     req_off = _chk(None if req_off is None else np.asarray(req_off, np.int32), np.int32)
@@ -318,9 +323,10 @@ def match_spans_req(hist: np.ndarray, req_off, query: np.ndarray, w: int = 4, ma
     ref_row = np.full(N, -1, np.int32)
     spans = np.zeros((N // max(w, 1) + 1, 3), np.int32)
     ns = C.c_int32(0)
-    rc = lib().orc_match_spans_req(_p(hist, _i32p), hist.size, _p(req_off, _i32p),
-                                   0 if req_off is None else req_off.size - 1, _p(query, _i32p), N, int(w),
-                                   int(max_hits), int(bool(intra)), _p(ref_row, _i32p), _p(spans, _i32p), C.byref(ns))
+    rc = lib().orc_match_spans_live(_p(hist, _i32p), hist.size, _p(req_off, _i32p),
+                                    0 if req_off is None else req_off.size - 1, _p(query, _i32p), N, int(w),
+                                    int(max_hits), int(bool(intra)), int(first_live), _p(ref_row, _i32p), _p(spans, _i32p),
+                                    C.byref(ns))
     if rc != 0:
         raise ValueError(f"orc_match_spans_req failed: {rc}")
     return ref_row, spans[: ns.value].copy()

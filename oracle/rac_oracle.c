@@ -732,12 +732,15 @@ static int cmp_hist_query(const int32_t *hist, int32_t p, const int32_t *query, 
  * n_spans  out
  * max_hits K: only the K largest history starts of each distinct window are
  *          candidates; 0 = all of them.
+ * first_live  a bounded history ("recent hits"): only windows that START at or after
+ *          this history position are candidates; a match still extends forward as far
+ *          as it goes.  0 = the whole history.
  * Not thread safe (qsort comparator state).
  */
-int orc_match_spans_req(const int32_t *hist, int64_t n_hist, const int32_t *req_off, int32_t n_req,
-                        const int32_t *query, int64_t n_query, int w, int max_hits, int intra,
-                        int32_t *ref_row, int32_t *spans, int32_t *n_spans) {
-    if (w < 1 || max_hits < 0) return -1;
+int orc_match_spans_live(const int32_t *hist, int64_t n_hist, const int32_t *req_off, int32_t n_req,
+                         const int32_t *query, int64_t n_query, int w, int max_hits, int intra, int64_t first_live,
+                         int32_t *ref_row, int32_t *spans, int32_t *n_spans) {
+    if (w < 1 || max_hits < 0 || first_live < 0) return -1;
     if (req_off) {
         if (n_req < 0 || req_off[0] != 0 || req_off[n_req] != n_hist) return -1;
         for (int32_t r = 0; r < n_req; r++) if (req_off[r] > req_off[r + 1]) return -1;
@@ -755,7 +758,7 @@ int orc_match_spans_req(const int32_t *hist, int64_t n_hist, const int32_t *req_
     /* windows that lie inside one request, sorted by content then position */
     int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_hist > 0 ? n_hist : 1));
     int64_t nwin = 0;
-    for (int64_t j = 0; j + w <= n_hist; j++)
+    for (int64_t j = first_live; j + w <= n_hist; j++)
         if (j + w <= end_of[j]) order[nwin++] = (int32_t)j;
     g_sort_tok = hist; g_sort_w = w;
     qsort(order, (size_t)nwin, sizeof(int32_t), cmp_window_pos);
@@ -804,6 +807,12 @@ int orc_match_spans_req(const int32_t *hist, int64_t n_hist, const int32_t *req_
     }
     free(order); free(end_of);
     return 0;
+}
+
+int orc_match_spans_req(const int32_t *hist, int64_t n_hist, const int32_t *req_off, int32_t n_req,
+                        const int32_t *query, int64_t n_query, int w, int max_hits, int intra,
+                        int32_t *ref_row, int32_t *spans, int32_t *n_spans) {
+    return orc_match_spans_live(hist, n_hist, req_off, n_req, query, n_query, w, max_hits, intra, 0, ref_row, spans, n_spans);
 }
 
 int orc_match_spans(const int32_t *hist, int64_t n_hist, const int32_t *query, int64_t n_query,

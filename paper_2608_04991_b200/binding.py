@@ -31,6 +31,7 @@ EXPORTS = [
     "rac_match_workspace_bytes", "rac_match_spans", "rac_spans_to_rows",
     "rac_match_spans_static",
     "rac_index_bytes", "rac_index_reset", "rac_index_append", "rac_index_query_workspace_bytes", "rac_index_query",
+    "rac_index_query_live",
     "rac_encode_workspace_bytes", "rac_encode", "rac_encode_reconstruct", "rac_decode_reconstruct",
     "rac_sender_reconstruct",
     "rac_split_waves", "rac_encode_reconstruct_list", "rac_decode_reconstruct_list",
@@ -112,6 +113,8 @@ def load() -> C.CDLL:
     l.rac_index_query_workspace_bytes.argtypes = [i64]
     l.rac_index_query.restype = C.c_int
     l.rac_index_query.argtypes = [icfgp, vp, sz, vp, i64, vp, i64, i32, vp, vp, vp, vp, sz, vp]
+    l.rac_index_query_live.restype = C.c_int
+    l.rac_index_query_live.argtypes = [icfgp, vp, sz, vp, i64, i64, vp, i64, i32, vp, vp, vp, vp, sz, vp]
     l.rac_spans_to_rows.restype = C.c_int
     l.rac_spans_to_rows.argtypes = [vp, vp, i64, vp, vp]
     l.rac_encode.restype = C.c_int
@@ -345,6 +348,17 @@ def rac_index_append(cfg, index, index_bytes, hist_tok, n_before, n_after, strea
                                  _ptr(hist_tok, _I32, "hist_tok"), int(n_before), int(n_after),
                                  _stream() if stream is None else stream)
     _check("rac_index_append", rc)
+
+
+def rac_index_query_live(cfg, index, index_bytes, hist_tok, n_hist, first_live, query_tok, n_query, intra, ref_row, spans,
+                         n_spans, workspace, workspace_bytes, stream=None) -> None:
+    rc = load().rac_index_query_live(C.byref(cfg), _ptr(index, None, "index"), int(index_bytes),
+                                     _ptr(hist_tok, _I32, "hist_tok"), int(n_hist), int(first_live),
+                                     _ptr(query_tok, _I32, "query_tok"), int(n_query), int(bool(intra)),
+                                     _ptr(ref_row, _I32, "ref_row"), _ptr(spans, _I32, "spans"), _ptr(n_spans, _I32, "n_spans"),
+                                     _ptr(workspace, None, "workspace"), int(workspace_bytes),
+                                     _stream() if stream is None else stream)
+    _check("rac_index_query_live", rc)
 
 
 def rac_index_query(cfg, index, index_bytes, hist_tok, n_hist, query_tok, n_query, intra, ref_row, spans, n_spans,

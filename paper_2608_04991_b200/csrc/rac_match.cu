@@ -39,6 +39,7 @@ struct MatchParams {
     int n_hist, n_query, nwin, w, K;
     unsigned int mask;     // M - 1
     const int32_t *end_of; // [n_hist] end of the request that holds each history position; null = one request
+    int first_live;        // only windows that start at or after this history position are candidates (0 = all)
     int32_t *next;         // [nwin]   unlimited hits (max_hits = 0) only: another start of the same window, -1 = none;
                            //          top[slot] is then the head of the slot's chain (K = 1 entry per slot)
 };
@@ -138,14 +139,14 @@ __global__ void match_query_kernel(MatchParams p) {
                 // every occurrence of the window (at most nwin of them: the walk is bounded by construction)
                 int j = p.top[slot];
                 for (int n = 0; j >= 0 && n < p.nwin; n++) {
-                    consider(j);
+                    if (j >= p.first_live) consider(j);
                     j = p.next[j];
                 }
             } else {
                 const int32_t *lst = p.top + (long long)slot * p.K;
                 for (int r = 0; r < p.K; r++) {
                     const int j = lst[r];
-                    if (j < 0) break;
+                    if (j < p.first_live) break;   // descending: the rest is empty (-1) or older than the live window
                     consider(j);
                 }
             }
@@ -571,6 +572,7 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
     p.nwin = (int)(n_hist - min_ngram + 1 > 0 ? n_hist - min_ngram + 1 : 0);
     p.w = min_ngram;
     p.K = max_hits > 0 ? max_hits : 1;
+    p.first_live = 0;
     p.next = max_hits == 0 ? reinterpret_cast<int32_t *>(ws + L.next) : nullptr;
     p.mask = L.M - 1;
 
@@ -732,8 +734,17 @@ size_t rac_index_query_workspace_bytes(int64_t n_query) {
 int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_bytes, const int32_t *hist_tok,
                     int64_t n_hist, const int32_t *query_tok, int64_t n_query, int32_t intra, int32_t *ref_row,
                     rac_span *spans, int32_t *n_spans, void *workspace, size_t workspace_bytes, void *stream) {
+    return rac_index_query_live(cfg, index, index_bytes, hist_tok, n_hist, 0, query_tok, n_query, intra, ref_row, spans,
+                                n_spans, workspace, workspace_bytes, stream);
+}
+
+int rac_index_query_live(const rac_index_cfg *cfg, const void *index, size_t index_bytes, const int32_t *hist_tok,
+                         int64_t n_hist, int64_t first_live, const int32_t *query_tok, int64_t n_query, int32_t intra,
+                         int32_t *ref_row, rac_span *spans, int32_t *n_spans, void *workspace, size_t workspace_bytes,
+                         void *stream) {
     if (!index_cfg_ok(cfg)) return cfg ? RAC_EUNSUPPORTED : RAC_EINVAL;
     if (!index || !n_spans || n_hist < 0 || n_query < 0 || !workspace) return RAC_EINVAL;
+    if (first_live < 0 || first_live > n_hist) return RAC_EINVAL;
     if (n_hist > cfg->capacity) return RAC_ESIZE;
     if (n_query >= (1ll << 30) || n_hist + n_query >= (1ll << 31)) return RAC_EUNSUPPORTED;
     if ((n_hist > 0 && !hist_tok) || (n_query > 0 && (!query_tok || !ref_row))) return RAC_EINVAL;
@@ -768,6 +779,7 @@ int rac_index_query(const rac_index_cfg *cfg, const void *index, size_t index_by
     p.K = cfg->max_hits;
     p.mask = L.M - 1;
     p.next = nullptr;
+    p.first_live = (int)first_live;
     p.end_of = reinterpret_cast<const int32_t *>(ix + L.end_of);
     const int tb = 256;
     // rows to -1, span count to 0, and (for the intra-sequence pass) the token table to empty

@@ -189,7 +189,7 @@ class GpuIndex:
         self.rac.rac_index_append(self.cfg, self.mem[:self.nb], self.nb, self.hist, self.n, self.n + req.size)
         self.n += req.size
 
-    def query(self, query, intra=False):
+    def query(self, query, intra=False, first_live=None):
         q = torch.from_numpy(np.ascontiguousarray(query, np.int32)).to(self.dev)
         N = q.numel()
         nws = self.rac.rac_index_query_workspace_bytes(N)
@@ -198,8 +198,13 @@ class GpuIndex:
         cap = N // self.w + 1
         spans = torch.full((cap + 2, 3), 777, dtype=torch.int32, device=self.dev)
         n_spans = torch.full((1,), -5, dtype=torch.int32, device=self.dev)
-        self.rac.rac_index_query(self.cfg, self.mem[:self.nb], self.nb, self.hist, self.n, q if N else None, N, intra,
-                                 rows[:N] if N else None, spans[:cap], n_spans, ws[:nws], nws)
+        if first_live is None:
+            self.rac.rac_index_query(self.cfg, self.mem[:self.nb], self.nb, self.hist, self.n, q if N else None, N, intra,
+                                     rows[:N] if N else None, spans[:cap], n_spans, ws[:nws], nws)
+        else:
+            self.rac.rac_index_query_live(self.cfg, self.mem[:self.nb], self.nb, self.hist, self.n, first_live,
+                                          q if N else None, N, intra, rows[:N] if N else None, spans[:cap], n_spans,
+                                          ws[:nws], nws)
         torch.cuda.synchronize()
         assert torch.all(rows[N:] == 12345) and torch.all(spans[cap:] == 777) and torch.all(ws[nws:] == 0xA5)
         assert torch.all(self.mem[self.nb:] == 0x5A)
@@ -242,6 +247,43 @@ def test_index_appended_request_by_request_matches_oracle(env, seed):
     rr, sp = ix.query(query)
     o_rr, o_sp = env.orc.match_spans_req(np.concatenate(reqs), np.array(off, np.int32), query, w=w, max_hits=K)
     assert np.array_equal(sp, o_sp) and np.array_equal(rr, o_rr)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_index_live_window(env, seed):
+    """A bounded history: old requests are dropped by raising `first_live`; nothing in the index changes.  After
+    every append the prompt is matched with the cut at several places (request boundaries and inside requests)
+    and compared with the oracle's live-window matcher; the cut at 0 equals the plain query."""
+    rng = np.random.default_rng(1300 + seed)
+    vocab = [2, 3, 6, 40][seed % 4]
+    w = [1, 2, 3, 4][seed % 4]
+    K = [1, 2, 8, 16][seed % 4]
+    ix = GpuIndex(env, 4096, w, K)
+    reqs, off = [], [0]
+    for step in range(6):
+        req = rng.integers(0, vocab, int(rng.integers(0, 200))).astype(np.int32)
+        ix.append(req)
+        reqs.append(req)
+        off.append(off[-1] + req.size)
+        hist = np.concatenate(reqs)
+        N = int(rng.integers(1, 250))
+        query = rng.integers(0, vocab, N).astype(np.int32)
+        if hist.size >= 8:
+            L = min(N, hist.size, 50)
+            a = int(rng.integers(0, hist.size - L + 1))
+            query[:L] = hist[a:a + L]
+        cuts = sorted({0, off[len(off) // 2], int(rng.integers(0, hist.size + 1)), hist.size})
+        for cut in cuts:
+            for intra in (False, True):
+                rr, sp = ix.query(query, intra=intra, first_live=cut)
+                o_rr, o_sp = env.orc.match_spans_req(hist, np.array(off, np.int32), query, w=w, max_hits=K, intra=intra,
+                                                     first_live=cut)
+                assert np.array_equal(sp, o_sp) and np.array_equal(rr, o_rr), (step, cut, intra)
+        rr0, sp0 = ix.query(query)
+        rr1, sp1 = ix.query(query, first_live=0)
+        assert np.array_equal(rr0, rr1) and np.array_equal(sp0, sp1)
+    with pytest.raises(Exception):
+        ix.query(query, first_live=ix.n + 1)
 
 
 def test_index_one_request_equals_the_one_shot_matcher_and_reset(env):

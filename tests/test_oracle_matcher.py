@@ -164,7 +164,7 @@ def test_cap_changes_result_only_for_frequent_windows(orc):
 
 
 # ------------------------------------------------------------------ earlier requests and intra-sequence references
-def brute_force_requests(reqs, query, w, K, intra):
+def brute_force_requests(reqs, query, w, K, intra, first_live=0):
     """The definition per request: candidate (r, j, L) with query[i:i+L] == reqs[r][j:j+L], L >= w maximal inside
     request r; recency = (r, j); the K most recent hits per distinct window; longest, then most recent."""
     N = len(query)
@@ -177,7 +177,7 @@ def brute_force_requests(reqs, query, w, K, intra):
         if i + w <= N:
             for r, req in enumerate(reqs):
                 for j in range(len(req) - w + 1):
-                    if list(req[j:j + w]) == list(query[i:i + w]):
+                    if list(req[j:j + w]) == list(query[i:i + w]) and off[r] + j >= first_live:
                         hits.append((r, j))
         if K > 0:
             hits = sorted(hits)[-K:]
@@ -225,6 +225,34 @@ def test_requests_match_brute_force(orc, seed, K):
     rr, sp = orc.match_spans_req(hist, off, query, w=w, max_hits=K, intra=bool(seed % 2))
     assert np.array_equal(rr, brr)
     assert np.array_equal(sp, bsp)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_live_window_of_the_history(orc, seed):
+    """A bounded history: only windows that start at or after `first_live` are candidates.  Against the brute force
+    with the same filter, and against the matcher itself on the history cut at `first_live` (the request that
+    contains the cut starts there; rows shifted back) -- the cut history must give the same spans."""
+    rng = np.random.default_rng(900 + seed)
+    vocab = [2, 3, 6][seed % 3]
+    w = [1, 2, 3, 4][seed % 4]
+    K = [0, 1, 3, 8][seed % 4]
+    reqs = [rng.integers(0, vocab, int(rng.integers(0, 25))).astype(np.int32) for _ in range(int(rng.integers(1, 6)))]
+    N = int(rng.integers(1, 50))
+    query = rng.integers(0, vocab, N).astype(np.int32)
+    hist = np.concatenate(reqs + [np.zeros(0, np.int32)]).astype(np.int32)
+    off = np.concatenate([[0], np.cumsum([len(r) for r in reqs])]).astype(np.int32)
+    for first_live in sorted({0, 1, int(rng.integers(0, hist.size + 1)), int(hist.size // 2), int(hist.size)}):
+        brr, bsp, _ = brute_force_requests(reqs, query, w, K, intra=False, first_live=first_live)
+        rr, sp = orc.match_spans_req(hist, off, query, w=w, max_hits=K, first_live=first_live)
+        assert np.array_equal(rr, brr) and np.array_equal(sp, bsp), (first_live,)
+        assert not len(sp) or sp[:, 1].min() >= first_live
+        # the same through the cut history
+        cut_off = np.unique(np.clip(off, first_live, None)) - first_live
+        if cut_off[0] != 0:
+            cut_off = np.concatenate([[0], cut_off])
+        crr, csp = orc.match_spans_req(hist[first_live:].copy(), cut_off.astype(np.int32), query, w=w, max_hits=K)
+        assert np.array_equal(np.where(crr >= 0, crr + first_live, -1), rr)
+        assert np.array_equal(csp + np.array([0, first_live, 0], np.int32) if len(csp) else csp, sp)
 
 
 def test_request_boundaries_cut_matches_and_one_request_is_the_flat_matcher(orc):
