@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode-steps", action="store_true", help="skip the decode-step latency extra")
     ap.add_argument("--no-sweep", action="store_true", help="skip the b x group sweep at T=16384, d=4096")
+    ap.add_argument("--sweep-only", action="store_true",
+                    help="run only the b x group sweep and print its JSON (a small case for profiler captures)")
     ap.add_argument("--no-family", action="store_true", help="skip the extras beyond the graded path (Eq. 8 family, persistent index)")
     return ap.parse_args()
 
@@ -513,7 +515,18 @@ def decode_step_latency(dev, n_steps=64, reps=20):
         for t in range(n_steps):
             rac.rac_decode_reconstruct(cfg, pays[t], B, recv_state, B, None, gain, bias, step, recv_state, status)
 
+    # the same calls with their arguments marshalled once (binding.prepare): what a decode loop with fixed buffers does
+    send_calls = [rac.prepare(rac.rac_encode_reconstruct, cfg, xs[t + 1], B, send_state, B, None, gain, bias, step, inv,
+                              pays[t], pays[t].numel(), send_state, None, 0, status) for t in range(n_steps)]
+    recv_calls = [rac.prepare(rac.rac_decode_reconstruct, cfg, pays[t], B, recv_state, B, None, gain, bias, step,
+                              recv_state, status) for t in range(n_steps)]
+
+    def run_prepared(calls):
+        for c in calls:
+            c()
+
     out = {}
+    prepared = {"sender_encode_plus_xhat": send_calls, "receiver_reconstruct": recv_calls}
     for name, fn, state in (("sender_encode_plus_xhat", sender, send_state), ("receiver_reconstruct", receiver, recv_state)):
         fn()                                                    # warm-up (also does the one-time function set-up)
         torch.cuda.synchronize()
@@ -524,6 +537,14 @@ def decode_step_latency(dev, n_steps=64, reps=20):
         e1.record()
         torch.cuda.synchronize()
         eager = e0.elapsed_time(e1) * 1e3 / (reps * n_steps)
+        run_prepared(prepared[name])
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            run_prepared(prepared[name])
+        e1.record()
+        torch.cuda.synchronize()
+        prep = e0.elapsed_time(e1) * 1e3 / (reps * n_steps)
         graph = torch.cuda.CUDAGraph()
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -538,7 +559,8 @@ def decode_step_latency(dev, n_steps=64, reps=20):
             graph.replay()
         e1.record()
         torch.cuda.synchronize()
-        out[name] = {"us_per_step_eager": eager, "us_per_step_cuda_graph": e0.elapsed_time(e1) * 1e3 / (reps * n_steps)}
+        out[name] = {"us_per_step_eager": eager, "us_per_step_prepared_call": prep,
+                     "us_per_step_cuda_graph": e0.elapsed_time(e1) * 1e3 / (reps * n_steps)}
     # one clean chain from the common first state: both ends must arrive at the same state
     send_state.copy_(xs[0])
     recv_state.copy_(xs[0])
@@ -681,6 +703,10 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE {world}"
 
+    if args.sweep_only:
+        if rank == 0:
+            print(json.dumps({"sweep": config3_sweep(dev, measured_peak()[0])}))
+        return 0
     strong = args.scaling == "strong"
     if strong:
         # one tensor, the same on every rank; rank r codes the token range shard.token_range(T, r, world) against its
@@ -748,8 +774,9 @@ def main():
         pin = lambda t_: torch.empty(t_.shape, dtype=t_.dtype, pin_memory=True).copy_(t_)
         hX, hY, hq = pin(rt.X), pin(rt.Y), pin(rt.query)
         o_up = torch.empty(rt.pay_up.shape, dtype=torch.uint8, pin_memory=True)
-        o_dn = torch.empty_like(o_up).pin_memory()
+        o_dn = torch.empty(rt.pay_dn.shape, dtype=torch.uint8, pin_memory=True)
         o_Y = torch.empty(rt.Yh.shape, dtype=torch.bfloat16, pin_memory=True)
+        assert all(t_.is_pinned() for t_ in (hX, hY, hq, o_up, o_dn, o_Y)), "end-to-end buffers must be pinned"
         h2d = hX.numel() * 2 + hY.numel() * 2 + hq.numel() * 4
         d2h = o_up.numel() * 2 + o_Y.numel() * 2
         n_e2e = max(4, min(steps, 12))

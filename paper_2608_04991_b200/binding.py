@@ -73,9 +73,61 @@ class IndexCfg(C.Structure):
 _lib: Optional[C.CDLL] = None
 
 
-def load() -> C.CDLL:
+class _Recorder:
+    """Stands in for the library while `prepare` runs a wrapper once: launches are recorded instead of made."""
+
+    def __init__(self, lib):
+        self._lib = lib
+        self.calls = []
+
+    def __getattr__(self, name):
+        real = getattr(self._lib, name)
+        if real.restype is not C.c_int:      # size queries, strings: answer them
+            return real
+
+        def record(*args):
+            self.calls.append((name, real, args))
+            return RAC_OK
+        return record
+
+
+_recorder = None
+
+
+def prepare(wrapper, *args, **kwargs):
+    """Marshals the arguments of one call ONCE and returns a function without arguments that repeats the call.
+
+    ``wrapper`` is one of the functions of this module that launch work (``rac_encode_reconstruct``,
+    ``rac_decode_reconstruct``, ...), ``args`` what it would be given.  Tensor addresses, sizes and the stream
+    (``stream=`` or the current one at the time of this call) are fixed here; the tensors must stay alive and in
+    place.  For loops that issue the same small call many times (a decode step per token), where looking at a dozen
+    tensors costs more than the launch.  Not thread safe while it prepares."""
+    global _recorder
+    lib = load()
+    rec = _Recorder(lib)
+    _recorder = rec
+    try:
+        wrapper(*args, **kwargs)
+    finally:
+        _recorder = None
+    if len(rec.calls) != 1:
+        raise ValueError("prepare() wants a wrapper that makes exactly one library call")
+    name, real, cargs = rec.calls[0]
+    keep = (args, kwargs)      # the tensors (and the configuration struct the pointers refer to) stay referenced
+
+    def call():
+        rc = real(*cargs)
+        if rc != RAC_OK:
+            _check(name, rc)
+    call.keepalive = keep
+    return call
+
+
+def load():
     """Load the C-ABI library.  Raises if it has not been built (``__graft_entry__.build()``)."""
     global _lib
+    if _recorder is not None:
+        return _recorder
     if _lib is not None:
         return _lib
     if not os.path.exists(LIB_PATH):

@@ -291,6 +291,38 @@ def test_waits_that_cannot_complete_give_up_and_leave_the_stream_usable(env, d, 
         assert st == 0 and torch.equal(again_x, good_x)
 
 
+def test_prepared_calls_repeat_the_plain_calls(env):
+    """binding.prepare marshals the arguments of a call once; the function it returns launches the same work."""
+    d, g, bits, T = 3584, 128, 3, 64
+    s, rac, dev = env.synth, env.rac, env.dev
+    gen = s.generator(19, dev)
+    prev = s.activations(T, d, s.channel_scale(d, 19, dev), gen)
+    X = s.random_walk_step(prev, gen)
+    step, inv = env.orc.calibrate(d, g, bits, s.bf16_bits(X), ref_base=s.bf16_bits(prev))
+    step_d, inv_d = env.P.to_dev(step, dev), env.P.to_dev(inv, dev)
+    cfg = rac.CodecCfg(d, g, bits, 0)
+    rec = rac.rac_record_bytes(cfg)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pay_a, pay_b = (torch.zeros(T * rec, dtype=torch.uint8, device=dev) for _ in range(2))
+    xa, xb = torch.empty_like(X), torch.empty_like(X)
+    rac.rac_encode_reconstruct(cfg, X, T, prev, T, None, None, None, step_d, inv_d, pay_a, pay_a.numel(), xa, None, 0, status)
+    call = rac.prepare(rac.rac_encode_reconstruct, cfg, X, T, prev, T, None, None, None, step_d, inv_d, pay_b, pay_b.numel(),
+                       xb, None, 0, status)
+    torch.cuda.synchronize()
+    assert not pay_b.any()                      # preparing launches nothing
+    call()
+    call()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(pay_a, pay_b) and torch.equal(xa, xb)
+    dec = rac.prepare(rac.rac_decode_reconstruct, cfg, pay_b, T, prev, T, None, None, None, step_d, xb, status)
+    xb.zero_()
+    dec()
+    torch.cuda.synchronize()
+    assert torch.equal(xa, xb)
+    with pytest.raises(ValueError):             # a wrapper that launches nothing cannot be prepared
+        rac.prepare(rac.rac_record_bytes, cfg)
+
+
 def test_zero_tokens_is_a_no_op(env):
     cfg = env.rac.CodecCfg(4096, 128, 4, 8)
     t = torch.zeros(16, dtype=torch.uint8, device=env.dev)
