@@ -157,7 +157,8 @@ int rac_match_spans(const int32_t *hist_tok, int64_t n_hist, const int32_t *quer
  * launched.  The call allocates nothing and frees nothing, on the host side of CUDA or through any library.
  *
  * First call on a device: looks up the device address of the built-in array (one cudaGetSymbolAddress with
- * that device current).  Make that first call outside any stream capture.
+ * that device current).  Make that first call outside any stream capture.  The address is kept for the life of the
+ * process: after a cudaDeviceReset of that device it is stale, and this entry point must not be used again.
  * All calls on a device share the one array.  Its contents survive from call to call, but every call
  * re-initialises what it reads (hash table, rows, span count), so stale contents never matter.  Two calls that
  * overlap on the GPU (different streams, or several host threads) race on the array and give garbage: keep the
