@@ -130,7 +130,7 @@ int rac_header_parse(const void *header /* host, 64 bytes */, rac_codec_cfg *cfg
  *              match of the paper, the K-hit cap being a bucket policy).  The cost of a query position then
  *              grows with the number of occurrences of its window times the length they match over, so a
  *              history that repeats one token thousands of times is slow; keep the cap for token streams
- *              you do not control.  The persistent index (rac_index_*) takes 1..16 only.
+ *              you do not control.  The persistent index (rac_index_*) takes the same values.
  *   ref_row    int32[n_query]    out: history row of every covered position, -1 elsewhere
  *   spans      rac_span[n_query/min_ngram + 1]  out, in query order; may be NULL
  *   n_spans    int32[1]          out (device)
@@ -200,7 +200,7 @@ int rac_match_spans_static(const int32_t *hist_tok, int64_t n_hist, const int32_
 typedef struct {
     int64_t capacity;      /* history tokens the index can hold, 1 .. 2^30 - 1 */
     int32_t min_ngram;     /* w, 1..32 */
-    int32_t max_hits;      /* K, 1..16 */
+    int32_t max_hits;      /* K, 1..16, or 0 = no cap (every occurrence of a window is a candidate) */
 } rac_index_cfg;
 size_t rac_index_bytes(const rac_index_cfg *cfg);
 int rac_index_reset(const rac_index_cfg *cfg, void *index, size_t index_bytes, void *stream);

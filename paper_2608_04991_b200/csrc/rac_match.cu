@@ -371,8 +371,8 @@ struct IndexParams {
     int32_t *rep;       // [M]
     int32_t *top;       // [M*K]
     int32_t *end_of;    // [capacity]
-    int32_t *slot_of;   // [capacity]  slot of the window starting at each history position (append scratch)
-    int32_t *cnt;       // [M]         windows of the request being appended, per slot; zero between calls
+    int32_t *next;      // [capacity]  no cap on the hits: another start of the same window (chain link), else null
+    int32_t *cnt;       // [M]         unused (kept so that the layout of an index does not change)
     int a, b;           // the request: tokens [a, b)
     int w, K;
     unsigned int mask;
@@ -394,7 +394,9 @@ __global__ void index_append_kernel(IndexParams p) {
         if (cur == -1 || cur == j || same_window(p.hist + cur, win, p.w)) { slot = (int)s; break; }
         s = (s + 1) & p.mask;
     }
-    if (slot >= 0) cascade_insert(p.top + (long long)slot * p.K, p.K, j);
+    if (slot < 0) return;
+    if (p.next) p.next[j] = atomicExch(&p.top[slot], j);   // every start, on the slot's chain (order irrelevant)
+    else cascade_insert(p.top + (long long)slot * p.K, p.K, j);
 }
 
 // Intra-sequence references: first occurrence of every token of the prompt (a hash table keyed by a position
@@ -633,7 +635,7 @@ struct IndexLayout {
 };
 bool index_cfg_ok(const rac_index_cfg *c) {
     return c && c->capacity >= 1 && c->capacity < (1ll << 30) && c->min_ngram >= 1 && c->min_ngram <= 32 &&
-           c->max_hits >= 1 && c->max_hits <= 16;
+           c->max_hits >= 0 && c->max_hits <= 16;   // 0 = no cap: chains instead of K-lists
 }
 IndexLayout index_layout(const rac_index_cfg *c) {
     IndexLayout L;
@@ -642,7 +644,7 @@ IndexLayout index_layout(const rac_index_cfg *c) {
     L.M = (unsigned int)M;
     size_t o = 0;
     L.rep = o;      o += (size_t)M * 4;                        // rep and top contiguous: one fill with -1
-    L.top = o;      o = align16(o + (size_t)M * c->max_hits * 4);
+    L.top = o;      o = align16(o + (size_t)M * (c->max_hits > 0 ? c->max_hits : 1) * 4);
     L.cnt = o;      o = align16(o + (size_t)M * 4);
     L.end_of = o;   o = align16(o + (size_t)c->capacity * 4);
     L.slot_of = o;  o = align16(o + (size_t)c->capacity * 4);
@@ -690,7 +692,7 @@ int rac_index_reset(const rac_index_cfg *cfg, void *index, size_t index_bytes, v
     const IndexLayout L = index_layout(cfg);
     if (index_bytes < L.total) return RAC_ESIZE;
     unsigned char *ix = static_cast<unsigned char *>(index);
-    const long long table = (long long)L.M * (1 + cfg->max_hits);
+    const long long table = (long long)L.M * (1 + (cfg->max_hits > 0 ? cfg->max_hits : 1));
     fill2_i32_kernel<<<grid_for(table, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         reinterpret_cast<int32_t *>(ix + L.rep), table, -1, reinterpret_cast<int32_t *>(ix + L.cnt), (long long)L.M, 0);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
@@ -713,11 +715,11 @@ int rac_index_append(const rac_index_cfg *cfg, void *index, size_t index_bytes, 
     p.top = reinterpret_cast<int32_t *>(ix + L.top);
     p.cnt = reinterpret_cast<int32_t *>(ix + L.cnt);
     p.end_of = reinterpret_cast<int32_t *>(ix + L.end_of);
-    p.slot_of = reinterpret_cast<int32_t *>(ix + L.slot_of);
+    p.next = cfg->max_hits == 0 ? reinterpret_cast<int32_t *>(ix + L.slot_of) : nullptr;
     p.a = (int)n_before;
     p.b = (int)n_after;
     p.w = cfg->min_ngram;
-    p.K = cfg->max_hits;
+    p.K = cfg->max_hits > 0 ? cfg->max_hits : 1;
     p.mask = L.M - 1;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int tb = 256;
@@ -776,9 +778,9 @@ int rac_index_query_live(const rac_index_cfg *cfg, const void *index, size_t ind
     p.n_query = (int)n_query;
     p.nwin = (int)(n_hist - cfg->min_ngram + 1 > 0 ? n_hist - cfg->min_ngram + 1 : 0);
     p.w = cfg->min_ngram;
-    p.K = cfg->max_hits;
+    p.K = cfg->max_hits > 0 ? cfg->max_hits : 1;
     p.mask = L.M - 1;
-    p.next = nullptr;
+    p.next = cfg->max_hits == 0 ? const_cast<int32_t *>(reinterpret_cast<const int32_t *>(ix + L.slot_of)) : nullptr;
     p.first_live = (int)first_live;
     p.end_of = reinterpret_cast<const int32_t *>(ix + L.end_of);
     const int tb = 256;

@@ -217,7 +217,7 @@ def test_index_appended_request_by_request_matches_oracle(env, seed):
     rng = np.random.default_rng(700 + seed)
     vocab = [2, 3, 6, 40][seed % 4]
     w = [1, 2, 3, 4, 5][seed % 5]
-    K = [1, 2, 8, 16][seed % 4]
+    K = [1, 2, 8, 0][seed % 4]          # 0: no cap on the hits (chains instead of K-lists)
     ix = GpuIndex(env, 4096, w, K)
     reqs, off = [], [0]
     for step in range(7):
@@ -257,7 +257,7 @@ def test_index_live_window(env, seed):
     rng = np.random.default_rng(1300 + seed)
     vocab = [2, 3, 6, 40][seed % 4]
     w = [1, 2, 3, 4][seed % 4]
-    K = [1, 2, 8, 16][seed % 4]
+    K = [1, 0, 8, 16][seed % 4]
     ix = GpuIndex(env, 4096, w, K)
     reqs, off = [], [0]
     for step in range(6):
@@ -315,7 +315,8 @@ def test_index_argument_checks(env):
     rac = env.rac
     assert rac.rac_index_bytes(rac.IndexCfg(0, 4, 8)) == 0
     assert rac.rac_index_bytes(rac.IndexCfg(100, 0, 8)) == 0
-    assert rac.rac_index_bytes(rac.IndexCfg(100, 4, 17)) == 0
+    assert rac.rac_index_bytes(rac.IndexCfg(100, 4, 17)) == 0 and rac.rac_index_bytes(rac.IndexCfg(100, 4, -1)) == 0
+    assert 0 < rac.rac_index_bytes(rac.IndexCfg(100, 4, 0)) <= rac.rac_index_bytes(rac.IndexCfg(100, 4, 1))
     cfg = rac.IndexCfg(100, 4, 8)
     nb = rac.rac_index_bytes(cfg)
     mem = torch.zeros(nb, dtype=torch.uint8, device=env.dev)
