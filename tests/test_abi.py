@@ -130,3 +130,18 @@ def test_payload_header_round_trip_and_rejections(rac):
         rac.rac_header_write(rac.CodecCfg(4096, 100, 4, 0), 5)
     with pytest.raises(rac.RacError):
         rac.rac_header_write(cfgs[0], -1)
+
+
+def test_prepare_marshals_once_and_launches_nothing(rac):
+    """binding.prepare runs a wrapper against a recorder: the arguments are checked and marshalled, nothing is
+    called; the function it returns holds the library entry point and the marshalled arguments."""
+    A = 1 << 20          # a made-up, 16-byte aligned device address: never dereferenced here
+    cfg = rac.CodecCfg(4096, 128, 4, 0)
+    call = rac.prepare(rac.rac_decode_reconstruct, cfg, A, 16, A, 16, None, None, None, A, A, A, stream=0)
+    assert callable(call) and call.keepalive[0][0] is cfg
+    assert rac.load() is not None and not isinstance(rac.load(), rac._Recorder)      # the recorder is gone again
+    with pytest.raises(ValueError):
+        rac.prepare(rac.rac_record_bytes, cfg)                                       # a size query launches nothing
+    with pytest.raises(TypeError):
+        rac.prepare(rac.rac_decode_reconstruct, cfg, "not a tensor", 16, A, 16, None, None, None, A, A, A, stream=0)
+    assert not isinstance(rac.load(), rac._Recorder)                                 # also after a failed prepare
