@@ -248,7 +248,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                 find();
 #pragma unroll
                 for (int n = 0; n < KG; n++) {
-                    if (n < p.kg) {
+                    if (KG <= 2 || n < p.kg) {   // the launcher compiles in exactly k_g rounds for k_g = 1, 2
                         float gm = mloc;
 #pragma unroll
                         for (int o = 1; o < 8; o <<= 1)
@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                             const int js = (cq - rot) & 3;
 #pragma unroll
                             for (int j = 0; j < 4; j++) sm[j] = (j == js) ? cnm : sm[j];
-                            if (n + 1 < p.kg) find();
+                            if (KG <= 2 ? n + 1 < KG : n + 1 < p.kg) find();
                         }
                         sel[n] = __shfl_sync(group_mask, word, owner);
                     }
@@ -274,11 +274,11 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                     unsigned short *gv = reinterpret_cast<unsigned short *>(rec + p.gval_off) + jq * p.kg;
 #pragma unroll
                     for (int n = 0; n < KG; n++) {
-                        if (n < p.kg) {
+                        if (KG <= 2 || n < p.kg) {
                             int rank = 0;
 #pragma unroll
                             for (int q = 0; q < KG; q++)
-                                if (q < p.kg && (sel[q] & 0xffffu) < (sel[n] & 0xffffu)) rank++;
+                                if ((KG <= 2 || q < p.kg) && (sel[q] & 0xffffu) < (sel[n] & 0xffffu)) rank++;
                             go[rank] = (unsigned char)(sel[n] & 0xffu);
                             gv[rank] = (unsigned short)(sel[n] >> 16);
                         }
