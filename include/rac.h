@@ -70,8 +70,8 @@ extern "C" {
  *   bits    code width q: 2, 3 or 4; also 8 in scale_mode 1     (Qmax = 2^(bits-1) - 1, Eq. 8a)
  *   topk    outliers per TOKEN kept as binary16, 0..16 (u16 channel index); scale_mode 0 only
  *   coef_fmt   0 = one binary16 pair per (token, group), in the record
- *              1 = one binary16 pair per (segment, group), outside the record (scale_mode 1 only; see
- *                  rac_fit_segments): the record then starts with the scales
+ *              1 = one binary16 pair per (segment, group), outside the record (see rac_fit_segments): the
+ *                  record then starts with the scales (scale_mode 1) or with the codes (scale_mode 0)
  *   scale_mode 0 = static per-channel step table `step`/`inv_step` (calibrated clip; dense values may clip);
  *                  g_q == g_a, `qgroup` 0 or == group, `topk_group` 0
  *              1 = Eq. 8 as printed: per quantisation group the scale s = RoundUp_binary16(max|E^d| / Qmax) is
@@ -351,8 +351,8 @@ int rac_decode_reconstruct_list(const rac_codec_cfg *cfg, const void *payload, i
  * Eq. 6 over several fitting positions: one coefficient pair per (segment of consecutive tokens, group)
  * instead of one per (token, group).  H_j and R_j of Eq. 6 are then the [positions x group] slices of the
  * segment; a token coded directly contributes r = 0.  The pairs are shared by the tokens of the segment and
- * travel once per segment, outside the records: rac_codec_cfg.coef_fmt = 1 (scale_mode 1 only) gives records
- * without coefficient words.
+ * travel once per segment, outside the records: rac_codec_cfg.coef_fmt = 1 gives records without coefficient
+ * words, in either scale mode (with the static table: [codes][outlier indices][outlier values]).
  *
  * rac_fit_segments
  *   seg_off   device int32[n_seg + 1], ascending, seg_off[0] = 0, seg_off[n_seg] = T; equal neighbours = an
@@ -394,6 +394,15 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T,
                         const void *ref_gain, const void *ref_bias, float clip_sigmas,
                         float *step, float *inv_step, void *workspace, size_t workspace_bytes,
                         uint32_t *dev_status, void *stream);
+/* The same for shared coefficients (cfg->coef_fmt = 1, scale_mode 0): the residual of every calibration token is
+ * taken with the pair of its segment, coef_seg[seg_of[t]] as rac_fit_segments wrote them over the same T tokens.
+ * rac_calibrate_steps wants coef_fmt = 0, this call coef_fmt = 1 and both arrays (RAC_EINVAL otherwise). */
+int rac_calibrate_steps_shared(const rac_codec_cfg *cfg, const void *X, int64_t T,
+                               const void *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                               const void *ref_gain, const void *ref_bias,
+                               const uint32_t *coef_seg, const int32_t *seg_of, float clip_sigmas,
+                               float *step, float *inv_step, void *workspace, size_t workspace_bytes,
+                               uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Reconstruction error of a sender-path run: the measurable half of the offline calibration of Sec. IV-C

@@ -89,6 +89,9 @@ def _declare(l: C.CDLL) -> None:
     l.orc_calibrate.restype = C.c_int
     l.orc_calibrate.argtypes = [C.c_int] * 3 + [_u16p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p,
                                                 C.c_double, _f32p, _f32p]
+    l.orc_calibrate_shared.restype = C.c_int
+    l.orc_calibrate_shared.argtypes = [C.c_int] * 3 + [_u16p, C.c_int64, _u16p, C.c_int64, _i32p, _u16p, _u16p, _u32p,
+                                                       C.c_double, _f32p, _f32p]
     l.orc_match_spans.restype = C.c_int
     l.orc_match_spans.argtypes = [_i32p, C.c_int64, _i32p, C.c_int64, C.c_int, C.c_int, _i32p, _i32p, _i32p]
     l.orc_match_spans_req.restype = C.c_int
@@ -277,8 +280,9 @@ def reconstruct(d, group, bits, topk, payload, T, ref_base=None, ref_row=None, g
     return (out, st.value) if return_status else out
 
 
-def calibrate(d, group, bits, X, ref_base=None, ref_row=None, gain=None, bias=None, clip_sigmas=3.0):
-    """Step tables (step, inv_step), float32[2,d] each, from a calibration draw."""
+def calibrate(d, group, bits, X, ref_base=None, ref_row=None, gain=None, bias=None, clip_sigmas=3.0, shared_coef=None):
+    """Step tables (step, inv_step), float32[2,d] each, from a calibration draw.  ``shared_coef`` uint32[T,J]: every
+    token's residual is taken with the wire words of its segment (Eq. 6 over several fitting positions)."""
     X = _chk(X, np.uint16)
     T = X.size // d
     ref_base = _chk(ref_base, np.uint16)
@@ -288,8 +292,14 @@ def calibrate(d, group, bits, X, ref_base=None, ref_row=None, gain=None, bias=No
     bias = _chk(bias, np.uint16, d)
     step = np.zeros((2, d), np.float32)
     inv = np.zeros((2, d), np.float32)
-    rc = lib().orc_calibrate(d, group, bits, _p(X, _u16p), T, _p(ref_base, _u16p), ref_rows, _p(ref_row, _i32p),
-                             _p(gain, _u16p), _p(bias, _u16p), float(clip_sigmas), _p(step, _f32p), _p(inv, _f32p))
+    if shared_coef is not None:
+        shared_coef = _chk(shared_coef, np.uint32, T * (d // group))
+        rc = lib().orc_calibrate_shared(d, group, bits, _p(X, _u16p), T, _p(ref_base, _u16p), ref_rows,
+                                        _p(ref_row, _i32p), _p(gain, _u16p), _p(bias, _u16p), _p(shared_coef, _u32p),
+                                        float(clip_sigmas), _p(step, _f32p), _p(inv, _f32p))
+    else:
+        rc = lib().orc_calibrate(d, group, bits, _p(X, _u16p), T, _p(ref_base, _u16p), ref_rows, _p(ref_row, _i32p),
+                                 _p(gain, _u16p), _p(bias, _u16p), float(clip_sigmas), _p(step, _f32p), _p(inv, _f32p))
     if rc != 0:
         raise ValueError(f"orc_calibrate failed: {rc}")
     return step, inv

@@ -27,6 +27,8 @@
  *   orc_calibrate        "offline calibration" of Sec. IV-C reduced to the one
  *                        thing the codec needs as an input: a per-channel step
  *                        from the RMS of the aligned residual.
+ *   orc_calibrate_shared the same with the wire words of every token given
+ *                        from outside (Eq. 6 solved over several positions).
  *
  * Readings taken where the paper is silent:
  *   - one fit per (token, group): the "fitting positions" of Eq. 6 are the
@@ -639,12 +641,15 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qg
  * binary32 residual of Eq. 7 with wire coefficients.  step = smallest
  * binary16 >= clip_sigmas*sigma/Qmax (held as float), inv_step = 1.0f/step in
  * binary32; a row without tokens, or a channel with sigma 0, gets step 0 and
- * inv_step 0. */
-int orc_calibrate(int d, int group, int bits,
-                  const uint16_t *X, int64_t T,
-                  const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
-                  const uint16_t *gain, const uint16_t *bias,
-                  double clip_sigmas, float *step, float *inv_step) {
+ * inv_step 0.
+ * shared_coef (u32[T,J] or NULL): with Eq. 6 solved over several fitting
+ * positions every token uses the wire words of its segment; the residual is
+ * then taken with those instead of the token's own fit. */
+static int calibrate_impl(int d, int group, int bits,
+                          const uint16_t *X, int64_t T,
+                          const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                          const uint16_t *gain, const uint16_t *bias, const uint32_t *shared_coef,
+                          double clip_sigmas, float *step, float *inv_step) {
     if (!cfg_ok(d, group, bits, 0)) return -1;
     const int J = d / group;
     const int qmax = (1 << (bits - 1)) - 1;
@@ -660,10 +665,17 @@ int orc_calibrate(int d, int group, int bits,
         int row = has_ref ? 0 : 1;
         cnt[row]++;
         for (int j = 0; j < J; j++) {
-            double as, bs;
-            orc_fit_group(h + j * group, r + j * group, group, has_ref, &as, &bs, NULL, NULL);
-            float a = orc_f16_to_f32(orc_f64_to_f16(as));
-            float b = orc_f16_to_f32(orc_f64_to_f16(bs));
+            float a, b;
+            if (shared_coef) {
+                const uint32_t w = shared_coef[t * (int64_t)J + j];
+                a = orc_f16_to_f32((uint16_t)(w & 0xffffu));
+                b = orc_f16_to_f32((uint16_t)(w >> 16));
+            } else {
+                double as, bs;
+                orc_fit_group(h + j * group, r + j * group, group, has_ref, &as, &bs, NULL, NULL);
+                a = orc_f16_to_f32(orc_f64_to_f16(as));
+                b = orc_f16_to_f32(orc_f64_to_f16(bs));
+            }
             for (int c = j * group; c < (j + 1) * group; c++) {
                 float rt = fmaf(a, r[c], b);
                 float e = h[c] - rt;
@@ -688,6 +700,23 @@ int orc_calibrate(int d, int group, int bits,
     }
     free(acc); free(h); free(r);
     return err;
+}
+
+int orc_calibrate(int d, int group, int bits,
+                  const uint16_t *X, int64_t T,
+                  const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                  const uint16_t *gain, const uint16_t *bias,
+                  double clip_sigmas, float *step, float *inv_step) {
+    return calibrate_impl(d, group, bits, X, T, ref_base, ref_rows, ref_row, gain, bias, NULL, clip_sigmas, step, inv_step);
+}
+
+int orc_calibrate_shared(int d, int group, int bits,
+                         const uint16_t *X, int64_t T,
+                         const uint16_t *ref_base, int64_t ref_rows, const int32_t *ref_row,
+                         const uint16_t *gain, const uint16_t *bias, const uint32_t *shared_coef,
+                         double clip_sigmas, float *step, float *inv_step) {
+    if (!shared_coef) return -1;
+    return calibrate_impl(d, group, bits, X, T, ref_base, ref_rows, ref_row, gain, bias, shared_coef, clip_sigmas, step, inv_step);
 }
 
 /* ------------------------------------------------------------------ */

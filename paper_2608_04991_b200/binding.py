@@ -36,7 +36,7 @@ EXPORTS = [
     "rac_sender_reconstruct",
     "rac_split_waves", "rac_encode_reconstruct_list", "rac_decode_reconstruct_list",
     "rac_fit_segments_workspace_bytes", "rac_fit_segments", "rac_spans_to_segments",
-    "rac_calibrate_workspace_bytes", "rac_calibrate_steps",
+    "rac_calibrate_workspace_bytes", "rac_calibrate_steps", "rac_calibrate_steps_shared",
     "rac_recon_error_workspace_bytes", "rac_recon_error",
     "rac_selftest_bounded_wait",
 ]
@@ -202,6 +202,8 @@ def load():
     l.rac_calibrate_workspace_bytes.argtypes = [cfgp]
     l.rac_calibrate_steps.restype = C.c_int
     l.rac_calibrate_steps.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, C.c_float, vp, vp, vp, sz, vp, vp]
+    l.rac_calibrate_steps_shared.restype = C.c_int
+    l.rac_calibrate_steps_shared.argtypes = [cfgp, vp, i64, vp, i64, vp, vp, vp, vp, vp, C.c_float, vp, vp, vp, sz, vp, vp]
     _lib = l
     return l
 
@@ -493,3 +495,16 @@ def rac_calibrate_steps(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bi
                                     int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"),
                                     _stream() if stream is None else stream)
     _check("rac_calibrate_steps", rc)
+
+
+def rac_calibrate_steps_shared(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, coef_seg, seg_of, clip_sigmas,
+                               step, inv_step, workspace, workspace_bytes, dev_status, stream=None) -> None:
+    rc = load().rac_calibrate_steps_shared(C.byref(cfg), _ptr(X, _BF16, "X"), int(T), _ptr(ref_base, _BF16, "ref_base"),
+                                           int(ref_rows), _ptr(ref_row, _I32, "ref_row"),
+                                           _ptr(ref_gain, _F16, "ref_gain"), _ptr(ref_bias, _F16, "ref_bias"),
+                                           _ptr(coef_seg, _I32, "coef_seg"), _ptr(seg_of, _I32, "seg_of"),
+                                           float(clip_sigmas), _ptr(step, _F32, "step"),
+                                           _ptr(inv_step, _F32, "inv_step"), _ptr(workspace, None, "workspace"),
+                                           int(workspace_bytes), _ptr(dev_status, _I32, "dev_status"),
+                                           _stream() if stream is None else stream)
+    _check("rac_calibrate_steps_shared", rc)

@@ -36,7 +36,6 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     if (cfg->d <= 0 || cfg->group <= 0 || cfg->topk < 0 || cfg->bits <= 0) return RAC_EINVAL;
     if (cfg->qgroup < 0 || cfg->topk_group < 0) return RAC_EINVAL;
     if ((cfg->coef_fmt != 0 && cfg->coef_fmt != 1) || cfg->flags != 0) return RAC_EUNSUPPORTED;
-    if (cfg->coef_fmt == 1 && cfg->scale_mode != 1) return RAC_EUNSUPPORTED;   // shared coefficients: Eq. 8 family only
     if (cfg->scale_mode != 0 && cfg->scale_mode != 1) return RAC_EUNSUPPORTED;
     if (cfg->d % cfg->group) return RAC_EINVAL;
     if (cfg->d % 32 || cfg->d > 8192) return RAC_EUNSUPPORTED;
@@ -182,7 +181,15 @@ __global__ void __launch_bounds__(256, 2) calib_kernel(const CodecParams p) {
             }
             u64 a2, b2;
             float4 st;
-            fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, nullptr, &st);
+            if (!MOMENTS && p.coef_ext) {
+                // shared coefficients: the residual of Eq. 7 with the words of the token's segment
+                const uint32_t cw = p.coef_ext[(long long)p.seg_of[tok] * p.J + (tid >> p.lpg_shift)];
+                const float a = half_bits_to_float(cw & 0xffffu), b = half_bits_to_float(cw >> 16);
+                a2 = pack2(a, a);
+                b2 = pack2(b, b);
+            } else {
+                fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, nullptr, &st);
+            }
             if (MOMENTS) {
                 if (!timed_out && (lane & (p.lpg - 1)) == 0) p.moments[tok * p.J + (tid >> p.lpg_shift)] = st;
             }
@@ -259,6 +266,7 @@ struct WsCtrl {
     unsigned long long full[kMaxStages];
     unsigned long long done[kMaxStages];
     int row[kMaxStages];
+    int seg[kMaxStages];   // segment of the token in each stage (shared coefficients only)
     int abort;
 };
 
@@ -306,6 +314,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         const long long t = token_at<SUB>(p, first + (long long)k * stride);
         const int row = resolve_row<SUB>(p, raw_row);
         ctrl->row[s] = row;
+        if constexpr (SUB) ctrl->seg[s] = p.seg_of ? p.seg_of[t] : 0;
         const uint32_t bar = smem_u32(&ctrl->full[s]);
         const uint32_t base = sbase + L.stage0 + s * L.stage_bytes;
         mbar_arrive_expect_tx(bar, p.test_extra_tx + row_bytes + (row >= 0 ? row_bytes : 0u));
@@ -321,9 +330,14 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         ctrl->abort = 0;
         mbar_init_fence();
     }
+    // shared coefficients (one pair per segment and group, Eq. 6 over several positions) come from outside the
+    // records: no coefficient words in front of the codes
+    bool shared = false;
+    if constexpr (SUB) shared = p.coef_ext != nullptr;
+    const int coff = shared ? 0 : 4 * p.J;
     {
         // padding words of the records are written once and never touched again
-        const int raw = 4 * p.J + p.code_bytes + 4 * p.topk;
+        const int raw = coff + p.code_bytes + 4 * p.topk;
         for (int s = 0; s < 2 * S; s++)
             for (int o = raw + 4 * tid; o < p.rec; o += 4 * nt)
                 *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * p.rec + o) = 0u;
@@ -375,13 +389,20 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             }
             // ---- (2) Eq. 6 and wire rounding
             u64 a2, b2;
-            uint32_t coef_word;
             constexpr int kShift = LPG == 4 ? 2 : 1;
             const int lpg = LPG ? LPG : p.lpg, lpg_shift = LPG ? kShift : p.lpg_shift;
-            fit_group(x2, r2, has_ref, lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
+            if (shared) {
+                const uint32_t cw = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> lpg_shift)];
+                const float a = half_bits_to_float(cw & 0xffffu), b = half_bits_to_float(cw >> 16);
+                a2 = pack2(a, a);
+                b2 = pack2(b, b);
+            } else {
+                uint32_t coef_word;
+                fit_group(x2, r2, has_ref, lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
+                if ((lane & (lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> lpg_shift] = coef_word;
+            }
 
             // ---- (3) Eq. 7 residual, Eq. 8 quantisation with the static table, packing
-            if ((lane & (lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> lpg_shift] = coef_word;
             const float *inv_tab = p.inv_step + (has_ref ? 0 : d);
             const float *step_tab = p.step + (has_ref ? 0 : d);
             uint32_t words[4];
@@ -459,7 +480,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                 }
             }
             rot_right4(words, rot);  // words[q] is now the code word of piece q
-            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + 4 * p.J) + tid * BITS;
+            uint32_t *cw = reinterpret_cast<uint32_t *>(rec + coff) + tid * BITS;
             if (BITS == 4) {
                 cw[0] = words[0]; cw[1] = words[1]; cw[2] = words[2]; cw[3] = words[3];
             } else if (BITS == 3) {
@@ -618,6 +639,9 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
     const int my0 = NV * lane;                  // first slab of this lane
     const int my_n = min(NV, max(0, nth - my0));  // how many of its NV slabs exist
     const int coef_shift = 5 + p.lpg_shift;
+    bool shared = false;   // coefficient words per segment, outside the records
+    if constexpr (SUB) shared = p.coef_ext != nullptr;
+    const int coff = shared ? 0 : 4 * p.J;
     // everything this kernel reads was written by the streaming pass launched just before it
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const long long n_tok = tokens_to_do<SUB>(p);
@@ -625,6 +649,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
     for (long long ti0 = ((long long)blockIdx.x * kOutWarps + warp) * U; ti0 < n_tok; ti0 += tstride) {
         long long t[U];
         const uint16_t *xrow[U], *rrow[U];
+        const uint32_t *coefp[U];
         unsigned char *rec[U];
         unsigned int tau[U];
         int nh[U], n[U];
@@ -658,6 +683,9 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
             xrow[u] = p.X + t[u] * d;
             rrow[u] = row >= 0 ? ref_row_ptr<SUB>(p, row) : nullptr;
             rec[u] = p.payload + t[u] * p.rec;
+            coefp[u] = reinterpret_cast<const uint32_t *>(rec[u]);
+            if constexpr (SUB)
+                if (shared) coefp[u] = p.coef_ext + (long long)(live[u] ? p.seg_of[t[u]] : 0) * p.J;
             // threshold.  Bit patterns of non-negative floats order like integers.
             unsigned int m1 = tv[0], m2 = 0u;
 #pragma unroll
@@ -709,7 +737,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
             if (act) {
                 xw = __ldg(reinterpret_cast<const uint4 *>(xrow[u] + c0));
                 if (rrow[u]) rw = __ldg(reinterpret_cast<const uint4 *>(rrow[u] + c0));
-                cf = reinterpret_cast<const uint32_t *>(rec[u])[c0 >> coef_shift];
+                cf = coefp[u][c0 >> coef_shift];
             }
         };
         auto use_round = [&](int u, int c0, bool act, const uint4 &xw, const uint4 &rw, uint32_t cf) {
@@ -812,8 +840,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
                     if (lane == 31 - __clz(bal)) { mag = 0xffffffffu; won = false; }   // among equals the highest channel
                 }
             } else {
-                select_whole_token(d, k, coef_shift, xrow[u], rrow[u], p.gain, p.bias,
-                                   reinterpret_cast<const uint32_t *>(rec[u]), lane, &wc, &we, &wrt);
+                select_whole_token(d, k, coef_shift, xrow[u], rrow[u], p.gain, p.bias, coefp[u], lane, &wc, &we, &wrt);
                 won = lane < k;
             }
             // ---- (d) outlier fields in channel order, dense codes at those channels cleared
@@ -826,14 +853,14 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
                 }
             }
             if (won) {
-                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec[u] + 4 * p.J + p.code_bytes);
+                unsigned short *oidx = reinterpret_cast<unsigned short *>(rec[u] + coff + p.code_bytes);
                 const uint32_t hv = float_to_half_bits_sat(we);
                 oidx[pos] = (unsigned short)wc;
                 oidx[k + pos] = (unsigned short)hv;
                 // the sender-side reconstruction of an outlier channel: (alpha*r + beta) + the binary16 value
                 if (want_xhat)
                     p.X_hat[t[u] * d + wc] = __bfloat16_as_ushort(__float2bfloat16_rn(__fadd_rn(wrt, half_bits_to_float(hv))));
-                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec[u] + 4 * p.J);
+                uint32_t *codes32 = reinterpret_cast<uint32_t *>(rec[u] + coff);
                 const int bit = wc * bits, wd = bit >> 5, sh = bit & 31;
                 atomicAnd(&codes32[wd], ~(cmask << sh));
                 if (sh + bits > 32) atomicAnd(&codes32[wd + 1], ~(cmask >> (32 - sh)));
@@ -906,6 +933,9 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
     }
     __syncthreads();
 
+    bool shared = false;   // coefficient words per segment, outside the records
+    if constexpr (SUB) shared = p.coef_ext != nullptr;
+    const int coff = shared ? 0 : 4 * p.J;
     const int first = blockIdx.x, stride = gridDim.x;
     const long long n_tok = tokens_to_do<SUB>(p);
     const int n_my = (n_tok > first) ? (int)((n_tok - first + stride - 1) / stride) : 0;
@@ -919,7 +949,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
         for (int k = 0; k < S - 1 && k < n_my; k++) {
             long long t = token_at<SUB>(p, first + (long long)k * stride);
             issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + k * L.stage_bytes, L.rec_pad, k, resolve_row<SUB>(p, raw_row_of(k)),
-                              p.payload + t * p.rec, (uint32_t)p.rec);
+                              p.payload + t * p.rec, (uint32_t)p.rec, t);
         }
         if (S - 1 < n_my) next_raw = raw_row_of(S - 1);
     }
@@ -952,7 +982,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             const int k = it + S - 1;
             const long long tk = token_at<SUB>(p, first + (long long)k * stride);
             issue_token_loads<SUB>(p, ctrl, sbase + L.stage0 + issue_stage * L.stage_bytes, L.rec_pad, issue_stage,
-                              resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec);
+                              resolve_row<SUB>(p, next_raw), p.payload + tk * p.rec, (uint32_t)p.rec, tk);
             if (k + 1 < n_my) next_raw = raw_row_of(k + 1);
         }
         const bool timed_out = !mbar_wait_bounded(smem_u32(&ctrl->bar[stage]), parity);
@@ -964,11 +994,13 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
         const uint32_t obs = smem_u32(ob);
 
         if (valid) {
-            const uint32_t cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
+            uint32_t cf;
+            if (shared) cf = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> p.lpg_shift)];
+            else cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
             const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
             const u64 a2 = pack2(a, a), b2 = pack2(b, b);
             // code words of the four pieces, in piece order, then rotated into slot order
-            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + 4 * p.J) + tid * BITS;
+            const uint32_t *cw = reinterpret_cast<const uint32_t *>(rec + coff) + tid * BITS;
             uint32_t words[4];
             if (BITS == 4) {
                 words[0] = cw[0]; words[1] = cw[1]; words[2] = cw[2]; words[3] = cw[3];
@@ -1021,7 +1053,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             }
             if (KT > 0) {
                 // outliers whose channel this thread owns replace what the dense pass wrote
-                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
+                const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + coff + p.code_bytes);
                 const unsigned short *oval = oidx + p.topk;
 #pragma unroll
                 for (int n = 0; n < KT; n++) {
@@ -1041,7 +1073,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const CodecParams p) {
             }
         }
         if (KT > 0 && tid == 0) {
-            const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + 4 * p.J + p.code_bytes);
+            const unsigned short *oidx = reinterpret_cast<const unsigned short *>(rec + coff + p.code_bytes);
             bool bad = false;
             for (int n = 0; n < p.topk; n++) bad |= oidx[n] >= d;
             if (bad && p.status) atomicOr(p.status, RAC_STATUS_OUTLIER_RANGE);
@@ -2004,10 +2036,10 @@ size_t rac_calibrate_workspace_bytes(const rac_codec_cfg *cfg) {
     return (size_t)kCalibGrid * 2 * (size_t)g.d * sizeof(float) + (size_t)kCalibGrid * 2 * sizeof(int);
 }
 
-int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
-                        const int32_t *ref_row, const void *ref_gain, const void *ref_bias, float clip_sigmas,
-                        float *step, float *inv_step, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
-                        void *stream) {
+static int calibrate_impl(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+                          const int32_t *ref_row, const void *ref_gain, const void *ref_bias, const uint32_t *coef_seg,
+                          const int32_t *seg_of, float clip_sigmas, float *step, float *inv_step, void *workspace,
+                          size_t workspace_bytes, uint32_t *dev_status, void *stream) {
     Geometry g;
     int rc = make_geometry(cfg, &g);
     if (rc != RAC_OK) return rc;
@@ -2015,6 +2047,9 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, cons
     rc = fill_common(g, &p, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, dev_status);
     if (rc != RAC_OK) return rc;
     if (g.scale_mode != 0) return RAC_EUNSUPPORTED;   // the tables belong to the static quantiser only
+    if ((g.coef_fmt == 1) != (coef_seg != nullptr) || (coef_seg != nullptr) != (seg_of != nullptr)) return RAC_EINVAL;
+    p.coef_ext = coef_seg;
+    p.seg_of = seg_of;
     if (!step || !inv_step || !workspace || !(clip_sigmas > 0.f)) return RAC_EINVAL;
     if (T > 0 && !X) return RAC_EINVAL;
     if (!aligned16(X) || !aligned16(workspace) || !aligned16(step) || !aligned16(inv_step)) return RAC_EALIGN;
@@ -2037,6 +2072,24 @@ int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, cons
     int n = 2 * g.d;
     calib_finalize_kernel<<<(n + 255) / 256, 256, 0, st>>>(p.calib_partial, kCalibGrid, g.d, g.bits, clip_sigmas, step, inv_step);
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
+}
+
+int rac_calibrate_steps(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+                        const int32_t *ref_row, const void *ref_gain, const void *ref_bias, float clip_sigmas,
+                        float *step, float *inv_step, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                        void *stream) {
+    return calibrate_impl(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, nullptr, nullptr, clip_sigmas, step,
+                          inv_step, workspace, workspace_bytes, dev_status, stream);
+}
+
+int rac_calibrate_steps_shared(const rac_codec_cfg *cfg, const void *X, int64_t T, const void *ref_base, int64_t ref_rows,
+                               const int32_t *ref_row, const void *ref_gain, const void *ref_bias,
+                               const uint32_t *coef_seg, const int32_t *seg_of, float clip_sigmas, float *step,
+                               float *inv_step, void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                               void *stream) {
+    if (!coef_seg || !seg_of) return RAC_EINVAL;
+    return calibrate_impl(cfg, X, T, ref_base, ref_rows, ref_row, ref_gain, ref_bias, coef_seg, seg_of, clip_sigmas, step,
+                          inv_step, workspace, workspace_bytes, dev_status, stream);
 }
 
 }  // extern "C"

@@ -119,7 +119,108 @@ def test_segment_fit_and_shared_coefficient_coding_match_oracle(env, d, g, T, kw
         assert e.value.code == -1
     with pytest.raises(rac.RacError):
         rac.rac_decode_reconstruct(cfg, pay[:T * rec], T, R, T, rows_d, None, None, None, xd, st)
-    assert rac.rac_record_bytes(rac.CodecCfg(d, g, 4, 0, coef_fmt=1)) == 0        # static table: per-token pairs only
+    assert rac.rac_record_bytes(rac.CodecCfg(d, g, 4, 0, coef_fmt=1)) == (d // 2 + 15) // 16 * 16   # static table: codes only
+
+
+@pytest.mark.parametrize("d,g,T,bits,k,with_gain", [
+    (1024, 128, 300, 4, 0, False),
+    (5120, 128, 257, 4, 8, False),
+    (4096, 64, 130, 3, 8, True),
+    (96, 32, 41, 2, 3, False),
+])
+def test_shared_coefficients_with_the_static_table(env, d, g, T, bits, k, with_gain):
+    """coef_fmt = 1 with scale_mode 0: records are [codes][outlier indices][outlier values]; the step table is
+    calibrated on the residuals of the shared fit; everything bit-identical to the oracle given the device's words."""
+    s, rac, orc, dev = env.synth, env.rac, env.orc, env.dev
+    J = d // g
+    gen = s.generator(1300 + d, dev)
+    scale = s.channel_scale(d, 13, dev)
+    X = s.activations(T, d, scale, gen)
+    R = s.affine_noisy_reference(X, g, gen)
+    rows = np.arange(T, dtype=np.int32)
+    rows[T // 3: T // 3 + 7] = -1
+    rows_d = torch.from_numpy(rows).to(dev)
+    gain = bias = gb = bb = None
+    if with_gain:
+        gain = (1.0 + 0.1 * torch.randn(d, generator=gen, device=dev)).to(torch.float16)
+        bias = (0.02 * torch.randn(d, generator=gen, device=dev)).to(torch.float16)
+        gb, bb = gain.cpu().numpy().view(np.uint16), bias.cpu().numpy().view(np.uint16)
+    rng = np.random.default_rng(d + k)
+    cuts = np.sort(rng.choice(np.arange(1, T), size=9, replace=False))
+    seg_off = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    cfg = rac.CodecCfg(d, g, bits, k, coef_fmt=1)
+    rec = rac.rac_record_bytes(cfg)
+    assert rec == orc.record_bytes(d, g, bits, k, 0, 0, 0, 1) == (d * bits // 8 + 4 * k + 15) // 16 * 16
+    coef_d, seg_of_d, _ = device_fit(env, cfg, X, R, rows_d, seg_off, gain, bias)
+    g_coef = coef_d.cpu().numpy().view(np.uint32)
+    seg_of = np.repeat(np.arange(len(seg_off) - 1), np.diff(seg_off)).astype(np.int32)
+    per_tok = np.ascontiguousarray(g_coef[seg_of])
+    Xb, Rb = s.bf16_bits(X), s.bf16_bits(R)
+
+    # ---- step table from the residuals of the shared fit
+    step = torch.empty((2, d), dtype=torch.float32, device=dev)
+    inv = torch.empty_like(step)
+    nb = rac.rac_calibrate_workspace_bytes(cfg)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    rac.rac_calibrate_steps_shared(cfg, X, T, R, T, rows_d, gain, bias, coef_d, seg_of_d, 3.0, step, inv, ws, nb, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    o_step, o_inv = orc.calibrate(d, g, bits, Xb, ref_base=Rb, ref_row=rows, gain=gb, bias=bb, shared_coef=per_tok)
+    gs = step.cpu().numpy()
+    ulp = np.spacing(o_step.astype(np.float16)).astype(np.float32)
+    assert np.all(np.abs(gs - o_step) <= ulp) and (gs != o_step).mean() < 0.02
+    # the residual of a shared fit is wider than that of the token's own fit
+    own = orc.calibrate(d, g, bits, Xb, ref_base=Rb, ref_row=rows, gain=gb, bias=bb)[0]
+    assert np.median(o_step[0] / own[0]) > 1.0
+    for c, cs in ((rac.CodecCfg(d, g, bits, k), coef_d), (cfg, None)):
+        with pytest.raises(rac.RacError) as e:
+            if cs is None:
+                rac.rac_calibrate_steps(c, X, T, R, T, rows_d, gain, bias, 3.0, step.clone(), inv.clone(), ws, nb, st)
+            else:
+                rac.rac_calibrate_steps_shared(c, X, T, R, T, rows_d, gain, bias, cs, seg_of_d, 3.0, step.clone(),
+                                               inv.clone(), ws, nb, st)
+        assert e.value.code == -1
+
+    # ---- coding: the device's table and words on both sides
+    gi = inv.cpu().numpy()
+    pay = torch.full((T * rec + 64,), 0xA5, dtype=torch.uint8, device=dev)
+    xh = torch.full((T + 1, d), -7.0, dtype=torch.bfloat16, device=dev)
+    nws = rac.rac_encode_workspace_bytes(cfg, T)
+    ews = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
+    rac.rac_encode_reconstruct_list(cfg, X, T, None, None, R, T, rows_d, None, 0, gain, bias, step, inv, pay, T * rec,
+                                    xh[:T], ews if nws else None, nws, st, coef_seg=coef_d, seg_of=seg_of_d)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and torch.all(pay[T * rec:] == 0xA5) and torch.all(xh[T] == -7.0)
+    o_pay = orc.encode(d, g, bits, k, Xb, ref_base=Rb, ref_row=rows, gain=gb, bias=bb, step=gs, inv_step=gi,
+                       forced_coef=per_tok.reshape(-1).copy(), coef_fmt=1, nthreads=orc.max_threads())
+    g_pay = pay[:T * rec].cpu().numpy()
+    if not np.array_equal(g_pay, o_pay):
+        bad = np.flatnonzero((g_pay.reshape(T, rec) != o_pay.reshape(T, rec)).any(axis=1))
+        off = np.flatnonzero(g_pay.reshape(T, rec)[bad[0]] != o_pay.reshape(T, rec)[bad[0]])
+        raise AssertionError(f"{bad.size} records differ; first token {bad[0]}, byte offsets {off[:8].tolist()} of {rec}")
+    o_x = orc.reconstruct(d, g, bits, k, o_pay, T, ref_base=Rb, ref_row=rows, gain=gb, bias=bb, step=gs, coef_fmt=1,
+                          shared_coef=per_tok, nthreads=orc.max_threads())
+    assert np.array_equal(o_x, s.bf16_bits(xh[:T]))
+    xd = torch.empty((T, d), dtype=torch.bfloat16, device=dev)
+    rac.rac_decode_reconstruct_list(cfg, pay[:T * rec], T, None, None, R, T, rows_d, None, 0, gain, bias, step, xd, st,
+                                    coef_seg=coef_d, seg_of=seg_of_d)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and torch.equal(xd, xh[:T])
+    # a token list: only those records and rows are written
+    lst = torch.from_numpy(np.arange(1, T, 3, dtype=np.int32)).to(dev)
+    cnt = torch.tensor([lst.numel()], dtype=torch.int32, device=dev)
+    pay2 = torch.full_like(pay, 0x3C)
+    rac.rac_encode_reconstruct_list(cfg, X, T, lst, cnt, R, T, rows_d, None, 0, gain, bias, step, inv, pay2, T * rec,
+                                    None, ews if nws else None, nws, st, coef_seg=coef_d, seg_of=seg_of_d)
+    torch.cuda.synchronize()
+    p2, p1 = pay2[:T * rec].view(T, rec), pay[:T * rec].view(T, rec)
+    sel = torch.zeros(T, dtype=torch.bool, device=dev)
+    sel[lst.long()] = True
+    assert int(st.item()) == 0 and torch.equal(p2[sel], p1[sel]) and torch.all(p2[~sel] == 0x3C)
+    # the per-token record format and the shared words do not mix
+    with pytest.raises(rac.RacError):
+        rac.rac_decode_reconstruct(cfg, pay[:T * rec], T, R, T, rows_d, gain, bias, step, xd, st)
 
 
 def test_one_long_segment_and_single_token_segments(env):

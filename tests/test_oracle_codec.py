@@ -344,6 +344,44 @@ def test_calibrated_step_is_three_sigma_rounded_up(orc):
     assert not step[1].any() and not inv[1].any()
 
 
+def test_calibration_with_shared_coefficient_words(orc):
+    """Residuals taken with words that come from outside (Eq. 6 over several positions): an independent numpy
+    evaluation with hand-picked words, and the reduction to the per-token form when the words are the tokens' own."""
+    d, g, bits, T = 128, 32, 3, 96
+    J = d // g
+    gen = synth.generator(71)
+    X = synth.activations(T, d, synth.channel_scale(d, 6), gen)
+    R = synth.affine_noisy_reference(X, g, gen)
+    Xb, Rb = synth.bf16_bits(X), synth.bf16_bits(R)
+    rows = np.arange(T, dtype=np.int32)
+    rows[10:20] = -1                                                     # direct tokens: table row 1, r = 0
+    rng = np.random.default_rng(5)
+    a16 = rng.choice(np.array([0.5, 0.75, 1.0, 1.25], np.float16), (T, J))
+    b16 = rng.choice(np.array([-0.25, 0.0, 0.125], np.float16), (T, J))
+    words = (a16.view(np.uint16).astype(np.uint32) | (b16.view(np.uint16).astype(np.uint32) << 16))
+    step, inv = orc.calibrate(d, g, bits, Xb, ref_base=Rb, ref_row=rows, shared_coef=words)
+    h = X.float().numpy().astype(np.float64)
+    r = R.float().numpy().astype(np.float64)
+    r[rows < 0] = 0.0
+    # binary32 fma and subtraction, as Eq. 7 is evaluated: emulate with float64 then round (exact for these inputs'
+    # products: bf16 x binary16 has <= 19 significant bits; the sum is rounded once to binary32)
+    rt = (np.repeat(a16.astype(np.float64), g, axis=1) * r + np.repeat(b16.astype(np.float64), g, axis=1)).astype(np.float32)
+    e = (X.float().numpy() - rt).astype(np.float64)
+    for row, mask in ((0, rows >= 0), (1, rows < 0)):
+        sigma = np.sqrt((e[mask] ** 2).mean(axis=0))
+        want = 3.0 * sigma / 3.0                                         # Qmax = 3 for 3-bit codes
+        ulp = np.spacing(step[row].astype(np.float16)).astype(np.float64)
+        assert np.all(step[row] >= want * (1 - 1e-6)) and np.all(step[row] <= want * (1 + 1e-6) + ulp)
+        assert np.array_equal(inv[row], (np.float32(1) / step[row]).astype(np.float32))
+    # the tokens' own wire words reproduce the per-token calibration exactly
+    _, dg = orc.encode(d, g, bits, 0, Xb, ref_base=Rb, ref_row=rows, step=step, inv_step=inv, diag=True)
+    pay = orc.encode(d, g, bits, 0, Xb, ref_base=Rb, ref_row=rows, step=step, inv_step=inv)
+    own = pay.reshape(T, -1)[:, :4 * J].copy().view(np.uint32).reshape(T, J)
+    s0, i0 = orc.calibrate(d, g, bits, Xb, ref_base=Rb, ref_row=rows)
+    s1, i1 = orc.calibrate(d, g, bits, Xb, ref_base=Rb, ref_row=rows, shared_coef=own)
+    assert np.array_equal(s0, s1) and np.array_equal(i0, i1)
+
+
 # ------------------------------------------------------------------ Eq. 8 as printed: dynamic per-group scale
 @pytest.mark.parametrize("bits,topk", [(4, 0), (3, 0), (2, 0), (4, 8)])
 def test_dynamic_scale_never_clips_and_rounds_up(orc, bits, topk):
