@@ -80,9 +80,11 @@ extern "C" {
  *   flags   must be 0
  *   qgroup  g_q, channels per quantisation group (scale_mode 1): 0 = same as `group`; a power of two 32..1024
  *           that divides d; or d itself (the paper's decode mode: one scale per token)
- *   topk_group  k_g, outliers per quantisation group (Sec. IV-C "Outlier Metadata"), 0..8, scale_mode 1 with
- *           qgroup <= 256: the k_g largest |e| of every group (ties to the lower channel) leave the dense base
- *           before its scale is taken; one-byte in-group offsets in ascending order + binary16 values */
+ *   topk_group  k_g, outliers per quantisation group (Sec. IV-C "Outlier Metadata"), 0..8, scale_mode 1 with a
+ *           power-of-two qgroup (not with qgroup = d unless d is such a value): the k_g largest |e| of every
+ *           group (ties to the lower channel) leave the dense base before its scale is taken; in-group offsets in
+ *           ascending order (one byte each for groups of up to 256 channels, two bytes little-endian for 512 and
+ *           1024; the field is padded to an even size) + binary16 values */
 typedef struct {
     int32_t d, group, bits, topk, coef_fmt, scale_mode, flags, qgroup, topk_group;
 } rac_codec_cfg;

@@ -164,7 +164,8 @@ def split_payload(payload: np.ndarray, T: int, d: int, group: int, bits: int, to
                   qgroup: int = 0, topk_group: int = 0, coef_fmt: int = 0):
     """Views into a payload: coef u32[T,J], codes u8[T,d*b/8], out_idx u16[T,k], out_val u16[T,k];
     for scale_mode 1 also scale u16[T,Jq] as a fifth item, and with per-group outliers
-    grp_off u8[T,Jq,kg] and grp_val u16[T,Jq,kg] as a sixth and seventh."""
+    grp_off u8[T,Jq,kg] (u16 when the group has more than 256 channels) and grp_val u16[T,Jq,kg] as a sixth and
+    seventh."""
     J = d // group
     qg = qgroup or group
     Jq = d // qg
@@ -185,8 +186,12 @@ def split_payload(payload: np.ndarray, T: int, d: int, group: int, bits: int, to
         return coef, codes, oi, ov, scale
     ng = Jq * topk_group
     g0 = o + nb + 4 * topk
-    g1 = g0 + (ng + 1) // 2 * 2
-    goff = np.ascontiguousarray(p[:, g0: g0 + ng]).reshape(T, Jq, topk_group)
+    wide = qg > 256                            # two-byte offsets for groups of more than 256 channels
+    g1 = g0 + (ng * (2 if wide else 1) + 1) // 2 * 2
+    if wide:
+        goff = np.ascontiguousarray(p[:, g0: g0 + 2 * ng]).view(np.uint16).reshape(T, Jq, topk_group)
+    else:
+        goff = np.ascontiguousarray(p[:, g0: g0 + ng]).reshape(T, Jq, topk_group)
     gval = np.ascontiguousarray(p[:, g1: g1 + 2 * ng]).view(np.uint16).reshape(T, Jq, topk_group)
     return coef, codes, oi, ov, scale, goff, gval
 

@@ -165,13 +165,18 @@ static int64_t scale_bytes(int d, int qgroup, int scale_mode) {
     return scale_mode == 1 ? (2 * (int64_t)(d / qgroup) + 3) / 4 * 4 : 0;
 }
 
+/* in-group offsets of the per-group outliers: one byte each while a group has at most 256 channels, two
+ * (little endian) for wider groups; the field is padded to an even number of bytes */
+static int goff_width(int qgroup) { return qgroup > 256 ? 2 : 1; }
+static int64_t goff_bytes(int64_t ng, int qgroup) { return (ng * goff_width(qgroup) + 1) / 2 * 2; }
+
 /* qgroup 0 means "same as group"; topk_group outliers per quantisation group; coef_fmt 1: the coefficient
  * pairs are shared by the tokens of a segment and travel outside the record */
 int64_t orc_record_bytes_full(int d, int group, int bits, int topk, int scale_mode, int qgroup, int topk_group, int coef_fmt) {
     if (qgroup == 0) qgroup = group;
     int64_t ng = (int64_t)(d / qgroup) * topk_group;
     int64_t raw = (coef_fmt == 1 ? 0 : 4 * (int64_t)(d / group)) + scale_bytes(d, qgroup, scale_mode) + ((int64_t)d * bits) / 8 +
-                  4 * (int64_t)topk + (ng + 1) / 2 * 2 + 2 * ng;
+                  4 * (int64_t)topk + goff_bytes(ng, qgroup) + 2 * ng;
     return (raw + 15) / 16 * 16;
 }
 
@@ -200,7 +205,7 @@ static int qcfg_ok(int d, int group, int topk, int scale_mode, int qgroup, int t
     if (scale_mode == 0) return (qgroup == 0 || qgroup == group) && topk_group == 0;
     if (qgroup == 0) qgroup = group;
     if (d % qgroup) return 0;
-    if (topk_group && (topk || qgroup > 256 || topk_group > qgroup)) return 0;
+    if (topk_group && (topk || qgroup > 65536 || topk_group > qgroup)) return 0;
     return 1;
 }
 
@@ -407,7 +412,7 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
             uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             uint8_t *oval = oidx + 2 * topk;
             uint8_t *goff = oval + 2 * topk;
-            uint8_t *gval = goff + ((int64_t)Jq * topk_group + 1) / 2 * 2;
+            uint8_t *gval = goff + goff_bytes((int64_t)Jq * topk_group, qgroup);
 
             for (int c = 0; c < d; c++) h[c] = orc_bf16_to_f32(X[t * (int64_t)d + c]);
             int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
@@ -477,7 +482,13 @@ int orc_encode(int d, int group, int bits, int topk, int scale_mode, int qgroup,
                 for (int c = j * qgroup; c < (j + 1) * qgroup; c++) {
                     if (!is_out[c]) continue;
                     uint16_t hv = orc_f64_to_f16((double)clampf(e[c], -65504.0f, 65504.0f));
-                    goff[j * topk_group + n] = (uint8_t)(c - j * qgroup);
+                    const int o = c - j * qgroup;
+                    if (goff_width(qgroup) == 1) {
+                        goff[j * topk_group + n] = (uint8_t)o;
+                    } else {
+                        goff[2 * (j * topk_group + n)] = (uint8_t)(o & 0xff);
+                        goff[2 * (j * topk_group + n) + 1] = (uint8_t)(o >> 8);
+                    }
                     memcpy(gval + 2 * (j * topk_group + n), &hv, 2);
                     n++;
                 }
@@ -572,7 +583,7 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qg
             const uint8_t *oidx = codes + ((int64_t)d * bits) / 8;
             const uint8_t *oval = oidx + 2 * topk;
             const uint8_t *goff = oval + 2 * topk;
-            const uint8_t *gval = goff + ((int64_t)Jq * topk_group + 1) / 2 * 2;
+            const uint8_t *gval = goff + goff_bytes((int64_t)Jq * topk_group, qgroup);
             int has_ref = resolve_ref(d, t, ref_base, ref_rows, ref_row, gain, bias, r);
             if (has_ref < 0) {
 #pragma omp atomic write
@@ -604,7 +615,7 @@ int orc_reconstruct(int d, int group, int bits, int topk, int scale_mode, int qg
             }
             for (int n = 0; n < Jq * topk_group; n++) {
                 uint16_t hv;
-                int o = goff[n];
+                int o = goff_width(qgroup) == 1 ? goff[n] : (goff[2 * n] | (goff[2 * n + 1] << 8));
                 memcpy(&hv, gval + 2 * n, 2);
                 if (o >= qgroup) {
 #pragma omp atomic write

@@ -59,7 +59,7 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
         else if (qgroup == cfg->d) lpq = 0;   // one scale per token, exchanged through shared memory
         else return RAC_EUNSUPPORTED;
         if (cfg->topk_group > 8) return RAC_EUNSUPPORTED;
-        if (cfg->topk_group > 0 && (lpq == 0 || qgroup > 256)) return RAC_EUNSUPPORTED;   // one-byte offsets
+        if (cfg->topk_group > 0 && lpq == 0) return RAC_EUNSUPPORTED;   // a group must lie within one warp
     }
     g->d = cfg->d;
     g->group = cfg->group;
@@ -79,7 +79,7 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     g->codes_off = g->scale_off + (cfg->scale_mode == 1 ? (2 * g->Jq + 3) / 4 * 4 : 0);
     const int ng = g->Jq * g->topk_group;
     g->goff_off = g->codes_off + g->code_bytes + 4 * cfg->topk;
-    g->gval_off = g->goff_off + (ng + 1) / 2 * 2;
+    g->gval_off = g->goff_off + (ng * (qgroup > 256 ? 2 : 1) + 1) / 2 * 2;   // one-byte offsets up to 256 channels, two beyond
     const int raw = g->gval_off + 2 * ng;
     g->rec = (raw + 15) / 16 * 16;
     return RAC_OK;

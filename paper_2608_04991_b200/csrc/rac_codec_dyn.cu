@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                     if (KG <= 2 || n < p.kg) {   // the launcher compiles in exactly k_g rounds for k_g = 1, 2
                         float gm = mloc;
 #pragma unroll
-                        for (int o = 1; o < 8; o <<= 1)
+                        for (int o = 1; o < 32; o <<= 1)
                             if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
                         const uint32_t gb = (__ballot_sync(group_mask, mloc == gm) >> qbase) & qlanes;
                         const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);   // gb == 0 only with NaNs around
@@ -270,7 +270,9 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                 }
                 if ((lane & (p.lpq - 1)) == 0) {
                     // the group's first lane serialises them in ascending offset order
+                    const bool wide = p.lpq > 8;   // more than 256 channels per group: two-byte offsets
                     unsigned char *go = rec + p.goff_off + jq * p.kg;
+                    unsigned short *go2 = reinterpret_cast<unsigned short *>(rec + p.goff_off) + jq * p.kg;
                     unsigned short *gv = reinterpret_cast<unsigned short *>(rec + p.gval_off) + jq * p.kg;
 #pragma unroll
                     for (int n = 0; n < KG; n++) {
@@ -279,7 +281,8 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
 #pragma unroll
                             for (int q = 0; q < KG; q++)
                                 if ((KG <= 2 || q < p.kg) && (sel[q] & 0xffffu) < (sel[n] & 0xffffu)) rank++;
-                            go[rank] = (unsigned char)(sel[n] & 0xffu);
+                            if (wide) go2[rank] = (unsigned short)(sel[n] & 0xffffu);
+                            else go[rank] = (unsigned char)(sel[n] & 0xffu);
                             gv[rank] = (unsigned short)(sel[n] >> 16);
                         }
                     }
@@ -601,14 +604,16 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
             }
             if (KG) {
                 // outliers of this thread's group that fall into its own 32 channels, in record order
+                const bool wide = p.lpq > 8;   // more than 256 channels per group: two-byte offsets
                 const unsigned char *go = rec + p.goff_off + jq * p.kg;
+                const unsigned short *go2 = reinterpret_cast<const unsigned short *>(rec + p.goff_off) + jq * p.kg;
                 const unsigned short *gv = reinterpret_cast<const unsigned short *>(rec + p.gval_off) + jq * p.kg;
                 const int qsize = p.lpq * 32;
                 bool bad = false;
 #pragma unroll
                 for (int n = 0; n < 8; n++) {
                     if (n < p.kg) {
-                        const int o = go[n];
+                        const int o = wide ? (int)go2[n] : (int)go[n];
                         if (o >= qsize) {
                             bad = true;
                         } else if ((o >> 5) == (tid & (p.lpq - 1))) {

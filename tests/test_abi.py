@@ -49,7 +49,9 @@ def test_record_geometry_matches_the_wire_format(rac, orc):
         assert rac.rac_record_bytes(rac.CodecCfg(d, g, b, 0, scale_mode=1, qgroup=qg, topk_group=kg)) == \
             orc.record_bytes(d, g, b, 0, 1, qg, kg)
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 8, 0)) == 0
-    assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 4, 0, scale_mode=1, qgroup=512, topk_group=1)) == 0
+    assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 4, 0, scale_mode=1, qgroup=512, topk_group=3)) == \
+        orc.record_bytes(4096, 128, 4, 0, 1, 512, 3)                   # wide groups: two-byte offsets
+    assert rac.rac_record_bytes(rac.CodecCfg(5120, 128, 4, 0, scale_mode=1, qgroup=5120, topk_group=1)) == 0   # group wider than a warp
     assert C.sizeof(rac.CodecCfg) == 36
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 100, 4, 0)) == 0   # group does not divide d
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 5, 0)) == 0   # unsupported width

@@ -487,6 +487,10 @@ def test_dynamic_group_scale_identity_and_rejections(env):
     (4096, 128, 4, 0, 8, 70),       # eight outliers per group of 128
     (5120, 128, 4, 256, 6, 41),     # six, groups of eight lanes
     (4096, 64, 8, 32, 5, 23),       # five in groups of one lane, 8-bit codes
+    (4096, 128, 4, 512, 3, 40),     # groups of 16 lanes: two-byte offsets
+    (5120, 128, 8, 1024, 8, 25),    # groups of a whole warp
+    (1024, 128, 4, 1024, 2, 30),    # g_q = d inside one warp, with outliers
+    (2048, 64, 3, 512, 5, 33),
 ])
 def test_family_matches_oracle(env, d, g, bits, qg, kg, T):
     X, R, _, _ = prefill_inputs(env, T, d, g, seed=3000 + d + bits + qg + kg)
@@ -532,7 +536,7 @@ def test_family_ties_zero_groups_and_bad_offsets(env):
     diff = (xb != good).nonzero().cpu().numpy()
     assert len(diff) == 1 and diff[0][0] == 3 and diff[0][1] == 5 * 32 + keep   # only the outlier that was dropped
     # configurations this build has no kernel for
-    for bad_cfg in [env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=512, topk_group=1),   # one-byte offsets
+    for bad_cfg in [env.rac.CodecCfg(5120, g, 4, 0, scale_mode=1, qgroup=5120, topk_group=1),   # a group wider than a warp
                     env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, topk_group=9),
                     env.rac.CodecCfg(d, g, 8, 0),                                           # 8 bits: Eq. 8 family only
                     env.rac.CodecCfg(d, g, 4, 0, qgroup=64),                                # static table: g_q = g_a
@@ -686,7 +690,7 @@ def test_random_configurations_on_stressed_inputs(env):
         T = int(rng.integers(1, 400 if d <= 2080 else 120))
         if fam:
             cfg = rac.CodecCfg(d, g, int(rng.choice([2, 3, 4, 8])), 0, scale_mode=1,
-                               qgroup=int(rng.choice([0, 32, 64, 128, 256, d])), topk_group=int(rng.choice([0, 0, 1, 2, 3, 4, 7, 8])))
+                               qgroup=int(rng.choice([0, 32, 64, 128, 256, 512, 1024, d])), topk_group=int(rng.choice([0, 0, 1, 2, 3, 4, 7, 8])))
             if rac.rac_record_bytes(cfg) == 0:
                 continue
         else:

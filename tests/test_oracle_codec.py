@@ -479,6 +479,7 @@ def test_family_record_by_hand(orc):
 @pytest.mark.parametrize("bits,g,qg,kg", [
     (4, 64, 64, 1), (4, 64, 64, 2), (8, 64, 64, 1), (4, 128, 32, 4), (4, 32, 128, 2), (3, 64, 256, 3),
     (8, 64, 0, 0), (8, 64, 512, 0), (4, 64, 512, 0), (2, 128, 512, 0), (4, 128, 16, 1),
+    (4, 64, 512, 3), (8, 128, 512, 6),     # groups of more than 256 channels: two-byte offsets
 ])
 def test_family_outliers_per_group_and_token_scale(orc, bits, g, qg, kg):
     d, T = 512, 24
@@ -492,7 +493,8 @@ def test_family_outliers_per_group_and_token_scale(orc, bits, g, qg, kg):
     pay = orc.encode(d, g, bits, 0, Xb, ref_base=Rb, **kw)
     # record size from the layout, typed out
     ng = Jq * kg
-    raw = 4 * (d // g) + (2 * Jq + 3) // 4 * 4 + d * bits // 8 + (ng + 1) // 2 * 2 + 2 * ng
+    off_bytes = 2 if q_g > 256 else 1
+    raw = 4 * (d // g) + (2 * Jq + 3) // 4 * 4 + d * bits // 8 + (ng * off_bytes + 1) // 2 * 2 + 2 * ng
     assert orc.record_bytes(d, g, bits, 0, 1, qg, kg) == (raw + 15) // 16 * 16 == pay.size // T
     parts = orc.split_payload(pay, T, d, g, bits, 0, 1, qg, kg)
     coef, codes, scale = parts[0], parts[1], parts[4]
@@ -552,9 +554,13 @@ def test_family_token_scale_is_the_token_maximum_and_rejections(orc):
     q = np.stack([orc.unpack_codes(codes[t], d, 8) for t in range(T)])
     assert np.all(np.abs(q).max(axis=1) == 127)          # one scale per token: exactly the token's largest |e| is at the end
     assert np.array_equal(codes.view(np.int8).astype(np.int32), q)   # 8-bit codes are plain signed bytes
-    orc.encode(d, g, 4, 0, Xb, scale_mode=1, qgroup=d, topk_group=1)        # offsets are one byte: g_q = 256 still fits
+    # offsets are one byte up to g_q = 256 and two beyond: one more byte per outlier in the record
+    r256 = orc.encode(d, g, 4, 0, Xb, scale_mode=1, qgroup=d, topk_group=2).size // T
+    assert r256 == (4 * (d // g) + 4 + d // 2 + 2 + 4 + 15) // 16 * 16
+    r512 = orc.encode(512, g, 4, 0, np.zeros((1, 512), np.uint16), scale_mode=1, qgroup=512, topk_group=2).size
+    assert r512 == (4 * (512 // g) + 4 + 512 // 2 + 4 + 4 + 15) // 16 * 16
     with pytest.raises(ValueError):
-        orc.encode(512, g, 4, 0, np.zeros((1, 512), np.uint16), scale_mode=1, qgroup=512, topk_group=1)
+        orc.encode(d, g, 4, 0, Xb, scale_mode=1, qgroup=d, topk_group=d + 1)    # more outliers than channels in a group
     with pytest.raises(ValueError):
         orc.encode(d, g, 4, 2, Xb, scale_mode=1, topk_group=1)              # one outlier rule at a time
     with pytest.raises(ValueError):
