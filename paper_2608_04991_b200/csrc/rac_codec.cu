@@ -566,7 +566,6 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
 // all-zero residual): k rounds of a maximum over the whole token instead.  (d) The winners go into the record's
 // outlier fields in channel order, their dense codes are cleared (E^d = E - O), and with the sender-side
 // reconstruction those channels of x_hat are replaced.
-constexpr int kOutWarps = 8;       // warps per CTA
 constexpr int kOutCap = 32;        // candidates per token: one per lane
 
 // eight values by a run-time index, as a select tree (no local-memory array)
@@ -621,18 +620,20 @@ __device__ __noinline__ void select_whole_token(int d, int k, int coef_shift, co
 // bound this pass) overlap.
 constexpr int kOutPair = 2;
 
-template <int NV, int KT, bool SUB>
-__global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecParams p, const int bits) {
+// W: warps per CTA.  7 = four CTAs of 72 registers per SM (56 tokens in flight), the faster shape without x_hat;
+// 8 = three CTAs of 80 registers (48 tokens), which the variant that also patches x_hat prefers.
+template <int NV, int KT, bool SUB, int W>
+__global__ void __launch_bounds__(W * 32, W == 7 ? 4 : 3) outlier_kernel(const CodecParams p, const int bits) {
     constexpr int U = kOutPair;
-    __shared__ float s_e[kOutWarps][U][kOutCap];
-    __shared__ float s_rt[kOutWarps][U][kOutCap];
-    __shared__ unsigned short s_c[kOutWarps][U][kOutCap];
-    __shared__ unsigned char s_hot[kOutWarps][U][32 * NV];
+    __shared__ float s_e[W][U][kOutCap];
+    __shared__ float s_rt[W][U][kOutCap];
+    __shared__ unsigned short s_c[W][U][kOutCap];
+    __shared__ unsigned char s_hot[W][U][32 * NV];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int d = p.d, nth = d >> 5;
     const int k = KT ? KT : p.topk;
     const uint32_t cmask = (1u << bits) - 1u;
-    const long long tstride = (long long)gridDim.x * kOutWarps * U;
+    const long long tstride = (long long)gridDim.x * W * U;
     const unsigned int lt_mask = (1u << lane) - 1u;
     const int tm_stride = (nth + 3) & ~3;       // rows of slab maxima are padded to 16 bytes
     const bool want_xhat = p.X_hat != nullptr;
@@ -646,7 +647,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 3) outlier_kernel(const CodecP
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const long long n_tok = tokens_to_do<SUB>(p);
 
-    for (long long ti0 = ((long long)blockIdx.x * kOutWarps + warp) * U; ti0 < n_tok; ti0 += tstride) {
+    for (long long ti0 = ((long long)blockIdx.x * W + warp) * U; ti0 < n_tok; ti0 += tstride) {
         long long t[U];
         const uint16_t *xrow[U], *rrow[U];
         const uint32_t *coefp[U];
@@ -1448,28 +1449,34 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != RAC_OK) return rc;
-    // a warp per token
-    // three CTAs of 80 registers per SM; with more work than one round of them, every warp gets the same number of
-    // rounds (a grid of whole rounds, not a full grid with a ragged last round)
-    const long long per_cta = kOutWarps * kOutPair;
+    // a warp per pair of tokens.  Without x_hat: four CTAs of seven warps per SM (72 registers); with x_hat (more state per
+    // token): three CTAs of eight warps (80 registers).  With more work than one round of them, every warp gets the same
+    // number of rounds (a grid of whole rounds, not a full grid with a ragged last round).
+    const bool wide = p.X_hat != nullptr || sub;
+    const int wpc = wide ? 8 : 7;
+    const long long per_cta = wpc * kOutPair;
     long long blocks = (p.T + per_cta - 1) / per_cta;
-    const long long resident = (long long)di.sms * 3;
+    const long long resident = (long long)di.sms * (wide ? 3 : 4);
     if (blocks > resident) {
         const long long rounds = (blocks + resident - 1) / resident;
         blocks = (blocks + rounds - 1) / rounds;
     }
     const int nth = g.d / 32;
-    const unsigned nb = (unsigned)blocks, nt = kOutWarps * 32;
-    if (sub) launch_after(outlier_kernel<8, 0, true>, nb, nt, stream, p, g.bits);
+    const unsigned nb = (unsigned)blocks, nt = wpc * 32;
+#define RAC_OUT(NV, KT)                                                                    \
+    (wide ? launch_after(outlier_kernel<NV, KT, false, 8>, nb, nt, stream, p, g.bits)     \
+          : launch_after(outlier_kernel<NV, KT, false, 7>, nb, nt, stream, p, g.bits))
+    if (sub) launch_after(outlier_kernel<8, 0, true, 8>, nb, nt, stream, p, g.bits);
     else if (g.topk == 8) {
-        if (nth <= 128) launch_after(outlier_kernel<4, 8, false>, nb, nt, stream, p, g.bits);
-        else if (nth <= 160) launch_after(outlier_kernel<5, 8, false>, nb, nt, stream, p, g.bits);
-        else launch_after(outlier_kernel<8, 8, false>, nb, nt, stream, p, g.bits);
+        if (nth <= 128) RAC_OUT(4, 8);
+        else if (nth <= 160) RAC_OUT(5, 8);
+        else RAC_OUT(8, 8);
     } else {
-        if (nth <= 128) launch_after(outlier_kernel<4, 0, false>, nb, nt, stream, p, g.bits);
-        else if (nth <= 160) launch_after(outlier_kernel<5, 0, false>, nb, nt, stream, p, g.bits);
-        else launch_after(outlier_kernel<8, 0, false>, nb, nt, stream, p, g.bits);
+        if (nth <= 128) RAC_OUT(4, 0);
+        else if (nth <= 160) RAC_OUT(5, 0);
+        else RAC_OUT(8, 0);
     }
+#undef RAC_OUT
     return cudaGetLastError() == cudaSuccess ? RAC_OK : RAC_ECUDA;
 }
 
