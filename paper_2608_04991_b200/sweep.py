@@ -2,8 +2,9 @@
 
 For every candidate configuration the sender path is run on the given activations (step tables from
 ``rac_calibrate_steps`` where the configuration needs them, then ``rac_encode_reconstruct``) and the packed bytes per
-token are reported beside the reconstruction error (``rac_recon_error``).  Picking a configuration against a
-model-quality target needs the model and its evaluation suites and is not done here.
+token are reported beside the reconstruction error (``rac_recon_error``).  Members with shared coefficient pairs
+(``coef_fmt = 1``) run ``rac_fit_segments`` first and count their shared words towards the bytes.  Picking a
+configuration against a model-quality target needs the model and its evaluation suites and is not done here.
 
 Every step runs in the CUDA kernels of the C-ABI library; this module only loops over configurations.
 
@@ -21,8 +22,11 @@ from . import synth
 
 
 def sweep(X: torch.Tensor, ref_base: Optional[torch.Tensor], ref_row: Optional[torch.Tensor],
-          configs: Iterable[rac.CodecCfg], gain=None, bias=None, clip_sigmas: float = 3.0, reps: int = 3) -> List[dict]:
-    """X bf16[T,d] on a CUDA device; ``ref_base`` / ``ref_row`` / ``gain`` / ``bias`` as for ``rac_encode``."""
+          configs: Iterable[rac.CodecCfg], gain=None, bias=None, clip_sigmas: float = 3.0, reps: int = 3,
+          seg_off: Optional[torch.Tensor] = None) -> List[dict]:
+    """X bf16[T,d] on a CUDA device; ``ref_base`` / ``ref_row`` / ``gain`` / ``bias`` as for ``rac_encode``.
+    Configurations with ``coef_fmt = 1`` (one coefficient pair per segment and group, Eq. 6 over several positions) need
+    ``seg_off``, int32[n_seg + 1] on the device; their shared words count towards the bytes per token."""
     dev = X.device
     T, d = X.shape
     ref_rows = 0 if ref_base is None else ref_base.shape[0]
@@ -37,7 +41,29 @@ def sweep(X: torch.Tensor, ref_base: Optional[torch.Tensor], ref_row: Optional[t
         if rec == 0:
             raise ValueError(f"unsupported configuration {cfg!r}")
         step = inv = None
-        if cfg.scale_mode == 0:
+        shared = cfg.coef_fmt == 1
+        coef_seg = seg_of = None
+        extra = 0.0
+        if shared:
+            if seg_off is None:
+                raise ValueError("a configuration with coef_fmt = 1 needs seg_off")
+            n_seg = seg_off.numel() - 1
+            J = d // cfg.group
+            coef_seg = torch.empty((n_seg, J), dtype=torch.int32, device=dev)
+            seg_of = torch.empty(T, dtype=torch.int32, device=dev)
+            nbf = rac.rac_fit_segments_workspace_bytes(cfg, T)
+            wsf = torch.empty(nbf, dtype=torch.uint8, device=dev)
+            rac.rac_fit_segments(cfg, X, T, ref_base, ref_rows, ref_row, gain, bias, seg_off, n_seg, coef_seg, seg_of,
+                                 wsf, nbf, status)
+            extra = 4.0 * J * n_seg / T
+        if cfg.scale_mode == 0 and shared:
+            step = torch.empty((2, d), dtype=torch.float32, device=dev)
+            inv = torch.empty_like(step)
+            nb = rac.rac_calibrate_workspace_bytes(cfg)
+            ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+            rac.rac_calibrate_steps_shared(cfg, X, T, ref_base, ref_rows, ref_row, gain, bias, coef_seg, seg_of,
+                                           clip_sigmas, step, inv, ws, nb, status)
+        elif cfg.scale_mode == 0:
             step = torch.empty((2, d), dtype=torch.float32, device=dev)
             inv = torch.empty_like(step)
             nb = rac.rac_calibrate_workspace_bytes(cfg)
@@ -47,8 +73,13 @@ def sweep(X: torch.Tensor, ref_base: Optional[torch.Tensor], ref_row: Optional[t
         pay = torch.empty(T * rec, dtype=torch.uint8, device=dev)
         nws = rac.rac_encode_workspace_bytes(cfg, T)
         ws2 = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
-        run = lambda: rac.rac_encode_reconstruct(cfg, X, T, ref_base, ref_rows, ref_row, gain, bias, step, inv, pay,
-                                                 pay.numel(), x_hat, ws2 if nws else None, nws, status)
+        if shared:
+            run = lambda: rac.rac_encode_reconstruct_list(cfg, X, T, None, None, ref_base, ref_rows, ref_row, None, 0, gain,
+                                                          bias, step, inv, pay, pay.numel(), x_hat, ws2 if nws else None,
+                                                          nws, status, coef_seg=coef_seg, seg_of=seg_of)
+        else:
+            run = lambda: rac.rac_encode_reconstruct(cfg, X, T, ref_base, ref_rows, ref_row, gain, bias, step, inv, pay,
+                                                     pay.numel(), x_hat, ws2 if nws else None, nws, status)
         run()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
@@ -62,7 +93,8 @@ def sweep(X: torch.Tensor, ref_base: Optional[torch.Tensor], ref_row: Optional[t
         out.append({
             "group": cfg.group, "bits": cfg.bits, "topk": cfg.topk, "scale_mode": cfg.scale_mode,
             "qgroup": cfg.qgroup or cfg.group, "topk_group": cfg.topk_group,
-            "record_bytes": rec, "payload_over_raw": rec / (2.0 * d),
+            "coef_fmt": cfg.coef_fmt, "record_bytes": rec, "shared_bytes_per_token": extra,
+            "payload_over_raw": (rec + extra) / (2.0 * d),
             "rel_rms_error": (se / sx) ** 0.5 if sx > 0 else 0.0, "max_abs_error": mx,
             "encode_reconstruct_ms": e0.elapsed_time(e1) / reps, "status": int(status.item()),
         })
@@ -85,11 +117,19 @@ def default_grid(d: int) -> List[rac.CodecCfg]:
     return cfgs
 
 
+def shared_grid(d: int) -> List[rac.CodecCfg]:
+    """Members whose coefficient pairs are shared by the tokens of a segment (they need ``seg_off``)."""
+    return [rac.CodecCfg(d, 128, 4, 8, coef_fmt=1), rac.CodecCfg(d, 128, 4, 0, coef_fmt=1),
+            rac.CodecCfg(d, 128, 4, 0, scale_mode=1, coef_fmt=1), rac.CodecCfg(d, 128, 4, 0, scale_mode=1, topk_group=1, coef_fmt=1)]
+
+
 def main() -> int:
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
     ap.add_argument("--tokens", type=int, default=16384)
     ap.add_argument("--d", type=int, default=4096)
     ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--segment", type=int, default=64, help="tokens per segment for the members with shared coefficient "
+                    "pairs (0 leaves them out)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("the sweep runs the CUDA kernels: no CUDA device found")
@@ -99,14 +139,37 @@ def main() -> int:
     X = synth.activations(args.tokens, args.d, synth.channel_scale(args.d, args.seed, dev), gen)
     R = synth.affine_noisy_reference(X, 128, gen)
     rows = sweep(X, R, None, default_grid(args.d))
-    rows.sort(key=lambda r: (r["record_bytes"], r["rel_rms_error"]))
+    if args.segment > 0:
+        # the reference of these members carries ONE affine map per (segment, group): what a shared pair can undo
+        bounds = list(range(0, args.tokens, args.segment)) + [args.tokens]
+        seg_off = torch.tensor(bounds, dtype=torch.int32, device=dev)
+        a = torch.rand((len(bounds) - 1, args.d // 128, 1), generator=gen, device=dev) * 0.4 + 0.8
+        b = torch.randn((len(bounds) - 1, args.d // 128, 1), generator=gen, device=dev) * 0.1
+        seg = torch.repeat_interleave(torch.arange(len(bounds) - 1, device=dev),
+                                      torch.diff(seg_off.long()))
+        Rs = torch.empty_like(X)
+        for t0 in range(0, args.tokens, 4096):
+            t1 = min(args.tokens, t0 + 4096)
+            x = X[t0:t1].float().view(t1 - t0, args.d // 128, 128)
+            z = torch.randn(x.shape, generator=gen, device=dev) * 0.05
+            Rs[t0:t1] = ((x - b[seg[t0:t1]]) / a[seg[t0:t1]] + z).view(t1 - t0, args.d).to(torch.bfloat16)
+        more = sweep(X, Rs, None, shared_grid(args.d) + [rac.CodecCfg(args.d, 128, 4, 8), rac.CodecCfg(args.d, 128, 4, 0, scale_mode=1)],
+                     seg_off=seg_off)
+        for r in more:
+            r["segmented"] = True
+        rows += more
+    rows.sort(key=lambda r: (r["record_bytes"] + r["shared_bytes_per_token"], r["rel_rms_error"]))
     print(f"synthetic prefill uplink, {args.tokens} x {args.d}; reference = noisy affine image per (token, 128 channels)")
-    print(f"{'mode':>7} {'g_a':>4} {'g_q':>5} {'b':>2} {'k':>3} {'k_g':>3} {'bytes':>6} {'/raw':>6} {'rel rms':>9} {'max abs':>8} {'ms':>7}")
+    if args.segment > 0:
+        print(f"members marked 'seg': reference with one affine map per ({args.segment} tokens, 128 channels); 'shared' = one "
+              "coefficient pair per segment and group, outside the records")
+    print(f"{'mode':>7} {'coef':>7} {'g_a':>4} {'g_q':>5} {'b':>2} {'k':>3} {'k_g':>3} {'bytes':>8} {'/raw':>6} {'rel rms':>9} {'max abs':>8} {'ms':>7}")
     for r in rows:
         mode = "static" if r["scale_mode"] == 0 else "Eq.8"
-        print(f"{mode:>7} {r['group']:>4} {r['qgroup']:>5} {r['bits']:>2} {r['topk']:>3} {r['topk_group']:>3} "
-              f"{r['record_bytes']:>6} {r['payload_over_raw']:>6.3f} {r['rel_rms_error']:>9.5f} {r['max_abs_error']:>8.3f} "
-              f"{r['encode_reconstruct_ms']:>7.3f}")
+        coef = "shared" if r["coef_fmt"] == 1 else ("seg" if r.get("segmented") else "token")
+        print(f"{mode:>7} {coef:>7} {r['group']:>4} {r['qgroup']:>5} {r['bits']:>2} {r['topk']:>3} {r['topk_group']:>3} "
+              f"{r['record_bytes'] + r['shared_bytes_per_token']:>8.1f} {r['payload_over_raw']:>6.3f} {r['rel_rms_error']:>9.5f} "
+              f"{r['max_abs_error']:>8.3f} {r['encode_reconstruct_ms']:>7.3f}")
     return 0
 
 
