@@ -99,6 +99,18 @@ def test_host_side_rejections_happen_before_any_launch(rac):
     m = lambda **kw: lib.rac_match_spans(kw.get("h", A), kw.get("nh", 1000), A, 100, kw.get("w", 4), kw.get("K", 8), A, None, A,
                                          kw.get("ws", A), kw.get("wsb", need), 0)
     assert m(w=0) == -4 and m(K=-1) == -4 and m(K=17) == -4 and m(wsb=need - 1) == -3 and m(ws=A + 4) == -2 and m(h=None) == -1
+    # shared coefficient pairs: the record format and the words go together, in the calibration and in the list calls
+    sh = rac.CodecCfg(4096, 128, 4, 8, coef_fmt=1)
+    nbc = rac.rac_calibrate_workspace_bytes(sh)
+    assert nbc == rac.rac_calibrate_workspace_bytes(cfg) > 0
+    cal = lambda c, cs, so, wsb=nbc: lib.rac_calibrate_steps_shared(C.byref(c), A, 16, A, 16, None, None, None, cs, so, 3.0, A, A,
+                                                                  A, wsb, None, 0)
+    assert cal(sh, None, A) == -1 and cal(sh, A, None) == -1 and cal(cfg, A, A) == -1 and cal(sh, A, A, nbc - 1) == -3
+    assert lib.rac_calibrate_steps(C.byref(sh), A, 16, A, 16, None, None, None, 3.0, A, A, A, nbc, None, 0) == -1
+    assert cal(rac.CodecCfg(4096, 128, 4, 0, scale_mode=1, coef_fmt=1), A, A) == -4      # no table in that mode
+    lst = lambda c, cs, so: lib.rac_encode_reconstruct_list(C.byref(c), A, 16, None, None, A, 16, None, None, 0, cs, so, None,
+                                                            None, A, A, A, 16 * 4096, None, A, 16 * 128 * 4, None, 0)
+    assert lst(sh, None, None) == -1 and lst(cfg, A, A) == -1 and lst(sh, A, None) == -1
     assert rac.rac_strerror(-3) == "caller buffer too small"
     with pytest.raises(rac.RacError):
         rac._check("x", -1)
