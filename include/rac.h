@@ -79,7 +79,8 @@ extern "C" {
  *                  not read and may be NULL
  *   flags   must be 0
  *   qgroup  g_q, channels per quantisation group (scale_mode 1): 0 = same as `group`; a power of two 32..1024
- *           that divides d; or d itself (the paper's decode mode: one scale per token)
+ *           that divides d; d itself (the paper's decode mode: one scale per token); or any other multiple of 32
+ *           that divides d (without outliers)
  *   topk_group  k_g, outliers per quantisation group (Sec. IV-C "Outlier Metadata"), 0..8, scale_mode 1 with a
  *           power-of-two qgroup (not with qgroup = d unless d is such a value): the k_g largest |e| of every
  *           group (ties to the lower channel) leave the dense base before its scale is taken; in-group offsets in

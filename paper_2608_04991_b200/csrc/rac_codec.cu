@@ -42,7 +42,7 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     if (!is_pow2(cfg->group) || cfg->group < 32 || cfg->group > 1024) return RAC_EUNSUPPORTED;
     if (cfg->topk > 16 || cfg->topk > cfg->d) return RAC_EUNSUPPORTED;
     int qgroup = cfg->qgroup ? cfg->qgroup : cfg->group;
-    int lpq = 0;
+    int lpq = 0, qgen = 0;
     if (cfg->scale_mode == 0) {
         // the static table: one grouping, per-token outliers, 2..4 bits
         if (qgroup != cfg->group || cfg->topk_group != 0) return RAC_EUNSUPPORTED;
@@ -57,6 +57,7 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
         if (cfg->d % qgroup) return RAC_EINVAL;
         if (is_pow2(qgroup) && qgroup >= 32 && qgroup <= 1024) lpq = qgroup / 32;
         else if (qgroup == cfg->d) lpq = 0;   // one scale per token, exchanged through shared memory
+        else if (qgroup % 32 == 0) { lpq = 0; qgen = qgroup / 32; }   // any other whole number of lanes: the same exchange
         else return RAC_EUNSUPPORTED;
         if (cfg->topk_group > 8) return RAC_EUNSUPPORTED;
         if (cfg->topk_group > 0 && lpq == 0) return RAC_EUNSUPPORTED;   // a group must lie within one warp
@@ -73,6 +74,7 @@ int make_geometry(const rac_codec_cfg *cfg, Geometry *g) {
     g->qgroup = qgroup;
     g->Jq = cfg->d / qgroup;
     g->lpq = lpq;
+    g->qgen = qgen;
     g->topk_group = cfg->topk_group;
     g->coef_fmt = cfg->coef_fmt;
     g->scale_off = cfg->coef_fmt == 1 ? 0 : 4 * g->J;
@@ -1390,6 +1392,7 @@ static int fill_common(const Geometry &g, CodecParams *p, long long T, const voi
     p->inv_group = 1.0f / (float)g.group;
     p->Jq = g.Jq;
     p->lpq = g.lpq;
+    p->qgen = g.qgen;
     p->lpq_shift = 0;
     while ((1 << p->lpq_shift) < g.lpq) p->lpq_shift++;
     p->kg = g.topk_group;

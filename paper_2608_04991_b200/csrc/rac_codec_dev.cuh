@@ -47,6 +47,7 @@ struct CodecParams {
     float4 *moments;             // segment fit, first pass out: (mean r, mean h, Sxx, Sxy) per (token, group)
     // scale_mode 1 only: quantisation groups, per-group outliers, field offsets in the record
     int Jq, lpq, lpq_shift, kg, scale_off, codes_off, goff_off, gval_off;
+    int qgen;   // lanes per quantisation group that is neither a power of two nor the token (lpq == 0 then), else 0
     // only from rac_selftest_bounded_wait: bytes announced on top of what the copies of a stage deliver, so that the
     // (bounded) wait for them cannot complete
     uint32_t test_extra_tx;

@@ -138,7 +138,8 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
     const u64 magic2 = pack2(kMagic, kMagic);
     const int qbase = lane & ~(p.lpq - 1);              // first lane of this lane's quantisation group (lpq > 0)
     const uint32_t qlanes = p.lpq >= 32 ? 0xffffffffu : ((1u << p.lpq) - 1u);
-    const int jq = qtok ? 0 : (tid >> p.lpq_shift);     // quantisation group of this thread
+    // quantisation group of this thread (qgen: groups of any whole number of lanes, which may cross warps)
+    const int jq = qtok ? (p.qgen ? tid / p.qgen : 0) : (tid >> p.lpq_shift);
 
     int stage = 0, duty = 0;
     uint32_t parity = 0;
@@ -296,7 +297,21 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                     if (p.lpq > o) m = fmaxf(m, __shfl_xor_sync(group_mask, m, o));
             }
         }
-        if (qtok) {
+        if (qtok && p.qgen) {
+            // groups of any whole number of lanes: every thread leaves its maximum in the first word of its own slab of
+            // the reference row (read long ago, not needed again), the warps meet once, and every thread takes the
+            // largest of its group's entries
+            float *mine = reinterpret_cast<float *>(stg + row_bytes + 64 * tid);
+            if (valid) *mine = m;
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&ctrl->tokmax[stage])) : "memory");
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->tokmax[stage]), parity))) { timed_out = true; break; }
+            if (valid) {
+                const int l0 = jq * p.qgen;
+                for (int l = 0; l < p.qgen; l++)
+                    m = fmaxf(m, *reinterpret_cast<volatile float *>(stg + row_bytes + 64 * (l0 + l)));
+            }
+        } else if (qtok) {
             // one scale per token: the warps meet once
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -316,7 +331,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             const float sc = half_bits_to_float(s16);
             const float isc = sc != 0.f ? __fdiv_rn(1.0f, sc) : 0.f;   // zero marker: no division, codes 0
             const u64 inv2 = pack2(isc, isc), s2 = pack2(sc, sc);
-            if (qtok ? tid == 0 : (lane & (p.lpq - 1)) == 0)
+            if (qtok ? tid == jq * p.qgen : (lane & (p.lpq - 1)) == 0)
                 reinterpret_cast<unsigned short *>(rec + p.scale_off)[jq] = (unsigned short)s16;
 
             // No dense value can leave [-Qmax, Qmax] (Eq. 11): s >= max|E^d| / Qmax by the round-up, and the two
@@ -483,7 +498,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
     constexpr uint32_t highs = ones << (BITS - 1);
     constexpr float kBase = 8388608.0f + (float)H;  // 2^23 + H
     const uint32_t row_bytes = 2u * (uint32_t)d;
-    const int jq = p.lpq == 0 ? 0 : (tid >> p.lpq_shift);
+    const int jq = p.lpq == 0 ? (p.qgen ? tid / p.qgen : 0) : (tid >> p.lpq_shift);
 
     if (tid == 0) {
         for (int s = 0; s < S; s++) mbar_init(smem_u32(&ctrl->bar[s]), 1);

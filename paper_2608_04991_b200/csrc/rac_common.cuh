@@ -146,6 +146,7 @@ struct Geometry {
     int qgroup;     // channels per quantisation group (scale_mode 1; == group in mode 0)
     int Jq;         // quantisation groups per token
     int lpq;        // lanes per quantisation group, 0 when the group is the whole token and d/32 is no power of two <= 32
+    int qgen;       // lanes per quantisation group when that is neither a power of two nor the token (then lpq == 0), else 0
     int topk_group; // outliers per quantisation group (scale_mode 1)
     int coef_fmt;   // 0: coefficient words in the record; 1: shared per segment, outside the record (scale_mode 1)
     int scale_off;  // byte offset of the scales in a record: 4*J, or 0 when the record holds no coefficients

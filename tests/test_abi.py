@@ -45,7 +45,7 @@ def test_record_geometry_matches_the_wire_format(rac, orc):
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 4, 0, scale_mode=1)) == 2176 + 64
     # the quantiser family: geometry agrees with the oracle's, 8-bit and per-group outliers only with record scales
     for d, g, b, qg, kg in [(4096, 128, 8, 0, 0), (4096, 128, 4, 0, 2), (3584, 128, 4, 3584, 0), (2080, 32, 4, 0, 1),
-                            (5120, 128, 2, 256, 3), (96, 32, 8, 96, 0)]:
+                            (5120, 128, 2, 256, 3), (96, 32, 8, 96, 0), (5120, 128, 4, 160, 0), (3584, 64, 3, 1792, 0)]:
         assert rac.rac_record_bytes(rac.CodecCfg(d, g, b, 0, scale_mode=1, qgroup=qg, topk_group=kg)) == \
             orc.record_bytes(d, g, b, 0, 1, qg, kg)
     assert rac.rac_record_bytes(rac.CodecCfg(4096, 128, 8, 0)) == 0

@@ -491,6 +491,11 @@ def test_dynamic_group_scale_identity_and_rejections(env):
     (5120, 128, 8, 1024, 8, 25),    # groups of a whole warp
     (1024, 128, 4, 1024, 2, 30),    # g_q = d inside one warp, with outliers
     (2048, 64, 3, 512, 5, 33),
+    (5120, 128, 4, 160, 0, 40),     # groups of five lanes: neither a power of two nor the token, crossing warps
+    (5120, 128, 8, 640, 0, 25),
+    (3584, 128, 4, 224, 0, 33),     # seven lanes
+    (3584, 64, 3, 1792, 0, 21),     # 56 lanes: half a token
+    (96, 32, 2, 96, 0, 9),
 ])
 def test_family_matches_oracle(env, d, g, bits, qg, kg, T):
     X, R, _, _ = prefill_inputs(env, T, d, g, seed=3000 + d + bits + qg + kg)
@@ -540,7 +545,9 @@ def test_family_ties_zero_groups_and_bad_offsets(env):
                     env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, topk_group=9),
                     env.rac.CodecCfg(d, g, 8, 0),                                           # 8 bits: Eq. 8 family only
                     env.rac.CodecCfg(d, g, 4, 0, qgroup=64),                                # static table: g_q = g_a
-                    env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=96),
+                    env.rac.CodecCfg(d, g, 4, 0, scale_mode=1, qgroup=96),                  # does not divide d = 1024
+                    env.rac.CodecCfg(5120, g, 4, 0, scale_mode=1, qgroup=160, topk_group=1),  # outliers need groups inside a warp
+                    env.rac.CodecCfg(5120, g, 4, 0, scale_mode=1, qgroup=80),
                     env.rac.CodecCfg(d, g, 5, 0, scale_mode=1)]:
         assert env.rac.rac_record_bytes(bad_cfg) == 0
 
@@ -690,7 +697,7 @@ def test_random_configurations_on_stressed_inputs(env):
         T = int(rng.integers(1, 400 if d <= 2080 else 120))
         if fam:
             cfg = rac.CodecCfg(d, g, int(rng.choice([2, 3, 4, 8])), 0, scale_mode=1,
-                               qgroup=int(rng.choice([0, 32, 64, 128, 256, 512, 1024, d])), topk_group=int(rng.choice([0, 0, 1, 2, 3, 4, 7, 8])))
+                               qgroup=int(rng.choice([0, 32, 64, 128, 256, 512, 1024, d, 96, 160, 224])), topk_group=int(rng.choice([0, 0, 1, 2, 3, 4, 7, 8])))
             if rac.rac_record_bytes(cfg) == 0:
                 continue
         else:
