@@ -33,8 +33,8 @@
  *                          bit n%8 of byte n/8; two's complement; -2^(bits-1) is never produced
  *     out_idx topk x u16   channel indices, ascending
  *     out_val topk x u16   binary16 residuals of those channels (their dense code is 0)
- *     grp_off Jq*topk_group x u8   in-group offsets of the per-group outliers, ascending within a group,
- *                          padded to a multiple of 2 bytes (scale_mode 1 only)
+ *     grp_off Jq*topk_group x u8   in-group offsets of the per-group outliers, ascending within a group (u16 each
+ *                          when a group has more than 256 channels), padded to a multiple of 2 bytes (scale_mode 1 only)
  *     grp_val Jq*topk_group x u16  binary16 residuals of those channels (their dense code is 0)
  *     zero padding to a multiple of 16 bytes
  * rac_record_bytes() gives the stride.  A token range is a contiguous byte range.
