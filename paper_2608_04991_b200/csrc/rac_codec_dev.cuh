@@ -199,6 +199,20 @@ __device__ __forceinline__ void load_ref_slot(uint32_t addr, const uint16_t *gai
     }
 }
 
+// the same for one pair of channels (c even), operation for operation
+__device__ __forceinline__ u64 load_ref_pair(uint32_t addr, const uint16_t *gain, const uint16_t *bias, int c) {
+    const uint32_t w = lds32(addr);
+    if (gain) {
+        const uint32_t gw = __ldg(reinterpret_cast<const uint32_t *>(gain + c));
+        const uint32_t bw = __ldg(reinterpret_cast<const uint32_t *>(bias + c));
+        const float g0 = half_bits_to_float(gw & 0xffff), g1 = half_bits_to_float(gw >> 16);
+        const float b0 = half_bits_to_float(bw & 0xffff), b1 = half_bits_to_float(bw >> 16);
+        const float r0 = __uint_as_float(w << 16), r1 = __uint_as_float(w & 0xffff0000u);
+        return pack2(bf16_round(__fmaf_rn(g0, r0, b0)), bf16_round(__fmaf_rn(g1, r1, b1)));
+    }
+    return bf16x2_to_p(w);
+}
+
 // SUB = false compiles the plain form (all T tokens in order, one reference buffer); SUB = true the form of the
 // *_list entry points.  how many tokens this launch codes, and the idx-th of them:
 template <bool SUB>

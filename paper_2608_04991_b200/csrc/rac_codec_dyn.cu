@@ -208,67 +208,121 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             }
 
             // ---- outlier mask: k_g rounds of (largest |e| of the group, lowest channel among equals).  The
-            // registers are left alone.  Every lane first finds ITS candidate -- the lowest channel that holds the
-            // lane's own maximum -- by reading that piece of the rows in shared memory again (same operations, same
-            // bits); none of this depends on the other lanes, so it overlaps the group's shuffles.  A round is then
-            // the group maximum, one ballot for the lowest lane that holds it, and that lane handing out its
-            // candidate; only the winner looks for a new candidate, and only if another round follows.  Codes and
-            // x_hat of the outliers are patched after the dense pass.
+            // registers are left alone: what a round needs again is read from the rows in shared memory and formed by
+            // the same operations (same bits).  Codes and x_hat of the outliers are patched after the dense pass.
+            // Groups of four lanes and more that share one coefficient pair (the usual case) work on a round together:
+            // group maximum by shuffles, one ballot for the lowest lane that holds it, that lane names its lowest piece
+            // (8 channels) with that maximum and what was taken from it before; four lanes of the group then form one
+            // pair of that piece's residuals each, two ballots give the lowest channel that equals the maximum and was
+            // not taken, its value comes from the lane that formed it, and the largest of the rest is the piece's new
+            // maximum.  Nothing diverges.  Smaller groups (or quantisation groups that span alignment groups) keep the
+            // older form: every lane finds ITS candidate beforehand (off the critical path), a round is the group
+            // maximum, one ballot, the winner handing out its candidate and looking for its next one.
             if (KG) {
                 uint32_t taken = 0;  // channel order within the slab
-                float mloc, cval, cnm;
-                int cq, ck;
-                auto find = [&]() {
-                    mloc = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
-                    // lowest piece whose maximum is the lane's maximum; piece q sits in slot (q - rot) & 3
-                    float sp[4] = {sm[0], sm[1], sm[2], sm[3]};
-                    rot_right4f(sp, rot);
-                    const int q = sp[0] == mloc ? 0 : sp[1] == mloc ? 1 : sp[2] == mloc ? 2 : 3;
-                    const uint32_t pa = (uint32_t)(tid * 64 + q * 16);
-                    const uint4 xw = lds128(xs + pa);
-                    const uint32_t xws[4] = {xw.x, xw.y, xw.z, xw.w};
-                    u64 rr[4] = {0ull, 0ull, 0ull, 0ull};
-                    if (has_ref) load_ref_slot(rs + pa, p.gain, p.bias, (int)(pa >> 1), rr);
-                    float ev[8];
+                if (p.lpq >= 4 && p.lpg >= p.lpq) {
+                    const int pi = (lane - qbase) & 3;   // this lane's pair of the piece; with more than four lanes the upper ones repeat the lower four
 #pragma unroll
-                    for (int i = 0; i < 4; i++) unpack2(psub(bf16x2_to_p(xws[i]), pfma(a2, rr[i], b2)), ev[2 * i], ev[2 * i + 1]);
-                    uint32_t tq = (taken >> (8 * q)) & 0xffu;
-                    uint32_t eq = 0;
+                    for (int n = 0; n < KG; n++) {
+                        if (KG <= 2 || n < p.kg) {
+                            const float mloc = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
+                            float sp[4] = {sm[0], sm[1], sm[2], sm[3]};
+                            rot_right4f(sp, rot);
+                            const int q = sp[0] == mloc ? 0 : sp[1] == mloc ? 1 : sp[2] == mloc ? 2 : 3;
+                            float gm = mloc;
 #pragma unroll
-                    for (int k = 0; k < 8; k++) eq |= (fabsf(ev[k]) == mloc) ? (1u << k) : 0u;
-                    eq &= ~tq;
-                    const int k = eq ? __ffs(eq) - 1 : 0;   // eq == 0 only with NaNs around
-                    float val = ev[0];
+                            for (int o = 1; o < 32; o <<= 1)
+                                if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
+                            const uint32_t gb = (__ballot_sync(group_mask, mloc == gm) >> qbase) & qlanes;
+                            const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);
+                            const uint32_t info = __shfl_sync(group_mask, (uint32_t)(tid * 64 + q * 16) | (((taken >> (8 * q)) & 0xffu) << 20), owner);
+                            const uint32_t wpa = info & 0xfffffu, wtq = info >> 20;
+                            const uint32_t ad = wpa + 4u * (uint32_t)pi;
+                            u64 rr = 0ull;
+                            if (has_ref) rr = load_ref_pair(rs + ad, p.gain, p.bias, (int)(ad >> 1));
+                            float e0, e1;
+                            unpack2(psub(bf16x2_to_p(lds32(xs + ad)), pfma(a2, rr, b2)), e0, e1);
+                            const uint32_t mybits = (((fabsf(e0) == gm ? 1u : 0u) | (fabsf(e1) == gm ? 2u : 0u)) << (2 * pi)) & ~wtq;
+                            // the four lanes that hold the piece sit at qbase..qbase+3 of the group
+                            const uint32_t b0 = __ballot_sync(group_mask, mybits & (1u << (2 * pi)));
+                            const uint32_t b1 = __ballot_sync(group_mask, mybits & (2u << (2 * pi)));
+                            const uint32_t g0 = (b0 >> qbase) & 0xfu, g1 = (b1 >> qbase) & 0xfu;
+                            // channel 2*l is bit l of g0, channel 2*l+1 bit l of g1: the lowest channel that is set
+                            const int k0 = g0 ? 2 * (__ffs(g0) - 1) : 8, k1 = g1 ? 2 * (__ffs(g1) - 1) + 1 : 8;
+                            const int k = min(k0, k1) & 7;   // 8 (nothing set: only with NaNs around) -> 0
+                            const int kp = k >> 1;
+                            const uint32_t gone = (wtq | (1u << k)) >> (2 * pi);
+                            const float mine = (k & 1) ? e1 : e0;
+                            float rest = fmaxf((gone & 1u) ? 0.f : fabsf(e0), (gone & 2u) ? 0.f : fabsf(e1));
+                            const float val = __shfl_sync(group_mask, mine, qbase + kp);
+                            rest = fmaxf(rest, __shfl_xor_sync(group_mask, rest, 1));
+                            rest = fmaxf(rest, __shfl_xor_sync(group_mask, rest, 2));
+                            const int wq = (int)(wpa >> 4) & 3;
+                            sel[n] = (uint32_t)((owner - qbase) * 32 + 8 * wq + k) | (float_to_half_bits_sat(val) << 16);
+                            if (lane == owner) {
+                                own |= 1u << n;
+                                taken |= 1u << (8 * wq + k);
+                                const int js = (wq - rot) & 3;
 #pragma unroll
-                    for (int kk = 1; kk < 8; kk++) val = (kk == k) ? ev[kk] : val;
-                    cnm = abs_max8(ev, tq | (1u << k));     // E^d = E - O for this slot's maximum
-                    cq = q;
-                    ck = k;
-                    cval = val;
-                };
-                find();
-#pragma unroll
-                for (int n = 0; n < KG; n++) {
-                    if (KG <= 2 || n < p.kg) {   // the launcher compiles in exactly k_g rounds for k_g = 1, 2
-                        float gm = mloc;
-#pragma unroll
-                        for (int o = 1; o < 32; o <<= 1)
-                            if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
-                        const uint32_t gb = (__ballot_sync(group_mask, mloc == gm) >> qbase) & qlanes;
-                        const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);   // gb == 0 only with NaNs around
-                        uint32_t word = 0;
-                        if (lane == owner) {
-                            word = (uint32_t)((lane - qbase) * 32 + 8 * cq + ck) | (float_to_half_bits_sat(cval) << 16);
-                            own |= 1u << n;
-                            taken |= 1u << (8 * cq + ck);
-                            const int js = (cq - rot) & 3;
-#pragma unroll
-                            for (int j = 0; j < 4; j++) sm[j] = (j == js) ? cnm : sm[j];
-                            if (KG <= 2 ? n + 1 < KG : n + 1 < p.kg) find();
+                                for (int j = 0; j < 4; j++) sm[j] = (j == js) ? rest : sm[j];
+                            }
                         }
-                        sel[n] = __shfl_sync(group_mask, word, owner);
                     }
-                }
+                } else {
+                    float mloc, cval, cnm;
+                    int cq, ck;
+                    auto find = [&]() {
+                        mloc = fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
+                        // lowest piece whose maximum is the lane's maximum; piece q sits in slot (q - rot) & 3
+                        float sp[4] = {sm[0], sm[1], sm[2], sm[3]};
+                        rot_right4f(sp, rot);
+                        const int q = sp[0] == mloc ? 0 : sp[1] == mloc ? 1 : sp[2] == mloc ? 2 : 3;
+                        const uint32_t pa = (uint32_t)(tid * 64 + q * 16);
+                        const uint4 xw = lds128(xs + pa);
+                        const uint32_t xws[4] = {xw.x, xw.y, xw.z, xw.w};
+                        u64 rr[4] = {0ull, 0ull, 0ull, 0ull};
+                        if (has_ref) load_ref_slot(rs + pa, p.gain, p.bias, (int)(pa >> 1), rr);
+                        float ev[8];
+#pragma unroll
+                        for (int i = 0; i < 4; i++) unpack2(psub(bf16x2_to_p(xws[i]), pfma(a2, rr[i], b2)), ev[2 * i], ev[2 * i + 1]);
+                        uint32_t tq = (taken >> (8 * q)) & 0xffu;
+                        uint32_t eq = 0;
+#pragma unroll
+                        for (int k = 0; k < 8; k++) eq |= (fabsf(ev[k]) == mloc) ? (1u << k) : 0u;
+                        eq &= ~tq;
+                        const int k = eq ? __ffs(eq) - 1 : 0;   // eq == 0 only with NaNs around
+                        float val = ev[0];
+#pragma unroll
+                        for (int kk = 1; kk < 8; kk++) val = (kk == k) ? ev[kk] : val;
+                        cnm = abs_max8(ev, tq | (1u << k));     // E^d = E - O for this slot's maximum
+                        cq = q;
+                        ck = k;
+                        cval = val;
+                    };
+                    find();
+#pragma unroll
+                    for (int n = 0; n < KG; n++) {
+                        if (KG <= 2 || n < p.kg) {   // the launcher compiles in exactly k_g rounds for k_g = 1, 2
+                            float gm = mloc;
+#pragma unroll
+                            for (int o = 1; o < 32; o <<= 1)
+                                if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
+                            const uint32_t gb = (__ballot_sync(group_mask, mloc == gm) >> qbase) & qlanes;
+                            const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);   // gb == 0 only with NaNs around
+                            uint32_t word = 0;
+                            if (lane == owner) {
+                                word = (uint32_t)((lane - qbase) * 32 + 8 * cq + ck) | (float_to_half_bits_sat(cval) << 16);
+                                own |= 1u << n;
+                                taken |= 1u << (8 * cq + ck);
+                                const int js = (cq - rot) & 3;
+#pragma unroll
+                                for (int j = 0; j < 4; j++) sm[j] = (j == js) ? cnm : sm[j];
+                                if (KG <= 2 ? n + 1 < KG : n + 1 < p.kg) find();
+                            }
+                            sel[n] = __shfl_sync(group_mask, word, owner);
+                        }
+                    }
+}
                 if ((lane & (p.lpq - 1)) == 0) {
                     // the group's first lane serialises them in ascending offset order
                     const bool wide = p.lpq > 8;   // more than 256 channels per group: two-byte offsets
