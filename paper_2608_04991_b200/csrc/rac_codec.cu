@@ -295,14 +295,20 @@ template <int BITS, bool TOPK, bool XHAT, int MINB, bool SUB, int LPG = 0, int D
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
-    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = D ? (D / 32 + 31) / 32 : nt >> 5;
     const int rot = (lane >> 1) & 3;
     const int d = D ? D : p.d;
     const bool valid = tid * 32 < d;
-    const WsSmem L = ws_smem_layout(d, p.rec, p.stages, TOPK);
+    constexpr int S = 2;   // stages of the ring (the host sets p.stages to the same)
+    // with the width and the group compiled in, the record geometry is a constant too (those variants are launched for
+    // no outliers or eight per token only)
+    constexpr bool kGeo = D != 0 && LPG != 0;
+    const int Jc = kGeo ? D / (32 * (LPG ? LPG : 1)) : p.J;
+    const int codeb = kGeo ? D * BITS / 8 : p.code_bytes;
+    const int recb = kGeo ? (4 * (D / (32 * (LPG ? LPG : 1))) + D * BITS / 8 + (TOPK ? 32 : 0) + 15) / 16 * 16 : p.rec;
+    const WsSmem L = ws_smem_layout(d, recb, S, TOPK);
     WsCtrl *ctrl = reinterpret_cast<WsCtrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
-    const int S = p.stages;
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     const uint32_t row_bytes = 2u * (uint32_t)d;
 
@@ -338,13 +344,13 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
     // records: no coefficient words in front of the codes
     bool shared = false;
     if constexpr (SUB) shared = p.coef_ext != nullptr;
-    const int coff = shared ? 0 : 4 * p.J;
+    const int coff = shared ? 0 : 4 * Jc;
     {
         // padding words of the records are written once and never touched again
-        const int raw = coff + p.code_bytes + 4 * p.topk;
+        const int raw = coff + codeb + 4 * p.topk;
         for (int s = 0; s < 2 * S; s++)
-            for (int o = raw + 4 * tid; o < p.rec; o += 4 * nt)
-                *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * p.rec + o) = 0u;
+            for (int o = raw + 4 * tid; o < recb; o += 4 * nt)
+                *reinterpret_cast<uint32_t *>(smem + L.stage0 + (s >> 1) * L.stage_bytes + L.rec_off + (s & 1) * recb + o) = 0u;
     }
     __syncthreads();
     if (tid == 0)
@@ -364,7 +370,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         unsigned char *stg = smem + L.stage0 + stage * L.stage_bytes;
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
-        unsigned char *rec = stg + L.rec_off + parity * p.rec;
+        unsigned char *rec = stg + L.rec_off + parity * recb;
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
@@ -396,7 +402,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
             constexpr int kShift = LPG == 4 ? 2 : 1;
             const int lpg = LPG ? LPG : p.lpg, lpg_shift = LPG ? kShift : p.lpg_shift;
             if (shared) {
-                const uint32_t cw = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> lpg_shift)];
+                const uint32_t cw = p.coef_ext[(long long)ctrl->seg[stage] * Jc + (tid >> lpg_shift)];
                 const float a = half_bits_to_float(cw & 0xffffu), b = half_bits_to_float(cw >> 16);
                 a2 = pack2(a, a);
                 b2 = pack2(b, b);
@@ -519,14 +525,14 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
                 if (TOPK)  // the slab maxima travel like the record: one bulk copy from this parity's slot
                     bulk_store(p.tmax + t * (L.tm_bytes >> 2), xs + L.tm_off + parity * L.tm_bytes, (uint32_t)L.tm_bytes);
                 if (XHAT) {
-                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_store(p.payload + t * recb, smem_u32(rec), (uint32_t)recb);
                     bulk_store(p.X_hat + t * d, xs, row_bytes);
                     bulk_commit();
                     bulk_wait_read<0>();
                     if (k_next < n_my) issue(k_next, stage, raw_next);
                 } else {
                     if (k_next < n_my) issue(k_next, stage, raw_next);
-                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_store(p.payload + t * recb, smem_u32(rec), (uint32_t)recb);
                     bulk_commit();
                     bulk_wait_read<0>();
                 }
@@ -1435,10 +1441,13 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     const bool tight = g.nthreads > 96 && g.nthreads <= 160 && !p.X_hat;
     int rc = RAC_EUNSUPPORTED;
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;   // the subset form has one variant per width: it is not the hot path
+    // widths 4096 and 5120 with no or eight outliers per token run variants with the whole record geometry compiled in
+    const bool geo = (g.d == 5120 || g.d == 4096) && (g.topk == 0 || g.topk == 8);
 #define RAC_ENC4(B, K, X, G, W)                                                                                        \
     (tight ? launch_persistent(encode_ws_kernel<B, K, X, 4, false, G, W>, p, g.nthreads, L.total, max_ctas, stream) \
            : launch_persistent(encode_ws_kernel<B, K, X, 2, false, G, W>, p, g.nthreads, L.total, max_ctas, stream))
-#define RAC_ENC3(B, K, X, G) (g.d == 5120 ? RAC_ENC4(B, K, X, G, 5120) : g.d == 4096 ? RAC_ENC4(B, K, X, G, 4096) : RAC_ENC4(B, K, X, G, 0))
+#define RAC_ENC3(B, K, X, G)                                                        \
+    (!geo ? RAC_ENC4(B, K, X, G, 0) : g.d == 5120 ? RAC_ENC4(B, K, X, G, 5120) : RAC_ENC4(B, K, X, G, 4096))
 #define RAC_ENC2(B, K, X)                                                                                           \
     (sub ? launch_persistent(encode_ws_kernel<B, K, X, 2, true, 0>, p, g.nthreads, L.total, max_ctas, stream)      \
      : g.lpg == 4 ? RAC_ENC3(B, K, X, 4) : g.lpg == 2 ? RAC_ENC3(B, K, X, 2) : RAC_ENC4(B, K, X, 0, 0))
