@@ -78,19 +78,25 @@ __device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, 
 
 // MINB = 4 caps registers at 96 so that four 160-thread CTAs (d = 5120) fit on an SM.
 // KG: rounds compiled in (0, 1, 2, 4 or 8; p.kg <= KG is the number taken).
-template <int BITS, bool XHAT, int KG, int MINB, bool SUB>
+// G, D: lanes per group (alignment and quantisation group alike) and the hidden width as compile-time constants, or 0
+// to read them from the parameters; with them the reductions lose their uniform branches and the address arithmetic
+// of rows and stages folds.
+template <int BITS, bool XHAT, int KG, int MINB, bool SUB, int G = 0, int D = 0>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
-    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = D ? (D / 32 + 31) / 32 : nt >> 5;
     const int rot = (lane >> 1) & 3;
-    const int d = p.d;
+    const int d = D ? D : p.d;
+    constexpr int kGShift = G == 32 ? 5 : G == 16 ? 4 : G == 8 ? 3 : G == 4 ? 2 : G == 2 ? 1 : 0;
+    const int lpg = G ? G : p.lpg, lpg_shift = G ? kGShift : p.lpg_shift;
+    const int lpq = G ? G : p.lpq, lpq_shift = G ? kGShift : p.lpq_shift;
     const bool valid = tid * 32 < d;
-    const bool qtok = p.lpq == 0;
-    const DynSmem L = dyn_smem_layout(d, p.rec, p.stages);
+    const bool qtok = lpq == 0;
+    const int S = D ? 2 : p.stages;   // the host sets two stages
+    const DynSmem L = dyn_smem_layout(d, p.rec, S);
     DynCtrl *ctrl = reinterpret_cast<DynCtrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
-    const int S = p.stages;
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     constexpr int WPT = BITS;  // code words per thread (32 channels)
     const uint32_t row_bytes = 2u * (uint32_t)d;
@@ -136,10 +142,10 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
     for (int j = 0; j < 4; j++) off[j] = (uint32_t)(tid * 64 + ((j + rot) & 3) * 16);
     const unsigned int group_mask = __ballot_sync(0xffffffffu, valid);
     const u64 magic2 = pack2(kMagic, kMagic);
-    const int qbase = lane & ~(p.lpq - 1);              // first lane of this lane's quantisation group (lpq > 0)
-    const uint32_t qlanes = p.lpq >= 32 ? 0xffffffffu : ((1u << p.lpq) - 1u);
+    const int qbase = lane & ~(lpq - 1);              // first lane of this lane's quantisation group (lpq > 0)
+    const uint32_t qlanes = lpq >= 32 ? 0xffffffffu : ((1u << lpq) - 1u);
     // quantisation group of this thread (qgen: groups of any whole number of lanes, which may cross warps)
-    const int jq = qtok ? (p.qgen ? tid / p.qgen : 0) : (tid >> p.lpq_shift);
+    const int jq = qtok ? (p.qgen ? tid / p.qgen : 0) : (tid >> lpq_shift);
 
     int stage = 0, duty = 0;
     uint32_t parity = 0;
@@ -185,14 +191,14 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             if constexpr (SUB) shared = p.coef_ext != nullptr;
             if (shared) {
                 // Eq. 6 was solved over all positions of the token's segment beforehand: the words come from outside
-                const uint32_t cw = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> p.lpg_shift)];
+                const uint32_t cw = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> lpg_shift)];
                 const float a = half_bits_to_float(cw & 0xffffu), b = half_bits_to_float(cw >> 16);
                 a2 = pack2(a, a);
                 b2 = pack2(b, b);
             } else {
                 uint32_t coef_word;
-                fit_group(x2, r2, has_ref, p.lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
-                if ((lane & (p.lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> p.lpg_shift] = coef_word;
+                fit_group(x2, r2, has_ref, lpg, p.inv_group, group_mask, p.status, a2, b2, &coef_word);
+                if ((lane & (lpg - 1)) == 0) reinterpret_cast<uint32_t *>(rec)[tid >> lpg_shift] = coef_word;
             }
             // residual, and the largest magnitude of each slot of 8 channels
             float sm[4];
@@ -220,7 +226,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             // maximum, one ballot, the winner handing out its candidate and looking for its next one.
             if (KG) {
                 uint32_t taken = 0;  // channel order within the slab
-                if (p.lpq >= 4 && p.lpg >= p.lpq) {
+                if (lpq >= 4 && lpg >= lpq) {
                     const int pi = (lane - qbase) & 3;   // this lane's pair of the piece; with more than four lanes the upper ones repeat the lower four
 #pragma unroll
                     for (int n = 0; n < KG; n++) {
@@ -232,7 +238,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                             float gm = mloc;
 #pragma unroll
                             for (int o = 1; o < 32; o <<= 1)
-                                if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
+                                if (lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
                             const uint32_t gb = (__ballot_sync(group_mask, mloc == gm) >> qbase) & qlanes;
                             const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);
                             const uint32_t info = __shfl_sync(group_mask, (uint32_t)(tid * 64 + q * 16) | (((taken >> (8 * q)) & 0xffu) << 20), owner);
@@ -306,7 +312,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                             float gm = mloc;
 #pragma unroll
                             for (int o = 1; o < 32; o <<= 1)
-                                if (p.lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
+                                if (lpq > o) gm = fmaxf(gm, __shfl_xor_sync(group_mask, gm, o));
                             const uint32_t gb = (__ballot_sync(group_mask, mloc == gm) >> qbase) & qlanes;
                             const int owner = qbase + (gb ? __ffs(gb) - 1 : 0);   // gb == 0 only with NaNs around
                             uint32_t word = 0;
@@ -323,9 +329,9 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                         }
                     }
 }
-                if ((lane & (p.lpq - 1)) == 0) {
+                if ((lane & (lpq - 1)) == 0) {
                     // the group's first lane serialises them in ascending offset order
-                    const bool wide = p.lpq > 8;   // more than 256 channels per group: two-byte offsets
+                    const bool wide = lpq > 8;   // more than 256 channels per group: two-byte offsets
                     unsigned char *go = rec + p.goff_off + jq * p.kg;
                     unsigned short *go2 = reinterpret_cast<unsigned short *>(rec + p.goff_off) + jq * p.kg;
                     unsigned short *gv = reinterpret_cast<unsigned short *>(rec + p.gval_off) + jq * p.kg;
@@ -348,7 +354,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             if (!qtok) {
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1)
-                    if (p.lpq > o) m = fmaxf(m, __shfl_xor_sync(group_mask, m, o));
+                    if (lpq > o) m = fmaxf(m, __shfl_xor_sync(group_mask, m, o));
             }
         }
         if (qtok && p.qgen) {
@@ -385,7 +391,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             const float sc = half_bits_to_float(s16);
             const float isc = sc != 0.f ? __fdiv_rn(1.0f, sc) : 0.f;   // zero marker: no division, codes 0
             const u64 inv2 = pack2(isc, isc), s2 = pack2(sc, sc);
-            if (qtok ? tid == jq * p.qgen : (lane & (p.lpq - 1)) == 0)
+            if (qtok ? tid == jq * p.qgen : (lane & (lpq - 1)) == 0)
                 reinterpret_cast<unsigned short *>(rec + p.scale_off)[jq] = (unsigned short)s16;
 
             // No dense value can leave [-Qmax, Qmax] (Eq. 11): s >= max|E^d| / Qmax by the round-up, and the two
@@ -459,7 +465,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
 #pragma unroll
                 for (int n = 0; n < KG; n++) {
                     if ((own >> n) & 1u) {
-                        const int c = jq * (p.lpq * 32) + (int)(sel[n] & 0xffffu);
+                        const int c = jq * (lpq * 32) + (int)(sel[n] & 0xffffu);
                         const int bp = (c & 31) * BITS, w = bp >> 5, sh = bp & 31;
                         const unsigned long long mk = (unsigned long long)((1u << BITS) - 1u) << sh;
                         cw[w] &= ~(uint32_t)mk;
@@ -731,6 +737,18 @@ template <int B, bool X, int K>
 static int launch_encode_variant(bool tight, const Geometry &g, CodecParams &p, int smem, long long max_ctas, cudaStream_t stream) {
     if (p.tok_list || p.intra_base || p.coef_ext)   // the subset form: one variant, not the hot path
         return launch_persistent(encode_dyn_kernel<B, X, K, 2, true>, p, g.nthreads, smem, max_ctas, stream);
+    // the paper's code widths (4 and 8 bits) at widths 5120 and 4096 with groups of 128 channels (alignment and
+    // quantisation alike) run variants with those compiled in
+    if constexpr (B == 4 || B == 8) {
+        if (g.d == 5120 && g.lpg == 4 && g.lpq == 4) {
+            if constexpr (!X && (K == 0 || B != 8))
+                return launch_persistent(encode_dyn_kernel<B, X, K, 4, false, 4, 5120>, p, g.nthreads, smem, max_ctas, stream);
+            else
+                return launch_persistent(encode_dyn_kernel<B, X, K, 2, false, 4, 5120>, p, g.nthreads, smem, max_ctas, stream);
+        }
+        if (g.d == 4096 && g.lpg == 4 && g.lpq == 4)
+            return launch_persistent(encode_dyn_kernel<B, X, K, 2, false, 4, 4096>, p, g.nthreads, smem, max_ctas, stream);
+    }
     if constexpr (!X && (K == 0 || B != 8)) {
         if (tight) return launch_persistent(encode_dyn_kernel<B, X, K, 4, false>, p, g.nthreads, smem, max_ctas, stream);
     }
