@@ -81,7 +81,8 @@ __device__ __forceinline__ void pack_slot(const uint32_t (&t)[8], uint32_t &w0, 
 // G, D: lanes per group (alignment and quantisation group alike) and the hidden width as compile-time constants, or 0
 // to read them from the parameters; with them the reductions lose their uniform branches and the address arithmetic
 // of rows and stages folds.
-template <int BITS, bool XHAT, int KG, int MINB, bool SUB, int G = 0, int D = 0>
+// QT (with G): the quantisation group is the whole token (one scale per token) instead of the alignment group.
+template <int BITS, bool XHAT, int KG, int MINB, bool SUB, int G = 0, int D = 0, bool QT = false>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
     const int d = D ? D : p.d;
     constexpr int kGShift = G == 32 ? 5 : G == 16 ? 4 : G == 8 ? 3 : G == 4 ? 2 : G == 2 ? 1 : 0;
     const int lpg = G ? G : p.lpg, lpg_shift = G ? kGShift : p.lpg_shift;
-    const int lpq = G ? G : p.lpq, lpq_shift = G ? kGShift : p.lpq_shift;
+    const int lpq = G ? (QT ? 0 : G) : p.lpq, lpq_shift = G ? (QT ? 0 : kGShift) : p.lpq_shift;
     const bool valid = tid * 32 < d;
     const bool qtok = lpq == 0;
     const int S = D ? 2 : p.stages;   // the host sets two stages
@@ -537,18 +538,22 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
 // dequantises its 32 channels (code -> binary32 through the 2^23 trick, times its group's scale), adds the
 // aligned reference, rounds to bf16 into an output row in shared memory; then the per-group outliers replace
 // what the dense pass wrote, and the row leaves as one bulk store.
-template <int BITS, bool KG, bool SUB>
+// G, D: as for the encoder (lanes per group and hidden width compiled in, or 0)
+template <int BITS, bool KG, bool SUB, int G = 0, int D = 0>
 __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int rot = (lane >> 1) & 3;
-    const int d = p.d;
+    const int d = D ? D : p.d;
+    constexpr int kGShift = G == 32 ? 5 : G == 16 ? 4 : G == 8 ? 3 : G == 4 ? 2 : G == 2 ? 1 : 0;
+    const int lpg_shift = G ? kGShift : p.lpg_shift;
+    const int lpq = G ? G : p.lpq, lpq_shift = G ? kGShift : p.lpq_shift;
     const bool valid = tid * 32 < d;
-    const DecSmem L = dec_smem_layout(d, p.rec, p.stages);
+    const int S = D ? 2 : p.stages;   // the host sets two stages
+    const DecSmem L = dec_smem_layout(d, p.rec, S);
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
-    const int S = p.stages;
     constexpr int WPT = BITS;                     // code words per thread
     constexpr int WPP = BITS == 8 ? 2 : 1;        // code words per piece of 8 channels
     constexpr int FPW = 8 / WPP;                  // fields per word
@@ -558,7 +563,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
     constexpr uint32_t highs = ones << (BITS - 1);
     constexpr float kBase = 8388608.0f + (float)H;  // 2^23 + H
     const uint32_t row_bytes = 2u * (uint32_t)d;
-    const int jq = p.lpq == 0 ? (p.qgen ? tid / p.qgen : 0) : (tid >> p.lpq_shift);
+    const int jq = lpq == 0 ? (p.qgen ? tid / p.qgen : 0) : (tid >> lpq_shift);
 
     if (tid == 0) {
         for (int s = 0; s < S; s++) mbar_init(smem_u32(&ctrl->bar[s]), 1);
@@ -613,8 +618,8 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
             uint32_t cf;
             bool shared = false;
             if constexpr (SUB) shared = p.coef_ext != nullptr;
-            if (shared) cf = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> p.lpg_shift)];
-            else cf = reinterpret_cast<const uint32_t *>(rec)[tid >> p.lpg_shift];
+            if (shared) cf = p.coef_ext[(long long)ctrl->seg[stage] * p.J + (tid >> lpg_shift)];
+            else cf = reinterpret_cast<const uint32_t *>(rec)[tid >> lpg_shift];
             const float a = half_bits_to_float(cf & 0xffff), b = half_bits_to_float(cf >> 16);
             const u64 a2 = pack2(a, a), b2 = pack2(b, b);
             const float sc = half_bits_to_float(reinterpret_cast<const unsigned short *>(rec + p.scale_off)[jq]);
@@ -679,11 +684,11 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
             }
             if (KG) {
                 // outliers of this thread's group that fall into its own 32 channels, in record order
-                const bool wide = p.lpq > 8;   // more than 256 channels per group: two-byte offsets
+                const bool wide = lpq > 8;   // more than 256 channels per group: two-byte offsets
                 const unsigned char *go = rec + p.goff_off + jq * p.kg;
                 const unsigned short *go2 = reinterpret_cast<const unsigned short *>(rec + p.goff_off) + jq * p.kg;
                 const unsigned short *gv = reinterpret_cast<const unsigned short *>(rec + p.gval_off) + jq * p.kg;
-                const int qsize = p.lpq * 32;
+                const int qsize = lpq * 32;
                 bool bad = false;
 #pragma unroll
                 for (int n = 0; n < 8; n++) {
@@ -691,7 +696,7 @@ __global__ void __launch_bounds__(256) decode_dyn_kernel(const CodecParams p) {
                         const int o = wide ? (int)go2[n] : (int)go[n];
                         if (o >= qsize) {
                             bad = true;
-                        } else if ((o >> 5) == (tid & (p.lpq - 1))) {
+                        } else if ((o >> 5) == (tid & (lpq - 1))) {
                             const int c = jq * qsize + o;
                             float r = 0.f;
                             if (has_ref) {
@@ -748,6 +753,18 @@ static int launch_encode_variant(bool tight, const Geometry &g, CodecParams &p, 
         }
         if (g.d == 4096 && g.lpg == 4 && g.lpq == 4)
             return launch_persistent(encode_dyn_kernel<B, X, K, 2, false, 4, 4096>, p, g.nthreads, smem, max_ctas, stream);
+        if constexpr (K == 0) {   // the paper's decode mode: one scale per token
+            if (g.lpg == 4 && g.lpq == 0 && g.qgen == 0) {
+                if (g.d == 5120) {
+                    if constexpr (!X)
+                        return launch_persistent(encode_dyn_kernel<B, X, 0, 4, false, 4, 5120, true>, p, g.nthreads, smem, max_ctas, stream);
+                    else
+                        return launch_persistent(encode_dyn_kernel<B, X, 0, 2, false, 4, 5120, true>, p, g.nthreads, smem, max_ctas, stream);
+                }
+                if (g.d == 4096)
+                    return launch_persistent(encode_dyn_kernel<B, X, 0, 2, false, 4, 4096, true>, p, g.nthreads, smem, max_ctas, stream);
+            }
+        }
     }
     if constexpr (!X && (K == 0 || B != 8)) {
         if (tight) return launch_persistent(encode_dyn_kernel<B, X, K, 4, false>, p, g.nthreads, smem, max_ctas, stream);
@@ -790,9 +807,12 @@ int launch_decode_dyn(const Geometry &g, CodecParams &p, cudaStream_t stream) {
     const DecSmem L = dec_smem_layout(g.d, g.rec, p.stages);
     const bool kg = g.topk_group > 0;
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;
+    const bool spec = g.d == 5120 && g.lpg == 4 && g.lpq == 4;   // width and groups of 128 compiled in
 #define RAC_DYN_DEC(B) \
     (sub ? (kg ? launch_persistent(decode_dyn_kernel<B, true, true>, p, g.nthreads, L.total, p.T, stream) \
                : launch_persistent(decode_dyn_kernel<B, false, true>, p, g.nthreads, L.total, p.T, stream)) \
+     : spec ? (kg ? launch_persistent(decode_dyn_kernel<B, true, false, 4, 5120>, p, g.nthreads, L.total, p.T, stream) \
+                  : launch_persistent(decode_dyn_kernel<B, false, false, 4, 5120>, p, g.nthreads, L.total, p.T, stream)) \
          : (kg ? launch_persistent(decode_dyn_kernel<B, true, false>, p, g.nthreads, L.total, p.T, stream) \
                : launch_persistent(decode_dyn_kernel<B, false, false>, p, g.nthreads, L.total, p.T, stream)))
     switch (g.bits) {
