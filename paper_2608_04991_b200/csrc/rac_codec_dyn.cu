@@ -95,7 +95,16 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
     const bool valid = tid * 32 < d;
     const bool qtok = lpq == 0;
     const int S = D ? 2 : p.stages;   // the host sets two stages
-    const DynSmem L = dyn_smem_layout(d, p.rec, S);
+    // with the width, the groups and (for up to two outliers per group, where the launcher compiles in the exact count)
+    // the outlier count known, the record geometry is a constant: coefficient words, scales, codes, offsets, values
+    constexpr bool kGeo = G != 0 && D != 0 && !SUB && KG <= 2;
+    constexpr int kJ = kGeo ? D / (32 * (G ? G : 1)) : 0, kJq = QT ? 1 : kJ;   // QT: one scale per token (and KG = 0)
+    constexpr int kScaleOff = 4 * kJ, kCodesOff = kScaleOff + (2 * kJq + 3) / 4 * 4, kGoffOff = kCodesOff + D * BITS / 8;
+    constexpr int kGvalOff = kGoffOff + (kJq * KG + 1) / 2 * 2, kRec = (kGvalOff + 2 * kJq * KG + 15) / 16 * 16;
+    const int recb = kGeo ? kRec : p.rec, kgc = kGeo ? KG : p.kg;
+    const int scale_off = kGeo ? kScaleOff : p.scale_off, codes_off = kGeo ? kCodesOff : p.codes_off;
+    const int goff_off = kGeo ? kGoffOff : p.goff_off, gval_off = kGeo ? kGvalOff : p.gval_off;
+    const DynSmem L = dyn_smem_layout(d, recb, S);
     DynCtrl *ctrl = reinterpret_cast<DynCtrl *>(smem);
     const uint32_t sbase = smem_u32(smem);
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
@@ -132,7 +141,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
     }
     // padding bytes of the record slots are zero from here on: every field is rewritten per token, the gaps never
     for (int s = 0; s < S; s++)
-        for (int o = 4 * tid; o < 2 * p.rec; o += 4 * nt)
+        for (int o = 4 * tid; o < 2 * recb; o += 4 * nt)
             *reinterpret_cast<uint32_t *>(smem + L.stage0 + s * L.stage_bytes + L.rec_off + o) = 0u;
     __syncthreads();
     if (tid == 0)
@@ -156,7 +165,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
         unsigned char *stg = smem + L.stage0 + stage * L.stage_bytes;
         const uint32_t xs = sbase + L.stage0 + stage * L.stage_bytes;
         const uint32_t rs = xs + row_bytes;
-        unsigned char *rec = stg + L.rec_off + parity * p.rec;
+        unsigned char *rec = stg + L.rec_off + parity * recb;
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
         const bool has_ref = ctrl->row[stage] >= 0;
 
@@ -333,9 +342,9 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                 if ((lane & (lpq - 1)) == 0) {
                     // the group's first lane serialises them in ascending offset order
                     const bool wide = lpq > 8;   // more than 256 channels per group: two-byte offsets
-                    unsigned char *go = rec + p.goff_off + jq * p.kg;
-                    unsigned short *go2 = reinterpret_cast<unsigned short *>(rec + p.goff_off) + jq * p.kg;
-                    unsigned short *gv = reinterpret_cast<unsigned short *>(rec + p.gval_off) + jq * p.kg;
+                    unsigned char *go = rec + goff_off + jq * kgc;
+                    unsigned short *go2 = reinterpret_cast<unsigned short *>(rec + goff_off) + jq * kgc;
+                    unsigned short *gv = reinterpret_cast<unsigned short *>(rec + gval_off) + jq * kgc;
 #pragma unroll
                     for (int n = 0; n < KG; n++) {
                         if (KG <= 2 || n < p.kg) {
@@ -393,7 +402,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             const float isc = sc != 0.f ? __fdiv_rn(1.0f, sc) : 0.f;   // zero marker: no division, codes 0
             const u64 inv2 = pack2(isc, isc), s2 = pack2(sc, sc);
             if (qtok ? tid == jq * p.qgen : (lane & (lpq - 1)) == 0)
-                reinterpret_cast<unsigned short *>(rec + p.scale_off)[jq] = (unsigned short)s16;
+                reinterpret_cast<unsigned short *>(rec + scale_off)[jq] = (unsigned short)s16;
 
             // No dense value can leave [-Qmax, Qmax] (Eq. 11): s >= max|E^d| / Qmax by the round-up, and the two
             // binary32 roundings of e * (1/s) add a few 2^-24 relative, far from the next half.  The exception is a
@@ -439,7 +448,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             {
                 uint32_t lo[4] = {words[0][0], words[1][0], words[2][0], words[3][0]};
                 rot_right4(lo, rot);
-                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + p.codes_off) + tid * WPT;
+                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + codes_off) + tid * WPT;
                 if (BITS == 8) {
                     uint32_t hi[4] = {words[0][1], words[1][1], words[2][1], words[3][1]};
                     rot_right4(hi, rot);
@@ -462,7 +471,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
                 float a, b, unused;
                 unpack2(a2, a, unused);
                 unpack2(b2, b, unused);
-                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + p.codes_off) + tid * WPT;
+                uint32_t *cw = reinterpret_cast<uint32_t *>(rec + codes_off) + tid * WPT;
 #pragma unroll
                 for (int n = 0; n < KG; n++) {
                     if ((own >> n) & 1u) {
@@ -500,14 +509,14 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_dyn_kernel
             if (lane == 0) {
                 const long long t = token_at<SUB>(p, first + (long long)it * stride);
                 if (XHAT) {
-                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_store(p.payload + t * recb, smem_u32(rec), (uint32_t)recb);
                     bulk_store(p.X_hat + t * d, xs, row_bytes);
                     bulk_commit();
                     bulk_wait_read<0>();
                     if (k_next < n_my) issue(k_next, stage, raw_next);
                 } else {
                     if (k_next < n_my) issue(k_next, stage, raw_next);
-                    bulk_store(p.payload + t * p.rec, smem_u32(rec), (uint32_t)p.rec);
+                    bulk_store(p.payload + t * recb, smem_u32(rec), (uint32_t)recb);
                     bulk_commit();
                     bulk_wait_read<0>();
                 }
