@@ -291,7 +291,9 @@ __host__ __device__ inline WsSmem ws_smem_layout(int d, int rec, int stages, boo
 // read it from the parameters; the constant removes the uniform branches of the shuffle reductions.
 // D: the hidden width as a compile-time constant (4096 and 5120 are compiled in), or 0 to read it from the parameters;
 // the constant folds the address arithmetic of the rows and stages (downlink call at 131072 x 5120: 0.671 -> 0.658 ms).
-template <int BITS, bool TOPK, bool XHAT, int MINB, bool SUB, int LPG = 0, int D = 0>
+// REF: every token has a reference row (identity rows: no row list, a reference buffer): the per-token test and the
+// second row of the tables go away (downlink call 0.649 -> 0.634 ms).
+template <int BITS, bool TOPK, bool XHAT, int MINB, bool SUB, int LPG = 0, int D = 0, bool REF = false>
 __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(const CodecParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -372,7 +374,7 @@ __global__ void __launch_bounds__(MINB == 4 ? 160 : 256, MINB) encode_ws_kernel(
         const uint32_t rs = xs + row_bytes;
         unsigned char *rec = stg + L.rec_off + parity * recb;
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_u32(&ctrl->full[stage]), parity))) { timed_out = true; break; }
-        const bool has_ref = ctrl->row[stage] >= 0;
+        const bool has_ref = REF ? true : ctrl->row[stage] >= 0;
 
         if (valid) {
             // ---- (1) the slab: 4 slots of 8 channels, slot j holds piece (j + rot) & 3
@@ -1445,11 +1447,17 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
     const bool sub = p.tok_list || p.intra_base || p.coef_ext;   // the subset form has one variant per width: it is not the hot path
     // widths 4096 and 5120 with no or eight outliers per token run variants with the whole record geometry compiled in
     const bool geo = (g.d == 5120 || g.d == 4096) && (g.topk == 0 || g.topk == 8);
+    const bool allref = p.ref_row == nullptr && p.ref_base != nullptr;   // identity rows: every token has its reference
 #define RAC_ENC4(B, K, X, G, W)                                                                                        \
     (tight ? launch_persistent(encode_ws_kernel<B, K, X, 4, false, G, W>, p, g.nthreads, L.total, max_ctas, stream) \
            : launch_persistent(encode_ws_kernel<B, K, X, 2, false, G, W>, p, g.nthreads, L.total, max_ctas, stream))
-#define RAC_ENC3(B, K, X, G)                                                        \
-    (!geo ? RAC_ENC4(B, K, X, G, 0) : g.d == 5120 ? RAC_ENC4(B, K, X, G, 5120) : RAC_ENC4(B, K, X, G, 4096))
+    // (at those widths the register variant follows from x_hat alone: 96 registers without it, 128 with it)
+#define RAC_ENC5(B, K, X, G, W, R) \
+    launch_persistent(encode_ws_kernel<B, K, X, (X ? 2 : 4), false, G, W, R>, p, g.nthreads, L.total, max_ctas, stream)
+#define RAC_ENC3(B, K, X, G)                                                                              \
+    (!geo ? RAC_ENC4(B, K, X, G, 0)                                                                       \
+     : g.d == 5120 ? (allref ? RAC_ENC5(B, K, X, G, 5120, true) : RAC_ENC5(B, K, X, G, 5120, false))     \
+                   : (allref ? RAC_ENC5(B, K, X, G, 4096, true) : RAC_ENC5(B, K, X, G, 4096, false)))
 #define RAC_ENC2(B, K, X)                                                                                           \
     (sub ? launch_persistent(encode_ws_kernel<B, K, X, 2, true, 0>, p, g.nthreads, L.total, max_ctas, stream)      \
      : g.lpg == 4 ? RAC_ENC3(B, K, X, 4) : g.lpg == 2 ? RAC_ENC3(B, K, X, 2) : RAC_ENC4(B, K, X, 0, 0))
@@ -1459,6 +1467,7 @@ static int launch_encode(const Geometry &g, CodecParams &p, long long max_ctas, 
         case 3: rc = topk ? RAC_ENC(3, true) : RAC_ENC(3, false); break;
         case 2: rc = topk ? RAC_ENC(2, true) : RAC_ENC(2, false); break;
     }
+#undef RAC_ENC5
 #undef RAC_ENC4
 #undef RAC_ENC3
 #undef RAC_ENC2
